@@ -1,0 +1,337 @@
+/*
+ * BlossomRec block-level fused sparse attention -- fp64 CPU ORACLE.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+ * restatement of the paper's equations that the CUDA library is checked
+ * against.  It shares no code, header, table or helper with the CUDA path and
+ * must never be called from the product path (only from tests, the smoke
+ * check and the benchmark's cpu_baseline / reference arm).
+ *
+ * What it computes, per (batch n, head h), all in double precision, in the
+ * paper's order (section "Block-Level Fused Sparse Attention Mechanism"):
+ *
+ *   block splitting      Eq. 8  with l = s = l' = Bk (non-overlapping blocks,
+ *                               0-based half-open, ragged last block kept)
+ *   block compression    Eq. 9  with phi := mean over the valid keys of a block
+ *   importance scoring   Eq. 10 softmax over the strictly-past live blocks,
+ *                               logits scaled by sm_scale
+ *   score sharing        Eq. 12 rule (sum of the probabilities of everyone who
+ *                               shares one selection) applied to the queries
+ *                               of a query block
+ *   top-k selection      Eq. 13 own block always kept, ties -> lower index
+ *   selected-KV attention Eq. 14 + Eq. 16 (via Eq. 1 with the causal mask)
+ *   window attention     Eq. 15 first case (|i-j| < w), causal side, Eq. 17
+ *   gate combine         Eq. 19 with alpha_h = sigmoid(a[h][0] - a[h][1])
+ *   backward             chain rule through Eq. 19, Eq. 16/17 and Eq. 1 with
+ *                        the selection frozen (top-k is piecewise constant)
+ *
+ * Parity pins (tests/test_oracle_*.py): explicit dense-mask evaluation of
+ * Eq. 1, softmax/causality invariants, reductions to dense causal attention,
+ * constructed selections with known answers, an independent numpy scorer,
+ * finite differences, and Table 5's key-budget closed form.  The readings of
+ * the paper that no printed value pins (selection per query block, phi = mean,
+ * scalar gate, own block always selected) are "parity unpinned by the paper".
+ *
+ * Layout: q, k, v, out*, dout, dq, dk, dv are contiguous [B][H][L][D] doubles;
+ * lse is [2][B][H][L] (0 = long-term branch, 1 = short-term branch), natural
+ * log of the sum of exp(sm_scale * q.k); gate is [H][2]; idx is
+ * [B][H][M][topk] int32 ascending, -1 padded; scores is [B][H][M][M].
+ * seq_lens[n] = number of valid (right-aligned) positions; NULL = all valid.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static int n_blocks(int L, int Bk) { return (L + Bk - 1) / Bk; }
+static int imin(int a, int b) { return a < b ? a : b; }
+static int imax(int a, int b) { return a > b ? a : b; }
+
+int blossom_oracle_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ---- selection for one (n,h) unit: Eq. 8-10, 12, 13 --------------------- */
+static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0,
+                        const double *q, const double *k, int32_t *idx,
+                        double *scores /* [M][M] or NULL */) {
+  const int M = n_blocks(L, Bk);
+  double *ktil = (double *)calloc((size_t)M * D, sizeof(double));
+  int *live = (int *)calloc((size_t)M, sizeof(int));
+  double *S = (double *)malloc(sizeof(double) * (size_t)M);
+  double *z = (double *)malloc(sizeof(double) * (size_t)M);
+  char *taken = (char *)malloc((size_t)M);
+  int *chosen = (int *)malloc(sizeof(int) * (size_t)(topk + 1));
+
+  /* Eq. 8 + Eq. 9: block j = [j*Bk, min((j+1)*Bk, L)), summary = mean of its valid keys */
+  for (int j = 0; j < M; ++j) {
+    int lo = imax(j * Bk, pad0), hi = imin((j + 1) * Bk, L), cnt = 0;
+    for (int p = lo; p < hi; ++p) {
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] += k[(size_t)p * D + c];
+      ++cnt;
+    }
+    live[j] = cnt > 0;
+    if (cnt > 0)
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] /= (double)cnt;
+  }
+
+  for (int b = 0; b < M; ++b) {
+    int32_t *row = idx + (size_t)b * topk;
+    for (int s = 0; s < topk; ++s) row[s] = -1;
+    if (scores)
+      for (int j = 0; j < M; ++j) scores[(size_t)b * M + j] = 0.0;
+    int qlo = imax(b * Bk, pad0), qhi = imin((b + 1) * Bk, L);
+    if (qlo >= qhi) continue; /* query block holds only padding */
+
+    int ncand = 0;
+    for (int j = 0; j < b; ++j) {
+      S[j] = 0.0;
+      ncand += live[j];
+    }
+    /* Eq. 10 per query, summed over the queries that share the selection (Eq. 12's rule) */
+    if (ncand > 0) {
+      for (int t = qlo; t < qhi; ++t) {
+        double mx = -INFINITY;
+        for (int j = 0; j < b; ++j) {
+          if (!live[j]) continue;
+          double acc = 0.0;
+          for (int c = 0; c < D; ++c) acc += q[(size_t)t * D + c] * ktil[(size_t)j * D + c];
+          z[j] = scale * acc;
+          if (z[j] > mx) mx = z[j];
+        }
+        double den = 0.0;
+        for (int j = 0; j < b; ++j)
+          if (live[j]) den += exp(z[j] - mx);
+        for (int j = 0; j < b; ++j)
+          if (live[j]) S[j] += exp(z[j] - mx) / den;
+      }
+    }
+    if (scores)
+      for (int j = 0; j < b; ++j)
+        if (live[j]) scores[(size_t)b * M + j] = S[j];
+
+    /* Eq. 13: the own block plus the (topk-1) best past blocks, ties to the lower index */
+    int want = imin(topk - 1, ncand), nch = 0;
+    memset(taken, 0, (size_t)M);
+    for (int s = 0; s < want; ++s) {
+      int best = -1;
+      for (int j = 0; j < b; ++j) {
+        if (!live[j] || taken[j]) continue;
+        if (best < 0 || S[j] > S[best]) best = j; /* strict > keeps the lower index on ties */
+      }
+      taken[best] = 1;
+      chosen[nch++] = best;
+    }
+    /* ascending order: walk the flags, then the own block (largest index) */
+    int s = 0;
+    for (int j = 0; j < b; ++j)
+      if (taken[j]) row[s++] = j;
+    row[s++] = b;
+  }
+  free(ktil); free(live); free(S); free(z); free(taken); free(chosen);
+}
+
+int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double scale,
+                          const double *q, const double *k, const int32_t *seq_lens,
+                          int32_t *idx, double *scores) {
+  if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
+  const int M = n_blocks(L, Bk);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int n = 0; n < B; ++n)
+    for (int h = 0; h < H; ++h) {
+      size_t u = (size_t)n * H + h;
+      int len = seq_lens ? seq_lens[n] : L;
+      if (len < 0) len = 0;
+      if (len > L) len = L;
+      select_unit(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D,
+                  idx + u * M * topk, scores ? scores + u * M * M : NULL);
+    }
+  return 0;
+}
+
+/* ---- one softmax-attention row over an explicit key list: Eq. 1 ---------- */
+/* keys[0..nk) are key positions; writes out[D], returns lse (0 and zeros if nk == 0) */
+static double attend_row(int D, double scale, const double *qt, const double *k, const double *v,
+                         const int *keys, int nk, double *sbuf, double *out) {
+  for (int c = 0; c < D; ++c) out[c] = 0.0;
+  if (nk == 0) return 0.0;
+  double mx = -INFINITY;
+  for (int i = 0; i < nk; ++i) {
+    const double *kp = k + (size_t)keys[i] * D;
+    double acc = 0.0;
+    for (int c = 0; c < D; ++c) acc += qt[c] * kp[c];
+    sbuf[i] = scale * acc;
+    if (sbuf[i] > mx) mx = sbuf[i];
+  }
+  double den = 0.0;
+  for (int i = 0; i < nk; ++i) den += exp(sbuf[i] - mx);
+  for (int i = 0; i < nk; ++i) {
+    double p = exp(sbuf[i] - mx) / den;
+    const double *vp = v + (size_t)keys[i] * D;
+    for (int c = 0; c < D; ++c) out[c] += p * vp[c];
+  }
+  return mx + log(den);
+}
+
+/* key list of the long-term branch for query t (Eq. 14 + causal mask): valid p <= t inside the
+ * selected blocks of t's query block */
+static int ltis_keys(int L, int Bk, int topk, int pad0, const int32_t *row, int t, int *keys) {
+  int nk = 0;
+  const int M = n_blocks(L, Bk);
+  for (int s = 0; s < topk; ++s) {
+    int j = row[s];
+    if (j < 0 || j >= M) continue;
+    int lo = imax(j * Bk, pad0), hi = imin(imin((j + 1) * Bk, L), t + 1);
+    for (int p = lo; p < hi; ++p) keys[nk++] = p;
+  }
+  return nk;
+}
+
+/* key list of the short-term branch (Eq. 15 first case, causal side): t - w < p <= t, valid */
+static int stis_keys(int w, int pad0, int t, int *keys) {
+  int nk = 0;
+  for (int p = imax(pad0, t - w + 1); p <= t; ++p) keys[nk++] = p;
+  return nk;
+}
+
+static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
+
+int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int window, double scale,
+                           const double *q, const double *k, const double *v, const double *gate,
+                           const int32_t *seq_lens, const int32_t *idx, double *out,
+                           double *out_lt, double *out_st, double *lse) {
+  if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1 || window < 1) return 1;
+  const int M = n_blocks(L, Bk);
+  const size_t BHL = (size_t)B * H * L;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int n = 0; n < B; ++n)
+    for (int h = 0; h < H; ++h) {
+      size_t u = (size_t)n * H + h;
+      int len = seq_lens ? seq_lens[n] : L;
+      if (len < 0) len = 0;
+      if (len > L) len = L;
+      const int pad0 = L - len;
+      const double *qu = q + u * L * D, *ku = k + u * L * D, *vu = v + u * L * D;
+      const double alpha = sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]); /* Eq. 18 reduced to a scalar */
+      int *keys = (int *)malloc(sizeof(int) * (size_t)(L + 1));
+      double *sbuf = (double *)malloc(sizeof(double) * (size_t)(L + 1));
+      double *oL = (double *)malloc(sizeof(double) * (size_t)D);
+      double *oS = (double *)malloc(sizeof(double) * (size_t)D);
+      for (int t = 0; t < L; ++t) {
+        size_t ro = (u * L + t) * (size_t)D;
+        double lL = 0.0, lS = 0.0;
+        if (t < pad0) {
+          for (int c = 0; c < D; ++c) oL[c] = oS[c] = 0.0;
+        } else {
+          const int32_t *row = idx + (u * M + (size_t)(t / Bk)) * topk;
+          int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
+          lL = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oL); /* Eq. 16 */
+          nk = stis_keys(window, pad0, t, keys);
+          lS = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oS); /* Eq. 17 */
+        }
+        for (int c = 0; c < D; ++c) {
+          if (out_lt) out_lt[ro + c] = oL[c];
+          if (out_st) out_st[ro + c] = oS[c];
+          out[ro + c] = alpha * oL[c] + (1.0 - alpha) * oS[c]; /* Eq. 19 */
+        }
+        if (lse) {
+          lse[u * L + t] = lL;
+          lse[BHL + u * L + t] = lS;
+        }
+      }
+      free(keys); free(sbuf); free(oL); free(oS);
+    }
+  return 0;
+}
+
+/* gradient of one softmax-attention row (Eq. 1) given upstream g = dL/d(out row):
+ *   P = exp(s - lse); dV_p += P g; dP = <g, v_p>; delta = <g, o>; dS = P (dP - delta);
+ *   dq += scale dS k_p; dK_p += scale dS q */
+static void attend_row_bwd(int D, double scale, const double *qt, const double *k, const double *v,
+                           const int *keys, int nk, double lse, const double *o, const double *g,
+                           double *dqt, double *dk, double *dv) {
+  if (nk == 0) return;
+  double delta = 0.0;
+  for (int c = 0; c < D; ++c) delta += g[c] * o[c];
+  for (int i = 0; i < nk; ++i) {
+    const size_t p = (size_t)keys[i];
+    const double *kp = k + p * D, *vp = v + p * D;
+    double acc = 0.0, dP = 0.0;
+    for (int c = 0; c < D; ++c) {
+      acc += qt[c] * kp[c];
+      dP += g[c] * vp[c];
+    }
+    double P = exp(scale * acc - lse);
+    double dS = P * (dP - delta);
+    for (int c = 0; c < D; ++c) {
+      dv[p * D + c] += P * g[c];
+      dqt[c] += scale * dS * kp[c];
+      dk[p * D + c] += scale * dS * qt[c];
+    }
+  }
+}
+
+int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int window, double scale,
+                            const double *q, const double *k, const double *v, const double *gate,
+                            const int32_t *seq_lens, const int32_t *idx, const double *out_lt,
+                            const double *out_st, const double *lse, const double *dout,
+                            double *dq, double *dk, double *dv, double *dgate) {
+  if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1 || window < 1) return 1;
+  const int M = n_blocks(L, Bk);
+  const size_t BHL = (size_t)B * H * L;
+  double *dalpha_unit = (double *)calloc((size_t)B * H, sizeof(double));
+  memset(dq, 0, sizeof(double) * BHL * D);
+  memset(dk, 0, sizeof(double) * BHL * D);
+  memset(dv, 0, sizeof(double) * BHL * D);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int n = 0; n < B; ++n)
+    for (int h = 0; h < H; ++h) {
+      size_t u = (size_t)n * H + h;
+      int len = seq_lens ? seq_lens[n] : L;
+      if (len < 0) len = 0;
+      if (len > L) len = L;
+      const int pad0 = L - len;
+      const double *qu = q + u * L * D, *ku = k + u * L * D, *vu = v + u * L * D;
+      double *dqu = dq + u * L * D, *dku = dk + u * L * D, *dvu = dv + u * L * D;
+      const double alpha = sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]);
+      int *keys = (int *)malloc(sizeof(int) * (size_t)(L + 1));
+      double *gL = (double *)malloc(sizeof(double) * (size_t)D);
+      double *gS = (double *)malloc(sizeof(double) * (size_t)D);
+      double dalpha = 0.0;
+      for (int t = pad0; t < L; ++t) {
+        size_t ro = (u * L + t) * (size_t)D;
+        for (int c = 0; c < D; ++c) {
+          dalpha += dout[ro + c] * (out_lt[ro + c] - out_st[ro + c]); /* d/d alpha of Eq. 19 */
+          gL[c] = alpha * dout[ro + c];
+          gS[c] = (1.0 - alpha) * dout[ro + c];
+        }
+        const int32_t *row = idx + (u * M + (size_t)(t / Bk)) * topk;
+        int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
+        attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[u * L + t],
+                       out_lt + ro, gL, dqu + (size_t)t * D, dku, dvu);
+        nk = stis_keys(window, pad0, t, keys);
+        attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[BHL + u * L + t],
+                       out_st + ro, gS, dqu + (size_t)t * D, dku, dvu);
+      }
+      dalpha_unit[u] = dalpha;
+      free(keys); free(gL); free(gS);
+    }
+  /* gate logits: alpha = sigmoid(a0 - a1)  =>  d a0 = alpha (1 - alpha) d alpha = - d a1 */
+  for (int h = 0; h < H; ++h) {
+    double da = 0.0;
+    for (int n = 0; n < B; ++n) da += dalpha_unit[(size_t)n * H + h];
+    const double alpha = sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]);
+    dgate[h * 2 + 0] = alpha * (1.0 - alpha) * da;
+    dgate[h * 2 + 1] = -dgate[h * 2 + 0];
+  }
+  free(dalpha_unit);
+  return 0;
+}

@@ -1,0 +1,159 @@
+"""ctypes front end of the fp64 C oracle (``blossom_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  Every function widens its inputs to float64 and calls
+the plain-C restatement of the paper's equations; nothing here is shared with
+the CUDA library.
+
+Shapes: q, k, v, dout ``[B, H, L, D]``; gate ``[H, 2]`` (column 0 = long-term
+branch logit, column 1 = short-term branch logit); seq_lens ``[B]`` valid
+lengths of left-padded sequences or ``None``; idx ``[B, H, M, topk]`` int32,
+ascending, -1 padded, ``M = ceil(L / block)``.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "blossom_oracle.c")
+_LIB = os.path.join(_HERE, "_build", "libblossom_oracle.so")
+_lib = None
+
+_dp = ctypes.POINTER(ctypes.c_double)
+_ip = ctypes.POINTER(ctypes.c_int32)
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (-O2 -fopenmp) if it is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    os.makedirs(os.path.dirname(_LIB), exist_ok=True)
+    tmp = _LIB + ".tmp.%d" % os.getpid()
+    subprocess.check_call(["gcc", "-O2", "-fopenmp", "-std=c99", "-fPIC", "-shared",
+                           "-o", tmp, _SRC, "-lm"])
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i = ctypes.c_int
+        d = ctypes.c_double
+        lib.blossom_oracle_threads.restype = i
+        lib.blossom_oracle_select.restype = i
+        lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp]
+        lib.blossom_oracle_forward.restype = i
+        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+                                               _ip, _dp, _dp, _dp, _dp]
+        lib.blossom_oracle_backward.restype = i
+        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+                                                _ip, _dp, _dp, _dp, _dp, _dp, _dp, _dp, _dp]
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the oracle uses (parallel over (batch, head) only)."""
+    return int(_load().blossom_oracle_threads())
+
+
+def _f64(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _ptr(a, ty):
+    return a.ctypes.data_as(ty) if a is not None else None
+
+
+def _lens(seq_lens, B):
+    if seq_lens is None:
+        return None
+    s = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    assert s.shape == (B,)
+    return s
+
+
+def _scale(sm_scale, D):
+    return float(sm_scale) if sm_scale else 1.0 / math.sqrt(D)
+
+
+def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False):
+    """Eq. 8-10, 12, 13: block summaries, block scores and the top-k block set."""
+    q, k = _f64(q), _f64(k)
+    B, H, L, D = q.shape
+    M = -(-L // block)
+    idx = np.empty((B, H, M, topk), dtype=np.int32)
+    scores = np.zeros((B, H, M, M), dtype=np.float64) if return_scores else None
+    sl = _lens(seq_lens, B)
+    rc = _load().blossom_oracle_select(B, H, L, D, block, topk, _scale(sm_scale, D),
+                                       _ptr(q, _dp), _ptr(k, _dp), _ptr(sl, _ip),
+                                       _ptr(idx, _ip), _ptr(scores, _dp))
+    if rc:
+        raise ValueError("blossom_oracle_select: bad arguments")
+    return (idx, scores) if return_scores else idx
+
+
+def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None):
+    """Eq. 14, 16, 17, 19.  ``idx`` overrides the selection when given.
+
+    Returns a dict: out, out_lt, out_st ``[B,H,L,D]``, lse ``[2,B,H,L]``, idx.
+    """
+    q, k, v, gate = _f64(q), _f64(k), _f64(v), _f64(gate)
+    B, H, L, D = q.shape
+    M = -(-L // block)
+    assert gate.shape == (H, 2)
+    if idx is None:
+        idx = select_blocks(q, k, block, topk, seq_lens, sm_scale)
+    idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
+    assert idx.shape == (B, H, M, topk)
+    sl = _lens(seq_lens, B)
+    out = np.empty_like(q)
+    out_lt = np.empty_like(q)
+    out_st = np.empty_like(q)
+    lse = np.empty((2, B, H, L), dtype=np.float64)
+    rc = _load().blossom_oracle_forward(B, H, L, D, block, topk, window, _scale(sm_scale, D),
+                                        _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp), _ptr(gate, _dp),
+                                        _ptr(sl, _ip), _ptr(idx, _ip), _ptr(out, _dp),
+                                        _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp))
+    if rc:
+        raise ValueError("blossom_oracle_forward: bad arguments")
+    return {"out": out, "out_lt": out_lt, "out_st": out_st, "lse": lse, "idx": idx}
+
+
+def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None):
+    """Gradients of sum(out * dout) with the selection frozen.
+
+    ``fwd`` is the dict ``forward`` returned.  Returns dq, dk, dv, dgate ``[H,2]``.
+    """
+    q, k, v, gate, dout = _f64(q), _f64(k), _f64(v), _f64(gate), _f64(dout)
+    B, H, L, D = q.shape
+    sl = _lens(seq_lens, B)
+    idx = np.ascontiguousarray(fwd["idx"], dtype=np.int32)
+    out_lt, out_st, lse = _f64(fwd["out_lt"]), _f64(fwd["out_st"]), _f64(fwd["lse"])
+    dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    dgate = np.empty((H, 2), dtype=np.float64)
+    rc = _load().blossom_oracle_backward(B, H, L, D, block, topk, window, _scale(sm_scale, D),
+                                         _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp),
+                                         _ptr(gate, _dp), _ptr(sl, _ip), _ptr(idx, _ip),
+                                         _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp),
+                                         _ptr(dout, _dp), _ptr(dq, _dp), _ptr(dk, _dp),
+                                         _ptr(dv, _dp), _ptr(dgate, _dp))
+    if rc:
+        raise ValueError("blossom_oracle_backward: bad arguments")
+    return {"dq": dq, "dk": dk, "dv": dv, "dgate": dgate}
+
+
+def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm_scale=None,
+                     idx=None):
+    """Convenience: forward then backward; returns the two dicts merged."""
+    f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx)
+    b = backward(q, k, v, gate, block, topk, window, f, dout, seq_lens, sm_scale)
+    f.update(b)
+    return f
