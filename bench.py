@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the BlossomRec sparse-attention hot path (selection + forward + backward).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 4] [--impl ours|reference]
+
+One "step" = one pass of the whole hot path over one synthetic batch: block summary + scoring
++ top-k selection, the fused two-branch forward (training mode: per-branch outputs and
+log-sum-exps saved) and the backward.  Prints ONE JSON line (rank 0).
+
+value     tokens/s with every input already resident in HBM (CUDA events, max over ranks)
+e2e       the same metric with HOST (pinned) inputs: host->device copies of q, k, v, dout, gate
+          and device->host copies of out, dq, dk, dv, dgate inside the timed region
+roofline  the kernel with the largest share of the timed region: its algorithmic FLOPs (or
+          bytes) per launch over its average device time (per-launch CUDA events recorded by
+          the library inside the timed region) against the measured peak of this machine
+cpu_baseline  the fp64 oracle, as it stands, on the host cores, on a bounded sample
+N > 1     every rank runs the same batch on its own GPU (independent replicas, no collective
+          on the data path): weak scaling, value = N * tokens / max-over-ranks time.
+--impl reference  times the oracle itself (rank 0 only), same metric and config.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sparse-attn fwd+bwd tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ algorithmic work model
+def work_model(w):
+    """Visited (query block, key block) tiles and the FLOPs / bytes they imply.
+
+    tile FLOPs = 2 * Bk * Bk * D per GEMM per visited tile and branch; forward 2 GEMMs
+    (QK^T, PV), backward 5 (S recompute, dP, dV, dK, dQ).  Compulsory bytes: forward reads
+    q, k, v and writes out, out_lt, out_st (+ lse, indices); backward reads q, k, v, dout,
+    out_lt, out_st, lse and writes dq, dk, dv: 15 q-shaped tensors in total.
+    """
+    import numpy as np
+    M, Bk = w.n_blocks, w.block
+    lens = np.full(w.B, w.L) if w.seq_lens is None else w.seq_lens.astype(np.int64)
+    tiles_L = tiles_S = 0
+    for ln in np.unique(lens):
+        cnt = int((lens == ln).sum())
+        pad0 = w.L - int(ln)
+        first = pad0 // Bk if ln > 0 else M
+        tl = ts = 0
+        for qb in range(first, M):
+            tl += min(w.topk, qb - first + 1)
+            lo_pos = max(pad0, qb * Bk - (w.window - 1))
+            ts += qb - lo_pos // Bk + 1
+        tiles_L += cnt * tl * w.H
+        tiles_S += cnt * ts * w.H
+    esz = 2 if w.dtype == "bf16" else 4
+    T = w.B * w.H * w.L * w.D * esz
+    tile_flops = 2.0 * Bk * Bk * w.D
+    tb = tiles_L + tiles_S
+    lse_b = 2 * w.B * w.H * w.L * 4
+    idx_b = w.B * w.H * M * w.topk * 4
+    gemms = {"fwd": 2, "bwd": 5, "fwd_simt": 2, "fwd_tc": 2, "bwd_dq_simt": 3, "bwd_dkdv_simt": 2,
+             "bwd_tc": 5}
+    byts = {"fwd": 6 * T + lse_b + idx_b, "bwd": 9 * T + 2 * lse_b + idx_b}
+    byts.update({"fwd_simt": byts["fwd"], "fwd_tc": byts["fwd"], "bwd_tc": byts["bwd"],
+                 "bwd_dq_simt": 7 * T + 2 * lse_b, "bwd_dkdv_simt": 6 * T + 2 * lse_b,
+                 "summary": T, "score_select": T})
+    return {"tiles_lt": tiles_L, "tiles_st": tiles_S, "tile_flops": tile_flops,
+            "flops": {k: g * tb * tile_flops for k, g in gemms.items()}, "bytes": byts,
+            "step_flops": 7 * tb * tile_flops, "step_bytes": 15 * T + 3 * lse_b + 2 * idx_b}
+
+
+# ------------------------------------------------------------------------ clock sampling
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------- oracle timing
+def oracle_sample(w, max_batch):
+    """The bounded sample of the workload the oracle is timed on: its first `max_batch`
+    batch entries (all heads)."""
+    from paper_2512_13368_b200.workloads import Workload
+    nb = min(max_batch, w.B)
+    sl = None if w.seq_lens is None else w.seq_lens[:nb].copy()
+    return Workload(w.name + f"[first {nb} of {w.B} batch entries]", w.dtype, nb, w.H, w.L, w.D,
+                    w.block, w.topk, w.window, w.seed, w.q[:nb], w.k[:nb], w.v[:nb], w.gate,
+                    w.dout[:nb], sl)
+
+
+def time_oracle(ws):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.forward_backward(ws.q, ws.k, ws.v, ws.gate, ws.dout, ws.block, ws.topk, ws.window,
+                            ws.seq_lens)
+    return time.perf_counter() - t0
+
+
+SAMPLE_BATCH = {1: 4, 2: 256, 3: 16, 4: 8, 5: 32}   # ~10-30 s of oracle work each
+
+
+def run_reference(args, w, cfg_desc):
+    import oracle
+    ws = oracle_sample(w, SAMPLE_BATCH[args.config])
+    for _ in range(args.warmup):
+        time_oracle(ws)
+    times = [time_oracle(ws) for _ in range(args.steps)]
+    sec = sum(times) / len(times)
+    value = ws.tokens / sec
+    cores = min(oracle.threads(), ws.B * ws.H)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": cfg_desc,
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": ws.name},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_2512_13368_b200 import workloads
+    if args.impl == "reference" and rank != 0:
+        return 0
+    w = workloads.CONFIGS[args.config]()
+    cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "seq_len": w.L, "head_dim": w.D,
+                "block_size": w.block, "top_k": w.topk, "window": w.window, "storage": w.dtype,
+                "padding": "left, lengths U{5..200}" if w.seq_lens is not None else "none",
+                "l2": "no flush: a step touches ~1 GB of distinct tensors, more than the 126 MB L2"
+                if w.B * w.H * w.L * w.D * 2 * 15 > 4 * 126e6 else
+                "working set fits L2; a 256 MB buffer is written between timed steps"}
+    if args.impl == "reference":
+        if args.steps == 20 and args.warmup == 5:
+            args.steps, args.warmup = 3, 1
+        run_reference(args, w, cfg_desc)
+        return 0
+
+    import torch
+    from paper_2512_13368_b200 import binding, runner
+    binding.load()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    args.warmup = max(args.warmup, 3)
+    dev = torch.device("cuda", local_rank if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return x
+
+    p = runner.DeviceProblem(w, device=dev)
+    model = work_model(w)
+    peaks, peak_kind = load_peaks()
+    flush = None
+    if not cfg_desc["l2"].startswith("no flush"):
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def step():
+        if flush is not None:
+            flush.fill_(1)
+        p.step()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, device-resident inputs, per-launch events recorded by the library
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = binding.blossom_launch_count()
+    cap = 16 * args.steps
+    binding.blossom_profile_start(cap)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_events = []
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        if flush is not None:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            flush.fill_(1)
+            a.record()
+            p.step()
+            b.record()
+            step_events.append((a, b))
+        else:
+            p.step()
+    e1.record()
+    barrier()
+    launches = binding.blossom_launch_count() - launches0
+    per_launch = binding.blossom_profile_stop(cap)
+    if step_events:
+        total_ms = sum(a.elapsed_time(b) for a, b in step_events)
+    else:
+        total_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    assert binding.blossom_device_status(p.workspace) == 0
+    ms_per_step = max_over_ranks(total_ms / args.steps)
+    value = world * w.tokens / (ms_per_step * 1e-3)
+
+    # ---- roofline of the kernel with the largest share
+    agg = {}
+    for name, ms in per_launch:
+        a = agg.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += ms
+    tot_kernel_ms = sum(v[1] for v in agg.values()) or 1.0
+    top = max(agg, key=lambda k: agg[k][1])
+    avg_ms = agg[top][1] / agg[top][0]
+    fl, by = model["flops"].get(top, 0.0), model["bytes"].get(top, 0.0)
+    tensor_peak = peaks["bf16_tflops_sustained"]
+    hbm_peak = peaks["hbm_gbs"]
+    if fl / (tensor_peak * 1e12) >= by / (hbm_peak * 1e9):
+        ach = fl / (avg_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": tensor_peak, "unit": "TFLOP/s",
+                "frac": ach / tensor_peak}
+    else:
+        ach = by / (avg_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak}
+    roof.update({"traffic": None, "kernel": top, "kernel_ms": avg_ms,
+                 "kernel_share": agg[top][1] / tot_kernel_ms,
+                 "peak_source": f"of {peak_kind} (MEASURED_PEAKS.json, sustained bf16 / copy bandwidth)"
+                 if peak_kind == "measured" else "of fallback",
+                 "kernels": {k: {"launches": v[0], "ms_per_launch": v[1] / v[0],
+                                 "share": v[1] / tot_kernel_ms} for k, v in sorted(agg.items())}})
+    t_roof = max(model["step_flops"] / (tensor_peak * 1e12), model["step_bytes"] / (hbm_peak * 1e9))
+    roof["step"] = {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step,
+                    "tile_gflop": model["step_flops"] / 1e9, "hbm_mb": model["step_bytes"] / 1e6}
+
+    # ---- end to end through the C ABI with host buffers
+    pin = lambda t: t.detach().cpu().pin_memory()  # noqa: E731
+    h_in = {k: pin(getattr(p, k)) for k in ("q", "k", "v", "dout", "gate")}
+    h_out = {k: pin(getattr(p, k)) for k in ("out", "dq", "dk", "dv", "dgate")}
+    h_sl = pin(p.seq_lens) if p.seq_lens is not None else None
+
+    def e2e_step():
+        for k, h in h_in.items():
+            getattr(p, k).copy_(h, non_blocking=True)
+        if h_sl is not None:
+            p.seq_lens.copy_(h_sl, non_blocking=True)
+        p.step()
+        for k, h in h_out.items():
+            h.copy_(getattr(p, k), non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+    nb = lambda t: t.numel() * t.element_size()  # noqa: E731
+    e2e = {"value": world * w.tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": sum(nb(t) for t in h_in.values()) + (nb(h_sl) if h_sl is not None else 0),
+           "d2h_bytes_per_step": sum(nb(t) for t in h_out.values())}
+
+    # ---- the oracle on the host cores (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        ws = oracle_sample(w, SAMPLE_BATCH[args.config])
+        sec = time_oracle(ws)
+        cpu = {"value": ws.tokens / sec, "unit": "tokens/s", "cores": min(oracle.threads(), ws.B * ws.H),
+               "kind": "oracle", "sample": f"{ws.name}: one fwd+bwd incl. selection, {sec:.1f} s"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+                "data": "synthetic", "config": cfg_desc, "clocks": clocks, "e2e": e2e,
+                "gpu_launches": int(launches), "roofline": roof, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,169 @@
+/*
+ * blossom.h -- C ABI of the B200 (sm_100a) BlossomRec block-sparse attention library.
+ *
+ * One operation, forward and backward: for every (batch, head) the long-term branch scores
+ * key-block summaries, keeps the top-k key blocks per query block and attends over them; the
+ * short-term branch attends over a causal sliding window; a per-head gate mixes the two.
+ *
+ * General conventions (all entry points)
+ *   - Every pointer is DEVICE memory unless a comment says "host".  The caller owns every
+ *     buffer; except where an entry point says otherwise the library allocates nothing, keeps
+ *     no state between calls, launches only on the given stream and never synchronises.
+ *   - q-shaped tensors (q, k, v, out, out_lt, out_st, dout, dq, dk, dv) are [B][H][L][D] with
+ *     element strides (stride_b, stride_h, stride_l, 1) shared by all of them; the element type
+ *     is params.dtype.  Base pointers must be 16-byte aligned and the three strides multiples
+ *     of 8 elements.
+ *   - seq_lens[B] (int32, may be NULL = every position valid) is the number of valid,
+ *     right-aligned positions of a left-padded sequence.  Padded keys never take part; padded
+ *     query rows produce 0 in out / out_lt / out_st / lse and in every gradient.
+ *   - block_idx is int32 [B][H][M][top_k], M = ceil(seq_len / block_size): for each query block
+ *     the selected key blocks in ascending order, -1 padded.  The query block's own block is
+ *     always one of them.
+ *   - lse is float [2][B][H][L]: plane 0 long-term branch, plane 1 short-term branch; natural log
+ *     of the sum over the branch's visible keys of exp(sm_scale * <q, k>).
+ *   - gate_logits is float [H][2]: column 0 long-term, column 1 short-term logit;
+ *     alpha_h = sigmoid(g[h][0] - g[h][1]) and out = alpha_h * out_lt + (1 - alpha_h) * out_st.
+ *   - Outputs are overwritten, never accumulated into; they need no zeroing.
+ *   - Return value: a blossom_status.  Arguments are checked on the host before any launch
+ *     (BLOSSOM_ERR_INVALID_ARG / _UNSUPPORTED / _WORKSPACE, nothing launched); a failed launch
+ *     gives BLOSSOM_ERR_CUDA.  Device-side bounded waits report through the status word read by
+ *     blossom_device_status.
+ *   - Calls on different streams are independent as long as their workspaces are distinct.
+ */
+#ifndef BLOSSOM_H_
+#define BLOSSOM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BLOSSOM_OK = 0,
+  BLOSSOM_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, non-positive size, bad stride      */
+  BLOSSOM_ERR_UNSUPPORTED = 2, /* a legal request this version does not implement               */
+  BLOSSOM_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned (256 B) or smaller than required   */
+  BLOSSOM_ERR_CUDA = 4,        /* a CUDA launch or runtime call failed                          */
+  BLOSSOM_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see blossom_device_status)*/
+} blossom_status;
+
+enum { BLOSSOM_DTYPE_FP32 = 0, BLOSSOM_DTYPE_BF16 = 1 };
+
+/* CUDA stream handle (same object as cudaStream_t / CUstream); NULL = the default stream. */
+typedef struct CUstream_st *blossom_stream_t;
+
+typedef struct {
+  int32_t batch, heads;
+  int32_t kv_heads;    /* must equal heads (grouped-query sharing is not implemented)            */
+  int32_t seq_len;     /* L >= 1, ceil(L / block_size) <= 1024                                   */
+  int32_t head_dim;    /* D in {32, 64}                                                          */
+  int32_t block_size;  /* key block = query block size Bk in {8, 16, 32, 64}                     */
+  int32_t top_k;       /* 1 <= top_k <= 64 blocks per query block, the own block included        */
+  int32_t window;      /* w >= 1: query t sees keys t - w < p <= t in the short-term branch      */
+  int32_t causal;      /* must be 1                                                              */
+  int32_t select_mode; /* 0 = one selection per query block (the only mode implemented)          */
+  int32_t dtype;       /* BLOSSOM_DTYPE_FP32 or BLOSSOM_DTYPE_BF16                               */
+  float sm_scale;      /* 0 -> 1/sqrt(head_dim); scales block scores and attention logits alike  */
+  int64_t stride_b, stride_h, stride_l; /* element strides of every q-shaped tensor              */
+} blossom_params;
+
+/* Bytes of device scratch the calls below need for these params (one size serves all three);
+ * 0 if the params are invalid or unsupported.  The workspace must be 256-byte aligned.  Its
+ * contents carry nothing from one call to the next, except that blossom_attn_bwd reads nothing
+ * from it that blossom_attn_fwd wrote (the saved tensors are the caller's).  Host function. */
+size_t blossom_workspace_bytes(const blossom_params *params /* host */);
+
+/*
+ * Block summary, importance scoring and top-k selection (paper: LTIS "Block Splitting",
+ * "Block Compression", "Importance Scoring", "Top-k Selection"; Eq. 8-10, 12, 13 with
+ * compression size = stride = selection size = block_size and the summary = mean of a block's
+ * valid keys).  For each query block b: every valid query of the block takes a softmax of
+ * sm_scale * <q, mean-key_j> over the live blocks j < b; the probabilities are summed over the
+ * block's queries; the top_k - 1 largest sums (ties to the lower j) plus b itself are written
+ * ascending to block_idx.  Scores are evaluated in double precision so that the choice matches
+ * an fp64 evaluation except for ties below 1e-12 relative.
+ *   q, k        in   q-shaped
+ *   seq_lens    in   [B] or NULL
+ *   block_idx   out  [B][H][M][top_k]
+ */
+int blossom_select_blocks(const blossom_params *params /* host */, const void *q, const void *k,
+                          const int32_t *seq_lens, int32_t *block_idx, void *workspace,
+                          size_t workspace_bytes, blossom_stream_t stream);
+
+/*
+ * Forward (paper: Eq. 14 and 16 for the selected-block branch, Eq. 15 first case under the
+ * causal mask and Eq. 17 for the window branch, Eq. 19 for the gate, each branch being the
+ * masked softmax attention of Eq. 1 with online softmax in fp32).
+ *   q, k, v      in   q-shaped
+ *   gate_logits  in   [H][2]
+ *   seq_lens     in   [B] or NULL
+ *   block_idx    in/out [B][H][M][top_k]; idx_is_input = 0: selection is computed (as by
+ *                blossom_select_blocks) and written here; != 0: used as given (entries outside
+ *                [0, M) are ignored; blocks after the query block contribute nothing)
+ *   out          out  q-shaped, the gated mix
+ *   out_lt,out_st out q-shaped per-branch outputs, needed by the backward; both may be NULL
+ *                (inference: nothing is saved), else both non-NULL
+ *   lse          out  [2][B][H][L]; may be NULL only when out_lt and out_st are NULL
+ */
+int blossom_attn_fwd(const blossom_params *params /* host */, const void *q, const void *k,
+                     const void *v, const float *gate_logits, const int32_t *seq_lens,
+                     int32_t *block_idx, int32_t idx_is_input, void *out, void *out_lt,
+                     void *out_st, float *lse, void *workspace, size_t workspace_bytes,
+                     blossom_stream_t stream);
+
+/*
+ * Backward of blossom_attn_fwd for upstream gradient dout = dLoss/d out, with the selection
+ * frozen (top-k is piecewise constant, no gradient flows through the scores).  Chain rule through
+ * Eq. 19 (gate), Eq. 16 / 17 and the softmax of Eq. 1, recomputing the probabilities from the
+ * saved log-sum-exps: P = exp(sm_scale <q,k> - lse), dV += P^T G, dP = G V^T,
+ * dS = P o (dP - rowsum(G o O)), dQ += sm_scale dS K, dK += sm_scale dS^T Q per branch with
+ * G_lt = alpha G, G_st = (1 - alpha) G; d alpha_h = sum G o (out_lt - out_st),
+ * dgate[h][0] = alpha (1 - alpha) d alpha = -dgate[h][1].
+ *   q, k, v, gate_logits, seq_lens, block_idx   in   as given to / produced by the forward
+ *   out_lt, out_st, lse                          in   saved by the forward
+ *   dout                                         in   q-shaped
+ *   dq, dk, dv                                   out  q-shaped
+ *   dgate                                        out  float [H][2]
+ */
+int blossom_attn_bwd(const blossom_params *params /* host */, const void *q, const void *k,
+                     const void *v, const float *gate_logits, const int32_t *seq_lens,
+                     const int32_t *block_idx, const void *out_lt, const void *out_st,
+                     const float *lse, const void *dout, void *dq, void *dk, void *dv,
+                     float *dgate, void *workspace, size_t workspace_bytes,
+                     blossom_stream_t stream);
+
+/* Synchronises the stream and copies the workspace's device status word to *host_out (host):
+ * 0 = no device-side error since the workspace was last used, else a blossom_status.  Returns
+ * BLOSSOM_ERR_CUDA if the synchronise or the copy fails. */
+int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out);
+
+/* Human-readable name of a blossom_status (host string, static storage). */
+const char *blossom_status_string(int status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int blossom_version(void);
+
+/* Number of kernels the library launched from this process since it was loaded (all streams);
+ * a host-side counter for benchmarks. */
+uint64_t blossom_launch_count(void);
+
+/*
+ * Measurement aid (no counterpart in the paper): per-launch device times of the library's own
+ * kernels.  blossom_profile_start creates 2 * max_launches CUDA events; from then on every
+ * kernel the library launches (any stream) is bracketed by two event records until
+ * blossom_profile_stop, which waits for the recorded events, writes for launch i its kernel id
+ * and its device time in milliseconds to kernel_ids[i] / ms[i] (host arrays of `capacity`
+ * entries), destroys the events and returns the number of launches written (-1 on error or if
+ * no profile is running).  Process-wide and not thread-safe; off by default; launches beyond
+ * max_launches are not recorded.  blossom_kernel_name maps an id to a static host string.
+ */
+int blossom_profile_start(int max_launches);
+int blossom_profile_stop(int32_t *kernel_ids /* host */, float *ms /* host */, int capacity);
+const char *blossom_kernel_name(int kernel_id);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BLOSSOM_H_ */

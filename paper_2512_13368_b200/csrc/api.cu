@@ -1,0 +1,234 @@
+// C ABI of the blossom library: argument validation, workspace carving and dispatch.
+// Every check happens on the host before anything is launched.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace blossom {
+
+unsigned long long g_launches = 0;
+
+// ---- optional per-launch event profile (process-wide, off by default) ---------------------
+static cudaEvent_t *g_prof_events = nullptr;  // [2 * cap]: before / after each launch
+static int *g_prof_ids = nullptr;
+static int g_prof_cap = 0, g_prof_n = 0;
+
+void prof_mark(int id, int phase, cudaStream_t st) {
+  if (!g_prof_events) return;
+  if (phase == 0) {
+    if (g_prof_n >= g_prof_cap) return;
+    g_prof_ids[g_prof_n] = id;
+    cudaEventRecord(g_prof_events[2 * g_prof_n], st);
+  } else {
+    if (g_prof_n >= g_prof_cap) return;
+    cudaEventRecord(g_prof_events[2 * g_prof_n + 1], st);
+    ++g_prof_n;
+  }
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+Workspace carve_workspace(const Shape &s, void *base) {
+  Workspace w;
+  char *p = static_cast<char *>(base);
+  size_t off = 0;
+  const size_t units = (size_t)s.B * s.H;
+  auto take = [&](size_t bytes) {
+    char *r = p ? p + off : nullptr;
+    off += align_up(bytes, 256);
+    return r;
+  };
+  w.status = reinterpret_cast<int32_t *>(take(256));
+  w.kmean = reinterpret_cast<double *>(take(units * s.M * s.D * sizeof(double)));
+  w.klive = reinterpret_cast<int32_t *>(take(units * s.M * sizeof(int32_t)));
+  w.delta = reinterpret_cast<float *>(take(2 * units * s.L * sizeof(float)));
+  w.dalpha = reinterpret_cast<double *>(take(units * s.M * sizeof(double)));
+  w.dq_acc = nullptr;
+  w.bytes = off;
+  return w;
+}
+
+// Returns BLOSSOM_OK and fills the shape, or the status describing what is wrong.
+static int make_shape(const blossom_params *p, Shape *out) {
+  if (!p) return BLOSSOM_ERR_INVALID_ARG;
+  if (p->batch < 1 || p->heads < 1 || p->seq_len < 1 || p->head_dim < 1 || p->block_size < 1 ||
+      p->top_k < 1 || p->window < 1)
+    return BLOSSOM_ERR_INVALID_ARG;
+  if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return BLOSSOM_ERR_INVALID_ARG;
+  if (p->dtype != BLOSSOM_DTYPE_FP32 && p->dtype != BLOSSOM_DTYPE_BF16)
+    return BLOSSOM_ERR_INVALID_ARG;
+  if (p->stride_l < p->head_dim || p->stride_h < 1 || p->stride_b < 1) return BLOSSOM_ERR_INVALID_ARG;
+  if (p->stride_l % 8 || p->stride_h % 8 || p->stride_b % 8) return BLOSSOM_ERR_INVALID_ARG;
+  if (p->kv_heads != p->heads) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->causal != 1 || p->select_mode != 0) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->head_dim != 32 && p->head_dim != 64) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->block_size != 8 && p->block_size != 16 && p->block_size != 32 && p->block_size != 64)
+    return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->top_k > 64) return BLOSSOM_ERR_UNSUPPORTED;
+  const int64_t M = ((int64_t)p->seq_len + p->block_size - 1) / p->block_size;
+  if (M > 1024) return BLOSSOM_ERR_UNSUPPORTED;
+  if ((int64_t)p->batch * p->heads * M > 0x7fffffffLL) return BLOSSOM_ERR_UNSUPPORTED;
+  Shape s;
+  s.B = p->batch; s.H = p->heads; s.L = p->seq_len; s.D = p->head_dim; s.Bk = p->block_size;
+  s.topk = p->top_k; s.window = p->window; s.M = (int)M;
+  s.scale_d = p->sm_scale > 0.f ? (double)p->sm_scale : 1.0 / sqrt((double)p->head_dim);
+  s.scale = (float)s.scale_d;
+  s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;
+  *out = s;
+  return BLOSSOM_OK;
+}
+
+static bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
+// Validates the workspace and clears its status word on the stream (a memset, not a kernel).
+static int check_workspace(const Shape &s, void *ws, size_t bytes, cudaStream_t st, Workspace *out) {
+  if (!ws || misaligned(ws, 256)) return BLOSSOM_ERR_WORKSPACE;
+  *out = carve_workspace(s, ws);
+  if (bytes < out->bytes) return BLOSSOM_ERR_WORKSPACE;
+  if (cudaMemsetAsync(out->status, 0, 16, st) != cudaSuccess) return BLOSSOM_ERR_CUDA;
+  return BLOSSOM_OK;
+}
+
+}  // namespace blossom
+
+using namespace blossom;
+
+extern "C" {
+
+size_t blossom_workspace_bytes(const blossom_params *params) {
+  Shape s;
+  if (make_shape(params, &s) != BLOSSOM_OK) return 0;
+  return carve_workspace(s, nullptr).bytes;
+}
+
+int blossom_select_blocks(const blossom_params *params, const void *q, const void *k,
+                          const int32_t *seq_lens, int32_t *block_idx, void *workspace,
+                          size_t workspace_bytes, blossom_stream_t stream) {
+  Shape s;
+  int rc = make_shape(params, &s);
+  if (rc) return rc;
+  if (!q || !k || !block_idx) return BLOSSOM_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(block_idx, 4) || misaligned(seq_lens, 4))
+    return BLOSSOM_ERR_INVALID_ARG;
+  Workspace ws;
+  rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
+  if (rc) return rc;
+  return launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, (cudaStream_t)stream);
+}
+
+int blossom_attn_fwd(const blossom_params *params, const void *q, const void *k, const void *v,
+                     const float *gate_logits, const int32_t *seq_lens, int32_t *block_idx,
+                     int32_t idx_is_input, void *out, void *out_lt, void *out_st, float *lse,
+                     void *workspace, size_t workspace_bytes, blossom_stream_t stream) {
+  Shape s;
+  int rc = make_shape(params, &s);
+  if (rc) return rc;
+  if (!q || !k || !v || !gate_logits || !block_idx || !out) return BLOSSOM_ERR_INVALID_ARG;
+  if ((out_lt == nullptr) != (out_st == nullptr)) return BLOSSOM_ERR_INVALID_ARG;
+  if (out_lt && !lse) return BLOSSOM_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out, 16) ||
+      misaligned(out_lt, 16) || misaligned(out_st, 16) || misaligned(lse, 4) ||
+      misaligned(gate_logits, 4) || misaligned(block_idx, 4) || misaligned(seq_lens, 4))
+    return BLOSSOM_ERR_INVALID_ARG;
+  Workspace ws;
+  rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!idx_is_input) {
+    rc = launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, st);
+    if (rc) return rc;
+  }
+  return launch_fwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out, out_lt,
+                         out_st, lse, ws, st);
+}
+
+int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k, const void *v,
+                     const float *gate_logits, const int32_t *seq_lens, const int32_t *block_idx,
+                     const void *out_lt, const void *out_st, const float *lse, const void *dout,
+                     void *dq, void *dk, void *dv, float *dgate, void *workspace,
+                     size_t workspace_bytes, blossom_stream_t stream) {
+  Shape s;
+  int rc = make_shape(params, &s);
+  if (rc) return rc;
+  if (!q || !k || !v || !gate_logits || !block_idx || !out_lt || !out_st || !lse || !dout || !dq ||
+      !dk || !dv || !dgate)
+    return BLOSSOM_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out_lt, 16) ||
+      misaligned(out_st, 16) || misaligned(dout, 16) || misaligned(dq, 16) || misaligned(dk, 16) ||
+      misaligned(dv, 16) || misaligned(lse, 4) || misaligned(dgate, 4) ||
+      misaligned(gate_logits, 4) || misaligned(block_idx, 4) || misaligned(seq_lens, 4))
+    return BLOSSOM_ERR_INVALID_ARG;
+  Workspace ws;
+  rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
+  if (rc) return rc;
+  return launch_bwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out_lt,
+                         out_st, lse, dout, dq, dk, dv, dgate, ws, (cudaStream_t)stream);
+}
+
+int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out) {
+  if (!workspace || !host_out) return BLOSSOM_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BLOSSOM_ERR_CUDA;
+  if (cudaMemcpy(host_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  return BLOSSOM_OK;
+}
+
+const char *blossom_status_string(int status) {
+  switch (status) {
+    case BLOSSOM_OK: return "ok";
+    case BLOSSOM_ERR_INVALID_ARG: return "invalid argument";
+    case BLOSSOM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case BLOSSOM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case BLOSSOM_ERR_CUDA: return "CUDA error";
+    case BLOSSOM_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int blossom_version(void) { return 100; }
+
+int blossom_profile_start(int max_launches) {
+  if (max_launches < 1 || g_prof_events) return BLOSSOM_ERR_INVALID_ARG;
+  cudaEvent_t *ev = new cudaEvent_t[2 * (size_t)max_launches];
+  for (int i = 0; i < 2 * max_launches; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+      for (int j = 0; j < i; ++j) cudaEventDestroy(ev[j]);
+      delete[] ev;
+      return BLOSSOM_ERR_CUDA;
+    }
+  g_prof_ids = new int[max_launches];
+  g_prof_cap = max_launches;
+  g_prof_n = 0;
+  g_prof_events = ev;
+  return BLOSSOM_OK;
+}
+
+int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
+  if (!g_prof_events) return -1;
+  cudaEvent_t *ev = g_prof_events;
+  g_prof_events = nullptr;  // stop recording
+  int n = g_prof_n < capacity ? g_prof_n : capacity, bad = 0;
+  for (int i = 0; i < n; ++i) {
+    if (cudaEventSynchronize(ev[2 * i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms[i], ev[2 * i], ev[2 * i + 1]) != cudaSuccess)
+      bad = 1;
+    kernel_ids[i] = g_prof_ids[i];
+  }
+  for (int i = 0; i < 2 * g_prof_cap; ++i) cudaEventDestroy(ev[i]);
+  delete[] ev;
+  delete[] g_prof_ids;
+  g_prof_ids = nullptr;
+  g_prof_cap = g_prof_n = 0;
+  return bad ? -1 : n;
+}
+
+const char *blossom_kernel_name(int id) {
+  static const char *names[K_COUNT] = {
+      "summary", "score_select", "fwd_simt", "bwd_dq_simt", "bwd_dkdv_simt", "gate_grad",
+      "fwd_tc", "bwd_pre_tc", "bwd_tc", "bwd_cvt_tc"};
+  return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
+}
+
+uint64_t blossom_launch_count(void) { return g_launches; }
+
+}  // extern "C"

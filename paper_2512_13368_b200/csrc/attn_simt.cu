@@ -1,0 +1,486 @@
+// fp32 CUDA-core path of the fused two-branch attention (forward + backward).
+//
+// It serves fp32 inputs (whose 1e-4 tolerance rules out reduced-precision tensor-core products)
+// and every shape the tensor-core path does not take.  One CTA per (unit, query block) for the
+// forward and dQ kernels, one CTA per (unit, key block) for dK/dV; a query (or key) row is owned
+// by 4 adjacent lanes, each holding D/4 columns as interleaved float4 chunks, so dot products
+// finish with two shuffles and shared-memory reads are conflict-free 128-bit loads.
+//
+// Paper: selected-block attention Eq. 14 + 16, window attention Eq. 15 (first case, causal) + 17,
+// both instances of the masked softmax attention of Eq. 1; gate combine Eq. 19.
+#include "common.cuh"
+
+namespace blossom {
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float group_sum(float x, unsigned gmask) {
+  x += __shfl_xor_sync(gmask, x, 1);
+  x += __shfl_xor_sync(gmask, x, 2);
+  return x;
+}
+__device__ __forceinline__ float dot4(const float4 a, const float4 b, float acc) {
+  acc = fmaf(a.x, b.x, acc);
+  acc = fmaf(a.y, b.y, acc);
+  acc = fmaf(a.z, b.z, acc);
+  return fmaf(a.w, b.w, acc);
+}
+__device__ __forceinline__ void axpy4(float4 &y, float a, const float4 x) {
+  y.x = fmaf(a, x.x, y.x); y.y = fmaf(a, x.y, y.y); y.z = fmaf(a, x.z, y.z); y.w = fmaf(a, x.w, y.w);
+}
+__device__ __forceinline__ void scale_axpy4(float4 &y, float c, float a, const float4 x) {
+  y.x = fmaf(a, x.x, y.x * c); y.y = fmaf(a, x.y, y.y * c);
+  y.z = fmaf(a, x.z, y.z * c); y.w = fmaf(a, x.w, y.w * c);
+}
+__device__ __forceinline__ float4 zero4() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
+
+// Stage rows [row0, row0 + Bk) of a q-shaped tensor into shared memory as fp32 (zero past L).
+template <typename T, int D>
+__device__ __forceinline__ void stage_tile(const Shape &s, const T *base, int n, int h, int row0,
+                                           float *dst) {
+  constexpr int CH = D / 4;
+  for (int i = threadIdx.x; i < s.Bk * CH; i += blockDim.x) {
+    const int pr = i / CH, ch = i % CH, p = row0 + pr;
+    float4 x = zero4();
+    if (p < s.L) x = ld4(base + row_offset(s, n, h, p) + ch * 4);
+    reinterpret_cast<float4 *>(dst)[i] = x;
+  }
+}
+
+// flags[blk], blk <= qb: bit 0 = blk is one of the query block's selected blocks,
+// bit 1 = blk intersects the causal window of some query of the block.
+__device__ __forceinline__ void build_visit_flags(const Shape &s, const int32_t *idxrow, int qb,
+                                                  int *flags) {
+  const int wpos = qb * s.Bk - (s.window - 1);
+  const int wlo = wpos > 0 ? wpos / s.Bk : 0;
+  for (int blk = threadIdx.x; blk <= qb; blk += blockDim.x) {
+    int f = blk >= wlo ? 2 : 0;
+    for (int i = 0; i < s.topk; ++i) f |= (idxrow[i] == blk) ? 1 : 0;
+    flags[blk] = f;
+  }
+}
+
+// ------------------------------------------------------------------------------- forward
+template <typename T, int D>
+__global__ void __launch_bounds__(256) fwd_simt_kernel(
+    Shape s, const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
+    const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
+    const int32_t *__restrict__ idx, T *__restrict__ out, T *__restrict__ out_lt,
+    T *__restrict__ out_st, float *__restrict__ lse) {
+  constexpr int NV = D / 16, CH = D / 4;
+  extern __shared__ float smf[];
+  float *Ks = smf, *Vs = Ks + s.Bk * D;
+  int *flags = reinterpret_cast<int *>(Vs + s.Bk * D);
+  const int qb = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int tid = threadIdx.x, r = tid >> 2, sub = tid & 3;
+  const unsigned gmask = 0xFu << ((tid & 31) & ~3);
+  const int t = qb * s.Bk + r;
+  const bool inrange = t < s.L, active = inrange && t >= pad0;
+
+  build_visit_flags(s, idx + ((int64_t)u * s.M + qb) * s.topk, qb, flags);
+
+  float4 qv[NV], aL[NV], aS[NV];
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    qv[c] = active ? ld4(q + row_offset(s, n, h, t) + (c * 4 + sub) * 4) : zero4();
+    aL[c] = zero4();
+    aS[c] = zero4();
+  }
+  float mL = -INFINITY, lL = 0.f, mS = -INFINITY, lS = 0.f;
+  const float sc2 = s.scale * kLog2e;
+  const bool block_live = min((qb + 1) * s.Bk, s.L) > pad0;
+  __syncthreads();
+
+  if (block_live) {
+    for (int blk = 0; blk <= qb; ++blk) {
+      const int f = flags[blk];
+      if (!f) continue;
+      __syncthreads();
+      stage_tile<T, D>(s, k, n, h, blk * s.Bk, Ks);
+      stage_tile<T, D>(s, v, n, h, blk * s.Bk, Vs);
+      __syncthreads();
+      if (!active) continue;
+      const int p0 = blk * s.Bk;
+      const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
+      const bool selb = f & 1;
+      for (int pi = pbeg; pi < pend; ++pi) {
+        const bool inS = (t - (p0 + pi)) < s.window;
+        if (!selb && !inS) continue;
+        const float4 *kr = reinterpret_cast<const float4 *>(Ks) + pi * CH;
+        const float4 *vr = reinterpret_cast<const float4 *>(Vs) + pi * CH;
+        float part = 0.f;
+#pragma unroll
+        for (int c = 0; c < NV; ++c) part = dot4(qv[c], kr[c * 4 + sub], part);
+        const float sv = group_sum(part, gmask) * sc2;
+        if (selb) {
+          const float mn = fmaxf(mL, sv), corr = exp2f(mL - mn), pe = exp2f(sv - mn);
+          lL = fmaf(lL, corr, pe);
+#pragma unroll
+          for (int c = 0; c < NV; ++c) scale_axpy4(aL[c], corr, pe, vr[c * 4 + sub]);
+          mL = mn;
+        }
+        if (inS) {
+          const float mn = fmaxf(mS, sv), corr = exp2f(mS - mn), pe = exp2f(sv - mn);
+          lS = fmaf(lS, corr, pe);
+#pragma unroll
+          for (int c = 0; c < NV; ++c) scale_axpy4(aS[c], corr, pe, vr[c * 4 + sub]);
+          mS = mn;
+        }
+      }
+    }
+  }
+
+  if (!inrange) return;
+  const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]);
+  const float iL = lL > 0.f ? 1.f / lL : 0.f, iS = lS > 0.f ? 1.f / lS : 0.f;
+  const int64_t ro = row_offset(s, n, h, t);
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    const float4 oL = make_float4(aL[c].x * iL, aL[c].y * iL, aL[c].z * iL, aL[c].w * iL);
+    const float4 oS = make_float4(aS[c].x * iS, aS[c].y * iS, aS[c].z * iS, aS[c].w * iS);
+    const float be = 1.f - alpha;
+    const float4 o = make_float4(alpha * oL.x + be * oS.x, alpha * oL.y + be * oS.y,
+                                 alpha * oL.z + be * oS.z, alpha * oL.w + be * oS.w);
+    const int64_t off = ro + (c * 4 + sub) * 4;
+    st4(out + off, o);
+    if (out_lt) st4(out_lt + off, oL);
+    if (out_st) st4(out_st + off, oS);
+  }
+  if (sub == 0 && lse) {
+    const int64_t BHL = (int64_t)s.B * s.H * s.L;
+    lse[(int64_t)u * s.L + t] = lL > 0.f ? mL * kLn2 + __logf(lL) : 0.f;
+    lse[BHL + (int64_t)u * s.L + t] = lS > 0.f ? mS * kLn2 + __logf(lS) : 0.f;
+  }
+}
+
+// ------------------------------------------------------------------------- backward: dQ
+// Also produces delta[2][B][H][L] and the per-query-block partial of d alpha for the later kernels.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
+    Shape s, const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
+    const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
+    const int32_t *__restrict__ idx, const T *__restrict__ out_lt, const T *__restrict__ out_st,
+    const float *__restrict__ lse, const T *__restrict__ dout, T *__restrict__ dq,
+    float *__restrict__ delta, double *__restrict__ dalpha_part) {
+  constexpr int NV = D / 16, CH = D / 4;
+  extern __shared__ float smf[];
+  float *Ks = smf, *Vs = Ks + s.Bk * D;
+  int *flags = reinterpret_cast<int *>(Vs + s.Bk * D);
+  double *red = reinterpret_cast<double *>(flags + s.M + (s.M & 1));  // [Bk]
+  const int qb = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int tid = threadIdx.x, r = tid >> 2, sub = tid & 3;
+  const unsigned gmask = 0xFu << ((tid & 31) & ~3);
+  const int t = qb * s.Bk + r;
+  const bool inrange = t < s.L, active = inrange && t >= pad0;
+  const int64_t BHL = (int64_t)s.B * s.H * s.L;
+  const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
+
+  build_visit_flags(s, idx + ((int64_t)u * s.M + qb) * s.topk, qb, flags);
+
+  float4 qv[NV], gv[NV], acc[NV];
+  float dL = 0.f, dS = 0.f;
+  const int64_t ro = row_offset(s, n, h, inrange ? t : 0);
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    const int64_t off = ro + (c * 4 + sub) * 4;
+    qv[c] = active ? ld4(q + off) : zero4();
+    gv[c] = active ? ld4(dout + off) : zero4();
+    acc[c] = zero4();
+    if (active) {
+      dL = dot4(gv[c], ld4(out_lt + off), dL);
+      dS = dot4(gv[c], ld4(out_st + off), dS);
+    }
+  }
+  dL = group_sum(dL, gmask);
+  dS = group_sum(dS, gmask);
+  const float deltaL = alpha * dL, deltaS = beta * dS;
+  float lseL2 = 0.f, lseS2 = 0.f;
+  if (active) {
+    lseL2 = lse[(int64_t)u * s.L + t] * kLog2e;
+    lseS2 = lse[BHL + (int64_t)u * s.L + t] * kLog2e;
+  }
+  if (inrange && sub == 0) {
+    delta[(int64_t)u * s.L + t] = deltaL;
+    delta[BHL + (int64_t)u * s.L + t] = deltaS;
+  }
+  if (sub == 0) red[r] = active ? (double)dL - (double)dS : 0.0;
+  const float sc2 = s.scale * kLog2e;
+  const bool block_live = min((qb + 1) * s.Bk, s.L) > pad0;
+  __syncthreads();
+  if (tid == 0) {
+    double a = 0.0;
+    for (int i = 0; i < s.Bk; ++i) a += red[i];  // fixed order
+    dalpha_part[(int64_t)u * s.M + qb] = a;
+  }
+
+  if (block_live) {
+    for (int blk = 0; blk <= qb; ++blk) {
+      const int f = flags[blk];
+      if (!f) continue;
+      __syncthreads();
+      stage_tile<T, D>(s, k, n, h, blk * s.Bk, Ks);
+      stage_tile<T, D>(s, v, n, h, blk * s.Bk, Vs);
+      __syncthreads();
+      if (!active) continue;
+      const int p0 = blk * s.Bk;
+      const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
+      const bool selb = f & 1;
+      for (int pi = pbeg; pi < pend; ++pi) {
+        const bool inS = (t - (p0 + pi)) < s.window;
+        if (!selb && !inS) continue;
+        const float4 *kr = reinterpret_cast<const float4 *>(Ks) + pi * CH;
+        const float4 *vr = reinterpret_cast<const float4 *>(Vs) + pi * CH;
+        float part = 0.f, dpart = 0.f;
+#pragma unroll
+        for (int c = 0; c < NV; ++c) {
+          part = dot4(qv[c], kr[c * 4 + sub], part);
+          dpart = dot4(gv[c], vr[c * 4 + sub], dpart);
+        }
+        const float sv = group_sum(part, gmask) * sc2;
+        const float dP = group_sum(dpart, gmask);
+        float dSsum = 0.f;
+        if (selb) dSsum += exp2f(sv - lseL2) * (alpha * dP - deltaL);
+        if (inS) dSsum += exp2f(sv - lseS2) * (beta * dP - deltaS);
+        const float w = s.scale * dSsum;
+#pragma unroll
+        for (int c = 0; c < NV; ++c) axpy4(acc[c], w, kr[c * 4 + sub]);
+      }
+    }
+  }
+  if (!inrange) return;
+#pragma unroll
+  for (int c = 0; c < NV; ++c) st4(dq + ro + (c * 4 + sub) * 4, acc[c]);
+}
+
+// -------------------------------------------------------------------- backward: dK, dV
+template <typename T, int D>
+__global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
+    Shape s, const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
+    const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
+    const int32_t *__restrict__ idx, const float *__restrict__ lse,
+    const float *__restrict__ delta, const T *__restrict__ dout, T *__restrict__ dk,
+    T *__restrict__ dv) {
+  constexpr int NV = D / 16, CH = D / 4;
+  extern __shared__ float smf[];
+  float *Qs = smf, *Gs = Qs + s.Bk * D;
+  float *lLs = Gs + s.Bk * D, *lSs = lLs + s.Bk, *dLs = lSs + s.Bk, *dSs = dLs + s.Bk;
+  int *flags = reinterpret_cast<int *>(dSs + s.Bk);
+  const int j = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int tid = threadIdx.x, r = tid >> 2, sub = tid & 3;
+  const unsigned gmask = 0xFu << ((tid & 31) & ~3);
+  const int p = j * s.Bk + r;
+  const bool inrange = p < s.L, active = inrange && p >= pad0;
+  const int64_t BHL = (int64_t)s.B * s.H * s.L;
+  const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
+
+  // which query blocks visit this key block: bit 0 = selected it, bit 1 = window reaches it
+  for (int qb = j + tid; qb < s.M; qb += blockDim.x) {
+    const int32_t *row = idx + ((int64_t)u * s.M + qb) * s.topk;
+    int f = (qb * s.Bk - (j * s.Bk + s.Bk - 1) < s.window) ? 2 : 0;
+    for (int i = 0; i < s.topk; ++i) f |= (row[i] == j) ? 1 : 0;
+    flags[qb] = f;
+  }
+
+  float4 kv[NV], vv[NV], dka[NV], dva[NV];
+  const int64_t ro = row_offset(s, n, h, inrange ? p : 0);
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    const int64_t off = ro + (c * 4 + sub) * 4;
+    kv[c] = active ? ld4(k + off) : zero4();
+    vv[c] = active ? ld4(v + off) : zero4();
+    dka[c] = zero4();
+    dva[c] = zero4();
+  }
+  const float sc2 = s.scale * kLog2e;
+  const bool block_live = min((j + 1) * s.Bk, s.L) > pad0;
+  __syncthreads();
+
+  if (block_live) {
+    for (int qb = j; qb < s.M; ++qb) {
+      const int f = flags[qb];
+      if (!f) continue;
+      __syncthreads();
+      stage_tile<T, D>(s, q, n, h, qb * s.Bk, Qs);
+      stage_tile<T, D>(s, dout, n, h, qb * s.Bk, Gs);
+      for (int i = tid; i < s.Bk; i += blockDim.x) {
+        const int t = qb * s.Bk + i;
+        const bool ok = t < s.L;
+        lLs[i] = ok ? lse[(int64_t)u * s.L + t] * kLog2e : 0.f;
+        lSs[i] = ok ? lse[BHL + (int64_t)u * s.L + t] * kLog2e : 0.f;
+        dLs[i] = ok ? delta[(int64_t)u * s.L + t] : 0.f;
+        dSs[i] = ok ? delta[BHL + (int64_t)u * s.L + t] : 0.f;
+      }
+      __syncthreads();
+      if (!active) continue;
+      const int t0 = qb * s.Bk;
+      const int tbeg = max(0, p - t0), tend = min(s.Bk, s.L - t0);  // t >= p >= pad0
+      const bool selb = f & 1;
+      for (int ti = tbeg; ti < tend; ++ti) {
+        const bool inS = (t0 + ti - p) < s.window;
+        if (!selb && !inS) continue;
+        const float4 *qr = reinterpret_cast<const float4 *>(Qs) + ti * CH;
+        const float4 *gr = reinterpret_cast<const float4 *>(Gs) + ti * CH;
+        float part = 0.f, dpart = 0.f;
+#pragma unroll
+        for (int c = 0; c < NV; ++c) {
+          part = dot4(qr[c * 4 + sub], kv[c], part);
+          dpart = dot4(gr[c * 4 + sub], vv[c], dpart);
+        }
+        const float sv = group_sum(part, gmask) * sc2;
+        const float dP = group_sum(dpart, gmask);
+        float wv = 0.f, dSsum = 0.f;
+        if (selb) {
+          const float P = exp2f(sv - lLs[ti]);
+          wv = alpha * P;
+          dSsum = P * (alpha * dP - dLs[ti]);
+        }
+        if (inS) {
+          const float P = exp2f(sv - lSs[ti]);
+          wv = fmaf(beta, P, wv);
+          dSsum = fmaf(P, beta * dP - dSs[ti], dSsum);
+        }
+        const float wk = s.scale * dSsum;
+#pragma unroll
+        for (int c = 0; c < NV; ++c) {
+          axpy4(dva[c], wv, gr[c * 4 + sub]);
+          axpy4(dka[c], wk, qr[c * 4 + sub]);
+        }
+      }
+    }
+  }
+  if (!inrange) return;
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
+    st4(dk + ro + (c * 4 + sub) * 4, dka[c]);
+    st4(dv + ro + (c * 4 + sub) * 4, dva[c]);
+  }
+}
+
+}  // namespace
+
+// d alpha partials -> dgate[H][2]; one block per head, fixed reduction shape (deterministic).
+__global__ void __launch_bounds__(256) gate_grad_kernel(Shape s, const float *__restrict__ gate,
+                                                        const double *__restrict__ dalpha_part,
+                                                        float *__restrict__ dgate) {
+  __shared__ double red[256];
+  const int h = blockIdx.x;
+  double a = 0.0;
+  const int per = s.M, total = s.B * per;
+  for (int i = threadIdx.x; i < total; i += 256) {
+    const int n = i / per, qb = i % per;
+    a += dalpha_part[((int64_t)n * s.H + h) * s.M + qb];
+  }
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double al = 1.0 / (1.0 + exp(-((double)gate[h * 2 + 0] - (double)gate[h * 2 + 1])));
+    const double g0 = al * (1.0 - al) * red[0];
+    dgate[h * 2 + 0] = (float)g0;
+    dgate[h * 2 + 1] = (float)(-g0);
+  }
+}
+
+namespace {
+
+template <typename T, int D>
+int launch_fwd_t(const Shape &s, const T *q, const T *k, const T *v, const float *gate,
+                 const int32_t *seq_lens, const int32_t *idx, T *out, T *out_lt, T *out_st,
+                 float *lse, cudaStream_t st) {
+  const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.H);
+  const size_t smem = (size_t)2 * s.Bk * D * sizeof(float) + (size_t)s.M * sizeof(int);
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(fwd_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  {
+    LaunchScope ls(K_FWD_SIMT, st);
+    fwd_simt_kernel<T, D><<<grid, s.Bk * 4, smem, st>>>(s, q, k, v, gate, seq_lens, idx, out, out_lt,
+                                                        out_st, lse);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
+template <typename T, int D>
+int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float *gate,
+                 const int32_t *seq_lens, const int32_t *idx, const T *out_lt, const T *out_st,
+                 const float *lse, const T *dout, T *dq, T *dk, T *dv, float *dgate,
+                 const Workspace &ws, cudaStream_t st) {
+  const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.H);
+  const size_t smem_q = (size_t)2 * s.Bk * D * sizeof(float) +
+                        (size_t)(s.M + (s.M & 1)) * sizeof(int) + (size_t)s.Bk * sizeof(double);
+  if (smem_q > 48 * 1024 &&
+      cudaFuncSetAttribute(bwd_dq_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem_q) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  {
+    LaunchScope ls(K_BWD_DQ_SIMT, st);
+    bwd_dq_simt_kernel<T, D><<<grid, s.Bk * 4, smem_q, st>>>(s, q, k, v, gate, seq_lens, idx, out_lt,
+                                                             out_st, lse, dout, dq, ws.delta,
+                                                             ws.dalpha);
+  }
+  const size_t smem_k = (size_t)(2 * s.Bk * D + 4 * s.Bk) * sizeof(float) + (size_t)s.M * sizeof(int);
+  if (smem_k > 48 * 1024 &&
+      cudaFuncSetAttribute(bwd_dkdv_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem_k) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  {
+    LaunchScope ls(K_BWD_DKDV_SIMT, st);
+    bwd_dkdv_simt_kernel<T, D><<<grid, s.Bk * 4, smem_k, st>>>(s, q, k, v, gate, seq_lens, idx, lse,
+                                                               ws.delta, dout, dk, dv);
+  }
+  {
+    LaunchScope ls(K_GATE_GRAD, st);
+    gate_grad_kernel<<<s.H, 256, 0, st>>>(s, gate, ws.dalpha, dgate);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_fwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,
+                    const float *gate, const int32_t *seq_lens, const int32_t *idx, void *out,
+                    void *out_lt, void *out_st, float *lse, const Workspace &, cudaStream_t st) {
+  typedef __nv_bfloat16 bf;
+  if (dtype == BLOSSOM_DTYPE_FP32) {
+    if (s.D == 32)
+      return launch_fwd_t<float, 32>(s, (const float *)q, (const float *)k, (const float *)v, gate, seq_lens, idx, (float *)out, (float *)out_lt, (float *)out_st, lse, st);
+    return launch_fwd_t<float, 64>(s, (const float *)q, (const float *)k, (const float *)v, gate, seq_lens, idx, (float *)out, (float *)out_lt, (float *)out_st, lse, st);
+  }
+  if (s.D == 32)
+    return launch_fwd_t<bf, 32>(s, (const bf *)q, (const bf *)k, (const bf *)v, gate, seq_lens, idx, (bf *)out, (bf *)out_lt, (bf *)out_st, lse, st);
+  return launch_fwd_t<bf, 64>(s, (const bf *)q, (const bf *)k, (const bf *)v, gate, seq_lens, idx, (bf *)out, (bf *)out_lt, (bf *)out_st, lse, st);
+}
+
+int launch_bwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,
+                    const float *gate, const int32_t *seq_lens, const int32_t *idx,
+                    const void *out_lt, const void *out_st, const float *lse, const void *dout,
+                    void *dq, void *dk, void *dv, float *dgate, const Workspace &ws,
+                    cudaStream_t st) {
+  typedef __nv_bfloat16 bf;
+  if (dtype == BLOSSOM_DTYPE_FP32) {
+    if (s.D == 32)
+      return launch_bwd_t<float, 32>(s, (const float *)q, (const float *)k, (const float *)v, gate, seq_lens, idx, (const float *)out_lt, (const float *)out_st, lse, (const float *)dout, (float *)dq, (float *)dk, (float *)dv, dgate, ws, st);
+    return launch_bwd_t<float, 64>(s, (const float *)q, (const float *)k, (const float *)v, gate, seq_lens, idx, (const float *)out_lt, (const float *)out_st, lse, (const float *)dout, (float *)dq, (float *)dk, (float *)dv, dgate, ws, st);
+  }
+  if (s.D == 32)
+    return launch_bwd_t<bf, 32>(s, (const bf *)q, (const bf *)k, (const bf *)v, gate, seq_lens, idx, (const bf *)out_lt, (const bf *)out_st, lse, (const bf *)dout, (bf *)dq, (bf *)dk, (bf *)dv, dgate, ws, st);
+  return launch_bwd_t<bf, 64>(s, (const bf *)q, (const bf *)k, (const bf *)v, gate, seq_lens, idx, (const bf *)out_lt, (const bf *)out_st, lse, (const bf *)dout, (bf *)dq, (bf *)dk, (bf *)dv, dgate, ws, st);
+}
+
+}  // namespace blossom

@@ -1,0 +1,88 @@
+// Shared device/host declarations of the blossom CUDA library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/blossom.h"
+
+namespace blossom {
+
+// Problem shape handed to every kernel by value.
+struct Shape {
+  int B, H, L, D, Bk, topk, window, M;
+  float scale;     // attention logit scale (fp32 arithmetic of the attention kernels)
+  double scale_d;  // the same scale in double for the fp64 block scoring
+  int64_t sb, sh, sl;  // element strides of q-shaped tensors
+};
+
+// Device scratch carved out of the caller's workspace.
+struct Workspace {
+  int32_t *status;   // [4] word 0: device status (0 = ok)
+  double *kmean;     // [B][H][M][D]  mean of each block's valid keys (Eq. 9 summary)
+  int32_t *klive;    // [B][H][M]     number of valid keys in the block
+  float *delta;      // [2][B][H][L]  rowsum(G_branch o O_branch) for the backward
+  double *dalpha;    // [B][H][M]     per query block partial of d alpha
+  float *dq_acc;     // [B][H][L][D]  fp32 dQ accumulator of the tensor-core backward
+  size_t bytes;
+};
+
+Workspace carve_workspace(const Shape &s, void *base);
+
+extern unsigned long long g_launches;  // host-side launch counter
+
+// Kernel identifiers reported by the optional per-launch event profile.
+enum KernelId {
+  K_SUMMARY = 0, K_SCORE_SELECT, K_FWD_SIMT, K_BWD_DQ_SIMT, K_BWD_DKDV_SIMT, K_GATE_GRAD,
+  K_FWD_TC, K_BWD_PRE_TC, K_BWD_TC, K_BWD_CVT_TC, K_COUNT
+};
+void prof_mark(int id, int phase, cudaStream_t st);  // no-op unless a profile is running
+
+// Wrap every kernel launch: counts it and, when a profile is running, brackets it with events.
+struct LaunchScope {
+  int id;
+  cudaStream_t st;
+  LaunchScope(int id_, cudaStream_t st_) : id(id_), st(st_) { ++g_launches; prof_mark(id, 0, st); }
+  ~LaunchScope() { prof_mark(id, 1, st); }
+};
+
+// ---- element access: 4 consecutive elements as float4 ------------------------------------
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 ld4(const __nv_bfloat16 *p) {
+  uint2 r = *reinterpret_cast<const uint2 *>(p);
+  float4 o;
+  o.x = __uint_as_float(r.x << 16);
+  o.y = __uint_as_float(r.x & 0xffff0000u);
+  o.z = __uint_as_float(r.y << 16);
+  o.w = __uint_as_float(r.y & 0xffff0000u);
+  return o;
+}
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void st4(__nv_bfloat16 *p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);  // round to nearest even, once
+  __nv_bfloat162 b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 r;
+  r.x = *reinterpret_cast<uint32_t *>(&a);
+  r.y = *reinterpret_cast<uint32_t *>(&b);
+  *reinterpret_cast<uint2 *>(p) = r;
+}
+__device__ __forceinline__ float ld1(const float *p) { return *p; }
+__device__ __forceinline__ float ld1(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+
+__device__ __forceinline__ int64_t row_offset(const Shape &s, int n, int h, int t) {
+  return (int64_t)n * s.sb + (int64_t)h * s.sh + (int64_t)t * s.sl;
+}
+
+// launchers (one translation unit each)
+int launch_select(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
+                  int32_t *idx, const Workspace &ws, cudaStream_t st);
+int launch_fwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,
+                    const float *gate, const int32_t *seq_lens, const int32_t *idx, void *out,
+                    void *out_lt, void *out_st, float *lse, const Workspace &ws, cudaStream_t st);
+int launch_bwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,
+                    const float *gate, const int32_t *seq_lens, const int32_t *idx,
+                    const void *out_lt, const void *out_st, const float *lse, const void *dout,
+                    void *dq, void *dk, void *dv, float *dgate, const Workspace &ws,
+                    cudaStream_t st);
+
+}  // namespace blossom

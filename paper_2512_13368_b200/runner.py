@@ -1,0 +1,75 @@
+"""Device-buffer plumbing around the C ABI: upload a workload, allocate outputs and the
+workspace with PyTorch, call the library, hand results back.  No arithmetic of the method
+happens here."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding
+from .workloads import Workload
+
+_TORCH_DTYPE = {"fp32": torch.float32, "bf16": torch.bfloat16}
+
+
+class DeviceProblem:
+    """All device buffers of one forward + backward call for a workload."""
+
+    def __init__(self, w: Workload, device="cuda:0", sm_scale=0.0, training=True):
+        self.w = w
+        self.device = torch.device(device)
+        dt = _TORCH_DTYPE[w.dtype]
+        self.dt = dt
+        up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(self.device).to(dt)  # noqa: E731
+        self.q, self.k, self.v, self.dout = up(w.q), up(w.k), up(w.v), up(w.dout)
+        self.gate = torch.from_numpy(np.ascontiguousarray(w.gate, dtype=np.float32)).to(self.device)
+        self.seq_lens = None
+        if w.seq_lens is not None:
+            self.seq_lens = torch.from_numpy(w.seq_lens.astype(np.int32)).to(self.device)
+        self.params = binding.make_params(w.B, w.H, w.L, w.D, w.block, w.topk, w.window, w.dtype,
+                                          sm_scale=sm_scale)
+        self.alloc_outputs(training)
+
+    def alloc_outputs(self, training=True):
+        w, dev = self.w, self.device
+        shape = (w.B, w.H, w.L, w.D)
+        e = lambda: torch.empty(shape, dtype=self.dt, device=dev)  # noqa: E731
+        self.idx = torch.empty((w.B, w.H, w.n_blocks, w.topk), dtype=torch.int32, device=dev)
+        self.out = e()
+        self.out_lt = e() if training else None
+        self.out_st = e() if training else None
+        self.lse = torch.empty((2, w.B, w.H, w.L), dtype=torch.float32, device=dev) if training else None
+        self.dq, self.dk, self.dv = (e(), e(), e()) if training else (None, None, None)
+        self.dgate = torch.empty((w.H, 2), dtype=torch.float32, device=dev)
+        nbytes = binding.blossom_workspace_bytes(self.params)
+        if nbytes == 0:
+            raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+
+    # -- calls ---------------------------------------------------------------------------
+    def select(self, stream=None):
+        binding.blossom_select_blocks(self.params, self.q, self.k, self.seq_lens, self.idx,
+                                      self.workspace, stream=stream)
+
+    def forward(self, idx_is_input=False, stream=None):
+        binding.blossom_attn_fwd(self.params, self.q, self.k, self.v, self.gate, self.seq_lens,
+                                 self.idx, int(idx_is_input), self.out, self.out_lt, self.out_st,
+                                 self.lse, self.workspace, stream=stream)
+
+    def backward(self, stream=None):
+        binding.blossom_attn_bwd(self.params, self.q, self.k, self.v, self.gate, self.seq_lens,
+                                 self.idx, self.out_lt, self.out_st, self.lse, self.dout, self.dq,
+                                 self.dk, self.dv, self.dgate, self.workspace, stream=stream)
+
+    def step(self, stream=None):
+        """One pass of the whole hot path: selection + forward + backward."""
+        self.forward(False, stream)
+        self.backward(stream)
+
+    # -- results -------------------------------------------------------------------------
+    def results(self) -> dict:
+        torch.cuda.synchronize(self.device)
+        f = lambda t: None if t is None else t.float().cpu().numpy()  # noqa: E731
+        return {"idx": self.idx.cpu().numpy(), "out": f(self.out), "out_lt": f(self.out_lt),
+                "out_st": f(self.out_st), "lse": f(self.lse), "dq": f(self.dq), "dk": f(self.dk),
+                "dv": f(self.dv), "dgate": f(self.dgate)}

@@ -1,0 +1,91 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, sizes workspaces, names its statuses and rejects bad arguments before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2512_13368_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def header_functions():
+    text = open(os.path.join(ROOT, "include", "blossom.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(blossom_[a-z_]+)\s*\(", text)))
+
+
+def test_exports_match_header(lib):
+    names = header_functions()
+    assert set(names) == set(binding.EXPORTS), names
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert binding.blossom_version() >= 100
+    seen = {binding.blossom_status_string(i) for i in range(6)}
+    assert len(seen) == 6 and "ok" in seen
+    assert binding.blossom_status_string(99) == "unknown status"
+
+
+def good(**kw):
+    d = dict(batch=4, heads=2, seq_len=64, head_dim=32, block_size=8, top_k=2, window=16, dtype="fp32")
+    d.update(kw)
+    return binding.make_params(**d)
+
+
+def test_workspace_bytes(lib):
+    n = binding.blossom_workspace_bytes(good())
+    assert n > 0 and n % 256 == 0
+    assert binding.blossom_workspace_bytes(good(batch=8)) > n
+    for bad in (dict(batch=0), dict(head_dim=48), dict(block_size=12), dict(top_k=0), dict(window=0),
+                dict(kv_heads=1), dict(causal=0), dict(select_mode=1), dict(dtype=7),
+                dict(seq_len=8 * 1025), dict(strides=(4096, 2048, 33)), dict(sm_scale=-1.0)):
+        assert binding.blossom_workspace_bytes(good(**bad)) == 0, bad
+
+
+def test_argument_validation_precedes_any_launch(lib):
+    p = good()
+    A = 1 << 20  # a fake, aligned, never-dereferenced device address
+    ws_bytes = binding.blossom_workspace_bytes(p)
+    E = binding
+    # NULL tensors
+    assert E.blossom_attn_fwd(p, None, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
+    # misaligned q
+    assert E.blossom_attn_fwd(p, A + 4, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
+    # only one of the saved outputs
+    assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
+    # training outputs without lse
+    assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, None, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
+    # workspace: missing, misaligned, short
+    assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, None, 0, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
+    assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, A + 64, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
+    assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes - 1, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
+    # unsupported but legal requests
+    assert E.blossom_attn_fwd(good(kv_heads=1), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
+    assert E.blossom_select_blocks(good(head_dim=128), A, A, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
+    assert E.blossom_select_blocks(p, A, None, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
+    # backward: every tensor is required
+    args = [A] * 14          # q k v gate seq_lens idx out_lt out_st lse dout dq dk dv dgate
+    for i in (0, 3, 5, 6, 8, 9, 10, 13):
+        a = list(args)
+        a[i] = None
+        a[4] = None              # seq_lens may always be NULL
+        assert E.blossom_attn_bwd(p, *a, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG, i
+    with pytest.raises(E.BlossomError):
+        E.blossom_select_blocks(p, None, None, None, None, None, 0, stream=0)
+
+
+def test_params_struct_layout_matches_header():
+    # 12 x 4-byte fields then three int64 strides: 72 bytes with natural alignment
+    assert ctypes.sizeof(binding.blossom_params) == 72
+    assert binding.blossom_params.stride_b.offset == 48
