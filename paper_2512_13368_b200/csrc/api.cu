@@ -1,6 +1,7 @@
 // C ABI of the blossom library: argument validation, workspace carving and dispatch.
 // Every check happens on the host before anything is launched.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -24,6 +25,11 @@ void prof_mark(int id, int phase, cudaStream_t st) {
     cudaEventRecord(g_prof_events[2 * g_prof_n + 1], st);
     ++g_prof_n;
   }
+}
+
+bool force_simt() {
+  const char *e = getenv("BLOSSOM_FORCE_SIMT");
+  return e && e[0] && e[0] != '0';
 }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -138,6 +144,9 @@ int blossom_attn_fwd(const blossom_params *params, const void *q, const void *k,
     rc = launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, st);
     if (rc) return rc;
   }
+  if (!force_simt() && tc::fwd_tc_supported(s, params->dtype))
+    return tc::launch_fwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out, out_lt, out_st, lse, ws,
+                             st);
   return launch_fwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out, out_lt,
                          out_st, lse, ws, st);
 }

@@ -212,15 +212,12 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
     delta[(int64_t)u * s.L + t] = deltaL;
     delta[BHL + (int64_t)u * s.L + t] = deltaS;
   }
-  if (sub == 0) red[r] = active ? (double)dL - (double)dS : 0.0;
   const float sc2 = s.scale * kLog2e;
   const bool block_live = min((qb + 1) * s.Bk, s.L) > pad0;
+  // d alpha of the row = <G, O_lt - O_st> = sum_p (P_lt - P_st) dP, accumulated from the fp32
+  // probabilities below rather than from the stored (rounded) branch outputs
+  float dal = 0.f;
   __syncthreads();
-  if (tid == 0) {
-    double a = 0.0;
-    for (int i = 0; i < s.Bk; ++i) a += red[i];  // fixed order
-    dalpha_part[(int64_t)u * s.M + qb] = a;
-  }
 
   if (block_live) {
     for (int blk = 0; blk <= qb; ++blk) {
@@ -248,13 +245,28 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
         const float sv = group_sum(part, gmask) * sc2;
         const float dP = group_sum(dpart, gmask);
         float dSsum = 0.f;
-        if (selb) dSsum += exp2f(sv - lseL2) * (alpha * dP - deltaL);
-        if (inS) dSsum += exp2f(sv - lseS2) * (beta * dP - deltaS);
+        if (selb) {
+          const float P = exp2f(sv - lseL2);
+          dSsum = P * (alpha * dP - deltaL);
+          dal = fmaf(P, dP, dal);
+        }
+        if (inS) {
+          const float P = exp2f(sv - lseS2);
+          dSsum = fmaf(P, beta * dP - deltaS, dSsum);
+          dal = fmaf(-P, dP, dal);
+        }
         const float w = s.scale * dSsum;
 #pragma unroll
         for (int c = 0; c < NV; ++c) axpy4(acc[c], w, kr[c * 4 + sub]);
       }
     }
+  }
+  if (sub == 0) red[r] = active ? (double)dal : 0.0;
+  __syncthreads();
+  if (tid == 0) {
+    double a = 0.0;
+    for (int i = 0; i < s.Bk; ++i) a += red[i];  // fixed order
+    dalpha_part[(int64_t)u * s.M + qb] = a;
   }
   if (!inrange) return;
 #pragma unroll

@@ -85,4 +85,14 @@ int launch_bwd_simt(const Shape &s, int dtype, const void *q, const void *k, con
                     void *dq, void *dk, void *dv, float *dgate, const Workspace &ws,
                     cudaStream_t st);
 
+namespace tc {
+bool fwd_tc_supported(const Shape &s, int dtype);
+int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                  const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt, void *out_st,
+                  float *lse, const Workspace &ws, cudaStream_t st);
+}  // namespace tc
+
+// BLOSSOM_FORCE_SIMT=1 in the environment routes every call to the fp32 CUDA-core kernels.
+bool force_simt();
+
 }  // namespace blossom

@@ -19,9 +19,10 @@ BF16_REL = 2e-2
 TIE_REL = 1e-6
 
 
-def check_indices(w, gpu_idx):
+def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
-    ref_idx, scores = oracle.select_blocks(w.q, w.k, w.block, w.topk, w.seq_lens, return_scores=True)
+    ref_idx, scores = oracle.select_blocks(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
+                                            return_scores=True)
     assert gpu_idx.shape == ref_idx.shape and gpu_idx.dtype == np.int32
     bad = np.argwhere((gpu_idx != ref_idx).any(-1))
     forgiven = 0
@@ -52,7 +53,7 @@ def tolerance(w, ref):
 
 def check_forward_backward(w, res, sm_scale=None, backward=True):
     """res: dict of numpy arrays from the CUDA path.  Returns a dict of max-abs errors."""
-    forgiven = check_indices(w, res["idx"])
+    forgiven = check_indices(w, res["idx"], sm_scale)
     ref = oracle.forward(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
                          idx=res["idx"])
     errs = {"near_tie_rows": forgiven}
