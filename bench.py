@@ -75,10 +75,11 @@ def work_model(w):
     lse_b = 2 * w.B * w.H * w.L * 4
     idx_b = w.B * w.H * M * w.topk * 4
     gemms = {"fwd": 2, "bwd": 5, "fwd_simt": 2, "fwd_tc": 2, "bwd_dq_simt": 3, "bwd_dkdv_simt": 2,
-             "bwd_tc": 5}
+             "bwd_dq_tc": 3, "bwd_dkdv_tc": 2}
     byts = {"fwd": 6 * T + lse_b + idx_b, "bwd": 9 * T + 2 * lse_b + idx_b}
-    byts.update({"fwd_simt": byts["fwd"], "fwd_tc": byts["fwd"], "bwd_tc": byts["bwd"],
+    byts.update({"fwd_simt": byts["fwd"], "fwd_tc": byts["fwd"],
                  "bwd_dq_simt": 7 * T + 2 * lse_b, "bwd_dkdv_simt": 6 * T + 2 * lse_b,
+                 "bwd_dq_tc": 7 * T + 2 * lse_b, "bwd_dkdv_tc": 6 * T + 2 * lse_b,
                  "summary": T, "score_select": T})
     return {"tiles_lt": tiles_L, "tiles_st": tiles_S, "tile_flops": tile_flops,
             "flops": {k: g * tb * tile_flops for k, g in gemms.items()}, "bytes": byts,

@@ -170,6 +170,12 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
   Workspace ws;
   rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
   if (rc) return rc;
+  if (!force_simt() && tc::fwd_tc_supported(s, params->dtype)) {
+    rc = tc::launch_bwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out_lt, out_st, lse, dout, dq,
+                           dk, dv, ws, (cudaStream_t)stream);
+    if (rc) return rc;
+    return launch_gate_grad(s, gate_logits, ws, dgate, (cudaStream_t)stream);
+  }
   return launch_bwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out_lt,
                          out_st, lse, dout, dq, dk, dv, dgate, ws, (cudaStream_t)stream);
 }
@@ -234,7 +240,7 @@ int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
 const char *blossom_kernel_name(int id) {
   static const char *names[K_COUNT] = {
       "summary", "score_select", "fwd_simt", "bwd_dq_simt", "bwd_dkdv_simt", "gate_grad",
-      "fwd_tc", "bwd_pre_tc", "bwd_tc", "bwd_cvt_tc"};
+      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc"};
   return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

@@ -456,14 +456,19 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
     bwd_dkdv_simt_kernel<T, D><<<grid, s.Bk * 4, smem_k, st>>>(s, q, k, v, gate, seq_lens, idx, lse,
                                                                ws.delta, dout, dk, dv);
   }
+  return launch_gate_grad(s, gate, ws, dgate, st);
+}
+
+}  // namespace
+
+int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, float *dgate,
+                     cudaStream_t st) {
   {
     LaunchScope ls(K_GATE_GRAD, st);
     gate_grad_kernel<<<s.H, 256, 0, st>>>(s, gate, ws.dalpha, dgate);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
-
-}  // namespace
 
 int launch_fwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,
                     const float *gate, const int32_t *seq_lens, const int32_t *idx, void *out,

@@ -34,7 +34,7 @@ extern unsigned long long g_launches;  // host-side launch counter
 // Kernel identifiers reported by the optional per-launch event profile.
 enum KernelId {
   K_SUMMARY = 0, K_SCORE_SELECT, K_FWD_SIMT, K_BWD_DQ_SIMT, K_BWD_DKDV_SIMT, K_GATE_GRAD,
-  K_FWD_TC, K_BWD_PRE_TC, K_BWD_TC, K_BWD_CVT_TC, K_COUNT
+  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_COUNT
 };
 void prof_mark(int id, int phase, cudaStream_t st);  // no-op unless a profile is running
 
@@ -85,8 +85,15 @@ int launch_bwd_simt(const Shape &s, int dtype, const void *q, const void *k, con
                     void *dq, void *dk, void *dv, float *dgate, const Workspace &ws,
                     cudaStream_t st);
 
+int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, float *dgate,
+                     cudaStream_t st);
+
 namespace tc {
 bool fwd_tc_supported(const Shape &s, int dtype);
+int launch_bwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                  const int32_t *seq_lens, const int32_t *idx, const void *out_lt, const void *out_st,
+                  const float *lse, const void *dout, void *dq, void *dk, void *dv,
+                  const Workspace &ws, cudaStream_t st);
 int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                   const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt, void *out_st,
                   float *lse, const Workspace &ws, cudaStream_t st);
