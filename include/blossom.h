@@ -46,7 +46,8 @@ typedef enum {
   BLOSSOM_ERR_UNSUPPORTED = 2, /* a legal request this version does not implement               */
   BLOSSOM_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned (256 B) or smaller than required   */
   BLOSSOM_ERR_CUDA = 4,        /* a CUDA launch or runtime call failed                          */
-  BLOSSOM_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see blossom_device_status)*/
+  BLOSSOM_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (see blossom_device_status)*/
+  BLOSSOM_ERR_TOO_LARGE = 6    /* problem exceeds the fixed capacity of a no-allocation entry   */
 } blossom_status;
 
 enum { BLOSSOM_DTYPE_FP32 = 0, BLOSSOM_DTYPE_BF16 = 1 };
@@ -91,6 +92,34 @@ size_t blossom_workspace_bytes(const blossom_params *params /* host */);
 int blossom_select_blocks(const blossom_params *params /* host */, const void *q, const void *k,
                           const int32_t *seq_lens, int32_t *block_idx, void *workspace,
                           size_t workspace_bytes, blossom_stream_t stream);
+
+/*
+ * blossom_select_blocks for callers that cannot provide a workspace.  (The paper has no
+ * counterpart: this is a packaging variant of the selection above, same inputs, same result.)
+ *
+ * Who needs it: code that runs where device memory can no longer be requested -- inside a
+ * serving process whose memory pool was handed out in full at start-up, in a plug-in that is
+ * given tensors but no allocator, or on a thread that must not take the allocator's lock.  Such a
+ * caller cannot size and allocate the workspace the other entry points ask for, so here the
+ * scratch (per-block key means and live counts) is a fixed array inside the library image.
+ *
+ *   - Nothing on this call path allocates or frees memory: no cudaMalloc / cudaFree, no library
+ *     allocator.  The array (4 MiB + 32 KiB) is resident on every GPU that loads the library,
+ *     from load to exit, whether or not this function is ever called.
+ *   - Capacity: batch * heads * M <= 8192 and batch * heads * M * head_dim <= 524288
+ *     (M = ceil(seq_len / block_size)); larger problems return BLOSSOM_ERR_TOO_LARGE before
+ *     anything is launched.  All other argument rules are those of blossom_select_blocks.
+ *   - The first call on each device looks up the array's device address (a runtime query, done
+ *     once per device with that device current).  Make that first call outside any stream
+ *     capture; later calls only launch kernels on `stream`.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left in it;
+ *     each call overwrites every entry before reading it, so no clearing is needed.  Two calls
+ *     whose kernels may run at the same time on one device (different streams, or different
+ *     host threads) race on it and must be serialised by the caller.
+ */
+int blossom_select_blocks_static(const blossom_params *params /* host */, const void *q,
+                                 const void *k, const int32_t *seq_lens, int32_t *block_idx,
+                                 blossom_stream_t stream);
 
 /*
  * Forward (paper: Eq. 14 and 16 for the selected-block branch, Eq. 15 first case under the

@@ -19,11 +19,13 @@ BLOSSOM_ERR_UNSUPPORTED = 2
 BLOSSOM_ERR_WORKSPACE = 3
 BLOSSOM_ERR_CUDA = 4
 BLOSSOM_ERR_TIMEOUT = 5
+BLOSSOM_ERR_TOO_LARGE = 6
 DTYPE_FP32 = 0
 DTYPE_BF16 = 1
 
 EXPORTS = (
-    "blossom_workspace_bytes", "blossom_select_blocks", "blossom_attn_fwd", "blossom_attn_bwd",
+    "blossom_workspace_bytes", "blossom_select_blocks", "blossom_select_blocks_static",
+    "blossom_attn_fwd", "blossom_attn_bwd",
     "blossom_device_status", "blossom_status_string", "blossom_version", "blossom_launch_count",
     "blossom_profile_start", "blossom_profile_stop", "blossom_kernel_name",
 )
@@ -64,6 +66,8 @@ def load():
     lib.blossom_workspace_bytes.argtypes = [pp]
     lib.blossom_select_blocks.restype = ctypes.c_int
     lib.blossom_select_blocks.argtypes = [pp, vp, vp, vp, vp, vp, sz, vp]
+    lib.blossom_select_blocks_static.restype = ctypes.c_int
+    lib.blossom_select_blocks_static.argtypes = [pp, vp, vp, vp, vp, vp]
     lib.blossom_attn_fwd.restype = ctypes.c_int
     lib.blossom_attn_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.blossom_attn_bwd.restype = ctypes.c_int
@@ -143,6 +147,18 @@ def blossom_select_blocks(params, q, k, seq_lens, block_idx, workspace, workspac
                                       _stream(stream))
     if rc and check:
         raise BlossomError(rc, "blossom_select_blocks")
+    return rc
+
+
+def blossom_select_blocks_static(params, q, k, seq_lens, block_idx, stream=None, check=True) -> int:
+    """Selection without a caller workspace: the scratch is a fixed array inside the library, so
+    nothing on the path allocates.  For callers that are handed tensors but may not allocate
+    device memory themselves.  Capacity-limited (see include/blossom.h); calls that could overlap
+    on one device must be serialised by the caller."""
+    rc = load().blossom_select_blocks_static(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(seq_lens),
+                                             _ptr(block_idx), _stream(stream))
+    if rc and check:
+        raise BlossomError(rc, "blossom_select_blocks_static")
     return rc
 
 

@@ -122,6 +122,18 @@ int blossom_select_blocks(const blossom_params *params, const void *q, const voi
   return launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, (cudaStream_t)stream);
 }
 
+int blossom_select_blocks_static(const blossom_params *params, const void *q, const void *k,
+                                 const int32_t *seq_lens, int32_t *block_idx,
+                                 blossom_stream_t stream) {
+  Shape s;
+  int rc = make_shape(params, &s);
+  if (rc) return rc;
+  if (!q || !k || !block_idx) return BLOSSOM_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(block_idx, 4) || misaligned(seq_lens, 4))
+    return BLOSSOM_ERR_INVALID_ARG;
+  return launch_select_static(s, params->dtype, q, k, seq_lens, block_idx, (cudaStream_t)stream);
+}
+
 int blossom_attn_fwd(const blossom_params *params, const void *q, const void *k, const void *v,
                      const float *gate_logits, const int32_t *seq_lens, int32_t *block_idx,
                      int32_t idx_is_input, void *out, void *out_lt, void *out_st, float *lse,
@@ -196,6 +208,7 @@ const char *blossom_status_string(int status) {
     case BLOSSOM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case BLOSSOM_ERR_CUDA: return "CUDA error";
     case BLOSSOM_ERR_TIMEOUT: return "device-side wait timed out";
+    case BLOSSOM_ERR_TOO_LARGE: return "problem exceeds the built-in scratch capacity";
     default: return "unknown status";
   }
 }

@@ -85,6 +85,9 @@ int launch_bwd_simt(const Shape &s, int dtype, const void *q, const void *k, con
                     void *dq, void *dk, void *dv, float *dgate, const Workspace &ws,
                     cudaStream_t st);
 
+int launch_select_static(const Shape &s, int dtype, const void *q, const void *k,
+                         const int32_t *seq_lens, int32_t *idx, cudaStream_t st);
+size_t select_static_capacity_bytes();
 int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, float *dgate,
                      cudaStream_t st);
 

@@ -215,4 +215,39 @@ int launch_select(const Shape &s, int dtype, const void *q, const void *k, const
   return launch_select_t<__nv_bfloat16, 64>(s, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, seq_lens, idx, ws, st);
 }
 
+// ---- selection with built-in scratch (no allocation anywhere on the call path) -------------
+// The block means and live counts that blossom_select_blocks keeps in the caller's workspace
+// live here in one array that is part of the loaded module.  Every launch overwrites each entry
+// it later reads, so nothing has to start at zero and stale contents of earlier calls are
+// harmless; two calls in flight at once on one device would overwrite each other's means.
+constexpr size_t kStaticMeanElems = 524288;  // doubles: batch * heads * M * head_dim may not exceed this
+constexpr size_t kStaticBlocks = 8192;       // int32:   batch * heads * M may not exceed this
+constexpr size_t kStaticBytes = kStaticMeanElems * sizeof(double) + kStaticBlocks * sizeof(int32_t);
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+static void *g_scratch_addr[kMaxDevices] = {nullptr};  // device address of the array, per device
+
+size_t select_static_capacity_bytes() { return kStaticBytes; }
+
+int launch_select_static(const Shape &s, int dtype, const void *q, const void *k,
+                         const int32_t *seq_lens, int32_t *idx, cudaStream_t st) {
+  const size_t blocks = (size_t)s.B * s.H * s.M;
+  if (blocks > kStaticBlocks || blocks * (size_t)s.D > kStaticMeanElems) return BLOSSOM_ERR_TOO_LARGE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BLOSSOM_ERR_CUDA;
+  if (!g_scratch_addr[dev]) {
+    // In host code the array's name is only a handle: ask the runtime for its device address on
+    // the current device (once per device) and hand that to the kernels.
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || !p) return BLOSSOM_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  unsigned char *base = static_cast<unsigned char *>(g_scratch_addr[dev]);
+  Workspace ws = {};
+  ws.kmean = reinterpret_cast<double *>(base);
+  ws.klive = reinterpret_cast<int32_t *>(base + kStaticMeanElems * sizeof(double));
+  return launch_select(s, dtype, q, k, seq_lens, idx, ws, st);
+}
+
 }  // namespace blossom
