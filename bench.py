@@ -191,6 +191,9 @@ def main():
     ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the batch size (profiling captures on a smaller case; not a bench line)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -200,7 +203,8 @@ def main():
     from paper_2512_13368_b200 import workloads
     if args.impl == "reference" and rank != 0:
         return 0
-    w = workloads.CONFIGS[args.config]()
+    w = workloads.CONFIGS[args.config](B=args.batch) if (args.batch and args.config != 1) \
+        else workloads.CONFIGS[args.config]()
     cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "seq_len": w.L, "head_dim": w.D,
                 "block_size": w.block, "top_k": w.topk, "window": w.window, "storage": w.dtype,
                 "padding": "left, lengths U{5..200}" if w.seq_lens is not None else "none",
@@ -330,20 +334,22 @@ def main():
         for k, h in h_out.items():
             h.copy_(getattr(p, k), non_blocking=True)
 
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    e1.record()
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
-    nb = lambda t: t.numel() * t.element_size()  # noqa: E731
-    e2e = {"value": world * w.tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": sum(nb(t) for t in h_in.values()) + (nb(h_sl) if h_sl is not None else 0),
-           "d2h_bytes_per_step": sum(nb(t) for t in h_out.values())}
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+        nb = lambda t: t.numel() * t.element_size()  # noqa: E731
+        e2e = {"value": world * w.tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": sum(nb(t) for t in h_in.values()) + (nb(h_sl) if h_sl is not None else 0),
+               "d2h_bytes_per_step": sum(nb(t) for t in h_out.values())}
 
     # ---- the oracle on the host cores (rank 0, N = 1 only)
     cpu = None
