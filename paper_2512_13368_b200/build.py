@@ -40,6 +40,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     headers = glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(HERE, "..", "include", "blossom.h")]
     objs = []
     procs = []
+    live = {os.path.basename(x)[:-3] + ".o" for x in sources()}
+    for f in os.listdir(OBJ):  # stale objects of sources that no longer exist
+        if f.endswith(".o") and f not in live:
+            os.remove(os.path.join(OBJ, f))
     for src in sources():
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
