@@ -49,7 +49,7 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.klive = reinterpret_cast<int32_t *>(take(units * s.M * sizeof(int32_t)));
   w.delta = reinterpret_cast<float *>(take(2 * units * s.L * sizeof(float)));
   w.dalpha = reinterpret_cast<double *>(take(units * s.M * sizeof(double)));
-  w.dq_acc = nullptr;
+  w.qstats = reinterpret_cast<float4 *>(take(units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4)));
   w.bytes = off;
   return w;
 }

@@ -1,0 +1,710 @@
+// Tensor-core backward of the fused two-branch attention (bf16 storage, fp32 accumulate): two
+// kernels, both deterministic (no atomics on any gradient), both recomputing the probabilities
+// from the saved log-sum-exps.
+//
+// CTA = 288 threads: warps 0..7 compute, warp 8 is the producer (one lane issues every TMA load
+// and every tcgen05.mma).  A CTA owns a resident 128-row tile (rows = TMEM lanes) and streams
+// 64-row tiles past it.  Row r of the 128 is shared by two compute threads: warp w and warp w + 4
+// both address TMEM lane quarter w % 4; the first takes columns 0..31 of a 64-column tile, the
+// second columns 32..63.  The bf16 operands of the second-stage products (dS, and in the dK/dV
+// kernel W^T and dS^T) are written to tensor memory and read from there by the MMA.
+//
+//  dQ     resident Q, dO (128 queries); streams K, V 64-key tiles (same walk as the forward).
+//         Tensor memory: S [0,64), dP [64,128), dS [128,160) (bf16 pairs), dQ [160,160+D).
+//         S = Q K^T, dP = dO V^T; P_x = exp(S - lse_x);
+//         dS = alpha P_lt (dP - Delta_lt) + beta P_st (dP - Delta_st), Delta_x = rowsum(dO o O_x)
+//         (one tile for both branches, they share K); dQ += dS K.  The first-stage MMAs of tile
+//         i+1 run while the compute warps work on tile i.
+//         Prologue: Delta and the per-row record (lse_lt*log2e - log2 alpha, lse_st*log2e -
+//         log2 beta, Delta_lt, Delta_st) that the dK/dV kernel streams.
+//         d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
+//  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
+//         records) that selected one of its key blocks or whose window reaches them.
+//         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D); each thread
+//         overwrites the first half of its own S^T / dP^T columns with W^T / dS^T.
+//         S^T = K Q^T, dP^T = V dO^T; thread = key row; W^T = alpha P_lt + beta P_st and
+//         dS^T as above; dV += W^T dO, dK += dS^T Q.
+// Every wait is bounded (tc_common.cuh).
+#include "tc_common.cuh"
+
+namespace blossom {
+namespace tc {
+namespace {
+
+constexpr int kBwdThreads = 288;
+constexpr int kComputeWarps = 8;
+constexpr int kDqStages = 4;
+constexpr int kKvStages = 3;
+constexpr uint32_t kBwdTmemCols = 256;
+constexpr int kStatBytes = 64 * 16;  // one 64-query tile of row records
+// The dK/dV kernel lets S^T(i+1) overwrite the columns W^T(i) was read from.  With this switch
+// off it waits for the products that read them to complete before it issues the overwriting
+// ones; with it on it relies on the tensor pipe executing one thread's MMAs in issue order.
+constexpr bool kTrustMmaIssueOrder = false;
+
+__device__ __forceinline__ bool bit(uint32_t w, int c) { return (w >> c) & 1u; }
+
+// ---------------------------------------------------------------------------- backward dQ
+// 16 columns of one tile for one row: dS packed to bf16 pairs, d alpha partial.
+template <bool HAS_L, bool HAS_S, bool FULL>
+__device__ __forceinline__ void dq_tile(const float (&sv)[16], const float (&dp)[16], uint32_t hL,
+                                        uint32_t hS, float sc2, float lseL2, float lseS2, float DL,
+                                        float DS, float alpha, float beta, float &dal,
+                                        uint32_t (&dw)[8]) {
+#pragma unroll
+  for (int c = 0; c < 16; c += 2) {
+    float d[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const float dpv = dp[c + e];
+      float acc = 0.f;
+      if (HAS_L) {
+        float p = exp2f(fmaf(sv[c + e], sc2, -lseL2));
+        if (!FULL) p = bit(hL, c + e) ? p : 0.f;
+        dal = fmaf(p, dpv, dal);
+        acc = (alpha * p) * (dpv - DL);
+      }
+      if (HAS_S) {
+        float p = exp2f(fmaf(sv[c + e], sc2, -lseS2));
+        if (!FULL) p = bit(hS, c + e) ? p : 0.f;
+        dal = fmaf(-p, dpv, dal);
+        acc = fmaf(beta * p, dpv - DS, acc);
+      }
+      d[e] = acc;
+    }
+    dw[c >> 1] = pack_bf16(d[0], d[1]);
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
+    const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+    const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
+    const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
+    const int32_t *__restrict__ idx, const __nv_bfloat16 *__restrict__ out_lt,
+    const __nv_bfloat16 *__restrict__ out_st, const float *__restrict__ lse,
+    const __nv_bfloat16 *__restrict__ dout, __nv_bfloat16 *__restrict__ dq,
+    float4 *__restrict__ qstats, double *__restrict__ dalpha_part, int32_t *__restrict__ status,
+    int nT) {
+  using C = Cfg<D>;
+  constexpr int STAGES = kDqStages;
+  constexpr int OC = D / 2;  // accumulator columns per thread
+  extern __shared__ uint8_t smem_raw[];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, t_full, mma_done
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ int nvis_s;
+  __shared__ float2 xch[2][128];
+  __shared__ double red[256];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nST = (s.L + 127) >> 7;
+  const int st = nST - 1 - (int)(blockIdx.x % nST);
+  const int u = blockIdx.x / nST, n = u / s.H, h = u % s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int row0 = st * 128;
+  const int G = 128 / s.Bk;
+  const int Lpad = nT * 64;
+
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t *tiles = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+  uint8_t *q_tile = tiles;
+  uint8_t *g_tile = q_tile + C::kBigBytes;
+  uint8_t *kv_tiles = g_tile + C::kBigBytes;
+  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;
+  uint32_t *selw = reinterpret_cast<uint32_t *>(meta);
+  uint8_t *selb = meta;
+  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
+  uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
+
+  const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
+  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
+  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 3]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 4]);
+
+  if (tid == 0) {
+    abort_flag = (*status != 0) ? 1 : 0;
+    tma_prefetch_desc(&tmq);
+    tma_prefetch_desc(&tmk);
+    tma_prefetch_desc(&tmv);
+    tma_prefetch_desc(&tmg);
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(b_full + 8 * i, 1);
+      mbar_init(b_empty + 8 * i, 1);
+    }
+    mbar_init(b_res, 1);
+    mbar_init(b_sfull, 1);
+    mbar_init(b_sempty, kComputeWarps);
+    mbar_init(b_tfull, kComputeWarps);
+    mbar_init(b_done, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(smem_u32(&tmem_slot), kBwdTmemCols);
+    tmem_relinquish();
+  }
+  build_query_major_list(s, idx, u, st, pad0, nT, selw, selb, list, lflags, &nvis_s);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const int nvis = nvis_s;
+  const uint32_t tmem_base = tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_ds = tmem_base + 128,
+                 tmem_dq = tmem_base + 160;
+
+  if (warp == kComputeWarps) {
+    if (lane == 0 && nvis > 0) {
+      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
+      constexpr uint32_t idesc_dq = instr_desc(128, D, 0, 1);
+      auto load_stage = [&](int j) {
+        const int sj = j % STAGES;
+        const uint32_t bar = b_full + 8 * sj;
+        uint8_t *kt = kv_tiles + sj * 2 * C::kSmallBytes;
+        mbar_expect_tx(bar, 2 * C::kSmallBytes);
+        tma_load_4d(smem_u32(kt), &tmk, bar, 0, (int)list[j] * 64, h, n);
+        tma_load_4d(smem_u32(kt + C::kSmallBytes), &tmv, bar, 0, (int)list[j] * 64, h, n);
+      };
+      int acc = 0;
+      auto second_stage = [&](int j) {  // dQ += dS K of tile j (dS from tensor memory, K MN-major)
+        uint8_t *k_tile = kv_tiles + (j % STAGES) * 2 * C::kSmallBytes;
+        const uint64_t dkm = smem_desc(smem_u32(k_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16_ts(tmem_dq, tmem_ds + 8 * k, dkm + k * C::kKStep, idesc_dq, (acc | k) != 0);
+        acc = 1;
+        umma_commit(b_done);
+        umma_commit(b_empty + 8 * (j % STAGES));
+      };
+      mbar_expect_tx(b_res, 2 * C::kBigBytes);
+      tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+      tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
+      for (int j = 0; j < min(STAGES - 1, nvis); ++j) load_stage(j);
+      const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
+      const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
+      for (int i = 0; i < nvis; ++i) {
+        if (i == 0) mbar_wait(b_res, 0, &abort_flag, 201);
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 202);
+        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 203);
+        tc_fence_after();
+        uint8_t *k_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes, *v_tile = k_tile + C::kSmallBytes;
+        const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dvd = smem_desc(smem_u32(v_tile), 16, C::kAtomBytes, C::kSwizzle);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dqd + 2 * k, dkd + 2 * k, idesc_s, k > 0);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dgd + 2 * k, dvd + 2 * k, idesc_s, k > 0);
+        umma_commit(b_sfull);
+        if (i >= 1) {
+          mbar_wait(b_tfull, (i - 1) & 1, &abort_flag, 204);
+          tc_fence_after();
+          second_stage(i - 1);
+          const int j = i + STAGES - 2;
+          if (j < nvis) {
+            if (i >= 2) mbar_wait(b_empty + 8 * ((i - 2) % STAGES), ((i - 2) / STAGES) & 1, &abort_flag, 205);
+            load_stage(j);
+          }
+        }
+      }
+      mbar_wait(b_tfull, (nvis - 1) & 1, &abort_flag, 206);
+      tc_fence_after();
+      second_stage(nvis - 1);
+    }
+  } else {
+    const int quarter = warp & 3, half = warp >> 2;
+    const int r = quarter * 32 + lane, t = row0 + r, g = r / s.Bk;
+    const bool row_ok = t < s.L, row_valid = row_ok && t >= pad0;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
+    const int64_t BHL = (int64_t)s.B * s.H * s.L;
+    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0);
+    // Delta of both branches: each thread sums its half of the row, the halves meet in shared memory
+    float DL = 0.f, DS = 0.f, lseL2 = 0.f, lseS2 = 0.f;
+    {
+      float aL = 0.f, aS = 0.f;
+      if (row_valid) {
+#pragma unroll
+        for (int c = 0; c < OC; c += 8) {
+          const int64_t off = ro + half * OC + c;
+          const uint4 gv = *reinterpret_cast<const uint4 *>(dout + off);
+          const uint4 lv = *reinterpret_cast<const uint4 *>(out_lt + off);
+          const uint4 sv4 = *reinterpret_cast<const uint4 *>(out_st + off);
+          const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, lw[4] = {lv.x, lv.y, lv.z, lv.w},
+                         sw[4] = {sv4.x, sv4.y, sv4.z, sv4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float g0 = __uint_as_float(gw[e] << 16), g1 = __uint_as_float(gw[e] & 0xffff0000u);
+            aL = fmaf(g0, __uint_as_float(lw[e] << 16), aL);
+            aL = fmaf(g1, __uint_as_float(lw[e] & 0xffff0000u), aL);
+            aS = fmaf(g0, __uint_as_float(sw[e] << 16), aS);
+            aS = fmaf(g1, __uint_as_float(sw[e] & 0xffff0000u), aS);
+          }
+        }
+        lseL2 = lse[(int64_t)u * s.L + t] * kLog2e;
+        lseS2 = lse[BHL + (int64_t)u * s.L + t] * kLog2e;
+      }
+      xch[half][r] = make_float2(aL, aS);
+      named_bar_sync(1 + quarter, 64);
+      const float2 o0 = xch[0][r], o1 = xch[1][r];  // fixed order: both threads get the same sums
+      DL = o0.x + o1.x;
+      DS = o0.y + o1.y;
+    }
+    if (half == 0 && t < Lpad)  // the row record the dK/dV kernel streams (zeros for rows that do not exist)
+      qstats[(int64_t)u * Lpad + t] = row_valid ? make_float4(lseL2 - log2f(alpha), lseS2 - log2f(beta), DL, DS)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+    float dal = 0.f;
+    bool ds_zero = false;
+    const float sc2 = s.scale * kLog2e;
+
+    for (int i = 0; i < nvis; ++i) {
+      const int jt = list[i], f = lflags[i], p0 = jt * 64;
+      uint64_t maskL = 0ull, maskS = 0ull;
+      if (row_valid) {
+        const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
+        if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
+        if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
+      }
+      const uint32_t hL = (uint32_t)(maskL >> (half * 32)), hS = (uint32_t)(maskS >> (half * 32));
+      const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);
+      const bool full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffffffu) && (!anyS || hS == 0xffffffffu));
+
+      mbar_wait(b_sfull, i & 1, &abort_flag, 207);
+      __syncwarp();
+      tc_fence_after();
+      const bool mine = anyL || anyS;
+      float sv[2][16], dp[2][16];
+      if (mine) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv[q]);
+          tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp[q]);
+        }
+        tmem_wait_ld();
+      }
+      tc_fence_before();
+      warp_arrive(b_sempty, lane);
+
+      if (mine || !ds_zero) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          uint32_t dw[8];
+          const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
+          if (anyL && anyS) {
+            if (full) dq_tile<true, true, true>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            else dq_tile<true, true, false>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+          } else if (anyL) {
+            if (full) dq_tile<true, false, true>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            else dq_tile<true, false, false>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+          } else if (anyS) {
+            if (full) dq_tile<false, true, true>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            else dq_tile<false, true, false>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) dw[c] = 0u;
+          }
+          if (q == 0 && i >= 1) {  // the dS columns are free once dQ += dS K of tile i-1 has completed
+            mbar_wait(b_done, (i - 1) & 1, &abort_flag, 208);
+            __syncwarp();
+            tc_fence_after();
+          }
+          tmem_st8u(tmem_ds + lane_off + half * 16 + q * 8, dw);
+        }
+        tmem_wait_st();
+        ds_zero = !mine;
+      } else if (i >= 1) {
+        // nothing to write, but keep in step with the barrier: a parity wait only tells the last
+        // two phases apart, so no warp may fall further behind than that
+        mbar_wait(b_done, (i - 1) & 1, &abort_flag, 219);
+        __syncwarp();
+      }
+      tc_fence_before();
+      warp_arrive(b_tfull, lane);
+    }
+
+    if (nvis > 0) {
+      mbar_wait(b_done, (nvis - 1) & 1, &abort_flag, 209);
+      __syncwarp();
+      tc_fence_after();
+    }
+    float o[OC];
+    if (nvis > 0) {
+      tmem_ld<OC>(tmem_dq + lane_off + half * OC, o);
+      tmem_wait_ld();
+    }
+    if (row_ok) {
+      const bool live = nvis > 0 && row_valid;
+#pragma unroll
+      for (int ch = 0; ch < OC / 8; ++ch) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = ch * 8 + e * 2;
+          w[e] = live ? pack_bf16(o[c] * s.scale, o[c + 1] * s.scale) : 0u;
+        }
+        *reinterpret_cast<uint4 *>(dq + ro + half * OC + ch * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+    red[tid] = row_valid ? (double)dal : 0.0;
+  }
+  tc_fence_before();
+  __syncthreads();
+  // d alpha partial of this CTA -> first query-block slot of the super-tile, zeros in the rest
+  if (tid == 0) {
+    double a = 0.0;
+    for (int i = 0; i < 256; ++i) a += red[i];  // fixed order
+    for (int gq = 0; gq < G; ++gq)
+      if (st * G + gq < s.M) dalpha_part[(int64_t)u * s.M + st * G + gq] = gq == 0 ? a : 0.0;
+  }
+  finish(warp, tmem_base, kBwdTmemCols, &abort_flag, status);
+}
+
+// ------------------------------------------------------------------------- backward dK, dV
+// 16 query columns of one tile for one key row: W^T and dS^T packed to bf16 pairs.  st points at
+// the row records (lse_lt', lse_st', Delta_lt, Delta_st) of these 16 queries.
+template <bool HAS_L, bool HAS_S, bool FULL>
+__device__ __forceinline__ void dkdv_tile(const float (&sv)[16], const float (&dp)[16], uint32_t hL,
+                                          uint32_t hS, float sc2, const float4 *st, uint32_t (&ww)[8],
+                                          uint32_t (&dw)[8]) {
+#pragma unroll
+  for (int c = 0; c < 16; c += 2) {
+    float wv[2], d[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const float4 q4 = st[c + e];
+      const float dpv = dp[c + e];
+      float wa = 0.f, da = 0.f;
+      if (HAS_L) {
+        float p = exp2f(fmaf(sv[c + e], sc2, -q4.x));
+        if (!FULL) p = bit(hL, c + e) ? p : 0.f;
+        wa = p;
+        da = p * (dpv - q4.z);
+      }
+      if (HAS_S) {
+        float p = exp2f(fmaf(sv[c + e], sc2, -q4.y));
+        if (!FULL) p = bit(hS, c + e) ? p : 0.f;
+        wa += p;
+        da = fmaf(p, dpv - q4.w, da);
+      }
+      wv[e] = wa;
+      d[e] = da;
+    }
+    ww[c >> 1] = pack_bf16(wv[0], wv[1]);
+    dw[c >> 1] = pack_bf16(d[0], d[1]);
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
+    const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+    const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
+    const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ idx,
+    const float4 *__restrict__ qstats, __nv_bfloat16 *__restrict__ dk, __nv_bfloat16 *__restrict__ dv,
+    int32_t *__restrict__ status, int nT) {
+  using C = Cfg<D>;
+  constexpr int STAGES = kKvStages;
+  constexpr int OC = D / 2;
+  constexpr int kStageBytes = 2 * C::kSmallBytes + kStatBytes;  // Q, dO, row records
+  extern __shared__ uint8_t smem_raw[];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ int nvis_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nKT = (s.L + 127) >> 7;
+  const int kt = (int)(blockIdx.x % nKT);  // early keys have the most visitors: first
+  const int u = blockIdx.x / nKT, n = u / s.H, h = u % s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int key0 = kt * 128, key_last = min(s.L - 1, key0 + 127);
+  const int G = 128 / s.Bk, nb = 64 / s.Bk;
+  const int Lpad = nT * 64;
+
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t *tiles = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+  uint8_t *k_tile = tiles;
+  uint8_t *v_tile = k_tile + C::kBigBytes;
+  uint8_t *qg_tiles = v_tile + C::kBigBytes;  // [stage][Q, dO, row records]
+  uint8_t *meta = qg_tiles + STAGES * kStageBytes;
+  uint32_t *invw = reinterpret_cast<uint32_t *>(meta);  // [8][nT] bytes: per key block, per query tile
+  uint8_t *invb = meta;
+  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
+  uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
+
+  const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
+  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
+  const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 2]), b_done = smem_u32(&bars[2 * STAGES + 3]);
+
+  if (tid == 0) {
+    abort_flag = (*status != 0) ? 1 : 0;
+    tma_prefetch_desc(&tmq);
+    tma_prefetch_desc(&tmk);
+    tma_prefetch_desc(&tmv);
+    tma_prefetch_desc(&tmg);
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(b_full + 8 * i, 1);
+      mbar_init(b_empty + 8 * i, 1);
+    }
+    mbar_init(b_res, 1);
+    mbar_init(b_sfull, 1);
+    mbar_init(b_tfull, kComputeWarps);
+    mbar_init(b_done, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(smem_u32(&tmem_slot), kBwdTmemCols);
+    tmem_relinquish();
+  }
+  for (int i = tid; i < (8 * nT + 3) / 4; i += kBwdThreads) invw[i] = 0u;
+  __syncthreads();
+  {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
+    const int qb0 = kt * G, nq = s.M - qb0;
+    for (int i = tid; i < nq * s.topk; i += kBwdThreads) {
+      const int qb = qb0 + i / s.topk;
+      const int blk = idx[((int64_t)u * s.M + qb) * s.topk + (i % s.topk)];
+      if (blk >= qb0 && blk < qb0 + G && blk <= qb) {
+        const int a = (blk - qb0) * nT + qb / nb;
+        atomicOr(&invw[a >> 2], (1u << (qb % nb)) << ((a & 3) * 8));
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int qt_min = key0 >> 6, qt_max = (s.L - 1) >> 6;
+    int count = 0;
+    for (int base = qt_min; base <= qt_max; base += 32) {
+      const int qt = base + lane;
+      int f = 0;
+      if (qt <= qt_max && key_last >= pad0) {
+        for (int g = 0; g < G; ++g) f |= invb[g * nT + qt] ? 1 : 0;
+        if (qt * 64 <= key_last + s.window - 1) f |= 2;
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
+      if (f) {
+        const int pos = count + __popc(bal & ((1u << lane) - 1u));
+        list[pos] = (uint16_t)qt;
+        lflags[pos] = (uint8_t)f;
+      }
+      count += __popc(bal);
+    }
+    if (lane == 0) nvis_s = count;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const int nvis = nvis_s;
+  const uint32_t tmem_base = tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_dv = tmem_base + 128,
+                 tmem_dk = tmem_base + 192;
+
+  if (warp == kComputeWarps) {
+    if (lane == 0 && nvis > 0) {
+      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
+      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
+      auto load_stage = [&](int j) {
+        const int sj = j % STAGES;
+        const uint32_t bar = b_full + 8 * sj;
+        uint8_t *qt_ = qg_tiles + sj * kStageBytes;
+        mbar_expect_tx(bar, kStageBytes);
+        tma_load_4d(smem_u32(qt_), &tmq, bar, 0, (int)list[j] * 64, h, n);
+        tma_load_4d(smem_u32(qt_ + C::kSmallBytes), &tmg, bar, 0, (int)list[j] * 64, h, n);
+        bulk_load(smem_u32(qt_ + 2 * C::kSmallBytes), qstats + (int64_t)u * Lpad + (int64_t)list[j] * 64,
+                  kStatBytes, bar);
+      };
+      int acc = 0;
+      // dV += W^T dO, dK += dS^T Q of tile j; the 16 queries of K step k sit in columns
+      // 32 * (k / 2) + 8 * (k % 2) of the S^T / dP^T regions
+      auto second_stage = [&](int j) {
+        uint8_t *q_tile = qg_tiles + (j % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
+        const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16_ts(tmem_dv, tmem_s + 32 * (k >> 1) + 8 * (k & 1), dgm + k * C::kKStep, idesc_o, (acc | k) != 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16_ts(tmem_dk, tmem_dp + 32 * (k >> 1) + 8 * (k & 1), dqm + k * C::kKStep, idesc_o, (acc | k) != 0);
+        acc = 1;
+        umma_commit(b_empty + 8 * (j % STAGES));
+        umma_commit(b_done);
+      };
+      mbar_expect_tx(b_res, 2 * C::kBigBytes);
+      tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
+      tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
+      for (int j = 0; j < min(STAGES, nvis); ++j) load_stage(j);
+      const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
+      const uint64_t dvd = smem_desc(smem_u32(v_tile), 16, C::kAtomBytes, C::kSwizzle);
+      for (int i = 0; i < nvis; ++i) {
+        if (i == 0) mbar_wait(b_res, 0, &abort_flag, 210);
+        if (i >= 1) {
+          mbar_wait(b_tfull, (i - 1) & 1, &abort_flag, 211);
+          tc_fence_after();
+          second_stage(i - 1);
+          if (!kTrustMmaIssueOrder) mbar_wait(b_done, (i - 1) & 1, &abort_flag, 212);
+        }
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 213);
+        tc_fence_after();
+        uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
+        const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
+        umma_commit(b_sfull);
+        // tile i + STAGES - 1 goes into the stage tile i - 1 occupied
+        const int j = i + STAGES - 1;
+        if (i >= 1 && j < nvis) {
+          mbar_wait(b_empty + 8 * ((i - 1) % STAGES), ((i - 1) / STAGES) & 1, &abort_flag, 214);
+          load_stage(j);
+        }
+      }
+      mbar_wait(b_tfull, (nvis - 1) & 1, &abort_flag, 215);
+      tc_fence_after();
+      second_stage(nvis - 1);
+    }
+  } else {
+    const int quarter = warp & 3, half = warp >> 2;
+    const int r = quarter * 32 + lane, p = key0 + r, g = r / s.Bk;
+    const bool row_ok = p < s.L, row_valid = row_ok && p >= pad0;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const float sc2 = s.scale * kLog2e;
+
+    for (int i = 0; i < nvis; ++i) {
+      const int qt = list[i], f = lflags[i], t0 = qt * 64;
+      uint64_t maskL = 0ull, maskS = 0ull;
+      if (row_valid) {
+        const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
+        if (f & 1) maskL = mc & expand_block_bits(invb[g * nT + qt], s.Bk);
+        if (f & 2) maskS = mc & cols_le(p + s.window - 1 - t0);
+      }
+      const uint32_t hL = (uint32_t)(maskL >> (half * 32)), hS = (uint32_t)(maskS >> (half * 32));
+      const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);
+      const bool full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffffffu) && (!anyS || hS == 0xffffffffu));
+
+      mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 216);  // the row records have landed
+      mbar_wait(b_sfull, i & 1, &abort_flag, 217);
+      __syncwarp();
+      tc_fence_after();
+      // 16 query columns at a time; W^T / dS^T always written: the fresh S^T / dP^T erased
+      // whatever this thread had left in those columns
+      const float4 *stt =
+          reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes) + half * 32;
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        uint32_t ww[8], dw[8];
+        if (anyL || anyS) {
+          float sv[16], dp[16];
+          tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
+          tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
+          tmem_wait_ld();
+          const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
+          const float4 *sq = stt + q * 16;
+          if (anyL && anyS) {
+            if (full) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+            else dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          } else if (anyL) {
+            if (full) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+            else dkdv_tile<true, false, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          } else {
+            if (full) dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+            else dkdv_tile<false, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }
+        }
+        tmem_st8u(tmem_s + lane_off + half * 32 + q * 8, ww);
+        tmem_st8u(tmem_dp + lane_off + half * 32 + q * 8, dw);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      warp_arrive(b_tfull, lane);
+    }
+
+    if (nvis > 0) {
+      mbar_wait(b_done, (nvis - 1) & 1, &abort_flag, 218);
+      __syncwarp();
+      tc_fence_after();
+    }
+    float ov[OC], okk[OC];
+    if (nvis > 0) {
+      tmem_ld<OC>(tmem_dv + lane_off + half * OC, ov);
+      tmem_ld<OC>(tmem_dk + lane_off + half * OC, okk);
+      tmem_wait_ld();
+    }
+    if (row_ok) {
+      const bool live = nvis > 0 && row_valid;
+      const int64_t ro = row_offset(s, n, h, p) + half * OC;
+#pragma unroll
+      for (int ch = 0; ch < OC / 8; ++ch) {
+        uint32_t wv[4], wk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = ch * 8 + e * 2;
+          wv[e] = live ? pack_bf16(ov[c], ov[c + 1]) : 0u;
+          wk[e] = live ? pack_bf16(okk[c] * s.scale, okk[c + 1] * s.scale) : 0u;
+        }
+        *reinterpret_cast<uint4 *>(dv + ro + ch * 8) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+        *reinterpret_cast<uint4 *>(dk + ro + ch * 8) = make_uint4(wk[0], wk[1], wk[2], wk[3]);
+      }
+    }
+  }
+  finish(warp, tmem_base, kBwdTmemCols, &abort_flag, status);
+}
+
+}  // namespace
+
+template <int D>
+int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                    const int32_t *seq_lens, const int32_t *idx, const void *out_lt,
+                    const void *out_st, const float *lse, const void *dout, void *dq, void *dk,
+                    void *dv, const Workspace &ws, cudaStream_t st) {
+  typedef __nv_bfloat16 bf;
+  using C = Cfg<D>;
+  CUtensorMap q128, k64, v64, g128, q64, k128, v128, g64;
+  if (make_tensor_map(&q128, q, s, 128) || make_tensor_map(&k64, k, s, 64) ||
+      make_tensor_map(&v64, v, s, 64) || make_tensor_map(&g128, dout, s, 128) ||
+      make_tensor_map(&q64, q, s, 64) || make_tensor_map(&k128, k, s, 128) ||
+      make_tensor_map(&v128, v, s, 128) || make_tensor_map(&g64, dout, s, 64))
+    return BLOSSOM_ERR_CUDA;
+  const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
+  const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
+  const size_t smem_dq = 1024 + 2 * C::kBigBytes + kDqStages * 2 * C::kSmallBytes + meta_bytes(nT);
+  const size_t smem_kv =
+      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT);
+  if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
+      cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  {
+    LaunchScope ls(K_BWD_DQ_TC, st);
+    bwd_dq_tc_kernel<D><<<grid, kBwdThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, idx,
+                                                           (const bf *)out_lt, (const bf *)out_st, lse,
+                                                           (const bf *)dout, (bf *)dq, ws.qstats, ws.dalpha,
+                                                           ws.status, nT);
+  }
+  {
+    LaunchScope ls(K_BWD_DKDV_TC, st);
+    bwd_dkdv_tc_kernel<D><<<grid, kBwdThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, idx,
+                                                             ws.qstats, (bf *)dk, (bf *)dv, ws.status, nT);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
+template int launch_bwd_tc_t<32>(const Shape &, const void *, const void *, const void *, const float *,
+                                 const int32_t *, const int32_t *, const void *, const void *,
+                                 const float *, const void *, void *, void *, void *, const Workspace &,
+                                 cudaStream_t);
+template int launch_bwd_tc_t<64>(const Shape &, const void *, const void *, const void *, const float *,
+                                 const int32_t *, const int32_t *, const void *, const void *,
+                                 const float *, const void *, void *, void *, void *, const Workspace &,
+                                 cudaStream_t);
+
+}  // namespace tc
+}  // namespace blossom

@@ -1,0 +1,397 @@
+// Tensor-core forward of the fused two-branch attention (bf16 storage, fp32 accumulate).
+//
+// CTA = 160 threads: warps 0..3 are the softmax warps (thread = query row = TMEM lane), warp 4 is
+// the producer (one lane issues every TMA load and every tcgen05.mma).  A CTA owns 128 query rows
+// (128 / Bk query blocks) and streams the 64-key tiles that any of its query blocks selected
+// (Eq. 14, 16) or that its rows reach through the window (Eq. 15, 17).  Tensor memory (256
+// columns): S = Q K^T [0,64), P_lt [64,96), P_st [96,128) (bf16 pairs), O_lt [128,128+D),
+// O_st [192,192+D).  Per streamed tile i:
+//
+//   producer : wait TMA(i) and "S(i-1) is in registers" -> S(i) = Q K_i^T -> commit s_full
+//              wait "P(i-1) written" -> O_lt += P_lt V, O_st += P_st V with the probabilities read
+//              straight from tensor memory -> commit mma_done, release the K/V stage, refill it
+//   softmax  : wait s_full(i) -> tcgen05.ld the row's 64 logits -> arrive s_empty -> masks, the two
+//              online softmaxes (maximum raised, and the accumulator rescaled, only when a tile's
+//              maximum exceeds it by > 2^8) -> wait mma_done(i-1) -> tcgen05.st P -> arrive t_full
+//
+// so S(i+1) is computed while the softmax warps work on tile i, probabilities never touch shared
+// memory, and nothing in the loop is a block-wide barrier.  Rows whose query block does not need a
+// tile skip its exponentials (warp-uniform) and contribute zero rows to P.
+// Epilogue: normalise, gate mix (Eq. 19), store out / out_lt / out_st / lse.
+// Every wait is bounded (tc_common.cuh).
+#include "tc_common.cuh"
+
+namespace blossom {
+namespace tc {
+namespace {
+
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr int kFwdThreads = 160;
+constexpr int kSoftmaxWarps = 4;
+constexpr int kFwdStages = 4;
+constexpr uint32_t kFwdTmemCols = 256;
+
+// One branch of one tile for one query row: masked maximum, lazy rescale decision, probabilities
+// relative to the running maximum packed as bf16 pairs, running sum.  FULL = no column is masked
+// for any lane of the warp.
+template <bool FULL>
+__device__ __forceinline__ void tile_softmax(const float (&sv)[64], uint64_t mask, float sc2, float &m,
+                                             float &l, float &fac, bool &need, uint32_t (&pk)[32]) {
+  const uint32_t mlo = (uint32_t)mask, mhi = (uint32_t)(mask >> 32);
+  float a0 = -INFINITY, a1 = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < 64; c += 4) {
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int cc = c + e;
+      const bool on = FULL || (((cc < 32 ? mlo : mhi) >> (cc & 31)) & 1u);
+      v[e] = on ? sv[cc] : -INFINITY;
+    }
+    a0 = max3(a0, v[0], v[1]);
+    a1 = max3(a1, v[2], v[3]);
+  }
+  const float mt = fmaxf(a0, a1) * sc2;
+  need = mt > m + kRescaleThreshold;  // also true on the row's first keys
+  fac = 1.f;
+  if (need) {
+    fac = exp2f(m - mt);
+    l *= fac;
+    m = mt;
+  }
+  const float nm = -m;
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < 64; c += 2) {
+    float a = exp2f(fmaf(sv[c], sc2, nm)), b = exp2f(fmaf(sv[c + 1], sc2, nm));
+    if (!FULL) {
+      const uint32_t w = c < 32 ? mlo : mhi;
+      a = ((w >> (c & 31)) & 1u) ? a : 0.f;
+      b = ((w >> ((c + 1) & 31)) & 1u) ? b : 0.f;
+    }
+    s0 += a;
+    s1 += b;
+    pk[c >> 1] = pack_bf16(a, b);
+  }
+  l += s0 + s1;
+}
+
+// multiply the row's accumulator by fac (all lanes of the warp take part)
+template <int D>
+__device__ __forceinline__ void rescale_acc(uint32_t taddr, float fac) {
+#pragma unroll
+  for (int c0 = 0; c0 < D; c0 += 32) {
+    float o[32];
+    tmem_ld32(taddr + c0, o);
+    tmem_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; ++c) o[c] *= fac;
+    tmem_st32(taddr + c0, o);
+  }
+  tmem_wait_st();
+}
+
+template <int D>
+__global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
+    const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+    const __grid_constant__ CUtensorMap tmv, Shape s, const float *__restrict__ gate,
+    const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ idx,
+    __nv_bfloat16 *__restrict__ out, __nv_bfloat16 *__restrict__ out_lt,
+    __nv_bfloat16 *__restrict__ out_st, float *__restrict__ lse, int32_t *__restrict__ status,
+    int nT) {
+  using C = Cfg<D>;
+  constexpr int STAGES = kFwdStages;
+  extern __shared__ uint8_t smem_raw[];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, t_full, mma_done
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ int nvis_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nST = (s.L + 127) >> 7;
+  const int st = nST - 1 - (int)(blockIdx.x % nST);  // long rows first
+  const int u = blockIdx.x / nST, n = u / s.H, h = u % s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int row0 = st * 128;
+
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t *tiles = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+  uint8_t *q_tile = tiles;
+  uint8_t *kv_tiles = q_tile + C::kBigBytes;  // [stage][K, V]
+  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;
+  uint32_t *selw = reinterpret_cast<uint32_t *>(meta);
+  uint8_t *selb = meta;
+  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
+  uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
+
+  const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
+  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
+  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 3]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 4]);
+
+  if (tid == 0) {
+    abort_flag = (*status != 0) ? 1 : 0;  // an earlier CTA timed out: do not wait again
+    tma_prefetch_desc(&tmq);
+    tma_prefetch_desc(&tmk);
+    tma_prefetch_desc(&tmv);
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(b_full + 8 * i, 1);
+      mbar_init(b_empty + 8 * i, 1);
+    }
+    mbar_init(b_res, 1);
+    mbar_init(b_sfull, 1);
+    mbar_init(b_sempty, kSoftmaxWarps);
+    mbar_init(b_tfull, kSoftmaxWarps);
+    mbar_init(b_done, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(smem_u32(&tmem_slot), kFwdTmemCols);
+    tmem_relinquish();
+  }
+  build_query_major_list(s, idx, u, st, pad0, nT, selw, selb, list, lflags, &nvis_s);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const int nvis = nvis_s;
+  const uint32_t tmem_base = tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_pl = tmem_base + 64, tmem_ps = tmem_base + 96,
+                 tmem_ol = tmem_base + 128, tmem_os = tmem_base + 192;
+
+  if (warp == kSoftmaxWarps) {
+    // ================================ producer ================================
+    if (lane == 0 && nvis > 0) {
+      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
+      constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
+      auto load_stage = [&](int j) {
+        const int sj = j % STAGES;
+        const uint32_t bar = b_full + 8 * sj;
+        uint8_t *kt = kv_tiles + sj * 2 * C::kSmallBytes;
+        mbar_expect_tx(bar, 2 * C::kSmallBytes);
+        tma_load_4d(smem_u32(kt), &tmk, bar, 0, (int)list[j] * 64, h, n);
+        tma_load_4d(smem_u32(kt + C::kSmallBytes), &tmv, bar, 0, (int)list[j] * 64, h, n);
+      };
+      int accL = 0, accS = 0;
+      auto second_stage = [&](int j) {  // O += P V of tile j, P read from tensor memory
+        const int f = lflags[j];
+        uint8_t *v_tile = kv_tiles + (j % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes;
+        const uint64_t dv = smem_desc(smem_u32(v_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        if (f & 1) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16_ts(tmem_ol, tmem_pl + 8 * k, dv + k * C::kKStep, idesc_pv, (accL | k) != 0);
+          accL = 1;
+        }
+        if (f & 2) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16_ts(tmem_os, tmem_ps + 8 * k, dv + k * C::kKStep, idesc_pv, (accS | k) != 0);
+          accS = 1;
+        }
+        umma_commit(b_done);
+        umma_commit(b_empty + 8 * (j % STAGES));
+      };
+      mbar_expect_tx(b_res, C::kBigBytes);
+      tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+      for (int j = 0; j < min(STAGES - 1, nvis); ++j) load_stage(j);
+      const uint64_t dq = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
+      for (int i = 0; i < nvis; ++i) {
+        if (i == 0) mbar_wait(b_res, 0, &abort_flag, 101);
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 102);
+        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 103);
+        tc_fence_after();
+        uint8_t *k_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes;
+        const uint64_t dk = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dq + 2 * k, dk + 2 * k, idesc_s, k > 0);
+        umma_commit(b_sfull);
+        if (i >= 1) {
+          mbar_wait(b_tfull, (i - 1) & 1, &abort_flag, 104);
+          tc_fence_after();
+          second_stage(i - 1);
+          // tile i + STAGES - 2 goes into the stage tile i - 2 occupied
+          const int j = i + STAGES - 2;
+          if (j < nvis) {
+            if (i >= 2) mbar_wait(b_empty + 8 * ((i - 2) % STAGES), ((i - 2) / STAGES) & 1, &abort_flag, 105);
+            load_stage(j);
+          }
+        }
+      }
+      mbar_wait(b_tfull, (nvis - 1) & 1, &abort_flag, 106);
+      tc_fence_after();
+      second_stage(nvis - 1);
+    }
+  } else {
+    // ================================ softmax =================================
+    const int r = warp * 32 + lane, t = row0 + r, g = r / s.Bk;
+    const bool row_ok = t < s.L;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    float mL = -INFINITY, lL = 0.f, mS = -INFINITY, lS = 0.f;
+    bool zeroL = false, zeroS = false;
+    int accL = 0, accS = 0;
+    const float sc2 = s.scale * kLog2e;
+
+    for (int i = 0; i < nvis; ++i) {
+      const int jt = list[i], f = lflags[i], p0 = jt * 64;
+      uint64_t maskL = 0ull, maskS = 0ull;
+      if (row_ok) {
+        const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
+        if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
+        if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
+      }
+      const bool doL = __any_sync(0xffffffffu, maskL != 0ull);
+      const bool doS = __any_sync(0xffffffffu, maskS != 0ull);
+      const bool fullL = __all_sync(0xffffffffu, maskL == ~0ull);
+      const bool fullS = __all_sync(0xffffffffu, maskS == ~0ull);
+
+      mbar_wait(b_sfull, i & 1, &abort_flag, 107);
+      __syncwarp();
+      tc_fence_after();
+      float sv[64];
+      if (doL || doS) {
+        tmem_ld32(tmem_s + lane_off, sv);
+        tmem_ld32(tmem_s + lane_off + 32, sv + 32);
+        tmem_wait_ld();
+      }
+      tc_fence_before();
+      warp_arrive(b_sempty, lane);
+
+      uint32_t pk[32];
+      float fac = 1.f;
+      bool need = false;
+      // ---- long-term branch ----
+      if (f & 1) {
+        if (doL) {
+          if (fullL) tile_softmax<true>(sv, maskL, sc2, mL, lL, fac, need, pk);
+          else tile_softmax<false>(sv, maskL, sc2, mL, lL, fac, need, pk);
+        }
+        if (i >= 1) {  // P regions and accumulators are free once the MMAs of tile i-1 completed
+          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 108);
+          __syncwarp();
+          tc_fence_after();
+        }
+        if (doL) {
+          if (accL && __any_sync(0xffffffffu, need)) rescale_acc<D>(tmem_ol + lane_off, fac);
+          tmem_st32u(tmem_pl + lane_off, pk);
+          zeroL = false;
+        } else if (!zeroL) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) pk[c] = 0u;
+          tmem_st32u(tmem_pl + lane_off, pk);
+          zeroL = true;
+        }
+      }
+      // ---- short-term branch ----
+      if (f & 2) {
+        fac = 1.f;
+        need = false;
+        if (doS) {
+          if (fullS) tile_softmax<true>(sv, maskS, sc2, mS, lS, fac, need, pk);
+          else tile_softmax<false>(sv, maskS, sc2, mS, lS, fac, need, pk);
+        }
+        if (!(f & 1) && i >= 1) {
+          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 109);
+          __syncwarp();
+          tc_fence_after();
+        }
+        if (doS) {
+          if (accS && __any_sync(0xffffffffu, need)) rescale_acc<D>(tmem_os + lane_off, fac);
+          tmem_st32u(tmem_ps + lane_off, pk);
+          zeroS = false;
+        } else if (!zeroS) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) pk[c] = 0u;
+          tmem_st32u(tmem_ps + lane_off, pk);
+          zeroS = true;
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      warp_arrive(b_tfull, lane);
+      accL |= (f & 1);
+      accS |= (f & 2);
+    }
+
+    // ---- epilogue ----
+    if (nvis > 0) {
+      mbar_wait(b_done, (nvis - 1) & 1, &abort_flag, 110);
+      __syncwarp();
+      tc_fence_after();
+    }
+    const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
+    const float iL = lL > 0.f ? 1.f / lL : 0.f, iS = lS > 0.f ? 1.f / lS : 0.f;
+    const bool haveL = accL && lL > 0.f, haveS = accS && lS > 0.f;
+    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0);
+#pragma unroll
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      float oL[32], oS[32];
+      if (accL) tmem_ld32(tmem_ol + lane_off + c0, oL);  // accL / accS are CTA-uniform
+      if (accS) tmem_ld32(tmem_os + lane_off + c0, oS);
+      tmem_wait_ld();
+      if (row_ok) {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t wo[4], wl[4], ws[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = ch * 8 + e * 2;
+            const float a0 = haveL ? oL[c] * iL : 0.f, a1 = haveL ? oL[c + 1] * iL : 0.f;
+            const float b0 = haveS ? oS[c] * iS : 0.f, b1 = haveS ? oS[c + 1] * iS : 0.f;
+            wl[e] = pack_bf16(a0, a1);
+            ws[e] = pack_bf16(b0, b1);
+            wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
+          }
+          const int64_t off = ro + c0 + ch * 8;
+          *reinterpret_cast<uint4 *>(out + off) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+          if (out_lt) *reinterpret_cast<uint4 *>(out_lt + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+          if (out_st) *reinterpret_cast<uint4 *>(out_st + off) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+        }
+      }
+    }
+    if (row_ok && lse) {
+      const int64_t BHL = (int64_t)s.B * s.H * s.L;
+      lse[(int64_t)u * s.L + t] = lL > 0.f ? (mL + log2f(lL)) * kLn2 : 0.f;
+      lse[BHL + (int64_t)u * s.L + t] = lS > 0.f ? (mS + log2f(lS)) * kLn2 : 0.f;
+    }
+  }
+  finish(warp, tmem_base, kFwdTmemCols, &abort_flag, status);
+}
+
+}  // namespace
+
+template <int D>
+int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                    const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt,
+                    void *out_st, float *lse, const Workspace &ws, cudaStream_t st) {
+  using C = Cfg<D>;
+  CUtensorMap tq, tk, tv;
+  if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64) || make_tensor_map(&tv, v, s, 64))
+    return BLOSSOM_ERR_CUDA;
+  const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
+  const size_t smem = 1024 + C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT);
+  if (cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
+  {
+    LaunchScope ls(K_FWD_TC, st);
+    fwd_tc_kernel<D><<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, s, gate, seq_lens, idx,
+                                                     (__nv_bfloat16 *)out, (__nv_bfloat16 *)out_lt,
+                                                     (__nv_bfloat16 *)out_st, lse, ws.status, nT);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
+template int launch_fwd_tc_t<32>(const Shape &, const void *, const void *, const void *, const float *,
+                                 const int32_t *, const int32_t *, void *, void *, void *, float *,
+                                 const Workspace &, cudaStream_t);
+template int launch_fwd_tc_t<64>(const Shape &, const void *, const void *, const void *, const float *,
+                                 const int32_t *, const int32_t *, void *, void *, void *, float *,
+                                 const Workspace &, cudaStream_t);
+
+}  // namespace tc
+}  // namespace blossom

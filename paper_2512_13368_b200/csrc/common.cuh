@@ -23,7 +23,8 @@ struct Workspace {
   int32_t *klive;    // [B][H][M]     number of valid keys in the block
   float *delta;      // [2][B][H][L]  rowsum(G_branch o O_branch) for the backward
   double *dalpha;    // [B][H][M]     per query block partial of d alpha
-  float *dq_acc;     // [B][H][L][D]  fp32 dQ accumulator of the tensor-core backward
+  float4 *qstats;    // [B][H][ceil(L/64)*64]  per query row: (lse_lt*log2e - log2 alpha,
+                     //   lse_st*log2e - log2 beta, Delta_lt, Delta_st) for the dK/dV kernel
   size_t bytes;
 };
 

@@ -48,14 +48,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// `site` (non-zero) names the wait in the kernel's source; the first wait of a CTA that runs out
+// leaves it in the abort flag, from where it reaches word 1 of the workspace status.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int site = 1) {
   if (mbar_try_wait(bar, parity)) return;
   if (*abort_flag) return;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
     if (*abort_flag) return;
     if (clock64() - t0 > kTimeoutCycles) {
-      *abort_flag = 1;
+      *abort_flag = site;
       return;
     }
   }
@@ -72,6 +75,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+// 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion on an
+// mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+      : "memory");
 }
 // generic-proxy shared-memory writes -> visible to the async proxy (TMA / tcgen05 operands)
 __device__ __forceinline__ void fence_async_smem() {
@@ -105,6 +116,18 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]: A is a bf16 matrix held in tensor memory, row m in lane m, two
+// consecutive K elements per 32-bit column (the lower K index in the low half), 8 columns per
+// K = 16 step.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // arrive on the mbarrier once every MMA this thread issued so far has completed
@@ -181,6 +204,36 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *v) {
       "r"(__float_as_uint(v[15]))
       : "memory");
 }
+// packed words (two bf16 per 32-bit column) -> tensor memory
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t *v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+      "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+      "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+      "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16u(uint32_t taddr, const uint32_t *v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+      "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8u(uint32_t taddr, const uint32_t *v) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
+               "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 template <int N>
 __device__ __forceinline__ void tmem_ld(uint32_t taddr, float *v) {
   static_assert(N == 16 || N == 32, "16 or 32 columns");
@@ -243,8 +296,107 @@ __device__ __forceinline__ void store_row_sw128(uint8_t *tile, int r, int ch, ui
   *reinterpret_cast<uint4 *>(tile + r * 128 + ((ch ^ (r & 7)) << 4)) = v;
 }
 
+// ---- pieces shared by the forward and backward kernels ------------------------------------
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+template <int D>
+struct Cfg {
+  static constexpr int kRowBytes = D * 2;
+  static constexpr int kBigBytes = 128 * kRowBytes;   // resident 128-row tile
+  static constexpr int kSmallBytes = 64 * kRowBytes;  // streamed 64-row tile
+  static constexpr int kAtomBytes = 8 * kRowBytes;    // 8-row swizzle atom of a D-wide tile
+  static constexpr uint32_t kSwizzle = (D == 64) ? 2u : 4u;  // 128-byte / 64-byte swizzle
+  static constexpr int kKStep = (16 * kRowBytes) >> 4;       // descriptor advance of 16 rows
+};
+
+// bytes of the per-CTA tile bookkeeping: [8][nT] selection bytes, nT list entries, nT flags
+__host__ __device__ inline int meta_bytes(int nT) { return ((11 * nT + 15) / 16) * 16 + 16; }
+
+// one arrival per warp, after all its lanes are done
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+}
+
+// common kernel end: everyone is done with tensor memory -> free it; report a timed-out wait
+__device__ __forceinline__ void finish(int warp, uint32_t tmem_base, uint32_t ncols, int *abort_flag,
+                                       int32_t *status) {
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, ncols);
+  if (threadIdx.x == 0 && *abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {}  // grace period for copies still in flight
+    if (atomicCAS(status, 0, (int32_t)BLOSSOM_ERR_TIMEOUT) == 0) {  // first reporter: where it happened
+      status[1] = *abort_flag;
+      status[2] = (int32_t)blockIdx.x;
+    }
+  }
+}
+
+__device__ __forceinline__ float gate_alpha(const float *gate, int h) {
+  return 1.f / (1.f + __expf(-(gate[h * 2 + 0] - gate[h * 2 + 1])));
+}
+
+// Query-major tile list (forward and dQ): per 64-key tile, which key blocks each of the CTA's
+// query blocks selected (selb[g * nT + tile]), and the ascending list of tiles to visit with
+// flags (bit 0: some selected block lies in the tile, bit 1: the window of some row reaches it).
+// Called by every thread of the CTA; contains block-wide barriers.
+__device__ __forceinline__ void build_query_major_list(const Shape &s, const int32_t *idx, int u, int st,
+                                                       int pad0, int nT, uint32_t *selw, uint8_t *selb,
+                                                       uint16_t *list, uint8_t *lflags, int *nvis_out) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nthr = blockDim.x;
+  const int G = 128 / s.Bk, nb = 64 / s.Bk;
+  const int row0 = st * 128, row_last = min(s.L - 1, row0 + 127);
+  for (int i = tid; i < (8 * nT + 3) / 4; i += nthr) selw[i] = 0u;
+  __syncthreads();
+  for (int i = tid; i < G * s.topk; i += nthr) {
+    const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
+    if (qb < s.M) {
+      const int blk = idx[((int64_t)u * s.M + qb) * s.topk + slot];
+      if (blk >= 0 && blk <= qb) {
+        const int a = g * nT + blk / nb;
+        atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int jt_max = row_last >> 6;
+    int count = 0;
+    for (int base = 0; base <= jt_max; base += 32) {
+      const int jt = base + lane;
+      int f = 0;
+      if (jt <= jt_max && row_last >= pad0 && jt * 64 + 63 >= pad0) {
+        for (int g = 0; g < G; ++g) f |= selb[g * nT + jt] ? 1 : 0;
+        if (jt * 64 + 63 >= row0 - s.window + 1) f |= 2;
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
+      if (f) {
+        const int pos = count + __popc(bal & ((1u << lane) - 1u));
+        list[pos] = (uint16_t)jt;
+        lflags[pos] = (uint8_t)f;
+      }
+      count += __popc(bal);
+    }
+    if (lane == 0) *nvis_out = count;
+  }
+}
+
 // ---- host: TMA descriptor of a q-shaped bf16 tensor, box = (D, rows, 1, 1) -----------------
 int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows);
+
+// per-file launchers behind launch_fwd_tc / launch_bwd_tc
+template <int D>
+int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                    const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt,
+                    void *out_st, float *lse, const Workspace &ws, cudaStream_t st);
+template <int D>
+int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                    const int32_t *seq_lens, const int32_t *idx, const void *out_lt,
+                    const void *out_st, const float *lse, const void *dout, void *dq, void *dk,
+                    void *dv, const Workspace &ws, cudaStream_t st);
 
 }  // namespace tc
 }  // namespace blossom

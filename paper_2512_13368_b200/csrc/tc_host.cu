@@ -1,0 +1,62 @@
+// Host side of the tensor-core path: TMA descriptors and dispatch on the head dimension.
+#include "tc_common.cuh"
+
+namespace blossom {
+namespace tc {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// q-shaped bf16 tensor [B][H][L][D] with the caller's strides, box = (D, box_rows, 1, 1); rows
+// past L read as zeros.  The swizzle matches the shared-memory descriptors of the kernels.
+int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return 1;
+  const cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.L, (cuuint64_t)s.H, (cuuint64_t)s.B};
+  const cuuint64_t strides[3] = {(cuuint64_t)s.sl * 2, (cuuint64_t)s.sh * 2, (cuuint64_t)s.sb * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)s.D, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUtensorMapSwizzle sw = s.D == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? 0 : 1;
+}
+
+bool fwd_tc_supported(const Shape &s, int dtype) {
+  return dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+         (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
+}
+
+int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                  const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt, void *out_st,
+                  float *lse, const Workspace &ws, cudaStream_t st) {
+  if (s.D == 32) return launch_fwd_tc_t<32>(s, q, k, v, gate, seq_lens, idx, out, out_lt, out_st, lse, ws, st);
+  return launch_fwd_tc_t<64>(s, q, k, v, gate, seq_lens, idx, out, out_lt, out_st, lse, ws, st);
+}
+
+int launch_bwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                  const int32_t *seq_lens, const int32_t *idx, const void *out_lt, const void *out_st,
+                  const float *lse, const void *dout, void *dq, void *dk, void *dv,
+                  const Workspace &ws, cudaStream_t st) {
+  if (s.D == 32)
+    return launch_bwd_tc_t<32>(s, q, k, v, gate, seq_lens, idx, out_lt, out_st, lse, dout, dq, dk, dv, ws, st);
+  return launch_bwd_tc_t<64>(s, q, k, v, gate, seq_lens, idx, out_lt, out_st, lse, dout, dq, dk, dv, ws, st);
+}
+
+}  // namespace tc
+}  // namespace blossom
