@@ -83,8 +83,9 @@ size_t blossom_workspace_bytes(const blossom_params *params /* host */);
  * valid keys).  For each query block b: every valid query of the block takes a softmax of
  * sm_scale * <q, mean-key_j> over the live blocks j < b; the probabilities are summed over the
  * block's queries; the top_k - 1 largest sums (ties to the lower j) plus b itself are written
- * ascending to block_idx.  Scores are evaluated in double precision so that the choice matches
- * an fp64 evaluation except for ties below 1e-12 relative.
+ * ascending to block_idx.  The choice is the one a double-precision evaluation makes (ties below
+ * 1e-12 relative excepted): query blocks are first scored in single precision with an error
+ * bound, and only those whose choice the bound cannot certify are re-scored in double precision.
  *   q, k        in   q-shaped
  *   seq_lens    in   [B] or NULL
  *   block_idx   out  [B][H][M][top_k]
@@ -101,10 +102,11 @@ int blossom_select_blocks(const blossom_params *params /* host */, const void *q
  * serving process whose memory pool was handed out in full at start-up, in a plug-in that is
  * given tensors but no allocator, or on a thread that must not take the allocator's lock.  Such a
  * caller cannot size and allocate the workspace the other entry points ask for, so here the
- * scratch (per-block key means and live counts) is a fixed array inside the library image.
+ * scratch (per-block key means, live counts and the list of query blocks that need the
+ * double-precision pass) is a fixed array inside the library image.
  *
  *   - Nothing on this call path allocates or frees memory: no cudaMalloc / cudaFree, no library
- *     allocator.  The array (4 MiB + 32 KiB) is resident on every GPU that loads the library,
+ *     allocator.  The array (6 MiB + 96.25 KiB) is resident on every GPU that loads the library,
  *     from load to exit, whether or not this function is ever called.
  *   - Capacity: batch * heads * M <= 8192 and batch * heads * M * head_dim <= 524288
  *     (M = ceil(seq_len / block_size)); larger problems return BLOSSOM_ERR_TOO_LARGE before
@@ -113,7 +115,8 @@ int blossom_select_blocks(const blossom_params *params /* host */, const void *q
  *     once per device with that device current).  Make that first call outside any stream
  *     capture; later calls only launch kernels on `stream`.
  *   - All calls on a device share the one array.  It keeps whatever the previous call left in it;
- *     each call overwrites every entry before reading it, so no clearing is needed.  Two calls
+ *     each call overwrites every entry before reading it and its first kernel resets the one
+ *     counter that must start at zero, so the caller clears nothing.  Two calls
  *     whose kernels may run at the same time on one device (different streams, or different
  *     host threads) race on it and must be serialised by the caller.
  */

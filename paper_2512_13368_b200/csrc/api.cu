@@ -32,6 +32,11 @@ bool force_simt() {
   return e && e[0] && e[0] != '0';
 }
 
+bool exact_select_only() {
+  const char *e = getenv("BLOSSOM_EXACT_SELECT");
+  return e && e[0] && e[0] != '0';
+}
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 Workspace carve_workspace(const Shape &s, void *base) {
@@ -47,6 +52,10 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.status = reinterpret_cast<int32_t *>(take(256));
   w.kmean = reinterpret_cast<double *>(take(units * s.M * s.D * sizeof(double)));
   w.klive = reinterpret_cast<int32_t *>(take(units * s.M * sizeof(int32_t)));
+  w.kmean32 = reinterpret_cast<float *>(take(units * s.M * s.D * sizeof(float)));
+  w.knorm = reinterpret_cast<float *>(take(units * s.M * sizeof(float)));
+  w.sel_list = reinterpret_cast<int32_t *>(take(units * s.M * sizeof(int32_t)));
+  w.sel_count = reinterpret_cast<int32_t *>(take(256));
   w.delta = reinterpret_cast<float *>(take(2 * units * s.L * sizeof(float)));
   w.dalpha = reinterpret_cast<double *>(take(units * s.M * sizeof(double)));
   w.qstats = reinterpret_cast<float4 *>(take(units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4)));
@@ -253,7 +262,7 @@ int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
 const char *blossom_kernel_name(int id) {
   static const char *names[K_COUNT] = {
       "summary", "score_select", "fwd_simt", "bwd_dq_simt", "bwd_dkdv_simt", "gate_grad",
-      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc"};
+      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast"};
   return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

@@ -275,35 +275,33 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
       __syncwarp();
       tc_fence_after();
       const bool mine = anyL || anyS;
-      float sv[2][16], dp[2][16];
-      if (mine) {
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv[q]);
-          tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp[q]);
-        }
-        tmem_wait_ld();
-      }
-      tc_fence_before();
-      warp_arrive(b_sempty, lane);
-
       if (mine || !ds_zero) {
-#pragma unroll
+        // two passes of 16 columns (a rolled loop: one copy of each code path)
+#pragma unroll 1
         for (int q = 0; q < 2; ++q) {
+          float sv[16], dp[16];
           uint32_t dw[8];
+          if (mine) {
+            tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
+            tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
+            tmem_wait_ld();
+          }
+          if (q == 1) {  // S and dP of this tile are in registers: the next tile's may overwrite them
+            tc_fence_before();
+            warp_arrive(b_sempty, lane);
+          }
           const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
-          if (anyL && anyS) {
-            if (full) dq_tile<true, true, true>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
-            else dq_tile<true, true, false>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
-          } else if (anyL) {
-            if (full) dq_tile<true, false, true>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
-            else dq_tile<true, false, false>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
-          } else if (anyS) {
-            if (full) dq_tile<false, true, true>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
-            else dq_tile<false, true, false>(sv[q], dp[q], qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
-          } else {
+          if (!mine) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) dw[c] = 0u;
+          } else if (!full) {
+            dq_tile<true, true, false>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+          } else if (anyL && anyS) {
+            dq_tile<true, true, true>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+          } else if (anyL) {
+            dq_tile<true, false, true>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+          } else {
+            dq_tile<false, true, true>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
           }
           if (q == 0 && i >= 1) {  // the dS columns are free once dQ += dS K of tile i-1 has completed
             mbar_wait(b_done, (i - 1) & 1, &abort_flag, 208);
@@ -314,11 +312,15 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
         }
         tmem_wait_st();
         ds_zero = !mine;
-      } else if (i >= 1) {
-        // nothing to write, but keep in step with the barrier: a parity wait only tells the last
-        // two phases apart, so no warp may fall further behind than that
-        mbar_wait(b_done, (i - 1) & 1, &abort_flag, 219);
-        __syncwarp();
+      } else {
+        tc_fence_before();
+        warp_arrive(b_sempty, lane);
+        if (i >= 1) {
+          // nothing to write, but keep in step with the barrier: a parity wait only tells the last
+          // two phases apart, so no warp may fall further behind than that
+          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 219);
+          __syncwarp();
+        }
       }
       tc_fence_before();
       warp_arrive(b_tfull, lane);
@@ -596,7 +598,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
       // whatever this thread had left in those columns
       const float4 *stt =
           reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes) + half * 32;
-#pragma unroll
+#pragma unroll 1
       for (int q = 0; q < 2; ++q) {
         uint32_t ww[8], dw[8];
         if (anyL || anyS) {
@@ -606,16 +608,10 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
           tmem_wait_ld();
           const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
           const float4 *sq = stt + q * 16;
-          if (anyL && anyS) {
-            if (full) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-            else dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          } else if (anyL) {
-            if (full) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-            else dkdv_tile<true, false, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          } else {
-            if (full) dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-            else dkdv_tile<false, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          }
+          if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          else dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
         } else {
 #pragma unroll
           for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }

@@ -260,54 +260,39 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       tc_fence_before();
       warp_arrive(b_sempty, lane);
 
-      uint32_t pk[32];
-      float fac = 1.f;
-      bool need = false;
-      // ---- long-term branch ----
-      if (f & 1) {
-        if (doL) {
-          if (fullL) tile_softmax<true>(sv, maskL, sc2, mL, lL, fac, need, pk);
-          else tile_softmax<false>(sv, maskL, sc2, mL, lL, fac, need, pk);
+      // the two branches, one after the other through one copy of the code (a rolled loop)
+      bool waited = i == 0;
+#pragma unroll 1
+      for (int br = 0; br < 2; ++br) {
+        if (!(f & (1 << br))) continue;
+        const bool isL = br == 0;
+        const uint64_t mask = isL ? maskL : maskS;
+        const bool doB = isL ? doL : doS, fullB = isL ? fullL : fullS;
+        float m = isL ? mL : mS, l = isL ? lL : lS;
+        uint32_t pk[32];
+        float fac = 1.f;
+        bool need = false;
+        if (doB) {
+          if (fullB) tile_softmax<true>(sv, mask, sc2, m, l, fac, need, pk);
+          else tile_softmax<false>(sv, mask, sc2, m, l, fac, need, pk);
         }
-        if (i >= 1) {  // P regions and accumulators are free once the MMAs of tile i-1 completed
+        if (!waited) {  // P regions and accumulators are free once the MMAs of tile i-1 completed
           mbar_wait(b_done, (i - 1) & 1, &abort_flag, 108);
           __syncwarp();
           tc_fence_after();
+          waited = true;
         }
-        if (doL) {
-          if (accL && __any_sync(0xffffffffu, need)) rescale_acc<D>(tmem_ol + lane_off, fac);
-          tmem_st32u(tmem_pl + lane_off, pk);
-          zeroL = false;
-        } else if (!zeroL) {
+        const uint32_t t_p = (isL ? tmem_pl : tmem_ps) + lane_off, t_o = (isL ? tmem_ol : tmem_os) + lane_off;
+        const bool zero = isL ? zeroL : zeroS;
+        if (doB) {
+          if ((isL ? accL : accS) && __any_sync(0xffffffffu, need)) rescale_acc<D>(t_o, fac);
+          tmem_st32u(t_p, pk);
+        } else if (!zero) {
 #pragma unroll
           for (int c = 0; c < 32; ++c) pk[c] = 0u;
-          tmem_st32u(tmem_pl + lane_off, pk);
-          zeroL = true;
+          tmem_st32u(t_p, pk);
         }
-      }
-      // ---- short-term branch ----
-      if (f & 2) {
-        fac = 1.f;
-        need = false;
-        if (doS) {
-          if (fullS) tile_softmax<true>(sv, maskS, sc2, mS, lS, fac, need, pk);
-          else tile_softmax<false>(sv, maskS, sc2, mS, lS, fac, need, pk);
-        }
-        if (!(f & 1) && i >= 1) {
-          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 109);
-          __syncwarp();
-          tc_fence_after();
-        }
-        if (doS) {
-          if (accS && __any_sync(0xffffffffu, need)) rescale_acc<D>(tmem_os + lane_off, fac);
-          tmem_st32u(tmem_ps + lane_off, pk);
-          zeroS = false;
-        } else if (!zeroS) {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) pk[c] = 0u;
-          tmem_st32u(tmem_ps + lane_off, pk);
-          zeroS = true;
-        }
+        if (isL) { mL = m; lL = l; zeroL = !doB; } else { mS = m; lS = l; zeroS = !doB; }
       }
       tmem_wait_st();
       tc_fence_before();

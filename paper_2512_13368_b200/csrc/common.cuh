@@ -21,6 +21,10 @@ struct Workspace {
   int32_t *status;   // [4] word 0: device status (0 = ok)
   double *kmean;     // [B][H][M][D]  mean of each block's valid keys (Eq. 9 summary)
   int32_t *klive;    // [B][H][M]     number of valid keys in the block
+  float *kmean32;    // [B][H][M][D]  the means rounded to fp32 (single-precision scoring stage)
+  float *knorm;      // [B][H][M]     upper bound of the Euclidean norm of each fp32 mean
+  int32_t *sel_list; // [B][H][M]     query blocks whose choice the fp32 stage could not certify
+  int32_t *sel_count;// [1]           length of that list
   float *delta;      // [2][B][H][L]  rowsum(G_branch o O_branch) for the backward
   double *dalpha;    // [B][H][M]     per query block partial of d alpha
   float4 *qstats;    // [B][H][ceil(L/64)*64]  per query row: (lse_lt*log2e - log2 alpha,
@@ -35,7 +39,7 @@ extern unsigned long long g_launches;  // host-side launch counter
 // Kernel identifiers reported by the optional per-launch event profile.
 enum KernelId {
   K_SUMMARY = 0, K_SCORE_SELECT, K_FWD_SIMT, K_BWD_DQ_SIMT, K_BWD_DKDV_SIMT, K_GATE_GRAD,
-  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_COUNT
+  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_COUNT
 };
 void prof_mark(int id, int phase, cudaStream_t st);  // no-op unless a profile is running
 
@@ -105,5 +109,7 @@ int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, c
 
 // BLOSSOM_FORCE_SIMT=1 in the environment routes every call to the fp32 CUDA-core kernels.
 bool force_simt();
+// BLOSSOM_EXACT_SELECT=1 scores every query block in double precision (skips the fp32 stage).
+bool exact_select_only();
 
 }  // namespace blossom

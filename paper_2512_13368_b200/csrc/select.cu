@@ -1,9 +1,15 @@
 // Block summary, importance scoring and top-k selection (paper Eq. 8-10, 12, 13 with
 // compression size = stride = selection size = Bk and the summary = mean of a block's valid keys).
 //
-// Scores are evaluated in double precision: the selection is a discrete decision taken from
-// floating-point sums whose neighbours differ by ~1e-3 relative on Gaussian inputs, and the
-// library promises the fp64 choice (ties below ~1e-12 relative excepted).
+// The selection is a discrete decision taken from floating-point sums whose neighbours differ by
+// ~1e-3 relative on Gaussian inputs, and the library promises the choice a double-precision
+// evaluation makes (ties below ~1e-12 relative excepted).  Two stages deliver it:
+//   1. every query block is scored in single precision together with a rigorous bound on the
+//      distance of each score from its exact value; if the last kept and the first dropped
+//      candidate are further apart than the bound allows them to move, the choice is certain and
+//      is written out;
+//   2. the (few per cent of) query blocks whose choice is not certain are appended to a work
+//      list and re-scored in double precision by a second kernel.
 #include "common.cuh"
 
 namespace blossom {
@@ -19,10 +25,15 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restrict__ k,
                                                       const int32_t *__restrict__ seq_lens,
                                                       double *__restrict__ kmean,
-                                                      int32_t *__restrict__ klive) {
+                                                      int32_t *__restrict__ klive,
+                                                      float *__restrict__ kmean32,
+                                                      float *__restrict__ knorm,
+                                                      int32_t *__restrict__ sel_count) {
   constexpr int CH = D / 4;        // chunks per row
   constexpr int RG = 256 / CH;     // row groups
   __shared__ double part[RG][D];
+  __shared__ float sq[D];
+  if (blockIdx.x == 0 && threadIdx.x == 0) *sel_count = 0;  // work list of the scoring kernel
   const int j = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
@@ -41,9 +52,19 @@ __global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restri
   if (threadIdx.x < D) {
     double acc = 0;
     for (int r = 0; r < RG; ++r) acc += part[r][threadIdx.x];  // fixed order
-    kmean[((int64_t)u * s.M + j) * D + threadIdx.x] = cnt > 0 ? acc / (double)cnt : 0.0;
+    const double mean = cnt > 0 ? acc / (double)cnt : 0.0;
+    kmean[((int64_t)u * s.M + j) * D + threadIdx.x] = mean;
+    const float m32 = (float)mean;
+    kmean32[((int64_t)u * s.M + j) * D + threadIdx.x] = m32;
+    sq[threadIdx.x] = m32 * m32;
   }
-  if (threadIdx.x == 0) klive[(int64_t)u * s.M + j] = cnt;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    klive[(int64_t)u * s.M + j] = cnt;
+    float a = 0.f;
+    for (int c = 0; c < D; ++c) a += sq[c];
+    knorm[(int64_t)u * s.M + j] = sqrtf(a) * 1.0001f;  // an upper bound of the fp32 mean's norm
+  }
 }
 
 // ---- Eq. 10 + 12 + 13: scores of one query block and its top-k --------------------------
@@ -51,12 +72,11 @@ __global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restri
 // softmax over the candidates, per-warp partial sums, fixed-order combine, then warp 0 runs
 // top_k - 1 arg-max passes (value desc, index asc).
 template <typename T, int D>
-__global__ void __launch_bounds__(kSelThreads) score_select_kernel(
-    Shape s, const T *__restrict__ q, const double *__restrict__ kmean,
+__device__ __forceinline__ void score_select_row(
+    const Shape &s, const T *__restrict__ q, const double *__restrict__ kmean,
     const int32_t *__restrict__ klive, const int32_t *__restrict__ seq_lens,
-    int32_t *__restrict__ idx, int kt_in_smem) {
-  extern __shared__ double sm[];
-  const int b = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
+    int32_t *__restrict__ idx, int kt_in_smem, int row_id, double *sm) {
+  const int b = row_id % s.M, u = row_id / s.M, n = u / s.H, h = u % s.H;
   const int M = s.M;
   const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
   int len = seq_lens ? seq_lens[n] : s.L;
@@ -172,6 +192,258 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
   }
 }
 
+// The double-precision scoring of the query blocks on the work list (all of them when
+// worklist == nullptr).  grid: any; each CTA takes rows blockIdx.x, blockIdx.x + gridDim.x, ...
+template <typename T, int D>
+__global__ void __launch_bounds__(kSelThreads) score_select_kernel(
+    Shape s, const T *__restrict__ q, const double *__restrict__ kmean,
+    const int32_t *__restrict__ klive, const int32_t *__restrict__ seq_lens,
+    int32_t *__restrict__ idx, int kt_in_smem, const int32_t *__restrict__ worklist,
+    const int32_t *__restrict__ work_count) {
+  extern __shared__ double sm[];
+  const int total = worklist ? *work_count : s.M * s.B * s.H;
+  for (int w = blockIdx.x; w < total; w += gridDim.x) {
+    score_select_row<T, D>(s, q, kmean, klive, seq_lens, idx, kt_in_smem, worklist ? worklist[w] : w, sm);
+    __syncthreads();  // shared memory is reused by the next row
+  }
+}
+
+// ---- stage 1: single-precision scoring with an error bound ----------------------------------
+// grid M*B*H (unit-major), 256 threads, one query block per CTA.  Logits z[t][j] of the block's
+// (up to 64) queries against 64 candidate means at a time come from a register-blocked fp32
+// product out of shared memory (thread = 4 queries x 4 candidates); softmax per query row by 4
+// lanes; column sums in fixed order; warp 0 runs the top_k - 1 arg-max passes.
+//
+// Error bound.  With u = 2^-24: every logit is within E = (D + 4) u scale max|q_t| max|mean_j| of
+// its exact value (D roundings of the accumulation, the rounding of the mean to fp32, the scale),
+// so every exact probability lies within a factor exp(+-2E) of the exact softmax of the computed
+// logits; evaluating that softmax and the column sum in fp32 adds 2^-21 (exp2 approximation and
+// division), 2^-22 per unit of logit range, and (b/4 + 80 + 8 chunks) u for the sums.  R is the
+// total, relative; two scores a > b are in certain order when a - b > R (a + b).
+constexpr int kFastThreads = 256;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kFastThreads) score_select_fast_kernel(
+    Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
+    const float *__restrict__ knorm, const int32_t *__restrict__ klive,
+    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
+    int32_t *__restrict__ work_count) {
+  constexpr int P = D + 4;   // row pitch of the operand tiles (floats): conflict-free 128-bit reads
+  constexpr int ZP = 65;     // row pitch of the logit tile
+  extern __shared__ float fsm[];
+  __shared__ float rn[64];
+  __shared__ int kn_bits;
+  const int M = s.M;
+  float *qs = fsm;                 // [64][P]   the block's queries
+  float *ks = qs + 64 * P;         // [64][P]   a chunk of candidate means; reused as zs [64][ZP]
+  float *zs = ks;
+  float *S = ks + 64 * (P > ZP ? P : ZP);  // [M]
+  int *live = reinterpret_cast<int *>(S + M);  // [M]
+  int *taken = live + M;                       // [M]
+
+  const int b = blockIdx.x % M, u = blockIdx.x / M, n = u / s.H, h = u % s.H;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int qlo = max(b * s.Bk, pad0), qhi = min((b + 1) * s.Bk, s.L);
+  int32_t *row = idx + ((int64_t)u * M + b) * s.topk;
+  if (qlo >= qhi) {  // the query block holds only padding
+    for (int i = tid; i < s.topk; i += kFastThreads) row[i] = -1;
+    return;
+  }
+  if (tid == 0) kn_bits = 0;
+  for (int j = tid; j < b; j += kFastThreads) {
+    live[j] = klive[(int64_t)u * M + j] > 0;
+    taken[j] = 0;
+  }
+  __syncthreads();
+  int ncand = 0;
+  for (int j = 0; j < b; ++j) ncand += live[j];  // uniform
+  const int want = min(s.topk - 1, ncand);
+  bool certain = true;
+
+  if (ncand > want) {  // a real choice: score the candidates
+    // the query block, fp32, invalid rows zero
+    for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {
+      const int lt = i / (D / 4), c = (i % (D / 4)) * 4, t = b * s.Bk + lt;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (lt < s.Bk && t >= qlo && t < qhi) v = ld4(q + row_offset(s, n, h, t) + c);
+      *reinterpret_cast<float4 *>(qs + lt * P + c) = v;
+    }
+    {
+      float km = 0.f;
+      for (int j = tid; j < b; j += kFastThreads)
+        if (live[j]) km = fmaxf(km, knorm[(int64_t)u * M + j]);
+      if (km > 0.f) atomicMax(&kn_bits, __float_as_int(km));  // positive floats order like ints
+    }
+    __syncthreads();
+    if (tid < 64) {
+      float a = 0.f;
+      for (int c = 0; c < D; ++c) a = fmaf(qs[tid * P + c], qs[tid * P + c], a);
+      rn[tid] = sqrtf(a) * 1.0001f;
+    }
+    const int ty = tid >> 4, tx = tid & 15;          // product: queries ty + 16 a, candidates tx + 16 c
+    const int rt = tid >> 2, part = tid & 3;          // softmax: row rt, candidates part, part + 4, ...
+    const bool row_valid = rt < s.Bk && b * s.Bk + rt >= qlo && b * s.Bk + rt < qhi;
+    const int nchunks = (b + 63) / 64;
+    const float *kbase = kmean32 + (int64_t)u * M * D;
+    float mx = -INFINITY, den = 0.f;  // online softmax statistics of row rt (passes > 1 chunk)
+
+    auto logits_of_chunk = [&](int j0) {  // zs[t][j] = scale <q_t, mean_{j0+j}>
+      const int nb = min(64, b - j0);
+      __syncthreads();  // previous users of ks / zs are done
+      for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {
+        const int lj = i / (D / 4), c = (i % (D / 4)) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (lj < nb && live[j0 + lj]) v = *reinterpret_cast<const float4 *>(kbase + (int64_t)(j0 + lj) * D + c);
+        *reinterpret_cast<float4 *>(ks + lj * P + c) = v;
+      }
+      __syncthreads();
+      float acc[4][4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[a][c] = 0.f;
+#pragma unroll 4
+      for (int c = 0; c < D; c += 4) {
+        float4 qa[4], kb[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + c);
+          kb[a] = *reinterpret_cast<const float4 *>(ks + (tx + 16 * a) * P + c);
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
+            acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
+            acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
+            acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
+          }
+      }
+      __syncthreads();  // everyone has read ks: it becomes zs
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) zs[(ty + 16 * a) * ZP + tx + 16 * e] = s.scale * acc[a][e];
+      __syncthreads();
+    };
+    // probabilities of the chunk in place (zs[t][j] = p_t[j0 + j], 0 where there is none), then
+    // their column sums
+    auto probabilities_and_sums = [&](int j0) {
+      const int nb = min(64, b - j0);
+      const float inv = den > 0.f ? 1.f / den : 0.f;
+      for (int j = part; j < nb; j += 4) {
+        const bool on = row_valid && live[j0 + j];
+        zs[rt * ZP + j] = on ? __expf(zs[rt * ZP + j] - mx) * inv : 0.f;
+      }
+      __syncthreads();
+      if (tid < nb) {
+        float a = 0.f;
+        for (int t = 0; t < 64; ++t) a += zs[t * ZP + tid];  // fixed order
+        S[j0 + tid] = a;
+      }
+    };
+    auto row_statistics = [&](int j0) {  // fold the chunk into (mx, den) of row rt
+      const int nb = min(64, b - j0);
+      float cm = -INFINITY;
+      for (int j = part; j < nb; j += 4)
+        if (live[j0 + j]) cm = fmaxf(cm, zs[rt * ZP + j]);
+      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+      const float nm = fmaxf(mx, cm);
+      float e = 0.f;
+      if (nm > -INFINITY) {
+        for (int j = part; j < nb; j += 4)
+          if (live[j0 + j]) e += __expf(zs[rt * ZP + j] - nm);
+      }
+      e += __shfl_xor_sync(0xffffffffu, e, 1);
+      e += __shfl_xor_sync(0xffffffffu, e, 2);
+      den = (mx > -INFINITY ? den * __expf(mx - nm) : 0.f) + e;
+      mx = nm;
+    };
+
+    if (nchunks == 1) {
+      logits_of_chunk(0);
+      row_statistics(0);
+      probabilities_and_sums(0);
+    } else {
+      for (int ch = 0; ch < nchunks; ++ch) {
+        logits_of_chunk(ch * 64);
+        row_statistics(ch * 64);
+      }
+      for (int ch = 0; ch < nchunks; ++ch) {
+        logits_of_chunk(ch * 64);
+        probabilities_and_sums(ch * 64);
+      }
+    }
+    __syncthreads();
+  }
+
+  if (warp == 0) {
+    float smin = INFINITY;
+    for (int r = 0; r < want + 1; ++r) {  // the extra pass finds the best candidate left out
+      if (r == want && ncand <= want) break;
+      float bv = -INFINITY;
+      int bj = 0x7fffffff;
+      for (int j = lane; j < b; j += 32) {
+        if (!live[j] || taken[j]) continue;
+        const float vj = ncand > want ? S[j] : 0.f;
+        if (bj == 0x7fffffff || vj > bv) { bv = vj; bj = j; }  // ascending j: strict > keeps lower
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        if (oj != 0x7fffffff && (bj == 0x7fffffff || ov > bv || (ov == bv && oj < bj))) {
+          bv = ov;
+          bj = oj;
+        }
+      }
+      if (r < want) {
+        smin = bv;  // picks come in descending order: the last one is the smallest kept
+        if (lane == 0) taken[bj] = 1;
+        __syncwarp();
+      } else {
+        // bv = best dropped score.  Certain iff the gap exceeds what the errors can bridge.
+        float qn = fmaxf(rn[lane], rn[lane + 32]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, o));
+        const float kn = __int_as_float(kn_bits);
+        const float uu = 5.9604645e-8f;  // 2^-24
+        const float bound = s.scale * qn * kn;  // >= every |logit|
+        const float E = (float)(D + 4) * uu * bound * 1.01f;
+        const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f +
+                        ((float)b * 0.25f + 80.f + 8.f * (float)((b + 63) / 64)) * uu;
+        certain = (smin - bv) > R * (smin + bv) * 1.001f;
+      }
+    }
+    certain = __shfl_sync(0xffffffffu, certain ? 1 : 0, 0) != 0;
+    if (certain) {
+      // emit ascending: ballot over 32-wide chunks of the flags, then the own block
+      int pos = 0;
+      for (int base = 0; base < b; base += 32) {
+        const int j = base + lane;
+        const bool f = j < b && taken[j];
+        const unsigned m = __ballot_sync(0xffffffffu, f);
+        if (f) row[pos + __popc(m & ((1u << lane) - 1u))] = j;
+        pos += __popc(m);
+      }
+      if (lane == 0) row[pos] = b;
+      for (int i = pos + 1 + lane; i < s.topk; i += 32) row[i] = -1;
+    } else if (lane == 0) {
+      worklist[atomicAdd(work_count, 1)] = blockIdx.x;  // re-scored in double precision
+    }
+  }
+}
+
+size_t select_fast_smem_bytes(int M, int D) {
+  const int P = D + 4, ZP = 65;
+  return (size_t)(64 * P + 64 * (P > ZP ? P : ZP)) * sizeof(float) + (size_t)M * (sizeof(float) + 2 * sizeof(int));
+}
+
 size_t select_smem_bytes(int M, int D, bool kt_in_smem) {
   size_t dbl = (size_t)kSelWarps * M * 2 + (size_t)kSelWarps * D + M;
   size_t ints = 2 * (size_t)M;
@@ -185,7 +457,19 @@ int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_l
   const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.H);  // block = (unit, query block), unit-major
   {
     LaunchScope ls(K_SUMMARY, st);
-    summary_kernel<T, D><<<grid, 256, 0, st>>>(s, k, seq_lens, ws.kmean, ws.klive);
+    summary_kernel<T, D><<<grid, 256, 0, st>>>(s, k, seq_lens, ws.kmean, ws.klive, ws.kmean32, ws.knorm,
+                                               ws.sel_count);
+  }
+  const bool exact_only = exact_select_only();
+  if (!exact_only) {
+    const size_t fsm = select_fast_smem_bytes(s.M, D);
+    if (fsm > 48 * 1024 &&
+        cudaFuncSetAttribute(score_select_fast_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)fsm) != cudaSuccess)
+      return BLOSSOM_ERR_CUDA;
+    LaunchScope ls(K_SCORE_FAST, st);
+    score_select_fast_kernel<T, D><<<grid, kFastThreads, fsm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive,
+                                                                   seq_lens, idx, ws.sel_list, ws.sel_count);
   }
   bool in_smem = select_smem_bytes(s.M, D, true) <= 160 * 1024;
   size_t smem = select_smem_bytes(s.M, D, in_smem);
@@ -195,9 +479,12 @@ int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_l
       return BLOSSOM_ERR_CUDA;
   }
   {
+    // double precision: every query block (exact_only) or the work list of the kernel above
     LaunchScope ls(K_SCORE_SELECT, st);
-    score_select_kernel<T, D><<<grid, kSelThreads, smem, st>>>(s, q, ws.kmean, ws.klive, seq_lens,
-                                                               idx, in_smem ? 1 : 0);
+    const unsigned g2 = exact_only ? grid : (grid < 592u ? grid : 592u);
+    score_select_kernel<T, D><<<g2, kSelThreads, smem, st>>>(s, q, ws.kmean, ws.klive, seq_lens, idx,
+                                                            in_smem ? 1 : 0, exact_only ? nullptr : ws.sel_list,
+                                                            ws.sel_count);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
@@ -222,7 +509,13 @@ int launch_select(const Shape &s, int dtype, const void *q, const void *k, const
 // harmless; two calls in flight at once on one device would overwrite each other's means.
 constexpr size_t kStaticMeanElems = 524288;  // doubles: batch * heads * M * head_dim may not exceed this
 constexpr size_t kStaticBlocks = 8192;       // int32:   batch * heads * M may not exceed this
-constexpr size_t kStaticBytes = kStaticMeanElems * sizeof(double) + kStaticBlocks * sizeof(int32_t);
+// doubles (means) | floats (fp32 means) | int32 live counts | float norms | int32 work list | counter
+constexpr size_t kStaticOffMean32 = kStaticMeanElems * sizeof(double);
+constexpr size_t kStaticOffLive = kStaticOffMean32 + kStaticMeanElems * sizeof(float);
+constexpr size_t kStaticOffNorm = kStaticOffLive + kStaticBlocks * sizeof(int32_t);
+constexpr size_t kStaticOffList = kStaticOffNorm + kStaticBlocks * sizeof(float);
+constexpr size_t kStaticOffCount = kStaticOffList + kStaticBlocks * sizeof(int32_t);
+constexpr size_t kStaticBytes = kStaticOffCount + 256;
 static __device__ __align__(256) unsigned char g_select_scratch[kStaticBytes];
 
 constexpr int kMaxDevices = 64;
@@ -246,7 +539,11 @@ int launch_select_static(const Shape &s, int dtype, const void *q, const void *k
   unsigned char *base = static_cast<unsigned char *>(g_scratch_addr[dev]);
   Workspace ws = {};
   ws.kmean = reinterpret_cast<double *>(base);
-  ws.klive = reinterpret_cast<int32_t *>(base + kStaticMeanElems * sizeof(double));
+  ws.kmean32 = reinterpret_cast<float *>(base + kStaticOffMean32);
+  ws.klive = reinterpret_cast<int32_t *>(base + kStaticOffLive);
+  ws.knorm = reinterpret_cast<float *>(base + kStaticOffNorm);
+  ws.sel_list = reinterpret_cast<int32_t *>(base + kStaticOffList);
+  ws.sel_count = reinterpret_cast<int32_t *>(base + kStaticOffCount);
   return launch_select(s, dtype, q, k, seq_lens, idx, ws, st);
 }
 

@@ -206,3 +206,24 @@ def test_config2_full_size_sampled(runner):
     pad0 = w.L - w.seq_lens
     live_block = (np.minimum((np.arange(M) + 1) * w.block, w.L)[None, :] > pad0[:, None])
     assert np.all(np.where(live_block[:, None, :], last == own, last == -1))
+
+
+def test_certified_selection_equals_double_precision_selection(runner, monkeypatch):
+    """The two-stage selection (fp32 scores with an error bound, fp64 only for the uncertain query
+    blocks) must return exactly what scoring every query block in fp64 returns."""
+    import torch
+    for w in (workloads.config4(B=1), workloads.config2(B=16), workloads.config3(B=1),
+              workloads.make("many-blocks", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9)):
+        p = runner.DeviceProblem(w)
+        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
+        p.select()
+        torch.cuda.synchronize()
+        fast = p.idx.cpu().numpy().copy()
+        monkeypatch.setenv("BLOSSOM_EXACT_SELECT", "1")
+        p.idx.fill_(-7)
+        p.select()
+        torch.cuda.synchronize()
+        exact = p.idx.cpu().numpy()
+        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
+        assert np.array_equal(fast, exact), w.name
+        check_indices(w, fast)
