@@ -26,7 +26,8 @@ namespace tc {
 namespace {
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
-constexpr int kFwdThreads = 160;
+constexpr int kFwdThreads = 256;  // warps 0..3 softmax; 4 loader, 5 S issuer, 6 PV issuer, 7 spare
+constexpr int kProducerRegs = 40, kSoftmaxRegs = 216;  // (128 - 40) * 128 = (216 - 128) * 128
 constexpr int kSoftmaxWarps = 4;
 constexpr int kFwdStages = 4;
 constexpr uint32_t kFwdTmemCols = 256;
@@ -162,24 +163,48 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   const uint32_t tmem_s = tmem_base, tmem_pl = tmem_base + 64, tmem_ps = tmem_base + 96,
                  tmem_ol = tmem_base + 128, tmem_os = tmem_base + 192;
 
-  if (warp == kSoftmaxWarps) {
-    // ================================ producer ================================
-    if (lane == 0 && nvis > 0) {
-      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
-      constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
-      auto load_stage = [&](int j) {
+  if (warp >= kSoftmaxWarps) {
+    // ===================== three single-thread roles, one warp each =====================
+    setmaxnreg_dec<kProducerRegs>();
+    if (warp == kSoftmaxWarps && lane == 0 && nvis > 0) {
+      // ---- loader: K/V tiles, up to STAGES ahead of their consumers ----
+      mbar_expect_tx(b_res, C::kBigBytes);
+      tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+      for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
+        if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 105);
         const uint32_t bar = b_full + 8 * sj;
         uint8_t *kt = kv_tiles + sj * 2 * C::kSmallBytes;
         mbar_expect_tx(bar, 2 * C::kSmallBytes);
         tma_load_4d(smem_u32(kt), &tmk, bar, 0, (int)list[j] * 64, h, n);
         tma_load_4d(smem_u32(kt + C::kSmallBytes), &tmv, bar, 0, (int)list[j] * 64, h, n);
-      };
+      }
+    } else if (warp == kSoftmaxWarps + 1 && lane == 0 && nvis > 0) {
+      // ---- S = Q K^T of tile i as soon as the softmax warps hold S(i-1) in registers ----
+      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
+      const uint64_t dq = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
+      mbar_wait(b_res, 0, &abort_flag, 101);
+      for (int i = 0; i < nvis; ++i) {
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 102);
+        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 103);
+        tc_fence_after();
+        uint8_t *k_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes;
+        const uint64_t dk = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dq + 2 * k, dk + 2 * k, idesc_s, k > 0);
+        umma_commit(b_sfull);
+      }
+    } else if (warp == kSoftmaxWarps + 2 && lane == 0 && nvis > 0) {
+      // ---- O += P V of tile i once its probabilities are in tensor memory ----
+      constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
       int accL = 0, accS = 0;
-      auto second_stage = [&](int j) {  // O += P V of tile j, P read from tensor memory
-        const int f = lflags[j];
-        uint8_t *v_tile = kv_tiles + (j % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes;
+      for (int i = 0; i < nvis; ++i) {
+        const int f = lflags[i];
+        uint8_t *v_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes;
         const uint64_t dv = smem_desc(smem_u32(v_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 106);
+        mbar_wait(b_tfull, i & 1, &abort_flag, 104);
+        tc_fence_after();
         if (f & 1) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)
@@ -193,40 +218,12 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
           accS = 1;
         }
         umma_commit(b_done);
-        umma_commit(b_empty + 8 * (j % STAGES));
-      };
-      mbar_expect_tx(b_res, C::kBigBytes);
-      tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
-      for (int j = 0; j < min(STAGES - 1, nvis); ++j) load_stage(j);
-      const uint64_t dq = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
-      for (int i = 0; i < nvis; ++i) {
-        if (i == 0) mbar_wait(b_res, 0, &abort_flag, 101);
-        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 102);
-        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 103);
-        tc_fence_after();
-        uint8_t *k_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes;
-        const uint64_t dk = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dq + 2 * k, dk + 2 * k, idesc_s, k > 0);
-        umma_commit(b_sfull);
-        if (i >= 1) {
-          mbar_wait(b_tfull, (i - 1) & 1, &abort_flag, 104);
-          tc_fence_after();
-          second_stage(i - 1);
-          // tile i + STAGES - 2 goes into the stage tile i - 2 occupied
-          const int j = i + STAGES - 2;
-          if (j < nvis) {
-            if (i >= 2) mbar_wait(b_empty + 8 * ((i - 2) % STAGES), ((i - 2) / STAGES) & 1, &abort_flag, 105);
-            load_stage(j);
-          }
-        }
+        umma_commit(b_empty + 8 * (i % STAGES));  // S(i) completed before the softmax warps read it
       }
-      mbar_wait(b_tfull, (nvis - 1) & 1, &abort_flag, 106);
-      tc_fence_after();
-      second_stage(nvis - 1);
     }
   } else {
     // ================================ softmax =================================
+    setmaxnreg_inc<kSoftmaxRegs>();
     const int r = warp * 32 + lane, t = row0 + r, g = r / s.Bk;
     const bool row_ok = t < s.L;
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
