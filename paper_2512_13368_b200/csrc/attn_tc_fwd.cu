@@ -231,19 +231,43 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     bool zeroL = false, zeroS = false;
     int accL = 0, accS = 0;
     const float sc2 = s.scale * kLog2e;
+    const int t_lo = row0 + warp * 32;               // first row of this warp
+    const bool uni = s.Bk >= 32;                     // the warp's rows share one query block
+    const int gw = (warp * 32) / s.Bk;
+    const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
+    const bool rows_all = t_lo >= pad0 && t_lo + 31 < s.L;
 
     for (int i = 0; i < nvis; ++i) {
       const int jt = list[i], f = lflags[i], p0 = jt * 64;
+      // Classify the tile for this warp with warp-uniform integer tests (0 = no row needs it,
+      // 1 = every row sees all 64 keys, 2 = mixed); per-lane column masks only for mixed tiles.
       uint64_t maskL = 0ull, maskS = 0ull;
-      if (row_ok) {
-        const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
-        if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
-        if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
+      int cL = 0, cS = 0;
+      const bool some = p0 <= t_lo + 31 && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
+      const bool inner = rows_all && p0 >= pad0 && p0 + 63 <= t_lo;  // valid and causal for every row
+      if ((f & 1) && some) {
+        if (!uni) cL = 2;
+        else {
+          const uint32_t bits = selb[gw * nT + jt];
+          cL = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
+        }
       }
-      const bool doL = __any_sync(0xffffffffu, maskL != 0ull);
-      const bool doS = __any_sync(0xffffffffu, maskS != 0ull);
-      const bool fullL = __all_sync(0xffffffffu, maskL == ~0ull);
-      const bool fullS = __all_sync(0xffffffffu, maskS == ~0ull);
+      if ((f & 2) && some && p0 + 63 >= t_lo - s.window + 1) cS = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;
+      bool doL = cL == 1, doS = cS == 1, fullL = cL == 1, fullS = cS == 1;
+      if (cL == 2 || cS == 2) {
+        uint64_t mc = 0ull;
+        if (row_ok) mc = cols_le(t - p0) & cols_ge(pad0 - p0);
+        if (cL == 2) {
+          maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
+          doL = __any_sync(0xffffffffu, maskL != 0ull);
+          fullL = __all_sync(0xffffffffu, maskL == ~0ull);
+        }
+        if (cS == 2) {
+          maskS = mc & cols_ge(t - s.window + 1 - p0);
+          doS = __any_sync(0xffffffffu, maskS != 0ull);
+          fullS = __all_sync(0xffffffffu, maskS == ~0ull);
+        }
+      }
 
       mbar_wait(b_sfull, i & 1, &abort_flag, 107);
       __syncwarp();
