@@ -26,49 +26,43 @@ namespace tc {
 namespace {
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
-constexpr int kFwdThreads = 256;  // warps 0..3 softmax; 4 loader, 5 S issuer, 6 PV issuer, 7 spare
-constexpr int kProducerRegs = 40, kSoftmaxRegs = 216;  // (128 - 40) * 128 = (216 - 128) * 128
-constexpr int kSoftmaxWarps = 4;
+// warps 0..7 softmax (warp w: TMEM lane quarter w % 4, column half w / 4); 8 loader, 9 S issuer,
+// 10 PV issuer, 11 spare
+constexpr int kFwdThreads = 384;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kProducerRegs = 32, kSoftmaxRegs = 104;  // 256 * 104 + 128 * 32 = 384 * 80
 constexpr int kFwdStages = 4;
 constexpr uint32_t kFwdTmemCols = 256;
 
-// One branch of one tile for one query row: masked maximum, lazy rescale decision, probabilities
-// relative to the running maximum packed as bf16 pairs, running sum.  FULL = no column is masked
-// for any lane of the warp.
+__device__ __forceinline__ bool bit(uint32_t w, int c) { return (w >> c) & 1u; }
+
+// maximum of 32 logits (those whose bit is set, all of them when FULL)
 template <bool FULL>
-__device__ __forceinline__ void tile_softmax(const float (&sv)[64], uint64_t mask, float sc2, float &m,
-                                             float &l, float &fac, bool &need, uint32_t (&pk)[32]) {
-  const uint32_t mlo = (uint32_t)mask, mhi = (uint32_t)(mask >> 32);
+__device__ __forceinline__ float half_max(const float (&v)[32], uint32_t bits) {
   float a0 = -INFINITY, a1 = -INFINITY;
 #pragma unroll
-  for (int c = 0; c < 64; c += 4) {
-    float v[4];
+  for (int c = 0; c < 32; c += 4) {
+    float x[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int cc = c + e;
-      const bool on = FULL || (((cc < 32 ? mlo : mhi) >> (cc & 31)) & 1u);
-      v[e] = on ? sv[cc] : -INFINITY;
-    }
-    a0 = max3(a0, v[0], v[1]);
-    a1 = max3(a1, v[2], v[3]);
+    for (int e = 0; e < 4; ++e) x[e] = (FULL || bit(bits, c + e)) ? v[c + e] : -INFINITY;
+    a0 = max3(a0, x[0], x[1]);
+    a1 = max3(a1, x[2], x[3]);
   }
-  const float mt = fmaxf(a0, a1) * sc2;
-  need = mt > m + kRescaleThreshold;  // also true on the row's first keys
-  fac = 1.f;
-  if (need) {
-    fac = exp2f(m - mt);
-    l *= fac;
-    m = mt;
-  }
-  const float nm = -m;
+  return fmaxf(a0, a1);
+}
+
+// probabilities of 32 logits relative to the running maximum (nm = -m, log2 units), packed as
+// bf16 pairs; their sum is added to l
+template <bool FULL>
+__device__ __forceinline__ void half_probs(const float (&sv)[32], uint32_t bits, float sc2, float nm,
+                                           float &l, uint32_t (&pk)[16]) {
   float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-  for (int c = 0; c < 64; c += 2) {
+  for (int c = 0; c < 32; c += 2) {
     float a = exp2f(fmaf(sv[c], sc2, nm)), b = exp2f(fmaf(sv[c + 1], sc2, nm));
     if (!FULL) {
-      const uint32_t w = c < 32 ? mlo : mhi;
-      a = ((w >> (c & 31)) & 1u) ? a : 0.f;
-      b = ((w >> ((c + 1) & 31)) & 1u) ? b : 0.f;
+      a = bit(bits, c) ? a : 0.f;
+      b = bit(bits, c + 1) ? b : 0.f;
     }
     s0 += a;
     s1 += b;
@@ -77,18 +71,15 @@ __device__ __forceinline__ void tile_softmax(const float (&sv)[64], uint64_t mas
   l += s0 + s1;
 }
 
-// multiply the row's accumulator by fac (all lanes of the warp take part)
-template <int D>
+// multiply this thread's N accumulator columns by fac (all lanes of the warp take part)
+template <int N>
 __device__ __forceinline__ void rescale_acc(uint32_t taddr, float fac) {
+  float o[N];
+  tmem_ld<N>(taddr, o);
+  tmem_wait_ld();
 #pragma unroll
-  for (int c0 = 0; c0 < D; c0 += 32) {
-    float o[32];
-    tmem_ld32(taddr + c0, o);
-    tmem_wait_ld();
-#pragma unroll
-    for (int c = 0; c < 32; ++c) o[c] *= fac;
-    tmem_st32(taddr + c0, o);
-  }
+  for (int c = 0; c < N; ++c) o[c] *= fac;
+  tmem_st<N>(taddr, o);
   tmem_wait_st();
 }
 
@@ -103,11 +94,14 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   using C = Cfg<D>;
   constexpr int STAGES = kFwdStages;
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, t_full, mma_done
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, done[2], t_full[2] (tile parity:
+  // a softmax warp may be one tile ahead of the slowest one, so consecutive tiles must not share
+  // an arrival counter)
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 7];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int nvis_s;
+  __shared__ float2 xl[2][128];  // [column half][row]: partial sums (lt, st) for the epilogue
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
@@ -130,8 +124,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
-  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 4]);
+  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 2]), b_done = smem_u32(&bars[2 * STAGES + 3]);
+  const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 5]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;  // an earlier CTA timed out: do not wait again
@@ -146,7 +140,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     mbar_init(b_sfull, 1);
     mbar_init(b_sempty, kSoftmaxWarps);
     mbar_init(b_tfull, kSoftmaxWarps);
+    mbar_init(b_tfull + 8, kSoftmaxWarps);
     mbar_init(b_done, 1);
+    mbar_init(b_done + 8, 1);
     mbar_fence_init();
   }
   if (warp == 0) {
@@ -160,7 +156,10 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   tc_fence_after();
   const int nvis = nvis_s;
   const uint32_t tmem_base = tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_pl = tmem_base + 64, tmem_ps = tmem_base + 96,
+  // columns: S [0,64), probability buffers A [64,96) and B [96,128) (bf16 pairs), O_lt, O_st.
+  // A tile with one branch writes its probabilities to buffer (tile parity); a tile with both
+  // branches uses A for the long-term and B for the short-term branch.
+  const uint32_t tmem_s = tmem_base, tmem_pa = tmem_base + 64, tmem_pb = tmem_base + 96,
                  tmem_ol = tmem_base + 128, tmem_os = tmem_base + 192;
 
   if (warp >= kSoftmaxWarps) {
@@ -203,37 +202,43 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         uint8_t *v_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes;
         const uint64_t dv = smem_desc(smem_u32(v_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 106);
-        mbar_wait(b_tfull, i & 1, &abort_flag, 104);
+        mbar_wait(b_tfull + 8 * (i & 1), (i >> 1) & 1, &abort_flag, 104);
         tc_fence_after();
+        const uint32_t pl = f == 3 ? tmem_pa : ((i & 1) ? tmem_pb : tmem_pa);
+        const uint32_t ps = f == 3 ? tmem_pb : pl;
         if (f & 1) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_bf16_ts(tmem_ol, tmem_pl + 8 * k, dv + k * C::kKStep, idesc_pv, (accL | k) != 0);
+            umma_bf16_ts(tmem_ol, pl + 8 * k, dv + k * C::kKStep, idesc_pv, (accL | k) != 0);
           accL = 1;
         }
         if (f & 2) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_bf16_ts(tmem_os, tmem_ps + 8 * k, dv + k * C::kKStep, idesc_pv, (accS | k) != 0);
+            umma_bf16_ts(tmem_os, ps + 8 * k, dv + k * C::kKStep, idesc_pv, (accS | k) != 0);
           accS = 1;
         }
-        umma_commit(b_done);
+        umma_commit(b_done + 8 * (i & 1));
         umma_commit(b_empty + 8 * (i % STAGES));  // S(i) completed before the softmax warps read it
       }
     }
   } else {
     // ================================ softmax =================================
     setmaxnreg_inc<kSoftmaxRegs>();
-    const int r = warp * 32 + lane, t = row0 + r, g = r / s.Bk;
+    constexpr int OC = D / 2;  // accumulator columns per thread
+    const int quarter = warp & 3, half = warp >> 2;
+    const int r = quarter * 32 + lane, t = row0 + r, g = r / s.Bk;
     const bool row_ok = t < s.L;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    // Both threads of a row keep the same running maxima (each looks at all 64 logits of a tile)
+    // and the partial sums of their own 32 columns.
     float mL = -INFINITY, lL = 0.f, mS = -INFINITY, lS = 0.f;
-    bool zeroL = false, zeroS = false;
+    bool zeroA = false, zeroB = false;  // this thread's columns of buffer A / B hold zeros
     int accL = 0, accS = 0;
     const float sc2 = s.scale * kLog2e;
-    const int t_lo = row0 + warp * 32;               // first row of this warp
+    const int t_lo = row0 + quarter * 32;            // first row of this warp
     const bool uni = s.Bk >= 32;                     // the warp's rows share one query block
-    const int gw = (warp * 32) / s.Bk;
+    const int gw = (quarter * 32) / s.Bk;
     const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
     const bool rows_all = t_lo >= pad0 && t_lo + 31 < s.L;
 
@@ -272,93 +277,121 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       mbar_wait(b_sfull, i & 1, &abort_flag, 107);
       __syncwarp();
       tc_fence_after();
-      float sv[64];
+      float sv[32];                           // this thread's 32 logits
+      float oxL = -INFINITY, oxS = -INFINITY; // maxima of the other 32 logits of the row
       if (doL || doS) {
-        tmem_ld32(tmem_s + lane_off, sv);
-        tmem_ld32(tmem_s + lane_off + 32, sv + 32);
+        float ov[32];
+        tmem_ld32(tmem_s + lane_off + half * 32, sv);
+        tmem_ld32(tmem_s + lane_off + (half ^ 1) * 32, ov);
         tmem_wait_ld();
+        const uint32_t oL = (uint32_t)(maskL >> ((half ^ 1) * 32)), oS = (uint32_t)(maskS >> ((half ^ 1) * 32));
+        if (doL) oxL = fullL ? half_max<true>(ov, 0u) : half_max<false>(ov, oL);
+        if (doS) oxS = (fullS && fullL && doL) ? oxL : (fullS ? half_max<true>(ov, 0u) : half_max<false>(ov, oS));
       }
       tc_fence_before();
       warp_arrive(b_sempty, lane);
 
       // the two branches, one after the other through one copy of the code (a rolled loop)
-      bool waited = i == 0;
+      const bool both = f == 3;
+      bool waited_prev = i == 0;  // the MMAs of tile i-1 have completed
+      bool waited_buf = false;    // this tile's probability buffer(s) are free
 #pragma unroll 1
       for (int br = 0; br < 2; ++br) {
         if (!(f & (1 << br))) continue;
         const bool isL = br == 0;
-        const uint64_t mask = isL ? maskL : maskS;
+        const uint32_t bits = (uint32_t)((isL ? maskL : maskS) >> (half * 32));
         const bool doB = isL ? doL : doS, fullB = isL ? fullL : fullS;
         float m = isL ? mL : mS, l = isL ? lL : lS;
-        uint32_t pk[32];
+        uint32_t pk[16];
         float fac = 1.f;
         bool need = false;
         if (doB) {
-          if (fullB) tile_softmax<true>(sv, mask, sc2, m, l, fac, need, pk);
-          else tile_softmax<false>(sv, mask, sc2, m, l, fac, need, pk);
+          const float own = fullB ? half_max<true>(sv, 0u) : half_max<false>(sv, bits);
+          const float mt = fmaxf(own, isL ? oxL : oxS) * sc2;
+          need = mt > m + kRescaleThreshold;  // also true on the row's first keys
+          if (need) {
+            fac = exp2f(m - mt);
+            l *= fac;
+            m = mt;
+          }
+          if (fullB) half_probs<true>(sv, 0u, sc2, -m, l, pk);
+          else half_probs<false>(sv, bits, sc2, -m, l, pk);
         }
-        if (!waited) {  // P regions and accumulators are free once the MMAs of tile i-1 completed
-          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 108);
-          __syncwarp();
-          tc_fence_after();
-          waited = true;
+        // The buffer written now was last read by the MMAs of tile i-2 (tile i-1 when either of
+        // the two tiles carries both branches); rescaling needs those of tile i-1.
+        const bool rescale = doB && (isL ? accL : accS) && __any_sync(0xffffffffu, need);
+        const bool prev_both = i >= 1 && lflags[i - 1] == 3;
+        if (!waited_prev && (both || prev_both || rescale)) {
+          mbar_wait(b_done + 8 * ((i - 1) & 1), ((i - 1) >> 1) & 1, &abort_flag, 108);
+          waited_prev = waited_buf = true;
+        } else if (!waited_buf) {
+          if (i >= 2) mbar_wait(b_done + 8 * (i & 1), ((i - 2) >> 1) & 1, &abort_flag, 109);
+          waited_buf = true;
         }
-        const uint32_t t_p = (isL ? tmem_pl : tmem_ps) + lane_off, t_o = (isL ? tmem_ol : tmem_os) + lane_off;
-        const bool zero = isL ? zeroL : zeroS;
+        __syncwarp();
+        tc_fence_after();
+        const bool useB = both ? !isL : (i & 1);
+        const uint32_t t_p = (useB ? tmem_pb : tmem_pa) + lane_off + half * 16;
+        const bool zero = useB ? zeroB : zeroA;
         if (doB) {
-          if ((isL ? accL : accS) && __any_sync(0xffffffffu, need)) rescale_acc<D>(t_o, fac);
-          tmem_st32u(t_p, pk);
+          if (rescale) rescale_acc<OC>((isL ? tmem_ol : tmem_os) + lane_off + half * OC, fac);
+          tmem_st16u(t_p, pk);
         } else if (!zero) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) pk[c] = 0u;
-          tmem_st32u(t_p, pk);
+          for (int c = 0; c < 16; ++c) pk[c] = 0u;
+          tmem_st16u(t_p, pk);
         }
-        if (isL) { mL = m; lL = l; zeroL = !doB; } else { mS = m; lS = l; zeroS = !doB; }
+        if (useB) zeroB = !doB; else zeroA = !doB;
+        if (isL) { mL = m; lL = l; } else { mS = m; lS = l; }
       }
       tmem_wait_st();
       tc_fence_before();
-      warp_arrive(b_tfull, lane);
+      warp_arrive(b_tfull + 8 * (i & 1), lane);
       accL |= (f & 1);
       accS |= (f & 2);
     }
 
     // ---- epilogue ----
     if (nvis > 0) {
-      mbar_wait(b_done, (nvis - 1) & 1, &abort_flag, 110);
+      mbar_wait(b_done + 8 * ((nvis - 1) & 1), ((nvis - 1) >> 1) & 1, &abort_flag, 110);
       __syncwarp();
       tc_fence_after();
+    }
+    xl[half][r] = make_float2(lL, lS);
+    named_bar_sync(1 + quarter, 64);
+    {
+      const float2 a = xl[0][r], b = xl[1][r];  // fixed order: both threads get the same sums
+      lL = a.x + b.x;
+      lS = a.y + b.y;
     }
     const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
     const float iL = lL > 0.f ? 1.f / lL : 0.f, iS = lS > 0.f ? 1.f / lS : 0.f;
     const bool haveL = accL && lL > 0.f, haveS = accS && lS > 0.f;
-    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0);
+    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0) + half * OC;
+    float oL[OC], oS[OC];
+    if (accL) tmem_ld<OC>(tmem_ol + lane_off + half * OC, oL);  // accL / accS are CTA-uniform
+    if (accS) tmem_ld<OC>(tmem_os + lane_off + half * OC, oS);
+    tmem_wait_ld();
+    if (row_ok) {
 #pragma unroll
-    for (int c0 = 0; c0 < D; c0 += 32) {
-      float oL[32], oS[32];
-      if (accL) tmem_ld32(tmem_ol + lane_off + c0, oL);  // accL / accS are CTA-uniform
-      if (accS) tmem_ld32(tmem_os + lane_off + c0, oS);
-      tmem_wait_ld();
-      if (row_ok) {
+      for (int ch = 0; ch < OC / 8; ++ch) {
+        uint32_t wo[4], wl[4], ws[4];
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t wo[4], wl[4], ws[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int c = ch * 8 + e * 2;
-            const float a0 = haveL ? oL[c] * iL : 0.f, a1 = haveL ? oL[c + 1] * iL : 0.f;
-            const float b0 = haveS ? oS[c] * iS : 0.f, b1 = haveS ? oS[c + 1] * iS : 0.f;
-            wl[e] = pack_bf16(a0, a1);
-            ws[e] = pack_bf16(b0, b1);
-            wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
-          }
-          const int64_t off = ro + c0 + ch * 8;
-          *reinterpret_cast<uint4 *>(out + off) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
-          if (out_lt) *reinterpret_cast<uint4 *>(out_lt + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-          if (out_st) *reinterpret_cast<uint4 *>(out_st + off) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+        for (int e = 0; e < 4; ++e) {
+          const int c = ch * 8 + e * 2;
+          const float a0 = haveL ? oL[c] * iL : 0.f, a1 = haveL ? oL[c + 1] * iL : 0.f;
+          const float b0 = haveS ? oS[c] * iS : 0.f, b1 = haveS ? oS[c + 1] * iS : 0.f;
+          wl[e] = pack_bf16(a0, a1);
+          ws[e] = pack_bf16(b0, b1);
+          wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
         }
+        const int64_t off = ro + ch * 8;
+        *reinterpret_cast<uint4 *>(out + off) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+        if (out_lt) *reinterpret_cast<uint4 *>(out_lt + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+        if (out_st) *reinterpret_cast<uint4 *>(out_st + off) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
       }
     }
-    if (row_ok && lse) {
+    if (row_ok && lse && half == 0) {
       const int64_t BHL = (int64_t)s.B * s.H * s.L;
       lse[(int64_t)u * s.L + t] = lL > 0.f ? (mL + log2f(lL)) * kLn2 : 0.f;
       lse[BHL + (int64_t)u * s.L + t] = lS > 0.f ? (mS + log2f(lS)) * kLn2 : 0.f;
