@@ -37,14 +37,17 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
+// One probe of the barrier.  The last operand lets the hardware park the thread (up to that many
+// nanoseconds) until the phase completes instead of returning at once, so a waiting warp does
+// not compete for issue slots with the warps doing the arithmetic.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(1000000u)
       : "memory");
   return ok != 0;
 }
@@ -320,8 +323,9 @@ struct Cfg {
   static constexpr int kKStep = (16 * kRowBytes) >> 4;       // descriptor advance of 16 rows
 };
 
-// bytes of the per-CTA tile bookkeeping: [8][nT] selection bytes, nT list entries, nT flags
-__host__ __device__ inline int meta_bytes(int nT) { return ((11 * nT + 15) / 16) * 16 + 16; }
+// bytes of the per-CTA tile bookkeeping: [8][nT] selection bytes, nT list entries, nT flags, and
+// (forward) 2 nT per-phase items
+__host__ __device__ inline int meta_bytes(int nT) { return ((11 * nT + 15) / 16) * 16 + ((4 * nT + 15) / 16) * 16 + 16; }
 
 // one arrival per warp, after all its lanes are done
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
