@@ -3,15 +3,13 @@
 // A CTA owns 128 query rows (128 / Bk query blocks) and walks a list of items, one 64-key tile of
 // one branch each: first the tiles any of its query blocks selected (Eq. 14, 16), then the tiles
 // its rows reach through the window (Eq. 15, 17).  One accumulator serves both phases: when the
-// long-term phase ends its rows are parked in shared memory and the short-term phase starts the
+// long-term phase ends each thread parks its row in registers and the short-term phase starts the
 // accumulator afresh.  A tile that belongs to both branches is visited once per phase.
 //
-// CTA = 384 threads.  Warps 0..7 are softmax warps: warp w owns TMEM lane quarter w % 4 (32 query
-// rows) and column half w / 4 (32 of the 64 keys of a tile); both threads of a row look at all 64
-// logits for the row maximum, so they keep identical running maxima without talking to each
-// other, and each keeps the partial sum of its own columns.  Warp 8 lane 0 loads K/V tiles (TMA),
-// warp 9 lane 0 issues S = Q K^T, warp 10 lane 0 issues O += P V with P read from tensor memory.
-// Registers move from the three single-thread warps to the softmax warps (setmaxnreg).
+// CTA = 256 threads.  Warps 0..3 are softmax warps (thread = query row = TMEM lane: no exchange
+// between threads in the loop).  Warp 4 lane 0 loads K/V tiles (TMA), warp 5 lane 0 issues
+// S = Q K^T, warp 6 lane 0 issues O += P V with P read from tensor memory.  Registers move from
+// those single-thread warps to the softmax warps (setmaxnreg).
 //
 // Tensor memory (256 columns): S buffers [0,64) [64,128), probability buffers (bf16 pairs)
 // [128,160) [160,192), accumulator [192,192+D).  Item i uses S buffer and probability buffer
@@ -36,60 +34,73 @@ namespace tc {
 namespace {
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
-// warps 0..7 softmax (warp w: TMEM lane quarter w % 4, column half w / 4); 8 loader, 9 S issuer,
-// 10 PV issuer, 11 spare
-constexpr int kFwdThreads = 384;
-constexpr int kSoftmaxWarps = 8;
-constexpr int kProducerRegs = 32, kSoftmaxRegs = 104;  // 256 * 104 + 128 * 32 = 384 * 80
-constexpr int kFwdStages = 3;
+constexpr int kFwdThreads = 256;  // warps 0..3 softmax; 4 loader, 5 S issuer, 6 PV issuer, 7 spare
+constexpr int kSoftmaxWarps = 4;
+constexpr int kProducerRegs = 40, kSoftmaxRegs = 216;  // (128 - 40) * 128 = (216 - 128) * 128
+constexpr int kFwdStages = 5;
 constexpr uint32_t kFwdTmemCols = 256;
 
-__device__ __forceinline__ bool bit(uint32_t w, int c) { return (w >> c) & 1u; }
-
-// maximum of 32 logits (those whose bit is set, all of them when FULL)
+// maximum of a row's 64 logits (those whose mask bit is set, all of them when FULL)
 template <bool FULL>
-__device__ __forceinline__ float half_max(const float (&v)[32], uint32_t bits) {
-  float a0 = -INFINITY, a1 = -INFINITY;
+__device__ __forceinline__ float row_max(const float (&v)[64], uint64_t mask) {
+  const uint32_t mlo = (uint32_t)mask, mhi = (uint32_t)(mask >> 32);
+  float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
 #pragma unroll
-  for (int c = 0; c < 32; c += 4) {
-    float x[4];
+  for (int c = 0; c < 64; c += 8) {
+    float x[8];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) x[e] = (FULL || bit(bits, c + e)) ? v[c + e] : -INFINITY;
+    for (int e = 0; e < 8; ++e) {
+      const int cc = c + e;
+      x[e] = (FULL || (((cc < 32 ? mlo : mhi) >> (cc & 31)) & 1u)) ? v[cc] : -INFINITY;
+    }
     a0 = max3(a0, x[0], x[1]);
     a1 = max3(a1, x[2], x[3]);
+    a2 = max3(a2, x[4], x[5]);
+    a3 = max3(a3, x[6], x[7]);
   }
-  return fmaxf(a0, a1);
+  return fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
 }
 
-// probabilities of 32 logits relative to the running maximum (nm = -m, log2 units), packed as
-// bf16 pairs; their sum is added to l
+// probabilities of a row's 64 logits relative to the running maximum (nm = -m, log2 units),
+// packed as bf16 pairs; their sum is added to l.  Two logits per FMA / ADD instruction.
 template <bool FULL>
-__device__ __forceinline__ void half_probs(const float (&sv)[32], uint32_t bits, float sc2, float nm,
-                                           float &l, uint32_t (&pk)[16]) {
-  float s0 = 0.f, s1 = 0.f;
+__device__ __forceinline__ void row_probs(const float (&sv)[64], uint64_t mask, float sc2, float nm,
+                                          float &l, uint32_t (&pk)[32]) {
+  const uint32_t mlo = (uint32_t)mask, mhi = (uint32_t)(mask >> 32);
+  const float2 sc = make_float2(sc2, sc2), nn = make_float2(nm, nm);
+  float2 s0 = make_float2(0.f, 0.f), s1 = make_float2(0.f, 0.f);
 #pragma unroll
-  for (int c = 0; c < 32; c += 2) {
-    float a = exp2f(fmaf(sv[c], sc2, nm)), b = exp2f(fmaf(sv[c + 1], sc2, nm));
+  for (int c = 0; c < 64; c += 4) {
+    const float2 x0 = ffma2(make_float2(sv[c], sv[c + 1]), sc, nn);
+    const float2 x1 = ffma2(make_float2(sv[c + 2], sv[c + 3]), sc, nn);
+    float2 e0 = make_float2(exp2f(x0.x), exp2f(x0.y)), e1 = make_float2(exp2f(x1.x), exp2f(x1.y));
     if (!FULL) {
-      a = bit(bits, c) ? a : 0.f;
-      b = bit(bits, c + 1) ? b : 0.f;
+      const uint32_t w = (c < 32 ? mlo : mhi) >> (c & 31);
+      e0.x = (w & 1u) ? e0.x : 0.f;
+      e0.y = (w & 2u) ? e0.y : 0.f;
+      e1.x = (w & 4u) ? e1.x : 0.f;
+      e1.y = (w & 8u) ? e1.y : 0.f;
     }
-    s0 += a;
-    s1 += b;
-    pk[c >> 1] = pack_bf16(a, b);
+    s0 = fadd2(s0, e0);
+    s1 = fadd2(s1, e1);
+    pk[c >> 1] = pack_bf16(e0.x, e0.y);
+    pk[(c >> 1) + 1] = pack_bf16(e1.x, e1.y);
   }
-  l += s0 + s1;
+  l += (s0.x + s0.y) + (s1.x + s1.y);
 }
 
-// multiply this thread's N accumulator columns by fac (all lanes of the warp take part)
-template <int N>
+// multiply the row's accumulator by fac (all lanes of the warp take part)
+template <int D>
 __device__ __forceinline__ void rescale_acc(uint32_t taddr, float fac) {
-  float o[N];
-  tmem_ld<N>(taddr, o);
-  tmem_wait_ld();
 #pragma unroll
-  for (int c = 0; c < N; ++c) o[c] *= fac;
-  tmem_st<N>(taddr, o);
+  for (int c0 = 0; c0 < D; c0 += 32) {
+    float o[32];
+    tmem_ld32(taddr + c0, o);
+    tmem_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; ++c) o[c] *= fac;
+    tmem_st32(taddr + c0, o);
+  }
   tmem_wait_st();
 }
 
@@ -103,7 +114,6 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     int nT) {
   using C = Cfg<D>;
   constexpr int STAGES = kFwdStages;
-  constexpr int OC = D / 2;  // accumulator columns per thread
   extern __shared__ uint8_t smem_raw[];
   // barriers: full[STAGES], empty[STAGES], res, then pairs by item parity: s_full, s_empty,
   // t_full, done
@@ -111,7 +121,6 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int nvis_s, nL_s, nS_s;
-  __shared__ float2 xl[2][128];  // [column half][row]: partial sums (lt, st) for the epilogue
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
@@ -126,8 +135,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   uint8_t *tiles = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
   uint8_t *q_tile = tiles;
   uint8_t *kv_tiles = q_tile + C::kBigBytes;  // [stage][K, V]
-  float *park = reinterpret_cast<float *>(kv_tiles + STAGES * 2 * C::kSmallBytes);  // [D][128]
-  uint8_t *meta = reinterpret_cast<uint8_t *>(park + D * 128);
+  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;
   uint32_t *selw = reinterpret_cast<uint32_t *>(meta);
   uint8_t *selb = meta;
   uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
@@ -241,19 +249,17 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   } else {
     // ================================ softmax =================================
     setmaxnreg_inc<kSoftmaxRegs>();
-    const int quarter = warp & 3, half = warp >> 2;
-    const int r = quarter * 32 + lane, t = row0 + r, g = r / s.Bk;
+    const int r = warp * 32 + lane, t = row0 + r, g = r / s.Bk;
     const bool row_ok = t < s.L;
-    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    // Both threads of a row keep the same running maximum (each looks at all 64 logits of a tile)
-    // and the partial sum of their own 32 columns.
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     float m = -INFINITY, l = 0.f, mL = -INFINITY, lL = 0.f;
-    bool zeroA = false, zeroB = false;  // this thread's columns of probability buffer 0 / 1 hold zeros
+    float park[D];  // the row's long-term accumulator while the short-term phase runs
+    bool zeroA = false, zeroB = false;  // this row of probability buffer 0 / 1 holds zeros
     int acc = 0;                        // the current phase has written the accumulator
     const float sc2 = s.scale * kLog2e;
-    const int t_lo = row0 + quarter * 32;            // first row of this warp
+    const int t_lo = row0 + warp * 32;               // first row of this warp
     const bool uni = s.Bk >= 32;                     // the warp's rows share one query block
-    const int gw = (quarter * 32) / s.Bk;
+    const int gw = (warp * 32) / s.Bk;
     const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
     const bool rows_all = t_lo >= pad0 && t_lo + 31 < s.L;
 
@@ -290,14 +296,11 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       mbar_wait(b_sfull + 8 * par, (i >> 1) & 1, &abort_flag, 107);
       __syncwarp();
       tc_fence_after();
-      float sv[32];         // this thread's 32 logits
-      float ox = -INFINITY; // maximum of the other 32 logits of the row
+      float sv[64];
       if (doB) {
-        float ov[32];
-        tmem_ld32(tmem_s + 64 * par + lane_off + half * 32, sv);
-        tmem_ld32(tmem_s + 64 * par + lane_off + (half ^ 1) * 32, ov);
+        tmem_ld32(tmem_s + 64 * par + lane_off, sv);
+        tmem_ld32(tmem_s + 64 * par + lane_off + 32, sv + 32);
         tmem_wait_ld();
-        ox = fullB ? half_max<true>(ov, 0u) : half_max<false>(ov, (uint32_t)(mask >> ((half ^ 1) * 32)));
       }
       tc_fence_before();
       warp_arrive(b_sempty + 8 * par, lane);
@@ -310,11 +313,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         __syncwarp();
         tc_fence_after();
         waited_prev = true;
-        float o[OC];
-        tmem_ld<OC>(tmem_o + lane_off + half * OC, o);
-        tmem_wait_ld();
 #pragma unroll
-        for (int c = 0; c < OC; ++c) park[(half * OC + c) * 128 + r] = o[c];
+        for (int c0 = 0; c0 < D; c0 += 32) tmem_ld32(tmem_o + lane_off + c0, park + c0);
+        tmem_wait_ld();
         mL = m;
         lL = l;
         m = -INFINITY;
@@ -322,21 +323,19 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         acc = 0;
       }
 
-      const uint32_t bits = (uint32_t)(mask >> (half * 32));
-      uint32_t pk[16];
+      uint32_t pk[32];
       float fac = 1.f;
       bool need = false;
       if (doB) {
-        const float own = fullB ? half_max<true>(sv, 0u) : half_max<false>(sv, bits);
-        const float mt = fmaxf(own, ox) * sc2;
+        const float mt = (fullB ? row_max<true>(sv, 0ull) : row_max<false>(sv, mask)) * sc2;
         need = mt > m + kRescaleThreshold;  // also true on the row's first keys
         if (need) {
           fac = exp2f(m - mt);
           l *= fac;
           m = mt;
         }
-        if (fullB) half_probs<true>(sv, 0u, sc2, -m, l, pk);
-        else half_probs<false>(sv, bits, sc2, -m, l, pk);
+        if (fullB) row_probs<true>(sv, 0ull, sc2, -m, l, pk);
+        else row_probs<false>(sv, mask, sc2, -m, l, pk);
       }
       // Probability buffer i % 2 was last read by the MMAs of item i-2; rescaling the accumulator
       // needs those of item i-1.
@@ -348,15 +347,15 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       }
       __syncwarp();
       tc_fence_after();
-      const uint32_t t_p = tmem_p + 32 * par + lane_off + half * 16;
+      const uint32_t t_p = tmem_p + 32 * par + lane_off;
       const bool zero = par ? zeroB : zeroA;
       if (doB) {
-        if (rescale) rescale_acc<OC>(tmem_o + lane_off + half * OC, fac);
-        tmem_st16u(t_p, pk);
+        if (rescale) rescale_acc<D>(tmem_o + lane_off, fac);
+        tmem_st32u(t_p, pk);
       } else if (!zero) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) pk[c] = 0u;
-        tmem_st16u(t_p, pk);
+        for (int c = 0; c < 32; ++c) pk[c] = 0u;
+        tmem_st32u(t_p, pk);
       }
       if (par) zeroB = !doB; else zeroA = !doB;
       tmem_wait_st();
@@ -373,50 +372,46 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     }
     float mS = -INFINITY, lS = 0.f;
     if (nS > 0) { mS = m; lS = l; } else { mL = m; lL = l; }
-    xl[half][r] = make_float2(lL, lS);
-    named_bar_sync(1 + quarter, 64);
-    {
-      const float2 a = xl[0][r], b = xl[1][r];  // fixed order: both threads get the same sums
-      lL = a.x + b.x;
-      lS = a.y + b.y;
-    }
     const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
     const float iL = lL > 0.f ? 1.f / lL : 0.f, iS = lS > 0.f ? 1.f / lS : 0.f;
     const bool haveL = nL > 0 && lL > 0.f, haveS = nS > 0 && lS > 0.f;
-    const bool parked = nL > 0 && nS > 0;  // long-term rows in shared memory, short-term in TMEM
-    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0) + half * OC;
-    float o[OC];
-    if (nI > 0) {
-      tmem_ld<OC>(tmem_o + lane_off + half * OC, o);
-      tmem_wait_ld();
-    }
-    if (row_ok) {
+    const bool parked = nL > 0 && nS > 0;  // long-term rows in registers, short-term in TMEM
+    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0);
 #pragma unroll
-      for (int ch = 0; ch < OC / 8; ++ch) {
-        uint32_t wo[4], wl[4], ws[4];
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      float o[32];
+      if (nI > 0) {
+        tmem_ld32(tmem_o + lane_off + c0, o);
+        tmem_wait_ld();
+      }
+      if (row_ok) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int c = ch * 8 + e * 2;
-          float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-          if (haveL) {
-            a0 = (parked ? park[(half * OC + c) * 128 + r] : o[c]) * iL;
-            a1 = (parked ? park[(half * OC + c + 1) * 128 + r] : o[c + 1]) * iL;
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t wo[4], wl[4], ws[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = ch * 8 + e * 2;
+            float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+            if (haveL) {
+              a0 = (parked ? park[c0 + c] : o[c]) * iL;
+              a1 = (parked ? park[c0 + c + 1] : o[c + 1]) * iL;
+            }
+            if (haveS) {
+              b0 = o[c] * iS;
+              b1 = o[c + 1] * iS;
+            }
+            wl[e] = pack_bf16(a0, a1);
+            ws[e] = pack_bf16(b0, b1);
+            wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
           }
-          if (haveS) {
-            b0 = o[c] * iS;
-            b1 = o[c + 1] * iS;
-          }
-          wl[e] = pack_bf16(a0, a1);
-          ws[e] = pack_bf16(b0, b1);
-          wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
+          const int64_t off = ro + c0 + ch * 8;
+          *reinterpret_cast<uint4 *>(out + off) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+          if (out_lt) *reinterpret_cast<uint4 *>(out_lt + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+          if (out_st) *reinterpret_cast<uint4 *>(out_st + off) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
         }
-        const int64_t off = ro + ch * 8;
-        *reinterpret_cast<uint4 *>(out + off) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
-        if (out_lt) *reinterpret_cast<uint4 *>(out_lt + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-        if (out_st) *reinterpret_cast<uint4 *>(out_st + off) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
       }
     }
-    if (row_ok && lse && half == 0) {
+    if (row_ok && lse) {
       const int64_t BHL = (int64_t)s.B * s.H * s.L;
       lse[(int64_t)u * s.L + t] = lL > 0.f ? (mL + log2f(lL)) * kLn2 : 0.f;
       lse[BHL + (int64_t)u * s.L + t] = lS > 0.f ? (mS + log2f(lS)) * kLn2 : 0.f;
@@ -436,7 +431,7 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64) || make_tensor_map(&tv, v, s, 64))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
-  const size_t smem = 1024 + C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + (size_t)s.D * 128 * sizeof(float) + meta_bytes(nT);
+  const size_t smem = 1024 + C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT);
   if (cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return BLOSSOM_ERR_CUDA;
