@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
 constexpr int kFastThreads = 256;
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kFastThreads) score_select_fast_kernel(
+__global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
     Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
     const float *__restrict__ knorm, const int32_t *__restrict__ klive,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
@@ -232,6 +232,7 @@ __global__ void __launch_bounds__(kFastThreads) score_select_fast_kernel(
   constexpr int ZP = 65;     // row pitch of the logit tile
   extern __shared__ float fsm[];
   __shared__ float rn[64];
+  __shared__ float bound_s[2];
   __shared__ int kn_bits;
   const int M = s.M;
   float *qs = fsm;                 // [64][P]   the block's queries
@@ -253,17 +254,23 @@ __global__ void __launch_bounds__(kFastThreads) score_select_fast_kernel(
     return;
   }
   if (tid == 0) kn_bits = 0;
+  int mine = 0;
   for (int j = tid; j < b; j += kFastThreads) {
-    live[j] = klive[(int64_t)u * M + j] > 0;
+    const int lv = klive[(int64_t)u * M + j] > 0;
+    live[j] = lv;
     taken[j] = 0;
+    mine += lv;
   }
-  __syncthreads();
   int ncand = 0;
-  for (int j = 0; j < b; ++j) ncand += live[j];  // uniform
+  for (int base = 0; base < b; base += kFastThreads * 1) {  // one round unless b > 256
+    ncand += __syncthreads_count(base + tid < b && live[base + tid]);
+  }
+  (void)mine;
   const int want = min(s.topk - 1, ncand);
+  const bool choose = ncand > want && want > 0;  // a real choice: score the candidates
   bool certain = true;
 
-  if (ncand > want) {  // a real choice: score the candidates
+  if (choose) {
     // the query block, fp32, invalid rows zero
     for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {
       const int lt = i / (D / 4), c = (i % (D / 4)) * 4, t = b * s.Bk + lt;
@@ -382,45 +389,49 @@ __global__ void __launch_bounds__(kFastThreads) score_select_fast_kernel(
     __syncthreads();
   }
 
-  if (warp == 0) {
-    float smin = INFINITY;
-    for (int r = 0; r < want + 1; ++r) {  // the extra pass finds the best candidate left out
-      if (r == want && ncand <= want) break;
-      float bv = -INFINITY;
-      int bj = 0x7fffffff;
-      for (int j = lane; j < b; j += 32) {
-        if (!live[j] || taken[j]) continue;
-        const float vj = ncand > want ? S[j] : 0.f;
-        if (bj == 0x7fffffff || vj > bv) { bv = vj; bj = j; }  // ascending j: strict > keeps lower
+  // Selection by rank: candidate j is kept iff fewer than `want` live candidates beat it
+  // (larger score, or equal score and lower index).  4 lanes share a candidate.
+  if (choose) {
+    for (int j0 = 0; j0 < b; j0 += kFastThreads / 4) {
+      const int j = j0 + (tid >> 2), part = tid & 3;
+      int rank = 0;
+      if (j < b && live[j]) {
+        const float sj = S[j];
+        for (int i = part; i < b; i += 4)
+          if (live[i]) {
+            const float si = S[i];
+            rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
+          }
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-        if (oj != 0x7fffffff && (bj == 0x7fffffff || ov > bv || (ov == bv && oj < bj))) {
-          bv = ov;
-          bj = oj;
-        }
-      }
-      if (r < want) {
-        smin = bv;  // picks come in descending order: the last one is the smallest kept
-        if (lane == 0) taken[bj] = 1;
-        __syncwarp();
-      } else {
-        // bv = best dropped score.  Certain iff the gap exceeds what the errors can bridge.
-        float qn = fmaxf(rn[lane], rn[lane + 32]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, o));
-        const float kn = __int_as_float(kn_bits);
-        const float uu = 5.9604645e-8f;  // 2^-24
-        const float bound = s.scale * qn * kn;  // >= every |logit|
-        const float E = (float)(D + 4) * uu * bound * 1.01f;
-        const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f +
-                        ((float)b * 0.25f + 80.f + 8.f * (float)((b + 63) / 64)) * uu;
-        certain = (smin - bv) > R * (smin + bv) * 1.001f;
+      rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+      rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+      if (part == 0 && j < b && live[j]) {
+        taken[j] = rank < want;
+        if (rank == want - 1) bound_s[0] = S[j];  // the smallest kept score
+        if (rank == want) bound_s[1] = S[j];      // the largest dropped score
       }
     }
-    certain = __shfl_sync(0xffffffffu, certain ? 1 : 0, 0) != 0;
+  } else {
+    for (int j = tid; j < b; j += kFastThreads) taken[j] = want > 0 ? live[j] : 0;
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    if (choose) {
+      // Certain iff the gap between the last kept and the first dropped score exceeds what the
+      // errors can bridge.
+      float qn = fmaxf(rn[lane], rn[lane + 32]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, o));
+      const float kn = __int_as_float(kn_bits);
+      const float uu = 5.9604645e-8f;  // 2^-24
+      const float bound = s.scale * qn * kn;  // >= every |logit|
+      const float E = (float)(D + 4) * uu * bound * 1.01f;
+      const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f +
+                      ((float)b * 0.25f + 80.f + 8.f * (float)((b + 63) / 64)) * uu;
+      const float smin = bound_s[0], umax = bound_s[1];
+      certain = (smin - umax) > R * (smin + umax) * 1.001f;
+    }
     if (certain) {
       // emit ascending: ballot over 32-wide chunks of the flags, then the own block
       int pos = 0;
