@@ -160,7 +160,7 @@ def time_oracle(ws):
     return time.perf_counter() - t0
 
 
-SAMPLE_BATCH = {1: 4, 2: 256, 3: 16, 4: 8, 5: 32}   # ~10-30 s of oracle work each
+SAMPLE_BATCH = {1: 4, 2: 256, 3: 128, 4: 16, 5: 128}  # batch entries the oracle is timed on (a few to ~10 s of host work)
 
 
 def run_reference(args, w, cfg_desc):
