@@ -44,21 +44,21 @@ constexpr uint32_t kFwdTmemCols = 256;
 template <bool FULL>
 __device__ __forceinline__ float row_max(const float (&v)[64], uint64_t mask) {
   const uint32_t mlo = (uint32_t)mask, mhi = (uint32_t)(mask >> 32);
-  float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
+  float a[8];
 #pragma unroll
-  for (int c = 0; c < 64; c += 8) {
-    float x[8];
+  for (int e = 0; e < 8; ++e) a[e] = -INFINITY;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
+  for (int c = 0; c < 64; c += 16) {
+    float x[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
       const int cc = c + e;
       x[e] = (FULL || (((cc < 32 ? mlo : mhi) >> (cc & 31)) & 1u)) ? v[cc] : -INFINITY;
     }
-    a0 = max3(a0, x[0], x[1]);
-    a1 = max3(a1, x[2], x[3]);
-    a2 = max3(a2, x[4], x[5]);
-    a3 = max3(a3, x[6], x[7]);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] = max3(a[e], x[2 * e], x[2 * e + 1]);
   }
-  return fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+  return fmaxf(max3(a[0], a[1], a[2]), max3(max3(a[3], a[4], a[5]), a[6], a[7]));
 }
 
 // probabilities of a row's 64 logits relative to the running maximum (nm = -m, log2 units),
@@ -141,6 +141,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
   uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
   uint16_t *items = reinterpret_cast<uint16_t *>(meta + ((11 * nT + 15) / 16) * 16);  // [2 nT]
+  uint8_t *icls = reinterpret_cast<uint8_t *>(items + 2 * nT);                         // [2 nT][4]
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]);
@@ -188,6 +189,30 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     if (lane == 0) {
       nL_s = nl;
       nS_s = count - nl;
+    }
+    __syncwarp();
+    // Class of every (item, softmax warp): 0 = no row of the warp needs the tile, 1 = every row
+    // sees all 64 keys, 2 = mixed (the warp builds per-lane column masks).
+    const bool uni = s.Bk >= 32;  // a warp's 32 rows share one query block
+    const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
+    for (int e = lane; e < count * kSoftmaxWarps; e += 32) {
+      const int it = e / kSoftmaxWarps, w = e % kSoftmaxWarps;
+      const int jt = items[it], p0 = jt * 64, t_lo = row0 + w * 32;
+      const bool some = p0 <= t_lo + 31 && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
+      const bool inner = t_lo >= pad0 && t_lo + 31 < s.L && p0 >= pad0 && p0 + 63 <= t_lo;
+      int cls = 0;
+      if (some) {
+        if (it < nl) {
+          if (!uni) cls = 2;
+          else {
+            const uint32_t bits = selb[((w * 32) / s.Bk) * nT + jt];
+            cls = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
+          }
+        } else if (p0 + 63 >= t_lo - s.window + 1) {
+          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;
+        }
+      }
+      icls[e] = (uint8_t)cls;
     }
   }
   tc_fence_before();
@@ -257,31 +282,11 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     bool zeroA = false, zeroB = false;  // this row of probability buffer 0 / 1 holds zeros
     int acc = 0;                        // the current phase has written the accumulator
     const float sc2 = s.scale * kLog2e;
-    const int t_lo = row0 + warp * 32;               // first row of this warp
-    const bool uni = s.Bk >= 32;                     // the warp's rows share one query block
-    const int gw = (warp * 32) / s.Bk;
-    const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
-    const bool rows_all = t_lo >= pad0 && t_lo + 31 < s.L;
 
     for (int i = 0; i < nI; ++i) {
       const bool isL = i < nL;
       const int jt = items[i], p0 = jt * 64, par = i & 1;
-      // Classify the tile for this warp with warp-uniform integer tests (0 = no row needs it,
-      // 1 = every row sees all 64 keys, 2 = mixed); per-lane column masks only for mixed tiles.
-      const bool some = p0 <= t_lo + 31 && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
-      const bool inner = rows_all && p0 >= pad0 && p0 + 63 <= t_lo;  // valid and causal for every row
-      int cls = 0;
-      if (some) {
-        if (isL) {
-          if (!uni) cls = 2;
-          else {
-            const uint32_t bits = selb[gw * nT + jt];
-            cls = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
-          }
-        } else if (p0 + 63 >= t_lo - s.window + 1) {
-          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;
-        }
-      }
+      const int cls = icls[i * kSoftmaxWarps + warp];
       uint64_t mask = 0ull;
       bool doB = cls == 1, fullB = cls == 1;
       if (cls == 2) {
@@ -302,8 +307,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         tmem_ld32(tmem_s + 64 * par + lane_off + 32, sv + 32);
         tmem_wait_ld();
       }
-      tc_fence_before();
-      warp_arrive(b_sempty + 8 * par, lane);
+      warp_arrive(b_sempty + 8 * par, lane);  // the loads have completed (wait::ld)
 
       bool waited_prev = i == 0;  // the MMAs of item i-1 have completed
       if (i == nL && nL > 0) {
@@ -359,8 +363,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       }
       if (par) zeroB = !doB; else zeroA = !doB;
       tmem_wait_st();
-      tc_fence_before();
-      warp_arrive(b_tfull + 8 * par, lane);
+      warp_arrive(b_tfull + 8 * par, lane);  // the stores have completed (wait::st)
       acc = 1;
     }
 

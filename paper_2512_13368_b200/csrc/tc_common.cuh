@@ -340,8 +340,8 @@ struct Cfg {
 };
 
 // bytes of the per-CTA tile bookkeeping: [8][nT] selection bytes, nT list entries, nT flags, and
-// (forward) 2 nT per-phase items
-__host__ __device__ inline int meta_bytes(int nT) { return ((11 * nT + 15) / 16) * 16 + ((4 * nT + 15) / 16) * 16 + 16; }
+// (forward) 2 nT per-phase items with 4 class bytes each
+__host__ __device__ inline int meta_bytes(int nT) { return ((11 * nT + 15) / 16) * 16 + ((12 * nT + 15) / 16) * 16 + 16; }
 
 // one arrival per warp, after all its lanes are done
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
