@@ -15,8 +15,10 @@
 //         dS = alpha P_lt (dP - Delta_lt) + beta P_st (dP - Delta_st), Delta_x = rowsum(dO o O_x)
 //         (one tile for both branches, they share K); dQ += dS K.  The first-stage MMAs of tile
 //         i+1 run while the compute warps work on tile i.
-//         Prologue: Delta and the per-row record (lse_lt*log2e - log2 alpha, lse_st*log2e -
-//         log2 beta, Delta_lt, Delta_st) that the dK/dV kernel streams.
+//         Prologue: Delta and the records the dK/dV kernel streams: per pair of rows
+//         {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)}, nl = -(lse*log2e - log2 weight) (the
+//         branch weights alpha, beta ride in the exponent: alpha P_lt = exp2(s*log2e + nl_lt)).
+//         The tile arithmetic handles two columns per FMA / ADD / MUL (packed f32x2).
 //         d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
 //  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
 //         records) that selected one of its key blocks or whose window reaches them.
@@ -45,34 +47,40 @@ constexpr bool kTrustMmaIssueOrder = false;
 __device__ __forceinline__ bool bit(uint32_t w, int c) { return (w >> c) & 1u; }
 
 // ---------------------------------------------------------------------------- backward dQ
-// 16 columns of one tile for one row: dS packed to bf16 pairs, d alpha partial.
+// 16 columns of one tile for one row: dS packed to bf16 pairs, partial sums of P' dP.
+// nlL / nlS = -(lse * log2e - log2 alpha) resp. beta: the branch weight rides in the exponent, so
+// P' = alpha P_lt (beta P_st) comes straight out of the exponential; nDL / nDS = -Delta.
+// Two columns per FMA / ADD / MUL instruction.
 template <bool HAS_L, bool HAS_S, bool FULL>
 __device__ __forceinline__ void dq_tile(const float (&sv)[16], const float (&dp)[16], uint32_t hL,
-                                        uint32_t hS, float sc2, float lseL2, float lseS2, float DL,
-                                        float DS, float alpha, float beta, float &dal,
-                                        uint32_t (&dw)[8]) {
+                                        uint32_t hS, float sc2, float nlL, float nlS, float nDL,
+                                        float nDS, float2 &dalL, float2 &dalS, uint32_t (&dw)[8]) {
+  const float2 sc = make_float2(sc2, sc2);
 #pragma unroll
   for (int c = 0; c < 16; c += 2) {
-    float d[2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const float dpv = dp[c + e];
-      float acc = 0.f;
-      if (HAS_L) {
-        float p = exp2f(fmaf(sv[c + e], sc2, -lseL2));
-        if (!FULL) p = bit(hL, c + e) ? p : 0.f;
-        dal = fmaf(p, dpv, dal);
-        acc = (alpha * p) * (dpv - DL);
+    const float2 s2 = make_float2(sv[c], sv[c + 1]), dp2 = make_float2(dp[c], dp[c + 1]);
+    float2 acc = make_float2(0.f, 0.f);
+    if (HAS_L) {
+      const float2 x = ffma2(s2, sc, make_float2(nlL, nlL));
+      float2 p = make_float2(exp2f(x.x), exp2f(x.y));
+      if (!FULL) {
+        p.x = bit(hL, c) ? p.x : 0.f;
+        p.y = bit(hL, c + 1) ? p.y : 0.f;
       }
-      if (HAS_S) {
-        float p = exp2f(fmaf(sv[c + e], sc2, -lseS2));
-        if (!FULL) p = bit(hS, c + e) ? p : 0.f;
-        dal = fmaf(-p, dpv, dal);
-        acc = fmaf(beta * p, dpv - DS, acc);
-      }
-      d[e] = acc;
+      dalL = ffma2(p, dp2, dalL);
+      acc = fmul2(p, fadd2(dp2, make_float2(nDL, nDL)));
     }
-    dw[c >> 1] = pack_bf16(d[0], d[1]);
+    if (HAS_S) {
+      const float2 x = ffma2(s2, sc, make_float2(nlS, nlS));
+      float2 p = make_float2(exp2f(x.x), exp2f(x.y));
+      if (!FULL) {
+        p.x = bit(hS, c) ? p.x : 0.f;
+        p.y = bit(hS, c + 1) ? p.y : 0.f;
+      }
+      dalS = ffma2(p, dp2, dalS);
+      acc = ffma2(p, fadd2(dp2, make_float2(nDS, nDS)), acc);
+    }
+    dw[c >> 1] = pack_bf16(acc.x, acc.y);
   }
 }
 
@@ -252,10 +260,18 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
       DL = o0.x + o1.x;
       DS = o0.y + o1.y;
     }
-    if (half == 0 && t < Lpad)  // the row record the dK/dV kernel streams (zeros for rows that do not exist)
-      qstats[(int64_t)u * Lpad + t] = row_valid ? make_float4(lseL2 - log2f(alpha), lseS2 - log2f(beta), DL, DS)
-                                                : make_float4(0.f, 0.f, 0.f, 0.f);
-    float dal = 0.f;
+    // the branch weights ride in the exponent: P' = alpha P_lt = exp2(s - (lse - log2 alpha))
+    const float nlL = -(lseL2 - log2f(alpha)), nlS = -(lseS2 - log2f(beta));
+    if (half == 0 && t < Lpad) {
+      // The record the dK/dV kernel streams, laid out for two queries per instruction: per pair
+      // of rows {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)}; zeros for rows that do not exist.
+      float *rec = reinterpret_cast<float *>(qstats) + ((int64_t)u * Lpad + (t & ~1)) * 4 + (t & 1);
+      rec[0] = row_valid ? nlL : 0.f;
+      rec[2] = row_valid ? -DL : 0.f;
+      rec[4] = row_valid ? nlS : 0.f;
+      rec[6] = row_valid ? -DS : 0.f;
+    }
+    float2 dalL = make_float2(0.f, 0.f), dalS = make_float2(0.f, 0.f);  // sums of P' dP per branch
     bool ds_zero = false;
     const float sc2 = s.scale * kLog2e;
 
@@ -295,13 +311,13 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
 #pragma unroll
             for (int c = 0; c < 8; ++c) dw[c] = 0u;
           } else if (!full) {
-            dq_tile<true, true, false>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            dq_tile<true, true, false>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
           } else if (anyL && anyS) {
-            dq_tile<true, true, true>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            dq_tile<true, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
           } else if (anyL) {
-            dq_tile<true, false, true>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            dq_tile<true, false, true>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
           } else {
-            dq_tile<false, true, true>(sv, dp, qL, qS, sc2, lseL2, lseS2, DL, DS, alpha, beta, dal, dw);
+            dq_tile<false, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
           }
           if (q == 0 && i >= 1) {  // the dS columns are free once dQ += dS K of tile i-1 has completed
             mbar_wait(b_done, (i - 1) & 1, &abort_flag, 208);
@@ -349,6 +365,9 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
         *reinterpret_cast<uint4 *>(dq + ro + half * OC + ch * 8) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
+    // d alpha = sum (P_lt - P_st) dP; a weight of exactly 0 makes its branch's sum 0 and the gate
+    // gradient alpha (1 - alpha) d alpha 0 whatever d alpha is
+    const float dal = (alpha > 0.f ? (dalL.x + dalL.y) / alpha : 0.f) - (beta > 0.f ? (dalS.x + dalS.y) / beta : 0.f);
     red[tid] = row_valid ? (double)dal : 0.0;
   }
   tc_fence_before();
@@ -365,36 +384,42 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
 
 // ------------------------------------------------------------------------- backward dK, dV
 // 16 query columns of one tile for one key row: W^T and dS^T packed to bf16 pairs.  st points at
-// the row records (lse_lt', lse_st', Delta_lt, Delta_st) of these 16 queries.
+// the records of these 8 query pairs: {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)} per pair
+// (nl = -(lse * log2e - log2 weight): the branch weight rides in the exponent).  Two columns per
+// FMA / ADD / MUL instruction.
 template <bool HAS_L, bool HAS_S, bool FULL>
 __device__ __forceinline__ void dkdv_tile(const float (&sv)[16], const float (&dp)[16], uint32_t hL,
                                           uint32_t hS, float sc2, const float4 *st, uint32_t (&ww)[8],
                                           uint32_t (&dw)[8]) {
+  const float2 sc = make_float2(sc2, sc2);
 #pragma unroll
   for (int c = 0; c < 16; c += 2) {
-    float wv[2], d[2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const float4 q4 = st[c + e];
-      const float dpv = dp[c + e];
-      float wa = 0.f, da = 0.f;
-      if (HAS_L) {
-        float p = exp2f(fmaf(sv[c + e], sc2, -q4.x));
-        if (!FULL) p = bit(hL, c + e) ? p : 0.f;
-        wa = p;
-        da = p * (dpv - q4.z);
+    const float2 s2 = make_float2(sv[c], sv[c + 1]), dp2 = make_float2(dp[c], dp[c + 1]);
+    float2 w = make_float2(0.f, 0.f), d = make_float2(0.f, 0.f);
+    if (HAS_L) {
+      const float4 r = st[c];  // pair c / 2, long-term half of the record
+      const float2 x = ffma2(s2, sc, make_float2(r.x, r.y));
+      float2 p = make_float2(exp2f(x.x), exp2f(x.y));
+      if (!FULL) {
+        p.x = bit(hL, c) ? p.x : 0.f;
+        p.y = bit(hL, c + 1) ? p.y : 0.f;
       }
-      if (HAS_S) {
-        float p = exp2f(fmaf(sv[c + e], sc2, -q4.y));
-        if (!FULL) p = bit(hS, c + e) ? p : 0.f;
-        wa += p;
-        da = fmaf(p, dpv - q4.w, da);
-      }
-      wv[e] = wa;
-      d[e] = da;
+      w = p;
+      d = fmul2(p, fadd2(dp2, make_float2(r.z, r.w)));
     }
-    ww[c >> 1] = pack_bf16(wv[0], wv[1]);
-    dw[c >> 1] = pack_bf16(d[0], d[1]);
+    if (HAS_S) {
+      const float4 r = st[c + 1];  // short-term half
+      const float2 x = ffma2(s2, sc, make_float2(r.x, r.y));
+      float2 p = make_float2(exp2f(x.x), exp2f(x.y));
+      if (!FULL) {
+        p.x = bit(hS, c) ? p.x : 0.f;
+        p.y = bit(hS, c + 1) ? p.y : 0.f;
+      }
+      w = HAS_L ? fadd2(w, p) : p;
+      d = ffma2(p, fadd2(dp2, make_float2(r.z, r.w)), d);
+    }
+    ww[c >> 1] = pack_bf16(w.x, w.y);
+    dw[c >> 1] = pack_bf16(d.x, d.y);
   }
 }
 
@@ -607,7 +632,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
           tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
           tmem_wait_ld();
           const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
-          const float4 *sq = stt + q * 16;
+          const float4 *sq = stt + q * 16;  // 8 pairs x 2 float4
           if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
           else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
           else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);

@@ -27,8 +27,8 @@ struct Workspace {
   int32_t *sel_count;// [1]           length of that list
   float *delta;      // [2][B][H][L]  rowsum(G_branch o O_branch) for the backward
   double *dalpha;    // [B][H][M]     per query block partial of d alpha
-  float4 *qstats;    // [B][H][ceil(L/64)*64]  per query row: (lse_lt*log2e - log2 alpha,
-                     //   lse_st*log2e - log2 beta, Delta_lt, Delta_st) for the dK/dV kernel
+  float4 *qstats;    // [B][H][ceil(L/64)*64]  16 bytes per query row, laid out per pair of rows as
+                     //   {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)} for the dK/dV kernel
   size_t bytes;
 };
 
