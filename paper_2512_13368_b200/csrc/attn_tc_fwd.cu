@@ -107,11 +107,11 @@ __device__ __forceinline__ void rescale_acc(uint32_t taddr, float fac) {
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-    const __grid_constant__ CUtensorMap tmv, Shape s, const float *__restrict__ gate,
-    const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ idx,
-    __nv_bfloat16 *__restrict__ out, __nv_bfloat16 *__restrict__ out_lt,
-    __nv_bfloat16 *__restrict__ out_st, float *__restrict__ lse, int32_t *__restrict__ status,
-    int nT) {
+    const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
+    const __grid_constant__ CUtensorMap tmol, const __grid_constant__ CUtensorMap tmos, Shape s,
+    const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
+    const int32_t *__restrict__ idx, int training, float *__restrict__ lse,
+    int32_t *__restrict__ status, int nT) {
   using C = Cfg<D>;
   constexpr int STAGES = kFwdStages;
   extern __shared__ uint8_t smem_raw[];
@@ -379,7 +379,10 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const float iL = lL > 0.f ? 1.f / lL : 0.f, iS = lS > 0.f ? 1.f / lS : 0.f;
     const bool haveL = nL > 0 && lL > 0.f, haveS = nS > 0 && lS > 0.f;
     const bool parked = nL > 0 && nS > 0;  // long-term rows in registers, short-term in TMEM
-    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0);
+    // Rows go to shared memory in the layout TMA stores expect (the K/V stages are free: every
+    // load has landed and every MMA has completed), then three bulk stores write whole lines;
+    // rows past L are clipped by the hardware, padded rows are written as zeros.
+    uint8_t *so = kv_tiles, *sl = so + C::kBigBytes, *ss = sl + C::kBigBytes;
 #pragma unroll
     for (int c0 = 0; c0 < D; c0 += 32) {
       float o[32];
@@ -387,32 +390,42 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         tmem_ld32(tmem_o + lane_off + c0, o);
         tmem_wait_ld();
       }
-      if (row_ok) {
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t wo[4], wl[4], ws[4];
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t wo[4], wl[4], ws[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int c = ch * 8 + e * 2;
-            float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-            if (haveL) {
-              a0 = (parked ? park[c0 + c] : o[c]) * iL;
-              a1 = (parked ? park[c0 + c + 1] : o[c + 1]) * iL;
-            }
-            if (haveS) {
-              b0 = o[c] * iS;
-              b1 = o[c + 1] * iS;
-            }
-            wl[e] = pack_bf16(a0, a1);
-            ws[e] = pack_bf16(b0, b1);
-            wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
+        for (int e = 0; e < 4; ++e) {
+          const int c = ch * 8 + e * 2;
+          float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+          if (haveL) {
+            a0 = (parked ? park[c0 + c] : o[c]) * iL;
+            a1 = (parked ? park[c0 + c + 1] : o[c + 1]) * iL;
           }
-          const int64_t off = ro + c0 + ch * 8;
-          *reinterpret_cast<uint4 *>(out + off) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
-          if (out_lt) *reinterpret_cast<uint4 *>(out_lt + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-          if (out_st) *reinterpret_cast<uint4 *>(out_st + off) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+          if (haveS) {
+            b0 = o[c] * iS;
+            b1 = o[c + 1] * iS;
+          }
+          wl[e] = pack_bf16(a0, a1);
+          ws[e] = pack_bf16(b0, b1);
+          wo[e] = pack_bf16(alpha * a0 + beta * b0, alpha * a1 + beta * b1);
+        }
+        const int chunk = c0 / 8 + ch;
+        store_row_chunk<D>(so, r, chunk, make_uint4(wo[0], wo[1], wo[2], wo[3]));
+        if (training) {
+          store_row_chunk<D>(sl, r, chunk, make_uint4(wl[0], wl[1], wl[2], wl[3]));
+          store_row_chunk<D>(ss, r, chunk, make_uint4(ws[0], ws[1], ws[2], ws[3]));
         }
       }
+    }
+    fence_async_smem();
+    named_bar_sync(1, kSoftmaxWarps * 32);
+    if (tid == 0) {
+      tma_store_4d(&tmo, smem_u32(so), 0, row0, h, n);
+      if (training) {
+        tma_store_4d(&tmol, smem_u32(sl), 0, row0, h, n);
+        tma_store_4d(&tmos, smem_u32(ss), 0, row0, h, n);
+      }
+      tma_store_commit_and_wait();
     }
     if (row_ok && lse) {
       const int64_t BHL = (int64_t)s.B * s.H * s.L;
@@ -430,8 +443,11 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
                     const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt,
                     void *out_st, float *lse, const Workspace &ws, cudaStream_t st) {
   using C = Cfg<D>;
-  CUtensorMap tq, tk, tv;
-  if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64) || make_tensor_map(&tv, v, s, 64))
+  CUtensorMap tq, tk, tv, to, tol, tos;
+  const int training = out_lt != nullptr;
+  if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64) || make_tensor_map(&tv, v, s, 64) ||
+      make_tensor_map(&to, out, s, 128) || make_tensor_map(&tol, training ? out_lt : out, s, 128) ||
+      make_tensor_map(&tos, training ? out_st : out, s, 128))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const size_t smem = 1024 + C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT);
@@ -441,9 +457,8 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
   {
     LaunchScope ls(K_FWD_TC, st);
-    fwd_tc_kernel<D><<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, s, gate, seq_lens, idx,
-                                                     (__nv_bfloat16 *)out, (__nv_bfloat16 *)out_lt,
-                                                     (__nv_bfloat16 *)out_st, lse, ws.status, nT);
+    fwd_tc_kernel<D><<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, idx,
+                                                     training, lse, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

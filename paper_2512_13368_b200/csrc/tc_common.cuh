@@ -86,6 +86,20 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
       "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
+// 4-D tiled store shared -> global (rows past the tensor's extent are not written); the caller
+// commits and waits for the bulk group before the shared memory is reused or the CTA exits.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2,
+                                             int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+          reinterpret_cast<uint64_t>(map)),
+      "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_commit_and_wait() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -419,6 +433,14 @@ __device__ __forceinline__ void build_query_major_list(const Shape &s, const int
     }
     if (lane == 0) *nvis_out = count;
   }
+}
+
+// Store 16-byte chunk ch of row r of a D-wide bf16 tile laid out as TMA expects it (128-byte
+// swizzle for D = 64, 64-byte swizzle for D = 32).  `tile` must be 1024-byte aligned.
+template <int D>
+__device__ __forceinline__ void store_row_chunk(uint8_t *tile, int r, int ch, uint4 v) {
+  if constexpr (D == 64) *reinterpret_cast<uint4 *>(tile + r * 128 + ((ch ^ (r & 7)) << 4)) = v;
+  else *reinterpret_cast<uint4 *>(tile + r * 64 + ((ch ^ ((r >> 1) & 3)) << 4)) = v;
 }
 
 // ---- host: TMA descriptor of a q-shaped bf16 tensor, box = (D, rows, 1, 1) -----------------
