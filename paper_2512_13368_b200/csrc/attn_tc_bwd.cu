@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
     const int32_t *__restrict__ idx, const __nv_bfloat16 *__restrict__ out_lt,
     const __nv_bfloat16 *__restrict__ out_st, const float *__restrict__ lse,
-    const __nv_bfloat16 *__restrict__ dout, __nv_bfloat16 *__restrict__ dq,
+    const __nv_bfloat16 *__restrict__ dout, const __grid_constant__ CUtensorMap tmdq,
     float4 *__restrict__ qstats, double *__restrict__ dalpha_part, int32_t *__restrict__ status,
     int nT) {
   using C = Cfg<D>;
@@ -352,7 +352,10 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
       tmem_ld<OC>(tmem_dq + lane_off + half * OC, o);
       tmem_wait_ld();
     }
-    if (row_ok) {
+    {
+      // The rows go to shared memory in the layout a TMA store expects (the K/V stages are free:
+      // every load has landed and every MMA has completed); one bulk store then writes whole lines,
+      // clipped at L by the hardware.  Padded rows are written as zeros.
       const bool live = nvis > 0 && row_valid;
 #pragma unroll
       for (int ch = 0; ch < OC / 8; ++ch) {
@@ -362,7 +365,13 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
           const int c = ch * 8 + e * 2;
           w[e] = live ? pack_bf16(o[c] * s.scale, o[c + 1] * s.scale) : 0u;
         }
-        *reinterpret_cast<uint4 *>(dq + ro + half * OC + ch * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+        store_row_chunk<D>(kv_tiles, r, half * (OC / 8) + ch, make_uint4(w[0], w[1], w[2], w[3]));
+      }
+      fence_async_smem();
+      named_bar_sync(5, kComputeWarps * 32);
+      if (tid == 0) {
+        tma_store_4d(&tmdq, smem_u32(kv_tiles), 0, row0, h, n);
+        tma_store_commit_and_wait();
       }
     }
     // d alpha = sum (P_lt - P_st) dP; a weight of exactly 0 makes its branch's sum 0 and the gate
@@ -428,8 +437,8 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
     const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ idx,
-    const float4 *__restrict__ qstats, __nv_bfloat16 *__restrict__ dk, __nv_bfloat16 *__restrict__ dv,
-    int32_t *__restrict__ status, int nT) {
+    const float4 *__restrict__ qstats, const __grid_constant__ CUtensorMap tmdk,
+    const __grid_constant__ CUtensorMap tmdv, int32_t *__restrict__ status, int nT) {
   using C = Cfg<D>;
   constexpr int STAGES = kKvStages;
   constexpr int OC = D / 2;
@@ -660,9 +669,10 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
       tmem_ld<OC>(tmem_dk + lane_off + half * OC, okk);
       tmem_wait_ld();
     }
-    if (row_ok) {
+    {
+      // staged in the (now free) Q/dO stages, then two whole-line bulk stores clipped at L
       const bool live = nvis > 0 && row_valid;
-      const int64_t ro = row_offset(s, n, h, p) + half * OC;
+      uint8_t *sv_t = qg_tiles, *sk_t = qg_tiles + C::kBigBytes;
 #pragma unroll
       for (int ch = 0; ch < OC / 8; ++ch) {
         uint32_t wv[4], wk[4];
@@ -672,8 +682,15 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
           wv[e] = live ? pack_bf16(ov[c], ov[c + 1]) : 0u;
           wk[e] = live ? pack_bf16(okk[c] * s.scale, okk[c + 1] * s.scale) : 0u;
         }
-        *reinterpret_cast<uint4 *>(dv + ro + ch * 8) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
-        *reinterpret_cast<uint4 *>(dk + ro + ch * 8) = make_uint4(wk[0], wk[1], wk[2], wk[3]);
+        store_row_chunk<D>(sv_t, r, half * (OC / 8) + ch, make_uint4(wv[0], wv[1], wv[2], wv[3]));
+        store_row_chunk<D>(sk_t, r, half * (OC / 8) + ch, make_uint4(wk[0], wk[1], wk[2], wk[3]));
+      }
+      fence_async_smem();
+      named_bar_sync(5, kComputeWarps * 32);
+      if (tid == 0) {
+        tma_store_4d(&tmdv, smem_u32(sv_t), 0, key0, h, n);
+        tma_store_4d(&tmdk, smem_u32(sk_t), 0, key0, h, n);
+        tma_store_commit_and_wait();
       }
     }
   }
@@ -689,11 +706,12 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
                     void *dv, const Workspace &ws, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   using C = Cfg<D>;
-  CUtensorMap q128, k64, v64, g128, q64, k128, v128, g64;
+  CUtensorMap q128, k64, v64, g128, q64, k128, v128, g64, tdq, tdk, tdv;
   if (make_tensor_map(&q128, q, s, 128) || make_tensor_map(&k64, k, s, 64) ||
       make_tensor_map(&v64, v, s, 64) || make_tensor_map(&g128, dout, s, 128) ||
       make_tensor_map(&q64, q, s, 64) || make_tensor_map(&k128, k, s, 128) ||
-      make_tensor_map(&v128, v, s, 128) || make_tensor_map(&g64, dout, s, 64))
+      make_tensor_map(&v128, v, s, 128) || make_tensor_map(&g64, dout, s, 64) ||
+      make_tensor_map(&tdq, dq, s, 128) || make_tensor_map(&tdk, dk, s, 128) || make_tensor_map(&tdv, dv, s, 128))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
@@ -707,13 +725,13 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
     LaunchScope ls(K_BWD_DQ_TC, st);
     bwd_dq_tc_kernel<D><<<grid, kBwdThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, idx,
                                                            (const bf *)out_lt, (const bf *)out_st, lse,
-                                                           (const bf *)dout, (bf *)dq, ws.qstats, ws.dalpha,
+                                                           (const bf *)dout, tdq, ws.qstats, ws.dalpha,
                                                            ws.status, nT);
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
     bwd_dkdv_tc_kernel<D><<<grid, kBwdThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, idx,
-                                                             ws.qstats, (bf *)dk, (bf *)dv, ws.status, nT);
+                                                             ws.qstats, tdk, tdv, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
