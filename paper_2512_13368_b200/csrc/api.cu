@@ -262,7 +262,7 @@ int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
 const char *blossom_kernel_name(int id) {
   static const char *names[K_COUNT] = {
       "summary", "score_select", "fwd_simt", "bwd_dq_simt", "bwd_dkdv_simt", "gate_grad",
-      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast"};
+      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast", "bwd_prep"};
   return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

@@ -1,5 +1,5 @@
-// Tensor-core backward of the fused two-branch attention (bf16 storage, fp32 accumulate): two
-// kernels, both deterministic (no atomics on any gradient), both recomputing the probabilities
+// Tensor-core backward of the fused two-branch attention (bf16 storage, fp32 accumulate): a small
+// pre-pass and two main kernels, all deterministic (no atomics on any gradient), both recomputing the probabilities
 // from the saved log-sum-exps.
 //
 // CTA = 288 threads: warps 0..7 compute, warp 8 is the producer (one lane issues every TMA load
@@ -15,9 +15,10 @@
 //         dS = alpha P_lt (dP - Delta_lt) + beta P_st (dP - Delta_st), Delta_x = rowsum(dO o O_x)
 //         (one tile for both branches, they share K); dQ += dS K.  The first-stage MMAs of tile
 //         i+1 run while the compute warps work on tile i.
-//         Prologue: Delta and the records the dK/dV kernel streams: per pair of rows
-//         {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)}, nl = -(lse*log2e - log2 weight) (the
-//         branch weights alpha, beta ride in the exponent: alpha P_lt = exp2(s*log2e + nl_lt)).
+//         Row statistics come from the pre-pass kernel (coalesced reads of dO, O_lt, O_st):
+//         per pair of rows {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)},
+//         nl = -(lse*log2e - log2 weight) (the branch weights alpha, beta ride in the exponent:
+//         alpha P_lt = exp2(s*log2e + nl_lt)); the dK/dV kernel streams the same records.
 //         The tile arithmetic handles two columns per FMA / ADD / MUL (packed f32x2).
 //         d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
 //  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
@@ -45,6 +46,68 @@ constexpr int kStatBytes = 64 * 16;  // one 64-query tile of row records
 constexpr bool kTrustMmaIssueOrder = false;
 
 __device__ __forceinline__ bool bit(uint32_t w, int c) { return (w >> c) & 1u; }
+
+// ------------------------------------------------------------------ backward pre-pass
+// Delta_x = rowsum(dO o O_x) of both branches and the per-row records both backward kernels read:
+// per pair of rows {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)} with
+// nl = -(lse * log2e - log2 weight), the branch weight (alpha, beta) riding in the exponent;
+// zeros for padded rows and for the rows that pad L to a multiple of 64.
+// D / 8 lanes share a row (one 16-byte load per tensor each): fully coalesced reads.
+template <int D>
+__global__ void __launch_bounds__(256) bwd_prep_kernel(Shape s, const float *__restrict__ gate,
+                                                       const int32_t *__restrict__ seq_lens,
+                                                       const __nv_bfloat16 *__restrict__ out_lt,
+                                                       const __nv_bfloat16 *__restrict__ out_st,
+                                                       const float *__restrict__ lse,
+                                                       const __nv_bfloat16 *__restrict__ dout,
+                                                       float4 *__restrict__ qstats, int Lpad) {
+  constexpr int LPR = D / 8;         // lanes per row
+  constexpr int RPB = 256 / LPR;     // rows per block
+  const int blocks_per_unit = (Lpad + RPB - 1) / RPB;
+  const int u = blockIdx.x / blocks_per_unit, n = u / s.H, h = u % s.H;
+  const int t = (blockIdx.x % blocks_per_unit) * RPB + threadIdx.x / LPR, ch = threadIdx.x % LPR;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const bool row_valid = t < s.L && t >= s.L - len;
+  float aL = 0.f, aS = 0.f;
+  if (row_valid) {
+    const int64_t off = row_offset(s, n, h, t) + ch * 8;
+    const uint4 gv = *reinterpret_cast<const uint4 *>(dout + off);
+    const uint4 lv = *reinterpret_cast<const uint4 *>(out_lt + off);
+    const uint4 sv4 = *reinterpret_cast<const uint4 *>(out_st + off);
+    const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, lw[4] = {lv.x, lv.y, lv.z, lv.w},
+                   sw[4] = {sv4.x, sv4.y, sv4.z, sv4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float g0 = __uint_as_float(gw[e] << 16), g1 = __uint_as_float(gw[e] & 0xffff0000u);
+      aL = fmaf(g0, __uint_as_float(lw[e] << 16), aL);
+      aL = fmaf(g1, __uint_as_float(lw[e] & 0xffff0000u), aL);
+      aS = fmaf(g0, __uint_as_float(sw[e] << 16), aS);
+      aS = fmaf(g1, __uint_as_float(sw[e] & 0xffff0000u), aS);
+    }
+  }
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) {  // fixed-shape tree over the row's lanes
+    aL += __shfl_xor_sync(0xffffffffu, aL, o);
+    aS += __shfl_xor_sync(0xffffffffu, aS, o);
+  }
+  if (ch == 0 && t < Lpad) {
+    float r0 = 0.f, r2 = 0.f, r4 = 0.f, r6 = 0.f;
+    if (row_valid) {
+      const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
+      const int64_t BHL = (int64_t)s.B * s.H * s.L;
+      r0 = -(lse[(int64_t)u * s.L + t] * kLog2e - log2f(alpha));
+      r4 = -(lse[BHL + (int64_t)u * s.L + t] * kLog2e - log2f(beta));
+      r2 = -aL;
+      r6 = -aS;
+    }
+    float *rec = reinterpret_cast<float *>(qstats) + ((int64_t)u * Lpad + (t & ~1)) * 4 + (t & 1);
+    rec[0] = r0;
+    rec[2] = r2;
+    rec[4] = r4;
+    rec[6] = r6;
+  }
+}
 
 // ---------------------------------------------------------------------------- backward dQ
 // 16 columns of one tile for one row: dS packed to bf16 pairs, partial sums of P' dP.
@@ -89,10 +152,8 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
-    const int32_t *__restrict__ idx, const __nv_bfloat16 *__restrict__ out_lt,
-    const __nv_bfloat16 *__restrict__ out_st, const float *__restrict__ lse,
-    const __nv_bfloat16 *__restrict__ dout, const __grid_constant__ CUtensorMap tmdq,
-    float4 *__restrict__ qstats, double *__restrict__ dalpha_part, int32_t *__restrict__ status,
+    const int32_t *__restrict__ idx, const __grid_constant__ CUtensorMap tmdq,
+    const float4 *__restrict__ qstats, double *__restrict__ dalpha_part, int32_t *__restrict__ status,
     int nT) {
   using C = Cfg<D>;
   constexpr int STAGES = kDqStages;
@@ -103,7 +164,6 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int nvis_s;
-  __shared__ float2 xch[2][128];
   __shared__ double red[256];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -227,49 +287,14 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
     const bool row_ok = t < s.L, row_valid = row_ok && t >= pad0;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
-    const int64_t BHL = (int64_t)s.B * s.H * s.L;
-    const int64_t ro = row_offset(s, n, h, row_ok ? t : 0);
-    // Delta of both branches: each thread sums its half of the row, the halves meet in shared memory
-    float DL = 0.f, DS = 0.f, lseL2 = 0.f, lseS2 = 0.f;
-    {
-      float aL = 0.f, aS = 0.f;
-      if (row_valid) {
-#pragma unroll
-        for (int c = 0; c < OC; c += 8) {
-          const int64_t off = ro + half * OC + c;
-          const uint4 gv = *reinterpret_cast<const uint4 *>(dout + off);
-          const uint4 lv = *reinterpret_cast<const uint4 *>(out_lt + off);
-          const uint4 sv4 = *reinterpret_cast<const uint4 *>(out_st + off);
-          const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, lw[4] = {lv.x, lv.y, lv.z, lv.w},
-                         sw[4] = {sv4.x, sv4.y, sv4.z, sv4.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float g0 = __uint_as_float(gw[e] << 16), g1 = __uint_as_float(gw[e] & 0xffff0000u);
-            aL = fmaf(g0, __uint_as_float(lw[e] << 16), aL);
-            aL = fmaf(g1, __uint_as_float(lw[e] & 0xffff0000u), aL);
-            aS = fmaf(g0, __uint_as_float(sw[e] << 16), aS);
-            aS = fmaf(g1, __uint_as_float(sw[e] & 0xffff0000u), aS);
-          }
-        }
-        lseL2 = lse[(int64_t)u * s.L + t] * kLog2e;
-        lseS2 = lse[BHL + (int64_t)u * s.L + t] * kLog2e;
-      }
-      xch[half][r] = make_float2(aL, aS);
-      named_bar_sync(1 + quarter, 64);
-      const float2 o0 = xch[0][r], o1 = xch[1][r];  // fixed order: both threads get the same sums
-      DL = o0.x + o1.x;
-      DS = o0.y + o1.y;
-    }
-    // the branch weights ride in the exponent: P' = alpha P_lt = exp2(s - (lse - log2 alpha))
-    const float nlL = -(lseL2 - log2f(alpha)), nlS = -(lseS2 - log2f(beta));
-    if (half == 0 && t < Lpad) {
-      // The record the dK/dV kernel streams, laid out for two queries per instruction: per pair
-      // of rows {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)}; zeros for rows that do not exist.
-      float *rec = reinterpret_cast<float *>(qstats) + ((int64_t)u * Lpad + (t & ~1)) * 4 + (t & 1);
-      rec[0] = row_valid ? nlL : 0.f;
-      rec[2] = row_valid ? -DL : 0.f;
-      rec[4] = row_valid ? nlS : 0.f;
-      rec[6] = row_valid ? -DS : 0.f;
+    // this row's record from the pre-pass: nl = -(lse * log2e - log2 weight), nD = -Delta
+    float nlL = 0.f, nlS = 0.f, nDL = 0.f, nDS = 0.f;
+    if (row_valid) {
+      const float *rec = reinterpret_cast<const float *>(qstats) + ((int64_t)u * Lpad + (t & ~1)) * 4 + (t & 1);
+      nlL = rec[0];
+      nDL = rec[2];
+      nlS = rec[4];
+      nDS = rec[6];
     }
     float2 dalL = make_float2(0.f, 0.f), dalS = make_float2(0.f, 0.f);  // sums of P' dP per branch
     bool ds_zero = false;
@@ -311,13 +336,13 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
 #pragma unroll
             for (int c = 0; c < 8; ++c) dw[c] = 0u;
           } else if (!full) {
-            dq_tile<true, true, false>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
+            dq_tile<true, true, false>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
           } else if (anyL && anyS) {
-            dq_tile<true, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
+            dq_tile<true, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
           } else if (anyL) {
-            dq_tile<true, false, true>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
+            dq_tile<true, false, true>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
           } else {
-            dq_tile<false, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, -DL, -DS, dalL, dalS, dw);
+            dq_tile<false, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
           }
           if (q == 0 && i >= 1) {  // the dS columns are free once dQ += dS K of tile i-1 has completed
             mbar_wait(b_done, (i - 1) & 1, &abort_flag, 208);
@@ -722,10 +747,16 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
       cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   {
+    LaunchScope ls(K_BWD_PREP, st);
+    const int Lpad = nT * 64, rpb = 256 / (D / 8);
+    const unsigned gp = (unsigned)(s.B * s.H) * (unsigned)((Lpad + rpb - 1) / rpb);
+    bwd_prep_kernel<D><<<gp, 256, 0, st>>>(s, gate, seq_lens, (const bf *)out_lt, (const bf *)out_st, lse,
+                                          (const bf *)dout, ws.qstats, Lpad);
+  }
+  {
     LaunchScope ls(K_BWD_DQ_TC, st);
     bwd_dq_tc_kernel<D><<<grid, kBwdThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, idx,
-                                                           (const bf *)out_lt, (const bf *)out_st, lse,
-                                                           (const bf *)dout, tdq, ws.qstats, ws.dalpha,
+                                                           tdq, ws.qstats, ws.dalpha,
                                                            ws.status, nT);
   }
   {

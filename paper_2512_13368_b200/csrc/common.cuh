@@ -39,7 +39,7 @@ extern unsigned long long g_launches;  // host-side launch counter
 // Kernel identifiers reported by the optional per-launch event profile.
 enum KernelId {
   K_SUMMARY = 0, K_SCORE_SELECT, K_FWD_SIMT, K_BWD_DQ_SIMT, K_BWD_DKDV_SIMT, K_GATE_GRAD,
-  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_COUNT
+  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_BWD_PREP, K_COUNT
 };
 void prof_mark(int id, int phase, cudaStream_t st);  // no-op unless a profile is running
 
