@@ -35,15 +35,14 @@ namespace tc {
 namespace {
 
 constexpr int kBwdThreads = 288;
+// dK/dV kernel: warps 0..7 compute; 8 loader, 9 first-stage issuer, 10 second-stage issuer, 11 spare
+constexpr int kKvThreads = 384;
+constexpr int kProducerRegs = 32, kKvComputeRegs = 104;  // 256 * 104 + 128 * 32 = 384 * 80
 constexpr int kComputeWarps = 8;
 constexpr int kDqStages = 4;
-constexpr int kKvStages = 3;
+constexpr int kKvStages = 2;
 constexpr uint32_t kBwdTmemCols = 256;
 constexpr int kStatBytes = 64 * 16;  // one 64-query tile of row records
-// The dK/dV kernel lets S^T(i+1) overwrite the columns W^T(i) was read from.  With this switch
-// off it waits for the products that read them to complete before it issues the overwriting
-// ones; with it on it relies on the tensor pipe executing one thread's MMAs in issue order.
-constexpr bool kTrustMmaIssueOrder = false;
 
 __device__ __forceinline__ bool bit(uint32_t w, int c) { return (w >> c) & 1u; }
 
@@ -458,7 +457,7 @@ __device__ __forceinline__ void dkdv_tile(const float (&sv)[16], const float (&d
 }
 
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
+__global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
     const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ idx,
@@ -469,8 +468,8 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
   constexpr int OC = D / 2;
   constexpr int kStageBytes = 2 * C::kSmallBytes + kStatBytes;  // Q, dO, row records
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done, s_empty
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int nvis_s;
@@ -491,7 +490,9 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
   uint8_t *k_tile = tiles;
   uint8_t *v_tile = k_tile + C::kBigBytes;
   uint8_t *qg_tiles = v_tile + C::kBigBytes;  // [stage][Q, dO, row records]
-  uint8_t *meta = qg_tiles + STAGES * kStageBytes;
+  uint8_t *w_tile = qg_tiles + STAGES * kStageBytes;  // W^T  [128 keys][64 queries] bf16, 128-byte swizzle
+  uint8_t *ds_tile = w_tile + 128 * 128;               // dS^T, same layout
+  uint8_t *meta = ds_tile + 128 * 128;
   uint32_t *invw = reinterpret_cast<uint32_t *>(meta);  // [8][nT] bytes: per key block, per query tile
   uint8_t *invb = meta;
   uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
@@ -500,6 +501,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
   const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 2]), b_done = smem_u32(&bars[2 * STAGES + 3]);
+  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 4]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -515,6 +517,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
     mbar_init(b_sfull, 1);
     mbar_init(b_tfull, kComputeWarps);
     mbar_init(b_done, 1);
+    mbar_init(b_sempty, kComputeWarps);
     mbar_fence_init();
   }
   if (warp == 0) {
@@ -522,11 +525,11 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
     tmem_alloc(smem_u32(&tmem_slot), kBwdTmemCols);
     tmem_relinquish();
   }
-  for (int i = tid; i < (8 * nT + 3) / 4; i += kBwdThreads) invw[i] = 0u;
+  for (int i = tid; i < (8 * nT + 3) / 4; i += kKvThreads) invw[i] = 0u;
   __syncthreads();
   {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
     const int qb0 = kt * G, nq = s.M - qb0;
-    for (int i = tid; i < nq * s.topk; i += kBwdThreads) {
+    for (int i = tid; i < nq * s.topk; i += kKvThreads) {
       const int qb = qb0 + i / s.topk;
       const int blk = idx[((int64_t)u * s.M + qb) * s.topk + (i % s.topk)];
       if (blk >= qb0 && blk < qb0 + G && blk <= qb) {
@@ -564,12 +567,17 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
   const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_dv = tmem_base + 128,
                  tmem_dk = tmem_base + 192;
 
-  if (warp == kComputeWarps) {
-    if (lane == 0 && nvis > 0) {
-      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
-      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
-      auto load_stage = [&](int j) {
+  if (warp >= kComputeWarps) {
+    // ===================== three single-thread roles, one warp each =====================
+    setmaxnreg_dec<kProducerRegs>();
+    if (warp == kComputeWarps && lane == 0 && nvis > 0) {
+      // ---- loader: K, V once; Q, dO tiles and their row records up to STAGES ahead ----
+      mbar_expect_tx(b_res, 2 * C::kBigBytes);
+      tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
+      tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
+      for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
+        if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 214);
         const uint32_t bar = b_full + 8 * sj;
         uint8_t *qt_ = qg_tiles + sj * kStageBytes;
         mbar_expect_tx(bar, kStageBytes);
@@ -577,39 +585,16 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
         tma_load_4d(smem_u32(qt_ + C::kSmallBytes), &tmg, bar, 0, (int)list[j] * 64, h, n);
         bulk_load(smem_u32(qt_ + 2 * C::kSmallBytes), qstats + (int64_t)u * Lpad + (int64_t)list[j] * 64,
                   kStatBytes, bar);
-      };
-      int acc = 0;
-      // dV += W^T dO, dK += dS^T Q of tile j; the 16 queries of K step k sit in columns
-      // 32 * (k / 2) + 8 * (k % 2) of the S^T / dP^T regions
-      auto second_stage = [&](int j) {
-        uint8_t *q_tile = qg_tiles + (j % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
-        const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-        const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_bf16_ts(tmem_dv, tmem_s + 32 * (k >> 1) + 8 * (k & 1), dgm + k * C::kKStep, idesc_o, (acc | k) != 0);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_bf16_ts(tmem_dk, tmem_dp + 32 * (k >> 1) + 8 * (k & 1), dqm + k * C::kKStep, idesc_o, (acc | k) != 0);
-        acc = 1;
-        umma_commit(b_empty + 8 * (j % STAGES));
-        umma_commit(b_done);
-      };
-      mbar_expect_tx(b_res, 2 * C::kBigBytes);
-      tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
-      tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
-      for (int j = 0; j < min(STAGES, nvis); ++j) load_stage(j);
+      }
+    } else if (warp == kComputeWarps + 1 && lane == 0 && nvis > 0) {
+      // ---- S^T = K Q^T and dP^T = V dO^T of tile i once the compute warps hold tile i-1's ----
+      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
       const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
       const uint64_t dvd = smem_desc(smem_u32(v_tile), 16, C::kAtomBytes, C::kSwizzle);
+      mbar_wait(b_res, 0, &abort_flag, 210);
       for (int i = 0; i < nvis; ++i) {
-        if (i == 0) mbar_wait(b_res, 0, &abort_flag, 210);
-        if (i >= 1) {
-          mbar_wait(b_tfull, (i - 1) & 1, &abort_flag, 211);
-          tc_fence_after();
-          second_stage(i - 1);
-          if (!kTrustMmaIssueOrder) mbar_wait(b_done, (i - 1) & 1, &abort_flag, 212);
-        }
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 213);
+        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 212);
         tc_fence_after();
         uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
         const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
@@ -619,20 +604,32 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
         umma_commit(b_sfull);
-        // tile i + STAGES - 1 goes into the stage tile i - 1 occupied
-        const int j = i + STAGES - 1;
-        if (i >= 1 && j < nvis) {
-          mbar_wait(b_empty + 8 * ((i - 1) % STAGES), ((i - 1) / STAGES) & 1, &abort_flag, 214);
-          load_stage(j);
-        }
       }
-      mbar_wait(b_tfull, (nvis - 1) & 1, &abort_flag, 215);
-      tc_fence_after();
-      second_stage(nvis - 1);
+    } else if (warp == kComputeWarps + 2 && lane == 0 && nvis > 0) {
+      // ---- dV += W^T dO, dK += dS^T Q of tile i (W^T, dS^T from shared memory, K-major) ----
+      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
+      const uint64_t dwd = smem_desc(smem_u32(w_tile), 16, 1024, 2u);
+      const uint64_t dsd = smem_desc(smem_u32(ds_tile), 16, 1024, 2u);
+      for (int i = 0; i < nvis; ++i) {
+        uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
+        const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 215);
+        mbar_wait(b_tfull, i & 1, &abort_flag, 211);
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < 4; ++k) umma_bf16(tmem_dv, dwd + 2 * k, dgm + k * C::kKStep, idesc_o, (i | k) != 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) umma_bf16(tmem_dk, dsd + 2 * k, dqm + k * C::kKStep, idesc_o, (i | k) != 0);
+        umma_commit(b_done);
+        umma_commit(b_empty + 8 * (i % STAGES));  // S^T(i), dP^T(i) completed before the compute warps read them
+      }
     }
   } else {
+    setmaxnreg_inc<kKvComputeRegs>();
     const int quarter = warp & 3, half = warp >> 2;
     const int r = quarter * 32 + lane, p = key0 + r, g = r / s.Bk;
+    bool w_zero = false;  // this thread's part of the W^T / dS^T tiles holds zeros
     const bool row_ok = p < s.L, row_valid = row_ok && p >= pad0;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float sc2 = s.scale * kLog2e;
@@ -653,33 +650,53 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkdv_tc_kernel(
       mbar_wait(b_sfull, i & 1, &abort_flag, 217);
       __syncwarp();
       tc_fence_after();
-      // 16 query columns at a time; W^T / dS^T always written: the fresh S^T / dP^T erased
-      // whatever this thread had left in those columns
+      const bool mine = anyL || anyS;
       const float4 *stt =
           reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes) + half * 32;
+      if (mine || !w_zero) {
+        // two passes of 16 query columns (a rolled loop: one copy of each code path)
 #pragma unroll 1
-      for (int q = 0; q < 2; ++q) {
-        uint32_t ww[8], dw[8];
-        if (anyL || anyS) {
+        for (int q = 0; q < 2; ++q) {
+          uint32_t ww[8], dw[8];
           float sv[16], dp[16];
-          tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
-          tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
-          tmem_wait_ld();
-          const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
-          const float4 *sq = stt + q * 16;  // 8 pairs x 2 float4
-          if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          else dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-        } else {
+          if (mine) {
+            tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
+            tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
+            tmem_wait_ld();
+          }
+          if (q == 1) warp_arrive(b_sempty, lane);  // S^T, dP^T of this tile are in registers
+          if (mine) {
+            const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
+            const float4 *sq = stt + q * 16;  // 8 pairs x 2 float4
+            if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
+            else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+            else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+            else dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          } else {
 #pragma unroll
-          for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }
+            for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }
+          }
+          if (q == 0 && i >= 1) {  // the W^T / dS^T tiles are free once the products of tile i-1 completed
+            mbar_wait(b_done, (i - 1) & 1, &abort_flag, 219);
+            __syncwarp();
+          }
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            store_row_sw128(w_tile, r, half * 4 + q * 2 + ch,
+                            make_uint4(ww[ch * 4], ww[ch * 4 + 1], ww[ch * 4 + 2], ww[ch * 4 + 3]));
+            store_row_sw128(ds_tile, r, half * 4 + q * 2 + ch,
+                            make_uint4(dw[ch * 4], dw[ch * 4 + 1], dw[ch * 4 + 2], dw[ch * 4 + 3]));
+          }
         }
-        tmem_st8u(tmem_s + lane_off + half * 32 + q * 8, ww);
-        tmem_st8u(tmem_dp + lane_off + half * 32 + q * 8, dw);
+        w_zero = !mine;
+      } else {
+        warp_arrive(b_sempty, lane);
+        if (i >= 1) {  // keep in step with the barrier (a parity wait tells only two phases apart)
+          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 220);
+          __syncwarp();
+        }
       }
-      tmem_wait_st();
-      tc_fence_before();
+      fence_async_smem();
       warp_arrive(b_tfull, lane);
     }
 
@@ -742,7 +759,7 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
   const size_t smem_dq = 1024 + 2 * C::kBigBytes + kDqStages * 2 * C::kSmallBytes + meta_bytes(nT);
   const size_t smem_kv =
-      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT);
+      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + 2 * 128 * 128 + meta_bytes(nT);
   if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
@@ -761,7 +778,7 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
-    bwd_dkdv_tc_kernel<D><<<grid, kBwdThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, idx,
+    bwd_dkdv_tc_kernel<D><<<grid, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, idx,
                                                              ws.qstats, tdk, tdv, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;

@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
 constexpr int kFastThreads = 256;
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
+__global__ void __launch_bounds__(kFastThreads, 5) score_select_fast_kernel(
     Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
     const float *__restrict__ knorm, const int32_t *__restrict__ klive,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
