@@ -225,20 +225,26 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   if (warp >= kSoftmaxWarps) {
     // ===================== three single-thread roles, one warp each =====================
     setmaxnreg_dec<kProducerRegs>();
-    if (warp == kSoftmaxWarps && lane == 0 && nI > 0) {
+    if (warp == kSoftmaxWarps && nI > 0) {
       // ---- loader: K/V tiles, up to STAGES ahead of their consumers ----
-      mbar_expect_tx(b_res, C::kBigBytes);
-      tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+      if (elect_one()) {
+        mbar_expect_tx(b_res, C::kBigBytes);
+        tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+      }
       for (int j = 0; j < nI; ++j) {
         const int sj = j % STAGES;
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 105);
         const uint32_t bar = b_full + 8 * sj;
-        uint8_t *kt = kv_tiles + sj * 2 * C::kSmallBytes;
-        mbar_expect_tx(bar, 2 * C::kSmallBytes);
-        tma_load_4d(smem_u32(kt), &tmk, bar, 0, (int)items[j] * 64, h, n);
-        tma_load_4d(smem_u32(kt + C::kSmallBytes), &tmv, bar, 0, (int)items[j] * 64, h, n);
+        const uint32_t kt = smem_u32(kv_tiles + sj * 2 * C::kSmallBytes);
+        const int row = (int)items[j] * 64;
+        if (elect_one()) {
+          mbar_expect_tx(bar, 2 * C::kSmallBytes);
+          tma_load_4d(kt, &tmk, bar, 0, row, h, n);
+          tma_load_4d(kt + C::kSmallBytes, &tmv, bar, 0, row, h, n);
+        }
+        __syncwarp();
       }
-    } else if (warp == kSoftmaxWarps + 1 && lane == 0 && nI > 0) {
+    } else if (warp == kSoftmaxWarps + 1 && nI > 0) {
       // ---- S(i) = Q K^T into S buffer i % 2 once the softmax warps hold S(i-2) in registers ----
       constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
       const uint64_t dq = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
@@ -247,28 +253,35 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 102);
         if (i >= 2) mbar_wait(b_sempty + 8 * (i & 1), ((i - 2) >> 1) & 1, &abort_flag, 103);
         tc_fence_after();
-        uint8_t *k_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes;
-        const uint64_t dk = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dk =
+            smem_desc(smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes), 16, C::kAtomBytes, C::kSwizzle);
         const uint32_t ts = tmem_s + 64 * (i & 1);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) umma_bf16(ts, dq + 2 * k, dk + 2 * k, idesc_s, k > 0);
-        umma_commit(b_sfull + 8 * (i & 1));
+          for (int k = 0; k < D / 16; ++k) umma_bf16(ts, dq + 2 * k, dk + 2 * k, idesc_s, k > 0);
+          umma_commit(b_sfull + 8 * (i & 1));
+        }
+        __syncwarp();
       }
-    } else if (warp == kSoftmaxWarps + 2 && lane == 0 && nI > 0) {
+    } else if (warp == kSoftmaxWarps + 2 && nI > 0) {
       // ---- O += P(i) V once the probabilities of item i are in tensor memory ----
       constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
       for (int i = 0; i < nI; ++i) {
-        uint8_t *v_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes;
-        const uint64_t dv = smem_desc(smem_u32(v_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dv = smem_desc(smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes),
+                                      C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
         const uint32_t tp = tmem_p + 32 * (i & 1);
-        const int first = (i == 0 || i == nL) ? 0 : 1;  // a phase starts the accumulator afresh
+        const uint32_t first = (i == 0 || i == nL) ? 0u : 1u;  // a phase starts the accumulator afresh
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 106);
         mbar_wait(b_tfull + 8 * (i & 1), (i >> 1) & 1, &abort_flag, 104);
         tc_fence_after();
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma_bf16_ts(tmem_o, tp + 8 * k, dv + k * C::kKStep, idesc_pv, (first | k) != 0);
-        umma_commit(b_done + 8 * (i & 1));
-        umma_commit(b_empty + 8 * (i % STAGES));  // S(i) completed before the softmax warps read it
+          for (int k = 0; k < 4; ++k)
+            umma_bf16_ts(tmem_o, tp + 8 * k, dv + k * C::kKStep, idesc_pv, (first | (uint32_t)k) != 0u);
+          umma_commit(b_done + 8 * (i & 1));
+          umma_commit(b_empty + 8 * (i % STAGES));  // S(i) completed before the softmax warps read it
+        }
+        __syncwarp();
       }
     }
   } else {

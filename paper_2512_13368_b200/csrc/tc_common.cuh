@@ -77,6 +77,20 @@ __device__ __forceinline__ void setmaxnreg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
+// True in exactly one lane of a converged warp.  The single-thread roles keep their whole warp
+// converged (every lane waits on the barriers and computes the uniform addresses) and put only the
+// asynchronous instructions under this predicate, so that descriptors and addresses can live in
+// uniform registers.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // ---- TMA: 4-D tiled load global -> shared, completion on an mbarrier ----------------------
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
                                             int c0, int c1, int c2, int c3) {
