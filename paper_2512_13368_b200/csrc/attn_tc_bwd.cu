@@ -34,8 +34,7 @@ namespace blossom {
 namespace tc {
 namespace {
 
-constexpr int kBwdThreads = 288;
-// dK/dV kernel: warps 0..7 compute; 8 loader, 9 first-stage issuer, 10 second-stage issuer, 11 spare
+// warps 0..7 compute; 8 loader, 9 first-stage issuer, 10 second-stage issuer, 11 spare
 constexpr int kKvThreads = 384;
 constexpr int kProducerRegs = 32, kKvComputeRegs = 104;  // 256 * 104 + 128 * 32 = 384 * 80
 constexpr int kComputeWarps = 8;
@@ -147,7 +146,7 @@ __device__ __forceinline__ void dq_tile(const float (&sv)[16], const float (&dp)
 }
 
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
+__global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
@@ -223,64 +222,72 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_tc_kernel(
   const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_ds = tmem_base + 128,
                  tmem_dq = tmem_base + 160;
 
-  if (warp == kComputeWarps) {
-    if (lane == 0 && nvis > 0) {
-      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
-      constexpr uint32_t idesc_dq = instr_desc(128, D, 0, 1);
-      auto load_stage = [&](int j) {
+  if (warp >= kComputeWarps) {
+    // ============ three single-thread roles, one converged warp each ============
+    setmaxnreg_dec<kProducerRegs>();
+    if (warp == kComputeWarps && nvis > 0) {
+      // ---- loader: Q, dO once; K/V tiles up to STAGES ahead of their consumers ----
+      if (elect_one()) {
+        mbar_expect_tx(b_res, 2 * C::kBigBytes);
+        tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+        tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
+      }
+      for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
+        if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 205);
         const uint32_t bar = b_full + 8 * sj;
-        uint8_t *kt = kv_tiles + sj * 2 * C::kSmallBytes;
-        mbar_expect_tx(bar, 2 * C::kSmallBytes);
-        tma_load_4d(smem_u32(kt), &tmk, bar, 0, (int)list[j] * 64, h, n);
-        tma_load_4d(smem_u32(kt + C::kSmallBytes), &tmv, bar, 0, (int)list[j] * 64, h, n);
-      };
-      int acc = 0;
-      auto second_stage = [&](int j) {  // dQ += dS K of tile j (dS from tensor memory, K MN-major)
-        uint8_t *k_tile = kv_tiles + (j % STAGES) * 2 * C::kSmallBytes;
-        const uint64_t dkm = smem_desc(smem_u32(k_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_bf16_ts(tmem_dq, tmem_ds + 8 * k, dkm + k * C::kKStep, idesc_dq, (acc | k) != 0);
-        acc = 1;
-        umma_commit(b_done);
-        umma_commit(b_empty + 8 * (j % STAGES));
-      };
-      mbar_expect_tx(b_res, 2 * C::kBigBytes);
-      tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
-      tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
-      for (int j = 0; j < min(STAGES - 1, nvis); ++j) load_stage(j);
+        const uint32_t kt = smem_u32(kv_tiles + sj * 2 * C::kSmallBytes);
+        const int row = (int)list[j] * 64;
+        if (elect_one()) {
+          mbar_expect_tx(bar, 2 * C::kSmallBytes);
+          tma_load_4d(kt, &tmk, bar, 0, row, h, n);
+          tma_load_4d(kt + C::kSmallBytes, &tmv, bar, 0, row, h, n);
+        }
+        __syncwarp();
+      }
+    } else if (warp == kComputeWarps + 1 && nvis > 0) {
+      // ---- S = Q K^T and dP = dO V^T of tile i once the compute warps hold tile i-1's ----
+      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
       const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
       const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
+      mbar_wait(b_res, 0, &abort_flag, 201);
       for (int i = 0; i < nvis; ++i) {
-        if (i == 0) mbar_wait(b_res, 0, &abort_flag, 201);
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 202);
         if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 203);
         tc_fence_after();
-        uint8_t *k_tile = kv_tiles + (i % STAGES) * 2 * C::kSmallBytes, *v_tile = k_tile + C::kSmallBytes;
-        const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
-        const uint64_t dvd = smem_desc(smem_u32(v_tile), 16, C::kAtomBytes, C::kSwizzle);
+        const uint32_t kt = smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes);
+        const uint64_t dkd = smem_desc(kt, 16, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dvd = smem_desc(kt + C::kSmallBytes, 16, C::kAtomBytes, C::kSwizzle);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dqd + 2 * k, dkd + 2 * k, idesc_s, k > 0);
+          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dqd + 2 * k, dkd + 2 * k, idesc_s, k > 0);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dgd + 2 * k, dvd + 2 * k, idesc_s, k > 0);
-        umma_commit(b_sfull);
-        if (i >= 1) {
-          mbar_wait(b_tfull, (i - 1) & 1, &abort_flag, 204);
-          tc_fence_after();
-          second_stage(i - 1);
-          const int j = i + STAGES - 2;
-          if (j < nvis) {
-            if (i >= 2) mbar_wait(b_empty + 8 * ((i - 2) % STAGES), ((i - 2) / STAGES) & 1, &abort_flag, 205);
-            load_stage(j);
-          }
+          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dgd + 2 * k, dvd + 2 * k, idesc_s, k > 0);
+          umma_commit(b_sfull);
         }
+        __syncwarp();
       }
-      mbar_wait(b_tfull, (nvis - 1) & 1, &abort_flag, 206);
-      tc_fence_after();
-      second_stage(nvis - 1);
+    } else if (warp == kComputeWarps + 2 && nvis > 0) {
+      // ---- dQ += dS K of tile i (dS from tensor memory, K MN-major) ----
+      constexpr uint32_t idesc_dq = instr_desc(128, D, 0, 1);
+      for (int i = 0; i < nvis; ++i) {
+        const uint64_t dkm = smem_desc(smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes), C::kSmallBytes,
+                                       C::kAtomBytes, C::kSwizzle);
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 206);
+        mbar_wait(b_tfull, i & 1, &abort_flag, 204);
+        tc_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16_ts(tmem_dq, tmem_ds + 8 * k, dkm + k * C::kKStep, idesc_dq, (i | k) != 0);
+          umma_commit(b_done);
+          umma_commit(b_empty + 8 * (i % STAGES));  // S(i), dP(i) completed before the compute warps read them
+        }
+        __syncwarp();
+      }
     }
   } else {
+    setmaxnreg_inc<kKvComputeRegs>();
     const int quarter = warp & 3, half = warp >> 2;
     const int r = quarter * 32 + lane, t = row0 + r, g = r / s.Bk;
     const bool row_ok = t < s.L, row_valid = row_ok && t >= pad0;
@@ -570,23 +577,28 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   if (warp >= kComputeWarps) {
     // ===================== three single-thread roles, one warp each =====================
     setmaxnreg_dec<kProducerRegs>();
-    if (warp == kComputeWarps && lane == 0 && nvis > 0) {
+    if (warp == kComputeWarps && nvis > 0) {
       // ---- loader: K, V once; Q, dO tiles and their row records up to STAGES ahead ----
-      mbar_expect_tx(b_res, 2 * C::kBigBytes);
-      tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
-      tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
+      if (elect_one()) {
+        mbar_expect_tx(b_res, 2 * C::kBigBytes);
+        tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
+        tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
+      }
       for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 214);
         const uint32_t bar = b_full + 8 * sj;
-        uint8_t *qt_ = qg_tiles + sj * kStageBytes;
-        mbar_expect_tx(bar, kStageBytes);
-        tma_load_4d(smem_u32(qt_), &tmq, bar, 0, (int)list[j] * 64, h, n);
-        tma_load_4d(smem_u32(qt_ + C::kSmallBytes), &tmg, bar, 0, (int)list[j] * 64, h, n);
-        bulk_load(smem_u32(qt_ + 2 * C::kSmallBytes), qstats + (int64_t)u * Lpad + (int64_t)list[j] * 64,
-                  kStatBytes, bar);
+        const uint32_t qt_ = smem_u32(qg_tiles + sj * kStageBytes);
+        const int row = (int)list[j] * 64;
+        if (elect_one()) {
+          mbar_expect_tx(bar, kStageBytes);
+          tma_load_4d(qt_, &tmq, bar, 0, row, h, n);
+          tma_load_4d(qt_ + C::kSmallBytes, &tmg, bar, 0, row, h, n);
+          bulk_load(qt_ + 2 * C::kSmallBytes, qstats + (int64_t)u * Lpad + row, kStatBytes, bar);
+        }
+        __syncwarp();
       }
-    } else if (warp == kComputeWarps + 1 && lane == 0 && nvis > 0) {
+    } else if (warp == kComputeWarps + 1 && nvis > 0) {
       // ---- S^T = K Q^T and dP^T = V dO^T of tile i once the compute warps hold tile i-1's ----
       constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
       const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
@@ -599,13 +611,16 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
         uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
         const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
         const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
+          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
-        umma_commit(b_sfull);
+          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
+          umma_commit(b_sfull);
+        }
+        __syncwarp();
       }
-    } else if (warp == kComputeWarps + 2 && lane == 0 && nvis > 0) {
+    } else if (warp == kComputeWarps + 2 && nvis > 0) {
       // ---- dV += W^T dO, dK += dS^T Q of tile i (W^T, dS^T from shared memory, K-major) ----
       constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
       const uint64_t dwd = smem_desc(smem_u32(w_tile), 16, 1024, 2u);
@@ -617,12 +632,15 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 215);
         mbar_wait(b_tfull, i & 1, &abort_flag, 211);
         tc_fence_after();
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma_bf16(tmem_dv, dwd + 2 * k, dgm + k * C::kKStep, idesc_o, (i | k) != 0);
+          for (int k = 0; k < 4; ++k) umma_bf16(tmem_dv, dwd + 2 * k, dgm + k * C::kKStep, idesc_o, (i | k) != 0);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma_bf16(tmem_dk, dsd + 2 * k, dqm + k * C::kKStep, idesc_o, (i | k) != 0);
-        umma_commit(b_done);
-        umma_commit(b_empty + 8 * (i % STAGES));  // S^T(i), dP^T(i) completed before the compute warps read them
+          for (int k = 0; k < 4; ++k) umma_bf16(tmem_dk, dsd + 2 * k, dqm + k * C::kKStep, idesc_o, (i | k) != 0);
+          umma_commit(b_done);
+          umma_commit(b_empty + 8 * (i % STAGES));  // S^T(i), dP^T(i) completed before the compute warps read them
+        }
+        __syncwarp();
       }
     }
   } else {
@@ -772,7 +790,7 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   }
   {
     LaunchScope ls(K_BWD_DQ_TC, st);
-    bwd_dq_tc_kernel<D><<<grid, kBwdThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, idx,
+    bwd_dq_tc_kernel<D><<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, idx,
                                                            tdq, ws.qstats, ws.dalpha,
                                                            ws.status, nT);
   }
