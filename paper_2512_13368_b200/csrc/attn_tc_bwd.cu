@@ -1,32 +1,34 @@
 // Tensor-core backward of the fused two-branch attention (bf16 storage, fp32 accumulate): a small
-// pre-pass and two main kernels, all deterministic (no atomics on any gradient), both recomputing the probabilities
-// from the saved log-sum-exps.
+// pre-pass and two main kernels, all deterministic (no atomics on any gradient); the main kernels
+// recompute the probabilities from the saved log-sum-exps.
 //
-// CTA = 288 threads: warps 0..7 compute, warp 8 is the producer (one lane issues every TMA load
-// and every tcgen05.mma).  A CTA owns a resident 128-row tile (rows = TMEM lanes) and streams
-// 64-row tiles past it.  Row r of the 128 is shared by two compute threads: warp w and warp w + 4
-// both address TMEM lane quarter w % 4; the first takes columns 0..31 of a 64-column tile, the
-// second columns 32..63.  The bf16 operands of the second-stage products (dS, and in the dK/dV
-// kernel W^T and dS^T) are written to tensor memory and read from there by the MMA.
+//  pre-pass  Delta_x = rowsum(dO o O_x) of both branches from coalesced reads, and the per-row
+//            records the main kernels read: per pair of rows {nl_lt(2), -Delta_lt(2)}
+//            {nl_st(2), -Delta_st(2)}, nl = -(lse*log2e - log2 weight): the branch weights alpha,
+//            beta ride in the exponent, alpha P_lt = exp2(s*log2e + nl_lt).
+//
+// Main kernels: CTA = 384 threads.  Warps 0..7 compute; warps 8, 9, 10 stay converged and one
+// elected lane of each issues the TMA loads, the first-stage MMAs and the second-stage MMAs;
+// registers move from those warps to the compute warps (setmaxnreg).  A CTA owns a resident
+// 128-row tile (rows = TMEM lanes) and streams 64-row tiles past it.  Row r of the 128 is shared by
+// two compute threads: warp w and warp w + 4 both address TMEM lane quarter w % 4; the first takes
+// columns 0..31 of a 64-column tile, the second columns 32..63.  The tile arithmetic runs in
+// 16-column passes, two columns per FMA / ADD / MUL (packed f32x2); outputs are staged in shared
+// memory and written with whole-line TMA stores.
 //
 //  dQ     resident Q, dO (128 queries); streams K, V 64-key tiles (same walk as the forward).
 //         Tensor memory: S [0,64), dP [64,128), dS [128,160) (bf16 pairs), dQ [160,160+D).
-//         S = Q K^T, dP = dO V^T; P_x = exp(S - lse_x);
-//         dS = alpha P_lt (dP - Delta_lt) + beta P_st (dP - Delta_st), Delta_x = rowsum(dO o O_x)
-//         (one tile for both branches, they share K); dQ += dS K.  The first-stage MMAs of tile
-//         i+1 run while the compute warps work on tile i.
-//         Row statistics come from the pre-pass kernel (coalesced reads of dO, O_lt, O_st):
-//         per pair of rows {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)},
-//         nl = -(lse*log2e - log2 weight) (the branch weights alpha, beta ride in the exponent:
-//         alpha P_lt = exp2(s*log2e + nl_lt)); the dK/dV kernel streams the same records.
-//         The tile arithmetic handles two columns per FMA / ADD / MUL (packed f32x2).
+//         S = Q K^T, dP = dO V^T; P'_x = weight_x exp(S - lse_x);
+//         dS = P'_lt (dP - Delta_lt) + P'_st (dP - Delta_st) (one tile for both branches, they share
+//         K), written to tensor memory and read from there by dQ += dS K.  The first-stage MMAs of
+//         tile i+1 run while the compute warps work on tile i.
 //         d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
 //  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
-//         records) that selected one of its key blocks or whose window reaches them.
-//         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D); each thread
-//         overwrites the first half of its own S^T / dP^T columns with W^T / dS^T.
-//         S^T = K Q^T, dP^T = V dO^T; thread = key row; W^T = alpha P_lt + beta P_st and
-//         dS^T as above; dV += W^T dO, dK += dS^T Q.
+//         records, by bulk copy) that selected one of its key blocks or whose window reaches them.
+//         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D): no room for
+//         the bf16 operands, so W^T = P'_lt + P'_st and dS^T go through two 128-byte-swizzled
+//         shared-memory tiles.  S^T = K Q^T, dP^T = V dO^T; thread = key row;
+//         dV += W^T dO, dK += dS^T Q.  As in dQ, tile i+1's first stage overlaps tile i's arithmetic.
 // Every wait is bounded (tc_common.cuh).
 #include "tc_common.cuh"
 

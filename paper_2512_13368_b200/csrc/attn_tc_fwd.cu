@@ -7,9 +7,9 @@
 // accumulator afresh.  A tile that belongs to both branches is visited once per phase.
 //
 // CTA = 256 threads.  Warps 0..3 are softmax warps (thread = query row = TMEM lane: no exchange
-// between threads in the loop).  Warp 4 lane 0 loads K/V tiles (TMA), warp 5 lane 0 issues
-// S = Q K^T, warp 6 lane 0 issues O += P V with P read from tensor memory.  Registers move from
-// those single-thread warps to the softmax warps (setmaxnreg).
+// between threads in the loop).  Warps 4, 5, 6 stay converged and one elected lane of each loads
+// K/V tiles (TMA), issues S = Q K^T, and issues O += P V with P read from tensor memory.
+// Registers move from those warps to the softmax warps (setmaxnreg).
 //
 // Tensor memory (256 columns): S buffers [0,64) [64,128), probability buffers (bf16 pairs)
 // [128,160) [160,192), accumulator [192,192+D).  Item i uses S buffer and probability buffer
@@ -25,7 +25,8 @@
 // Every barrier that counts warp arrivals exists once per item parity: a warp can be one item
 // ahead of the slowest warp, never two.  Rows whose query block does not need a tile skip its
 // exponentials (warp-uniform) and contribute zero rows to P.
-// Epilogue: normalise, gate mix (Eq. 19), store out / out_lt / out_st / lse.
+// Epilogue: normalise, gate mix (Eq. 19), stage the rows in shared memory and write out / out_lt /
+// out_st with whole-line TMA stores; lse directly.
 // Every wait is bounded (tc_common.cuh).
 #include "tc_common.cuh"
 
