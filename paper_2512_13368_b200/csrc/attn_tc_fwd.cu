@@ -11,20 +11,23 @@
 // K/V tiles (TMA), issues S = Q K^T, and issues O += P V with P read from tensor memory.
 // Registers move from those warps to the softmax warps (setmaxnreg).
 //
-// Tensor memory (256 columns): S buffers [0,64) [64,128), probability buffers (bf16 pairs)
-// [128,160) [160,192), accumulator [192,192+D).  Item i uses S buffer and probability buffer
-// i % 2, so that S(i+1) is computed and O += P(i-1) V runs while the softmax warps work on item i:
+// Tensor memory (256 columns): three logits / probability buffers [0,64) [64,128) [128,192) and
+// the accumulator [192,192+D).  Item i uses buffer i % 3: S(i) = Q K^T lands there as fp32, each
+// softmax thread reads its row and writes the row's probabilities (bf16 pairs) over the first 32
+// columns of the same buffer, and O += P(i) V reads them from there.  A row's probabilities only
+// replace that row's own logits, so the softmax warps wait for one thing per item:
 //
 //   loader   : stage j <- K, V of item j once O += P V of item j - STAGES has completed
-//   S issuer : wait K(i) and "S(i-2) is in registers" -> S(i) -> commit s_full[i%2]
-//   softmax  : wait s_full -> tcgen05.ld 64 logits -> arrive s_empty -> online softmax of the row
-//              (maximum raised, and the accumulator rescaled, only when it grows by > 2^8)
-//              -> wait "O += P(i-2) V done" -> tcgen05.st P -> arrive t_full[i%2]
-//   PV issuer: wait t_full -> O += P(i) V -> commit done[i%2], release the stage
+//   S issuer : wait K(i) and "O += P(i-3) V done" (the buffer is free) -> S(i) -> commit s_full[i%3]
+//   softmax  : wait s_full -> tcgen05.ld 64 logits -> online softmax of the row (maximum raised,
+//              and the accumulator rescaled, only when it grows by > 2^8) -> tcgen05.st P over the
+//              logits -> arrive t_full[i%3]
+//   PV issuer: wait t_full -> O += P(i) V -> commit done[i%3], release the stage
 //
-// Every barrier that counts warp arrivals exists once per item parity: a warp can be one item
-// ahead of the slowest warp, never two.  Rows whose query block does not need a tile skip its
-// exponentials (warp-uniform) and contribute zero rows to P.
+// so S(i+1) and S(i+2) are computed, and O += P(i-1) V runs, while the softmax warps work on item
+// i.  A softmax warp cannot pass s_full(i+3) before every warp has arrived on t_full(i), so a
+// barrier never collects two arrivals of one warp in one phase.  Rows whose query block does not
+// need a tile skip its exponentials (warp-uniform) and write zero rows.
 // Epilogue: normalise, gate mix (Eq. 19), stage the rows in shared memory and write out / out_lt /
 // out_st with whole-line TMA stores; lse directly.
 // Every wait is bounded (tc_common.cuh).
@@ -116,9 +119,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   using C = Cfg<D>;
   constexpr int STAGES = kFwdStages;
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, then pairs by item parity: s_full, s_empty,
-  // t_full, done
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 9];
+  // barriers: full[STAGES], empty[STAGES], res, then one per buffer: s_full[3], t_full[3], done[3]
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 10];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int nvis_s, nL_s, nS_s;
@@ -146,8 +148,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]);
-  const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 1]), b_sempty = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 5]), b_done = smem_u32(&bars[2 * STAGES + 7]);
+  const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 1]), b_tfull = smem_u32(&bars[2 * STAGES + 4]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 7]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;  // an earlier CTA timed out: do not wait again
@@ -159,9 +161,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       mbar_init(b_empty + 8 * i, 1);
     }
     mbar_init(b_res, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 3; ++i) {
       mbar_init(b_sfull + 8 * i, 1);
-      mbar_init(b_sempty + 8 * i, kSoftmaxWarps);
       mbar_init(b_tfull + 8 * i, kSoftmaxWarps);
       mbar_init(b_done + 8 * i, 1);
     }
@@ -176,16 +177,52 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   __syncthreads();
   if (warp == 0) {  // items: the tiles of the long-term phase, then those of the short-term phase
     const int nv = nvis_s;
-    int count = 0, nl = 0;
-    for (int ph = 1; ph <= 2; ++ph) {
+    // Long-term items: the tiles both 64-row halves of the CTA need, then alternately a tile only
+    // rows 0..63 need and a tile only rows 64..127 need.  A softmax warp may run one item ahead
+    // of the slowest one, so with alternating items both pairs of warps have work at once.
+    const int G = 128 / s.Bk, gh = G / 2;
+    const unsigned lt = (1u << lane) - 1u;
+    int nA = 0, nB = 0, nC = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+      int cA = 0, cB = 0, cC = 0;
       for (int base = 0; base < nv; base += 32) {
         const int j = base + lane;
-        const bool on = j < nv && (lflags[j] & ph);
-        const unsigned bal = __ballot_sync(0xffffffffu, on);
-        if (on) items[count + __popc(bal & ((1u << lane) - 1u))] = list[j];
-        count += __popc(bal);
+        int c = 0;
+        if (j < nv && (lflags[j] & 1)) {
+          const int jt = list[j];
+          for (int g = 0; g < G; ++g)
+            if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
+        }
+        const unsigned bA = __ballot_sync(0xffffffffu, c == 1), bB = __ballot_sync(0xffffffffu, c == 2),
+                       bC = __ballot_sync(0xffffffffu, c == 3);
+        if (pass == 1 && c) {
+          int pos;
+          if (c == 3) pos = cC + __popc(bC & lt);
+          else if (c == 1) {
+            const int k = cA + __popc(bA & lt);
+            pos = nC + (k < nB ? 2 * k : nB + k);
+          } else {
+            const int k = cB + __popc(bB & lt);
+            pos = nC + (k < nA ? 2 * k + 1 : nA + k);
+          }
+          items[pos] = list[j];
+        }
+        cA += __popc(bA);
+        cB += __popc(bB);
+        cC += __popc(bC);
       }
-      if (ph == 1) nl = count;
+      nA = cA;
+      nB = cB;
+      nC = cC;
+    }
+    const int nl = nA + nB + nC;
+    int count = nl;
+    for (int base = 0; base < nv; base += 32) {  // short-term items in ascending order
+      const int j = base + lane;
+      const bool on = j < nv && (lflags[j] & 2);
+      const unsigned bal = __ballot_sync(0xffffffffu, on);
+      if (on) items[count + __popc(bal & lt)] = list[j];
+      count += __popc(bal);
     }
     if (lane == 0) {
       nL_s = nl;
@@ -221,7 +258,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   tc_fence_after();
   const int nL = nL_s, nS = nS_s, nI = nL + nS;
   const uint32_t tmem_base = tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_p = tmem_base + 128, tmem_o = tmem_base + 192;
+  const uint32_t tmem_o = tmem_base + 192;  // buffers at tmem_base + 64 * (item % 3)
 
   if (warp >= kSoftmaxWarps) {
     // ===================== three single-thread roles, one warp each =====================
@@ -246,43 +283,51 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         __syncwarp();
       }
     } else if (warp == kSoftmaxWarps + 1 && nI > 0) {
-      // ---- S(i) = Q K^T into S buffer i % 2 once the softmax warps hold S(i-2) in registers ----
+      // ---- S(i) = Q K^T into buffer i % 3 once O += P(i-3) V has read that buffer ----
       constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
       const uint64_t dq = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
       mbar_wait(b_res, 0, &abort_flag, 101);
-      for (int i = 0; i < nI; ++i) {
+      for (int i = 0, b = 0, ph = 0; i < nI; ++i) {  // b = i % 3, ph = (i / 3) & 1
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 102);
-        if (i >= 2) mbar_wait(b_sempty + 8 * (i & 1), ((i - 2) >> 1) & 1, &abort_flag, 103);
+        if (i >= 3) mbar_wait(b_done + 8 * b, ph ^ 1, &abort_flag, 103);
         tc_fence_after();
         const uint64_t dk =
             smem_desc(smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes), 16, C::kAtomBytes, C::kSwizzle);
-        const uint32_t ts = tmem_s + 64 * (i & 1);
+        const uint32_t ts = tmem_base + 64 * b;
         if (elect_one()) {
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) umma_bf16(ts, dq + 2 * k, dk + 2 * k, idesc_s, k > 0);
-          umma_commit(b_sfull + 8 * (i & 1));
+          umma_commit(b_sfull + 8 * b);
         }
         __syncwarp();
+        if (++b == 3) {
+          b = 0;
+          ph ^= 1;
+        }
       }
     } else if (warp == kSoftmaxWarps + 2 && nI > 0) {
       // ---- O += P(i) V once the probabilities of item i are in tensor memory ----
       constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
-      for (int i = 0; i < nI; ++i) {
+      for (int i = 0, b = 0, ph = 0; i < nI; ++i) {
         const uint64_t dv = smem_desc(smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes + C::kSmallBytes),
                                       C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-        const uint32_t tp = tmem_p + 32 * (i & 1);
+        const uint32_t tp = tmem_base + 64 * b;
         const uint32_t first = (i == 0 || i == nL) ? 0u : 1u;  // a phase starts the accumulator afresh
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 106);
-        mbar_wait(b_tfull + 8 * (i & 1), (i >> 1) & 1, &abort_flag, 104);
+        mbar_wait(b_tfull + 8 * b, ph, &abort_flag, 104);
         tc_fence_after();
         if (elect_one()) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             umma_bf16_ts(tmem_o, tp + 8 * k, dv + k * C::kKStep, idesc_pv, (first | (uint32_t)k) != 0u);
-          umma_commit(b_done + 8 * (i & 1));
+          umma_commit(b_done + 8 * b);
           umma_commit(b_empty + 8 * (i % STAGES));  // S(i) completed before the softmax warps read it
         }
         __syncwarp();
+        if (++b == 3) {
+          b = 0;
+          ph ^= 1;
+        }
       }
     }
   } else {
@@ -293,14 +338,18 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     float m = -INFINITY, l = 0.f, mL = -INFINITY, lL = 0.f;
     float park[D];  // the row's long-term accumulator while the short-term phase runs
-    bool zeroA = false, zeroB = false;  // this row of probability buffer 0 / 1 holds zeros
-    int acc = 0;                        // the current phase has written the accumulator
+    int acc = 0;    // the current phase has written the accumulator
     const float sc2 = s.scale * kLog2e;
+    int b = 0, ph = 0;  // buffer i % 3 and the parity (i / 3) & 1 of its barriers
+    int jt_n = nI > 0 ? items[0] : 0, cls_n = nI > 0 ? icls[warp] : 0;
 
     for (int i = 0; i < nI; ++i) {
       const bool isL = i < nL;
-      const int jt = items[i], p0 = jt * 64, par = i & 1;
-      const int cls = icls[i * kSoftmaxWarps + warp];
+      const int jt = jt_n, cls = cls_n, p0 = jt * 64;
+      if (i + 1 < nI) {  // the next item's tile and class, ahead of their use
+        jt_n = items[i + 1];
+        cls_n = icls[(i + 1) * kSoftmaxWarps + warp];
+      }
       uint64_t mask = 0ull;
       bool doB = cls == 1, fullB = cls == 1;
       if (cls == 2) {
@@ -311,23 +360,24 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         doB = __any_sync(0xffffffffu, mask != 0ull);
         fullB = __all_sync(0xffffffffu, mask == ~0ull);
       }
+      const uint32_t t_b = tmem_base + 64 * b + lane_off;
+      const uint32_t b_prev = b_done + 8 * (b == 0 ? 2 : b - 1), ph_prev = b == 0 ? ph ^ 1 : ph;  // item i-1
 
-      mbar_wait(b_sfull + 8 * par, (i >> 1) & 1, &abort_flag, 107);
+      mbar_wait(b_sfull + 8 * b, ph, &abort_flag, 107);
       __syncwarp();
       tc_fence_after();
       float sv[64];
       if (doB) {
-        tmem_ld32(tmem_s + 64 * par + lane_off, sv);
-        tmem_ld32(tmem_s + 64 * par + lane_off + 32, sv + 32);
+        tmem_ld32(t_b, sv);
+        tmem_ld32(t_b + 32, sv + 32);
         tmem_wait_ld();
       }
-      warp_arrive(b_sempty + 8 * par, lane);  // the loads have completed (wait::ld)
 
-      bool waited_prev = i == 0;  // the MMAs of item i-1 have completed
+      bool waited_prev = false;  // the MMAs of item i-1 have completed
       if (i == nL && nL > 0) {
         // End of the long-term phase: park its accumulator rows and statistics; the first P V
         // product of the short-term phase overwrites the accumulator.
-        mbar_wait(b_done + 8 * ((i - 1) & 1), ((i - 1) >> 1) & 1, &abort_flag, 111);
+        mbar_wait(b_prev, ph_prev, &abort_flag, 111);
         __syncwarp();
         tc_fence_after();
         waited_prev = true;
@@ -342,9 +392,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       }
 
       uint32_t pk[32];
-      float fac = 1.f;
-      bool need = false;
       if (doB) {
+        float fac = 1.f;
+        bool need = false;
         const float mt = (fullB ? row_max<true>(sv, 0ull) : row_max<false>(sv, mask)) * sc2;
         need = mt > m + kRescaleThreshold;  // also true on the row's first keys
         if (need) {
@@ -354,36 +404,32 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         }
         if (fullB) row_probs<true>(sv, 0ull, sc2, -m, l, pk);
         else row_probs<false>(sv, mask, sc2, -m, l, pk);
-      }
-      // Probability buffer i % 2 was last read by the MMAs of item i-2; rescaling the accumulator
-      // needs those of item i-1.
-      const bool rescale = doB && acc && __any_sync(0xffffffffu, need);
-      if (rescale && !waited_prev) {
-        mbar_wait(b_done + 8 * ((i - 1) & 1), ((i - 1) >> 1) & 1, &abort_flag, 108);
-      } else if (i >= 2) {
-        mbar_wait(b_done + 8 * par, ((i - 2) >> 1) & 1, &abort_flag, 109);
-      }
-      __syncwarp();
-      tc_fence_after();
-      const uint32_t t_p = tmem_p + 32 * par + lane_off;
-      const bool zero = par ? zeroB : zeroA;
-      if (doB) {
-        if (rescale) rescale_acc<D>(tmem_o + lane_off, fac);
-        tmem_st32u(t_p, pk);
-      } else if (!zero) {
+        if (acc && __any_sync(0xffffffffu, need)) {  // rescaling needs the MMAs of item i-1
+          if (!waited_prev) {
+            mbar_wait(b_prev, ph_prev, &abort_flag, 108);
+            __syncwarp();
+            tc_fence_after();
+          }
+          rescale_acc<D>(tmem_o + lane_off, fac);
+        }
+      } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) pk[c] = 0u;
-        tmem_st32u(t_p, pk);
       }
-      if (par) zeroB = !doB; else zeroA = !doB;
+      tmem_st32u(t_b, pk);  // the row's probabilities replace its logits
       tmem_wait_st();
-      warp_arrive(b_tfull + 8 * par, lane);  // the stores have completed (wait::st)
+      tc_fence_before();
+      warp_arrive(b_tfull + 8 * b, lane);  // the stores have completed (wait::st)
       acc = 1;
+      if (++b == 3) {
+        b = 0;
+        ph ^= 1;
+      }
     }
 
     // ---- epilogue ----
     if (nI > 0) {
-      mbar_wait(b_done + 8 * ((nI - 1) & 1), ((nI - 1) >> 1) & 1, &abort_flag, 110);
+      mbar_wait(b_done + 8 * ((nI - 1) % 3), ((nI - 1) / 3) & 1, &abort_flag, 110);
       __syncwarp();
       tc_fence_after();
     }
