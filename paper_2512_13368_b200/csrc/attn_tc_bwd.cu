@@ -209,6 +209,10 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     mbar_init(b_tfull, kComputeWarps);
     mbar_init(b_done, 1);
     mbar_fence_init();
+    // the resident tiles are needed whatever the lists say: their loads run while those are built
+    mbar_expect_tx(b_res, 2 * C::kBigBytes);
+    tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
+    tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
   }
   if (warp == 0) {
     __syncwarp();
@@ -229,11 +233,6 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     setmaxnreg_dec<kProducerRegs>();
     if (warp == kComputeWarps && nvis > 0) {
       // ---- loader: Q, dO once; K/V tiles up to STAGES ahead of their consumers ----
-      if (elect_one()) {
-        mbar_expect_tx(b_res, 2 * C::kBigBytes);
-        tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
-        tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
-      }
       for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 205);
@@ -421,6 +420,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     for (int gq = 0; gq < G; ++gq)
       if (st * G + gq < s.M) dalpha_part[(int64_t)u * s.M + st * G + gq] = gq == 0 ? a : 0.0;
   }
+  if (nvis == 0 && tid == 0) mbar_wait(b_res, 0, &abort_flag, 221);  // no load may outlive the CTA
   finish(warp, tmem_base, kBwdTmemCols, &abort_flag, status);
 }
 
@@ -528,6 +528,10 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     mbar_init(b_done, 1);
     mbar_init(b_sempty, kComputeWarps);
     mbar_fence_init();
+    // the resident tiles are needed whatever the lists say: their loads run while those are built
+    mbar_expect_tx(b_res, 2 * C::kBigBytes);
+    tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
+    tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
   }
   if (warp == 0) {
     __syncwarp();
@@ -581,11 +585,6 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     setmaxnreg_dec<kProducerRegs>();
     if (warp == kComputeWarps && nvis > 0) {
       // ---- loader: K, V once; Q, dO tiles and their row records up to STAGES ahead ----
-      if (elect_one()) {
-        mbar_expect_tx(b_res, 2 * C::kBigBytes);
-        tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
-        tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
-      }
       for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 214);
@@ -756,6 +755,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       }
     }
   }
+  if (nvis == 0 && tid == 0) mbar_wait(b_res, 0, &abort_flag, 222);  // no load may outlive the CTA
   finish(warp, tmem_base, kBwdTmemCols, &abort_flag, status);
 }
 

@@ -167,6 +167,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       mbar_init(b_done + 8 * i, 1);
     }
     mbar_fence_init();
+    // the query tile is needed whatever the lists say: its load runs while they are built
+    mbar_expect_tx(b_res, C::kBigBytes);
+    tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
   }
   if (warp == 0) {
     __syncwarp();
@@ -265,10 +268,6 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     setmaxnreg_dec<kProducerRegs>();
     if (warp == kSoftmaxWarps && nI > 0) {
       // ---- loader: K/V tiles, up to STAGES ahead of their consumers ----
-      if (elect_one()) {
-        mbar_expect_tx(b_res, C::kBigBytes);
-        tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
-      }
       for (int j = 0; j < nI; ++j) {
         const int sj = j % STAGES;
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 105);
@@ -493,6 +492,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       lse[BHL + (int64_t)u * s.L + t] = lS > 0.f ? (mS + log2f(lS)) * kLn2 : 0.f;
     }
   }
+  if (nI == 0 && tid == 0) mbar_wait(b_res, 0, &abort_flag, 112);  // no load may outlive the CTA
   finish(warp, tmem_base, kFwdTmemCols, &abort_flag, status);
 }
 
