@@ -59,6 +59,8 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.delta = reinterpret_cast<float *>(take(2 * units * s.L * sizeof(float)));
   w.dalpha = reinterpret_cast<double *>(take(units * s.M * sizeof(double)));
   w.qstats = reinterpret_cast<float4 *>(take(units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4)));
+  w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
+  w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.bytes = off;
   return w;
 }
@@ -262,7 +264,7 @@ int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
 const char *blossom_kernel_name(int id) {
   static const char *names[K_COUNT] = {
       "summary", "score_select", "fwd_simt", "bwd_dq_simt", "bwd_dkdv_simt", "gate_grad",
-      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast", "bwd_prep"};
+      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast", "bwd_prep", "tc_meta"};
   return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

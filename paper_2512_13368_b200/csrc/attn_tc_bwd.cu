@@ -152,18 +152,17 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
-    const int32_t *__restrict__ idx, const __grid_constant__ CUtensorMap tmdq,
+    const uint8_t *__restrict__ qmeta, const __grid_constant__ CUtensorMap tmdq,
     const float4 *__restrict__ qstats, double *__restrict__ dalpha_part, int32_t *__restrict__ status,
     int nT) {
   using C = Cfg<D>;
   constexpr int STAGES = kDqStages;
   constexpr int OC = D / 2;  // accumulator columns per thread
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, t_full, mma_done
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, t_full, mma_done, meta
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 6];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ int nvis_s;
   __shared__ double red[256];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -182,16 +181,16 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   uint8_t *q_tile = tiles;
   uint8_t *g_tile = q_tile + C::kBigBytes;
   uint8_t *kv_tiles = g_tile + C::kBigBytes;
-  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;
-  uint32_t *selw = reinterpret_cast<uint32_t *>(meta);
-  uint8_t *selb = meta;
-  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
-  uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
+  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;  // image built by tc_meta_kernel
+  const MetaLayout ml = meta_layout(nT);
+  const uint8_t *selb = meta;
+  const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
+  const uint8_t *lflags = meta + ml.flags;
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
   const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 4]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 4]), b_meta = smem_u32(&bars[2 * STAGES + 5]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -208,8 +207,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     mbar_init(b_sempty, kComputeWarps);
     mbar_init(b_tfull, kComputeWarps);
     mbar_init(b_done, 1);
+    mbar_init(b_meta, 1);
     mbar_fence_init();
-    // the resident tiles are needed whatever the lists say: their loads run while those are built
+    // the CTA's tile lists and its resident tiles
+    mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
+    bulk_load(smem_u32(meta), qmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, 2 * C::kBigBytes);
     tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
     tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
@@ -219,11 +221,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     tmem_alloc(smem_u32(&tmem_slot), kBwdTmemCols);
     tmem_relinquish();
   }
-  build_query_major_list(s, idx, u, st, pad0, nT, selw, selb, list, lflags, &nvis_s);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const int nvis = nvis_s;
+  mbar_wait(b_meta, 0, &abort_flag, 223);
+  const int nvis = *reinterpret_cast<const int *>(meta + ml.counts);
   const uint32_t tmem_base = tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_ds = tmem_base + 128,
                  tmem_dq = tmem_base + 160;
@@ -469,7 +471,7 @@ template <int D>
 __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
-    const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ idx,
+    const int32_t *__restrict__ seq_lens, const uint8_t *__restrict__ kmeta,
     const float4 *__restrict__ qstats, const __grid_constant__ CUtensorMap tmdk,
     const __grid_constant__ CUtensorMap tmdv, int32_t *__restrict__ status, int nT) {
   using C = Cfg<D>;
@@ -477,11 +479,10 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   constexpr int OC = D / 2;
   constexpr int kStageBytes = 2 * C::kSmallBytes + kStatBytes;  // Q, dO, row records
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done, s_empty
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done, s_empty, meta
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 6];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ int nvis_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nKT = (s.L + 127) >> 7;
@@ -491,7 +492,6 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
   const int key0 = kt * 128, key_last = min(s.L - 1, key0 + 127);
-  const int G = 128 / s.Bk, nb = 64 / s.Bk;
   const int Lpad = nT * 64;
 
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -501,16 +501,16 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   uint8_t *qg_tiles = v_tile + C::kBigBytes;  // [stage][Q, dO, row records]
   uint8_t *w_tile = qg_tiles + STAGES * kStageBytes;  // W^T  [128 keys][64 queries] bf16, 128-byte swizzle
   uint8_t *ds_tile = w_tile + 128 * 128;               // dS^T, same layout
-  uint8_t *meta = ds_tile + 128 * 128;
-  uint32_t *invw = reinterpret_cast<uint32_t *>(meta);  // [8][nT] bytes: per key block, per query tile
-  uint8_t *invb = meta;
-  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
-  uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
+  uint8_t *meta = ds_tile + 128 * 128;                  // image built by tc_meta_kernel
+  const MetaLayout ml = meta_layout(nT);
+  const uint8_t *invb = meta;                           // [8][nT] bytes: per key block, per query tile
+  const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
+  const uint8_t *lflags = meta + ml.flags;
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
   const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 2]), b_done = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 4]);
+  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 4]), b_meta = smem_u32(&bars[2 * STAGES + 5]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -527,8 +527,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     mbar_init(b_tfull, kComputeWarps);
     mbar_init(b_done, 1);
     mbar_init(b_sempty, kComputeWarps);
+    mbar_init(b_meta, 1);
     mbar_fence_init();
-    // the resident tiles are needed whatever the lists say: their loads run while those are built
+    // the CTA's tile lists and its resident tiles
+    mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
+    bulk_load(smem_u32(meta), kmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, 2 * C::kBigBytes);
     tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
     tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
@@ -538,44 +541,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     tmem_alloc(smem_u32(&tmem_slot), kBwdTmemCols);
     tmem_relinquish();
   }
-  for (int i = tid; i < (8 * nT + 3) / 4; i += kKvThreads) invw[i] = 0u;
-  __syncthreads();
-  {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
-    const int qb0 = kt * G, nq = s.M - qb0;
-    for (int i = tid; i < nq * s.topk; i += kKvThreads) {
-      const int qb = qb0 + i / s.topk;
-      const int blk = idx[((int64_t)u * s.M + qb) * s.topk + (i % s.topk)];
-      if (blk >= qb0 && blk < qb0 + G && blk <= qb) {
-        const int a = (blk - qb0) * nT + qb / nb;
-        atomicOr(&invw[a >> 2], (1u << (qb % nb)) << ((a & 3) * 8));
-      }
-    }
-  }
-  __syncthreads();
-  if (warp == 0) {
-    const int qt_min = key0 >> 6, qt_max = (s.L - 1) >> 6;
-    int count = 0;
-    for (int base = qt_min; base <= qt_max; base += 32) {
-      const int qt = base + lane;
-      int f = 0;
-      if (qt <= qt_max && key_last >= pad0) {
-        for (int g = 0; g < G; ++g) f |= invb[g * nT + qt] ? 1 : 0;
-        if (qt * 64 <= key_last + s.window - 1) f |= 2;
-      }
-      const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
-      if (f) {
-        const int pos = count + __popc(bal & ((1u << lane) - 1u));
-        list[pos] = (uint16_t)qt;
-        lflags[pos] = (uint8_t)f;
-      }
-      count += __popc(bal);
-    }
-    if (lane == 0) nvis_s = count;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const int nvis = nvis_s;
+  mbar_wait(b_meta, 0, &abort_flag, 224);
+  const int nvis = *reinterpret_cast<const int *>(meta + ml.counts);
   const uint32_t tmem_base = tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_dv = tmem_base + 128,
                  tmem_dk = tmem_base + 192;
@@ -783,6 +753,7 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
+  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, ws.kmeta, st)) return rc;
   {
     LaunchScope ls(K_BWD_PREP, st);
     const int Lpad = nT * 64, rpb = 256 / (D / 8);
@@ -792,13 +763,13 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   }
   {
     LaunchScope ls(K_BWD_DQ_TC, st);
-    bwd_dq_tc_kernel<D><<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, idx,
+    bwd_dq_tc_kernel<D><<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
                                                            tdq, ws.qstats, ws.dalpha,
                                                            ws.status, nT);
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
-    bwd_dkdv_tc_kernel<D><<<grid, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, idx,
+    bwd_dkdv_tc_kernel<D><<<grid, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
                                                              ws.qstats, tdk, tdv, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;

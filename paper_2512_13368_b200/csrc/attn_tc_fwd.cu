@@ -114,16 +114,15 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
     const __grid_constant__ CUtensorMap tmol, const __grid_constant__ CUtensorMap tmos, Shape s,
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
-    const int32_t *__restrict__ idx, int training, float *__restrict__ lse,
+    const uint8_t *__restrict__ qmeta, int training, float *__restrict__ lse,
     int32_t *__restrict__ status, int nT) {
   using C = Cfg<D>;
   constexpr int STAGES = kFwdStages;
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, then one per buffer: s_full[3], t_full[3], done[3]
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 10];
+  // barriers: full[STAGES], empty[STAGES], res, one per buffer: s_full[3], t_full[3], done[3], meta
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 11];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ int nvis_s, nL_s, nS_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
@@ -138,18 +137,17 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   uint8_t *tiles = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
   uint8_t *q_tile = tiles;
   uint8_t *kv_tiles = q_tile + C::kBigBytes;  // [stage][K, V]
-  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;
-  uint32_t *selw = reinterpret_cast<uint32_t *>(meta);
-  uint8_t *selb = meta;
-  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ((8 * nT + 15) / 16) * 16);
-  uint8_t *lflags = reinterpret_cast<uint8_t *>(list + nT);
-  uint16_t *items = reinterpret_cast<uint16_t *>(meta + ((11 * nT + 15) / 16) * 16);  // [2 nT]
-  uint8_t *icls = reinterpret_cast<uint8_t *>(items + 2 * nT);                         // [2 nT][4]
+  uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;  // image built by tc_meta_kernel
+  const MetaLayout ml = meta_layout(nT);
+  const uint8_t *selb = meta;
+  const uint16_t *items = reinterpret_cast<const uint16_t *>(meta + ml.items);  // [2 nT]
+  const uint8_t *icls = meta + ml.icls;                                         // [2 nT][4]
+  const int *counts = reinterpret_cast<const int *>(meta + ml.counts);
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]);
   const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 1]), b_tfull = smem_u32(&bars[2 * STAGES + 4]);
-  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 7]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 7]), b_meta = smem_u32(&bars[2 * STAGES + 10]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;  // an earlier CTA timed out: do not wait again
@@ -166,8 +164,11 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       mbar_init(b_tfull + 8 * i, kSoftmaxWarps);
       mbar_init(b_done + 8 * i, 1);
     }
+    mbar_init(b_meta, 1);
     mbar_fence_init();
-    // the query tile is needed whatever the lists say: its load runs while they are built
+    // the CTA's tile lists and its query tile
+    mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
+    bulk_load(smem_u32(meta), qmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, C::kBigBytes);
     tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
   }
@@ -176,90 +177,11 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     tmem_alloc(smem_u32(&tmem_slot), kFwdTmemCols);
     tmem_relinquish();
   }
-  build_query_major_list(s, idx, u, st, pad0, nT, selw, selb, list, lflags, &nvis_s);
-  __syncthreads();
-  if (warp == 0) {  // items: the tiles of the long-term phase, then those of the short-term phase
-    const int nv = nvis_s;
-    // Long-term items: the tiles both 64-row halves of the CTA need, then alternately a tile only
-    // rows 0..63 need and a tile only rows 64..127 need.  A softmax warp may run one item ahead
-    // of the slowest one, so with alternating items both pairs of warps have work at once.
-    const int G = 128 / s.Bk, gh = G / 2;
-    const unsigned lt = (1u << lane) - 1u;
-    int nA = 0, nB = 0, nC = 0;
-    for (int pass = 0; pass < 2; ++pass) {
-      int cA = 0, cB = 0, cC = 0;
-      for (int base = 0; base < nv; base += 32) {
-        const int j = base + lane;
-        int c = 0;
-        if (j < nv && (lflags[j] & 1)) {
-          const int jt = list[j];
-          for (int g = 0; g < G; ++g)
-            if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
-        }
-        const unsigned bA = __ballot_sync(0xffffffffu, c == 1), bB = __ballot_sync(0xffffffffu, c == 2),
-                       bC = __ballot_sync(0xffffffffu, c == 3);
-        if (pass == 1 && c) {
-          int pos;
-          if (c == 3) pos = cC + __popc(bC & lt);
-          else if (c == 1) {
-            const int k = cA + __popc(bA & lt);
-            pos = nC + (k < nB ? 2 * k : nB + k);
-          } else {
-            const int k = cB + __popc(bB & lt);
-            pos = nC + (k < nA ? 2 * k + 1 : nA + k);
-          }
-          items[pos] = list[j];
-        }
-        cA += __popc(bA);
-        cB += __popc(bB);
-        cC += __popc(bC);
-      }
-      nA = cA;
-      nB = cB;
-      nC = cC;
-    }
-    const int nl = nA + nB + nC;
-    int count = nl;
-    for (int base = 0; base < nv; base += 32) {  // short-term items in ascending order
-      const int j = base + lane;
-      const bool on = j < nv && (lflags[j] & 2);
-      const unsigned bal = __ballot_sync(0xffffffffu, on);
-      if (on) items[count + __popc(bal & lt)] = list[j];
-      count += __popc(bal);
-    }
-    if (lane == 0) {
-      nL_s = nl;
-      nS_s = count - nl;
-    }
-    __syncwarp();
-    // Class of every (item, softmax warp): 0 = no row of the warp needs the tile, 1 = every row
-    // sees all 64 keys, 2 = mixed (the warp builds per-lane column masks).
-    const bool uni = s.Bk >= 32;  // a warp's 32 rows share one query block
-    const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
-    for (int e = lane; e < count * kSoftmaxWarps; e += 32) {
-      const int it = e / kSoftmaxWarps, w = e % kSoftmaxWarps;
-      const int jt = items[it], p0 = jt * 64, t_lo = row0 + w * 32;
-      const bool some = p0 <= t_lo + 31 && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
-      const bool inner = t_lo >= pad0 && t_lo + 31 < s.L && p0 >= pad0 && p0 + 63 <= t_lo;
-      int cls = 0;
-      if (some) {
-        if (it < nl) {
-          if (!uni) cls = 2;
-          else {
-            const uint32_t bits = selb[((w * 32) / s.Bk) * nT + jt];
-            cls = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
-          }
-        } else if (p0 + 63 >= t_lo - s.window + 1) {
-          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;
-        }
-      }
-      icls[e] = (uint8_t)cls;
-    }
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const int nL = nL_s, nS = nS_s, nI = nL + nS;
+  mbar_wait(b_meta, 0, &abort_flag, 113);
+  const int nL = counts[1], nS = counts[2], nI = nL + nS;
   const uint32_t tmem_base = tmem_slot;
   const uint32_t tmem_o = tmem_base + 192;  // buffers at tmem_base + 64 * (item % 3)
 
@@ -515,9 +437,10 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
       cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
+  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, nullptr, st)) return rc;
   {
     LaunchScope ls(K_FWD_TC, st);
-    fwd_tc_kernel<D><<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, idx,
+    fwd_tc_kernel<D><<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, ws.qmeta,
                                                      training, lse, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;

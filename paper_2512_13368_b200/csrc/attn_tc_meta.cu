@@ -1,0 +1,240 @@
+// Tile bookkeeping of the tensor-core attention kernels, built once per call.
+//
+// Which 64-key tiles a 128-row query tile has to visit (the blocks its query blocks selected,
+// Eq. 13, and the tiles its window reaches, Eq. 15), in which order, and which of its warps a tile
+// concerns, depends only on the block indices and the sequence lengths.  Building that inside the
+// attention kernels cost every CTA several thousand cycles before its first product; here one warp
+// per attention CTA builds the image of the bookkeeping the attention kernel wants in shared
+// memory, and the attention kernel fetches it with one bulk copy while its first tiles load.
+//
+// Query-major image (forward and dQ kernel), see meta_layout():
+//   [8][nT] selection bytes   bit c of byte (g, jt): query block g of the CTA selected key block
+//                             jt * (64 / Bk) + c
+//   list[nT], flags[nT]       the tiles any row of the CTA needs, ascending; bit 0: some selected
+//                             block lies in the tile, bit 1: the window of some row reaches it
+//   items[2 nT], icls[2 nT][4] (forward) the long-term tiles, then the short-term tiles, and the
+//                             class of every (item, softmax warp)
+//   counts                    {tiles on the list, long-term items, short-term items}
+// Key-major image (dK/dV kernel): [8][nT] bytes: bit c of byte (g, qt): query block
+// qt * (64 / Bk) + c selected key block g of the CTA; list / flags of the 64-query tiles that
+// visit the CTA's keys; counts {tiles on the list}.
+#include "tc_common.cuh"
+
+namespace blossom {
+namespace tc {
+namespace {
+
+constexpr int kMetaWarps = 4;  // images per CTA, one warp each
+
+// One warp builds one image: no block-wide barrier anywhere, so the (latency-bound) images of a
+// whole launch are in flight at once.
+__global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const int32_t *__restrict__ seq_lens,
+                                                                  const int32_t *__restrict__ idx,
+                                                                  uint8_t *__restrict__ qmeta,
+                                                                  uint8_t *__restrict__ kmeta, int nT,
+                                                                  int n_query_ctas, int n_images) {
+  extern __shared__ __align__(16) uint8_t meta_all[];
+  const MetaLayout ml = meta_layout(nT);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int image = (int)blockIdx.x * kMetaWarps + warp;
+  if (image >= n_images) return;
+  uint8_t *meta = meta_all + (size_t)warp * ml.bytes;
+  const int nST = (s.L + 127) >> 7;
+  const bool key_major = image >= n_query_ctas;
+  const int cta = key_major ? image - n_query_ctas : image;
+  const int u = cta / nST, n = u / s.H;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  uint32_t *selw = reinterpret_cast<uint32_t *>(meta);
+  uint8_t *selb = meta;
+  uint16_t *list = reinterpret_cast<uint16_t *>(meta + ml.list);
+  uint8_t *lflags = meta + ml.flags;
+  uint16_t *items = reinterpret_cast<uint16_t *>(meta + ml.items);
+  uint8_t *icls = meta + ml.icls;
+  int *counts = reinterpret_cast<int *>(meta + ml.counts);
+  const unsigned lt = (1u << lane) - 1u;
+  const int G = 128 / s.Bk, nb = 64 / s.Bk;
+
+  for (int i = lane; i < ml.bytes / 4; i += 32) selw[i] = 0u;  // the whole image
+  __syncwarp();
+
+  if (!key_major) {
+    const int st = nST - 1 - cta % nST;  // the attention kernels take long rows first
+    const int row0 = st * 128, row_last = min(s.L - 1, row0 + 127);
+    for (int i = lane; i < G * s.topk; i += 32) {  // the selections of the CTA's query blocks
+      const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
+      if (qb < s.M) {
+        const int blk = idx[((int64_t)u * s.M + qb) * s.topk + slot];
+        if (blk >= 0 && blk <= qb) {
+          const int a = g * nT + blk / nb;
+          atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
+        }
+      }
+    }
+    __syncwarp();
+    int nv = 0;
+    {  // the tiles any row of the CTA needs, ascending
+      const int jt_max = row_last >> 6;
+      for (int base = 0; base <= jt_max; base += 32) {
+        const int jt = base + lane;
+        int f = 0;
+        if (jt <= jt_max && row_last >= pad0 && jt * 64 + 63 >= pad0) {
+          for (int g = 0; g < G; ++g) f |= selb[g * nT + jt] ? 1 : 0;
+          if (jt * 64 + 63 >= row0 - s.window + 1) f |= 2;
+        }
+        const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
+        if (f) {
+          const int pos = nv + __popc(bal & lt);
+          list[pos] = (uint16_t)jt;
+          lflags[pos] = (uint8_t)f;
+        }
+        nv += __popc(bal);
+      }
+    }
+    __syncwarp();
+    // Long-term items: the tiles both 64-row halves of the CTA need, then alternately a tile only
+    // rows 0..63 need and a tile only rows 64..127 need.  A softmax warp may run ahead of the
+    // slowest one, so with alternating items both pairs of warps have work at once.
+    const int gh = G / 2;
+    int nA = 0, nB = 0, nC = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+      int cA = 0, cB = 0, cC = 0;
+      for (int base = 0; base < nv; base += 32) {
+        const int j = base + lane;
+        int c = 0;
+        if (j < nv && (lflags[j] & 1)) {
+          const int jt = list[j];
+          for (int g = 0; g < G; ++g)
+            if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
+        }
+        const unsigned bA = __ballot_sync(0xffffffffu, c == 1), bB = __ballot_sync(0xffffffffu, c == 2),
+                       bC = __ballot_sync(0xffffffffu, c == 3);
+        if (pass == 1 && c) {
+          int pos;
+          if (c == 3) pos = cC + __popc(bC & lt);
+          else if (c == 1) {
+            const int k = cA + __popc(bA & lt);
+            pos = nC + (k < nB ? 2 * k : nB + k);
+          } else {
+            const int k = cB + __popc(bB & lt);
+            pos = nC + (k < nA ? 2 * k + 1 : nA + k);
+          }
+          items[pos] = list[j];
+        }
+        cA += __popc(bA);
+        cB += __popc(bB);
+        cC += __popc(bC);
+      }
+      nA = cA;
+      nB = cB;
+      nC = cC;
+    }
+    const int nl = nA + nB + nC;
+    int count = nl;
+    for (int base = 0; base < nv; base += 32) {  // short-term items in ascending order
+      const int j = base + lane;
+      const bool on = j < nv && (lflags[j] & 2);
+      const unsigned bal = __ballot_sync(0xffffffffu, on);
+      if (on) items[count + __popc(bal & lt)] = list[j];
+      count += __popc(bal);
+    }
+    if (lane == 0) {
+      counts[0] = nv;
+      counts[1] = nl;
+      counts[2] = count - nl;
+    }
+    __syncwarp();
+    // Class of every (item, softmax warp): 0 = no row of the warp needs the tile, 1 = every row
+    // sees all 64 keys, 2 = mixed (the warp builds per-lane column masks).
+    const bool uni = s.Bk >= 32;  // a warp's 32 rows share one query block
+    const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
+    for (int e = lane; e < count * 4; e += 32) {
+      const int it = e >> 2, w = e & 3;
+      const int jt = items[it], p0 = jt * 64, t_lo = row0 + w * 32;
+      const bool some = p0 <= t_lo + 31 && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
+      const bool inner = t_lo >= pad0 && t_lo + 31 < s.L && p0 >= pad0 && p0 + 63 <= t_lo;
+      int cls = 0;
+      if (some) {
+        if (it < nl) {
+          if (!uni) cls = 2;
+          else {
+            const uint32_t bits = selb[((w * 32) / s.Bk) * nT + jt];
+            cls = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
+          }
+        } else if (p0 + 63 >= t_lo - s.window + 1) {
+          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;
+        }
+      }
+      icls[e] = (uint8_t)cls;
+    }
+  } else {
+    const int kt = cta % nST;  // the dK/dV kernel takes early keys first
+    const int key0 = kt * 128, key_last = min(s.L - 1, key0 + 127);
+    {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
+      // (the index rows of query blocks qb0 .. M-1 are contiguous; eight loads in flight per lane)
+      const int qb0 = kt * G, total = (s.M - qb0) * s.topk;
+      const int32_t *rows = idx + ((int64_t)u * s.M + qb0) * s.topk;
+      for (int base = 0; base < total; base += 256) {
+        int blk[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = base + e * 32 + lane;
+          blk[e] = i < total ? rows[i] : -1;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = base + e * 32 + lane, qb = qb0 + i / s.topk;
+          if (blk[e] >= qb0 && blk[e] < qb0 + G && blk[e] <= qb) {
+            const int a = (blk[e] - qb0) * nT + qb / nb;
+            atomicOr(&selw[a >> 2], (1u << (qb % nb)) << ((a & 3) * 8));
+          }
+        }
+      }
+    }
+    __syncwarp();
+    const int qt_min = key0 >> 6, qt_max = (s.L - 1) >> 6;
+    int count = 0;
+    for (int base = qt_min; base <= qt_max; base += 32) {
+      const int qt = base + lane;
+      int f = 0;
+      if (qt <= qt_max && key_last >= pad0) {
+        for (int g = 0; g < G; ++g) f |= selb[g * nT + qt] ? 1 : 0;
+        if (qt * 64 <= key_last + s.window - 1) f |= 2;
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
+      if (f) {
+        const int pos = count + __popc(bal & lt);
+        list[pos] = (uint16_t)qt;
+        lflags[pos] = (uint8_t)f;
+      }
+      count += __popc(bal);
+    }
+    if (lane == 0) counts[0] = count;
+  }
+  __syncwarp();
+  uint4 *dst = reinterpret_cast<uint4 *>((key_major ? kmeta : qmeta) + (size_t)cta * ml.bytes);
+  const uint4 *src = reinterpret_cast<const uint4 *>(meta);
+  for (int i = lane; i < ml.bytes / 16; i += 32) dst[i] = src[i];
+}
+
+}  // namespace
+
+int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
+                   uint8_t *kmeta, cudaStream_t st) {
+  const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
+  const int nq = nST * s.B * s.H, n_images = kmeta ? 2 * nq : nq;
+  const size_t smem = (size_t)kMetaWarps * meta_bytes(nT);
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(tc_meta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
+  {
+    LaunchScope ls(K_TC_META, st);
+    tc_meta_kernel<<<(unsigned)((n_images + kMetaWarps - 1) / kMetaWarps), kMetaWarps * 32, smem, st>>>(
+        s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
+}  // namespace tc
+}  // namespace blossom

@@ -29,6 +29,8 @@ struct Workspace {
   double *dalpha;    // [B][H][M]     per query block partial of d alpha
   float4 *qstats;    // [B][H][ceil(L/64)*64]  16 bytes per query row, laid out per pair of rows as
                      //   {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)} for the dK/dV kernel
+  uint8_t *qmeta;    // per query-major CTA of the tensor-core kernels: tile lists (tc_meta_kernel)
+  uint8_t *kmeta;    // per key-major CTA (dK/dV kernel): tile lists
   size_t bytes;
 };
 
@@ -39,7 +41,7 @@ extern unsigned long long g_launches;  // host-side launch counter
 // Kernel identifiers reported by the optional per-launch event profile.
 enum KernelId {
   K_SUMMARY = 0, K_SCORE_SELECT, K_FWD_SIMT, K_BWD_DQ_SIMT, K_BWD_DKDV_SIMT, K_GATE_GRAD,
-  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_BWD_PREP, K_COUNT
+  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_BWD_PREP, K_TC_META, K_COUNT
 };
 void prof_mark(int id, int phase, cudaStream_t st);  // no-op unless a profile is running
 
@@ -98,6 +100,7 @@ int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, flo
 
 namespace tc {
 bool fwd_tc_supported(const Shape &s, int dtype);
+size_t tc_meta_bytes(const Shape &s);  // bytes of one of the two tile-list areas of the workspace
 int launch_bwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                   const int32_t *seq_lens, const int32_t *idx, const void *out_lt, const void *out_st,
                   const float *lse, const void *dout, void *dq, void *dk, void *dv,

@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
 constexpr int kFastThreads = 256;
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kFastThreads, 5) score_select_fast_kernel(
+__global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
     Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
     const float *__restrict__ knorm, const int32_t *__restrict__ klive,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
@@ -312,22 +312,25 @@ __global__ void __launch_bounds__(kFastThreads, 5) score_select_fast_kernel(
       for (int a = 0; a < 4; ++a)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[a][c] = 0.f;
+      const int ne = (nb + 15) >> 4;  // groups of 16 candidates that hold any (block-uniform)
 #pragma unroll 4
       for (int c = 0; c < D; c += 4) {
         float4 qa[4], kb[4];
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
           qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + c);
-          kb[a] = *reinterpret_cast<const float4 *>(ks + (tx + 16 * a) * P + c);
+          if (a < ne) kb[a] = *reinterpret_cast<const float4 *>(ks + (tx + 16 * a) * P + c);
         }
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+        for (int e = 0; e < 4; ++e)
+          if (e < ne) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
-            acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
-            acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
-            acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
+            for (int a = 0; a < 4; ++a) {
+              acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
+              acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
+              acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
+              acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
+            }
           }
       }
       __syncthreads();  // everyone has read ks: it becomes zs

@@ -375,9 +375,24 @@ struct Cfg {
   static constexpr int kKStep = (16 * kRowBytes) >> 4;       // descriptor advance of 16 rows
 };
 
-// bytes of the per-CTA tile bookkeeping: [8][nT] selection bytes, nT list entries, nT flags, and
-// (forward) 2 nT per-phase items with 4 class bytes each
-__host__ __device__ inline int meta_bytes(int nT) { return ((11 * nT + 15) / 16) * 16 + ((12 * nT + 15) / 16) * 16 + 16; }
+// Per-CTA tile bookkeeping, built once per call by tc_meta_kernel and brought into shared memory
+// by one bulk copy: [8][nT] selection bytes, nT list entries, nT flags, (forward) 2 nT per-phase
+// items with 4 class bytes each, and the counts {tiles on the list, long-term items, short-term
+// items}.  Offsets in bytes; every part starts on a 16-byte boundary where a copy needs it.
+struct MetaLayout {
+  int list, flags, items, icls, counts, bytes;
+};
+__host__ __device__ inline MetaLayout meta_layout(int nT) {
+  MetaLayout m;
+  m.list = ((8 * nT + 15) / 16) * 16;
+  m.flags = m.list + 2 * nT;
+  m.items = ((m.flags + nT + 15) / 16) * 16;
+  m.icls = m.items + 4 * nT;
+  m.counts = ((m.icls + 8 * nT + 15) / 16) * 16;
+  m.bytes = m.counts + 16;
+  return m;
+}
+__host__ __device__ inline int meta_bytes(int nT) { return meta_layout(nT).bytes; }
 
 // one arrival per warp, after all its lanes are done
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
@@ -405,51 +420,6 @@ __device__ __forceinline__ float gate_alpha(const float *gate, int h) {
   return 1.f / (1.f + __expf(-(gate[h * 2 + 0] - gate[h * 2 + 1])));
 }
 
-// Query-major tile list (forward and dQ): per 64-key tile, which key blocks each of the CTA's
-// query blocks selected (selb[g * nT + tile]), and the ascending list of tiles to visit with
-// flags (bit 0: some selected block lies in the tile, bit 1: the window of some row reaches it).
-// Called by every thread of the CTA; contains block-wide barriers.
-__device__ __forceinline__ void build_query_major_list(const Shape &s, const int32_t *idx, int u, int st,
-                                                       int pad0, int nT, uint32_t *selw, uint8_t *selb,
-                                                       uint16_t *list, uint8_t *lflags, int *nvis_out) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nthr = blockDim.x;
-  const int G = 128 / s.Bk, nb = 64 / s.Bk;
-  const int row0 = st * 128, row_last = min(s.L - 1, row0 + 127);
-  for (int i = tid; i < (8 * nT + 3) / 4; i += nthr) selw[i] = 0u;
-  __syncthreads();
-  for (int i = tid; i < G * s.topk; i += nthr) {
-    const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
-    if (qb < s.M) {
-      const int blk = idx[((int64_t)u * s.M + qb) * s.topk + slot];
-      if (blk >= 0 && blk <= qb) {
-        const int a = g * nT + blk / nb;
-        atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
-      }
-    }
-  }
-  __syncthreads();
-  if (warp == 0) {
-    const int jt_max = row_last >> 6;
-    int count = 0;
-    for (int base = 0; base <= jt_max; base += 32) {
-      const int jt = base + lane;
-      int f = 0;
-      if (jt <= jt_max && row_last >= pad0 && jt * 64 + 63 >= pad0) {
-        for (int g = 0; g < G; ++g) f |= selb[g * nT + jt] ? 1 : 0;
-        if (jt * 64 + 63 >= row0 - s.window + 1) f |= 2;
-      }
-      const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
-      if (f) {
-        const int pos = count + __popc(bal & ((1u << lane) - 1u));
-        list[pos] = (uint16_t)jt;
-        lflags[pos] = (uint8_t)f;
-      }
-      count += __popc(bal);
-    }
-    if (lane == 0) *nvis_out = count;
-  }
-}
-
 // Store 16-byte chunk ch of row r of a D-wide bf16 tile laid out as TMA expects it (128-byte
 // swizzle for D = 64, 64-byte swizzle for D = 32).  `tile` must be 1024-byte aligned.
 template <int D>
@@ -460,6 +430,11 @@ __device__ __forceinline__ void store_row_chunk(uint8_t *tile, int r, int ch, ui
 
 // ---- host: TMA descriptor of a q-shaped bf16 tensor, box = (D, rows, 1, 1) -----------------
 int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows);
+
+// Builds the bookkeeping of every query-major CTA (forward, dQ) into qmeta and, if kmeta is not
+// null, of every key-major CTA (dK/dV) into kmeta: meta_bytes(nT) bytes per CTA, CTA-major.
+int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
+                   uint8_t *kmeta, cudaStream_t st);
 
 // per-file launchers behind launch_fwd_tc / launch_bwd_tc
 template <int D>

@@ -42,6 +42,11 @@ bool fwd_tc_supported(const Shape &s, int dtype) {
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 
+size_t tc_meta_bytes(const Shape &s) {
+  const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
+  return (size_t)s.B * s.H * nST * (size_t)meta_bytes(nT);
+}
+
 int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                   const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt, void *out_st,
                   float *lse, const Workspace &ws, cudaStream_t st) {
