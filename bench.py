@@ -80,7 +80,8 @@ def work_model(w):
     byts.update({"fwd_simt": byts["fwd"], "fwd_tc": byts["fwd"],
                  "bwd_dq_simt": 7 * T + 2 * lse_b, "bwd_dkdv_simt": 6 * T + 2 * lse_b,
                  "bwd_dq_tc": 7 * T + 2 * lse_b, "bwd_dkdv_tc": 6 * T + 2 * lse_b,
-                 "summary": T, "score_select": T, "score_fast": T, "bwd_prep": 3 * T + lse_b})
+                 "summary": T, "score_select": T, "score_fast": T, "bwd_prep": 3 * T + lse_b,
+                 "tc_meta": idx_b})
     return {"tiles_lt": tiles_L, "tiles_st": tiles_S, "tile_flops": tile_flops,
             "flops": {k: g * tb * tile_flops for k, g in gemms.items()}, "bytes": byts,
             "step_flops": 7 * tb * tile_flops, "step_bytes": 15 * T + 3 * lse_b + 2 * idx_b}
