@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   __shared__ __align__(8) uint64_t bars[2 * STAGES + 6];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ double red[256];
+  __shared__ double red[kComputeWarps];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
@@ -411,14 +411,17 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     // d alpha = sum (P_lt - P_st) dP; a weight of exactly 0 makes its branch's sum 0 and the gate
     // gradient alpha (1 - alpha) d alpha 0 whatever d alpha is
     const float dal = (alpha > 0.f ? (dalL.x + dalL.y) / alpha : 0.f) - (beta > 0.f ? (dalS.x + dalS.y) / beta : 0.f);
-    red[tid] = row_valid ? (double)dal : 0.0;
+    double a = row_valid ? (double)dal : 0.0;  // fixed-shape tree over the warp, then over the warps
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) red[warp] = a;
   }
   tc_fence_before();
   __syncthreads();
   // d alpha partial of this CTA -> first query-block slot of the super-tile, zeros in the rest
   if (tid == 0) {
     double a = 0.0;
-    for (int i = 0; i < 256; ++i) a += red[i];  // fixed order
+    for (int i = 0; i < kComputeWarps; ++i) a += red[i];  // fixed order
     for (int gq = 0; gq < G; ++gq)
       if (st * G + gq < s.M) dalpha_part[(int64_t)u * s.M + st * G + gq] = gq == 0 ? a : 0.0;
   }
