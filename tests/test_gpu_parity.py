@@ -81,6 +81,9 @@ def test_config5_attention_shape(runner):
     (257, 64, 8, 5, 9, [257, 100]),      # many small blocks, odd length
     (192, 32, 64, 2, 1, None),           # window 1: short-term branch returns v
     (512, 64, 64, 64, 64, None),         # top-k covers every block (long-term branch = dense)
+    (1000, 64, 32, 6, 100, [1000, 333]),   # several 128-row tiles, ragged last tile, padding inside a tile
+    (700, 32, 16, 9, 48, [700, 129, 64]),  # two query blocks per warp, padding ends on a tile border
+    (384, 64, 16, 3, 130, None),           # window wider than two tiles, few selected blocks
 ])
 def test_edge_shapes(runner, dtype, L, D, block, topk, window, lens):
     B = len(lens) if lens else 2
