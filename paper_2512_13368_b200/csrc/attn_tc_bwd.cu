@@ -16,13 +16,15 @@
 // 16-column passes, two columns per FMA / ADD / MUL (packed f32x2); outputs are staged in shared
 // memory and written with whole-line TMA stores.
 //
-//  dQ     resident Q, dO (128 queries); streams K, V 64-key tiles (same walk as the forward).
-//         Tensor memory: S [0,64), dP [64,128), dS [128,160) (bf16 pairs), dQ [160,160+D).
-//         S = Q K^T, dP = dO V^T; P'_x = weight_x exp(S - lse_x);
+//  dQ     resident Q, dO (128 queries); streams K, V 64-key tiles (same walk as the forward) and
+//         works through them in half tiles of 32 keys.  Tensor memory: three buffers of 64
+//         columns (half tile x uses buffer x % 3: S in its first 32 columns, dP in the other 32)
+//         and dQ [192,192+D).  S = Q K^T, dP = dO V^T; P'_x = weight_x exp(S - lse_x);
 //         dS = P'_lt (dP - Delta_lt) + P'_st (dP - Delta_st) (one tile for both branches, they share
-//         K), written to tensor memory and read from there by dQ += dS K.  The first-stage MMAs of
-//         tile i+1 run while the compute warps work on tile i.
-//         d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
+//         K).  A thread owns 16 of the 32 columns and writes its dS (bf16 pairs) over the first 8
+//         of its own S columns, from where dQ += dS K reads it: the compute warps wait for one
+//         thing per half tile (its S and dP), and the first stage of the next two half tiles runs
+//         meanwhile.  d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
 //  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
 //         records, by bulk copy) that selected one of its key blocks or whose window reaches them.
 //         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D): no room for
@@ -159,8 +161,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   constexpr int STAGES = kDqStages;
   constexpr int OC = D / 2;  // accumulator columns per thread
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, s_empty, t_full, mma_done, meta
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 6];
+  // barriers: full[STAGES], empty[STAGES], res, meta, then one per buffer: s_full[3], t_full[3],
+  // mma_done[3]
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 11];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ double red[kComputeWarps];
@@ -188,9 +191,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   const uint8_t *lflags = meta + ml.flags;
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
-  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
-  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 4]), b_meta = smem_u32(&bars[2 * STAGES + 5]);
+  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_meta = smem_u32(&bars[2 * STAGES + 1]);
+  const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 5]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 8]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -203,10 +206,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
       mbar_init(b_empty + 8 * i, 1);
     }
     mbar_init(b_res, 1);
-    mbar_init(b_sfull, 1);
-    mbar_init(b_sempty, kComputeWarps);
-    mbar_init(b_tfull, kComputeWarps);
-    mbar_init(b_done, 1);
+    for (int i = 0; i < 3; ++i) {
+      mbar_init(b_sfull + 8 * i, 1);
+      mbar_init(b_tfull + 8 * i, kComputeWarps);
+      mbar_init(b_done + 8 * i, 1);
+    }
     mbar_init(b_meta, 1);
     mbar_fence_init();
     // the CTA's tile lists and its resident tiles
@@ -227,8 +231,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   mbar_wait(b_meta, 0, &abort_flag, 223);
   const int nvis = *reinterpret_cast<const int *>(meta + ml.counts);
   const uint32_t tmem_base = tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_ds = tmem_base + 128,
-                 tmem_dq = tmem_base + 160;
+  const uint32_t tmem_dq = tmem_base + 192;  // buffers at tmem_base + 64 * (half tile % 3)
 
   if (warp >= kComputeWarps) {
     // ============ three single-thread roles, one converged warp each ============
@@ -249,44 +252,59 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         __syncwarp();
       }
     } else if (warp == kComputeWarps + 1 && nvis > 0) {
-      // ---- S = Q K^T and dP = dO V^T of tile i once the compute warps hold tile i-1's ----
-      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
+      // ---- S = Q K^T and dP = dO V^T of a half tile (32 keys) into buffer x % 3 once
+      // dQ += dS K of half tile x-3 has read that buffer ----
+      constexpr uint32_t idesc_s = instr_desc(128, 32, 0, 0);
       const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
       const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
       mbar_wait(b_res, 0, &abort_flag, 201);
-      for (int i = 0; i < nvis; ++i) {
+      for (int i = 0, x = 0, b = 0, ph = 0; i < nvis; ++i) {  // x = 2 i + hh, b = x % 3, ph = (x / 3) & 1
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 202);
-        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 203);
-        tc_fence_after();
-        const uint32_t kt = smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes);
-        const uint64_t dkd = smem_desc(kt, 16, C::kAtomBytes, C::kSwizzle);
-        const uint64_t dvd = smem_desc(kt + C::kSmallBytes, 16, C::kAtomBytes, C::kSwizzle);
-        if (elect_one()) {
+        for (int hh = 0; hh < 2; ++hh, ++x) {
+          if (x >= 3) mbar_wait(b_done + 8 * b, ph ^ 1, &abort_flag, 203);
+          tc_fence_after();
+          const uint32_t kt = smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes) + hh * 32 * C::kRowBytes;
+          const uint64_t dkd = smem_desc(kt, 16, C::kAtomBytes, C::kSwizzle);
+          const uint64_t dvd = smem_desc(kt + C::kSmallBytes, 16, C::kAtomBytes, C::kSwizzle);
+          const uint32_t ts = tmem_base + 64 * b;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dqd + 2 * k, dkd + 2 * k, idesc_s, k > 0);
+            for (int k = 0; k < D / 16; ++k) umma_bf16(ts, dqd + 2 * k, dkd + 2 * k, idesc_s, k > 0);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dgd + 2 * k, dvd + 2 * k, idesc_s, k > 0);
-          umma_commit(b_sfull);
+            for (int k = 0; k < D / 16; ++k) umma_bf16(ts + 32, dgd + 2 * k, dvd + 2 * k, idesc_s, k > 0);
+            umma_commit(b_sfull + 8 * b);
+          }
+          __syncwarp();
+          if (++b == 3) {
+            b = 0;
+            ph ^= 1;
+          }
         }
-        __syncwarp();
       }
     } else if (warp == kComputeWarps + 2 && nvis > 0) {
-      // ---- dQ += dS K of tile i (dS from tensor memory, K MN-major) ----
+      // ---- dQ += dS K of a half tile (dS from tensor memory, K MN-major) ----
       constexpr uint32_t idesc_dq = instr_desc(128, D, 0, 1);
-      for (int i = 0; i < nvis; ++i) {
+      for (int i = 0, b = 0, ph = 0; i < nvis; ++i) {
         const uint64_t dkm = smem_desc(smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes), C::kSmallBytes,
                                        C::kAtomBytes, C::kSwizzle);
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 206);
-        mbar_wait(b_tfull, i & 1, &abort_flag, 204);
-        tc_fence_after();
-        if (elect_one()) {
+        for (int hh = 0; hh < 2; ++hh) {
+          mbar_wait(b_tfull + 8 * b, ph, &abort_flag, 204);
+          tc_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16_ts(tmem_dq, tmem_ds + 8 * k, dkm + k * C::kKStep, idesc_dq, (i | k) != 0);
-          umma_commit(b_done);
-          umma_commit(b_empty + 8 * (i % STAGES));  // S(i), dP(i) completed before the compute warps read them
+            for (int kk = 0; kk < 2; ++kk)
+              umma_bf16_ts(tmem_dq, tmem_base + 64 * b + 16 * kk, dkm + (2 * hh + kk) * C::kKStep, idesc_dq,
+                           (i | hh | kk) != 0);
+            umma_commit(b_done + 8 * b);
+            if (hh == 1) umma_commit(b_empty + 8 * (i % STAGES));  // every product on this stage has completed
+          }
+          __syncwarp();
+          if (++b == 3) {
+            b = 0;
+            ph ^= 1;
+          }
         }
-        __syncwarp();
       }
     }
   } else {
@@ -306,8 +324,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
       nDS = rec[6];
     }
     float2 dalL = make_float2(0.f, 0.f), dalS = make_float2(0.f, 0.f);  // sums of P' dP per branch
-    bool ds_zero = false;
     const float sc2 = s.scale * kLog2e;
+    int b = 0, ph = 0;  // buffer x % 3 of half tile x = 2 i + hh and the parity (x / 3) & 1
 
     for (int i = 0; i < nvis; ++i) {
       const int jt = list[i], f = lflags[i], p0 = jt * 64;
@@ -317,67 +335,45 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
         if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
       }
-      const uint32_t hL = (uint32_t)(maskL >> (half * 32)), hS = (uint32_t)(maskS >> (half * 32));
-      const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);
-      const bool full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffffffu) && (!anyS || hS == 0xffffffffu));
-
-      mbar_wait(b_sfull, i & 1, &abort_flag, 207);
-      __syncwarp();
-      tc_fence_after();
-      const bool mine = anyL || anyS;
-      if (mine || !ds_zero) {
-        // two passes of 16 columns (a rolled loop: one copy of each code path)
 #pragma unroll 1
-        for (int q = 0; q < 2; ++q) {
+      for (int hh = 0; hh < 2; ++hh) {
+        // this thread's 16 keys of the half tile: keys 32 hh + 16 half ... of the tile
+        const uint32_t hL = (uint32_t)(maskL >> (32 * hh + 16 * half)) & 0xffffu;
+        const uint32_t hS = (uint32_t)(maskS >> (32 * hh + 16 * half)) & 0xffffu;
+        const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);
+        const bool full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffu) && (!anyS || hS == 0xffffu));
+        const uint32_t tb = tmem_base + 64 * b + lane_off + 16 * half;  // S; dP 32 columns further
+
+        mbar_wait(b_sfull + 8 * b, ph, &abort_flag, 207);
+        __syncwarp();
+        tc_fence_after();
+        uint32_t dw[8];
+        if (anyL || anyS) {
           float sv[16], dp[16];
-          uint32_t dw[8];
-          if (mine) {
-            tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
-            tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
-            tmem_wait_ld();
-          }
-          if (q == 1) {  // S and dP of this tile are in registers: the next tile's may overwrite them
-            tc_fence_before();
-            warp_arrive(b_sempty, lane);
-          }
-          const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
-          if (!mine) {
+          tmem_ld16(tb, sv);
+          tmem_ld16(tb + 32, dp);
+          tmem_wait_ld();
+          if (!full) dq_tile<true, true, false>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+          else if (anyL && anyS) dq_tile<true, true, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+          else if (anyL) dq_tile<true, false, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+          else dq_tile<false, true, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+        } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) dw[c] = 0u;
-          } else if (!full) {
-            dq_tile<true, true, false>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          } else if (anyL && anyS) {
-            dq_tile<true, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          } else if (anyL) {
-            dq_tile<true, false, true>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          } else {
-            dq_tile<false, true, true>(sv, dp, qL, qS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          }
-          if (q == 0 && i >= 1) {  // the dS columns are free once dQ += dS K of tile i-1 has completed
-            mbar_wait(b_done, (i - 1) & 1, &abort_flag, 208);
-            __syncwarp();
-            tc_fence_after();
-          }
-          tmem_st8u(tmem_ds + lane_off + half * 16 + q * 8, dw);
+          for (int c = 0; c < 8; ++c) dw[c] = 0u;
         }
+        tmem_st8u(tb, dw);  // dS (bf16 pairs) over the first 8 of this thread's own 16 S columns
         tmem_wait_st();
-        ds_zero = !mine;
-      } else {
         tc_fence_before();
-        warp_arrive(b_sempty, lane);
-        if (i >= 1) {
-          // nothing to write, but keep in step with the barrier: a parity wait only tells the last
-          // two phases apart, so no warp may fall further behind than that
-          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 219);
-          __syncwarp();
+        warp_arrive(b_tfull + 8 * b, lane);
+        if (++b == 3) {
+          b = 0;
+          ph ^= 1;
         }
       }
-      tc_fence_before();
-      warp_arrive(b_tfull, lane);
     }
 
     if (nvis > 0) {
-      mbar_wait(b_done, (nvis - 1) & 1, &abort_flag, 209);
+      mbar_wait(b_done + 8 * ((2 * nvis - 1) % 3), ((2 * nvis - 1) / 3) & 1, &abort_flag, 209);
       __syncwarp();
       tc_fence_after();
     }

@@ -38,7 +38,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int image = (int)blockIdx.x * kMetaWarps + warp;
   if (image >= n_images) return;
-  uint8_t *meta = meta_all + (size_t)warp * ml.bytes;
+  const int slice = ml.bytes + ((3 * nT + 15) / 16) * 16;  // the image and a scratch list behind it
+  uint8_t *meta = meta_all + (size_t)warp * slice;
   const int nST = (s.L + 127) >> 7;
   const bool key_major = image >= n_query_ctas;
   const int cta = key_major ? image - n_query_ctas : image;
@@ -168,6 +169,58 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
       icls[e] = (uint8_t)cls;
     }
+    __syncwarp();
+    // The dQ kernel walks `list` itself (a tile serves both branches there).  Same idea as above:
+    // tiles both 64-row halves need first, then alternately a tile only rows 0..63 need and one
+    // only rows 64..127 need, so that the two halves' warps work on neighbouring tiles at once.
+    {
+      uint16_t *tlist = reinterpret_cast<uint16_t *>(meta + ml.bytes);
+      uint8_t *tflags = meta + ml.bytes + 2 * nT;
+      int nA = 0, nB = 0, nC = 0;
+      for (int pass = 0; pass < 2; ++pass) {
+        int cA = 0, cB = 0, cC = 0;
+        for (int base = 0; base < nv; base += 32) {
+          const int j = base + lane;
+          int c = 0;
+          if (j < nv) {
+            const int jt = list[j], p0 = jt * 64;
+            if (lflags[j] & 1)
+              for (int g = 0; g < G; ++g)
+                if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
+            if (lflags[j] & 2)
+              for (int hf = 0; hf < 2; ++hf)
+                if (p0 + 63 >= row0 + 64 * hf - s.window + 1 && p0 <= row0 + 64 * hf + 63) c |= 1 << hf;
+            if (c == 0) c = 3;
+          }
+          const unsigned bA = __ballot_sync(0xffffffffu, c == 1), bB = __ballot_sync(0xffffffffu, c == 2),
+                         bC = __ballot_sync(0xffffffffu, c == 3);
+          if (pass == 1 && c) {
+            int pos;
+            if (c == 3) pos = cC + __popc(bC & lt);
+            else if (c == 1) {
+              const int k = cA + __popc(bA & lt);
+              pos = nC + (k < nB ? 2 * k : nB + k);
+            } else {
+              const int k = cB + __popc(bB & lt);
+              pos = nC + (k < nA ? 2 * k + 1 : nA + k);
+            }
+            tlist[pos] = list[j];
+            tflags[pos] = lflags[j];
+          }
+          cA += __popc(bA);
+          cB += __popc(bB);
+          cC += __popc(bC);
+        }
+        nA = cA;
+        nB = cB;
+        nC = cC;
+      }
+      __syncwarp();
+      for (int j = lane; j < nv; j += 32) {
+        list[j] = tlist[j];
+        lflags[j] = tflags[j];
+      }
+    }
   } else {
     const int kt = cta % nST;  // the dK/dV kernel takes early keys first
     const int key0 = kt * 128, key_last = min(s.L - 1, key0 + 127);
@@ -224,7 +277,7 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
                    uint8_t *kmeta, cudaStream_t st) {
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const int nq = nST * s.B * s.H, n_images = kmeta ? 2 * nq : nq;
-  const size_t smem = (size_t)kMetaWarps * meta_bytes(nT);
+  const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT) + ((3 * nT + 15) / 16) * 16);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(tc_meta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
