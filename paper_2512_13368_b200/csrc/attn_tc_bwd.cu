@@ -189,6 +189,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   const uint8_t *selb = meta;
   const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
   const uint8_t *lflags = meta + ml.flags;
+  const uint8_t *jcls = meta + ml.jcls;  // [tile][half tile][compute warp]
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_meta = smem_u32(&bars[2 * STAGES + 1]);
@@ -327,48 +328,52 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     const float sc2 = s.scale * kLog2e;
     int b = 0, ph = 0;  // buffer x % 3 of half tile x = 2 i + hh and the parity (x / 3) & 1
 
-    for (int i = 0; i < nvis; ++i) {
-      const int jt = list[i], f = lflags[i], p0 = jt * 64;
-      uint64_t maskL = 0ull, maskS = 0ull;
-      if (row_valid) {
-        const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
-        if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
-        if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
+    int cls_n = nvis > 0 ? jcls[warp] : 0;
+    for (int x = 0; x < 2 * nvis; ++x) {  // half tile x: keys 32 (x % 2) ... of tile list[x / 2]
+      const int cls = cls_n;
+      if (x + 1 < 2 * nvis) cls_n = jcls[(x + 1) * kComputeWarps + warp];  // ahead of its use
+      uint32_t hL = 0u, hS = 0u;  // this thread's 16 keys: keys 32 (x % 2) + 16 half ... of the tile
+      bool anyL = cls & 1, anyS = cls & 2, full = true;
+      if (cls & 8) {  // mixed: per-lane column masks
+        const int i = x >> 1, jt = list[i], f = lflags[i], p0 = jt * 64;
+        uint64_t maskL = 0ull, maskS = 0ull;
+        if (row_valid) {
+          const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
+          if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
+          if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
+        }
+        hL = (uint32_t)(maskL >> (32 * (x & 1) + 16 * half)) & 0xffffu;
+        hS = (uint32_t)(maskS >> (32 * (x & 1) + 16 * half)) & 0xffffu;
+        anyL = __any_sync(0xffffffffu, hL != 0u);
+        anyS = __any_sync(0xffffffffu, hS != 0u);
+        full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffu) && (!anyS || hS == 0xffffu));
       }
-#pragma unroll 1
-      for (int hh = 0; hh < 2; ++hh) {
-        // this thread's 16 keys of the half tile: keys 32 hh + 16 half ... of the tile
-        const uint32_t hL = (uint32_t)(maskL >> (32 * hh + 16 * half)) & 0xffffu;
-        const uint32_t hS = (uint32_t)(maskS >> (32 * hh + 16 * half)) & 0xffffu;
-        const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);
-        const bool full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffu) && (!anyS || hS == 0xffffu));
-        const uint32_t tb = tmem_base + 64 * b + lane_off + 16 * half;  // S; dP 32 columns further
+      const uint32_t tb = tmem_base + 64 * b + lane_off + 16 * half;  // S; dP 32 columns further
 
-        mbar_wait(b_sfull + 8 * b, ph, &abort_flag, 207);
-        __syncwarp();
-        tc_fence_after();
-        uint32_t dw[8];
-        if (anyL || anyS) {
-          float sv[16], dp[16];
-          tmem_ld16(tb, sv);
-          tmem_ld16(tb + 32, dp);
-          tmem_wait_ld();
-          if (!full) dq_tile<true, true, false>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          else if (anyL && anyS) dq_tile<true, true, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          else if (anyL) dq_tile<true, false, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-          else dq_tile<false, true, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
-        } else {
+      mbar_wait(b_sfull + 8 * b, ph, &abort_flag, 207);
+      __syncwarp();
+      tc_fence_after();
+      uint32_t dw[8];
+      if (anyL || anyS) {
+        float sv[16], dp[16];
+        tmem_ld16(tb, sv);
+        tmem_ld16(tb + 32, dp);
+        tmem_wait_ld();
+        if (!full) dq_tile<true, true, false>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+        else if (anyL && anyS) dq_tile<true, true, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+        else if (anyL) dq_tile<true, false, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+        else dq_tile<false, true, true>(sv, dp, hL, hS, sc2, nlL, nlS, nDL, nDS, dalL, dalS, dw);
+      } else {
 #pragma unroll
-          for (int c = 0; c < 8; ++c) dw[c] = 0u;
-        }
-        tmem_st8u(tb, dw);  // dS (bf16 pairs) over the first 8 of this thread's own 16 S columns
-        tmem_wait_st();
-        tc_fence_before();
-        warp_arrive(b_tfull + 8 * b, lane);
-        if (++b == 3) {
-          b = 0;
-          ph ^= 1;
-        }
+        for (int c = 0; c < 8; ++c) dw[c] = 0u;
+      }
+      tmem_st8u(tb, dw);  // dS (bf16 pairs) over the first 8 of this thread's own 16 S columns
+      tmem_wait_st();
+      tc_fence_before();
+      warp_arrive(b_tfull + 8 * b, lane);
+      if (++b == 3) {
+        b = 0;
+        ph ^= 1;
       }
     }
 

@@ -14,6 +14,7 @@
 //                             block lies in the tile, bit 1: the window of some row reaches it
 //   items[2 nT], icls[2 nT][4] (forward) the long-term tiles, then the short-term tiles, and the
 //                             class of every (item, softmax warp)
+//   jcls[nT][2][8]            (dQ) class of every (listed tile, half tile, compute warp)
 //   counts                    {tiles on the list, long-term items, short-term items}
 // Key-major image (dK/dV kernel): [8][nT] bytes: bit c of byte (g, qt): query block
 // qt * (64 / Bk) + c selected key block g of the CTA; list / flags of the 64-query tiles that
@@ -53,9 +54,11 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   uint8_t *lflags = meta + ml.flags;
   uint16_t *items = reinterpret_cast<uint16_t *>(meta + ml.items);
   uint8_t *icls = meta + ml.icls;
+  uint8_t *jcls = meta + ml.jcls;
   int *counts = reinterpret_cast<int *>(meta + ml.counts);
   const unsigned lt = (1u << lane) - 1u;
   const int G = 128 / s.Bk, nb = 64 / s.Bk;
+  const int bk_shift = __ffs(s.Bk) - 1;  // Bk is a power of two
 
   for (int i = lane; i < ml.bytes / 4; i += 32) selw[i] = 0u;  // the whole image
   __syncwarp();
@@ -220,6 +223,33 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         list[j] = tlist[j];
         lflags[j] = tflags[j];
       }
+    }
+    __syncwarp();
+    // dQ kernel: class of every (listed tile, half tile of 32 keys, compute warp).  Warp w works
+    // on rows 32 (w % 4) ... and keys 16 (w / 4) ... of the half tile.  Bit 0 / bit 1: every row of
+    // the warp sees all 16 keys through the long-term / short-term branch and no row sees only a
+    // part of them; 8: mixed, the warp builds per-lane column masks.  (A forward-only call has no
+    // use for them.)
+    for (int e = lane; e < (kmeta ? nv * 16 : 0); e += 32) {
+      const int it = e >> 4, hh = (e >> 3) & 1, w = e & 7, qtr = w & 3, c = w >> 2;
+      const int jt = list[it], f = lflags[it];
+      const int k_lo = jt * 64 + 32 * hh + 16 * c, k_hi = k_lo + 15, t_lo = row0 + qtr * 32, t_hi = t_lo + 31;
+      const bool rows_in = t_lo >= pad0 && t_hi < s.L, rows_none = t_hi < pad0 || t_lo >= s.L;
+      const bool past = rows_in && k_lo >= pad0 && k_hi <= t_lo;  // every key causally visible to every row
+      const bool reach = !rows_none && k_lo <= t_hi && k_hi >= pad0;  // some key may be visible to some row
+      int cL = 0, cS = 0;  // 0 none, 1 all, 2 mixed
+      if ((f & 1) && reach) {
+        const int kb = (32 * hh + 16 * c) >> bk_shift;  // key block within the tile
+        bool any_sel = false, all_sel = true;
+        for (int gq = (qtr * 32) >> bk_shift; gq <= (qtr * 32 + 31) >> bk_shift; ++gq) {
+          const bool sel = (selb[gq * nT + jt] >> kb) & 1u;
+          any_sel |= sel;
+          all_sel &= sel;
+        }
+        if (any_sel) cL = (all_sel && past) ? 1 : 2;
+      }
+      if ((f & 2) && reach && k_hi >= t_lo - s.window + 1) cS = (past && k_lo >= t_hi - s.window + 1) ? 1 : 2;
+      jcls[e] = (uint8_t)((cL == 2 || cS == 2) ? 8 : (cL | (cS << 1)));
     }
   } else {
     const int kt = cta % nST;  // the dK/dV kernel takes early keys first

@@ -377,10 +377,11 @@ struct Cfg {
 
 // Per-CTA tile bookkeeping, built once per call by tc_meta_kernel and brought into shared memory
 // by one bulk copy: [8][nT] selection bytes, nT list entries, nT flags, (forward) 2 nT per-phase
-// items with 4 class bytes each, and the counts {tiles on the list, long-term items, short-term
-// items}.  Offsets in bytes; every part starts on a 16-byte boundary where a copy needs it.
+// items with 4 class bytes each, (dQ kernel) 16 class bytes per listed tile, and the counts {tiles
+// on the list, long-term items, short-term items}.  Offsets in bytes; every part starts on a
+// 16-byte boundary where a copy needs it.
 struct MetaLayout {
-  int list, flags, items, icls, counts, bytes;
+  int list, flags, items, icls, jcls, counts, bytes;
 };
 __host__ __device__ inline MetaLayout meta_layout(int nT) {
   MetaLayout m;
@@ -388,7 +389,8 @@ __host__ __device__ inline MetaLayout meta_layout(int nT) {
   m.flags = m.list + 2 * nT;
   m.items = ((m.flags + nT + 15) / 16) * 16;
   m.icls = m.items + 4 * nT;
-  m.counts = ((m.icls + 8 * nT + 15) / 16) * 16;
+  m.jcls = ((m.icls + 8 * nT + 15) / 16) * 16;
+  m.counts = m.jcls + 16 * nT;
   m.bytes = m.counts + 16;
   return m;
 }
