@@ -69,8 +69,8 @@ __global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restri
 
 // ---- Eq. 10 + 12 + 13: scores of one query block and its top-k --------------------------
 // grid M*B*H (unit-major), 256 threads.  One warp per query row: lanes stride over the candidate blocks,
-// softmax over the candidates, per-warp partial sums, fixed-order combine, then warp 0 runs
-// top_k - 1 arg-max passes (value desc, index asc).
+// softmax over the candidates, per-warp partial sums, fixed-order combine, then a candidate is
+// kept iff fewer than top_k - 1 live candidates beat it (value desc, index asc).
 template <typename T, int D>
 __device__ __forceinline__ void score_select_row(
     const Shape &s, const T *__restrict__ q, const double *__restrict__ kmean,
@@ -117,18 +117,38 @@ __device__ __forceinline__ void score_select_row(
 
   if (ncand > 0 && s.topk > 1) {
     double *zw = zbuf + warp * M, *spw = sp + warp * M, *qw = qrow + warp * D;
+    constexpr int QPL = (D + 31) / 32;  // query elements per lane
+    double qreg[QPL];                   // the next row, loaded while the current one is scored
+    if (qlo + warp < qhi) {
+      const T *qp = q + row_offset(s, n, h, qlo + warp);
+#pragma unroll
+      for (int e = 0; e < QPL; ++e)
+        if (lane + 32 * e < D) qreg[e] = (double)ld1(qp + lane + 32 * e);
+    }
     for (int t = qlo + warp; t < qhi; t += kSelWarps) {
-      const T *qp = q + row_offset(s, n, h, t);
-      for (int c = lane; c < D; c += 32) qw[c] = (double)ld1(qp + c);
+#pragma unroll
+      for (int e = 0; e < QPL; ++e)
+        if (lane + 32 * e < D) qw[lane + 32 * e] = qreg[e];
       __syncwarp();
+      if (t + kSelWarps < qhi) {
+        const T *qp = q + row_offset(s, n, h, t + kSelWarps);
+#pragma unroll
+        for (int e = 0; e < QPL; ++e)
+          if (lane + 32 * e < D) qreg[e] = (double)ld1(qp + lane + 32 * e);
+      }
       double mx = -INFINITY;
       for (int j = lane; j < b; j += 32) {
         if (!live[j]) continue;
         const double *kj = kt + (int64_t)j * kstride;
-        double acc = 0.0;
-#pragma unroll 8
-        for (int c = 0; c < D; ++c) acc += qw[c] * kj[c];
-        const double z = s.scale_d * acc;
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;  // four chains: the FMA latency overlaps
+#pragma unroll 4
+        for (int c = 0; c < D; c += 4) {
+          a0 = fma(qw[c], kj[c], a0);
+          a1 = fma(qw[c + 1], kj[c + 1], a1);
+          a2 = fma(qw[c + 2], kj[c + 2], a2);
+          a3 = fma(qw[c + 3], kj[c + 3], a3);
+        }
+        const double z = s.scale_d * ((a0 + a1) + (a2 + a3));
         zw[j] = z;
         mx = fmax(mx, z);
       }
@@ -156,28 +176,25 @@ __device__ __forceinline__ void score_select_row(
   }
   __syncthreads();
 
-  if (warp == 0) {
+  {
+    // Selection by rank: candidate j is kept iff fewer than `want` live candidates beat it (larger
+    // score, or equal score and lower index).
     const int want = min(s.topk - 1, ncand);
-    for (int r = 0; r < want; ++r) {
-      double bv = -INFINITY;
-      int bj = 0x7fffffff;
-      for (int j = lane; j < b; j += 32) {
-        if (!live[j] || taken[j]) continue;
-        const double vj = S[j];
-        if (bj == 0x7fffffff || vj > bv) { bv = vj; bj = j; }  // ascending j: strict > keeps lower
+    for (int j = tid; j < b; j += kSelThreads) {
+      int rank = 0;
+      if (live[j]) {
+        const double sj = S[j];
+        for (int i = 0; i < b; ++i)
+          if (live[i]) {
+            const double si = S[i];
+            rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
+          }
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const double ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-        if (oj != 0x7fffffff && (bj == 0x7fffffff || ov > bv || (ov == bv && oj < bj))) {
-          bv = ov;
-          bj = oj;
-        }
-      }
-      if (lane == 0) taken[bj] = 1;
-      __syncwarp();
+      taken[j] = live[j] && rank < want;
     }
+  }
+  __syncthreads();
+  if (warp == 0) {
     // emit ascending: ballot over 32-wide chunks of the flags, then the own block
     int pos = 0;
     for (int base = 0; base < b; base += 32) {
