@@ -21,6 +21,9 @@
  *   top-k selection      Eq. 13 own block always kept, ties -> lower index
  *   selected-KV attention Eq. 14 + Eq. 16 (via Eq. 1 with the causal mask)
  *   window attention     Eq. 15 first case (|i-j| < w), causal side, Eq. 17
+ *   power-law mask       Eq. 15 all three cases (stis_mode 1), causal side:
+ *                               window, block-index distance a power of two,
+ *                               the last blk positions
  *   gate combine         Eq. 19 with alpha_h = sigmoid(a[h][0] - a[h][1])
  *   backward             chain rule through Eq. 19, Eq. 16/17 and Eq. 1 with
  *                        the selection frozen (top-k is piecewise constant)
@@ -195,20 +198,40 @@ static int ltis_keys(int L, int Bk, int topk, int pad0, const int32_t *row, int 
   return nk;
 }
 
-/* key list of the short-term branch (Eq. 15 first case, causal side): t - w < p <= t, valid */
-static int stis_keys(int w, int pad0, int t, int *keys) {
+/* Eq. 15, one (query i, key j) pair: 1 if the short-term branch lets i attend to j.
+ *   mode 0: the window alone, |i - j| < w;
+ *   mode 1: the paper's power-law mask: the window, or the block-index distance
+ *           |floor(i/blk) - floor(j/blk)| is 2^r for some integer r >= 0, or j is one of
+ *           the last blk positions of the sequence array. */
+static int stis_mask(int mode, int w, int blk, int L, int i, int j) {
+  int d = i > j ? i - j : j - i;
+  if (d < w) return 1;
+  if (mode == 0) return 0;
+  int bd = i / blk - j / blk;
+  if (bd < 0) bd = -bd;
+  if (bd >= 1 && (bd & (bd - 1)) == 0) return 1; /* a power of two */
+  if (j >= L - blk) return 1;
+  return 0;
+}
+
+/* key list of the short-term branch: Eq. 15 restricted to the causal side (p <= t) and to the
+ * valid (non-padding) positions */
+static int stis_keys(int mode, int w, int blk, int L, int pad0, int t, int *keys) {
   int nk = 0;
-  for (int p = imax(pad0, t - w + 1); p <= t; ++p) keys[nk++] = p;
+  for (int p = pad0; p <= t; ++p)
+    if (stis_mask(mode, w, blk, L, t, p)) keys[nk++] = p;
   return nk;
 }
 
 static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 
-int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int window, double scale,
+int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
+                           int stis_blk, double scale,
                            const double *q, const double *k, const double *v, const double *gate,
                            const int32_t *seq_lens, const int32_t *idx, double *out,
                            double *out_lt, double *out_st, double *lse) {
   if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1 || window < 1) return 1;
+  if (stis_mode < 0 || stis_mode > 1 || stis_blk < 1) return 1;
   const int M = n_blocks(L, Bk);
   const size_t BHL = (size_t)B * H * L;
 #pragma omp parallel for collapse(2) schedule(dynamic)
@@ -234,7 +257,7 @@ int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int win
           const int32_t *row = idx + (u * M + (size_t)(t / Bk)) * topk;
           int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
           lL = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oL); /* Eq. 16 */
-          nk = stis_keys(window, pad0, t, keys);
+          nk = stis_keys(stis_mode, window, stis_blk, L, pad0, t, keys);
           lS = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oS); /* Eq. 17 */
         }
         for (int c = 0; c < D; ++c) {
@@ -279,12 +302,14 @@ static void attend_row_bwd(int D, double scale, const double *qt, const double *
   }
 }
 
-int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int window, double scale,
+int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
+                            int stis_blk, double scale,
                             const double *q, const double *k, const double *v, const double *gate,
                             const int32_t *seq_lens, const int32_t *idx, const double *out_lt,
                             const double *out_st, const double *lse, const double *dout,
                             double *dq, double *dk, double *dv, double *dgate) {
   if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1 || window < 1) return 1;
+  if (stis_mode < 0 || stis_mode > 1 || stis_blk < 1) return 1;
   const int M = n_blocks(L, Bk);
   const size_t BHL = (size_t)B * H * L;
   double *dalpha_unit = (double *)calloc((size_t)B * H, sizeof(double));
@@ -317,7 +342,7 @@ int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int wi
         int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
         attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[u * L + t],
                        out_lt + ro, gL, dqu + (size_t)t * D, dku, dvu);
-        nk = stis_keys(window, pad0, t, keys);
+        nk = stis_keys(stis_mode, window, stis_blk, L, pad0, t, keys);
         attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[BHL + u * L + t],
                        out_st + ro, gS, dqu + (size_t)t * D, dku, dvu);
       }

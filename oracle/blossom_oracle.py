@@ -50,10 +50,10 @@ def _load():
         lib.blossom_oracle_select.restype = i
         lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp]
         lib.blossom_oracle_forward.restype = i
-        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
         lib.blossom_oracle_backward.restype = i
-        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                 _ip, _dp, _dp, _dp, _dp, _dp, _dp, _dp, _dp]
         _lib = lib
     return _lib
@@ -100,8 +100,12 @@ def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores
     return (idx, scores) if return_scores else idx
 
 
-def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None):
+def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None,
+            stis_mode=0, stis_block=1):
     """Eq. 14, 16, 17, 19.  ``idx`` overrides the selection when given.
+
+    ``stis_mode`` 0: the short-term branch is the causal window (Eq. 15, first case);
+    1: the power-law mask (all of Eq. 15, causal side) with mask block ``stis_block``.
 
     Returns a dict: out, out_lt, out_st ``[B,H,L,D]``, lse ``[2,B,H,L]``, idx.
     """
@@ -118,7 +122,8 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     out_lt = np.empty_like(q)
     out_st = np.empty_like(q)
     lse = np.empty((2, B, H, L), dtype=np.float64)
-    rc = _load().blossom_oracle_forward(B, H, L, D, block, topk, window, _scale(sm_scale, D),
+    rc = _load().blossom_oracle_forward(B, H, L, D, block, topk, window, int(stis_mode),
+                                        int(stis_block), _scale(sm_scale, D),
                                         _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp), _ptr(gate, _dp),
                                         _ptr(sl, _ip), _ptr(idx, _ip), _ptr(out, _dp),
                                         _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp))
@@ -127,7 +132,8 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     return {"out": out, "out_lt": out_lt, "out_st": out_st, "lse": lse, "idx": idx}
 
 
-def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None):
+def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None,
+             stis_mode=0, stis_block=1):
     """Gradients of sum(out * dout) with the selection frozen.
 
     ``fwd`` is the dict ``forward`` returned.  Returns dq, dk, dv, dgate ``[H,2]``.
@@ -139,7 +145,8 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
     out_lt, out_st, lse = _f64(fwd["out_lt"]), _f64(fwd["out_st"]), _f64(fwd["lse"])
     dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
     dgate = np.empty((H, 2), dtype=np.float64)
-    rc = _load().blossom_oracle_backward(B, H, L, D, block, topk, window, _scale(sm_scale, D),
+    rc = _load().blossom_oracle_backward(B, H, L, D, block, topk, window, int(stis_mode),
+                                         int(stis_block), _scale(sm_scale, D),
                                          _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp),
                                          _ptr(gate, _dp), _ptr(sl, _ip), _ptr(idx, _ip),
                                          _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp),
@@ -151,9 +158,10 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
 
 
 def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm_scale=None,
-                     idx=None):
+                     idx=None, stis_mode=0, stis_block=1):
     """Convenience: forward then backward; returns the two dicts merged."""
-    f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx)
-    b = backward(q, k, v, gate, block, topk, window, f, dout, seq_lens, sm_scale)
+    f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx, stis_mode, stis_block)
+    b = backward(q, k, v, gate, block, topk, window, f, dout, seq_lens, sm_scale, stis_mode,
+                 stis_block)
     f.update(b)
     return f
