@@ -66,6 +66,23 @@ def work_model(w):
             tl += min(w.topk, qb - first + 1)
             lo_pos = max(pad0, qb * Bk - (w.window - 1))
             ts += qb - lo_pos // Bk + 1
+        if w.stis_mode == 1:
+            # power-law mask: the work is counted per (query, key) pair of Eq. 15 and expressed in
+            # tiles of Bk x Bk pairs (fractional), since its links do not fill tiles
+            t = np.arange(pad0, w.L)
+            pairs = np.minimum(t - pad0 + 1, w.window).astype(np.float64)
+            blk, r = w.stis_block, 0
+            while (1 << r) * blk <= w.L:
+                d = 1 << r
+                kb = t // blk - d                      # the key block at distance 2^r
+                lo = np.maximum(kb * blk, pad0)
+                hi = np.minimum(kb * blk + blk - 1, t - w.window)   # keys the window does not hold already
+                pairs += np.maximum(hi - lo + 1, 0) * (kb >= 0)
+                r += 1
+            lastlo = np.maximum(w.L - blk, pad0)
+            own = (t // blk) * blk                       # last-block keys: distance 0 only, beyond the window
+            pairs += np.maximum(np.minimum(t - w.window, t) - np.maximum(lastlo, own) + 1, 0) * (t >= lastlo)
+            ts = float(pairs.sum()) / (Bk * Bk)
         tiles_L += cnt * tl * w.H
         tiles_S += cnt * ts * w.H
     esz = 2 if w.dtype == "bf16" else 4
@@ -150,14 +167,14 @@ def oracle_sample(w, max_batch):
     sl = None if w.seq_lens is None else w.seq_lens[:nb].copy()
     return Workload(w.name + f"[first {nb} of {w.B} batch entries]", w.dtype, nb, w.H, w.L, w.D,
                     w.block, w.topk, w.window, w.seed, w.q[:nb], w.k[:nb], w.v[:nb], w.gate,
-                    w.dout[:nb], sl)
+                    w.dout[:nb], sl, w.stis_mode, w.stis_block)
 
 
 def time_oracle(ws):
     import oracle
     t0 = time.perf_counter()
     oracle.forward_backward(ws.q, ws.k, ws.v, ws.gate, ws.dout, ws.block, ws.topk, ws.window,
-                            ws.seq_lens)
+                            ws.seq_lens, stis_mode=ws.stis_mode, stis_block=ws.stis_block)
     return time.perf_counter() - t0
 
 
@@ -193,6 +210,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--short-term", default="window", choices=["window", "power-law"],
+                    help="short-term branch: the configuration's causal window (headline) or the "
+                         "power-law mask of Eq. 15 with --mask-window and --mask-block")
+    ap.add_argument("--mask-window", type=int, default=8, help="w of the power-law mask (paper: 8 blocks of 1)")
+    ap.add_argument("--mask-block", type=int, default=1, help="blk of the power-law mask")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the batch size (profiling captures on a smaller case; not a bench line)")
     args = ap.parse_args()
@@ -206,8 +228,12 @@ def main():
         return 0
     w = workloads.CONFIGS[args.config](B=args.batch) if (args.batch and args.config != 1) \
         else workloads.CONFIGS[args.config]()
+    if args.short_term == "power-law":
+        w.stis_mode, w.stis_block, w.window = 1, args.mask_block, args.mask_window
+        w.name += f"+powerlaw(w{args.mask_window},blk{args.mask_block})"
     cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "seq_len": w.L, "head_dim": w.D,
-                "block_size": w.block, "top_k": w.topk, "window": w.window, "storage": w.dtype,
+                "block_size": w.block, "top_k": w.topk, "window": w.window, "short_term": args.short_term,
+                "mask_block": w.stis_block if w.stis_mode else None, "storage": w.dtype,
                 "padding": "left, lengths U{5..200}" if w.seq_lens is not None else "none",
                 "l2": "no flush: a step touches ~1 GB of distinct tensors, more than the 126 MB L2"
                 if w.B * w.H * w.L * w.D * 2 * 15 > 4 * 126e6 else

@@ -62,12 +62,17 @@ typedef struct {
   int32_t head_dim;    /* D in {32, 64}                                                          */
   int32_t block_size;  /* key block = query block size Bk in {8, 16, 32, 64}                     */
   int32_t top_k;       /* 1 <= top_k <= 64 blocks per query block, the own block included        */
-  int32_t window;      /* w >= 1: query t sees keys t - w < p <= t in the short-term branch      */
+  int32_t window;      /* w >= 1: query t sees keys t - w < p <= t in the short-term branch (and
+                        * more with stis_mode 1)                                                 */
   int32_t causal;      /* must be 1                                                              */
   int32_t select_mode; /* 0 = one selection per query block (the only mode implemented)          */
   int32_t dtype;       /* BLOSSOM_DTYPE_FP32 or BLOSSOM_DTYPE_BF16                               */
   float sm_scale;      /* 0 -> 1/sqrt(head_dim); scales block scores and attention logits alike  */
   int64_t stride_b, stride_h, stride_l; /* element strides of every q-shaped tensor              */
+  int32_t stis_mode;   /* short-term branch: 0 = causal window only; 1 = the power-law mask of
+                        * Eq. 15: window, or block-index distance floor(t/blk) - floor(p/blk) a
+                        * power of two, or p among the last blk positions (all with p <= t)      */
+  int32_t stis_block;  /* blk >= 1 of the power-law mask (0 reads as 1); ignored in mode 0       */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);
@@ -125,9 +130,11 @@ int blossom_select_blocks_static(const blossom_params *params /* host */, const 
                                  blossom_stream_t stream);
 
 /*
- * Forward (paper: Eq. 14 and 16 for the selected-block branch, Eq. 15 first case under the
- * causal mask and Eq. 17 for the window branch, Eq. 19 for the gate, each branch being the
- * masked softmax attention of Eq. 1 with online softmax in fp32).
+ * Forward (paper: Eq. 14 and 16 for the selected-block branch, Eq. 15 under the causal mask
+ * (its first case alone with stis_mode 0, all three with stis_mode 1) and Eq. 17 for the
+ * short-term branch, Eq. 19 for the gate, each branch being the masked softmax attention of
+ * Eq. 1 with online softmax in fp32).  With stis_mode 1 every dtype runs on the CUDA-core
+ * kernels.
  *   q, k, v      in   q-shaped
  *   gate_logits  in   [H][2]
  *   seq_lens     in   [B] or NULL

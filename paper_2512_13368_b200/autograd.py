@@ -16,7 +16,8 @@ _DT = {torch.float32: "fp32", torch.bfloat16: "bf16"}
 
 class _BlossomAttention(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale):
+    def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
+                stis_mode, stis_block):
         if q.dtype not in _DT or k.dtype != q.dtype or v.dtype != q.dtype:
             raise TypeError("q, k, v must share one dtype, float32 or bfloat16")
         if not (q.is_cuda and q.shape == k.shape == v.shape and q.dim() == 4):
@@ -25,7 +26,8 @@ class _BlossomAttention(torch.autograd.Function):
             q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
         B, H, L, D = q.shape
         params = binding.make_params(B, H, L, D, block_size, top_k, window, _DT[q.dtype],
-                                     sm_scale=sm_scale, strides=q.stride()[:3])
+                                     sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
+                                     stis_block=stis_block)
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -56,17 +58,22 @@ class _BlossomAttention(torch.autograd.Function):
         dgate = torch.empty((q.shape[1], 2), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
-        return dq, dk, dv, dgate.to(ctx.gate_dtype), None, None, None, None, None
+        return dq, dk, dv, dgate.to(ctx.gate_dtype), None, None, None, None, None, None, None
 
 
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
-                      return_indices=False):
+                      return_indices=False, short_term="window", mask_block=1):
     """Gated two-branch sparse attention of [B, H, L, D] tensors (float32 or bfloat16, CUDA).
 
     gate_logits: [H, 2] (column 0 long-term, column 1 short-term branch); seq_lens: optional int32
     [B] valid lengths of left-padded sequences; sm_scale 0 means 1/sqrt(D).  Differentiable in
     q, k, v and gate_logits.  Returns the output, and the selected block indices if asked.
+    short_term: "window" (keys t - window < p <= t) or "power-law" (Eq. 15: the window, blocks of
+    mask_block positions at power-of-two block distances, and the last mask_block positions).
     """
+    if short_term not in ("window", "power-law"):
+        raise ValueError("short_term must be 'window' or 'power-law'")
     out, idx = _BlossomAttention.apply(q, k, v, gate_logits, seq_lens, int(block_size), int(top_k),
-                                       int(window), float(sm_scale))
+                                       int(window), float(sm_scale),
+                                       1 if short_term == "power-law" else 0, int(mask_block))
     return (out, idx) if return_indices else out

@@ -78,6 +78,7 @@ static int make_shape(const blossom_params *p, Shape *out) {
   if (p->stride_l % 8 || p->stride_h % 8 || p->stride_b % 8) return BLOSSOM_ERR_INVALID_ARG;
   if (p->kv_heads != p->heads) return BLOSSOM_ERR_UNSUPPORTED;
   if (p->causal != 1 || p->select_mode != 0) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->stis_mode < 0 || p->stis_mode > 1 || p->stis_block < 0) return BLOSSOM_ERR_INVALID_ARG;
   if (p->head_dim != 32 && p->head_dim != 64) return BLOSSOM_ERR_UNSUPPORTED;
   if (p->block_size != 8 && p->block_size != 16 && p->block_size != 32 && p->block_size != 64)
     return BLOSSOM_ERR_UNSUPPORTED;
@@ -88,6 +89,7 @@ static int make_shape(const blossom_params *p, Shape *out) {
   Shape s;
   s.B = p->batch; s.H = p->heads; s.L = p->seq_len; s.D = p->head_dim; s.Bk = p->block_size;
   s.topk = p->top_k; s.window = p->window; s.M = (int)M;
+  s.stis_mode = p->stis_mode; s.stis_blk = p->stis_block > 0 ? p->stis_block : 1;
   s.scale_d = p->sm_scale > 0.f ? (double)p->sm_scale : 1.0 / sqrt((double)p->head_dim);
   s.scale = (float)s.scale_d;
   s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;

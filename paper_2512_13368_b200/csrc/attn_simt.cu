@@ -50,14 +50,34 @@ __device__ __forceinline__ void stage_tile(const Shape &s, const T *base, int n,
   }
 }
 
+// Eq. 15 on the causal side: may query t attend to key p <= t in the short-term branch?
+// Mode 0: the window alone.  Mode 1 (power-law mask): the window, or the block-index distance
+// floor(t / blk) - floor(p / blk) is a power of two, or p is one of the last blk positions.
+__device__ __forceinline__ bool st_visible(const Shape &s, int t, int p) {
+  if (t - p < s.window) return true;
+  if (s.stis_mode == 0) return false;
+  const int bd = t / s.stis_blk - p / s.stis_blk;
+  return (bd >= 1 && (bd & (bd - 1)) == 0) || p >= s.L - s.stis_blk;
+}
+// May some query in [t0, t1] see some key in [p0, p1] (p0 <= t1) through the short-term branch?
+// Exact for the window; for the power-law mask a superset (any power of two inside the range of
+// block distances counts), which only costs a visit: st_visible decides every pair.
+__device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, int p0, int p1) {
+  if (t0 - p1 < s.window) return true;
+  if (s.stis_mode == 0) return false;
+  if (p1 >= s.L - s.stis_blk) return true;
+  const int dmax = t1 / s.stis_blk - p0 / s.stis_blk;
+  const int dmin = max(1, t0 / s.stis_blk - p1 / s.stis_blk);
+  return dmax >= dmin && (1 << (31 - __clz(dmax))) >= dmin;  // largest power of two <= dmax
+}
+
 // flags[blk], blk <= qb: bit 0 = blk is one of the query block's selected blocks,
-// bit 1 = blk intersects the causal window of some query of the block.
+// bit 1 = the short-term branch of some query of the block may reach into blk.
 __device__ __forceinline__ void build_visit_flags(const Shape &s, const int32_t *idxrow, int qb,
                                                   int *flags) {
-  const int wpos = qb * s.Bk - (s.window - 1);
-  const int wlo = wpos > 0 ? wpos / s.Bk : 0;
+  const int t0 = qb * s.Bk, t1 = min(s.L, t0 + s.Bk) - 1;
   for (int blk = threadIdx.x; blk <= qb; blk += blockDim.x) {
-    int f = blk >= wlo ? 2 : 0;
+    int f = st_ranges_touch(s, t0, t1, blk * s.Bk, min(s.L, blk * s.Bk + s.Bk) - 1) ? 2 : 0;
     for (int i = 0; i < s.topk; ++i) f |= (idxrow[i] == blk) ? 1 : 0;
     flags[blk] = f;
   }
@@ -110,7 +130,7 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
       const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
       const bool selb = f & 1;
       for (int pi = pbeg; pi < pend; ++pi) {
-        const bool inS = (t - (p0 + pi)) < s.window;
+        const bool inS = st_visible(s, t, p0 + pi);
         if (!selb && !inS) continue;
         const float4 *kr = reinterpret_cast<const float4 *>(Ks) + pi * CH;
         const float4 *vr = reinterpret_cast<const float4 *>(Vs) + pi * CH;
@@ -232,7 +252,7 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
       const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
       const bool selb = f & 1;
       for (int pi = pbeg; pi < pend; ++pi) {
-        const bool inS = (t - (p0 + pi)) < s.window;
+        const bool inS = st_visible(s, t, p0 + pi);
         if (!selb && !inS) continue;
         const float4 *kr = reinterpret_cast<const float4 *>(Ks) + pi * CH;
         const float4 *vr = reinterpret_cast<const float4 *>(Vs) + pi * CH;
@@ -297,10 +317,12 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   const int64_t BHL = (int64_t)s.B * s.H * s.L;
   const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
 
-  // which query blocks visit this key block: bit 0 = selected it, bit 1 = window reaches it
+  // which query blocks visit this key block: bit 0 = selected it, bit 1 = their short-term branch
+  // may reach it
   for (int qb = j + tid; qb < s.M; qb += blockDim.x) {
     const int32_t *row = idx + ((int64_t)u * s.M + qb) * s.topk;
-    int f = (qb * s.Bk - (j * s.Bk + s.Bk - 1) < s.window) ? 2 : 0;
+    int f = st_ranges_touch(s, qb * s.Bk, min(s.L, qb * s.Bk + s.Bk) - 1, j * s.Bk,
+                            min(s.L, j * s.Bk + s.Bk) - 1) ? 2 : 0;
     for (int i = 0; i < s.topk; ++i) f |= (row[i] == j) ? 1 : 0;
     flags[qb] = f;
   }
@@ -340,7 +362,7 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
       const int tbeg = max(0, p - t0), tend = min(s.Bk, s.L - t0);  // t >= p >= pad0
       const bool selb = f & 1;
       for (int ti = tbeg; ti < tend; ++ti) {
-        const bool inS = (t0 + ti - p) < s.window;
+        const bool inS = st_visible(s, t0 + ti, p);
         if (!selb && !inS) continue;
         const float4 *qr = reinterpret_cast<const float4 *>(Qs) + ti * CH;
         const float4 *gr = reinterpret_cast<const float4 *>(Gs) + ti * CH;

@@ -11,6 +11,7 @@ namespace blossom {
 // Problem shape handed to every kernel by value.
 struct Shape {
   int B, H, L, D, Bk, topk, window, M;
+  int stis_mode, stis_blk;  // short-term mask: 0 = window, 1 = power-law (Eq. 15) with block stis_blk
   float scale;     // attention logit scale (fp32 arithmetic of the attention kernels)
   double scale_d;  // the same scale in double for the fp64 block scoring
   int64_t sb, sh, sl;  // element strides of q-shaped tensors

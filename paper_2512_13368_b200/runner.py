@@ -27,7 +27,8 @@ class DeviceProblem:
         if w.seq_lens is not None:
             self.seq_lens = torch.from_numpy(w.seq_lens.astype(np.int32)).to(self.device)
         self.params = binding.make_params(w.B, w.H, w.L, w.D, w.block, w.topk, w.window, w.dtype,
-                                          sm_scale=sm_scale)
+                                          sm_scale=sm_scale, stis_mode=w.stis_mode,
+                                          stis_block=w.stis_block)
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):

@@ -59,6 +59,8 @@ class Workload:
     gate: np.ndarray = field(repr=False)      # [H, 2] float32
     dout: np.ndarray = field(repr=False)
     seq_lens: np.ndarray | None = field(default=None, repr=False)  # [B] int32 or None
+    stis_mode: int = 0    # short-term branch: 0 = causal window, 1 = power-law mask (Eq. 15)
+    stis_block: int = 1   # mask block of the power-law mask
 
     @property
     def n_blocks(self) -> int:
@@ -75,11 +77,11 @@ class Workload:
                         self.topk, self.window, self.seed,
                         self.q[n:n + 1, h:h + 1].copy(), self.k[n:n + 1, h:h + 1].copy(),
                         self.v[n:n + 1, h:h + 1].copy(), self.gate[h:h + 1].copy(),
-                        self.dout[n:n + 1, h:h + 1].copy(), sl)
+                        self.dout[n:n + 1, h:h + 1].copy(), sl, self.stis_mode, self.stis_block)
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,
-         row_scales=False) -> Workload:
+         row_scales=False, stis_mode=0, stis_block=1) -> Workload:
     """Generic generator; see the module docstring for the draw order.
 
     lengths: None or (lo, hi) inclusive -> left-padded sequences, pad rows keep their
@@ -102,7 +104,7 @@ def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=No
             t *= rng.uniform(0.5, 2.0, size=(B, H, L, 1)).astype(np.float32)
     return Workload(name, dtype, B, H, L, D, block, topk, window, seed,
                     quantize(q, dtype), quantize(k, dtype), quantize(v, dtype),
-                    gate, quantize(dout, dtype), seq_lens)
+                    gate, quantize(dout, dtype), seq_lens, stis_mode, stis_block)
 
 
 # The five benchmark configurations (sizes fixed by the task's baseline file).

@@ -55,12 +55,13 @@ def check_forward_backward(w, res, sm_scale=None, backward=True):
     """res: dict of numpy arrays from the CUDA path.  Returns a dict of max-abs errors."""
     forgiven = check_indices(w, res["idx"], sm_scale)
     ref = oracle.forward(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
-                         idx=res["idx"])
+                         idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block)
     errs = {"near_tie_rows": forgiven}
     keys = ["out", "out_lt", "out_st", "lse"]
     if backward:
         ref.update(oracle.backward(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, ref, w.dout,
-                                   w.seq_lens, sm_scale))
+                                   w.seq_lens, sm_scale, stis_mode=w.stis_mode,
+                                   stis_block=w.stis_block))
         keys += ["dq", "dk", "dv", "dgate"]
     for key in keys:
         if res.get(key) is None:

@@ -94,6 +94,28 @@ def test_edge_shapes(runner, dtype, L, D, block, topk, window, lens):
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,block,topk,window,blk,lens", [
+    (64, 32, 8, 2, 8, 1, None),              # the paper's defaults: window 8, mask block 1
+    (200, 32, 16, 4, 8, 1, [200, 5, 1, 0]),  # ragged tail, length-1 and fully padded sequences
+    (300, 64, 32, 4, 16, 4, [300, 131]),     # mask block 4: whole blocks at power-of-two distances
+    (257, 64, 8, 5, 3, 2, None),             # window not a multiple of the mask block, odd length
+    (96, 64, 64, 2, 200, 1, None),           # window > L: the mask adds nothing to dense causal
+    (128, 32, 16, 3, 1, 128, None),          # mask block = L: every key is in the last block
+    (1024, 64, 64, 8, 8, 1, [1024, 700]),    # links up to distance 512 across many key blocks
+])
+def test_power_law_short_term_mask(runner, dtype, L, D, block, topk, window, blk, lens):
+    """Eq. 15 with all three cases (stis_mode 1) against the oracle, forward and backward."""
+    B = len(lens) if lens else 2
+    w = workloads.make("powerlaw", dtype, B, 2, L, D, block, topk, window, seed=13, stis_mode=1,
+                       stis_block=blk)
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    print(check_forward_backward(w, res))
+
+
 def test_explicit_scale_and_given_indices(runner):
     w = workloads.make("scale", "fp32", 2, 2, 96, 32, 16, 3, 20, seed=5)
     p, res = run(runner, w, sm_scale=0.37)
