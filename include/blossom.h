@@ -133,8 +133,7 @@ int blossom_select_blocks_static(const blossom_params *params /* host */, const 
  * Forward (paper: Eq. 14 and 16 for the selected-block branch, Eq. 15 under the causal mask
  * (its first case alone with stis_mode 0, all three with stis_mode 1) and Eq. 17 for the
  * short-term branch, Eq. 19 for the gate, each branch being the masked softmax attention of
- * Eq. 1 with online softmax in fp32).  With stis_mode 1 every dtype runs on the CUDA-core
- * kernels.
+ * Eq. 1 with online softmax in fp32).
  *   q, k, v      in   q-shaped
  *   gate_logits  in   [H][2]
  *   seq_lens     in   [B] or NULL

@@ -50,27 +50,6 @@ __device__ __forceinline__ void stage_tile(const Shape &s, const T *base, int n,
   }
 }
 
-// Eq. 15 on the causal side: may query t attend to key p <= t in the short-term branch?
-// Mode 0: the window alone.  Mode 1 (power-law mask): the window, or the block-index distance
-// floor(t / blk) - floor(p / blk) is a power of two, or p is one of the last blk positions.
-__device__ __forceinline__ bool st_visible(const Shape &s, int t, int p) {
-  if (t - p < s.window) return true;
-  if (s.stis_mode == 0) return false;
-  const int bd = t / s.stis_blk - p / s.stis_blk;
-  return (bd >= 1 && (bd & (bd - 1)) == 0) || p >= s.L - s.stis_blk;
-}
-// May some query in [t0, t1] see some key in [p0, p1] (p0 <= t1) through the short-term branch?
-// Exact for the window; for the power-law mask a superset (any power of two inside the range of
-// block distances counts), which only costs a visit: st_visible decides every pair.
-__device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, int p0, int p1) {
-  if (t0 - p1 < s.window) return true;
-  if (s.stis_mode == 0) return false;
-  if (p1 >= s.L - s.stis_blk) return true;
-  const int dmax = t1 / s.stis_blk - p0 / s.stis_blk;
-  const int dmin = max(1, t0 / s.stis_blk - p1 / s.stis_blk);
-  return dmax >= dmin && (1 << (31 - __clz(dmax))) >= dmin;  // largest power of two <= dmax
-}
-
 // flags[blk], blk <= qb: bit 0 = blk is one of the query block's selected blocks,
 // bit 1 = the short-term branch of some query of the block may reach into blk.
 __device__ __forceinline__ void build_visit_flags(const Shape &s, const int32_t *idxrow, int qb,

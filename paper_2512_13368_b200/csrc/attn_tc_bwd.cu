@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         if (row_valid) {
           const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
           if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
-          if (f & 2) maskS = mc & cols_ge(t - s.window + 1 - p0);
+          if (f & 2) maskS = mc & st_key_cols(s, t, p0);
         }
         hL = (uint32_t)(maskL >> (32 * (x & 1) + 16 * half)) & 0xffffu;
         hS = (uint32_t)(maskS >> (32 * (x & 1) + 16 * half)) & 0xffffu;
@@ -633,7 +633,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       if (row_valid) {
         const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
         if (f & 1) maskL = mc & expand_block_bits(invb[g * nT + qt], s.Bk);
-        if (f & 2) maskS = mc & cols_le(p + s.window - 1 - t0);
+        if (f & 2) maskS = mc & st_query_cols(s, p, t0);
       }
       const uint32_t hL = (uint32_t)(maskL >> (half * 32)), hS = (uint32_t)(maskS >> (half * 32));
       const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);

@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       if (cls == 2) {
         if (row_ok) {
           mask = cols_le(t - p0) & cols_ge(pad0 - p0);
-          mask &= isL ? expand_block_bits(selb[g * nT + jt], s.Bk) : cols_ge(t - s.window + 1 - p0);
+          mask &= isL ? expand_block_bits(selb[g * nT + jt], s.Bk) : st_key_cols(s, t, p0);
         }
         doB = __any_sync(0xffffffffu, mask != 0ull);
         fullB = __all_sync(0xffffffffu, mask == ~0ull);

@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         int f = 0;
         if (jt <= jt_max && row_last >= pad0 && jt * 64 + 63 >= pad0) {
           for (int g = 0; g < G; ++g) f |= selb[g * nT + jt] ? 1 : 0;
-          if (jt * 64 + 63 >= row0 - s.window + 1) f |= 2;
+          if (st_ranges_touch(s, row0, row_last, jt * 64, jt * 64 + 63)) f |= 2;
         }
         const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
         if (f) {
@@ -166,8 +166,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
             const uint32_t bits = selb[((w * 32) / s.Bk) * nT + jt];
             cls = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
           }
-        } else if (p0 + 63 >= t_lo - s.window + 1) {
-          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;
+        } else if (st_ranges_touch(s, t_lo, t_lo + 31, p0, p0 + 63)) {
+          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;  // 1: inside every row's window
         }
       }
       icls[e] = (uint8_t)cls;
@@ -192,7 +192,9 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                 if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
             if (lflags[j] & 2)
               for (int hf = 0; hf < 2; ++hf)
-                if (p0 + 63 >= row0 + 64 * hf - s.window + 1 && p0 <= row0 + 64 * hf + 63) c |= 1 << hf;
+                if (p0 <= row0 + 64 * hf + 63 &&
+                    st_ranges_touch(s, row0 + 64 * hf, row0 + 64 * hf + 63, p0, p0 + 63))
+                  c |= 1 << hf;
             if (c == 0) c = 3;
           }
           const unsigned bA = __ballot_sync(0xffffffffu, c == 1), bB = __ballot_sync(0xffffffffu, c == 2),
@@ -248,7 +250,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         }
         if (any_sel) cL = (all_sel && past) ? 1 : 2;
       }
-      if ((f & 2) && reach && k_hi >= t_lo - s.window + 1) cS = (past && k_lo >= t_hi - s.window + 1) ? 1 : 2;
+      if ((f & 2) && reach && st_ranges_touch(s, t_lo, t_hi, k_lo, k_hi))
+        cS = (past && k_lo >= t_hi - s.window + 1) ? 1 : 2;  // 1: inside every row's window
       jcls[e] = (uint8_t)((cL == 2 || cS == 2) ? 8 : (cL | (cS << 1)));
     }
   } else {
@@ -283,7 +286,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       int f = 0;
       if (qt <= qt_max && key_last >= pad0) {
         for (int g = 0; g < G; ++g) f |= selb[g * nT + qt] ? 1 : 0;
-        if (qt * 64 <= key_last + s.window - 1) f |= 2;
+        if (st_ranges_touch(s, qt * 64, min(qt * 64 + 63, s.L - 1), key0, key_last)) f |= 2;
       }
       const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
       if (f) {

@@ -81,6 +81,28 @@ __device__ __forceinline__ int64_t row_offset(const Shape &s, int n, int h, int 
   return (int64_t)n * s.sb + (int64_t)h * s.sh + (int64_t)t * s.sl;
 }
 
+// ---- the short-term mask (Eq. 15), shared by the CUDA-core and the tensor-core kernels ----
+// Eq. 15 on the causal side: may query t attend to key p <= t in the short-term branch?
+// Mode 0: the window alone.  Mode 1 (power-law mask): the window, or the block-index distance
+// floor(t / blk) - floor(p / blk) is a power of two, or p is one of the last blk positions.
+__device__ __forceinline__ bool st_visible(const Shape &s, int t, int p) {
+  if (t - p < s.window) return true;
+  if (s.stis_mode == 0) return false;
+  const int bd = t / s.stis_blk - p / s.stis_blk;
+  return (bd >= 1 && (bd & (bd - 1)) == 0) || p >= s.L - s.stis_blk;
+}
+// May some query in [t0, t1] see some key in [p0, p1] (p0 <= t1) through the short-term branch?
+// Exact for the window; for the power-law mask a superset (any power of two inside the range of
+// block distances counts), which only costs a visit: st_visible decides every pair.
+__device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, int p0, int p1) {
+  if (t0 - p1 < s.window) return true;
+  if (s.stis_mode == 0) return false;
+  if (p1 >= s.L - s.stis_blk) return true;
+  const int dmax = t1 / s.stis_blk - p0 / s.stis_blk;
+  const int dmin = max(1, t0 / s.stis_blk - p1 / s.stis_blk);
+  return dmax >= dmin && (1 << (31 - __clz(dmax))) >= dmin;  // largest power of two <= dmax
+}
+
 // launchers (one translation unit each)
 int launch_select(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
                   int32_t *idx, const Workspace &ws, cudaStream_t st);

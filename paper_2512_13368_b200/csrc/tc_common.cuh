@@ -350,6 +350,38 @@ __device__ __forceinline__ uint64_t expand_block_bits(uint32_t bits, int bk) {
   return m;
 }
 
+// Short-term mask of Eq. 15 over the 64 keys p0 ... p0 + 63 for query t, without the causal and
+// the padding condition (the caller ANDs those): the window, and with the power-law mask the key
+// blocks at power-of-two block distances and the last block.
+__device__ __forceinline__ uint64_t st_key_cols(const Shape &s, int t, int p0) {
+  uint64_t m = cols_ge(t - s.window + 1 - p0);
+  if (s.stis_mode) {
+    m |= cols_ge(s.L - s.stis_blk - p0);
+    const int bq = t / s.stis_blk;
+    for (int d = 1; d <= bq; d <<= 1) {  // key block bq - d: later d lie further left
+      const int a = (bq - d) * s.stis_blk;
+      if (a + s.stis_blk - 1 < p0) break;
+      if (a <= p0 + 63) m |= cols_ge(a - p0) & cols_le(a + s.stis_blk - 1 - p0);
+    }
+  }
+  return m;
+}
+// The same mask seen from key p over the 64 queries t0 ... t0 + 63 (again without causality and
+// padding).
+__device__ __forceinline__ uint64_t st_query_cols(const Shape &s, int p, int t0) {
+  uint64_t m = cols_le(p + s.window - 1 - t0);
+  if (s.stis_mode) {
+    if (p >= s.L - s.stis_blk) return ~0ull;
+    const int bk = p / s.stis_blk;
+    for (int d = 1;; d <<= 1) {  // query block bk + d: later d lie further right
+      const int a = (bk + d) * s.stis_blk;
+      if (a > t0 + 63 || a >= s.L) break;
+      if (a + s.stis_blk - 1 >= t0) m |= cols_ge(a - t0) & cols_le(a + s.stis_blk - 1 - t0);
+    }
+  }
+  return m;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t *>(&h);

@@ -38,9 +38,7 @@ int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_
 }
 
 bool fwd_tc_supported(const Shape &s, int dtype) {
-  // (the tile lists and masks of the tensor-core kernels know the window only; the power-law
-  // short-term mask runs on the CUDA-core path)
-  return s.stis_mode == 0 && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  return dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 

@@ -218,6 +218,15 @@ def test_config4_full_size_sampled(runner):
     print(errs)
 
 
+def test_config4_full_size_power_law_sampled(runner):
+    """The headline shape with the paper's short-term mask (window 8, mask block 1), in the launch
+    configuration the benchmark's --short-term power-law option times."""
+    w = workloads.config4()
+    w.stis_mode, w.stis_block, w.window = 1, 1, 8
+    errs, _ = _sampled_units(runner, w, [(0, 0), (7, 3), (15, 7)])
+    print(errs)
+
+
 def test_config2_full_size_sampled(runner):
     w = workloads.config2()
     units = [(int(np.argmin(w.seq_lens)), 0), (int(np.argmax(w.seq_lens)), 1), (100, 0), (255, 1)]
