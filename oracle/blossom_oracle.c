@@ -19,6 +19,8 @@
  *                               shares one selection) applied to the queries
  *                               of a query block
  *   top-k selection      Eq. 13 own block always kept, ties -> lower index
+ *   overlapping blocks   Eq. 8 with l, s != Bk and the score remap of Eq. 11
+ *                               (blossom_oracle_select_cmp)
  *   selected-KV attention Eq. 14 + Eq. 16 (via Eq. 1 with the causal mask)
  *   window attention     Eq. 15 first case (|i-j| < w), causal side, Eq. 17
  *   power-law mask       Eq. 15 all three cases (stis_mode 1), causal side:
@@ -156,6 +158,137 @@ int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double s
       if (len > L) len = L;
       select_unit(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D,
                   idx + u * M * topk, scores ? scores + u * M * M : NULL);
+    }
+  return 0;
+}
+
+/* ---- selection with overlapping compression blocks for one (n,h) unit: Eq. 8-11, 13 -------
+ * Compression blocks K_i = positions [s i, s i + l), i = 0 .. Mc-1, Mc = floor((L - l)/s) + 1
+ * (Eq. 8, 0-based; none if L < l), summarised by the mean of their valid keys (Eq. 9 with
+ * phi := mean).  For query block b (selection blocks of lp = Bk positions) the candidates are the
+ * live compression blocks that end before the query block starts, s i + l <= lp b; Eq. 10 per
+ * query over the candidates, summed over the block's valid queries (Eq. 12's rule).  Eq. 11 maps
+ * the compression scores to selection blocks j < b,
+ *   S_ltis[j] = sum_{m < lp/s} sum_{n < l/s} S_cmp[(lp/s) j - m - n],
+ * terms whose index is out of range or not a candidate being zero.  Eq. 13 as in select_unit.
+ * scores_cmp [M][Mc] and scores [M][M] are optional outputs. */
+static void select_unit_cmp(int L, int D, int Bk, int topk, int l, int s, double scale, int pad0,
+                            const double *q, const double *k, int32_t *idx, double *scores,
+                            double *scores_cmp) {
+  const int M = n_blocks(L, Bk);
+  const int Mc = L >= l ? (L - l) / s + 1 : 0;
+  const int rs = Bk / s, rl = l / s;
+  double *ktil = (double *)calloc((size_t)(Mc > 0 ? Mc : 1) * D, sizeof(double));
+  int *livec = (int *)calloc((size_t)(Mc > 0 ? Mc : 1), sizeof(int));
+  double *Sc = (double *)malloc(sizeof(double) * (size_t)(Mc > 0 ? Mc : 1));
+  double *z = (double *)malloc(sizeof(double) * (size_t)(Mc > 0 ? Mc : 1));
+  double *S = (double *)malloc(sizeof(double) * (size_t)M);
+  char *taken = (char *)malloc((size_t)M);
+
+  for (int i = 0; i < Mc; ++i) { /* Eq. 8 + Eq. 9 */
+    int lo = imax(i * s, pad0), hi = i * s + l, cnt = 0;
+    for (int p = lo; p < hi; ++p) {
+      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] += k[(size_t)p * D + c];
+      ++cnt;
+    }
+    livec[i] = cnt > 0;
+    if (cnt > 0)
+      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] /= (double)cnt;
+  }
+
+  for (int b = 0; b < M; ++b) {
+    int32_t *row = idx + (size_t)b * topk;
+    for (int e = 0; e < topk; ++e) row[e] = -1;
+    if (scores)
+      for (int j = 0; j < M; ++j) scores[(size_t)b * M + j] = 0.0;
+    if (scores_cmp)
+      for (int i = 0; i < Mc; ++i) scores_cmp[(size_t)b * Mc + i] = 0.0;
+    int qlo = imax(b * Bk, pad0), qhi = imin((b + 1) * Bk, L);
+    if (qlo >= qhi) continue; /* query block holds only padding */
+
+    /* candidates: compression blocks 0 .. nc-1 end before the query block starts */
+    int nc = 0;
+    while (nc < Mc && nc * s + l <= b * Bk) ++nc;
+    int ncand = 0;
+    for (int i = 0; i < nc; ++i) {
+      Sc[i] = 0.0;
+      ncand += livec[i];
+    }
+    if (ncand > 0) { /* Eq. 10 per query, summed over the block's valid queries */
+      for (int t = qlo; t < qhi; ++t) {
+        double mx = -INFINITY;
+        for (int i = 0; i < nc; ++i) {
+          if (!livec[i]) continue;
+          double acc = 0.0;
+          for (int c = 0; c < D; ++c) acc += q[(size_t)t * D + c] * ktil[(size_t)i * D + c];
+          z[i] = scale * acc;
+          if (z[i] > mx) mx = z[i];
+        }
+        double den = 0.0;
+        for (int i = 0; i < nc; ++i)
+          if (livec[i]) den += exp(z[i] - mx);
+        for (int i = 0; i < nc; ++i)
+          if (livec[i]) Sc[i] += exp(z[i] - mx) / den;
+      }
+    }
+    if (scores_cmp)
+      for (int i = 0; i < nc; ++i)
+        if (livec[i]) scores_cmp[(size_t)b * Mc + i] = Sc[i];
+
+    /* Eq. 11, and which past selection blocks hold a valid key */
+    int nlive = 0;
+    for (int j = 0; j < b; ++j) {
+      double acc = 0.0;
+      for (int m = 0; m < rs; ++m)
+        for (int n = 0; n < rl; ++n) {
+          int i = rs * j - m - n;
+          if (i >= 0 && i < nc && livec[i]) acc += Sc[i];
+        }
+      S[j] = acc;
+      taken[j] = 0;
+      if (imin((j + 1) * Bk, L) > imax(j * Bk, pad0)) {
+        ++nlive;
+        if (scores) scores[(size_t)b * M + j] = acc;
+      } else {
+        taken[j] = 2; /* not selectable */
+      }
+    }
+    /* Eq. 13: the own block plus the (topk-1) best past blocks, ties to the lower index */
+    int want = imin(topk - 1, nlive);
+    for (int e = 0; e < want; ++e) {
+      int best = -1;
+      for (int j = 0; j < b; ++j) {
+        if (taken[j]) continue;
+        if (best < 0 || S[j] > S[best]) best = j;
+      }
+      taken[best] = 1;
+    }
+    int e = 0;
+    for (int j = 0; j < b; ++j)
+      if (taken[j] == 1) row[e++] = j;
+    row[e++] = b;
+  }
+  free(ktil); free(livec); free(Sc); free(z); free(S); free(taken);
+}
+
+int blossom_oracle_select_cmp(int B, int H, int L, int D, int Bk, int topk, int l, int s,
+                              double scale, const double *q, const double *k,
+                              const int32_t *seq_lens, int32_t *idx, double *scores,
+                              double *scores_cmp) {
+  if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
+  if (l < 1 || s < 1 || l % s || Bk % s) return 1;
+  const int M = n_blocks(L, Bk);
+  const int Mc = L >= l ? (L - l) / s + 1 : 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int n = 0; n < B; ++n)
+    for (int h = 0; h < H; ++h) {
+      size_t u = (size_t)n * H + h;
+      int len = seq_lens ? seq_lens[n] : L;
+      if (len < 0) len = 0;
+      if (len > L) len = L;
+      select_unit_cmp(L, D, Bk, topk, l, s, scale, L - len, q + u * L * D, k + u * L * D,
+                      idx + u * M * topk, scores ? scores + u * M * M : NULL,
+                      scores_cmp ? scores_cmp + u * M * Mc : NULL);
     }
   return 0;
 }

@@ -49,6 +49,8 @@ def _load():
         lib.blossom_oracle_threads.restype = i
         lib.blossom_oracle_select.restype = i
         lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp]
+        lib.blossom_oracle_select_cmp.restype = i
+        lib.blossom_oracle_select_cmp.argtypes = [i, i, i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp, _dp]
         lib.blossom_oracle_forward.restype = i
         lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
@@ -98,6 +100,38 @@ def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores
     if rc:
         raise ValueError("blossom_oracle_select: bad arguments")
     return (idx, scores) if return_scores else idx
+
+
+def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, sm_scale=None,
+                      return_scores=False):
+    """Eq. 8-11, 13 with overlapping compression blocks (length ``cmp_block``, stride
+    ``cmp_stride``) scored and mapped onto selection blocks of ``block`` positions.
+
+    With return_scores also returns the selection scores ``[B,H,M,M]`` and the compression
+    scores ``[B,H,M,Mc]``."""
+    q, k = _f64(q), _f64(k)
+    B, H, L, D = q.shape
+    M = -(-L // block)
+    if cmp_block < 1 or cmp_stride < 1 or cmp_block % cmp_stride or block % cmp_stride:
+        raise ValueError("blossom_oracle_select_cmp: bad arguments")
+    Mc = (L - cmp_block) // cmp_stride + 1 if L >= cmp_block else 0
+    idx = np.empty((B, H, M, topk), dtype=np.int32)
+    scores = np.zeros((B, H, M, M), dtype=np.float64) if return_scores else None
+    scores_cmp = np.zeros((B, H, M, max(Mc, 1)), dtype=np.float64) if return_scores else None
+    sl = _lens(seq_lens, B)
+    if return_scores and Mc == 0:
+        sc_arg = None
+    else:
+        sc_arg = scores_cmp
+    rc = _load().blossom_oracle_select_cmp(B, H, L, D, block, topk, int(cmp_block), int(cmp_stride),
+                                           _scale(sm_scale, D), _ptr(q, _dp), _ptr(k, _dp),
+                                           _ptr(sl, _ip), _ptr(idx, _ip), _ptr(scores, _dp),
+                                           _ptr(sc_arg, _dp))
+    if rc:
+        raise ValueError("blossom_oracle_select_cmp: bad arguments")
+    if return_scores:
+        return idx, scores, scores_cmp[..., :Mc]
+    return idx
 
 
 def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None,
