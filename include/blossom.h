@@ -73,6 +73,10 @@ typedef struct {
                         * Eq. 15: window, or block-index distance floor(t/blk) - floor(p/blk) a
                         * power of two, or p among the last blk positions (all with p <= t)      */
   int32_t stis_block;  /* blk >= 1 of the power-law mask (0 reads as 1); ignored in mode 0       */
+  int32_t cmp_block;   /* l: length of the compression blocks the selection scores (Eq. 8); 0 =
+                        * block_size.  With cmp_stride it allows overlapping blocks whose scores
+                        * Eq. 11 maps onto the selection blocks of block_size positions          */
+  int32_t cmp_stride;  /* s: their stride; 0 = block_size; must divide cmp_block and block_size  */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

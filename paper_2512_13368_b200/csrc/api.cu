@@ -59,6 +59,8 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.delta = reinterpret_cast<float *>(take(2 * units * s.L * sizeof(float)));
   w.dalpha = reinterpret_cast<double *>(take(units * s.M * sizeof(double)));
   w.qstats = reinterpret_cast<float4 *>(take(units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4)));
+  w.cmean = reinterpret_cast<double *>(take(units * (size_t)s.Mc * s.D * sizeof(double)));
+  w.clive = reinterpret_cast<int32_t *>(take(units * (size_t)s.Mc * sizeof(int32_t)));
   w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.bytes = off;
@@ -90,6 +92,18 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.B = p->batch; s.H = p->heads; s.L = p->seq_len; s.D = p->head_dim; s.Bk = p->block_size;
   s.topk = p->top_k; s.window = p->window; s.M = (int)M;
   s.stis_mode = p->stis_mode; s.stis_blk = p->stis_block > 0 ? p->stis_block : 1;
+  s.cmp_l = s.cmp_s = s.Mc = 0;
+  if (p->cmp_block < 0 || p->cmp_stride < 0) return BLOSSOM_ERR_INVALID_ARG;
+  if (p->cmp_block > 0 || p->cmp_stride > 0) {
+    const int l = p->cmp_block > 0 ? p->cmp_block : p->block_size;
+    const int st = p->cmp_stride > 0 ? p->cmp_stride : p->block_size;
+    if (l % st || p->block_size % st) return BLOSSOM_ERR_INVALID_ARG;
+    if (l != p->block_size || st != p->block_size) {
+      const int64_t mc = p->seq_len >= l ? ((int64_t)p->seq_len - l) / st + 1 : 0;
+      if (mc > 4096) return BLOSSOM_ERR_UNSUPPORTED;
+      s.cmp_l = l; s.cmp_s = st; s.Mc = (int)mc;
+    }
+  }
   s.scale_d = p->sm_scale > 0.f ? (double)p->sm_scale : 1.0 / sqrt((double)p->head_dim);
   s.scale = (float)s.scale_d;
   s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;

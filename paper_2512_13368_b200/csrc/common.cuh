@@ -12,6 +12,8 @@ namespace blossom {
 struct Shape {
   int B, H, L, D, Bk, topk, window, M;
   int stis_mode, stis_blk;  // short-term mask: 0 = window, 1 = power-law (Eq. 15) with block stis_blk
+  int cmp_l, cmp_s, Mc;     // overlapping compression blocks (Eq. 8, 11): length, stride, count;
+                            // cmp_l == 0: the compression blocks are the selection blocks
   float scale;     // attention logit scale (fp32 arithmetic of the attention kernels)
   double scale_d;  // the same scale in double for the fp64 block scoring
   int64_t sb, sh, sl;  // element strides of q-shaped tensors
@@ -30,6 +32,8 @@ struct Workspace {
   double *dalpha;    // [B][H][M]     per query block partial of d alpha
   float4 *qstats;    // [B][H][ceil(L/64)*64]  16 bytes per query row, laid out per pair of rows as
                      //   {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)} for the dK/dV kernel
+  double *cmean;     // [B][H][Mc][D]  means of the overlapping compression blocks (cmp_l > 0)
+  int32_t *clive;    // [B][H][Mc]     their numbers of valid keys
   uint8_t *qmeta;    // per query-major CTA of the tensor-core kernels: tile lists (tc_meta_kernel)
   uint8_t *kmeta;    // per key-major CTA (dK/dV kernel): tile lists
   size_t bytes;
@@ -104,6 +108,8 @@ __device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, 
 }
 
 // launchers (one translation unit each)
+int launch_select_cmp(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
+                      int32_t *idx, const Workspace &ws, cudaStream_t st);
 int launch_select(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
                   int32_t *idx, const Workspace &ws, cudaStream_t st);
 int launch_fwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,

@@ -524,6 +524,7 @@ int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_l
 
 int launch_select(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
                   int32_t *idx, const Workspace &ws, cudaStream_t st) {
+  if (s.cmp_l > 0) return launch_select_cmp(s, dtype, q, k, seq_lens, idx, ws, st);  // Eq. 8-11
   if (dtype == BLOSSOM_DTYPE_FP32) {
     if (s.D == 32) return launch_select_t<float, 32>(s, (const float *)q, (const float *)k, seq_lens, idx, ws, st);
     return launch_select_t<float, 64>(s, (const float *)q, (const float *)k, seq_lens, idx, ws, st);
@@ -556,6 +557,7 @@ size_t select_static_capacity_bytes() { return kStaticBytes; }
 
 int launch_select_static(const Shape &s, int dtype, const void *q, const void *k,
                          const int32_t *seq_lens, int32_t *idx, cudaStream_t st) {
+  if (s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // the built-in scratch has no room for that mode
   const size_t blocks = (size_t)s.B * s.H * s.M;
   if (blocks > kStaticBlocks || blocks * (size_t)s.D > kStaticMeanElems) return BLOSSOM_ERR_TOO_LARGE;
   int dev = -1;

@@ -28,7 +28,8 @@ class DeviceProblem:
             self.seq_lens = torch.from_numpy(w.seq_lens.astype(np.int32)).to(self.device)
         self.params = binding.make_params(w.B, w.H, w.L, w.D, w.block, w.topk, w.window, w.dtype,
                                           sm_scale=sm_scale, stis_mode=w.stis_mode,
-                                          stis_block=w.stis_block)
+                                          stis_block=w.stis_block, cmp_block=w.cmp_block,
+                                          cmp_stride=w.cmp_stride)
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):

@@ -61,6 +61,8 @@ class Workload:
     seq_lens: np.ndarray | None = field(default=None, repr=False)  # [B] int32 or None
     stis_mode: int = 0    # short-term branch: 0 = causal window, 1 = power-law mask (Eq. 15)
     stis_block: int = 1   # mask block of the power-law mask
+    cmp_block: int = 0    # compression block length l of the selection (0 = block)
+    cmp_stride: int = 0   # and its stride s (0 = block)
 
     @property
     def n_blocks(self) -> int:
@@ -77,7 +79,8 @@ class Workload:
                         self.topk, self.window, self.seed,
                         self.q[n:n + 1, h:h + 1].copy(), self.k[n:n + 1, h:h + 1].copy(),
                         self.v[n:n + 1, h:h + 1].copy(), self.gate[h:h + 1].copy(),
-                        self.dout[n:n + 1, h:h + 1].copy(), sl, self.stis_mode, self.stis_block)
+                        self.dout[n:n + 1, h:h + 1].copy(), sl, self.stis_mode, self.stis_block,
+                        self.cmp_block, self.cmp_stride)
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,

@@ -21,8 +21,13 @@ TIE_REL = 1e-6
 
 def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
-    ref_idx, scores = oracle.select_blocks(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
-                                            return_scores=True)
+    if w.cmp_block or w.cmp_stride:
+        ref_idx, scores, _ = oracle.select_blocks_cmp(w.q, w.k, w.block, w.topk, w.cmp_block or w.block,
+                                                      w.cmp_stride or w.block, w.seq_lens, sm_scale,
+                                                      return_scores=True)
+    else:
+        ref_idx, scores = oracle.select_blocks(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
+                                                return_scores=True)
     assert gpu_idx.shape == ref_idx.shape and gpu_idx.dtype == np.int32
     bad = np.argwhere((gpu_idx != ref_idx).any(-1))
     forgiven = 0

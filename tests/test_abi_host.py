@@ -50,9 +50,12 @@ def test_workspace_bytes(lib):
     for bad in (dict(batch=0), dict(head_dim=48), dict(block_size=12), dict(top_k=0), dict(window=0),
                 dict(kv_heads=1), dict(causal=0), dict(select_mode=1), dict(dtype=7),
                 dict(seq_len=8 * 1025), dict(strides=(4096, 2048, 33)), dict(sm_scale=-1.0),
-                dict(stis_mode=2), dict(stis_mode=-1), dict(stis_mode=1, stis_block=-3)):
+                dict(stis_mode=2), dict(stis_mode=-1), dict(stis_mode=1, stis_block=-3),
+                dict(cmp_block=12, cmp_stride=8), dict(cmp_block=16, cmp_stride=3), dict(cmp_block=-8)):
         assert binding.blossom_workspace_bytes(good(**bad)) == 0, bad
     assert binding.blossom_workspace_bytes(good(stis_mode=1, stis_block=4)) == n  # power-law mask
+    assert binding.blossom_workspace_bytes(good(cmp_block=8, cmp_stride=8)) == n    # same as the default
+    assert binding.blossom_workspace_bytes(good(cmp_block=16, cmp_stride=4)) > n    # overlapping blocks
 
 
 def test_argument_validation_precedes_any_launch(lib):
@@ -88,8 +91,9 @@ def test_argument_validation_precedes_any_launch(lib):
 
 
 def test_params_struct_layout_matches_header():
-    # 12 x 4-byte fields, three int64 strides, the two short-term mask fields: 80 bytes with
-    # natural alignment
-    assert ctypes.sizeof(binding.blossom_params) == 80
+    # 12 x 4-byte fields, three int64 strides, the two short-term mask fields and the two
+    # compression-block fields: 88 bytes with natural alignment
+    assert ctypes.sizeof(binding.blossom_params) == 88
+    assert binding.blossom_params.cmp_block.offset == 80 and binding.blossom_params.cmp_stride.offset == 84
     assert binding.blossom_params.stride_b.offset == 48
     assert binding.blossom_params.stis_mode.offset == 72 and binding.blossom_params.stis_block.offset == 76

@@ -116,6 +116,28 @@ def test_power_law_short_term_mask(runner, dtype, L, D, block, topk, window, blk
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,block,topk,l,s,lens,power_law", [
+    (256, 32, 16, 4, 32, 16, None, True),            # the paper's default sizes, with its short-term mask
+    (512, 64, 16, 4, 32, 16, [512, 200, 33], False),
+    (320, 64, 32, 3, 32, 16, [320, 150], False),     # two strides per selection block
+    (192, 32, 16, 5, 48, 8, None, False),            # long compression blocks, small stride
+    (20, 32, 16, 4, 32, 16, None, False),            # shorter than one compression block
+    (1024, 64, 64, 8, 128, 32, [1024, 611], False),  # tensor-core attention behind the new selection
+])
+def test_overlapping_compression_blocks(runner, dtype, L, D, block, topk, l, s, lens, power_law):
+    """Selection through overlapping compression blocks and the score remap (Eq. 8-11)."""
+    B = len(lens) if lens else 2
+    w = workloads.make("overlap", dtype, B, 2, L, D, block, topk, 8 if power_law else 24, seed=17,
+                       stis_mode=1 if power_law else 0)
+    w.cmp_block, w.cmp_stride = l, s
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    print(check_forward_backward(w, res))
+
+
 def test_explicit_scale_and_given_indices(runner):
     w = workloads.make("scale", "fp32", 2, 2, 96, 32, 16, 3, 20, seed=5)
     p, res = run(runner, w, sm_scale=0.37)
