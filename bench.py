@@ -167,14 +167,18 @@ def oracle_sample(w, max_batch):
     sl = None if w.seq_lens is None else w.seq_lens[:nb].copy()
     return Workload(w.name + f"[first {nb} of {w.B} batch entries]", w.dtype, nb, w.H, w.L, w.D,
                     w.block, w.topk, w.window, w.seed, w.q[:nb], w.k[:nb], w.v[:nb], w.gate,
-                    w.dout[:nb], sl, w.stis_mode, w.stis_block)
+                    w.dout[:nb], sl, w.stis_mode, w.stis_block, w.cmp_block, w.cmp_stride)
 
 
 def time_oracle(ws):
     import oracle
     t0 = time.perf_counter()
+    idx = None
+    if ws.cmp_block or ws.cmp_stride:   # selection through overlapping compression blocks (Eq. 8-11)
+        idx = oracle.select_blocks_cmp(ws.q, ws.k, ws.block, ws.topk, ws.cmp_block or ws.block,
+                                       ws.cmp_stride or ws.block, ws.seq_lens)
     oracle.forward_backward(ws.q, ws.k, ws.v, ws.gate, ws.dout, ws.block, ws.topk, ws.window,
-                            ws.seq_lens, stis_mode=ws.stis_mode, stis_block=ws.stis_block)
+                            ws.seq_lens, idx=idx, stis_mode=ws.stis_mode, stis_block=ws.stis_block)
     return time.perf_counter() - t0
 
 
@@ -215,6 +219,9 @@ def main():
                          "power-law mask of Eq. 15 with --mask-window and --mask-block")
     ap.add_argument("--mask-window", type=int, default=8, help="w of the power-law mask (paper: 8 blocks of 1)")
     ap.add_argument("--mask-block", type=int, default=1, help="blk of the power-law mask")
+    ap.add_argument("--cmp-block", type=int, default=0,
+                    help="length l of overlapping compression blocks for the selection (Eq. 8, 11); 0 = off")
+    ap.add_argument("--cmp-stride", type=int, default=0, help="their stride s")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the batch size (profiling captures on a smaller case; not a bench line)")
     args = ap.parse_args()
@@ -231,9 +238,13 @@ def main():
     if args.short_term == "power-law":
         w.stis_mode, w.stis_block, w.window = 1, args.mask_block, args.mask_window
         w.name += f"+powerlaw(w{args.mask_window},blk{args.mask_block})"
+    if args.cmp_block or args.cmp_stride:
+        w.cmp_block, w.cmp_stride = args.cmp_block or w.block, args.cmp_stride or w.block
+        w.name += f"+cmp(l{w.cmp_block},s{w.cmp_stride})"
     cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "seq_len": w.L, "head_dim": w.D,
                 "block_size": w.block, "top_k": w.topk, "window": w.window, "short_term": args.short_term,
-                "mask_block": w.stis_block if w.stis_mode else None, "storage": w.dtype,
+                "mask_block": w.stis_block if w.stis_mode else None,
+                "cmp_block": w.cmp_block or None, "cmp_stride": w.cmp_stride or None, "storage": w.dtype,
                 "padding": "left, lengths U{5..200}" if w.seq_lens is not None else "none",
                 "l2": "no flush: a step touches ~1 GB of distinct tensors, more than the 126 MB L2"
                 if w.B * w.H * w.L * w.D * 2 * 15 > 4 * 126e6 else

@@ -17,7 +17,7 @@ _DT = {torch.float32: "fp32", torch.bfloat16: "bf16"}
 class _BlossomAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
-                stis_mode, stis_block):
+                stis_mode, stis_block, cmp_block, cmp_stride):
         if q.dtype not in _DT or k.dtype != q.dtype or v.dtype != q.dtype:
             raise TypeError("q, k, v must share one dtype, float32 or bfloat16")
         if not (q.is_cuda and q.shape == k.shape == v.shape and q.dim() == 4):
@@ -27,7 +27,7 @@ class _BlossomAttention(torch.autograd.Function):
         B, H, L, D = q.shape
         params = binding.make_params(B, H, L, D, block_size, top_k, window, _DT[q.dtype],
                                      sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
-                                     stis_block=stis_block)
+                                     stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride)
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -58,11 +58,12 @@ class _BlossomAttention(torch.autograd.Function):
         dgate = torch.empty((q.shape[1], 2), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
-        return dq, dk, dv, dgate.to(ctx.gate_dtype), None, None, None, None, None, None, None
+        return dq, dk, dv, dgate.to(ctx.gate_dtype), None, None, None, None, None, None, None, None, None
 
 
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
-                      return_indices=False, short_term="window", mask_block=1):
+                      return_indices=False, short_term="window", mask_block=1, cmp_block=0,
+                      cmp_stride=0):
     """Gated two-branch sparse attention of [B, H, L, D] tensors (float32 or bfloat16, CUDA).
 
     gate_logits: [H, 2] (column 0 long-term, column 1 short-term branch); seq_lens: optional int32
@@ -70,10 +71,13 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     q, k, v and gate_logits.  Returns the output, and the selected block indices if asked.
     short_term: "window" (keys t - window < p <= t) or "power-law" (Eq. 15: the window, blocks of
     mask_block positions at power-of-two block distances, and the last mask_block positions).
+    cmp_block / cmp_stride: length and stride of overlapping compression blocks for the selection
+    (Eq. 8, 11); 0 = the selection blocks themselves.
     """
     if short_term not in ("window", "power-law"):
         raise ValueError("short_term must be 'window' or 'power-law'")
     out, idx = _BlossomAttention.apply(q, k, v, gate_logits, seq_lens, int(block_size), int(top_k),
                                        int(window), float(sm_scale),
-                                       1 if short_term == "power-law" else 0, int(mask_block))
+                                       1 if short_term == "power-law" else 0, int(mask_block),
+                                       int(cmp_block), int(cmp_stride))
     return (out, idx) if return_indices else out

@@ -56,12 +56,14 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kCmpThreads) cmp_score_select_kernel(
     Shape s, const T *__restrict__ q, const double *__restrict__ cmean,
     const int32_t *__restrict__ clive, const int32_t *__restrict__ seq_lens,
-    int32_t *__restrict__ idx) {
+    int32_t *__restrict__ idx, int means_in_smem) {
   extern __shared__ double smd[];
   const int M = s.M, Mc = max(s.Mc, 1);
   double *zbuf = smd, *sp = zbuf + kCmpWarps * Mc, *qrow = sp + kCmpWarps * Mc;
   double *Sc = qrow + kCmpWarps * D, *S = Sc + Mc;
   int *livec = reinterpret_cast<int *>(S + M), *taken = livec + Mc;
+  // the candidates' means, row pitch D + 1 doubles (conflict-free when lanes read different rows)
+  double *kt_s = reinterpret_cast<double *>(taken + M + ((Mc + M) & 1));
   const int b = blockIdx.x % M, u = blockIdx.x / M, n = u / s.H, h = u % s.H;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int len = seq_lens ? seq_lens[n] : s.L;
@@ -76,6 +78,12 @@ __global__ void __launch_bounds__(kCmpThreads) cmp_score_select_kernel(
   // candidates: compression blocks 0 .. nc-1 end before the query block starts
   const int nc = b * s.Bk >= s.cmp_l ? min(s.Mc, (b * s.Bk - s.cmp_l) / s.cmp_s + 1) : 0;
   const double *kt = cmean + (int64_t)u * s.Mc * D;
+  int kpitch = D;
+  if (means_in_smem) {
+    for (int i = tid; i < nc * D; i += kCmpThreads) kt_s[(i / D) * (D + 1) + (i % D)] = kt[i];
+    kt = kt_s;
+    kpitch = D + 1;
+  }
   for (int i = tid; i < nc; i += kCmpThreads) livec[i] = clive[(int64_t)u * s.Mc + i] > 0;
   for (int i = tid; i < kCmpWarps * Mc; i += kCmpThreads) sp[i] = 0.0;
   __syncthreads();
@@ -92,7 +100,7 @@ __global__ void __launch_bounds__(kCmpThreads) cmp_score_select_kernel(
       double mx = -INFINITY;
       for (int i = lane; i < nc; i += 32) {
         if (!livec[i]) continue;
-        const double *ki = kt + (int64_t)i * D;
+        const double *ki = kt + (int64_t)i * kpitch;
         double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
 #pragma unroll 4
         for (int c = 0; c < D; c += 4) {
@@ -177,10 +185,11 @@ __global__ void __launch_bounds__(kCmpThreads) cmp_score_select_kernel(
   }
 }
 
-size_t cmp_smem_bytes(const Shape &s, int D) {
+size_t cmp_smem_bytes(const Shape &s, int D, bool means_in_smem) {
   const size_t Mc = s.Mc > 0 ? s.Mc : 1;
   return (2 * (size_t)kCmpWarps * Mc + (size_t)kCmpWarps * D + Mc + s.M) * sizeof(double) +
-         (Mc + s.M) * sizeof(int);
+         (Mc + s.M + ((Mc + s.M) & 1)) * sizeof(int) +
+         (means_in_smem ? Mc * (size_t)(D + 1) * sizeof(double) : 0);
 }
 
 template <typename T, int D>
@@ -191,7 +200,8 @@ int launch_select_cmp_t(const Shape &s, const T *q, const T *k, const int32_t *s
     LaunchScope ls(K_SUMMARY, st);
     cmp_summary_kernel<T, D><<<(unsigned)s.Mc * units, 256, 0, st>>>(s, k, seq_lens, ws.cmean, ws.clive);
   }
-  const size_t smem = cmp_smem_bytes(s, D);
+  const bool in_smem = cmp_smem_bytes(s, D, true) <= 160 * 1024;
+  const size_t smem = cmp_smem_bytes(s, D, in_smem);
   if (smem > 200 * 1024) return BLOSSOM_ERR_UNSUPPORTED;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(cmp_score_select_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -200,7 +210,7 @@ int launch_select_cmp_t(const Shape &s, const T *q, const T *k, const int32_t *s
   {
     LaunchScope ls(K_SCORE_SELECT, st);
     cmp_score_select_kernel<T, D><<<(unsigned)s.M * units, kCmpThreads, smem, st>>>(s, q, ws.cmean, ws.clive,
-                                                                                   seq_lens, idx);
+                                                                                   seq_lens, idx, in_smem ? 1 : 0);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -240,6 +240,15 @@ def test_config4_full_size_sampled(runner):
     print(errs)
 
 
+def test_config4_full_size_overlapping_compression_sampled(runner):
+    """The headline shape with compression blocks of 128 keys at stride 32 behind the selection,
+    as the benchmark's --cmp-block 128 --cmp-stride 32 option times it."""
+    w = workloads.config4()
+    w.cmp_block, w.cmp_stride = 128, 32
+    errs, _ = _sampled_units(runner, w, [(0, 0), (11, 6)])
+    print(errs)
+
+
 def test_config4_full_size_power_law_sampled(runner):
     """The headline shape with the paper's short-term mask (window 8, mask block 1), in the launch
     configuration the benchmark's --short-term power-law option times."""
