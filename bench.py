@@ -204,6 +204,24 @@ def run_reference(args, w, cfg_desc):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ replicas on several GPUs
+def rank_max(x, world, device):
+    """The slowest rank's value of x (a time): every rank returns the same number."""
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return x
+
+
+def replicas_tokens_per_s(world, tokens_per_replica, ms_per_step):
+    """Whole-job throughput of `world` independent replicas that all take the slowest rank's
+    time per step (weak scaling: the work per GPU is fixed)."""
+    return world * tokens_per_replica / (ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -272,11 +290,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x):
-        if world > 1:
-            t = torch.tensor([x], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return x
+        return rank_max(x, world, dev)
 
     p = runner.DeviceProblem(w, device=dev)
     model = work_model(w)
@@ -326,7 +340,7 @@ def main():
     clocks = sampler.stop()
     assert binding.blossom_device_status(p.workspace) == 0
     ms_per_step = max_over_ranks(total_ms / args.steps)
-    value = world * w.tokens / (ms_per_step * 1e-3)
+    value = replicas_tokens_per_s(world, w.tokens, ms_per_step)
 
     # ---- roofline of the kernel with the largest share
     agg = {}
