@@ -110,7 +110,7 @@ def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=No
                     gate, quantize(dout, dtype), seq_lens, stis_mode, stis_block)
 
 
-# The five benchmark configurations (sizes fixed by the task's baseline file).
+# The five benchmark configurations.
 def config1() -> Workload:
     """tiny fp32 correctness case: B4 H2 L64 D32, block 8, top-k 2, window 16, seed 0."""
     return make("cfg1-tiny-fp32", "fp32", 4, 2, 64, 32, 8, 2, 16, seed=0)

@@ -1,6 +1,6 @@
 """GPU-vs-oracle comparison used by the ``-m gpu`` parity tests.
 
-Tolerances (from the task's acceptance bar):
+Tolerances:
   * selected block indices: bit-exact, except rows where the oracle's fp64 scores of the last
     kept and the first dropped candidate differ by < 1e-6 relative;
   * fp32 inputs: max-abs error <= 1e-4 on outputs and gradients;
