@@ -61,6 +61,8 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.qstats = reinterpret_cast<float4 *>(take(units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4)));
   w.cmean = reinterpret_cast<double *>(take(units * (size_t)s.Mc * s.D * sizeof(double)));
   w.clive = reinterpret_cast<int32_t *>(take(units * (size_t)s.Mc * sizeof(int32_t)));
+  w.cmean32 = reinterpret_cast<float *>(take(units * (size_t)s.Mc * s.D * sizeof(float)));
+  w.cnorm = reinterpret_cast<float *>(take(units * (size_t)s.Mc * sizeof(float)));
   w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.bytes = off;

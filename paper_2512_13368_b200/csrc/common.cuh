@@ -34,6 +34,8 @@ struct Workspace {
                      //   {nl_lt(2), -Delta_lt(2)} {nl_st(2), -Delta_st(2)} for the dK/dV kernel
   double *cmean;     // [B][H][Mc][D]  means of the overlapping compression blocks (cmp_l > 0)
   int32_t *clive;    // [B][H][Mc]     their numbers of valid keys
+  float *cmean32;    // [B][H][Mc][D]  the means rounded to fp32
+  float *cnorm;      // [B][H][Mc]     upper bounds of the norms of the fp32 means
   uint8_t *qmeta;    // per query-major CTA of the tensor-core kernels: tile lists (tc_meta_kernel)
   uint8_t *kmeta;    // per key-major CTA (dK/dV kernel): tile lists
   size_t bytes;

@@ -277,8 +277,15 @@ def test_certified_selection_equals_double_precision_selection(runner, monkeypat
     """The two-stage selection (fp32 scores with an error bound, fp64 only for the uncertain query
     blocks) must return exactly what scoring every query block in fp64 returns."""
     import torch
+    overlap4 = workloads.config4(B=1)
+    overlap4.cmp_block, overlap4.cmp_stride = 128, 32          # 125 compression blocks: two chunks
+    overlap2 = workloads.config2(B=16)
+    overlap2.cmp_block, overlap2.cmp_stride = 32, 16           # the paper's default sizes, padded rows
+    small_stride = workloads.make("small-stride", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9)
+    small_stride.cmp_block, small_stride.cmp_stride = 32, 8    # 253 compression blocks: four chunks
     for w in (workloads.config4(B=1), workloads.config2(B=16), workloads.config3(B=1),
-              workloads.make("many-blocks", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9)):
+              workloads.make("many-blocks", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9),
+              overlap4, overlap2, small_stride):
         p = runner.DeviceProblem(w)
         monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
         p.select()
