@@ -97,10 +97,12 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
     }
     __syncwarp();
+    const int gh = G / 2;
+    if (lane == 0) counts[0] = nv;
+    if (!kmeta) {  // ---- forward-only call: the forward's items and their classes ----
     // Long-term items: the tiles both 64-row halves of the CTA need, then alternately a tile only
     // rows 0..63 need and a tile only rows 64..127 need.  A softmax warp may run ahead of the
     // slowest one, so with alternating items both pairs of warps have work at once.
-    const int gh = G / 2;
     int nA = 0, nB = 0, nC = 0;
     for (int pass = 0; pass < 2; ++pass) {
       int cA = 0, cB = 0, cC = 0;
@@ -172,11 +174,13 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
       icls[e] = (uint8_t)cls;
     }
+    }  // forward-only
     __syncwarp();
     // The dQ kernel walks `list` itself (a tile serves both branches there).  Same idea as above:
     // tiles both 64-row halves need first, then alternately a tile only rows 0..63 need and one
     // only rows 64..127 need, so that the two halves' warps work on neighbouring tiles at once.
-    {
+    // (Backward call only; the forward reads `items`.)
+    if (kmeta) {
       uint16_t *tlist = reinterpret_cast<uint16_t *>(meta + ml.bytes);
       uint8_t *tflags = meta + ml.bytes + 2 * nT;
       int nA = 0, nB = 0, nC = 0;
