@@ -199,3 +199,70 @@ def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm
                  stis_block)
     f.update(b)
     return f
+
+
+# ---------------------------------------------------------------------------- grouped-query
+# Grouped-query attention: H query heads share Hkv key/value heads, G = H / Hkv query heads per
+# group, query head h using key/value head h // G.  The importance scores of the heads of a group
+# are summed before the top-k (the paper's group-shared scores, Eq. 12), so a group has one
+# selection.  Given the selection every query head is an ordinary head on its group's K and V, so
+# the attention and its gradients are the functions above applied to K, V repeated per query head,
+# with the K and V gradients of a group's heads summed (the chain rule through the repetition).
+def _group(H, Hkv):
+    if Hkv < 1 or H % Hkv:
+        raise ValueError("heads must be a multiple of kv_heads")
+    return H // Hkv
+
+
+def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False):
+    """q ``[B,H,L,D]``, k ``[B,Hkv,L,D]`` -> idx ``[B,Hkv,M,topk]`` from group-summed scores."""
+    q, k = _f64(q), _f64(k)
+    B, H, L, D = q.shape
+    Hkv = k.shape[1]
+    G = _group(H, Hkv)
+    M = -(-L // block)
+    _, per_head = select_blocks(q, np.repeat(k, G, axis=1), block, topk, seq_lens, sm_scale,
+                                return_scores=True)
+    scores = per_head.reshape(B, Hkv, G, M, M).sum(axis=2)            # Eq. 12
+    idx = np.full((B, Hkv, M, topk), -1, dtype=np.int32)
+    for n in range(B):
+        pad0 = 0 if seq_lens is None else L - int(seq_lens[n])
+        live = np.array([min((j + 1) * block, L) > max(j * block, pad0) for j in range(M)])
+        for g in range(Hkv):
+            for b in range(M):
+                if not live[b]:
+                    continue
+                cand = [j for j in range(b) if live[j]]
+                # Eq. 13: largest scores first, ties to the lower index; the own block always
+                best = sorted(cand, key=lambda j: (-scores[n, g, b, j], j))[:topk - 1]
+                row = sorted(best) + [b]
+                idx[n, g, b, :len(row)] = row
+    return (idx, scores) if return_scores else idx
+
+
+def forward_gqa(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None, **kw):
+    """``forward`` for q ``[B,H,L,D]`` and k, v ``[B,Hkv,L,D]``; idx is ``[B,Hkv,M,topk]``."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    G = _group(q.shape[1], k.shape[1])
+    if idx is None:
+        idx = select_blocks_gqa(q, k, block, topk, seq_lens, sm_scale)
+    idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
+    f = forward(q, np.repeat(k, G, axis=1), np.repeat(v, G, axis=1), gate, block, topk, window,
+                seq_lens, sm_scale, idx=np.repeat(idx, G, axis=1), **kw)
+    f["idx"] = idx
+    return f
+
+
+def backward_gqa(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None, **kw):
+    """``backward`` for grouped heads: dk, dv are ``[B,Hkv,L,D]`` (summed over a group's heads)."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, L, D = q.shape
+    Hkv = k.shape[1]
+    G = _group(H, Hkv)
+    f = dict(fwd)
+    f["idx"] = np.repeat(np.asarray(fwd["idx"], dtype=np.int32), G, axis=1)
+    r = backward(q, np.repeat(k, G, axis=1), np.repeat(v, G, axis=1), gate, block, topk, window, f,
+                 dout, seq_lens, sm_scale, **kw)
+    r["dk"] = r["dk"].reshape(B, Hkv, G, L, D).sum(axis=2)
+    r["dv"] = r["dv"].reshape(B, Hkv, G, L, D).sum(axis=2)
+    return r
