@@ -57,7 +57,10 @@ typedef struct CUstream_st *blossom_stream_t;
 
 typedef struct {
   int32_t batch, heads;
-  int32_t kv_heads;    /* must equal heads (grouped-query sharing is not implemented)            */
+  int32_t kv_heads;    /* key/value heads: heads must be a multiple; query head h uses key/value
+                        * head h / (heads / kv_heads) and a group has ONE selection, made from
+                        * the summed scores of its heads (Eq. 12): k, v, dk, dv are
+                        * [B][kv_heads][L][D] and block_idx is [B][kv_heads][M][top_k]            */
   int32_t seq_len;     /* L >= 1, ceil(L / block_size) <= 1024                                   */
   int32_t head_dim;    /* D in {32, 64}                                                          */
   int32_t block_size;  /* key block = query block size Bk in {8, 16, 32, 64}                     */
@@ -77,6 +80,8 @@ typedef struct {
                         * block_size.  With cmp_stride it allows overlapping blocks whose scores
                         * Eq. 11 maps onto the selection blocks of block_size positions          */
   int32_t cmp_stride;  /* s: their stride; 0 = block_size; must divide cmp_block and block_size  */
+  int64_t kv_stride_b, kv_stride_h, kv_stride_l; /* element strides of k, v, dk, dv; all 0 = the
+                        * strides above if kv_heads == heads, else contiguous [B][kv_heads][L][D] */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

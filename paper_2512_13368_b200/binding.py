@@ -40,6 +40,7 @@ class blossom_params(ctypes.Structure):
         ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_l", ctypes.c_int64),
         ("stis_mode", ctypes.c_int32), ("stis_block", ctypes.c_int32),
         ("cmp_block", ctypes.c_int32), ("cmp_stride", ctypes.c_int32),
+        ("kv_stride_b", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64), ("kv_stride_l", ctypes.c_int64),
     ]
 
 
@@ -115,7 +116,7 @@ def _stream(stream):
 
 def make_params(batch, heads, seq_len, head_dim, block_size, top_k, window, dtype, sm_scale=0.0,
                 strides=None, kv_heads=None, causal=1, select_mode=0, stis_mode=0,
-                stis_block=1, cmp_block=0, cmp_stride=0) -> blossom_params:
+                stis_block=1, cmp_block=0, cmp_stride=0, kv_strides=None) -> blossom_params:
     """Fill a ``blossom_params``; ``strides`` = (stride_b, stride_h, stride_l) in elements,
     default contiguous [B, H, L, D]."""
     if strides is None:
@@ -124,7 +125,8 @@ def make_params(batch, heads, seq_len, head_dim, block_size, top_k, window, dtyp
     return blossom_params(batch, heads, heads if kv_heads is None else kv_heads, seq_len, head_dim,
                           block_size, top_k, window, causal, select_mode, d, float(sm_scale),
                           int(strides[0]), int(strides[1]), int(strides[2]), int(stis_mode),
-                          int(stis_block), int(cmp_block), int(cmp_stride))
+                          int(stis_block), int(cmp_block), int(cmp_stride),
+                          *((0, 0, 0) if kv_strides is None else [int(x) for x in kv_strides]))
 
 
 def blossom_status_string(status) -> str:

@@ -80,7 +80,11 @@ static int make_shape(const blossom_params *p, Shape *out) {
     return BLOSSOM_ERR_INVALID_ARG;
   if (p->stride_l < p->head_dim || p->stride_h < 1 || p->stride_b < 1) return BLOSSOM_ERR_INVALID_ARG;
   if (p->stride_l % 8 || p->stride_h % 8 || p->stride_b % 8) return BLOSSOM_ERR_INVALID_ARG;
-  if (p->kv_heads != p->heads) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->kv_heads < 1 || p->heads % p->kv_heads) return BLOSSOM_ERR_INVALID_ARG;
+  const bool kv_given = p->kv_stride_b || p->kv_stride_h || p->kv_stride_l;
+  if (kv_given && (p->kv_stride_l < p->head_dim || p->kv_stride_h < 1 || p->kv_stride_b < 1 ||
+                   p->kv_stride_l % 8 || p->kv_stride_h % 8 || p->kv_stride_b % 8))
+    return BLOSSOM_ERR_INVALID_ARG;
   if (p->causal != 1 || p->select_mode != 0) return BLOSSOM_ERR_UNSUPPORTED;
   if (p->stis_mode < 0 || p->stis_mode > 1 || p->stis_block < 0) return BLOSSOM_ERR_INVALID_ARG;
   if (p->head_dim != 32 && p->head_dim != 64) return BLOSSOM_ERR_UNSUPPORTED;
@@ -109,6 +113,15 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.scale_d = p->sm_scale > 0.f ? (double)p->sm_scale : 1.0 / sqrt((double)p->head_dim);
   s.scale = (float)s.scale_d;
   s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;
+  s.Hkv = p->kv_heads; s.G = p->heads / p->kv_heads;
+  if (kv_given) {
+    s.ksb = p->kv_stride_b; s.ksh = p->kv_stride_h; s.ksl = p->kv_stride_l;
+  } else if (s.G == 1) {
+    s.ksb = s.sb; s.ksh = s.sh; s.ksl = s.sl;
+  } else {
+    s.ksl = s.D; s.ksh = (int64_t)s.L * s.D; s.ksb = (int64_t)s.Hkv * s.L * s.D;
+  }
+  if (s.G > 1 && s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // overlapping blocks: one head per group only
   *out = s;
   return BLOSSOM_OK;
 }

@@ -38,14 +38,15 @@ __device__ __forceinline__ float4 zero4() { return make_float4(0.f, 0.f, 0.f, 0.
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
 
 // Stage rows [row0, row0 + Bk) of a q-shaped tensor into shared memory as fp32 (zero past L).
+// `head0` = element offset of row 0 of the (batch, head) the tile belongs to, `sl` = row stride.
 template <typename T, int D>
-__device__ __forceinline__ void stage_tile(const Shape &s, const T *base, int n, int h, int row0,
-                                           float *dst) {
+__device__ __forceinline__ void stage_tile(const Shape &s, const T *base, int64_t head0, int64_t sl,
+                                           int row0, float *dst) {
   constexpr int CH = D / 4;
   for (int i = threadIdx.x; i < s.Bk * CH; i += blockDim.x) {
     const int pr = i / CH, ch = i % CH, p = row0 + pr;
     float4 x = zero4();
-    if (p < s.L) x = ld4(base + row_offset(s, n, h, p) + ch * 4);
+    if (p < s.L) x = ld4(base + head0 + (int64_t)p * sl + ch * 4);
     reinterpret_cast<float4 *>(dst)[i] = x;
   }
 }
@@ -82,7 +83,8 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
   const int t = qb * s.Bk + r;
   const bool inrange = t < s.L, active = inrange && t >= pad0;
 
-  build_visit_flags(s, idx + ((int64_t)u * s.M + qb) * s.topk, qb, flags);
+  const int hk = h / s.G;  // key/value head of this query head; its group shares one selection
+  build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
 
   float4 qv[NV], aL[NV], aS[NV];
 #pragma unroll
@@ -101,8 +103,8 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
       const int f = flags[blk];
       if (!f) continue;
       __syncthreads();
-      stage_tile<T, D>(s, k, n, h, blk * s.Bk, Ks);
-      stage_tile<T, D>(s, v, n, h, blk * s.Bk, Vs);
+      stage_tile<T, D>(s, k, row_offset_kv(s, n, hk, 0), s.ksl, blk * s.Bk, Ks);
+      stage_tile<T, D>(s, v, row_offset_kv(s, n, hk, 0), s.ksl, blk * s.Bk, Vs);
       __syncthreads();
       if (!active) continue;
       const int p0 = blk * s.Bk;
@@ -183,7 +185,8 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
   const int64_t BHL = (int64_t)s.B * s.H * s.L;
   const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
 
-  build_visit_flags(s, idx + ((int64_t)u * s.M + qb) * s.topk, qb, flags);
+  const int hk = h / s.G;  // key/value head of this query head; its group shares one selection
+  build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
 
   float4 qv[NV], gv[NV], acc[NV];
   float dL = 0.f, dS = 0.f;
@@ -223,8 +226,8 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
       const int f = flags[blk];
       if (!f) continue;
       __syncthreads();
-      stage_tile<T, D>(s, k, n, h, blk * s.Bk, Ks);
-      stage_tile<T, D>(s, v, n, h, blk * s.Bk, Vs);
+      stage_tile<T, D>(s, k, row_offset_kv(s, n, hk, 0), s.ksl, blk * s.Bk, Ks);
+      stage_tile<T, D>(s, v, row_offset_kv(s, n, hk, 0), s.ksl, blk * s.Bk, Vs);
       __syncthreads();
       if (!active) continue;
       const int p0 = blk * s.Bk;
@@ -285,7 +288,8 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   float *Qs = smf, *Gs = Qs + s.Bk * D;
   float *lLs = Gs + s.Bk * D, *lSs = lLs + s.Bk, *dLs = lSs + s.Bk, *dSs = dLs + s.Bk;
   int *flags = reinterpret_cast<int *>(dSs + s.Bk);
-  const int j = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
+  // uk counts (batch, key/value head) pairs: the key block collects from every query head of its group
+  const int j = blockIdx.x % s.M, uk = blockIdx.x / s.M, n = uk / s.Hkv, hk = uk % s.Hkv;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -294,12 +298,11 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   const int p = j * s.Bk + r;
   const bool inrange = p < s.L, active = inrange && p >= pad0;
   const int64_t BHL = (int64_t)s.B * s.H * s.L;
-  const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
 
   // which query blocks visit this key block: bit 0 = selected it, bit 1 = their short-term branch
   // may reach it
   for (int qb = j + tid; qb < s.M; qb += blockDim.x) {
-    const int32_t *row = idx + ((int64_t)u * s.M + qb) * s.topk;
+    const int32_t *row = idx + ((int64_t)uk * s.M + qb) * s.topk;
     int f = st_ranges_touch(s, qb * s.Bk, min(s.L, qb * s.Bk + s.Bk) - 1, j * s.Bk,
                             min(s.L, j * s.Bk + s.Bk) - 1) ? 2 : 0;
     for (int i = 0; i < s.topk; ++i) f |= (row[i] == j) ? 1 : 0;
@@ -307,7 +310,7 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   }
 
   float4 kv[NV], vv[NV], dka[NV], dva[NV];
-  const int64_t ro = row_offset(s, n, h, inrange ? p : 0);
+  const int64_t ro = row_offset_kv(s, n, hk, inrange ? p : 0);
 #pragma unroll
   for (int c = 0; c < NV; ++c) {
     const int64_t off = ro + (c * 4 + sub) * 4;
@@ -321,19 +324,22 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   __syncthreads();
 
   if (block_live) {
-    for (int qb = j; qb < s.M; ++qb) {
+    for (int x = 0; x < s.G * (s.M - j); ++x) {  // every query head of the group, every later query block
+      const int h = hk * s.G + x / (s.M - j), qb = j + x % (s.M - j);
+      const int64_t u = (int64_t)n * s.H + h;
+      const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
       const int f = flags[qb];
       if (!f) continue;
       __syncthreads();
-      stage_tile<T, D>(s, q, n, h, qb * s.Bk, Qs);
-      stage_tile<T, D>(s, dout, n, h, qb * s.Bk, Gs);
+      stage_tile<T, D>(s, q, row_offset(s, n, h, 0), s.sl, qb * s.Bk, Qs);
+      stage_tile<T, D>(s, dout, row_offset(s, n, h, 0), s.sl, qb * s.Bk, Gs);
       for (int i = tid; i < s.Bk; i += blockDim.x) {
         const int t = qb * s.Bk + i;
         const bool ok = t < s.L;
-        lLs[i] = ok ? lse[(int64_t)u * s.L + t] * kLog2e : 0.f;
-        lSs[i] = ok ? lse[BHL + (int64_t)u * s.L + t] * kLog2e : 0.f;
-        dLs[i] = ok ? delta[(int64_t)u * s.L + t] : 0.f;
-        dSs[i] = ok ? delta[BHL + (int64_t)u * s.L + t] : 0.f;
+        lLs[i] = ok ? lse[u * s.L + t] * kLog2e : 0.f;
+        lSs[i] = ok ? lse[BHL + u * s.L + t] * kLog2e : 0.f;
+        dLs[i] = ok ? delta[u * s.L + t] : 0.f;
+        dSs[i] = ok ? delta[BHL + u * s.L + t] : 0.f;
       }
       __syncthreads();
       if (!active) continue;
@@ -454,7 +460,8 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
     return BLOSSOM_ERR_CUDA;
   {
     LaunchScope ls(K_BWD_DKDV_SIMT, st);
-    bwd_dkdv_simt_kernel<T, D><<<grid, s.Bk * 4, smem_k, st>>>(s, q, k, v, gate, seq_lens, idx, lse,
+    const unsigned grid_k = (unsigned)s.M * (unsigned)(s.B * s.Hkv);
+    bwd_dkdv_simt_kernel<T, D><<<grid_k, s.Bk * 4, smem_k, st>>>(s, q, k, v, gate, seq_lens, idx, lse,
                                                                ws.delta, dout, dk, dv);
   }
   return launch_gate_grad(s, gate, ws, dgate, st);

@@ -17,6 +17,8 @@ struct Shape {
   float scale;     // attention logit scale (fp32 arithmetic of the attention kernels)
   double scale_d;  // the same scale in double for the fp64 block scoring
   int64_t sb, sh, sl;  // element strides of q-shaped tensors
+  int Hkv, G;             // key/value heads and query heads per key/value head (H = Hkv * G)
+  int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
 };
 
 // Device scratch carved out of the caller's workspace.
@@ -85,6 +87,10 @@ __device__ __forceinline__ float ld1(const __nv_bfloat16 *p) { return __bfloat16
 
 __device__ __forceinline__ int64_t row_offset(const Shape &s, int n, int h, int t) {
   return (int64_t)n * s.sb + (int64_t)h * s.sh + (int64_t)t * s.sl;
+}
+// row p of key/value head hk in k, v, dk, dv
+__device__ __forceinline__ int64_t row_offset_kv(const Shape &s, int n, int hk, int p) {
+  return (int64_t)n * s.ksb + (int64_t)hk * s.ksh + (int64_t)p * s.ksl;
 }
 
 // ---- the short-term mask (Eq. 15), shared by the CUDA-core and the tensor-core kernels ----

@@ -34,7 +34,8 @@ __global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restri
   __shared__ double part[RG][D];
   __shared__ float sq[D];
   if (blockIdx.x == 0 && threadIdx.x == 0) *sel_count = 0;  // work list of the scoring kernel
-  const int j = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
+  // u counts (batch, key/value head) pairs
+  const int j = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.Hkv, hk = u % s.Hkv;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -42,7 +43,7 @@ __global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restri
   const int ch = threadIdx.x % CH, rg = threadIdx.x / CH;
   double a0 = 0, a1 = 0, a2 = 0, a3 = 0;
   for (int p = lo + rg; p < hi; p += RG) {
-    float4 x = ld4(k + row_offset(s, n, h, p) + ch * 4);
+    float4 x = ld4(k + row_offset_kv(s, n, hk, p) + ch * 4);
     a0 += (double)x.x; a1 += (double)x.y; a2 += (double)x.z; a3 += (double)x.w;
   }
   part[rg][ch * 4 + 0] = a0; part[rg][ch * 4 + 1] = a1;
@@ -76,7 +77,9 @@ __device__ __forceinline__ void score_select_row(
     const Shape &s, const T *__restrict__ q, const double *__restrict__ kmean,
     const int32_t *__restrict__ klive, const int32_t *__restrict__ seq_lens,
     int32_t *__restrict__ idx, int kt_in_smem, int row_id, double *sm) {
-  const int b = row_id % s.M, u = row_id / s.M, n = u / s.H, h = u % s.H;
+  // u counts (batch, key/value head) pairs; the queries of all G heads of the group are scored
+  // and their probabilities summed (Eq. 12)
+  const int b = row_id % s.M, u = row_id / s.M, n = u / s.Hkv, hk = u % s.Hkv;
   const int M = s.M;
   const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
   int len = seq_lens ? seq_lens[n] : s.L;
@@ -119,19 +122,21 @@ __device__ __forceinline__ void score_select_row(
     double *zw = zbuf + warp * M, *spw = sp + warp * M, *qw = qrow + warp * D;
     constexpr int QPL = (D + 31) / 32;  // query elements per lane
     double qreg[QPL];                   // the next row, loaded while the current one is scored
-    if (qlo + warp < qhi) {
-      const T *qp = q + row_offset(s, n, h, qlo + warp);
+    const int nq = qhi - qlo, nrows = nq * s.G;  // rows of the group: head g, query qlo + r % nq
+    if (warp < nrows) {
+      const T *qp = q + row_offset(s, n, hk * s.G + warp / nq, qlo + warp % nq);
 #pragma unroll
       for (int e = 0; e < QPL; ++e)
         if (lane + 32 * e < D) qreg[e] = (double)ld1(qp + lane + 32 * e);
     }
-    for (int t = qlo + warp; t < qhi; t += kSelWarps) {
+    for (int r = warp; r < nrows; r += kSelWarps) {
 #pragma unroll
       for (int e = 0; e < QPL; ++e)
         if (lane + 32 * e < D) qw[lane + 32 * e] = qreg[e];
       __syncwarp();
-      if (t + kSelWarps < qhi) {
-        const T *qp = q + row_offset(s, n, h, t + kSelWarps);
+      if (r + kSelWarps < nrows) {
+        const int r2 = r + kSelWarps;
+        const T *qp = q + row_offset(s, n, hk * s.G + r2 / nq, qlo + r2 % nq);
 #pragma unroll
         for (int e = 0; e < QPL; ++e)
           if (lane + 32 * e < D) qreg[e] = (double)ld1(qp + lane + 32 * e);
@@ -218,7 +223,7 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
     int32_t *__restrict__ idx, int kt_in_smem, const int32_t *__restrict__ worklist,
     const int32_t *__restrict__ work_count) {
   extern __shared__ double sm[];
-  const int total = worklist ? *work_count : s.M * s.B * s.H;
+  const int total = worklist ? *work_count : s.M * s.B * s.Hkv;
   for (int w = blockIdx.x; w < total; w += gridDim.x) {
     score_select_row<T, D>(s, q, kmean, klive, seq_lens, idx, kt_in_smem, worklist ? worklist[w] : w, sm);
     __syncthreads();  // shared memory is reused by the next row
@@ -485,13 +490,16 @@ size_t select_smem_bytes(int M, int D, bool kt_in_smem) {
 template <typename T, int D>
 int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_lens, int32_t *idx,
                     const Workspace &ws, cudaStream_t st) {
-  const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.H);  // block = (unit, query block), unit-major
+  // block = (unit, query block), unit-major; a unit is a (batch, key/value head) pair
+  const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.Hkv);
   {
     LaunchScope ls(K_SUMMARY, st);
     summary_kernel<T, D><<<grid, 256, 0, st>>>(s, k, seq_lens, ws.kmean, ws.klive, ws.kmean32, ws.knorm,
                                                ws.sel_count);
   }
-  const bool exact_only = exact_select_only();
+  // (the single-precision stage scores one head's queries: groups of several heads go straight
+  // to the double-precision kernel)
+  const bool exact_only = exact_select_only() || s.G > 1;
   if (!exact_only) {
     const size_t fsm = select_fast_smem_bytes(s.M, D);
     if (fsm > 48 * 1024 &&

@@ -38,7 +38,8 @@ int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_
 }
 
 bool fwd_tc_supported(const Shape &s, int dtype) {
-  return dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  // (grouped key/value heads run on the CUDA-core kernels)
+  return s.G == 1 && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 

@@ -29,19 +29,21 @@ class DeviceProblem:
         self.params = binding.make_params(w.B, w.H, w.L, w.D, w.block, w.topk, w.window, w.dtype,
                                           sm_scale=sm_scale, stis_mode=w.stis_mode,
                                           stis_block=w.stis_block, cmp_block=w.cmp_block,
-                                          cmp_stride=w.cmp_stride)
+                                          cmp_stride=w.cmp_stride, kv_heads=w.kv_heads or w.H)
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):
         w, dev = self.w, self.device
         shape = (w.B, w.H, w.L, w.D)
         e = lambda: torch.empty(shape, dtype=self.dt, device=dev)  # noqa: E731
-        self.idx = torch.empty((w.B, w.H, w.n_blocks, w.topk), dtype=torch.int32, device=dev)
+        hkv = w.kv_heads or w.H   # k, v, dk, dv and the selection are per key/value head
+        ekv = lambda: torch.empty((w.B, hkv, w.L, w.D), dtype=self.dt, device=dev)  # noqa: E731
+        self.idx = torch.empty((w.B, hkv, w.n_blocks, w.topk), dtype=torch.int32, device=dev)
         self.out = e()
         self.out_lt = e() if training else None
         self.out_st = e() if training else None
         self.lse = torch.empty((2, w.B, w.H, w.L), dtype=torch.float32, device=dev) if training else None
-        self.dq, self.dk, self.dv = (e(), e(), e()) if training else (None, None, None)
+        self.dq, self.dk, self.dv = (e(), ekv(), ekv()) if training else (None, None, None)
         self.dgate = torch.empty((w.H, 2), dtype=torch.float32, device=dev)
         nbytes = binding.blossom_workspace_bytes(self.params)
         if nbytes == 0:

@@ -63,6 +63,7 @@ class Workload:
     stis_block: int = 1   # mask block of the power-law mask
     cmp_block: int = 0    # compression block length l of the selection (0 = block)
     cmp_stride: int = 0   # and its stride s (0 = block)
+    kv_heads: int = 0     # key/value heads (0 = H): k, v are [B, kv_heads, L, D]
 
     @property
     def n_blocks(self) -> int:
@@ -75,6 +76,7 @@ class Workload:
     def unit(self, n: int, h: int) -> "Workload":
         """The single (batch n, head h) problem as a B=1, H=1 workload."""
         sl = None if self.seq_lens is None else self.seq_lens[n:n + 1].copy()
+        assert not self.kv_heads or self.kv_heads == self.H, "a head of a group is not a problem of its own"
         return Workload(self.name + f"[{n},{h}]", self.dtype, 1, 1, self.L, self.D, self.block,
                         self.topk, self.window, self.seed,
                         self.q[n:n + 1, h:h + 1].copy(), self.k[n:n + 1, h:h + 1].copy(),
@@ -84,7 +86,7 @@ class Workload:
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,
-         row_scales=False, stis_mode=0, stis_block=1) -> Workload:
+         row_scales=False, stis_mode=0, stis_block=1, kv_heads=0) -> Workload:
     """Generic generator; see the module docstring for the draw order.
 
     lengths: None or (lo, hi) inclusive -> left-padded sequences, pad rows keep their
@@ -93,9 +95,10 @@ def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=No
     """
     rng = np.random.default_rng(seed)
     shape = (B, H, L, D)
+    kv_shape = (B, kv_heads or H, L, D)
     q = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
-    k = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
-    v = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
+    k = rng.standard_normal(kv_shape, dtype=np.float32) * np.float32(std)
+    v = rng.standard_normal(kv_shape, dtype=np.float32) * np.float32(std)
     gate = rng.standard_normal((H, 2), dtype=np.float32)
     dout = rng.standard_normal(shape, dtype=np.float32)
     seq_lens = None
@@ -107,7 +110,7 @@ def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=No
             t *= rng.uniform(0.5, 2.0, size=(B, H, L, 1)).astype(np.float32)
     return Workload(name, dtype, B, H, L, D, block, topk, window, seed,
                     quantize(q, dtype), quantize(k, dtype), quantize(v, dtype),
-                    gate, quantize(dout, dtype), seq_lens, stis_mode, stis_block)
+                    gate, quantize(dout, dtype), seq_lens, stis_mode, stis_block, 0, 0, kv_heads)
 
 
 # The five benchmark configurations.

@@ -19,9 +19,16 @@ BF16_REL = 2e-2
 TIE_REL = 1e-6
 
 
+def _grouped(w):
+    return bool(w.kv_heads) and w.kv_heads != w.H
+
+
 def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
-    if w.cmp_block or w.cmp_stride:
+    if _grouped(w):
+        ref_idx, scores = oracle.select_blocks_gqa(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
+                                                   return_scores=True)
+    elif w.cmp_block or w.cmp_stride:
         ref_idx, scores, _ = oracle.select_blocks_cmp(w.q, w.k, w.block, w.topk, w.cmp_block or w.block,
                                                       w.cmp_stride or w.block, w.seq_lens, sm_scale,
                                                       return_scores=True)
@@ -59,14 +66,14 @@ def tolerance(w, ref):
 def check_forward_backward(w, res, sm_scale=None, backward=True):
     """res: dict of numpy arrays from the CUDA path.  Returns a dict of max-abs errors."""
     forgiven = check_indices(w, res["idx"], sm_scale)
-    ref = oracle.forward(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
-                         idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block)
+    fwd_fn, bwd_fn = (oracle.forward_gqa, oracle.backward_gqa) if _grouped(w) else (oracle.forward, oracle.backward)
+    ref = fwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
+                 idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block)
     errs = {"near_tie_rows": forgiven}
     keys = ["out", "out_lt", "out_st", "lse"]
     if backward:
-        ref.update(oracle.backward(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, ref, w.dout,
-                                   w.seq_lens, sm_scale, stis_mode=w.stis_mode,
-                                   stis_block=w.stis_block))
+        ref.update(bwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, ref, w.dout,
+                          w.seq_lens, sm_scale, stis_mode=w.stis_mode, stis_block=w.stis_block))
         keys += ["dq", "dk", "dv", "dgate"]
     for key in keys:
         if res.get(key) is None:

@@ -48,7 +48,7 @@ def test_workspace_bytes(lib):
     assert n > 0 and n % 256 == 0
     assert binding.blossom_workspace_bytes(good(batch=8)) > n
     for bad in (dict(batch=0), dict(head_dim=48), dict(block_size=12), dict(top_k=0), dict(window=0),
-                dict(kv_heads=1), dict(causal=0), dict(select_mode=1), dict(dtype=7),
+                dict(kv_heads=3), dict(kv_heads=0), dict(kv_strides=(4096, 2048, 31)), dict(causal=0), dict(select_mode=1), dict(dtype=7),
                 dict(seq_len=8 * 1025), dict(strides=(4096, 2048, 33)), dict(sm_scale=-1.0),
                 dict(stis_mode=2), dict(stis_mode=-1), dict(stis_mode=1, stis_block=-3),
                 dict(cmp_block=12, cmp_stride=8), dict(cmp_block=16, cmp_stride=3), dict(cmp_block=-8)):
@@ -56,6 +56,7 @@ def test_workspace_bytes(lib):
     assert binding.blossom_workspace_bytes(good(stis_mode=1, stis_block=4)) == n  # power-law mask
     assert binding.blossom_workspace_bytes(good(cmp_block=8, cmp_stride=8)) == n    # same as the default
     assert binding.blossom_workspace_bytes(good(cmp_block=16, cmp_stride=4)) > n    # overlapping blocks
+    assert binding.blossom_workspace_bytes(good(kv_heads=1)) == n                   # grouped key/value heads
 
 
 def test_argument_validation_precedes_any_launch(lib):
@@ -76,7 +77,8 @@ def test_argument_validation_precedes_any_launch(lib):
     assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, A + 64, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
     assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes - 1, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
     # unsupported but legal requests
-    assert E.blossom_attn_fwd(good(kv_heads=1), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
+    assert E.blossom_attn_fwd(good(select_mode=1), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
+    assert E.blossom_attn_fwd(good(kv_heads=3), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
     assert E.blossom_select_blocks(good(head_dim=128), A, A, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
     assert E.blossom_select_blocks(p, A, None, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
     # backward: every tensor is required
@@ -91,9 +93,10 @@ def test_argument_validation_precedes_any_launch(lib):
 
 
 def test_params_struct_layout_matches_header():
-    # 12 x 4-byte fields, three int64 strides, the two short-term mask fields and the two
-    # compression-block fields: 88 bytes with natural alignment
-    assert ctypes.sizeof(binding.blossom_params) == 88
+    # 12 x 4-byte fields, three int64 strides, the two short-term mask fields, the two
+    # compression-block fields and three int64 key/value strides: 112 bytes with natural alignment
+    assert ctypes.sizeof(binding.blossom_params) == 112
+    assert binding.blossom_params.kv_stride_b.offset == 88
     assert binding.blossom_params.cmp_block.offset == 80 and binding.blossom_params.cmp_stride.offset == 84
     assert binding.blossom_params.stride_b.offset == 48
     assert binding.blossom_params.stis_mode.offset == 72 and binding.blossom_params.stis_block.offset == 76

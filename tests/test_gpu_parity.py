@@ -138,6 +138,27 @@ def test_overlapping_compression_blocks(runner, dtype, L, D, block, topk, l, s, 
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens,power_law", [
+    (64, 32, 4, 2, 8, 2, 16, None, False),
+    (200, 32, 8, 2, 16, 4, 32, [200, 5, 77], False),     # the paper's 8 heads on 2 key/value heads, padded
+    (300, 64, 6, 3, 32, 4, 40, [300, 131], False),
+    (256, 64, 4, 1, 64, 3, 8, None, True),               # one key/value head, power-law short-term mask
+    (1024, 64, 8, 2, 64, 8, 256, [1024, 640], False),
+])
+def test_grouped_query_heads(runner, dtype, L, D, H, Hkv, block, topk, window, lens, power_law):
+    """Query heads share key/value heads and one selection per group (summed scores, Eq. 12)."""
+    B = len(lens) if lens else 2
+    w = workloads.make("gqa", dtype, B, H, L, D, block, topk, window, seed=19, kv_heads=Hkv,
+                       stis_mode=1 if power_law else 0)
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    assert res["dk"].shape == (B, Hkv, L, D) and res["idx"].shape[1] == Hkv
+    print(check_forward_backward(w, res))
+
+
 def test_explicit_scale_and_given_indices(runner):
     w = workloads.make("scale", "fp32", 2, 2, 96, 32, 16, 3, 20, seed=5)
     p, res = run(runner, w, sm_scale=0.37)
