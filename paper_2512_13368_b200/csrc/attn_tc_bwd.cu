@@ -247,8 +247,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         const int row = (int)list[j] * 64;
         if (elect_one()) {
           mbar_expect_tx(bar, 2 * C::kSmallBytes);
-          tma_load_4d(kt, &tmk, bar, 0, row, h, n);
-          tma_load_4d(kt + C::kSmallBytes, &tmv, bar, 0, row, h, n);
+          tma_load_4d(kt, &tmk, bar, 0, row, h / s.G, n);  // the key/value head of this query head
+          tma_load_4d(kt + C::kSmallBytes, &tmv, bar, 0, row, h / s.G, n);
         }
         __syncwarp();
       }
@@ -491,7 +491,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nKT = (s.L + 127) >> 7;
   const int kt = (int)(blockIdx.x % nKT);  // early keys have the most visitors: first
-  const int u = blockIdx.x / nKT, n = u / s.H, h = u % s.H;
+  // a CTA owns 128 keys of one (batch, key/value head) and collects from every query head of the group
+  const int uk = blockIdx.x / nKT, n = uk / s.Hkv, hk = uk % s.Hkv;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -537,8 +538,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
     bulk_load(smem_u32(meta), kmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, 2 * C::kBigBytes);
-    tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, h, n);
-    tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, h, n);
+    tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, hk, n);
+    tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, hk, n);
   }
   if (warp == 0) {
     __syncwarp();
@@ -549,7 +550,10 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   __syncthreads();
   tc_fence_after();
   mbar_wait(b_meta, 0, &abort_flag, 224);
-  const int nvis = *reinterpret_cast<const int *>(meta + ml.counts);
+  // The tile list is the same for every query head of the group (one selection per group): the
+  // kernel walks it once per head, item x = (head x / nlist, tile list[x % nlist]).
+  const int nlist = *reinterpret_cast<const int *>(meta + ml.counts);
+  const int nvis = nlist * s.G;
   const uint32_t tmem_base = tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_dv = tmem_base + 128,
                  tmem_dk = tmem_base + 192;
@@ -564,12 +568,12 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 214);
         const uint32_t bar = b_full + 8 * sj;
         const uint32_t qt_ = smem_u32(qg_tiles + sj * kStageBytes);
-        const int row = (int)list[j] * 64;
+        const int row = (int)list[j % nlist] * 64, h = hk * s.G + j / nlist;
         if (elect_one()) {
           mbar_expect_tx(bar, kStageBytes);
           tma_load_4d(qt_, &tmq, bar, 0, row, h, n);
           tma_load_4d(qt_ + C::kSmallBytes, &tmg, bar, 0, row, h, n);
-          bulk_load(qt_ + 2 * C::kSmallBytes, qstats + (int64_t)u * Lpad + row, kStatBytes, bar);
+          bulk_load(qt_ + 2 * C::kSmallBytes, qstats + ((int64_t)n * s.H + h) * Lpad + row, kStatBytes, bar);
         }
         __syncwarp();
       }
@@ -628,7 +632,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const float sc2 = s.scale * kLog2e;
 
     for (int i = 0; i < nvis; ++i) {
-      const int qt = list[i], f = lflags[i], t0 = qt * 64;
+      const int qt = list[i % nlist], f = lflags[i % nlist], t0 = qt * 64;
       uint64_t maskL = 0ull, maskS = 0ull;
       if (row_valid) {
         const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
@@ -723,8 +727,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       fence_async_smem();
       named_bar_sync(5, kComputeWarps * 32);
       if (tid == 0) {
-        tma_store_4d(&tmdv, smem_u32(sv_t), 0, key0, h, n);
-        tma_store_4d(&tmdk, smem_u32(sk_t), 0, key0, h, n);
+        tma_store_4d(&tmdv, smem_u32(sv_t), 0, key0, hk, n);
+        tma_store_4d(&tmdk, smem_u32(sk_t), 0, key0, hk, n);
         tma_store_commit_and_wait();
       }
     }
@@ -743,11 +747,12 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   typedef __nv_bfloat16 bf;
   using C = Cfg<D>;
   CUtensorMap q128, k64, v64, g128, q64, k128, v128, g64, tdq, tdk, tdv;
-  if (make_tensor_map(&q128, q, s, 128) || make_tensor_map(&k64, k, s, 64) ||
-      make_tensor_map(&v64, v, s, 64) || make_tensor_map(&g128, dout, s, 128) ||
-      make_tensor_map(&q64, q, s, 64) || make_tensor_map(&k128, k, s, 128) ||
-      make_tensor_map(&v128, v, s, 128) || make_tensor_map(&g64, dout, s, 64) ||
-      make_tensor_map(&tdq, dq, s, 128) || make_tensor_map(&tdk, dk, s, 128) || make_tensor_map(&tdv, dv, s, 128))
+  if (make_tensor_map(&q128, q, s, 128) || make_tensor_map(&k64, k, s, 64, true) ||
+      make_tensor_map(&v64, v, s, 64, true) || make_tensor_map(&g128, dout, s, 128) ||
+      make_tensor_map(&q64, q, s, 64) || make_tensor_map(&k128, k, s, 128, true) ||
+      make_tensor_map(&v128, v, s, 128, true) || make_tensor_map(&g64, dout, s, 64) ||
+      make_tensor_map(&tdq, dq, s, 128) || make_tensor_map(&tdk, dk, s, 128, true) ||
+      make_tensor_map(&tdv, dv, s, 128, true))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
@@ -773,7 +778,8 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
-    bwd_dkdv_tc_kernel<D><<<grid, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
+    const unsigned grid_k = (unsigned)nST * (unsigned)(s.B * s.Hkv);
+    bwd_dkdv_tc_kernel<D><<<grid_k, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
                                                              ws.qstats, tdk, tdv, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;

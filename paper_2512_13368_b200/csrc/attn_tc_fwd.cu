@@ -198,8 +198,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         const int row = (int)items[j] * 64;
         if (elect_one()) {
           mbar_expect_tx(bar, 2 * C::kSmallBytes);
-          tma_load_4d(kt, &tmk, bar, 0, row, h, n);
-          tma_load_4d(kt + C::kSmallBytes, &tmv, bar, 0, row, h, n);
+          tma_load_4d(kt, &tmk, bar, 0, row, h / s.G, n);  // the key/value head of this query head
+          tma_load_4d(kt + C::kSmallBytes, &tmv, bar, 0, row, h / s.G, n);
         }
         __syncwarp();
       }
@@ -427,7 +427,8 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   using C = Cfg<D>;
   CUtensorMap tq, tk, tv, to, tol, tos;
   const int training = out_lt != nullptr;
-  if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64) || make_tensor_map(&tv, v, s, 64) ||
+  if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64, true) ||
+      make_tensor_map(&tv, v, s, 64, true) ||
       make_tensor_map(&to, out, s, 128) || make_tensor_map(&tol, training ? out_lt : out, s, 128) ||
       make_tensor_map(&tos, training ? out_st : out, s, 128))
     return BLOSSOM_ERR_CUDA;

@@ -44,7 +44,10 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   const int nST = (s.L + 127) >> 7;
   const bool key_major = image >= n_query_ctas;
   const int cta = key_major ? image - n_query_ctas : image;
-  const int u = cta / nST, n = u / s.H;
+  // query-major CTAs count (batch, query head) pairs, key-major CTAs (batch, key/value head) pairs;
+  // uk = the (batch, key/value head) pair whose selection the image is built from
+  const int u = cta / nST, n = key_major ? u / s.Hkv : u / s.H;
+  const int uk = key_major ? u : n * s.Hkv + (u % s.H) / s.G;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -69,7 +72,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     for (int i = lane; i < G * s.topk; i += 32) {  // the selections of the CTA's query blocks
       const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
       if (qb < s.M) {
-        const int blk = idx[((int64_t)u * s.M + qb) * s.topk + slot];
+        const int blk = idx[((int64_t)uk * s.M + qb) * s.topk + slot];
         if (blk >= 0 && blk <= qb) {
           const int a = g * nT + blk / nb;
           atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
@@ -264,7 +267,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
       // (the index rows of query blocks qb0 .. M-1 are contiguous; eight loads in flight per lane)
       const int qb0 = kt * G, total = (s.M - qb0) * s.topk;
-      const int32_t *rows = idx + ((int64_t)u * s.M + qb0) * s.topk;
+      const int32_t *rows = idx + ((int64_t)uk * s.M + qb0) * s.topk;
       for (int base = 0; base < total; base += 256) {
         int blk[8];
 #pragma unroll
@@ -313,7 +316,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
 int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
                    uint8_t *kmeta, cudaStream_t st) {
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
-  const int nq = nST * s.B * s.H, n_images = kmeta ? 2 * nq : nq;
+  const int nq = nST * s.B * s.H, n_images = kmeta ? nq + nST * s.B * s.Hkv : nq;
   const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT) + ((3 * nT + 15) / 16) * 16);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(tc_meta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

@@ -23,11 +23,13 @@ static EncodeTiledFn encode_fn() {
 
 // q-shaped bf16 tensor [B][H][L][D] with the caller's strides, box = (D, box_rows, 1, 1); rows
 // past L read as zeros.  The swizzle matches the shared-memory descriptors of the kernels.
-int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows) {
+int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows, bool kv) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return 1;
-  const cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.L, (cuuint64_t)s.H, (cuuint64_t)s.B};
-  const cuuint64_t strides[3] = {(cuuint64_t)s.sl * 2, (cuuint64_t)s.sh * 2, (cuuint64_t)s.sb * 2};
+  // kv: a key/value-shaped tensor [B][Hkv][L][D] with its own strides
+  const cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.L, (cuuint64_t)(kv ? s.Hkv : s.H), (cuuint64_t)s.B};
+  const cuuint64_t strides[3] = {(cuuint64_t)(kv ? s.ksl : s.sl) * 2, (cuuint64_t)(kv ? s.ksh : s.sh) * 2,
+                                 (cuuint64_t)(kv ? s.ksb : s.sb) * 2};
   const cuuint32_t box[4] = {(cuuint32_t)s.D, (cuuint32_t)box_rows, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   const CUtensorMapSwizzle sw = s.D == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
@@ -38,8 +40,7 @@ int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_
 }
 
 bool fwd_tc_supported(const Shape &s, int dtype) {
-  // (grouped key/value heads run on the CUDA-core kernels)
-  return s.G == 1 && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  return dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 
