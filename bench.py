@@ -51,7 +51,8 @@ def work_model(w):
     tile FLOPs = 2 * Bk * Bk * D per GEMM per visited tile and branch; forward 2 GEMMs
     (QK^T, PV), backward 5 (S recompute, dP, dV, dK, dQ).  Compulsory bytes: forward reads
     q, k, v and writes out, out_lt, out_st (+ lse, indices); backward reads q, k, v, dout,
-    out_lt, out_st, lse and writes dq, dk, dv: 15 q-shaped tensors in total.
+    out_lt, out_st, lse and writes dq, dk, dv: 15 q-shaped tensors in total (with grouped
+    key/value heads the k-, v-, dk- and dv-shaped ones are kv_heads / heads as large).
     """
     import numpy as np
     M, Bk = w.n_blocks, w.block
@@ -87,21 +88,22 @@ def work_model(w):
         tiles_S += cnt * ts * w.H
     esz = 2 if w.dtype == "bf16" else 4
     T = w.B * w.H * w.L * w.D * esz
+    Tk = T * (w.kv_heads or w.H) // w.H          # a k- or v-shaped tensor
     tile_flops = 2.0 * Bk * Bk * w.D
     tb = tiles_L + tiles_S
     lse_b = 2 * w.B * w.H * w.L * 4
-    idx_b = w.B * w.H * M * w.topk * 4
+    idx_b = w.B * (w.kv_heads or w.H) * M * w.topk * 4
     gemms = {"fwd": 2, "bwd": 5, "fwd_simt": 2, "fwd_tc": 2, "bwd_dq_simt": 3, "bwd_dkdv_simt": 2,
              "bwd_dq_tc": 3, "bwd_dkdv_tc": 2}
-    byts = {"fwd": 6 * T + lse_b + idx_b, "bwd": 9 * T + 2 * lse_b + idx_b}
+    byts = {"fwd": 4 * T + 2 * Tk + lse_b + idx_b, "bwd": 5 * T + 4 * Tk + 2 * lse_b + idx_b}
     byts.update({"fwd_simt": byts["fwd"], "fwd_tc": byts["fwd"],
-                 "bwd_dq_simt": 7 * T + 2 * lse_b, "bwd_dkdv_simt": 6 * T + 2 * lse_b,
-                 "bwd_dq_tc": 7 * T + 2 * lse_b, "bwd_dkdv_tc": 6 * T + 2 * lse_b,
-                 "summary": T, "score_select": T, "score_fast": T, "bwd_prep": 3 * T + lse_b,
+                 "bwd_dq_simt": 5 * T + 2 * Tk + 2 * lse_b, "bwd_dkdv_simt": 2 * T + 4 * Tk + 2 * lse_b,
+                 "bwd_dq_tc": 5 * T + 2 * Tk + 2 * lse_b, "bwd_dkdv_tc": 2 * T + 4 * Tk + 2 * lse_b,
+                 "summary": Tk, "score_select": T, "score_fast": T, "bwd_prep": 3 * T + lse_b,
                  "tc_meta": idx_b})
     return {"tiles_lt": tiles_L, "tiles_st": tiles_S, "tile_flops": tile_flops,
             "flops": {k: g * tb * tile_flops for k, g in gemms.items()}, "bytes": byts,
-            "step_flops": 7 * tb * tile_flops, "step_bytes": 15 * T + 3 * lse_b + 2 * idx_b}
+            "step_flops": 7 * tb * tile_flops, "step_bytes": 9 * T + 6 * Tk + 3 * lse_b + 2 * idx_b}
 
 
 # ------------------------------------------------------------------------ clock sampling
@@ -167,7 +169,7 @@ def oracle_sample(w, max_batch):
     sl = None if w.seq_lens is None else w.seq_lens[:nb].copy()
     return Workload(w.name + f"[first {nb} of {w.B} batch entries]", w.dtype, nb, w.H, w.L, w.D,
                     w.block, w.topk, w.window, w.seed, w.q[:nb], w.k[:nb], w.v[:nb], w.gate,
-                    w.dout[:nb], sl, w.stis_mode, w.stis_block, w.cmp_block, w.cmp_stride)
+                    w.dout[:nb], sl, w.stis_mode, w.stis_block, w.cmp_block, w.cmp_stride, w.kv_heads)
 
 
 def time_oracle(ws):
@@ -177,6 +179,12 @@ def time_oracle(ws):
     if ws.cmp_block or ws.cmp_stride:   # selection through overlapping compression blocks (Eq. 8-11)
         idx = oracle.select_blocks_cmp(ws.q, ws.k, ws.block, ws.topk, ws.cmp_block or ws.block,
                                        ws.cmp_stride or ws.block, ws.seq_lens)
+    if ws.kv_heads and ws.kv_heads != ws.H:   # grouped key/value heads: one selection per group (Eq. 12)
+        f = oracle.forward_gqa(ws.q, ws.k, ws.v, ws.gate, ws.block, ws.topk, ws.window, ws.seq_lens,
+                               stis_mode=ws.stis_mode, stis_block=ws.stis_block)
+        oracle.backward_gqa(ws.q, ws.k, ws.v, ws.gate, ws.block, ws.topk, ws.window, f, ws.dout,
+                            ws.seq_lens, stis_mode=ws.stis_mode, stis_block=ws.stis_block)
+        return time.perf_counter() - t0
     oracle.forward_backward(ws.q, ws.k, ws.v, ws.gate, ws.dout, ws.block, ws.topk, ws.window,
                             ws.seq_lens, idx=idx, stis_mode=ws.stis_mode, stis_block=ws.stis_block)
     return time.perf_counter() - t0
@@ -240,6 +248,8 @@ def main():
     ap.add_argument("--cmp-block", type=int, default=0,
                     help="length l of overlapping compression blocks for the selection (Eq. 8, 11); 0 = off")
     ap.add_argument("--cmp-stride", type=int, default=0, help="their stride s")
+    ap.add_argument("--kv-heads", type=int, default=0,
+                    help="key/value heads shared by groups of query heads (0: one per query head)")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the batch size (profiling captures on a smaller case; not a bench line)")
     args = ap.parse_args()
@@ -251,15 +261,21 @@ def main():
     from paper_2512_13368_b200 import workloads
     if args.impl == "reference" and rank != 0:
         return 0
-    w = workloads.CONFIGS[args.config](B=args.batch) if (args.batch and args.config != 1) \
-        else workloads.CONFIGS[args.config]()
+    kw = {}
+    if args.batch and args.config != 1:
+        kw["B"] = args.batch
+    if args.kv_heads and args.config != 1:
+        kw["kv_heads"] = args.kv_heads
+    w = workloads.CONFIGS[args.config](**kw)
+    if w.kv_heads:
+        w.name += f"+kv_heads{w.kv_heads}"
     if args.short_term == "power-law":
         w.stis_mode, w.stis_block, w.window = 1, args.mask_block, args.mask_window
         w.name += f"+powerlaw(w{args.mask_window},blk{args.mask_block})"
     if args.cmp_block or args.cmp_stride:
         w.cmp_block, w.cmp_stride = args.cmp_block or w.block, args.cmp_stride or w.block
         w.name += f"+cmp(l{w.cmp_block},s{w.cmp_stride})"
-    cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "seq_len": w.L, "head_dim": w.D,
+    cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "kv_heads": w.kv_heads or w.H, "seq_len": w.L, "head_dim": w.D,
                 "block_size": w.block, "top_k": w.topk, "window": w.window, "short_term": args.short_term,
                 "mask_block": w.stis_block if w.stis_mode else None,
                 "cmp_block": w.cmp_block or None, "cmp_stride": w.cmp_stride or None, "storage": w.dtype,

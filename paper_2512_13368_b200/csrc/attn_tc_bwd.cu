@@ -170,8 +170,10 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
-  const int st = nST - 1 - (int)(blockIdx.x % nST);
-  const int u = blockIdx.x / nST, n = u / s.H, h = u % s.H;
+  // long rows first, tile-major: every unit's last tile, then every unit's last but one, ...
+  const int nU = s.B * s.H;
+  const int st = nST - 1 - (int)(blockIdx.x / nU);
+  const int u = (int)(blockIdx.x % nU), n = u / s.H, h = u % s.H;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -216,7 +218,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     mbar_fence_init();
     // the CTA's tile lists and its resident tiles
     mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
-    bulk_load(smem_u32(meta), qmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
+    bulk_load(smem_u32(meta), qmeta + ((size_t)u * nST + (nST - 1 - st)) * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, 2 * C::kBigBytes);
     tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
     tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
@@ -490,9 +492,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nKT = (s.L + 127) >> 7;
-  const int kt = (int)(blockIdx.x % nKT);  // early keys have the most visitors: first
-  // a CTA owns 128 keys of one (batch, key/value head) and collects from every query head of the group
-  const int uk = blockIdx.x / nKT, n = uk / s.Hkv, hk = uk % s.Hkv;
+  // A CTA owns 128 keys of one (batch, key/value head) and collects from every query head of the
+  // group.  Early keys have the most visitors, so the grid runs tile-major: every unit's first
+  // tile, then every unit's second, ... and the light tiles fill the tail.
+  const int nU = s.B * s.Hkv;
+  const int kt = (int)(blockIdx.x / nU), uk = (int)(blockIdx.x % nU), n = uk / s.Hkv, hk = uk % s.Hkv;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -536,7 +540,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     mbar_fence_init();
     // the CTA's tile lists and its resident tiles
     mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
-    bulk_load(smem_u32(meta), kmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
+    bulk_load(smem_u32(meta), kmeta + ((size_t)uk * nKT + kt) * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, 2 * C::kBigBytes);
     tma_load_4d(smem_u32(k_tile), &tmk, b_res, 0, key0, hk, n);
     tma_load_4d(smem_u32(v_tile), &tmv, b_res, 0, key0, hk, n);
@@ -563,12 +567,14 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     setmaxnreg_dec<kProducerRegs>();
     if (warp == kComputeWarps && nvis > 0) {
       // ---- loader: K, V once; Q, dO tiles and their row records up to STAGES ahead ----
+      int lj = 0, h = hk * s.G;
       for (int j = 0; j < nvis; ++j) {
         const int sj = j % STAGES;
         if (j >= STAGES) mbar_wait(b_empty + 8 * sj, ((j - STAGES) / STAGES) & 1, &abort_flag, 214);
         const uint32_t bar = b_full + 8 * sj;
         const uint32_t qt_ = smem_u32(qg_tiles + sj * kStageBytes);
-        const int row = (int)list[j % nlist] * 64, h = hk * s.G + j / nlist;
+        if (lj == nlist) { lj = 0; ++h; }  // the next query head of the group walks the same list
+        const int row = (int)list[lj++] * 64;
         if (elect_one()) {
           mbar_expect_tx(bar, kStageBytes);
           tma_load_4d(qt_, &tmq, bar, 0, row, h, n);
@@ -631,8 +637,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float sc2 = s.scale * kLog2e;
 
+    int li = 0;
     for (int i = 0; i < nvis; ++i) {
-      const int qt = list[i % nlist], f = lflags[i % nlist], t0 = qt * 64;
+      if (li == nlist) li = 0;
+      const int qt = list[li], f = lflags[li], t0 = qt * 64;
+      ++li;
       uint64_t maskL = 0ull, maskS = 0ull;
       if (row_valid) {
         const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);

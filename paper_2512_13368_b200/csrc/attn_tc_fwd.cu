@@ -126,8 +126,10 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
-  const int st = nST - 1 - (int)(blockIdx.x % nST);  // long rows first
-  const int u = blockIdx.x / nST, n = u / s.H, h = u % s.H;
+  // long rows first, tile-major: every unit's last tile, then every unit's last but one, ...
+  const int nU = s.B * s.H;
+  const int st = nST - 1 - (int)(blockIdx.x / nU);
+  const int u = (int)(blockIdx.x % nU), n = u / s.H, h = u % s.H;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -168,7 +170,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     mbar_fence_init();
     // the CTA's tile lists and its query tile
     mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
-    bulk_load(smem_u32(meta), qmeta + (size_t)blockIdx.x * ml.bytes, (uint32_t)ml.bytes, b_meta);
+    bulk_load(smem_u32(meta), qmeta + ((size_t)u * nST + (nST - 1 - st)) * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, C::kBigBytes);
     tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
   }

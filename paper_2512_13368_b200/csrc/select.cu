@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
 }
 
 // ---- stage 1: single-precision scoring with an error bound ----------------------------------
-// grid M*B*H (unit-major), 256 threads, one query block per CTA.  Logits z[t][j] of the block's
+// grid M*B*Hkv (unit-major), 256 threads, one query block of one head group per CTA.  Logits z[t][j] of the block's
 // (up to 64) queries against 64 candidate means at a time come from a register-blocked fp32
 // product out of shared memory (thread = 4 queries x 4 candidates); softmax per query row by 4
 // lanes; column sums in fixed order; warp 0 runs the top_k - 1 arg-max passes.
@@ -244,8 +244,10 @@ __global__ void __launch_bounds__(kSelThreads) score_select_kernel(
 // total, relative; two scores a > b are in certain order when a - b > R (a + b).
 constexpr int kFastThreads = 256;
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
+// GROUPED: several query heads per key/value head (their number is a run-time value; the
+// one-head kernel keeps its loop-free body and its four CTAs per SM; the grouped one needs more registers).
+template <typename T, int D, bool GROUPED>
+__global__ void __launch_bounds__(kFastThreads, GROUPED ? 2 : 4) score_select_fast_kernel(
     Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
     const float *__restrict__ knorm, const int32_t *__restrict__ klive,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
   int *live = reinterpret_cast<int *>(S + M);  // [M]
   int *taken = live + M;                       // [M]
 
-  const int b = blockIdx.x % M, u = blockIdx.x / M, n = u / s.H, h = u % s.H;
+  const int b = blockIdx.x % M, u = blockIdx.x / M, n = u / s.Hkv, hk = u % s.Hkv;  // u: (batch, key/value head)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
@@ -292,7 +294,12 @@ __global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
   const bool choose = ncand > want && want > 0;  // a real choice: score the candidates
   bool certain = true;
 
-  if (choose) {
+  // The heads of the group take turns (Eq. 12): each adds its column sums to S.
+  const int G = GROUPED ? s.G : 1;
+  if (choose)
+#pragma unroll 1
+  for (int g = 0; g < G; ++g) {
+    const int h = hk * G + g;
     // the query block, fp32, invalid rows zero
     for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {
       const int lt = i / (D / 4), c = (i % (D / 4)) * 4, t = b * s.Bk + lt;
@@ -300,7 +307,7 @@ __global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
       if (lt < s.Bk && t >= qlo && t < qhi) v = ld4(q + row_offset(s, n, h, t) + c);
       *reinterpret_cast<float4 *>(qs + lt * P + c) = v;
     }
-    {
+    if (g == 0) {
       float km = 0.f;
       for (int j = tid; j < b; j += kFastThreads)
         if (live[j]) km = fmaxf(km, knorm[(int64_t)u * M + j]);
@@ -310,7 +317,8 @@ __global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
     if (tid < 64) {
       float a = 0.f;
       for (int c = 0; c < D; ++c) a = fmaf(qs[tid * P + c], qs[tid * P + c], a);
-      rn[tid] = sqrtf(a) * 1.0001f;
+      const float r = sqrtf(a) * 1.0001f;
+      rn[tid] = g == 0 ? r : fmaxf(rn[tid], r);  // the bound below takes the largest query of the group
     }
     const int ty = tid >> 4, tx = tid & 15;          // product: queries ty + 16 a, candidates tx + 16 c
     const int rt = tid >> 2, part = tid & 3;          // softmax: row rt, candidates part, part + 4, ...
@@ -375,7 +383,7 @@ __global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
       if (tid < nb) {
         float a = 0.f;
         for (int t = 0; t < 64; ++t) a += zs[t * ZP + tid];  // fixed order
-        S[j0 + tid] = a;
+        S[j0 + tid] = g == 0 ? a : S[j0 + tid] + a;  // heads in ascending order
       }
     };
     auto row_statistics = [&](int j0) {  // fold the chunk into (mx, den) of row rt
@@ -452,8 +460,10 @@ __global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_kernel(
       const float uu = 5.9604645e-8f;  // 2^-24
       const float bound = s.scale * qn * kn;  // >= every |logit|
       const float E = (float)(D + 4) * uu * bound * 1.01f;
+      // a sum of G non-negative head scores, each within R of its exact value, is within R of the
+      // exact sum, plus one rounding per addition
       const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f +
-                      ((float)b * 0.25f + 80.f + 8.f * (float)((b + 63) / 64)) * uu;
+                      ((float)b * 0.25f + 80.f + 8.f * (float)((b + 63) / 64) + (float)G) * uu;
       const float smin = bound_s[0], umax = bound_s[1];
       certain = (smin - umax) > R * (smin + umax) * 1.001f;
     }
@@ -497,18 +507,16 @@ int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_l
     summary_kernel<T, D><<<grid, 256, 0, st>>>(s, k, seq_lens, ws.kmean, ws.klive, ws.kmean32, ws.knorm,
                                                ws.sel_count);
   }
-  // (the single-precision stage scores one head's queries: groups of several heads go straight
-  // to the double-precision kernel)
-  const bool exact_only = exact_select_only() || s.G > 1;
+  const bool exact_only = exact_select_only();
   if (!exact_only) {
     const size_t fsm = select_fast_smem_bytes(s.M, D);
+    auto fast = s.G > 1 ? score_select_fast_kernel<T, D, true> : score_select_fast_kernel<T, D, false>;
     if (fsm > 48 * 1024 &&
-        cudaFuncSetAttribute(score_select_fast_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)fsm) != cudaSuccess)
+        cudaFuncSetAttribute(fast, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm) != cudaSuccess)
       return BLOSSOM_ERR_CUDA;
     LaunchScope ls(K_SCORE_FAST, st);
-    score_select_fast_kernel<T, D><<<grid, kFastThreads, fsm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive,
-                                                                   seq_lens, idx, ws.sel_list, ws.sel_count);
+    fast<<<grid, kFastThreads, fsm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive, seq_lens, idx, ws.sel_list,
+                                          ws.sel_count);
   }
   bool in_smem = select_smem_bytes(s.M, D, true) <= 160 * 1024;
   size_t smem = select_smem_bytes(s.M, D, in_smem);

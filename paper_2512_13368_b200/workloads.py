@@ -74,15 +74,17 @@ class Workload:
         return self.B * self.L
 
     def unit(self, n: int, h: int) -> "Workload":
-        """The single (batch n, head h) problem as a B=1, H=1 workload."""
+        """The single (batch n, key/value head h) problem as a B=1 workload: one head, or with
+        grouped heads the query heads that share key/value head h."""
         sl = None if self.seq_lens is None else self.seq_lens[n:n + 1].copy()
-        assert not self.kv_heads or self.kv_heads == self.H, "a head of a group is not a problem of its own"
-        return Workload(self.name + f"[{n},{h}]", self.dtype, 1, 1, self.L, self.D, self.block,
+        G = self.H // (self.kv_heads or self.H)
+        hq = slice(h * G, (h + 1) * G)
+        return Workload(self.name + f"[{n},{h}]", self.dtype, 1, G, self.L, self.D, self.block,
                         self.topk, self.window, self.seed,
-                        self.q[n:n + 1, h:h + 1].copy(), self.k[n:n + 1, h:h + 1].copy(),
-                        self.v[n:n + 1, h:h + 1].copy(), self.gate[h:h + 1].copy(),
-                        self.dout[n:n + 1, h:h + 1].copy(), sl, self.stis_mode, self.stis_block,
-                        self.cmp_block, self.cmp_stride)
+                        self.q[n:n + 1, hq].copy(), self.k[n:n + 1, h:h + 1].copy(),
+                        self.v[n:n + 1, h:h + 1].copy(), self.gate[hq].copy(),
+                        self.dout[n:n + 1, hq].copy(), sl, self.stis_mode, self.stis_block,
+                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0)
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,
@@ -107,7 +109,7 @@ def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=No
         seq_lens = rng.integers(lo, hi + 1, size=(B,), dtype=np.int64).astype(np.int32)
     if row_scales:
         for t in (q, k, v):
-            t *= rng.uniform(0.5, 2.0, size=(B, H, L, 1)).astype(np.float32)
+            t *= rng.uniform(0.5, 2.0, size=t.shape[:3] + (1,)).astype(np.float32)
     return Workload(name, dtype, B, H, L, D, block, topk, window, seed,
                     quantize(q, dtype), quantize(k, dtype), quantize(v, dtype),
                     gate, quantize(dout, dtype), seq_lens, stis_mode, stis_block, 0, 0, kv_heads)
@@ -119,27 +121,27 @@ def config1() -> Workload:
     return make("cfg1-tiny-fp32", "fp32", 4, 2, 64, 32, 8, 2, 16, seed=0)
 
 
-def config2(B: int = 256) -> Workload:
+def config2(B: int = 256, kv_heads: int = 0) -> Workload:
     """short-sequence batch: bf16, L200 D32, block 16, top-k 4, window 32, lengths U{5..200}."""
     return make("cfg2-short-padded", "bf16", B, 2, 200, 32, 16, 4, 32, seed=2, std=0.5,
-                lengths=(5, 200))
+                lengths=(5, 200), kv_heads=kv_heads)
 
 
-def config3(B: int = 128) -> Workload:
+def config3(B: int = 128, kv_heads: int = 0) -> Workload:
     """mid-length: bf16, H4 L1024 D64, block 32, top-k 8, window 64, per-row norm scales."""
-    return make("cfg3-mid", "bf16", B, 4, 1024, 64, 32, 8, 64, seed=3, row_scales=True)
+    return make("cfg3-mid", "bf16", B, 4, 1024, 64, 32, 8, 64, seed=3, row_scales=True, kv_heads=kv_heads)
 
 
-def config4(B: int = 16) -> Workload:
+def config4(B: int = 16, kv_heads: int = 0) -> Workload:
     """long-history headline: bf16, H8 L4096 D64, block 64, top-k 16, window 256."""
-    return make("cfg4-long", "bf16", B, 8, 4096, 64, 64, 16, 256, seed=4)
+    return make("cfg4-long", "bf16", B, 8, 4096, 64, 64, 16, 256, seed=4, kv_heads=kv_heads)
 
 
-def config5_attention(B: int = 128) -> Workload:
+def config5_attention(B: int = 128, kv_heads: int = 0) -> Workload:
     """attention-shaped slice of the end-to-end layer case: bf16, H2 L1024 D32, block 32,
     top-k 8, window 64 (the layer case gives no attention hyper-parameters; the mid-length
     case's are reused)."""
-    return make("cfg5-layer-attn", "bf16", B, 2, 1024, 32, 32, 8, 64, seed=1)
+    return make("cfg5-layer-attn", "bf16", B, 2, 1024, 32, 32, 8, 64, seed=1, kv_heads=kv_heads)
 
 
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5_attention}

@@ -240,8 +240,11 @@ def _sampled_units(runner, w, units):
     def one(nh):
         n, h = nh
         wu = w.unit(n, h)
-        ru = {k: (v[n:n + 1, h:h + 1] if k not in ("lse", "dgate") else None) for k, v in res.items()}
-        ru["lse"] = res["lse"][:, n:n + 1, h:h + 1]
+        G = w.H // (w.kv_heads or w.H)
+        hq = slice(h * G, (h + 1) * G)      # the query heads of key/value head h
+        ru = {k: (v[n:n + 1, h:h + 1] if k in ("idx", "dk", "dv") else v[n:n + 1, hq])
+              for k, v in res.items() if k not in ("lse", "dgate")}
+        ru["lse"] = res["lse"][:, n:n + 1, hq]
         ru["dgate"] = None          # summed over the batch: checked separately on small cases
         return check_forward_backward(wu, ru)
 
@@ -259,6 +262,15 @@ def test_config4_full_size_sampled(runner):
     w = workloads.config4()
     errs, _ = _sampled_units(runner, w, [(0, 0), (9, 5), (15, 7)])
     print(errs)
+
+
+def test_config4_full_size_grouped_heads_sampled(runner):
+    """The headline shape with its 8 query heads on 2 key/value heads, as the benchmark's
+    --kv-heads 2 option times it; a sampled unit is a whole group."""
+    w = workloads.config4(kv_heads=2)
+    errs, res = _sampled_units(runner, w, [(0, 0), (11, 1)])
+    print(errs)
+    assert res["idx"].shape == (w.B, 2, w.n_blocks, w.topk) and res["dk"].shape == w.k.shape
 
 
 def test_config4_full_size_overlapping_compression_sampled(runner):
@@ -305,6 +317,8 @@ def test_certified_selection_equals_double_precision_selection(runner, monkeypat
     small_stride = workloads.make("small-stride", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9)
     small_stride.cmp_block, small_stride.cmp_stride = 32, 8    # 253 compression blocks: four chunks
     for w in (workloads.config4(B=1), workloads.config2(B=16), workloads.config3(B=1),
+              workloads.config4(B=1, kv_heads=2), workloads.config2(B=16, kv_heads=1),
+              workloads.config3(B=1, kv_heads=1),
               workloads.make("many-blocks", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9),
               overlap4, overlap2, small_stride):
         p = runner.DeviceProblem(w)
