@@ -253,9 +253,10 @@ __global__ void __launch_bounds__(kFastThreads, GROUPED ? 2 : 4) score_select_fa
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
     int32_t *__restrict__ work_count) {
   constexpr int P = D + 4;   // row pitch of the operand tiles (floats): conflict-free 128-bit reads
-  constexpr int ZP = 65;     // row pitch of the logit tile
+  constexpr int ZP = 68;     // row pitch of the logit tile (4 mod 32: the softmax reads hit 32 banks)
   extern __shared__ float fsm[];
   __shared__ float rn[64];
+  __shared__ float csum[kFastThreads];
   __shared__ float bound_s[2];
   __shared__ int kn_bits;
   const int M = s.M;
@@ -380,9 +381,18 @@ __global__ void __launch_bounds__(kFastThreads, GROUPED ? 2 : 4) score_select_fa
         zs[rt * ZP + j] = on ? __expf(zs[rt * ZP + j] - mx) * inv : 0.f;
       }
       __syncthreads();
-      if (tid < nb) {
+      {  // column sums in a fixed order: four partial sums of 16 rows each, then their tree
+        const int j = tid & 63, quarter = tid >> 6;
         float a = 0.f;
-        for (int t = 0; t < 64; ++t) a += zs[t * ZP + tid];  // fixed order
+        if (j < nb) {
+#pragma unroll
+          for (int t = 0; t < 16; ++t) a += zs[(quarter * 16 + t) * ZP + j];
+        }
+        csum[tid] = a;
+      }
+      __syncthreads();
+      if (tid < nb) {
+        const float a = (csum[tid] + csum[64 + tid]) + (csum[128 + tid] + csum[192 + tid]);
         S[j0 + tid] = g == 0 ? a : S[j0 + tid] + a;  // heads in ascending order
       }
     };
@@ -486,7 +496,7 @@ __global__ void __launch_bounds__(kFastThreads, GROUPED ? 2 : 4) score_select_fa
 }
 
 size_t select_fast_smem_bytes(int M, int D) {
-  const int P = D + 4, ZP = 65;
+  const int P = D + 4, ZP = 68;
   return (size_t)(64 * P + 64 * (P > ZP ? P : ZP)) * sizeof(float) + (size_t)M * (sizeof(float) + 2 * sizeof(int));
 }
 

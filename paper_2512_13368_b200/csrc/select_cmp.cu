@@ -224,9 +224,10 @@ __global__ void __launch_bounds__(256, 4) cmp_score_select_fast_kernel(
     Shape s, const T *__restrict__ q, const float *__restrict__ cmean32, const float *__restrict__ cnorm,
     const int32_t *__restrict__ clive, const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx,
     int32_t *__restrict__ worklist, int32_t *__restrict__ work_count) {
-  constexpr int P = D + 4, ZP = 65, NT = 256;
+  constexpr int P = D + 4, ZP = 68, NT = 256;
   extern __shared__ float fsm[];
   __shared__ float rn[64];
+  __shared__ float csum[256];
   __shared__ float bound_s[2];
   __shared__ int kn_bits;
   const int M = s.M, Mc = max(s.Mc, 1);
@@ -357,11 +358,17 @@ __global__ void __launch_bounds__(256, 4) cmp_score_select_fast_kernel(
             zs[rt * ZP + j] = on ? __expf(zs[rt * ZP + j] - mx) * inv : 0.f;
           }
           __syncthreads();
-          if (tid < nb) {
+          {  // column sums in a fixed order: four partial sums of 16 rows each, then their tree
+            const int j = tid & 63, quarter = tid >> 6;
             float a = 0.f;
-            for (int t = 0; t < 64; ++t) a += zs[t * ZP + tid];  // fixed order
-            Sc[j0 + tid] = a;
+            if (j < nb) {
+#pragma unroll
+              for (int t = 0; t < 16; ++t) a += zs[(quarter * 16 + t) * ZP + j];
+            }
+            csum[tid] = a;
           }
+          __syncthreads();
+          if (tid < nb) Sc[j0 + tid] = (csum[tid] + csum[64 + tid]) + (csum[128 + tid] + csum[192 + tid]);
         }
       }
     }
@@ -429,7 +436,7 @@ __global__ void __launch_bounds__(256, 4) cmp_score_select_fast_kernel(
 }
 
 size_t cmp_fast_smem_bytes(const Shape &s, int D) {
-  const int P = D + 4, ZP = 65;
+  const int P = D + 4, ZP = 68;
   const size_t Mc = s.Mc > 0 ? s.Mc : 1;
   return (size_t)(64 * P + 64 * (P > ZP ? P : ZP)) * sizeof(float) + (Mc + s.M) * (sizeof(float) + sizeof(int));
 }
