@@ -80,6 +80,9 @@ def test_argument_validation_precedes_any_launch(lib):
     assert E.blossom_attn_fwd(good(select_mode=1), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
     assert E.blossom_attn_fwd(good(kv_heads=3), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
     assert E.blossom_select_blocks(good(head_dim=128), A, A, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
+    # one block more than the 1024 the lists are laid out for
+    big = good(seq_len=1024 * 16 + 1, block_size=16)
+    assert E.blossom_select_blocks(big, A, A, None, A, A, 1 << 40, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
     assert E.blossom_select_blocks(p, A, None, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
     # backward: every tensor is required
     args = [A] * 14          # q k v gate seq_lens idx out_lt out_st lse dout dq dk dv dgate

@@ -95,6 +95,18 @@ def test_edge_shapes(runner, dtype, L, D, block, topk, window, lens):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("D,topk,window,lens", [(32, 8, 128, None), (64, 4, 64, [65536 - 4097])])
+def test_maximum_number_of_blocks(runner, D, topk, window, lens):
+    """ceil(L / block) = 1024, the most the interface takes: 1024 entries on every tile list, 512
+    CTAs per unit, query blocks with more than a thousand candidates in the selection."""
+    w = workloads.make("max-blocks", "bf16", 1, 2, 65536, D, 64, topk, window, seed=23)
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    print(check_forward_backward(w, res))
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("L,D,block,topk,window,blk,lens", [
     (64, 32, 8, 2, 8, 1, None),              # the paper's defaults: window 8, mask block 1
