@@ -77,3 +77,75 @@ class DeviceProblem:
         return {"idx": self.idx.cpu().numpy(), "out": f(self.out), "out_lt": f(self.out_lt),
                 "out_st": f(self.out_st), "lse": f(self.lse), "dq": f(self.dq), "dk": f(self.dk),
                 "dv": f(self.dv), "dgate": f(self.dgate)}
+
+
+class HostPipeline:
+    """Steps whose inputs and results live in pinned host memory.
+
+    `slots` device problems take turns: while one computes, the next one's inputs are uploaded
+    and the previous one's results are downloaded, on three streams ordered by events (PCIe
+    carries both directions at once).  Every byte of every step crosses the bus; only the
+    waiting is taken out.  The host buffers of a submitted step must stay untouched until
+    `drain()` (or until `slots` further steps have been submitted).
+    """
+
+    IN = ("q", "k", "v", "dout", "gate")
+    OUT = ("out", "dq", "dk", "dv", "dgate")
+
+    def __init__(self, w: Workload, slots: int = 2, device="cuda:0", sm_scale=0.0):
+        self.device = torch.device(device)
+        self.slots = [DeviceProblem(w, device, sm_scale) for _ in range(slots)]
+        mk = lambda: [torch.cuda.Event() for _ in range(slots)]  # noqa: E731
+        self.uploaded, self.computed, self.downloaded = mk(), mk(), mk()
+        self.s_up, self.s_run, self.s_down = (torch.cuda.Stream(self.device) for _ in range(3))
+        self.n = 0
+
+    def pinned_inputs(self) -> dict:
+        p = self.slots[0]
+        d = {k: getattr(p, k).detach().cpu().pin_memory() for k in self.IN}
+        if p.seq_lens is not None:
+            d["seq_lens"] = p.seq_lens.cpu().pin_memory()
+        return d
+
+    def pinned_outputs(self) -> dict:
+        p = self.slots[0]
+        return {k: torch.empty(getattr(p, k).shape, dtype=getattr(p, k).dtype).pin_memory() for k in self.OUT}
+
+    def submit(self, h_in: dict, h_out: dict):
+        i = self.n % len(self.slots)
+        p = self.slots[i]
+        used = self.n >= len(self.slots)
+        with torch.cuda.stream(self.s_up):
+            if used:
+                self.s_up.wait_event(self.computed[i])      # the slot's last step has read its inputs
+            for k, h in h_in.items():
+                getattr(p, k).copy_(h, non_blocking=True)
+            self.uploaded[i].record(self.s_up)
+        with torch.cuda.stream(self.s_run):
+            self.s_run.wait_event(self.uploaded[i])
+            if used:
+                self.s_run.wait_event(self.downloaded[i])   # and its results have left the device
+            p.step()
+            self.computed[i].record(self.s_run)
+        with torch.cuda.stream(self.s_down):
+            self.s_down.wait_event(self.computed[i])
+            for k, h in h_out.items():
+                h.copy_(getattr(p, k), non_blocking=True)
+            self.downloaded[i].record(self.s_down)
+        self.n += 1
+
+    def fence(self, stream=None):
+        """Makes `stream` (default: the current one) wait for everything submitted so far, and the
+        pipeline's streams wait for what `stream` has done."""
+        cur = stream or torch.cuda.current_stream(self.device)
+        e = torch.cuda.Event()
+        e.record(cur)
+        for s in (self.s_up, self.s_run, self.s_down):
+            s.wait_event(e)
+            d = torch.cuda.Event()
+            d.record(s)
+            cur.wait_event(d)
+
+    def drain(self):
+        for s in (self.s_up, self.s_run, self.s_down):
+            s.synchronize()

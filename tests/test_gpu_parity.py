@@ -205,6 +205,25 @@ def test_inference_mode_and_select_only(runner):
     assert np.array_equal(q.results()["idx"], res["idx"])
 
 
+def test_host_pipeline_returns_the_device_resident_results(runner):
+    """Steps streamed from and to pinned host memory over alternating device slots give, step
+    after step, the bits of a device-resident step."""
+    import torch
+    w = workloads.make("pipe", "bf16", 3, 2, 700, 64, 32, 5, 70, seed=31, lengths=(100, 700))
+    p, res = run(runner, w)
+    pipe = runner.HostPipeline(w, slots=2)
+    h_in = pipe.pinned_inputs()
+    outs = [pipe.pinned_outputs() for _ in range(5)]
+    for o in outs:
+        for t in o.values():
+            t.fill_(7.0)
+        pipe.submit(h_in, o)
+    pipe.drain()
+    for o in outs:
+        for k in ("out", "dq", "dk", "dv", "dgate"):
+            assert np.array_equal(o[k].float().numpy(), res[k]), k
+
+
 def test_strided_layout(runner):
     """q-shaped tensors stored [B, L, H, D] (the layout a fused QKV projection produces)."""
     import torch
