@@ -27,10 +27,13 @@
 //         meanwhile.  d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
 //  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
 //         records, by bulk copy) that selected one of its key blocks or whose window reaches them.
-//         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D): no room for
-//         the bf16 operands, so W^T = P'_lt + P'_st and dS^T go through two 128-byte-swizzled
-//         shared-memory tiles.  S^T = K Q^T, dP^T = V dO^T; thread = key row;
-//         dV += W^T dO, dK += dS^T Q.  As in dQ, tile i+1's first stage overlaps tile i's arithmetic.
+//         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D).
+//         S^T = K Q^T, dP^T = V dO^T; thread = key row and 32 of the 64 query columns; it writes
+//         W^T = P'_lt + P'_st and dS^T (bf16 pairs) over the first 16 of its own S^T / dP^T
+//         columns, from where dV += W^T dO and dK += dS^T Q read their first operand: nothing of
+//         a tile's arithmetic goes through shared memory, whose data pipe (operand reads of the
+//         products, row records) is the busiest unit of this kernel.  With one buffer the first
+//         stage of tile i+1 follows the products of tile i; the SM's other CTA fills the gap.
 // Every wait is bounded (tc_common.cuh).
 #include "tc_common.cuh"
 
@@ -43,7 +46,7 @@ constexpr int kKvThreads = 384;
 constexpr int kProducerRegs = 32, kKvComputeRegs = 104;  // 256 * 104 + 128 * 32 = 384 * 80
 constexpr int kComputeWarps = 8;
 constexpr int kDqStages = 4;
-constexpr int kKvStages = 2;
+constexpr int kKvStages = 3;
 constexpr uint32_t kBwdTmemCols = 256;
 constexpr int kStatBytes = 64 * 16;  // one 64-query tile of row records
 
@@ -485,8 +488,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   constexpr int OC = D / 2;
   constexpr int kStageBytes = 2 * C::kSmallBytes + kStatBytes;  // Q, dO, row records
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done, s_empty, meta
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 6];
+  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done, meta
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -508,18 +511,17 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   uint8_t *k_tile = tiles;
   uint8_t *v_tile = k_tile + C::kBigBytes;
   uint8_t *qg_tiles = v_tile + C::kBigBytes;  // [stage][Q, dO, row records]
-  uint8_t *w_tile = qg_tiles + STAGES * kStageBytes;  // W^T  [128 keys][64 queries] bf16, 128-byte swizzle
-  uint8_t *ds_tile = w_tile + 128 * 128;               // dS^T, same layout
-  uint8_t *meta = ds_tile + 128 * 128;                  // image built by tc_meta_kernel
+  uint8_t *meta = qg_tiles + STAGES * kStageBytes;  // image built by tc_meta_kernel
   const MetaLayout ml = meta_layout(nT);
   const uint8_t *invb = meta;                           // [8][nT] bytes: per key block, per query tile
   const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
   const uint8_t *lflags = meta + ml.flags;
+  const uint8_t *kcls = meta + ml.jcls;                 // [listed tile][compute warp]
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
   const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 2]), b_done = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_sempty = smem_u32(&bars[2 * STAGES + 4]), b_meta = smem_u32(&bars[2 * STAGES + 5]);
+  const uint32_t b_meta = smem_u32(&bars[2 * STAGES + 4]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -535,7 +537,6 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     mbar_init(b_sfull, 1);
     mbar_init(b_tfull, kComputeWarps);
     mbar_init(b_done, 1);
-    mbar_init(b_sempty, kComputeWarps);
     mbar_init(b_meta, 1);
     mbar_fence_init();
     // the CTA's tile lists and its resident tiles
@@ -584,55 +585,61 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
         __syncwarp();
       }
     } else if (warp == kComputeWarps + 1 && nvis > 0) {
-      // ---- S^T = K Q^T and dP^T = V dO^T of tile i once the compute warps hold tile i-1's ----
+      // ---- one issuer: S^T = K Q^T, dP^T = V dO^T of tile i; then, once the compute warps have
+      // written W^T and dS^T over those logits, dV += W^T dO and dK += dS^T Q with the first
+      // operand read from tensor memory; tile i + 1's logits may replace them when these products
+      // have completed ----
       constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
+      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
       const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
       const uint64_t dvd = smem_desc(smem_u32(v_tile), 16, C::kAtomBytes, C::kSwizzle);
       mbar_wait(b_res, 0, &abort_flag, 210);
-      for (int i = 0; i < nvis; ++i) {
-        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 213);
-        if (i >= 1) mbar_wait(b_sempty, (i - 1) & 1, &abort_flag, 212);
-        tc_fence_after();
-        uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
-        const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
-        const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
-        if (elect_one()) {
+      for (int i = 0; i <= nvis; ++i) {
+        if (i >= 1) {  // second stage of tile i - 1
+          const int j = i - 1;
+          uint8_t *q_tile = qg_tiles + (j % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
+          const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+          const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+          mbar_wait(b_tfull, j & 1, &abort_flag, 211);
+          tc_fence_after();
+          if (elect_one()) {
+            // 16 queries per step: bf16 pairs in 8 columns; the compute warps of column half h keep
+            // theirs in the first 16 of their own 32 logit columns
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
+            for (int k = 0; k < 4; ++k)
+              umma_bf16_ts(tmem_dv, tmem_s + (k >> 1) * 32 + (k & 1) * 8, dgm + k * C::kKStep, idesc_o,
+                           (j | k) != 0);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
-          umma_commit(b_sfull);
+            for (int k = 0; k < 4; ++k)
+              umma_bf16_ts(tmem_dk, tmem_dp + (k >> 1) * 32 + (k & 1) * 8, dqm + k * C::kKStep, idesc_o,
+                           (j | k) != 0);
+            umma_commit(b_done);
+            umma_commit(b_empty + 8 * (j % STAGES));
+          }
+          __syncwarp();
         }
-        __syncwarp();
-      }
-    } else if (warp == kComputeWarps + 2 && nvis > 0) {
-      // ---- dV += W^T dO, dK += dS^T Q of tile i (W^T, dS^T from shared memory, K-major) ----
-      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
-      const uint64_t dwd = smem_desc(smem_u32(w_tile), 16, 1024, 2u);
-      const uint64_t dsd = smem_desc(smem_u32(ds_tile), 16, 1024, 2u);
-      for (int i = 0; i < nvis; ++i) {
-        uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
-        const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-        const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 215);
-        mbar_wait(b_tfull, i & 1, &abort_flag, 211);
-        tc_fence_after();
-        if (elect_one()) {
+        if (i < nvis) {  // first stage of tile i
+          mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 213);
+          if (i >= 1) mbar_wait(b_done, (i - 1) & 1, &abort_flag, 212);  // W^T(i-1), dS^T(i-1) have been read
+          tc_fence_after();
+          uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
+          const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
+          const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_bf16(tmem_dv, dwd + 2 * k, dgm + k * C::kKStep, idesc_o, (i | k) != 0);
+            for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_bf16(tmem_dk, dsd + 2 * k, dqm + k * C::kKStep, idesc_o, (i | k) != 0);
-          umma_commit(b_done);
-          umma_commit(b_empty + 8 * (i % STAGES));  // S^T(i), dP^T(i) completed before the compute warps read them
+            for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
+            umma_commit(b_sfull);
+          }
+          __syncwarp();
         }
-        __syncwarp();
       }
     }
   } else {
     setmaxnreg_inc<kKvComputeRegs>();
     const int quarter = warp & 3, half = warp >> 2;
     const int r = quarter * 32 + lane, p = key0 + r, g = r / s.Bk;
-    bool w_zero = false;  // this thread's part of the W^T / dS^T tiles holds zeros
     const bool row_ok = p < s.L, row_valid = row_ok && p >= pad0;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const float sc2 = s.scale * kLog2e;
@@ -642,15 +649,23 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       if (li == nlist) li = 0;
       const int qt = list[li], f = lflags[li], t0 = qt * 64;
       ++li;
-      uint64_t maskL = 0ull, maskS = 0ull;
-      if (row_valid) {
-        const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
-        if (f & 1) maskL = mc & expand_block_bits(invb[g * nT + qt], s.Bk);
-        if (f & 2) maskS = mc & st_query_cols(s, p, t0);
+      // the warp's class for this tile comes prebuilt; only a mixed tile needs the per-lane masks
+      const int cls = kcls[(li - 1) * kComputeWarps + warp];
+      uint32_t hL = 0u, hS = 0u;
+      bool anyL = (cls & 1) != 0, anyS = (cls & 2) != 0, full = true;
+      if (cls == 8) {
+        uint64_t maskL = 0ull, maskS = 0ull;
+        if (row_valid) {
+          const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
+          if (f & 1) maskL = mc & expand_block_bits(invb[g * nT + qt], s.Bk);
+          if (f & 2) maskS = mc & st_query_cols(s, p, t0);
+        }
+        hL = (uint32_t)(maskL >> (half * 32));
+        hS = (uint32_t)(maskS >> (half * 32));
+        anyL = __any_sync(0xffffffffu, hL != 0u);
+        anyS = __any_sync(0xffffffffu, hS != 0u);
+        full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffffffu) && (!anyS || hS == 0xffffffffu));
       }
-      const uint32_t hL = (uint32_t)(maskL >> (half * 32)), hS = (uint32_t)(maskS >> (half * 32));
-      const bool anyL = __any_sync(0xffffffffu, hL != 0u), anyS = __any_sync(0xffffffffu, hS != 0u);
-      const bool full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffffffu) && (!anyS || hS == 0xffffffffu));
 
       mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 216);  // the row records have landed
       mbar_wait(b_sfull, i & 1, &abort_flag, 217);
@@ -659,50 +674,32 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       const bool mine = anyL || anyS;
       const float4 *stt =
           reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes) + half * 32;
-      if (mine || !w_zero) {
-        // two passes of 16 query columns (a rolled loop: one copy of each code path)
+      // two passes of 16 query columns (a rolled loop: one copy of each code path); W^T and dS^T
+      // of a pass go, as bf16 pairs, over the first 16 of this thread's own 32 logit columns:
+      // pass 0 over columns it has just read, pass 1 behind them
 #pragma unroll 1
-        for (int q = 0; q < 2; ++q) {
-          uint32_t ww[8], dw[8];
+      for (int q = 0; q < 2; ++q) {
+        uint32_t ww[8], dw[8];
+        if (mine) {
           float sv[16], dp[16];
-          if (mine) {
-            tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
-            tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
-            tmem_wait_ld();
-          }
-          if (q == 1) warp_arrive(b_sempty, lane);  // S^T, dP^T of this tile are in registers
-          if (mine) {
-            const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
-            const float4 *sq = stt + q * 16;  // 8 pairs x 2 float4
-            if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
-            else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-            else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-            else dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          } else {
+          tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
+          tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
+          tmem_wait_ld();
+          const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
+          const float4 *sq = stt + q * 16;  // 8 pairs x 2 float4
+          if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          else dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+        } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }
-          }
-          if (q == 0 && i >= 1) {  // the W^T / dS^T tiles are free once the products of tile i-1 completed
-            mbar_wait(b_done, (i - 1) & 1, &abort_flag, 219);
-            __syncwarp();
-          }
-#pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
-            store_row_sw128(w_tile, r, half * 4 + q * 2 + ch,
-                            make_uint4(ww[ch * 4], ww[ch * 4 + 1], ww[ch * 4 + 2], ww[ch * 4 + 3]));
-            store_row_sw128(ds_tile, r, half * 4 + q * 2 + ch,
-                            make_uint4(dw[ch * 4], dw[ch * 4 + 1], dw[ch * 4 + 2], dw[ch * 4 + 3]));
-          }
+          for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }
         }
-        w_zero = !mine;
-      } else {
-        warp_arrive(b_sempty, lane);
-        if (i >= 1) {  // keep in step with the barrier (a parity wait tells only two phases apart)
-          mbar_wait(b_done, (i - 1) & 1, &abort_flag, 220);
-          __syncwarp();
-        }
+        tmem_st8u(tmem_s + lane_off + half * 32 + q * 8, ww);
+        tmem_st8u(tmem_dp + lane_off + half * 32 + q * 8, dw);
       }
-      fence_async_smem();
+      tmem_wait_st();
+      tc_fence_before();
       warp_arrive(b_tfull, lane);
     }
 
@@ -767,7 +764,7 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
   const size_t smem_dq = 1024 + 2 * C::kBigBytes + kDqStages * 2 * C::kSmallBytes + meta_bytes(nT);
   const size_t smem_kv =
-      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + 2 * 128 * 128 + meta_bytes(nT);
+      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT);
   if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
