@@ -27,13 +27,14 @@
 //         meanwhile.  d alpha = sum (P_lt - P_st) dP from the fp32 probabilities.
 //  dK/dV  transposed: resident K, V of 128 keys, streams Q, dO 64-query tiles (and their row
 //         records, by bulk copy) that selected one of its key blocks or whose window reaches them.
-//         Tensor memory: S^T [0,64), dP^T [64,128), dV [128,128+D), dK [192,192+D).
-//         S^T = K Q^T, dP^T = V dO^T; thread = key row and 32 of the 64 query columns; it writes
-//         W^T = P'_lt + P'_st and dS^T (bf16 pairs) over the first 16 of its own S^T / dP^T
-//         columns, from where dV += W^T dO and dK += dS^T Q read their first operand: nothing of
-//         a tile's arithmetic goes through shared memory, whose data pipe (operand reads of the
-//         products, row records) is the busiest unit of this kernel.  With one buffer the first
-//         stage of tile i+1 follows the products of tile i; the SM's other CTA fills the gap.
+//         It works through them in half tiles of 32 queries.  Tensor memory: two buffers of 64
+//         columns (half tile x uses buffer x % 2: S^T in its first 32 columns, dP^T in the other
+//         32), dV [128,128+D), dK [192,192+D).  S^T = K Q^T, dP^T = V dO^T; thread = key row and
+//         16 of the 32 query columns; it writes W^T = P'_lt + P'_st and dS^T (bf16 pairs) over the
+//         first 8 of its own S^T / dP^T columns, from where dV += W^T dO and dK += dS^T Q read
+//         their first operand: nothing of a tile's arithmetic goes through shared memory, whose
+//         data pipe (operand reads of the products, row records) is the busiest unit of this
+//         kernel, and the first stage of the next half tile runs during the arithmetic of this one.
 // Every wait is bounded (tc_common.cuh).
 #include "tc_common.cuh"
 
@@ -488,8 +489,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   constexpr int OC = D / 2;
   constexpr int kStageBytes = 2 * C::kSmallBytes + kStatBytes;  // Q, dO, row records
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, s_full, t_full, mma_done, meta
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];
+  // barriers: full[STAGES], empty[STAGES], res, meta, and per buffer s_full[2], t_full[2], done[2]
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 8];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -519,9 +520,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   const uint8_t *kcls = meta + ml.jcls;                 // [listed tile][compute warp]
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
-  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_sfull = smem_u32(&bars[2 * STAGES + 1]);
-  const uint32_t b_tfull = smem_u32(&bars[2 * STAGES + 2]), b_done = smem_u32(&bars[2 * STAGES + 3]);
-  const uint32_t b_meta = smem_u32(&bars[2 * STAGES + 4]);
+  const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_meta = smem_u32(&bars[2 * STAGES + 1]);
+  const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 4]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 6]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -534,9 +535,11 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       mbar_init(b_empty + 8 * i, 1);
     }
     mbar_init(b_res, 1);
-    mbar_init(b_sfull, 1);
-    mbar_init(b_tfull, kComputeWarps);
-    mbar_init(b_done, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(b_sfull + 8 * i, 1);
+      mbar_init(b_tfull + 8 * i, kComputeWarps);
+      mbar_init(b_done + 8 * i, 1);
+    }
     mbar_init(b_meta, 1);
     mbar_fence_init();
     // the CTA's tile lists and its resident tiles
@@ -560,8 +563,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   const int nlist = *reinterpret_cast<const int *>(meta + ml.counts);
   const int nvis = nlist * s.G;
   const uint32_t tmem_base = tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_dp = tmem_base + 64, tmem_dv = tmem_base + 128,
-                 tmem_dk = tmem_base + 192;
+  // half tile x uses buffer x % 2 at column 64 (x % 2): S^T in its first 32 columns, dP^T behind
+  const uint32_t tmem_dv = tmem_base + 128, tmem_dk = tmem_base + 192;
 
   if (warp >= kComputeWarps) {
     // ===================== three single-thread roles, one warp each =====================
@@ -585,52 +588,56 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
         __syncwarp();
       }
     } else if (warp == kComputeWarps + 1 && nvis > 0) {
-      // ---- one issuer: S^T = K Q^T, dP^T = V dO^T of tile i; then, once the compute warps have
-      // written W^T and dS^T over those logits, dV += W^T dO and dK += dS^T Q with the first
-      // operand read from tensor memory; tile i + 1's logits may replace them when these products
-      // have completed ----
-      constexpr uint32_t idesc_s = instr_desc(128, 64, 0, 0);
-      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
+      // ---- S^T = K Q^T, dP^T = V dO^T of half tile x into buffer x % 2 once the products of half
+      // tile x - 2 have read that buffer ----
+      constexpr uint32_t idesc_s = instr_desc(128, 32, 0, 0);
       const uint64_t dkd = smem_desc(smem_u32(k_tile), 16, C::kAtomBytes, C::kSwizzle);
       const uint64_t dvd = smem_desc(smem_u32(v_tile), 16, C::kAtomBytes, C::kSwizzle);
       mbar_wait(b_res, 0, &abort_flag, 210);
-      for (int i = 0; i <= nvis; ++i) {
-        if (i >= 1) {  // second stage of tile i - 1
-          const int j = i - 1;
-          uint8_t *q_tile = qg_tiles + (j % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
-          const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-          const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
-          mbar_wait(b_tfull, j & 1, &abort_flag, 211);
+      for (int i = 0, x = 0; i < nvis; ++i) {
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 213);
+        for (int hh = 0; hh < 2; ++hh, ++x) {
+          const int b = x & 1, ph = (x >> 1) & 1;
+          if (x >= 2) mbar_wait(b_done + 8 * b, ph ^ 1, &abort_flag, 212);
           tc_fence_after();
+          const uint32_t qt_ = smem_u32(qg_tiles + (i % STAGES) * kStageBytes) + hh * 32 * C::kRowBytes;
+          const uint64_t dqd = smem_desc(qt_, 16, C::kAtomBytes, C::kSwizzle);
+          const uint64_t dgd = smem_desc(qt_ + C::kSmallBytes, 16, C::kAtomBytes, C::kSwizzle);
+          const uint32_t ts = tmem_base + 64 * b;
           if (elect_one()) {
-            // 16 queries per step: bf16 pairs in 8 columns; the compute warps of column half h keep
-            // theirs in the first 16 of their own 32 logit columns
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16_ts(tmem_dv, tmem_s + (k >> 1) * 32 + (k & 1) * 8, dgm + k * C::kKStep, idesc_o,
-                           (j | k) != 0);
+            for (int k = 0; k < D / 16; ++k) umma_bf16(ts, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16_ts(tmem_dk, tmem_dp + (k >> 1) * 32 + (k & 1) * 8, dqm + k * C::kKStep, idesc_o,
-                           (j | k) != 0);
-            umma_commit(b_done);
-            umma_commit(b_empty + 8 * (j % STAGES));
+            for (int k = 0; k < D / 16; ++k) umma_bf16(ts + 32, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
+            umma_commit(b_sfull + 8 * b);
           }
           __syncwarp();
         }
-        if (i < nvis) {  // first stage of tile i
-          mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 213);
-          if (i >= 1) mbar_wait(b_done, (i - 1) & 1, &abort_flag, 212);  // W^T(i-1), dS^T(i-1) have been read
+      }
+    } else if (warp == kComputeWarps + 2 && nvis > 0) {
+      // ---- dV += W^T dO, dK += dS^T Q of a half tile; W^T and dS^T are read from tensor memory,
+      // where the compute warps wrote them over the half tile's logits ----
+      constexpr uint32_t idesc_o = instr_desc(128, D, 0, 1);
+      for (int i = 0, x = 0; i < nvis; ++i) {
+        uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
+        const uint64_t dgm = smem_desc(smem_u32(g_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        const uint64_t dqm = smem_desc(smem_u32(q_tile), C::kSmallBytes, C::kAtomBytes, C::kSwizzle);
+        mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 215);
+        for (int hh = 0; hh < 2; ++hh, ++x) {
+          const int b = x & 1, ph = (x >> 1) & 1;
+          mbar_wait(b_tfull + 8 * b, ph, &abort_flag, 211);
           tc_fence_after();
-          uint8_t *q_tile = qg_tiles + (i % STAGES) * kStageBytes, *g_tile = q_tile + C::kSmallBytes;
-          const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
-          const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
+          const uint32_t tb = tmem_base + 64 * b;
           if (elect_one()) {
+            // 16 queries per step: the bf16 pairs of the warps of column half kk, 8 columns
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_s, dkd + 2 * k, dqd + 2 * k, idesc_s, k > 0);
+            for (int kk = 0; kk < 2; ++kk)
+              umma_bf16_ts(tmem_dv, tb + 16 * kk, dgm + (2 * hh + kk) * C::kKStep, idesc_o, (x | kk) != 0);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) umma_bf16(tmem_dp, dvd + 2 * k, dgd + 2 * k, idesc_s, k > 0);
-            umma_commit(b_sfull);
+            for (int kk = 0; kk < 2; ++kk)
+              umma_bf16_ts(tmem_dk, tb + 32 + 16 * kk, dqm + (2 * hh + kk) * C::kKStep, idesc_o, (x | kk) != 0);
+            umma_commit(b_done + 8 * b);
+            if (hh == 1) umma_commit(b_empty + 8 * (i % STAGES));  // every product on this stage has completed
           }
           __syncwarp();
         }
@@ -645,66 +652,65 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const float sc2 = s.scale * kLog2e;
 
     int li = 0;
-    for (int i = 0; i < nvis; ++i) {
+    for (int i = 0, x = 0; i < nvis; ++i) {
       if (li == nlist) li = 0;
       const int qt = list[li], f = lflags[li], t0 = qt * 64;
+      const uint8_t *cls2 = kcls + li * 16 + warp;  // classes of the tile's two half tiles for this warp
       ++li;
-      // the warp's class for this tile comes prebuilt; only a mixed tile needs the per-lane masks
-      const int cls = kcls[(li - 1) * kComputeWarps + warp];
-      uint32_t hL = 0u, hS = 0u;
-      bool anyL = (cls & 1) != 0, anyS = (cls & 2) != 0, full = true;
-      if (cls == 8) {
-        uint64_t maskL = 0ull, maskS = 0ull;
+      uint64_t maskL = 0ull, maskS = 0ull;
+      if (cls2[0] == 8 || cls2[8] == 8) {  // a mixed half tile: per-lane column masks
         if (row_valid) {
           const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
           if (f & 1) maskL = mc & expand_block_bits(invb[g * nT + qt], s.Bk);
           if (f & 2) maskS = mc & st_query_cols(s, p, t0);
         }
-        hL = (uint32_t)(maskL >> (half * 32));
-        hS = (uint32_t)(maskS >> (half * 32));
-        anyL = __any_sync(0xffffffffu, hL != 0u);
-        anyS = __any_sync(0xffffffffu, hS != 0u);
-        full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffffffu) && (!anyS || hS == 0xffffffffu));
       }
-
       mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 216);  // the row records have landed
-      mbar_wait(b_sfull, i & 1, &abort_flag, 217);
-      __syncwarp();
-      tc_fence_after();
-      const bool mine = anyL || anyS;
-      const float4 *stt =
-          reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes) + half * 32;
-      // two passes of 16 query columns (a rolled loop: one copy of each code path); W^T and dS^T
-      // of a pass go, as bf16 pairs, over the first 16 of this thread's own 32 logit columns:
-      // pass 0 over columns it has just read, pass 1 behind them
+      const float4 *stt = reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes);
+      // A half tile = 32 queries; this thread's 16 columns of it are queries 32 hh + 16 half ...
+      // W^T and dS^T go, as bf16 pairs, over the first 8 of the thread's own 16 columns of S^T / dP^T.
 #pragma unroll 1
-      for (int q = 0; q < 2; ++q) {
+      for (int hh = 0; hh < 2; ++hh, ++x) {
+        const int b = x & 1, ph = (x >> 1) & 1, c0 = 32 * hh + 16 * half;
+        const int cls = cls2[8 * hh];
+        uint32_t hL = 0u, hS = 0u;
+        bool anyL = (cls & 1) != 0, anyS = (cls & 2) != 0, full = true;
+        if (cls == 8) {
+          hL = (uint32_t)(maskL >> c0) & 0xffffu;
+          hS = (uint32_t)(maskS >> c0) & 0xffffu;
+          anyL = __any_sync(0xffffffffu, hL != 0u);
+          anyS = __any_sync(0xffffffffu, hS != 0u);
+          full = __all_sync(0xffffffffu, (!anyL || hL == 0xffffu) && (!anyS || hS == 0xffffu));
+        }
+        const uint32_t tb = tmem_base + 64 * b + lane_off + 16 * half;
+        mbar_wait(b_sfull + 8 * b, ph, &abort_flag, 217);
+        __syncwarp();
+        tc_fence_after();
         uint32_t ww[8], dw[8];
-        if (mine) {
+        if (anyL || anyS) {
           float sv[16], dp[16];
-          tmem_ld16(tmem_s + lane_off + half * 32 + q * 16, sv);
-          tmem_ld16(tmem_dp + lane_off + half * 32 + q * 16, dp);
+          tmem_ld16(tb, sv);
+          tmem_ld16(tb + 32, dp);
           tmem_wait_ld();
-          const uint32_t qL = hL >> (q * 16), qS = hS >> (q * 16);
-          const float4 *sq = stt + q * 16;  // 8 pairs x 2 float4
-          if (!full) dkdv_tile<true, true, false>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          else if (anyL) dkdv_tile<true, false, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
-          else dkdv_tile<false, true, true>(sv, dp, qL, qS, sc2, sq, ww, dw);
+          const float4 *sq = stt + c0;  // 8 pairs x 2 float4
+          if (!full) dkdv_tile<true, true, false>(sv, dp, hL, hS, sc2, sq, ww, dw);
+          else if (anyL && anyS) dkdv_tile<true, true, true>(sv, dp, hL, hS, sc2, sq, ww, dw);
+          else if (anyL) dkdv_tile<true, false, true>(sv, dp, hL, hS, sc2, sq, ww, dw);
+          else dkdv_tile<false, true, true>(sv, dp, hL, hS, sc2, sq, ww, dw);
         } else {
 #pragma unroll
           for (int c = 0; c < 8; ++c) { ww[c] = 0u; dw[c] = 0u; }
         }
-        tmem_st8u(tmem_s + lane_off + half * 32 + q * 8, ww);
-        tmem_st8u(tmem_dp + lane_off + half * 32 + q * 8, dw);
+        tmem_st8u(tb, ww);
+        tmem_st8u(tb + 32, dw);
+        tmem_wait_st();
+        tc_fence_before();
+        warp_arrive(b_tfull + 8 * b, lane);
       }
-      tmem_wait_st();
-      tc_fence_before();
-      warp_arrive(b_tfull, lane);
     }
 
     if (nvis > 0) {
-      mbar_wait(b_done, (nvis - 1) & 1, &abort_flag, 218);
+      mbar_wait(b_done + 8, (nvis - 1) & 1, &abort_flag, 218);  // the last half tile used buffer 1
       __syncwarp();
       tc_fence_after();
     }

@@ -18,8 +18,8 @@
 //   counts                    {tiles on the list, long-term items, short-term items}
 // Key-major image (dK/dV kernel): [8][nT] bytes: bit c of byte (g, qt): query block
 // qt * (64 / Bk) + c selected key block g of the CTA; list / flags of the 64-query tiles that
-// visit the CTA's keys; jcls[nT][8] class of every (listed tile, compute warp); counts {tiles on
-// the list}.
+// visit the CTA's keys; jcls[nT][2][8] class of every (listed tile, half tile, compute warp);
+// counts {tiles on the list}.
 #include "tc_common.cuh"
 
 namespace blossom {
@@ -306,14 +306,14 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     }
     if (lane == 0) counts[0] = count;
     __syncwarp();
-    // dK/dV kernel: class of every (listed tile, compute warp).  Warp w works on key rows
-    // 32 (w % 4) ... of the CTA and on query columns 32 (w / 4) ... of the tile.  Same code as for
-    // the dQ kernel: bit 0 / bit 1 = every key row of the warp is seen in full by all 32 queries
-    // through the long-term / short-term branch and none in part; 8 = mixed.
-    for (int e = lane; e < count * 8; e += 32) {
-      const int it = e >> 3, w = e & 7, qtr = w & 3, hf = w >> 2;
-      const int qt = list[it], f = lflags[it];
-      const int p_lo = key0 + 32 * qtr, p_hi = p_lo + 31, t_lo = qt * 64 + 32 * hf, t_hi = t_lo + 31;
+    // dK/dV kernel: class of every (listed tile, half tile of 32 queries, compute warp).  Warp w
+    // works on key rows 32 (w % 4) ... of the CTA and on query columns 16 (w / 4) ... of the half
+    // tile.  Same code as for the dQ kernel: bit 0 / bit 1 = every key row of the warp is seen in
+    // full by all 16 queries through the long-term / short-term branch and none in part; 8 = mixed.
+    for (int e = lane; e < count * 16; e += 32) {
+      const int it = e >> 4, hh = (e >> 3) & 1, w = e & 7, qtr = w & 3, hf = w >> 2;
+      const int qt = list[it], f = lflags[it], c_lo = 32 * hh + 16 * hf;
+      const int p_lo = key0 + 32 * qtr, p_hi = p_lo + 31, t_lo = qt * 64 + c_lo, t_hi = t_lo + 15;
       const bool rows_in = p_lo >= pad0 && p_hi < s.L, rows_none = p_hi < pad0 || p_lo >= s.L;
       const bool past = rows_in && t_hi < s.L && t_lo >= p_hi;  // every query causally sees every key
       const bool reach = !rows_none && t_hi >= p_lo && t_lo < s.L;  // some query may see some key
@@ -322,7 +322,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         bool any_sel = false, all_sel = true;
         for (int gk = (qtr * 32) >> bk_shift; gk <= (qtr * 32 + 31) >> bk_shift; ++gk) {
           const uint32_t bits = selb[gk * nT + qt];
-          for (int c = (32 * hf) >> bk_shift; c <= (32 * hf + 31) >> bk_shift; ++c) {
+          for (int c = c_lo >> bk_shift; c <= (c_lo + 15) >> bk_shift; ++c) {
             const bool sel = (bits >> c) & 1u;
             any_sel |= sel;
             all_sel &= sel;
