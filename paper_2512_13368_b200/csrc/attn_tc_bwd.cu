@@ -47,7 +47,7 @@ constexpr int kKvThreads = 384;
 constexpr int kProducerRegs = 32, kKvComputeRegs = 104;  // 256 * 104 + 128 * 32 = 384 * 80
 constexpr int kComputeWarps = 8;
 constexpr int kDqStages = 4;
-constexpr int kKvStages = 3;
+constexpr int kKvStages = 4;
 constexpr uint32_t kBwdTmemCols = 256;
 constexpr int kStatBytes = 64 * 16;  // one 64-query tile of row records
 
@@ -669,7 +669,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       const float4 *stt = reinterpret_cast<const float4 *>(qg_tiles + (i % STAGES) * kStageBytes + 2 * C::kSmallBytes);
       // A half tile = 32 queries; this thread's 16 columns of it are queries 32 hh + 16 half ...
       // W^T and dS^T go, as bf16 pairs, over the first 8 of the thread's own 16 columns of S^T / dP^T.
-#pragma unroll 1
+#pragma unroll
       for (int hh = 0; hh < 2; ++hh, ++x) {
         const int b = x & 1, ph = (x >> 1) & 1, c0 = 32 * hh + 16 * half;
         const int cls = cls2[8 * hh];
