@@ -106,6 +106,14 @@ def work_model(w):
             "step_flops": 7 * tb * tile_flops, "step_bytes": 9 * T + 6 * Tk + 3 * lse_b + 2 * idx_b}
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernels from
+# the ncu capture summarised in profiles/cfg4_attention_and_selection_kernels.md.  It was taken at
+# batch 4 of the long-history case (255 MB of tensors, more than L2); traffic grows in proportion
+# to the batch, so a launch at batch B is charged B / 4 times these figures.  Other workloads and
+# kernels report null.
+NCU_TRAFFIC_CFG4_B4 = {"fwd_tc": 54.09e6 + 13.22e6, "bwd_dq_tc": 71.91e6 + 0.90e6, "bwd_dkdv_tc": 71.99e6 + 3.07e6}
+
+
 # ------------------------------------------------------------------------ clock sampling
 class ClockSampler:
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -377,7 +385,9 @@ def main():
     else:
         ach = by / (avg_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak}
-    roof.update({"traffic": None, "kernel": top, "kernel_ms": avg_ms,
+    plain_cfg4 = args.config == 4 and not (w.stis_mode or w.cmp_block or w.cmp_stride or w.kv_heads)
+    traffic = NCU_TRAFFIC_CFG4_B4.get(top) if plain_cfg4 else None
+    roof.update({"traffic": traffic * w.B / 4 if traffic else None, "kernel": top, "kernel_ms": avg_ms,
                  "kernel_share": agg[top][1] / tot_kernel_ms,
                  "peak_source": f"of {peak_kind} (MEASURED_PEAKS.json, sustained bf16 / copy bandwidth)"
                  if peak_kind == "measured" else "of fallback",
