@@ -224,6 +224,31 @@ def test_host_pipeline_returns_the_device_resident_results(runner):
             assert np.array_equal(o[k].float().numpy(), res[k]), k
 
 
+def test_step_replays_from_a_cuda_graph(runner):
+    """Selection, forward and backward launch on the caller's stream and allocate nothing, so a
+    step can be captured once and replayed; the replays give the bits of the eager step."""
+    import torch
+    w = workloads.make("graph", "bf16", 2, 2, 600, 64, 32, 4, 96, seed=37, lengths=(200, 600))
+    p, res = run(runner, w)
+    for name in ("out", "dq", "dk", "dv", "dgate", "idx"):
+        getattr(p, name).zero_()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        p.step()                      # warm-up on the capture stream (attributes, tensor maps)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            p.step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        for name in ("out", "dq", "dk", "dv", "dgate"):
+            getattr(p, name).zero_()
+        graph.replay()
+        got = p.results()
+        for k in ("idx", "out", "out_lt", "out_st", "lse", "dq", "dk", "dv", "dgate"):
+            assert np.array_equal(got[k], res[k]), k
+
+
 def test_strided_layout(runner):
     """q-shaped tensors stored [B, L, H, D] (the layout a fused QKV projection produces)."""
     import torch
