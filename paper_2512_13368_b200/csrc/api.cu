@@ -12,20 +12,35 @@ unsigned long long g_launches = 0;
 // ---- optional per-launch event profile (process-wide, off by default) ---------------------
 static cudaEvent_t *g_prof_events = nullptr;  // [2 * cap]: before / after each launch
 static int *g_prof_ids = nullptr;
+static int *g_prof_start = nullptr;           // index of the event a record's time starts at
 static int g_prof_cap = 0, g_prof_n = 0;
+static cudaStream_t g_prof_chain_stream = nullptr;
+static bool g_prof_chain = false;  // the last thing put on g_prof_chain_stream was a record's end event
 
 void prof_mark(int id, int phase, cudaStream_t st) {
   if (!g_prof_events) return;
   if (phase == 0) {
     if (g_prof_n >= g_prof_cap) return;
     g_prof_ids[g_prof_n] = id;
-    cudaEventRecord(g_prof_events[2 * g_prof_n], st);
+    // back-to-back launches of one call share an event: the end of one is the start of the next
+    if (g_prof_chain && g_prof_chain_stream == st && g_prof_n > 0) {
+      g_prof_start[g_prof_n] = 2 * (g_prof_n - 1) + 1;
+    } else {
+      g_prof_start[g_prof_n] = 2 * g_prof_n;
+      cudaEventRecord(g_prof_events[2 * g_prof_n], st);
+    }
   } else {
     if (g_prof_n >= g_prof_cap) return;
     cudaEventRecord(g_prof_events[2 * g_prof_n + 1], st);
+    g_prof_chain = true;
+    g_prof_chain_stream = st;
     ++g_prof_n;
   }
 }
+
+// Called on entry of every launching API call: whatever the caller put on the stream since the
+// last call must not be charged to this call's first kernel.
+void prof_break() { g_prof_chain = false; }
 
 bool force_simt() {
   const char *e = getenv("BLOSSOM_FORCE_SIMT");
@@ -152,6 +167,7 @@ size_t blossom_workspace_bytes(const blossom_params *params) {
 int blossom_select_blocks(const blossom_params *params, const void *q, const void *k,
                           const int32_t *seq_lens, int32_t *block_idx, void *workspace,
                           size_t workspace_bytes, blossom_stream_t stream) {
+  prof_break();
   Shape s;
   int rc = make_shape(params, &s);
   if (rc) return rc;
@@ -167,6 +183,7 @@ int blossom_select_blocks(const blossom_params *params, const void *q, const voi
 int blossom_select_blocks_static(const blossom_params *params, const void *q, const void *k,
                                  const int32_t *seq_lens, int32_t *block_idx,
                                  blossom_stream_t stream) {
+  prof_break();
   Shape s;
   int rc = make_shape(params, &s);
   if (rc) return rc;
@@ -180,6 +197,7 @@ int blossom_attn_fwd(const blossom_params *params, const void *q, const void *k,
                      const float *gate_logits, const int32_t *seq_lens, int32_t *block_idx,
                      int32_t idx_is_input, void *out, void *out_lt, void *out_st, float *lse,
                      void *workspace, size_t workspace_bytes, blossom_stream_t stream) {
+  prof_break();
   Shape s;
   int rc = make_shape(params, &s);
   if (rc) return rc;
@@ -210,6 +228,7 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
                      const void *out_lt, const void *out_st, const float *lse, const void *dout,
                      void *dq, void *dk, void *dv, float *dgate, void *workspace,
                      size_t workspace_bytes, blossom_stream_t stream) {
+  prof_break();
   Shape s;
   int rc = make_shape(params, &s);
   if (rc) return rc;
@@ -267,6 +286,8 @@ int blossom_profile_start(int max_launches) {
       return BLOSSOM_ERR_CUDA;
     }
   g_prof_ids = new int[max_launches];
+  g_prof_start = new int[max_launches];
+  g_prof_chain = false;
   g_prof_cap = max_launches;
   g_prof_n = 0;
   g_prof_events = ev;
@@ -280,14 +301,16 @@ int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
   int n = g_prof_n < capacity ? g_prof_n : capacity, bad = 0;
   for (int i = 0; i < n; ++i) {
     if (cudaEventSynchronize(ev[2 * i + 1]) != cudaSuccess ||
-        cudaEventElapsedTime(&ms[i], ev[2 * i], ev[2 * i + 1]) != cudaSuccess)
+        cudaEventElapsedTime(&ms[i], ev[g_prof_start[i]], ev[2 * i + 1]) != cudaSuccess)
       bad = 1;
     kernel_ids[i] = g_prof_ids[i];
   }
   for (int i = 0; i < 2 * g_prof_cap; ++i) cudaEventDestroy(ev[i]);
   delete[] ev;
   delete[] g_prof_ids;
+  delete[] g_prof_start;
   g_prof_ids = nullptr;
+  g_prof_start = nullptr;
   g_prof_cap = g_prof_n = 0;
   return bad ? -1 : n;
 }
