@@ -107,7 +107,7 @@ def work_model(w):
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernels from
-# the ncu capture summarised in profiles/cfg4_attention_and_selection_kernels.md.  It was taken at
+# an ncu capture (the summaries under profiles/ give the command).  It was taken at
 # batch 4 of the long-history case (255 MB of tensors, more than L2); traffic grows in proportion
 # to the batch, so a launch at batch B is charged B / 4 times these figures.  Other workloads and
 # kernels report null.
