@@ -495,6 +495,245 @@ __global__ void __launch_bounds__(kFastThreads, GROUPED ? 2 : 4) score_select_fa
   }
 }
 
+// ---- stage 1 for short sequences with small blocks ------------------------------------------
+// With blocks of 16 or 32 positions a CTA of the kernel above fills a quarter or half of its 64
+// query rows, and with few blocks per sequence its run time is all fixed cost (three rounds of
+// global loads, a dozen block-wide barriers).  This kernel takes NBLK = 64 / Bk consecutive query
+// blocks per CTA: the 64 rows are 64 consecutive positions, every row is scored against the
+// candidates of the CTA's last block in one chunk (M <= 64) and keeps those before its own block;
+// the column sums of a block are the sums of its 16-row quarters.  Same arithmetic per score and
+// the same error bound as above (with the largest query norm of the block and the largest
+// candidate norm of the CTA, both upper bounds).
+template <typename T, int D, int NBLK>
+__global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_packed_kernel(
+    Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
+    const float *__restrict__ knorm, const int32_t *__restrict__ klive,
+    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
+    int32_t *__restrict__ work_count) {
+  constexpr int P = D + 4, ZP = 68, BK = 64 / NBLK, QPB = 4 / NBLK;  // quarters (16 rows) per block
+  extern __shared__ float fsm[];
+  __shared__ float rn[64];
+  __shared__ float csum[kFastThreads];
+  __shared__ float S[NBLK][64];
+  __shared__ float bound_s[NBLK][2];
+  __shared__ int live[64], taken[NBLK][64];
+  __shared__ int kn_bits;
+  const int M = s.M, MC = (M + NBLK - 1) / NBLK;
+  float *qs = fsm;          // [64][P]  the CTA's 64 query positions
+  float *ks = qs + 64 * P;  // [64][P]  the candidate means; reused as zs [64][ZP]
+  float *zs = ks;
+
+  const int c = blockIdx.x % MC, u = blockIdx.x / MC, n = u / s.H, h = u % s.H;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int len = seq_lens ? seq_lens[n] : s.L;
+  len = min(max(len, 0), s.L);
+  const int pad0 = s.L - len;
+  const int b0 = c * NBLK;                      // first query block of the CTA
+  const int nbk = min(NBLK, M - b0);            // its query blocks
+  const int bmax = b0 + nbk - 1;                // candidates of the last one: blocks 0 .. bmax - 1
+  if (tid == 0) kn_bits = 0;
+  if (tid < 64) live[tid] = (tid < bmax && klive[(int64_t)u * M + tid] > 0) ? 1 : 0;
+  __syncthreads();
+  // per block: valid, number of live candidates, how many to keep, whether that is a real choice
+  int want[NBLK];
+  bool valid[NBLK], choose[NBLK], any_choose = false;
+#pragma unroll
+  for (int i = 0; i < NBLK; ++i) {
+    const int b = b0 + i;
+    valid[i] = i < nbk && max(b * BK, pad0) < min((b + 1) * BK, s.L);
+    int nc = 0;
+    for (int j = 0; j < b && i < nbk; ++j) nc += live[j];
+    want[i] = min(s.topk - 1, nc);
+    choose[i] = valid[i] && nc > want[i] && want[i] > 0;
+    any_choose |= choose[i];
+  }
+
+  if (any_choose) {
+    for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {  // the 64 positions, fp32, invalid rows zero
+      const int lt = i / (D / 4), cc = (i % (D / 4)) * 4, t = b0 * BK + lt;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (t >= pad0 && t < s.L) v = ld4(q + row_offset(s, n, h, t) + cc);
+      *reinterpret_cast<float4 *>(qs + lt * P + cc) = v;
+    }
+    for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {  // the candidate means
+      const int lj = i / (D / 4), cc = (i % (D / 4)) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (lj < bmax && live[lj])
+        v = *reinterpret_cast<const float4 *>(kmean32 + ((int64_t)u * M + lj) * D + cc);
+      *reinterpret_cast<float4 *>(ks + lj * P + cc) = v;
+    }
+    if (tid < bmax && live[tid]) {
+      const float km = knorm[(int64_t)u * M + tid];
+      if (km > 0.f) atomicMax(&kn_bits, __float_as_int(km));  // positive floats order like ints
+    }
+    __syncthreads();
+    if (tid < 64) {
+      float a = 0.f;
+      for (int cc = 0; cc < D; ++cc) a = fmaf(qs[tid * P + cc], qs[tid * P + cc], a);
+      rn[tid] = sqrtf(a) * 1.0001f;
+    }
+    const int ty = tid >> 4, tx = tid & 15;  // product: rows ty + 16 a, candidates tx + 16 e
+    const int ne = (bmax + 15) >> 4;         // groups of 16 candidates that hold any
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[a][e] = 0.f;
+#pragma unroll 4
+    for (int cc = 0; cc < D; cc += 4) {
+      float4 qa[4], kb[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + cc);
+        if (a < ne) kb[a] = *reinterpret_cast<const float4 *>(ks + (tx + 16 * a) * P + cc);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e < ne) {
+#pragma unroll
+          for (int a = 0; a < 4; ++a) {
+            acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
+            acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
+            acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
+            acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
+          }
+        }
+    }
+    __syncthreads();  // everyone has read ks: it becomes zs
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) zs[(ty + 16 * a) * ZP + tx + 16 * e] = s.scale * acc[a][e];
+    __syncthreads();
+    {  // softmax of row rt over the live candidates before its own block, by 4 lanes, in registers
+      const int rt = tid >> 2, part = tid & 3, t = b0 * BK + rt, brow = b0 + rt / BK;
+      const bool row_valid = t >= pad0 && t < s.L;
+      float z[16], e[16];
+      unsigned lm = 0u;
+      float cm = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int j = part + 4 * k;
+        const bool v = j < brow && live[j];
+        lm |= (v ? 1u : 0u) << k;
+        z[k] = v ? zs[rt * ZP + j] : -INFINITY;
+        cm = fmaxf(cm, z[k]);
+      }
+      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+      float sum = 0.f;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        e[k] = 0.f;
+        if (cm > -INFINITY && ((lm >> k) & 1u)) {
+          e[k] = __expf(z[k] - cm);
+          sum += e[k];
+        }
+      }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      const float inv = sum > 0.f ? 1.f / sum : 0.f;
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        zs[rt * ZP + part + 4 * k] = (row_valid && ((lm >> k) & 1u)) ? e[k] * inv : 0.f;
+    }
+    __syncthreads();
+    {  // column sums of every 16-row quarter in a fixed order, then the blocks' sums of quarters
+      const int j = tid & 63, quarter = tid >> 6;
+      float a = 0.f;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) a += zs[(quarter * 16 + t) * ZP + j];
+      csum[tid] = a;
+    }
+    __syncthreads();
+    for (int e = tid; e < NBLK * 64; e += kFastThreads) {
+      const int i = e >> 6, j = e & 63;
+      float a = csum[(i * QPB) * 64 + j];
+#pragma unroll
+      for (int qq = 1; qq < QPB; ++qq) a += csum[(i * QPB + qq) * 64 + j];
+      S[i][j] = a;
+    }
+    __syncthreads();
+  }
+
+  // Selection by rank within each block, 4 lanes per (block, candidate)
+  for (int e0 = 0; e0 < NBLK * 64; e0 += kFastThreads / 4) {
+    const int e = e0 + (tid >> 2), part = tid & 3, i = e >> 6, j = e & 63, b = b0 + i;
+    int rank = 0;
+    const bool cand = i < nbk && j < b && live[j];
+    bool ch = false;
+    int wt = 0;
+#pragma unroll
+    for (int ii = 0; ii < NBLK; ++ii)
+      if (ii == i) { ch = choose[ii]; wt = want[ii]; }
+    if (cand && ch) {
+      const float sj = S[i][j];
+      for (int x = part; x < b; x += 4)
+        if (live[x]) {
+          const float sx = S[i][x];
+          rank += (sx > sj || (sx == sj && x < j)) ? 1 : 0;
+        }
+    }
+    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+    rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+    if (part == 0 && i < nbk) {
+      if (ch) {
+        if (cand) {
+          taken[i][j] = rank < wt;
+          if (rank == wt - 1) bound_s[i][0] = S[i][j];  // the smallest kept score
+          if (rank == wt) bound_s[i][1] = S[i][j];      // the largest dropped score
+        } else {
+          taken[i][j] = 0;
+        }
+      } else {
+        taken[i][j] = (wt > 0 && cand) ? 1 : 0;
+      }
+    }
+  }
+  __syncthreads();
+
+  if (warp < nbk) {  // warp i finishes block b0 + i
+    const int i = warp, b = b0 + i;
+    bool ch = false, vd = false;
+#pragma unroll
+    for (int ii = 0; ii < NBLK; ++ii)
+      if (ii == i) { ch = choose[ii]; vd = valid[ii]; }
+    int32_t *row = idx + ((int64_t)u * M + b) * s.topk;
+    if (!vd) {  // the query block holds only padding
+      for (int x = lane; x < s.topk; x += 32) row[x] = -1;
+      return;
+    }
+    bool certain = true;
+    if (ch) {
+      float qn = 0.f;
+      for (int x = lane; x < BK; x += 32) qn = fmaxf(qn, rn[i * BK + x]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, o));
+      const float kn = __int_as_float(kn_bits);
+      const float uu = 5.9604645e-8f;  // 2^-24
+      const float bound = s.scale * qn * kn;  // >= every |logit|
+      const float E = (float)(D + 4) * uu * bound * 1.01f;
+      const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f + ((float)b * 0.25f + 80.f + 8.f + 1.f) * uu;
+      const float smin = bound_s[i][0], umax = bound_s[i][1];
+      certain = (smin - umax) > R * (smin + umax) * 1.001f;
+    }
+    if (certain) {
+      int pos = 0;
+      for (int base = 0; base < b; base += 32) {
+        const int j = base + lane;
+        const bool f = j < b && taken[i][j];
+        const unsigned mm = __ballot_sync(0xffffffffu, f);
+        if (f) row[pos + __popc(mm & ((1u << lane) - 1u))] = j;
+        pos += __popc(mm);
+      }
+      if (lane == 0) row[pos] = b;
+      for (int x = pos + 1 + lane; x < s.topk; x += 32) row[x] = -1;
+    } else if (lane == 0) {
+      worklist[atomicAdd(work_count, 1)] = u * M + b;  // re-scored in double precision
+    }
+  }
+}
+
 size_t select_fast_smem_bytes(int M, int D) {
   const int P = D + 4, ZP = 68;
   return (size_t)(64 * P + 64 * (P > ZP ? P : ZP)) * sizeof(float) + (size_t)M * (sizeof(float) + 2 * sizeof(int));
@@ -519,6 +758,16 @@ int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_l
   }
   const bool exact_only = exact_select_only();
   if (!exact_only) {
+    if (s.G == 1 && s.M <= 64 && (s.Bk == 16 || s.Bk == 32)) {
+      // short sequences of small blocks: 64 / Bk query blocks per CTA
+      const int nblk = 64 / s.Bk;
+      const size_t psm = (size_t)(64 * (D + 4) + 64 * 68) * sizeof(float);
+      auto packed = nblk == 2 ? score_select_fast_packed_kernel<T, D, 2> : score_select_fast_packed_kernel<T, D, 4>;
+      const unsigned gpk = (unsigned)((s.M + nblk - 1) / nblk) * (unsigned)(s.B * s.Hkv);
+      LaunchScope ls(K_SCORE_FAST, st);
+      packed<<<gpk, kFastThreads, psm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive, seq_lens, idx, ws.sel_list,
+                                             ws.sel_count);
+    } else {
     const size_t fsm = select_fast_smem_bytes(s.M, D);
     auto fast = s.G > 1 ? score_select_fast_kernel<T, D, true> : score_select_fast_kernel<T, D, false>;
     if (fsm > 48 * 1024 &&
@@ -527,6 +776,7 @@ int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_l
     LaunchScope ls(K_SCORE_FAST, st);
     fast<<<grid, kFastThreads, fsm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive, seq_lens, idx, ws.sel_list,
                                           ws.sel_count);
+    }
   }
   bool in_smem = select_smem_bytes(s.M, D, true) <= 160 * 1024;
   size_t smem = select_smem_bytes(s.M, D, in_smem);
