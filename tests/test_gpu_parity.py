@@ -390,3 +390,35 @@ def test_certified_selection_equals_double_precision_selection(runner, monkeypat
         monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
         assert np.array_equal(fast, exact), w.name
         check_indices(w, fast)
+
+
+def test_certified_selection_on_random_small_block_shapes(runner, monkeypatch):
+    """Short sequences of 16- and 32-position blocks take the first-stage kernel that packs
+    several query blocks into a CTA: over random shapes, lengths, scales and exact ties (identical
+    keys) its choice must be the double-precision one, bit for bit."""
+    import torch
+    rng = np.random.default_rng(123)
+    for it in range(48):
+        Bk = int(rng.choice([16, 32]))
+        M = int(rng.integers(1, 65))
+        L = int(rng.integers((M - 1) * Bk + 1, M * Bk + 1))
+        D = int(rng.choice([32, 64]))
+        H, B = int(rng.choice([1, 2, 3])), int(rng.integers(1, 5))
+        topk, dtype = int(rng.integers(1, 12)), str(rng.choice(["bf16", "fp32"]))
+        std = float(rng.choice([0.05, 0.5, 1.0, 3.0]))
+        lens = None if rng.random() < 0.4 else (1, L)
+        w = workloads.make("rand-small", dtype, B, H, L, D, Bk, topk, 16, seed=1000 + it, std=std, lengths=lens)
+        if it % 7 == 0:
+            w.k[:] = w.k[:, :, :1, :]      # every key equal: every score ties
+        p = runner.DeviceProblem(w)
+        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
+        p.select()
+        torch.cuda.synchronize()
+        fast = p.idx.cpu().numpy().copy()
+        monkeypatch.setenv("BLOSSOM_EXACT_SELECT", "1")
+        p.idx.fill_(-7)
+        p.select()
+        torch.cuda.synchronize()
+        exact = p.idx.cpu().numpy()
+        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
+        assert np.array_equal(fast, exact), (it, L, Bk, D, H, B, topk, dtype, std)
