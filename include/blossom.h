@@ -7,8 +7,10 @@
  *
  * General conventions (all entry points)
  *   - Every pointer is DEVICE memory unless a comment says "host".  The caller owns every
- *     buffer; except where an entry point says otherwise the library allocates nothing, keeps
- *     no state between calls, launches only on the given stream and never synchronises.
+ *     buffer; except where an entry point says otherwise the library allocates nothing,
+ *     launches only on the given stream and never synchronises.  State kept between calls: none
+ *     that a result depends on; process-wide there are a launch counter, the optional event
+ *     profile below, and the two debugging switches (blossom_debug_switch).
  *   - q-shaped tensors (q, k, v, out, out_lt, out_st, dout, dq, dk, dv) are [B][H][L][D] with
  *     element strides (stride_b, stride_h, stride_l, 1) shared by all of them; the element type
  *     is params.dtype.  Base pointers must be 16-byte aligned and the three strides multiples
@@ -124,7 +126,9 @@ int blossom_select_blocks(const blossom_params *params /* host */, const void *q
  *     from load to exit, whether or not this function is ever called.
  *   - Capacity: batch * heads * M <= 8192 and batch * heads * M * head_dim <= 524288
  *     (M = ceil(seq_len / block_size)); larger problems return BLOSSOM_ERR_TOO_LARGE before
- *     anything is launched.  All other argument rules are those of blossom_select_blocks.
+ *     anything is launched.  Overlapping compression blocks (cmp_block / cmp_stride other than
+ *     block_size) are not taken: BLOSSOM_ERR_UNSUPPORTED.  All other argument rules are those of
+ *     blossom_select_blocks (grouped heads included: the capacity then counts kv_heads).
  *   - The first call on each device looks up the array's device address (a runtime query, done
  *     once per device with that device current).  Make that first call outside any stream
  *     capture; later calls only launch kernels on `stream`.
@@ -181,10 +185,21 @@ int blossom_attn_bwd(const blossom_params *params /* host */, const void *q, con
                      float *dgate, void *workspace, size_t workspace_bytes,
                      blossom_stream_t stream);
 
-/* Synchronises the stream and copies the workspace's device status word to *host_out (host):
- * 0 = no device-side error since the workspace was last used, else a blossom_status.  Returns
- * BLOSSOM_ERR_CUDA if the synchronise or the copy fails. */
+/* Synchronises the stream and copies the workspace's device status to *host_out (host): 0 = no
+ * device-side error, else a blossom_status.  The workspace holds one status word for the forward
+ * (blossom_select_blocks and blossom_attn_fwd clear it when they start) and one for the backward
+ * (blossom_attn_bwd clears only that one), so a read after a forward + backward pair on one
+ * workspace reports a wait that ran out in either; the forward's word wins if both are set.
+ * Returns BLOSSOM_ERR_CUDA if the synchronise or the copy fails. */
 int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out);
+
+/* Debugging switches (no counterpart in the paper), process-wide, host only, not thread-safe.
+ * which = 0: route every call to the fp32 CUDA-core kernels instead of the tensor-core ones;
+ * which = 1: score every query block in double precision (skip the certified fp32 stage).
+ * value 1 = on, 0 = off, -1 = back to the default, which is the environment variable
+ * BLOSSOM_FORCE_SIMT resp. BLOSSOM_EXACT_SELECT as it stood when the library was loaded
+ * (unset or "0" = off).  Returns BLOSSOM_ERR_INVALID_ARG for other arguments. */
+int blossom_debug_switch(int which, int value);
 
 /* Human-readable name of a blossom_status (host string, static storage). */
 const char *blossom_status_string(int status);

@@ -14,20 +14,71 @@ from . import binding
 _DT = {torch.float32: "fp32", torch.bfloat16: "bf16"}
 
 
+def _dense(t) -> bool:
+    """True if the tensor's elements tile its storage span without gaps or overlap, so that a
+    buffer of ``numel`` elements laid out with the same strides holds every element."""
+    span = 1 + sum((n - 1) * st for n, st in zip(t.shape, t.stride()) if n > 0)
+    return t.numel() > 0 and span == t.numel() and all(st > 0 for st in t.stride())
+
+
+def _like(t):
+    """An uninitialised tensor with exactly t's shape AND strides (``empty_like`` does not keep the
+    strides of a non-dense view; the library writes every q-shaped buffer with the strides passed
+    in the params)."""
+    return torch.empty_strided(t.shape, t.stride(), dtype=t.dtype, device=t.device)
+
+
+def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True):
+    """Host-side validation before anything is launched: the library receives raw addresses, so a
+    host tensor, a tensor on another device, a wrong integer width or a wrong shape would become a
+    device memory fault instead of a Python error.  Returns seq_lens as the int32 CUDA tensor the
+    library reads (or None).  ``require_cuda=False`` (host-side tests only) skips the test that
+    the tensors are CUDA tensors and keeps every other check, the same-device one included."""
+    if q.dtype not in _DT or k.dtype != q.dtype or v.dtype != q.dtype:
+        raise TypeError("q, k, v must share one dtype, float32 or bfloat16")
+    if not ((q.is_cuda or not require_cuda) and q.dim() == 4 and k.dim() == 4 and k.shape == v.shape):
+        raise ValueError("q [B, H, L, D] and k, v [B, Hkv, L, D] must be CUDA tensors")
+    if k.device != q.device or v.device != q.device:
+        raise ValueError("q, k, v must live on one device")
+    B, H, L, D = q.shape
+    if k.shape[0] != B or k.shape[2] != L or k.shape[3] != D or k.shape[1] < 1 or H % k.shape[1]:
+        raise ValueError("k, v must be [B, Hkv, L, D] with Hkv dividing the number of query heads")
+    if not isinstance(gate_logits, torch.Tensor) or tuple(gate_logits.shape) != (H, 2):
+        raise ValueError("gate_logits must be a tensor of shape [H, 2]")
+    if (require_cuda and not gate_logits.is_cuda) or gate_logits.device != q.device:
+        raise ValueError("gate_logits must be a CUDA tensor on q's device")
+    if not gate_logits.dtype.is_floating_point:
+        raise TypeError("gate_logits must be a floating-point tensor")
+    if seq_lens is not None:
+        if not isinstance(seq_lens, torch.Tensor) or tuple(seq_lens.shape) != (B,):
+            raise ValueError("seq_lens must be None or a tensor of shape [B]")
+        if seq_lens.dtype not in (torch.int32, torch.int64):
+            raise TypeError("seq_lens must be int32 (int64 is converted)")
+        if (require_cuda and not seq_lens.is_cuda) or seq_lens.device != q.device:
+            raise ValueError("seq_lens must be a CUDA tensor on q's device")
+        seq_lens = seq_lens.to(torch.int32).contiguous()
+    return seq_lens
+
+
 class _BlossomAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
                 stis_mode, stis_block, cmp_block, cmp_stride):
-        if q.dtype not in _DT or k.dtype != q.dtype or v.dtype != q.dtype:
-            raise TypeError("q, k, v must share one dtype, float32 or bfloat16")
-        if not (q.is_cuda and q.shape == k.shape == v.shape and q.dim() == 4):
-            raise ValueError("q, k, v: CUDA tensors of one shape [B, H, L, D]")
-        if not (q.stride() == k.stride() == v.stride() and q.stride(3) == 1):
-            q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
+        seq_lens = check_arguments(q, k, v, gate_logits, seq_lens)
         B, H, L, D = q.shape
+        Hkv = k.shape[1]
+        # The library addresses every q-shaped buffer with q's strides and every k-shaped one with
+        # k's: views that are not dense (a slice of a packed projection) are copied first.
+        if not (_dense(q) and q.stride(3) == 1):
+            q = q.contiguous()
+        if not (_dense(k) and k.stride(3) == 1 and k.stride() == v.stride()):
+            k, v = k.contiguous(), v.contiguous()
+        if Hkv == H and k.stride() != q.stride():
+            k, v = _like(q).copy_(k), _like(q).copy_(v)
         params = binding.make_params(B, H, L, D, block_size, top_k, window, _DT[q.dtype],
                                      sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
-                                     stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride)
+                                     stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride,
+                                     kv_heads=Hkv, kv_strides=k.stride()[:3])
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -35,9 +86,8 @@ class _BlossomAttention(torch.autograd.Function):
         workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         gate = gate_logits.detach().to(torch.float32).contiguous()
         M = -(-L // block_size)
-        idx = torch.empty((B, H, M, top_k), dtype=torch.int32, device=dev)
-        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=dev)
-        out_lt, out_st = torch.empty_like(out), torch.empty_like(out)
+        idx = torch.empty((B, Hkv, M, top_k), dtype=torch.int32, device=dev)
+        out, out_lt, out_st = _like(q), _like(q), _like(q)
         lse = torch.empty((2, B, H, L), dtype=torch.float32, device=dev)
         binding.blossom_attn_fwd(params, q, k, v, gate, seq_lens, idx, 0, out, out_lt, out_st, lse,
                                  workspace)
@@ -51,10 +101,8 @@ class _BlossomAttention(torch.autograd.Function):
     def backward(ctx, dout, _didx):
         q, k, v, gate, idx, out_lt, out_st, lse = ctx.saved_tensors
         if dout.stride() != q.stride() or dout.dtype != q.dtype:  # the library wants q's layout
-            tmp = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
-            tmp.copy_(dout)
-            dout = tmp
-        dq, dk, dv = torch.empty_like(out_lt), torch.empty_like(out_lt), torch.empty_like(out_lt)
+            dout = _like(q).copy_(dout)
+        dq, dk, dv = _like(q), _like(k), _like(k)
         dgate = torch.empty((q.shape[1], 2), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
@@ -64,11 +112,15 @@ class _BlossomAttention(torch.autograd.Function):
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
                       return_indices=False, short_term="window", mask_block=1, cmp_block=0,
                       cmp_stride=0):
-    """Gated two-branch sparse attention of [B, H, L, D] tensors (float32 or bfloat16, CUDA).
+    """Gated two-branch sparse attention of q [B, H, L, D] and k, v [B, Hkv, L, D] (float32 or
+    bfloat16, CUDA; Hkv divides H: with Hkv < H the query heads of a group share key/value head
+    and selection, and the returned indices are [B, Hkv, M, top_k]).
 
     gate_logits: [H, 2] (column 0 long-term, column 1 short-term branch); seq_lens: optional int32
     [B] valid lengths of left-padded sequences; sm_scale 0 means 1/sqrt(D).  Differentiable in
     q, k, v and gate_logits.  Returns the output, and the selected block indices if asked.
+    A wait that runs out inside a kernel is reported through ``binding.blossom_device_status`` of
+    the call's workspace (it synchronises, so this front end does not poll it).
     short_term: "window" (keys t - window < p <= t) or "power-law" (Eq. 15: the window, blocks of
     mask_block positions at power-of-two block distances, and the last mask_block positions).
     cmp_block / cmp_stride: length and stride of overlapping compression blocks for the selection

@@ -27,7 +27,7 @@ EXPORTS = (
     "blossom_workspace_bytes", "blossom_select_blocks", "blossom_select_blocks_static",
     "blossom_attn_fwd", "blossom_attn_bwd",
     "blossom_device_status", "blossom_status_string", "blossom_version", "blossom_launch_count",
-    "blossom_profile_start", "blossom_profile_stop", "blossom_kernel_name",
+    "blossom_profile_start", "blossom_profile_stop", "blossom_kernel_name", "blossom_debug_switch",
 )
 
 
@@ -87,6 +87,8 @@ def load():
     lib.blossom_profile_stop.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     lib.blossom_kernel_name.restype = ctypes.c_char_p
     lib.blossom_kernel_name.argtypes = [ctypes.c_int]
+    lib.blossom_debug_switch.restype = ctypes.c_int
+    lib.blossom_debug_switch.argtypes = [ctypes.c_int, ctypes.c_int]
     _lib = lib
     return lib
 
@@ -220,3 +222,14 @@ def blossom_profile_stop(capacity: int):
 
 def blossom_kernel_name(kernel_id: int) -> str:
     return load().blossom_kernel_name(int(kernel_id)).decode()
+
+
+SWITCH_FORCE_SIMT = 0
+SWITCH_EXACT_SELECT = 1
+
+
+def blossom_debug_switch(which: int, value: int) -> None:
+    """Process-wide debugging switch: 1 on, 0 off, -1 back to the environment's default."""
+    rc = load().blossom_debug_switch(int(which), int(value))
+    if rc:
+        raise BlossomError(rc, "blossom_debug_switch")

@@ -42,14 +42,19 @@ void prof_mark(int id, int phase, cudaStream_t st) {
 // last call must not be charged to this call's first kernel.
 void prof_break() { g_prof_chain = false; }
 
-bool force_simt() {
-  const char *e = getenv("BLOSSOM_FORCE_SIMT");
+// The two environment switches are read once, when the library is loaded.
+static bool env_flag(const char *name) {
+  const char *e = getenv(name);
   return e && e[0] && e[0] != '0';
 }
+static const bool g_force_simt = env_flag("BLOSSOM_FORCE_SIMT");
+static const bool g_exact_select = env_flag("BLOSSOM_EXACT_SELECT");
+static int g_force_simt_override = -1, g_exact_select_override = -1;  // blossom_debug_switch
+
+bool force_simt() { return g_force_simt_override >= 0 ? g_force_simt_override != 0 : g_force_simt; }
 
 bool exact_select_only() {
-  const char *e = getenv("BLOSSOM_EXACT_SELECT");
-  return e && e[0] && e[0] != '0';
+  return g_exact_select_override >= 0 ? g_exact_select_override != 0 : g_exact_select;
 }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -65,6 +70,7 @@ Workspace carve_workspace(const Shape &s, void *base) {
     return r;
   };
   w.status = reinterpret_cast<int32_t *>(take(256));
+  w.status_bwd = w.status ? w.status + 4 : nullptr;
   w.kmean = reinterpret_cast<double *>(take(units * s.M * s.D * sizeof(double)));
   w.klive = reinterpret_cast<int32_t *>(take(units * s.M * sizeof(int32_t)));
   w.kmean32 = reinterpret_cast<float *>(take(units * s.M * s.D * sizeof(float)));
@@ -143,12 +149,17 @@ static int make_shape(const blossom_params *p, Shape *out) {
 
 static bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
-// Validates the workspace and clears its status word on the stream (a memset, not a kernel).
-static int check_workspace(const Shape &s, void *ws, size_t bytes, cudaStream_t st, Workspace *out) {
+// Validates the workspace and clears the status words of the calling pass on the stream (a
+// memset, not a kernel).  The forward (and the selection) own words 0..3, the backward words
+// 4..7, so a wait that ran out in the forward is still on record after the backward that
+// follows it on the same workspace.
+static int check_workspace(const Shape &s, void *ws, size_t bytes, cudaStream_t st, Workspace *out,
+                           bool backward = false) {
   if (!ws || misaligned(ws, 256)) return BLOSSOM_ERR_WORKSPACE;
   *out = carve_workspace(s, ws);
   if (bytes < out->bytes) return BLOSSOM_ERR_WORKSPACE;
-  if (cudaMemsetAsync(out->status, 0, 16, st) != cudaSuccess) return BLOSSOM_ERR_CUDA;
+  if (cudaMemsetAsync(backward ? out->status_bwd : out->status, 0, 16, st) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
   return BLOSSOM_OK;
 }
 
@@ -241,7 +252,7 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
       misaligned(gate_logits, 4) || misaligned(block_idx, 4) || misaligned(seq_lens, 4))
     return BLOSSOM_ERR_INVALID_ARG;
   Workspace ws;
-  rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
+  rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws, true);
   if (rc) return rc;
   if (!force_simt() && tc::fwd_tc_supported(s, params->dtype)) {
     rc = tc::launch_bwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out_lt, out_st, lse, dout, dq,
@@ -256,8 +267,18 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
 int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out) {
   if (!workspace || !host_out) return BLOSSOM_ERR_INVALID_ARG;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BLOSSOM_ERR_CUDA;
-  if (cudaMemcpy(host_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+  int32_t words[8];
+  if (cudaMemcpy(words, workspace, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
+  *host_out = words[0] ? words[0] : words[4];  // the forward's word, else the backward's
+  return BLOSSOM_OK;
+}
+
+int blossom_debug_switch(int which, int value) {
+  if (value < -1 || value > 1) return BLOSSOM_ERR_INVALID_ARG;
+  if (which == 0) g_force_simt_override = value;
+  else if (which == 1) g_exact_select_override = value;
+  else return BLOSSOM_ERR_INVALID_ARG;
   return BLOSSOM_OK;
 }
 

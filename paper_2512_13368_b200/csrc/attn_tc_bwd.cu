@@ -786,13 +786,13 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
     LaunchScope ls(K_BWD_DQ_TC, st);
     bwd_dq_tc_kernel<D><<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
                                                            tdq, ws.qstats, ws.dalpha,
-                                                           ws.status, nT);
+                                                           ws.status_bwd, nT);
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
     const unsigned grid_k = (unsigned)nST * (unsigned)(s.B * s.Hkv);
     bwd_dkdv_tc_kernel<D><<<grid_k, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
-                                                             ws.qstats, tdk, tdv, ws.status, nT);
+                                                             ws.qstats, tdk, tdv, ws.status_bwd, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -23,7 +23,8 @@ struct Shape {
 
 // Device scratch carved out of the caller's workspace.
 struct Workspace {
-  int32_t *status;   // [4] word 0: device status (0 = ok)
+  int32_t *status;   // [4] word 0: device status (0 = ok) of the selection / forward kernels
+  int32_t *status_bwd;  // [4] the same for the backward kernels (status + 4)
   double *kmean;     // [B][H][M][D]  mean of each block's valid keys (Eq. 9 summary)
   int32_t *klive;    // [B][H][M]     number of valid keys in the block
   float *kmean32;    // [B][H][M][D]  the means rounded to fp32 (single-precision scoring stage)

@@ -103,3 +103,72 @@ def test_params_struct_layout_matches_header():
     assert binding.blossom_params.cmp_block.offset == 80 and binding.blossom_params.cmp_stride.offset == 84
     assert binding.blossom_params.stride_b.offset == 48
     assert binding.blossom_params.stis_mode.offset == 72 and binding.blossom_params.stis_block.offset == 76
+
+
+# ---- the autograd front end validates what it hands to the library as raw addresses -------------
+def _qkv(B=2, H=4, L=16, D=32, Hkv=None, dtype=None):
+    import torch
+    dtype = dtype or torch.bfloat16
+    q = torch.zeros(B, H, L, D, dtype=dtype)
+    k = torch.zeros(B, Hkv or H, L, D, dtype=dtype)
+    return q, k, k.clone()
+
+
+def test_autograd_front_end_rejects_bad_arguments_before_any_launch():
+    import torch
+    from paper_2512_13368_b200.autograd import check_arguments
+    q, k, v = _qkv()
+    gate = torch.zeros(4, 2)
+    with pytest.raises(ValueError):           # host tensors: the library would dereference host addresses
+        check_arguments(q, k, v, gate, None)
+    chk = lambda *a: check_arguments(*a, require_cuda=False)  # noqa: E731
+    assert chk(q, k, v, gate, None) is None
+    with pytest.raises(ValueError):
+        chk(q, k, v, torch.zeros(4, 3), None)                 # gate shape
+    with pytest.raises(ValueError):
+        chk(q, k, v, torch.zeros(2, 2), None)
+    with pytest.raises(TypeError):
+        chk(q, k, v, torch.zeros(4, 2, dtype=torch.int32), None)
+    with pytest.raises(ValueError):
+        chk(q, k, v, gate.to("meta"), None)                   # another device
+    with pytest.raises(ValueError):
+        chk(q, k, v, gate, torch.zeros(3, dtype=torch.int32))  # wrong number of lengths
+    with pytest.raises(TypeError):
+        chk(q, k, v, gate, torch.zeros(2, dtype=torch.float32))
+    with pytest.raises(ValueError):
+        chk(q, k, v, gate, torch.zeros(2, dtype=torch.int32, device="meta"))
+    lens = chk(q, k, v, gate, torch.tensor([16, 3], dtype=torch.int64))
+    assert lens.dtype == torch.int32 and lens.tolist() == [16, 3]   # int64 would be read as int32 pairs
+    with pytest.raises(TypeError):
+        chk(q, k.float(), v.float(), gate, None)
+    with pytest.raises(ValueError):
+        chk(q, *_qkv(Hkv=3)[1:], gate, None)                  # 4 heads on 3 key/value heads
+    q2, k2, v2 = _qkv(Hkv=2)
+    assert chk(q2, k2, v2, gate, None) is None                # grouped heads
+
+
+def test_every_q_shaped_buffer_gets_q_strides():
+    import torch
+    from paper_2512_13368_b200.autograd import _dense, _like
+    qkv = torch.zeros(2, 16, 3, 4, 32)                        # packed projection [B, L, 3, H, D]
+    q = qkv[:, :, 0].permute(0, 2, 1, 3)                      # [B, H, L, D], equal strides, not dense
+    assert not _dense(q)
+    assert torch.empty_like(q).stride() != q.stride()         # what made the library overrun its outputs
+    assert _like(q).stride() == q.stride()
+    qc = q.contiguous()
+    assert _dense(qc) and _like(qc).stride() == qc.stride()
+    perm = torch.zeros(2, 16, 4, 32).permute(0, 2, 1, 3)      # [B, L, H, D] storage: dense, kept as is
+    assert _dense(perm) and _like(perm).stride() == perm.stride()
+
+
+def test_debug_switch_arguments(lib):
+    assert lib.blossom_debug_switch(0, -1) == 0 and lib.blossom_debug_switch(1, -1) == 0
+    assert lib.blossom_debug_switch(2, 0) == binding.BLOSSOM_ERR_INVALID_ARG
+    assert lib.blossom_debug_switch(0, 2) == binding.BLOSSOM_ERR_INVALID_ARG
+
+
+def test_static_selection_rejects_overlapping_compression_blocks(lib):
+    A = 1 << 20
+    prm = good(cmp_block=16, cmp_stride=4)
+    rc = binding.blossom_select_blocks_static(prm, A, A, None, A, stream=0, check=False)
+    assert rc == binding.BLOSSOM_ERR_UNSUPPORTED

@@ -27,6 +27,51 @@ def test_autograd_matches_oracle():
         assert err <= tolerance(w, ref[key]), (key, err)
 
 
+def test_autograd_packed_projection_views_and_grouped_heads():
+    """q, k, v cut out of one packed projection buffer (equal strides, not dense: the layout that
+    once made the outputs overrun their allocation), int64 lengths, and 4 query heads on 2
+    key/value heads: outputs and gradients against the oracle."""
+    import torch
+    import oracle
+    from paper_2512_13368_b200.autograd import blossom_attention
+    dev = torch.device("cuda:0")
+    bf = lambda a: torch.from_numpy(a).to(dev).to(torch.bfloat16)  # noqa: E731
+    # ---- packed [B, L, 3, H, D] buffer, views [B, H, L, D]
+    w = workloads.make("packed", "bf16", 2, 3, 200, 64, 32, 3, 40, seed=22, lengths=(50, 200))
+    qkv = torch.stack([bf(w.q), bf(w.k), bf(w.v)], dim=1)            # [B, 3, H, L, D]
+    qkv = qkv.permute(0, 3, 1, 2, 4).contiguous().requires_grad_(True)   # [B, L, 3, H, D]
+    q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    gate = torch.from_numpy(w.gate).to(dev).requires_grad_(True)
+    lens = torch.from_numpy(w.seq_lens.astype(np.int64)).to(dev)
+    guard = torch.full((1 << 20,), 7.0, device=dev)                  # a neighbour in the allocator's pool
+    out, idx = blossom_attention(q, k, v, gate, w.block, w.topk, w.window, seq_lens=lens, return_indices=True)
+    out.backward(bf(w.dout))
+    torch.cuda.synchronize()
+    assert bool((guard == 7.0).all())
+    ref = oracle.forward_backward(w.q, w.k, w.v, w.gate, w.dout, w.block, w.topk, w.window, w.seq_lens,
+                                  idx=idx.cpu().numpy())
+    g = qkv.grad.permute(0, 2, 3, 1, 4)                              # [B, 3, H, L, D]
+    got = {"out": out, "dq": g[:, 0], "dk": g[:, 1], "dv": g[:, 2], "dgate": gate.grad}
+    for key, val in got.items():
+        err = float(np.abs(val.detach().float().cpu().numpy() - ref[key]).max())
+        assert err <= tolerance(w, ref[key]), (key, err)
+    # ---- grouped heads
+    w = workloads.make("autograd-gqa", "bf16", 2, 4, 256, 32, 32, 3, 48, seed=23, kv_heads=2)
+    t = lambda a: bf(a).requires_grad_(True)  # noqa: E731
+    q, k, v = t(w.q), t(w.k), t(w.v)
+    gate = torch.from_numpy(w.gate).to(dev).requires_grad_(True)
+    out, idx = blossom_attention(q, k, v, gate, w.block, w.topk, w.window, return_indices=True)
+    out.backward(bf(w.dout))
+    assert tuple(idx.shape) == (2, 2, 8, 3) and k.grad.shape == k.shape
+    f = oracle.forward_gqa(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, idx=idx.cpu().numpy())
+    ref = dict(f)
+    ref.update(oracle.backward_gqa(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, f, w.dout))
+    got = {"out": out, "dq": q.grad, "dk": k.grad, "dv": v.grad, "dgate": gate.grad}
+    for key, val in got.items():
+        err = float(np.abs(val.detach().float().cpu().numpy() - ref[key]).max())
+        assert err <= tolerance(w, ref[key]), (key, err)
+
+
 def test_layer_step_runs_and_reports_attention_share():
     from paper_2512_13368_b200 import layer_step
     r = layer_step.attention_share(batch=8, seq_len=256, n_items=2000, negatives=15, steps=2, warmup=1)

@@ -1,7 +1,5 @@
 """Parity of the CUDA library (through its C ABI) against the fp64 oracle on the same seeded
 inputs.  Every test here needs a B200."""
-import concurrent.futures as cf
-
 import numpy as np
 import pytest
 
@@ -286,73 +284,69 @@ def test_constructed_ties_pick_lower_index(runner):
     assert check_indices(w, res["idx"]) == 0
 
 
-# ------------------------------------------------- full benchmark sizes, sampled outputs
-def _sampled_units(runner, w, units):
-    p, _ = None, None
+# ------------------------------------------------- full benchmark sizes, every output element
+def _whole_batch(runner, w):
+    """One step at the full benchmark size, in the launch configuration the benchmark times, and
+    every element of every output (indices, out, out_lt, out_st, lse, dq, dk, dv and the gate
+    gradient, which is a sum over the whole batch) compared with the oracle run on the whole
+    batch (it parallelises over (batch, head) units by itself)."""
     p = runner.DeviceProblem(w)
     p.step()
+    from paper_2512_13368_b200 import binding
+    assert binding.blossom_device_status(p.workspace) == 0
     res = p.results()
-
-    def one(nh):
-        n, h = nh
-        wu = w.unit(n, h)
-        G = w.H // (w.kv_heads or w.H)
-        hq = slice(h * G, (h + 1) * G)      # the query heads of key/value head h
-        ru = {k: (v[n:n + 1, h:h + 1] if k in ("idx", "dk", "dv") else v[n:n + 1, hq])
-              for k, v in res.items() if k not in ("lse", "dgate")}
-        ru["lse"] = res["lse"][:, n:n + 1, hq]
-        ru["dgate"] = None          # summed over the batch: checked separately on small cases
-        return check_forward_backward(wu, ru)
-
-    with cf.ThreadPoolExecutor(max_workers=4) as ex:
-        return list(ex.map(one, units)), res
+    errs = check_forward_backward(w, res)
+    assert "dgate" in errs and "dk" in errs
+    return errs, res
 
 
-def test_config3_full_size_sampled(runner):
-    w = workloads.config3()
-    errs, _ = _sampled_units(runner, w, [(0, 0), (37, 2), (127, 3)])
+def test_config3_full_size(runner):
+    errs, _ = _whole_batch(runner, workloads.config3())
     print(errs)
 
 
-def test_config4_full_size_sampled(runner):
-    w = workloads.config4()
-    errs, _ = _sampled_units(runner, w, [(0, 0), (9, 5), (15, 7)])
+def test_config4_full_size(runner):
+    errs, _ = _whole_batch(runner, workloads.config4())
     print(errs)
 
 
-def test_config4_full_size_grouped_heads_sampled(runner):
+def test_config5_attention_shape_full_batch(runner):
+    errs, _ = _whole_batch(runner, workloads.config5_attention())
+    print(errs)
+
+
+def test_config4_full_size_grouped_heads(runner):
     """The headline shape with its 8 query heads on 2 key/value heads, as the benchmark's
-    --kv-heads 2 option times it; a sampled unit is a whole group."""
+    --kv-heads 2 option times it."""
     w = workloads.config4(kv_heads=2)
-    errs, res = _sampled_units(runner, w, [(0, 0), (11, 1)])
+    errs, res = _whole_batch(runner, w)
     print(errs)
     assert res["idx"].shape == (w.B, 2, w.n_blocks, w.topk) and res["dk"].shape == w.k.shape
 
 
-def test_config4_full_size_overlapping_compression_sampled(runner):
+def test_config4_full_size_overlapping_compression(runner):
     """The headline shape with compression blocks of 128 keys at stride 32 behind the selection,
     as the benchmark's --cmp-block 128 --cmp-stride 32 option times it."""
     w = workloads.config4()
     w.cmp_block, w.cmp_stride = 128, 32
-    errs, _ = _sampled_units(runner, w, [(0, 0), (11, 6)])
+    errs, _ = _whole_batch(runner, w)
     print(errs)
 
 
-def test_config4_full_size_power_law_sampled(runner):
+def test_config4_full_size_power_law(runner):
     """The headline shape with the paper's short-term mask (window 8, mask block 1), in the launch
     configuration the benchmark's --short-term power-law option times."""
     w = workloads.config4()
     w.stis_mode, w.stis_block, w.window = 1, 1, 8
-    errs, _ = _sampled_units(runner, w, [(0, 0), (7, 3), (15, 7)])
+    errs, _ = _whole_batch(runner, w)
     print(errs)
 
 
-def test_config2_full_size_sampled(runner):
+def test_config2_full_size(runner):
     w = workloads.config2()
-    units = [(int(np.argmin(w.seq_lens)), 0), (int(np.argmax(w.seq_lens)), 1), (100, 0), (255, 1)]
-    errs, res = _sampled_units(runner, w, units)
+    errs, res = _whole_batch(runner, w)
     print(errs)
-    # properties that hold at any size: structure of every index row, zero padding
+    # structure of every index row, zero padding
     idx = res["idx"]
     M = w.n_blocks
     own = np.arange(M)[None, None, :]
@@ -360,9 +354,31 @@ def test_config2_full_size_sampled(runner):
     pad0 = w.L - w.seq_lens
     live_block = (np.minimum((np.arange(M) + 1) * w.block, w.L)[None, :] > pad0[:, None])
     assert np.all(np.where(live_block[:, None, :], last == own, last == -1))
+    for n in range(w.B):
+        for key in ("out", "out_lt", "out_st", "dq", "dk", "dv"):
+            assert np.all(res[key][n, :, :pad0[n]] == 0.0)
 
 
-def test_certified_selection_equals_double_precision_selection(runner, monkeypatch):
+def _fast_and_exact_selection(p):
+    """The indices of the two-stage selection and of the double-precision-only selection."""
+    import torch
+    from paper_2512_13368_b200 import binding
+    binding.blossom_debug_switch(binding.SWITCH_EXACT_SELECT, 0)
+    try:
+        p.select()
+        torch.cuda.synchronize()
+        fast = p.idx.cpu().numpy().copy()
+        binding.blossom_debug_switch(binding.SWITCH_EXACT_SELECT, 1)
+        p.idx.fill_(-7)
+        p.select()
+        torch.cuda.synchronize()
+        exact = p.idx.cpu().numpy().copy()
+    finally:
+        binding.blossom_debug_switch(binding.SWITCH_EXACT_SELECT, -1)
+    return fast, exact
+
+
+def test_certified_selection_equals_double_precision_selection(runner):
     """The two-stage selection (fp32 scores with an error bound, fp64 only for the uncertain query
     blocks) must return exactly what scoring every query block in fp64 returns."""
     import torch
@@ -378,21 +394,12 @@ def test_certified_selection_equals_double_precision_selection(runner, monkeypat
               workloads.make("many-blocks", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9),
               overlap4, overlap2, small_stride):
         p = runner.DeviceProblem(w)
-        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
-        p.select()
-        torch.cuda.synchronize()
-        fast = p.idx.cpu().numpy().copy()
-        monkeypatch.setenv("BLOSSOM_EXACT_SELECT", "1")
-        p.idx.fill_(-7)
-        p.select()
-        torch.cuda.synchronize()
-        exact = p.idx.cpu().numpy()
-        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
+        fast, exact = _fast_and_exact_selection(p)
         assert np.array_equal(fast, exact), w.name
         check_indices(w, fast)
 
 
-def test_certified_selection_on_random_small_block_shapes(runner, monkeypatch):
+def test_certified_selection_on_random_small_block_shapes(runner):
     """Short sequences of 16- and 32-position blocks take the first-stage kernel that packs
     several query blocks into a CTA: over random shapes, lengths, scales and exact ties (identical
     keys) its choice must be the double-precision one, bit for bit."""
@@ -411,14 +418,5 @@ def test_certified_selection_on_random_small_block_shapes(runner, monkeypatch):
         if it % 7 == 0:
             w.k[:] = w.k[:, :, :1, :]      # every key equal: every score ties
         p = runner.DeviceProblem(w)
-        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
-        p.select()
-        torch.cuda.synchronize()
-        fast = p.idx.cpu().numpy().copy()
-        monkeypatch.setenv("BLOSSOM_EXACT_SELECT", "1")
-        p.idx.fill_(-7)
-        p.select()
-        torch.cuda.synchronize()
-        exact = p.idx.cpu().numpy()
-        monkeypatch.delenv("BLOSSOM_EXACT_SELECT", raising=False)
+        fast, exact = _fast_and_exact_selection(p)
         assert np.array_equal(fast, exact), (it, L, Bk, D, H, B, topk, dtype, std)

@@ -2,9 +2,10 @@
 device memory (no workspace argument; its scratch is a fixed array inside the library).
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
-every other test.  The GPU test calls the entry point through the C ABI twice in a row, on two
-different problems, and wants exactly the indices the workspace-based entry point returns: the
-second call runs on scratch that still holds the first call's contents.
+every other test.  The GPU test calls the entry point through the C ABI several times in a row,
+on different problems, and wants exactly the indices the workspace-based entry point returns (the
+later calls run on scratch that still holds an earlier call's contents) and the indices the
+CPU oracle selects.
 """
 import numpy as np
 import pytest
@@ -34,8 +35,11 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
     import torch
     assert torch.cuda.is_available()
     from paper_2512_13368_b200 import runner
+    from parity_util import check_indices
     cases = [workloads.config3(B=4),        # first call: L1024, 32 blocks, no padding
-             workloads.config2(B=32)]       # second call: smaller, left-padded, stale scratch
+             workloads.config2(B=32),       # second call: smaller, left-padded, stale scratch
+             workloads.config2(B=24, kv_heads=1),   # grouped heads: scratch indexed per key/value head
+             workloads.make("static-gqa", "bf16", 2, 8, 1024, 64, 64, 5, 64, seed=41, kv_heads=2)]
     for w in cases:
         p = runner.DeviceProblem(w)
         p.select()                                           # existing entry point
@@ -46,6 +50,7 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
         torch.cuda.synchronize()
         got = got_t.cpu().numpy()
         assert np.array_equal(got, want), w.name             # integer output: bit-exact
+        check_indices(w, got)                                # and the oracle's choice (Eq. 13)
     # and once more on the first problem, now after the smaller one
     w = cases[0]
     p = runner.DeviceProblem(w)
