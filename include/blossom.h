@@ -187,8 +187,8 @@ int blossom_attn_bwd(const blossom_params *params /* host */, const void *q, con
 
 /* Synchronises the stream and copies the workspace's device status to *host_out (host): 0 = no
  * device-side error, else a blossom_status.  The workspace holds one status word for the forward
- * (blossom_select_blocks and blossom_attn_fwd clear it when they start) and one for the backward
- * (blossom_attn_bwd clears only that one), so a read after a forward + backward pair on one
+ * (blossom_select_blocks and blossom_attn_fwd clear both words when they start: a new step) and
+ * one for the backward (blossom_attn_bwd clears only that one), so a read after a forward + backward pair on one
  * workspace reports a wait that ran out in either; the forward's word wins if both are set.
  * Returns BLOSSOM_ERR_CUDA if the synchronise or the copy fails. */
 int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out);

@@ -149,16 +149,16 @@ static int make_shape(const blossom_params *p, Shape *out) {
 
 static bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
-// Validates the workspace and clears the status words of the calling pass on the stream (a
-// memset, not a kernel).  The forward (and the selection) own words 0..3, the backward words
-// 4..7, so a wait that ran out in the forward is still on record after the backward that
-// follows it on the same workspace.
+// Validates the workspace and clears status words on the stream (a memset, not a kernel).  The
+// forward (and the selection) report in words 0..3, the backward in words 4..7.  A forward or a
+// selection clears both sets (a new step begins), a backward only its own, so a wait that ran out
+// in the forward is still on record after the backward that follows it on the same workspace.
 static int check_workspace(const Shape &s, void *ws, size_t bytes, cudaStream_t st, Workspace *out,
                            bool backward = false) {
   if (!ws || misaligned(ws, 256)) return BLOSSOM_ERR_WORKSPACE;
   *out = carve_workspace(s, ws);
   if (bytes < out->bytes) return BLOSSOM_ERR_WORKSPACE;
-  if (cudaMemsetAsync(backward ? out->status_bwd : out->status, 0, 16, st) != cudaSuccess)
+  if (cudaMemsetAsync(backward ? out->status_bwd : out->status, 0, backward ? 16 : 32, st) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   return BLOSSOM_OK;
 }
