@@ -142,7 +142,6 @@ static int make_shape(const blossom_params *p, Shape *out) {
   } else {
     s.ksl = s.D; s.ksh = (int64_t)s.L * s.D; s.ksb = (int64_t)s.Hkv * s.L * s.D;
   }
-  if (s.G > 1 && s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // overlapping blocks: one head per group only
   *out = s;
   return BLOSSOM_OK;
 }

@@ -117,8 +117,6 @@ __device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, 
 }
 
 // launchers (one translation unit each)
-int launch_select_cmp(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
-                      int32_t *idx, const Workspace &ws, cudaStream_t st);
 int launch_select(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
                   int32_t *idx, const Workspace &ws, cudaStream_t st);
 int launch_fwd_simt(const Shape &s, int dtype, const void *q, const void *k, const void *v,

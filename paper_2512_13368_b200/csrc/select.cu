@@ -1,813 +1,767 @@
-// Block summary, importance scoring and top-k selection (paper Eq. 8-10, 12, 13 with
-// compression size = stride = selection size = Bk and the summary = mean of a block's valid keys).
+// Block summary, importance scoring and top-k selection (paper Eq. 8-13).
+//
+// One code path serves the plain selection (compression size = stride = selection size = Bk, the
+// ragged last block kept) and the selection through overlapping compression blocks (Eq. 8 with
+// length l and stride s, only whole blocks, and the score remap of Eq. 11), for one head per
+// key/value head or for groups of heads that share one selection (Eq. 12: the probabilities of the
+// group's heads are summed).  The "scored blocks" below are the compression blocks: positions
+// [s c, s c + l), summarised by the mean of their valid keys (Eq. 9 with the summary = mean).
+// Query block b scores the scored blocks that end before it starts (candidates c < nc(b)), every
+// valid query taking a softmax over the live candidates (Eq. 10), the probabilities being summed
+// over the block's queries and the group's heads; Eq. 11 maps those sums onto the selection blocks
+// j < b (the identity in the plain mode); the own block plus the top_k - 1 best selectable past
+// blocks are kept, ties to the lower index (Eq. 13).
 //
 // The selection is a discrete decision taken from floating-point sums whose neighbours differ by
 // ~1e-3 relative on Gaussian inputs, and the library promises the choice a double-precision
 // evaluation makes (ties below ~1e-12 relative excepted).  Two stages deliver it:
 //   1. every query block is scored in single precision together with a rigorous bound on the
 //      distance of each score from its exact value; if the last kept and the first dropped
-//      candidate are further apart than the bound allows them to move, the choice is certain and
-//      is written out;
+//      selection block are further apart than the bound allows them to move, the choice is certain
+//      and is written out;
 //   2. the (few per cent of) query blocks whose choice is not certain are appended to a work
 //      list and re-scored in double precision by a second kernel.
+// With left padding a block is live exactly when it reaches past the padding, so liveness is a
+// comparison of indices (cmin, jmin below); the counts of valid keys are kept for callers that
+// want them.
 #include "common.cuh"
 
 namespace blossom {
 
 namespace {
 
-constexpr int kSelThreads = 256;
-constexpr int kSelWarps = kSelThreads / 32;
+// Geometry of the scored blocks.
+struct SelGeom {
+  int n;       // scored blocks per (batch, key/value head): Mc, or M in the plain mode
+  int l, s;    // their length and stride in positions
+  int rs, rl;  // Bk / s and l / s, the two sums of Eq. 11 (1, 1 in the plain mode)
+  int plain;
+};
 
-// ---- Eq. 8 + 9: per key block, mean of the valid keys (fp64) ------------------------------
-// grid M*B*H (unit-major), 256 threads: thread = (row group, 4-element column chunk); 128-bit/64-bit loads.
+SelGeom sel_geom(const Shape &sh) {
+  SelGeom g;
+  if (sh.cmp_l > 0) {
+    g.n = sh.Mc; g.l = sh.cmp_l; g.s = sh.cmp_s; g.rs = sh.Bk / sh.cmp_s; g.rl = sh.cmp_l / sh.cmp_s;
+    g.plain = 0;
+  } else {
+    g.n = sh.M; g.l = sh.Bk; g.s = sh.Bk; g.rs = 1; g.rl = 1; g.plain = 1;
+  }
+  return g;
+}
+
+// scored blocks 0 .. nc - 1 end before query block b starts
+__device__ __forceinline__ int n_candidates(const Shape &sh, const SelGeom &g, int b) {
+  if (g.plain) return b;
+  const int start = b * sh.Bk;
+  return start >= g.l ? min(g.n, (start - g.l) / g.s + 1) : 0;
+}
+// the first scored block that holds a valid key (pad0 = number of padded positions)
+__device__ __forceinline__ int first_live_scored(const SelGeom &g, int pad0) {
+  return pad0 < g.l ? 0 : (pad0 - g.l) / g.s + 1;
+}
+
+// Eight consecutive elements as loaded (16 bytes of bf16, 32 of fp32), unpacked to floats on use.
+template <typename T>
+struct Raw8;
+template <>
+struct Raw8<__nv_bfloat16> {
+  uint4 r;
+  __device__ __forceinline__ void load(const __nv_bfloat16 *p) { r = *reinterpret_cast<const uint4 *>(p); }
+  __device__ __forceinline__ void zero() { r = make_uint4(0u, 0u, 0u, 0u); }
+  __device__ __forceinline__ void unpack(float (&x)[8]) const {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      x[2 * e] = __uint_as_float(w[e] << 16);
+      x[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    }
+  }
+};
+template <>
+struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float *p) {
+    a = *reinterpret_cast<const float4 *>(p);
+    b = *reinterpret_cast<const float4 *>(p + 4);
+  }
+  __device__ __forceinline__ void zero() { a = b = make_float4(0.f, 0.f, 0.f, 0.f); }
+  __device__ __forceinline__ void unpack(float (&x)[8]) const {
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  }
+};
+
+// ---- Eq. 8 + 9: mean of the valid keys of every scored block (fp64) ------------------------
+// One warp per scored block, 8 blocks per CTA.  A lane owns eight columns (one 16-byte load of
+// bf16, two of fp32) of every (32 / (D / 8))-th row and sums them in a fixed order with eight rows
+// in flight (kept as loaded until they are added); the lanes that share columns are combined by
+// shuffles in a fixed tree.
 template <typename T, int D>
-__global__ void __launch_bounds__(256) summary_kernel(Shape s, const T *__restrict__ k,
-                                                      const int32_t *__restrict__ seq_lens,
-                                                      double *__restrict__ kmean,
-                                                      int32_t *__restrict__ klive,
-                                                      float *__restrict__ kmean32,
-                                                      float *__restrict__ knorm,
-                                                      int32_t *__restrict__ sel_count) {
-  constexpr int CH = D / 4;        // chunks per row
-  constexpr int RG = 256 / CH;     // row groups
-  __shared__ double part[RG][D];
-  __shared__ float sq[D];
+__global__ void __launch_bounds__(256, 4) summary_kernel(Shape sh, SelGeom g, const T *__restrict__ k,
+                                                         const int32_t *__restrict__ seq_lens,
+                                                         double *__restrict__ mean,
+                                                         int32_t *__restrict__ live,
+                                                         float *__restrict__ mean32,
+                                                         float *__restrict__ norm,
+                                                         int32_t *__restrict__ sel_count) {
+  constexpr int LPR = D / 8;     // lanes per row
+  constexpr int RPI = 32 / LPR;  // rows per warp iteration
+  constexpr int NF = sizeof(T) == 2 ? 8 : 2;  // rows in flight per lane
   if (blockIdx.x == 0 && threadIdx.x == 0) *sel_count = 0;  // work list of the scoring kernel
-  // u counts (batch, key/value head) pairs
-  const int j = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.Hkv, hk = u % s.Hkv;
-  int len = seq_lens ? seq_lens[n] : s.L;
-  len = min(max(len, 0), s.L);
-  const int pad0 = s.L - len;
-  const int lo = max(j * s.Bk, pad0), hi = min((j + 1) * s.Bk, s.L);
-  const int ch = threadIdx.x % CH, rg = threadIdx.x / CH;
-  double a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-  for (int p = lo + rg; p < hi; p += RG) {
-    float4 x = ld4(k + row_offset_kv(s, n, hk, p) + ch * 4);
-    a0 += (double)x.x; a1 += (double)x.y; a2 += (double)x.z; a3 += (double)x.w;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t blk = (int64_t)blockIdx.x * 8 + warp;  // (batch, key/value head, scored block)
+  if (blk >= (int64_t)sh.B * sh.Hkv * g.n) return;
+  const int c = (int)(blk % g.n), u = (int)(blk / g.n), n = u / sh.Hkv, hk = u % sh.Hkv;
+  int len = seq_lens ? seq_lens[n] : sh.L;
+  len = min(max(len, 0), sh.L);
+  const int pad0 = sh.L - len;
+  const int lo = max(c * g.s, pad0), hi = min(c * g.s + g.l, sh.L);
+  const int sub = lane / LPR, col = (lane % LPR) * 8;
+  const T *base = k + row_offset_kv(sh, n, hk, 0) + col;
+  double a[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) a[e] = 0.0;
+  for (int p = lo + sub; p < hi; p += NF * RPI) {
+    Raw8<T> x[NF];
+#pragma unroll
+    for (int r = 0; r < NF; ++r) {
+      const int pp = p + r * RPI;
+      if (pp < hi) x[r].load(base + (int64_t)pp * sh.ksl);
+      else x[r].zero();
+    }
+#pragma unroll
+    for (int r = 0; r < NF; ++r) {
+      float f[8];
+      x[r].unpack(f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a[e] += (double)f[e];
+    }
   }
-  part[rg][ch * 4 + 0] = a0; part[rg][ch * 4 + 1] = a1;
-  part[rg][ch * 4 + 2] = a2; part[rg][ch * 4 + 3] = a3;
-  __syncthreads();
+#pragma unroll
+  for (int o = LPR; o < 32; o <<= 1)  // the lanes that took other rows of the same columns
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] += __shfl_xor_sync(0xffffffffu, a[e], o);
   const int cnt = max(hi - lo, 0);
-  if (threadIdx.x < D) {
-    double acc = 0;
-    for (int r = 0; r < RG; ++r) acc += part[r][threadIdx.x];  // fixed order
-    const double mean = cnt > 0 ? acc / (double)cnt : 0.0;
-    kmean[((int64_t)u * s.M + j) * D + threadIdx.x] = mean;
-    const float m32 = (float)mean;
-    kmean32[((int64_t)u * s.M + j) * D + threadIdx.x] = m32;
-    sq[threadIdx.x] = m32 * m32;
+  float sq = 0.f;
+  if (sub == 0) {
+    double m[8];
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      m[e] = cnt > 0 ? a[e] / (double)cnt : 0.0;
+      f[e] = (float)m[e];
+      sq = fmaf(f[e], f[e], sq);
+    }
+    double2 *md = reinterpret_cast<double2 *>(mean + blk * D + col);
+    md[0] = make_double2(m[0], m[1]); md[1] = make_double2(m[2], m[3]);
+    md[2] = make_double2(m[4], m[5]); md[3] = make_double2(m[6], m[7]);
+    float4 *mf = reinterpret_cast<float4 *>(mean32 + blk * D + col);
+    mf[0] = make_float4(f[0], f[1], f[2], f[3]);
+    mf[1] = make_float4(f[4], f[5], f[6], f[7]);
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    klive[(int64_t)u * s.M + j] = cnt;
-    float a = 0.f;
-    for (int c = 0; c < D; ++c) a += sq[c];
-    knorm[(int64_t)u * s.M + j] = sqrtf(a) * 1.0001f;  // an upper bound of the fp32 mean's norm
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  if (lane == 0) {
+    live[blk] = cnt;
+    norm[blk] = sqrtf(sq) * 1.0001f;  // an upper bound of the fp32 mean's norm
   }
 }
 
-// ---- Eq. 10 + 12 + 13: scores of one query block and its top-k --------------------------
-// grid M*B*H (unit-major), 256 threads.  One warp per query row: lanes stride over the candidate blocks,
-// softmax over the candidates, per-warp partial sums, fixed-order combine, then a candidate is
-// kept iff fewer than top_k - 1 live candidates beat it (value desc, index asc).
-template <typename T, int D>
-__device__ __forceinline__ void score_select_row(
-    const Shape &s, const T *__restrict__ q, const double *__restrict__ kmean,
-    const int32_t *__restrict__ klive, const int32_t *__restrict__ seq_lens,
-    int32_t *__restrict__ idx, int kt_in_smem, int row_id, double *sm) {
-  // u counts (batch, key/value head) pairs; the queries of all G heads of the group are scored
-  // and their probabilities summed (Eq. 12)
-  const int b = row_id % s.M, u = row_id / s.M, n = u / s.Hkv, hk = u % s.Hkv;
-  const int M = s.M;
-  const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-  int len = seq_lens ? seq_lens[n] : s.L;
-  len = min(max(len, 0), s.L);
-  const int pad0 = s.L - len;
-  const int qlo = max(b * s.Bk, pad0), qhi = min((b + 1) * s.Bk, s.L);
-  int32_t *row = idx + ((int64_t)u * M + b) * s.topk;
-
-  if (qlo >= qhi) {  // the query block holds only padding
-    for (int i = tid; i < s.topk; i += kSelThreads) row[i] = -1;
-    return;
-  }
-
-  double *zbuf = sm;                          // [warps][M]
-  double *sp = zbuf + kSelWarps * M;          // [warps][M]
-  double *qrow = sp + kSelWarps * M;          // [warps][D]
-  double *S = qrow + kSelWarps * D;           // [M]
-  int *live = reinterpret_cast<int *>(S + M);  // [M]
-  int *taken = live + M;                      // [M]
-  double *kt_s = reinterpret_cast<double *>(taken + M);  // [b][D+1] if it fits (2M ints keep 8-byte alignment)
-
-  const double *kt = kmean + (int64_t)u * M * D;
-  int kstride = D;
-  for (int j = tid; j < b; j += kSelThreads) {
-    live[j] = klive[(int64_t)u * M + j] > 0;
-    taken[j] = 0;
-  }
-  for (int i = tid; i < kSelWarps * M; i += kSelThreads) sp[i] = 0.0;
-  if (kt_in_smem) {
-    for (int i = tid; i < b * D; i += kSelThreads) kt_s[(i / D) * (D + 1) + (i % D)] = kt[i];
-    kt = kt_s;
-    kstride = D + 1;
-  }
-  __syncthreads();
-
-  int ncand = 0;
-  for (int j = 0; j < b; ++j) ncand += live[j];  // uniform
-
-  if (ncand > 0 && s.topk > 1) {
-    double *zw = zbuf + warp * M, *spw = sp + warp * M, *qw = qrow + warp * D;
-    constexpr int QPL = (D + 31) / 32;  // query elements per lane
-    double qreg[QPL];                   // the next row, loaded while the current one is scored
-    const int nq = qhi - qlo, nrows = nq * s.G;  // rows of the group: head g, query qlo + r % nq
-    if (warp < nrows) {
-      const T *qp = q + row_offset(s, n, hk * s.G + warp / nq, qlo + warp % nq);
-#pragma unroll
-      for (int e = 0; e < QPL; ++e)
-        if (lane + 32 * e < D) qreg[e] = (double)ld1(qp + lane + 32 * e);
-    }
-    for (int r = warp; r < nrows; r += kSelWarps) {
-#pragma unroll
-      for (int e = 0; e < QPL; ++e)
-        if (lane + 32 * e < D) qw[lane + 32 * e] = qreg[e];
-      __syncwarp();
-      if (r + kSelWarps < nrows) {
-        const int r2 = r + kSelWarps;
-        const T *qp = q + row_offset(s, n, hk * s.G + r2 / nq, qlo + r2 % nq);
-#pragma unroll
-        for (int e = 0; e < QPL; ++e)
-          if (lane + 32 * e < D) qreg[e] = (double)ld1(qp + lane + 32 * e);
+// ---- Eq. 11 for one query block: scores of the selection blocks j in [jmin, b) -------------
+// Sc[c], c in [cmin, nc): summed probabilities of the live candidates (anything outside counts as
+// zero).  One warp.
+template <typename F>
+__device__ __forceinline__ void map_scores(const SelGeom &g, const F *Sc, int cmin, int nc, int jmin, int b,
+                                           F *S, int lane) {
+  for (int j = jmin + lane; j < b; j += 32) {
+    F acc = (F)0;
+    for (int m = 0; m < g.rs; ++m)
+      for (int n = 0; n < g.rl; ++n) {
+        const int i = g.rs * j - m - n;
+        if (i >= cmin && i < nc) acc += Sc[i];
       }
-      double mx = -INFINITY;
-      for (int j = lane; j < b; j += 32) {
-        if (!live[j]) continue;
-        const double *kj = kt + (int64_t)j * kstride;
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;  // four chains: the FMA latency overlaps
-#pragma unroll 4
-        for (int c = 0; c < D; c += 4) {
-          a0 = fma(qw[c], kj[c], a0);
-          a1 = fma(qw[c + 1], kj[c + 1], a1);
-          a2 = fma(qw[c + 2], kj[c + 2], a2);
-          a3 = fma(qw[c + 3], kj[c + 3], a3);
-        }
-        const double z = s.scale_d * ((a0 + a1) + (a2 + a3));
-        zw[j] = z;
-        mx = fmax(mx, z);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      double den = 0.0;
-      for (int j = lane; j < b; j += 32)
-        if (live[j]) {
-          const double e = exp(zw[j] - mx);
-          zw[j] = e;
-          den += e;
-        }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-      for (int j = lane; j < b; j += 32)
-        if (live[j]) spw[j] += zw[j] / den;
-      __syncwarp();
-    }
-  }
-  __syncthreads();
-  for (int j = tid; j < b; j += kSelThreads) {
-    double acc = 0.0;
-    for (int w = 0; w < kSelWarps; ++w) acc += sp[w * M + j];  // fixed order
     S[j] = acc;
   }
-  __syncthreads();
+}
 
-  {
-    // Selection by rank: candidate j is kept iff fewer than `want` live candidates beat it (larger
-    // score, or equal score and lower index).
-    const int want = min(s.topk - 1, ncand);
-    for (int j = tid; j < b; j += kSelThreads) {
-      int rank = 0;
-      if (live[j]) {
-        const double sj = S[j];
-        for (int i = 0; i < b; ++i)
-          if (live[i]) {
-            const double si = S[i];
-            rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
-          }
-      }
-      taken[j] = live[j] && rank < want;
+// Eq. 13 by rank: block j in [jmin, b) is kept iff fewer than `want` selectable blocks beat it
+// (larger score, or equal score and lower index).  One warp; `bound` receives the smallest kept
+// and the largest dropped score.
+template <typename F>
+__device__ __forceinline__ void rank_select(const F *S, int jmin, int b, int want, uint8_t *taken, F *bound,
+                                            int lane) {
+  for (int j = jmin + lane; j < b; j += 32) {
+    const F sj = S[j];
+    int rank = 0;
+    for (int i = jmin; i < b; ++i) {
+      const F si = S[i];
+      rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
     }
-  }
-  __syncthreads();
-  if (warp == 0) {
-    // emit ascending: ballot over 32-wide chunks of the flags, then the own block
-    int pos = 0;
-    for (int base = 0; base < b; base += 32) {
-      const int j = base + lane;
-      const bool f = j < b && taken[j];
-      const unsigned m = __ballot_sync(0xffffffffu, f);
-      if (f) row[pos + __popc(m & ((1u << lane) - 1u))] = j;
-      pos += __popc(m);
-    }
-    if (lane == 0) row[pos] = b;
-    for (int i = pos + 1 + lane; i < s.topk; i += 32) row[i] = -1;
+    taken[j] = rank < want ? 1 : 0;
+    if (rank == want - 1) bound[0] = sj;  // the smallest kept score
+    if (rank == want) bound[1] = sj;      // the largest dropped score
   }
 }
 
-// The double-precision scoring of the query blocks on the work list (all of them when
-// worklist == nullptr).  grid: any; each CTA takes rows blockIdx.x, blockIdx.x + gridDim.x, ...
-template <typename T, int D>
-__global__ void __launch_bounds__(kSelThreads) score_select_kernel(
-    Shape s, const T *__restrict__ q, const double *__restrict__ kmean,
-    const int32_t *__restrict__ klive, const int32_t *__restrict__ seq_lens,
-    int32_t *__restrict__ idx, int kt_in_smem, const int32_t *__restrict__ worklist,
-    const int32_t *__restrict__ work_count) {
-  extern __shared__ double sm[];
-  const int total = worklist ? *work_count : s.M * s.B * s.Hkv;
-  for (int w = blockIdx.x; w < total; w += gridDim.x) {
-    score_select_row<T, D>(s, q, kmean, klive, seq_lens, idx, kt_in_smem, worklist ? worklist[w] : w, sm);
-    __syncthreads();  // shared memory is reused by the next row
+// ascending: the flagged blocks of [jmin, b), then the own block, then -1
+__device__ __forceinline__ void emit_row(int32_t *row, const uint8_t *taken, int jmin, int b, int topk, int lane) {
+  int pos = 0;
+  for (int base = jmin; base < b; base += 32) {
+    const int j = base + lane;
+    const bool f = j < b && taken[j];
+    const unsigned m = __ballot_sync(0xffffffffu, f);
+    if (f) row[pos + __popc(m & ((1u << lane) - 1u))] = j;
+    pos += __popc(m);
   }
+  if (lane == 0) row[pos] = b;
+  for (int i = pos + 1 + lane; i < topk; i += 32) row[i] = -1;
+}
+
+// Partial column sums of the probabilities p[a][e] of a thread's rows ty + 16 a: first over GA
+// consecutive a (rows of one query block when Bk >= 16 GA), then over the four lanes ty of the
+// warp (rows 4 warp .. 4 warp + 3 of each 16-row group), in that fixed order.  part[warp][group][64].
+template <int GA>
+__device__ __forceinline__ void row_group_sums(const float (&p)[8][8], float *part, int warp, int lane) {
+#pragma unroll
+  for (int gi = 0; gi < 8 / GA; ++gi)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      float v = p[gi * GA][e];
+#pragma unroll
+      for (int a = 1; a < GA; ++a) v += p[gi * GA + a][e];
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      if (lane < 8) part[(warp * 8 + gi) * 64 + lane + 8 * e] = v;
+    }
 }
 
 // ---- stage 1: single-precision scoring with an error bound ----------------------------------
-// grid M*B*Hkv (unit-major), 256 threads, one query block of one head group per CTA.  Logits z[t][j] of the block's
-// (up to 64) queries against 64 candidate means at a time come from a register-blocked fp32
-// product out of shared memory (thread = 4 queries x 4 candidates); softmax per query row by 4
-// lanes; column sums in fixed order; warp 0 runs the top_k - 1 arg-max passes.
+// A CTA of 128 threads takes 128 consecutive positions of one (batch, key/value head): 128 / Bk
+// query blocks.  Logits against 64 candidate means at a time come from a register-blocked fp32
+// product out of shared memory: thread (ty, tx) owns rows ty + 16 a and candidates tx + 8 e
+// (a, e < 8), so a row's 64 logits sit in the eight lanes tx = 0..7 and the softmax of a row needs
+// three shuffles.  Probabilities are summed over groups of four rows by shuffles and over a query
+// block's groups in a fixed order through shared memory.
 //
-// Error bound.  With u = 2^-24: every logit is within E = (D + 4) u scale max|q_t| max|mean_j| of
+// Error bound.  With u = 2^-24: every logit is within E = (D + 4) u scale max|q_t| max|mean_c| of
 // its exact value (D roundings of the accumulation, the rounding of the mean to fp32, the scale),
 // so every exact probability lies within a factor exp(+-2E) of the exact softmax of the computed
-// logits; evaluating that softmax and the column sum in fp32 adds 2^-21 (exp2 approximation and
-// division), 2^-22 per unit of logit range, and (b/4 + 80 + 8 chunks) u for the sums.  R is the
-// total, relative; two scores a > b are in certain order when a - b > R (a + b).
-constexpr int kFastThreads = 256;
+// logits; evaluating that softmax and the sums in fp32 adds 2^-21 (exp2 approximation and
+// division), 2^-22 per unit of logit range, and one u per addition: 16 per candidate chunk for
+// the normaliser, 2 + Bk / 4 for the column sum, one per head of the group, one per term of
+// Eq. 11, and a margin of 40.  R is the total, relative; two scores a > b are in certain order
+// when a - b > R (a + b).
+constexpr int kFastThreads = 128;
+constexpr int kRowTile = 128;  // positions per CTA
+constexpr int kChunk = 64;     // candidates per product
 
-// GROUPED: several query heads per key/value head (their number is a run-time value; the
-// one-head kernel keeps its loop-free body and its four CTAs per SM; the grouped one needs more registers).
-template <typename T, int D, bool GROUPED>
-__global__ void __launch_bounds__(kFastThreads, GROUPED ? 2 : 4) score_select_fast_kernel(
-    Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
-    const float *__restrict__ knorm, const int32_t *__restrict__ klive,
-    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
-    int32_t *__restrict__ work_count) {
-  constexpr int P = D + 4;   // row pitch of the operand tiles (floats): conflict-free 128-bit reads
-  constexpr int ZP = 68;     // row pitch of the logit tile (4 mod 32: the softmax reads hit 32 banks)
+template <typename T, int D>
+__global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
+    Shape sh, SelGeom g, const T *__restrict__ q, const float *__restrict__ mean32,
+    const float *__restrict__ norm, const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx,
+    int32_t *__restrict__ worklist, int32_t *__restrict__ work_count, int sc_pitch) {
+  constexpr int P = D + 4;  // row pitch of the operand tiles (floats): conflict-free 128-bit reads
   extern __shared__ float fsm[];
-  __shared__ float rn[64];
-  __shared__ float csum[kFastThreads];
-  __shared__ float bound_s[2];
+  __shared__ float rn[kRowTile];  // norm bound of every query row (largest over the group's heads)
+  __shared__ float bound_s[16][2];
   __shared__ int kn_bits;
-  const int M = s.M;
-  float *qs = fsm;                 // [64][P]   the block's queries
-  float *ks = qs + 64 * P;         // [64][P]   a chunk of candidate means; reused as zs [64][ZP]
-  float *zs = ks;
-  float *S = ks + 64 * (P > ZP ? P : ZP);  // [M]
-  int *live = reinterpret_cast<int *>(S + M);  // [M]
-  int *taken = live + M;                       // [M]
+  const int M = sh.M, Bk = sh.Bk;
+  const int nqb_full = kRowTile / Bk;
+  float *qs = fsm;                                      // [128][P]  the tile's queries of one head
+  float *ks = qs + kRowTile * P;                        // [64][P]   a chunk of candidate means
+  float *part = ks + kChunk * P;                        // [4 warps][8][64] sums over groups of four rows
+  float *Sc = part + 4 * 8 * 64;                        // [nqb][sc_pitch] summed probabilities per candidate
+  float *Ssel = Sc + nqb_full * sc_pitch;               // [nqb][M] selection-block scores (overlapping mode)
+  uint8_t *taken = reinterpret_cast<uint8_t *>(Ssel + (g.plain ? 0 : nqb_full * M));  // [nqb][M]
 
-  const int b = blockIdx.x % M, u = blockIdx.x / M, n = u / s.Hkv, hk = u % s.Hkv;  // u: (batch, key/value head)
+  const int ntiles = (sh.L + kRowTile - 1) / kRowTile, nU = sh.B * sh.Hkv;
+  // late tiles have the most candidates: they go first (tile-major)
+  const int tile = ntiles - 1 - (int)(blockIdx.x / nU), u = (int)(blockIdx.x % nU), n = u / sh.Hkv, hk = u % sh.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int len = seq_lens ? seq_lens[n] : s.L;
-  len = min(max(len, 0), s.L);
-  const int pad0 = s.L - len;
-  const int qlo = max(b * s.Bk, pad0), qhi = min((b + 1) * s.Bk, s.L);
-  int32_t *row = idx + ((int64_t)u * M + b) * s.topk;
-  if (qlo >= qhi) {  // the query block holds only padding
-    for (int i = tid; i < s.topk; i += kFastThreads) row[i] = -1;
-    return;
+  const int ty = tid >> 3, tx = tid & 7;
+  int len = seq_lens ? seq_lens[n] : sh.L;
+  len = min(max(len, 0), sh.L);
+  const int pad0 = sh.L - len;
+  const int row0 = tile * kRowTile;
+  const int qb0 = row0 / Bk, nqb = min(nqb_full, M - qb0);
+  const int cmin = first_live_scored(g, pad0);  // live candidates: c >= cmin
+  const int jmin = pad0 / Bk;                   // selectable selection blocks: j >= jmin
+  const int nc_max = n_candidates(sh, g, qb0 + nqb - 1);
+
+  // Does any query block of the tile have a real choice to make from non-zero scores?
+  bool need = false;
+  for (int i = 0; i < nqb; ++i) {
+    const int b = qb0 + i;
+    const bool valid = max(b * Bk, pad0) < min((b + 1) * Bk, sh.L);
+    const int nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
+    const int ncand = max(0, n_candidates(sh, g, b) - cmin);
+    need |= valid && nsel > want && want > 0 && ncand > 0;
   }
   if (tid == 0) kn_bits = 0;
-  int mine = 0;
-  for (int j = tid; j < b; j += kFastThreads) {
-    const int lv = klive[(int64_t)u * M + j] > 0;
-    live[j] = lv;
-    taken[j] = 0;
-    mine += lv;
-  }
-  int ncand = 0;
-  for (int base = 0; base < b; base += kFastThreads * 1) {  // one round unless b > 256
-    ncand += __syncthreads_count(base + tid < b && live[base + tid]);
-  }
-  (void)mine;
-  const int want = min(s.topk - 1, ncand);
-  const bool choose = ncand > want && want > 0;  // a real choice: score the candidates
-  bool certain = true;
+  rn[tid] = 0.f;
+  __syncthreads();
 
-  // The heads of the group take turns (Eq. 12): each adds its column sums to S.
-  const int G = GROUPED ? s.G : 1;
-  if (choose)
-#pragma unroll 1
-  for (int g = 0; g < G; ++g) {
-    const int h = hk * G + g;
-    // the query block, fp32, invalid rows zero
-    for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {
-      const int lt = i / (D / 4), c = (i % (D / 4)) * 4, t = b * s.Bk + lt;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (lt < s.Bk && t >= qlo && t < qhi) v = ld4(q + row_offset(s, n, h, t) + c);
-      *reinterpret_cast<float4 *>(qs + lt * P + c) = v;
-    }
-    if (g == 0) {
+  if (need) {
+    {  // the largest norm among the live candidates of the tile
       float km = 0.f;
-      for (int j = tid; j < b; j += kFastThreads)
-        if (live[j]) km = fmaxf(km, knorm[(int64_t)u * M + j]);
+      for (int c = cmin + tid; c < nc_max; c += kFastThreads) km = fmaxf(km, norm[(int64_t)u * g.n + c]);
       if (km > 0.f) atomicMax(&kn_bits, __float_as_int(km));  // positive floats order like ints
     }
-    __syncthreads();
-    if (tid < 64) {
-      float a = 0.f;
-      for (int c = 0; c < D; ++c) a = fmaf(qs[tid * P + c], qs[tid * P + c], a);
-      const float r = sqrtf(a) * 1.0001f;
-      rn[tid] = g == 0 ? r : fmaxf(rn[tid], r);  // the bound below takes the largest query of the group
+    const int ch_lo = cmin / kChunk, ch_hi = (nc_max + kChunk - 1) / kChunk;  // chunks that hold live candidates
+    const int npass = ch_hi - ch_lo > 1 ? 2 : 1;
+    // candidate limit of each of this thread's rows (the block of row ty + 16 a)
+    int nc_row[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+      const int t = row0 + ty + 16 * a;
+      nc_row[a] = (t >= pad0 && t < sh.L) ? n_candidates(sh, g, t / Bk) : 0;
     }
-    const int ty = tid >> 4, tx = tid & 15;          // product: queries ty + 16 a, candidates tx + 16 c
-    const int rt = tid >> 2, part = tid & 3;          // softmax: row rt, candidates part, part + 4, ...
-    const bool row_valid = rt < s.Bk && b * s.Bk + rt >= qlo && b * s.Bk + rt < qhi;
-    const int nchunks = (b + 63) / 64;
-    const float *kbase = kmean32 + (int64_t)u * M * D;
-    float mx = -INFINITY, den = 0.f;  // online softmax statistics of row rt (passes > 1 chunk)
+    const float *kbase = mean32 + (int64_t)u * g.n * D;
 
-    auto logits_of_chunk = [&](int j0) {  // zs[t][j] = scale <q_t, mean_{j0+j}>
-      const int nb = min(64, b - j0);
-      __syncthreads();  // previous users of ks / zs are done
-      for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {
-        const int lj = i / (D / 4), c = (i % (D / 4)) * 4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lj < nb && live[j0 + lj]) v = *reinterpret_cast<const float4 *>(kbase + (int64_t)(j0 + lj) * D + c);
-        *reinterpret_cast<float4 *>(ks + lj * P + c) = v;
-      }
-      __syncthreads();
-      float acc[4][4];
+#pragma unroll 1
+    for (int hg = 0; hg < sh.G; ++hg) {  // the heads of the group take turns (Eq. 12)
+      const int h = hk * sh.G + hg;
+      __syncthreads();  // the previous head's tiles are no longer read
+      // The tile's queries (fp32 in shared memory, invalid rows zero) and the first chunk of
+      // candidate means: every global load of the thread is in flight before the first store.
+      {
+        constexpr int CPR = D / 8, NQ = kRowTile * CPR / kFastThreads;  // 8-element chunks per row; loads per thread
+        constexpr int NK = kChunk * (D / 4) / kFastThreads;
+        Raw8<T> x[NQ];
+        float4 v[NK];
+        const int c0 = ch_lo * kChunk, nb = min(kChunk, nc_max - c0);
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[a][c] = 0.f;
-      const int ne = (nb + 15) >> 4;  // groups of 16 candidates that hold any (block-uniform)
-#pragma unroll 4
-      for (int c = 0; c < D; c += 4) {
-        float4 qa[4], kb[4];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-          qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + c);
-          if (a < ne) kb[a] = *reinterpret_cast<const float4 *>(ks + (tx + 16 * a) * P + c);
+        for (int it = 0; it < NQ; ++it) {
+          const int i = tid + it * kFastThreads, lt = i / CPR, c = (i % CPR) * 8, t = row0 + lt;
+          if (t >= pad0 && t < sh.L) x[it].load(q + row_offset(sh, n, h, t) + c);
+          else x[it].zero();
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (e < ne) {
+        for (int it = 0; it < NK; ++it) {
+          const int i = tid + it * kFastThreads, lj = i / (D / 4), c = (i % (D / 4)) * 4;
+          v[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (lj < nb && c0 + lj >= cmin) v[it] = *reinterpret_cast<const float4 *>(kbase + (int64_t)(c0 + lj) * D + c);
+        }
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
-              acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
-              acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
-              acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
-              acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
+        for (int it = 0; it < NQ; ++it) {
+          const int i = tid + it * kFastThreads, lt = i / CPR, c = (i % CPR) * 8;
+          float f[8];
+          x[it].unpack(f);
+          *reinterpret_cast<float4 *>(qs + lt * P + c) = make_float4(f[0], f[1], f[2], f[3]);
+          *reinterpret_cast<float4 *>(qs + lt * P + c + 4) = make_float4(f[4], f[5], f[6], f[7]);
+        }
+#pragma unroll
+        for (int it = 0; it < NK; ++it) {
+          const int i = tid + it * kFastThreads, lj = i / (D / 4), c = (i % (D / 4)) * 4;
+          *reinterpret_cast<float4 *>(ks + lj * P + c) = v[it];
+        }
+      }
+      __syncthreads();
+      {  // norm bound of row tid (128 rows, 128 threads)
+        float a = 0.f;
+#pragma unroll 8
+        for (int c = 0; c < D; ++c) a = fmaf(qs[tid * P + c], qs[tid * P + c], a);
+        rn[tid] = fmaxf(rn[tid], sqrtf(a) * 1.0001f);
+      }
+      float mx[8], den[8];  // online softmax statistics of this thread's rows
+#pragma unroll
+      for (int a = 0; a < 8; ++a) {
+        mx[a] = -INFINITY;
+        den[a] = 0.f;
+      }
+#pragma unroll 1
+      for (int pass = 0; pass < npass; ++pass) {
+#pragma unroll 1
+        for (int ch = ch_lo; ch < ch_hi; ++ch) {
+          const int c0 = ch * kChunk, nb = min(kChunk, nc_max - c0);
+          if (pass > 0 || ch > ch_lo) {  // (the head's first chunk is in place already)
+            constexpr int NK = kChunk * (D / 4) / kFastThreads;
+            float4 v[NK];
+            __syncthreads();  // previous users of ks and part are done
+#pragma unroll
+            for (int it = 0; it < NK; ++it) {
+              const int i = tid + it * kFastThreads, lj = i / (D / 4), c = (i % (D / 4)) * 4;
+              v[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (lj < nb && c0 + lj >= cmin) v[it] = *reinterpret_cast<const float4 *>(kbase + (int64_t)(c0 + lj) * D + c);
+            }
+#pragma unroll
+            for (int it = 0; it < NK; ++it) {
+              const int i = tid + it * kFastThreads, lj = i / (D / 4), c = (i % (D / 4)) * 4;
+              *reinterpret_cast<float4 *>(ks + lj * P + c) = v[it];
+            }
+            __syncthreads();
+          }
+          float acc[8][8];
+#pragma unroll
+          for (int a = 0; a < 8; ++a)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[a][e] = 0.f;
+          const int ne = (nb + 7) >> 3;  // groups of 8 candidates that hold any (block-uniform)
+#pragma unroll 2
+          for (int c = 0; c < D; c += 4) {
+            float4 qa[8], kb[8];
+#pragma unroll
+            for (int a = 0; a < 8; ++a) qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + c);
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if (e < ne) kb[e] = *reinterpret_cast<const float4 *>(ks + (tx + 8 * e) * P + c);
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if (e < ne) {
+#pragma unroll
+                for (int a = 0; a < 8; ++a) {
+                  acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
+                  acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
+                  acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
+                  acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
+                }
+              }
+          }
+          // logits; pairs that do not take part (dead candidates, candidates not before the row's
+          // block, invalid rows) become -inf and drop out of every sum below
+#pragma unroll
+          for (int a = 0; a < 8; ++a)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int c = c0 + tx + 8 * e;
+              acc[a][e] = (e < ne && c >= cmin && c < nc_row[a]) ? acc[a][e] * sh.scale : -INFINITY;
+            }
+          if (pass == 0) {  // fold the chunk into (mx, den) of every row
+#pragma unroll
+            for (int a = 0; a < 8; ++a) {
+              float cm = acc[a][0];
+#pragma unroll
+              for (int e = 1; e < 8; ++e) cm = fmaxf(cm, acc[a][e]);
+              cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+              cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+              cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 4));
+              const float nm = fmaxf(mx[a], cm), ref = nm > -INFINITY ? nm : 0.f;
+              float es = 0.f;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float ex = __expf(acc[a][e] - ref);  // exp(-inf) = 0
+                es += ex;
+                if (npass == 1) acc[a][e] = ex;  // one chunk: these are the numerators
+              }
+              es += __shfl_xor_sync(0xffffffffu, es, 1);
+              es += __shfl_xor_sync(0xffffffffu, es, 2);
+              es += __shfl_xor_sync(0xffffffffu, es, 4);
+              den[a] = (mx[a] > -INFINITY ? den[a] * __expf(mx[a] - nm) : 0.f) + es;
+              mx[a] = nm;
             }
           }
-      }
-      __syncthreads();  // everyone has read ks: it becomes zs
+          if (pass == npass - 1) {  // probabilities, summed over the thread's rows of one query block
+                                    // (rows 16 a + ty: Bk / 16 consecutive a) and over groups of four rows
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
+            for (int a = 0; a < 8; ++a) {
+              const float inv = den[a] > 0.f ? 1.f / den[a] : 0.f, ref = mx[a] > -INFINITY ? mx[a] : 0.f;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) zs[(ty + 16 * a) * ZP + tx + 16 * e] = s.scale * acc[a][e];
-      __syncthreads();
-    };
-    // probabilities of the chunk in place (zs[t][j] = p_t[j0 + j], 0 where there is none), then
-    // their column sums
-    auto probabilities_and_sums = [&](int j0) {
-      const int nb = min(64, b - j0);
-      const float inv = den > 0.f ? 1.f / den : 0.f;
-      for (int j = part; j < nb; j += 4) {
-        const bool on = row_valid && live[j0 + j];
-        zs[rt * ZP + j] = on ? __expf(zs[rt * ZP + j] - mx) * inv : 0.f;
-      }
-      __syncthreads();
-      {  // column sums in a fixed order: four partial sums of 16 rows each, then their tree
-        const int j = tid & 63, quarter = tid >> 6;
-        float a = 0.f;
-        if (j < nb) {
-#pragma unroll
-          for (int t = 0; t < 16; ++t) a += zs[(quarter * 16 + t) * ZP + j];
-        }
-        csum[tid] = a;
-      }
-      __syncthreads();
-      if (tid < nb) {
-        const float a = (csum[tid] + csum[64 + tid]) + (csum[128 + tid] + csum[192 + tid]);
-        S[j0 + tid] = g == 0 ? a : S[j0 + tid] + a;  // heads in ascending order
-      }
-    };
-    auto row_statistics = [&](int j0) {  // fold the chunk into (mx, den) of row rt
-      const int nb = min(64, b - j0);
-      float cm = -INFINITY;
-      for (int j = part; j < nb; j += 4)
-        if (live[j0 + j]) cm = fmaxf(cm, zs[rt * ZP + j]);
-      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
-      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
-      const float nm = fmaxf(mx, cm);
-      float e = 0.f;
-      if (nm > -INFINITY) {
-        for (int j = part; j < nb; j += 4)
-          if (live[j0 + j]) e += __expf(zs[rt * ZP + j] - nm);
-      }
-      e += __shfl_xor_sync(0xffffffffu, e, 1);
-      e += __shfl_xor_sync(0xffffffffu, e, 2);
-      den = (mx > -INFINITY ? den * __expf(mx - nm) : 0.f) + e;
-      mx = nm;
-    };
-
-    if (nchunks == 1) {
-      logits_of_chunk(0);
-      row_statistics(0);
-      probabilities_and_sums(0);
-    } else {
-      for (int ch = 0; ch < nchunks; ++ch) {
-        logits_of_chunk(ch * 64);
-        row_statistics(ch * 64);
-      }
-      for (int ch = 0; ch < nchunks; ++ch) {
-        logits_of_chunk(ch * 64);
-        probabilities_and_sums(ch * 64);
-      }
-    }
-    __syncthreads();
-  }
-
-  // Selection by rank: candidate j is kept iff fewer than `want` live candidates beat it
-  // (larger score, or equal score and lower index).  4 lanes share a candidate.
-  if (choose) {
-    for (int j0 = 0; j0 < b; j0 += kFastThreads / 4) {
-      const int j = j0 + (tid >> 2), part = tid & 3;
-      int rank = 0;
-      if (j < b && live[j]) {
-        const float sj = S[j];
-        for (int i = part; i < b; i += 4)
-          if (live[i]) {
-            const float si = S[i];
-            rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
+              for (int e = 0; e < 8; ++e) acc[a][e] = (npass == 1 ? acc[a][e] : __expf(acc[a][e] - ref)) * inv;
+            }
+            if (Bk >= 64) row_group_sums<4>(acc, part, warp, lane);
+            else if (Bk >= 32) row_group_sums<2>(acc, part, warp, lane);
+            else row_group_sums<1>(acc, part, warp, lane);
+            __syncthreads();
+            // a query block's column sums: the partial sums of its rows in a fixed order
+            const int ga = Bk >= 64 ? 4 : (Bk >= 32 ? 2 : 1);  // rows of a thread per partial sum
+            for (int o = tid; o < nqb * kChunk; o += kFastThreads) {
+              const int i = o / kChunk, col = o % kChunk;
+              if (col < nb) {
+                // block i: rows [i Bk, (i + 1) Bk) = partial sums (warp w, group gi) with 16 ga gi + 4 w inside
+                float a = 0.f;
+                for (int r4 = i * Bk / 4; r4 < (i + 1) * Bk / 4; ++r4)
+                  if ((r4 >> 2) % ga == 0) a += part[((r4 & 3) * 8 + (r4 >> 2) / ga) * 64 + col];
+                float *dst = Sc + i * sc_pitch + c0 + col;
+                *dst = hg == 0 ? a : *dst + a;  // heads in ascending order
+              }
+            }
           }
-      }
-      rank += __shfl_xor_sync(0xffffffffu, rank, 1);
-      rank += __shfl_xor_sync(0xffffffffu, rank, 2);
-      if (part == 0 && j < b && live[j]) {
-        taken[j] = rank < want;
-        if (rank == want - 1) bound_s[0] = S[j];  // the smallest kept score
-        if (rank == want) bound_s[1] = S[j];      // the largest dropped score
+        }
       }
     }
-  } else {
-    for (int j = tid; j < b; j += kFastThreads) taken[j] = want > 0 ? live[j] : 0;
   }
   __syncthreads();
 
-  if (warp == 0) {
-    if (choose) {
+  // Eq. 11, Eq. 13 and the certificate: one warp per query block
+  for (int i = warp; i < nqb; i += kFastThreads / 32) {
+    const int b = qb0 + i;
+    int32_t *row = idx + ((int64_t)u * M + b) * sh.topk;
+    if (max(b * Bk, pad0) >= min((b + 1) * Bk, sh.L)) {  // the query block holds only padding
+      for (int x = lane; x < sh.topk; x += 32) row[x] = -1;
+      continue;
+    }
+    const int nc = n_candidates(sh, g, b), ncand = max(0, nc - cmin);
+    const int nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
+    const bool choose = nsel > want && want > 0;
+    uint8_t *tk = taken + i * M;
+    bool certain = true;
+    if (!choose) {
+      for (int j = jmin + lane; j < b; j += 32) tk[j] = want > 0 ? 1 : 0;
+    } else if (ncand == 0) {  // every score is zero in any precision: the lowest blocks win the ties
+      for (int j = jmin + lane; j < b; j += 32) tk[j] = j - jmin < want ? 1 : 0;
+    } else {
+      float *S = Sc + i * sc_pitch;
+      if (!g.plain) {
+        S = Ssel + i * M;
+        map_scores<float>(g, Sc + i * sc_pitch, cmin, nc, jmin, b, S, lane);
+        __syncwarp();
+      }
+      rank_select<float>(S, jmin, b, want, tk, bound_s[i], lane);
+      __syncwarp();
       // Certain iff the gap between the last kept and the first dropped score exceeds what the
       // errors can bridge.
-      float qn = fmaxf(rn[lane], rn[lane + 32]);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, o));
-      const float kn = __int_as_float(kn_bits);
-      const float uu = 5.9604645e-8f;  // 2^-24
-      const float bound = s.scale * qn * kn;  // >= every |logit|
-      const float E = (float)(D + 4) * uu * bound * 1.01f;
-      // a sum of G non-negative head scores, each within R of its exact value, is within R of the
-      // exact sum, plus one rounding per addition
-      const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f +
-                      ((float)b * 0.25f + 80.f + 8.f * (float)((b + 63) / 64) + (float)G) * uu;
-      const float smin = bound_s[0], umax = bound_s[1];
-      certain = (smin - umax) > R * (smin + umax) * 1.001f;
-    }
-    if (certain) {
-      // emit ascending: ballot over 32-wide chunks of the flags, then the own block
-      int pos = 0;
-      for (int base = 0; base < b; base += 32) {
-        const int j = base + lane;
-        const bool f = j < b && taken[j];
-        const unsigned m = __ballot_sync(0xffffffffu, f);
-        if (f) row[pos + __popc(m & ((1u << lane) - 1u))] = j;
-        pos += __popc(m);
-      }
-      if (lane == 0) row[pos] = b;
-      for (int i = pos + 1 + lane; i < s.topk; i += 32) row[i] = -1;
-    } else if (lane == 0) {
-      worklist[atomicAdd(work_count, 1)] = blockIdx.x;  // re-scored in double precision
-    }
-  }
-}
-
-// ---- stage 1 for short sequences with small blocks ------------------------------------------
-// With blocks of 16 or 32 positions a CTA of the kernel above fills a quarter or half of its 64
-// query rows, and with few blocks per sequence its run time is all fixed cost (three rounds of
-// global loads, a dozen block-wide barriers).  This kernel takes NBLK = 64 / Bk consecutive query
-// blocks per CTA: the 64 rows are 64 consecutive positions, every row is scored against the
-// candidates of the CTA's last block in one chunk (M <= 64) and keeps those before its own block;
-// the column sums of a block are the sums of its 16-row quarters.  Same arithmetic per score and
-// the same error bound as above (with the largest query norm of the block and the largest
-// candidate norm of the CTA, both upper bounds).
-template <typename T, int D, int NBLK>
-__global__ void __launch_bounds__(kFastThreads, 4) score_select_fast_packed_kernel(
-    Shape s, const T *__restrict__ q, const float *__restrict__ kmean32,
-    const float *__restrict__ knorm, const int32_t *__restrict__ klive,
-    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, int32_t *__restrict__ worklist,
-    int32_t *__restrict__ work_count) {
-  constexpr int P = D + 4, ZP = 68, BK = 64 / NBLK, QPB = 4 / NBLK;  // quarters (16 rows) per block
-  extern __shared__ float fsm[];
-  __shared__ float rn[64];
-  __shared__ float csum[kFastThreads];
-  __shared__ float S[NBLK][64];
-  __shared__ float bound_s[NBLK][2];
-  __shared__ int live[64], taken[NBLK][64];
-  __shared__ int kn_bits;
-  const int M = s.M, MC = (M + NBLK - 1) / NBLK;
-  float *qs = fsm;          // [64][P]  the CTA's 64 query positions
-  float *ks = qs + 64 * P;  // [64][P]  the candidate means; reused as zs [64][ZP]
-  float *zs = ks;
-
-  const int c = blockIdx.x % MC, u = blockIdx.x / MC, n = u / s.H, h = u % s.H;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int len = seq_lens ? seq_lens[n] : s.L;
-  len = min(max(len, 0), s.L);
-  const int pad0 = s.L - len;
-  const int b0 = c * NBLK;                      // first query block of the CTA
-  const int nbk = min(NBLK, M - b0);            // its query blocks
-  const int bmax = b0 + nbk - 1;                // candidates of the last one: blocks 0 .. bmax - 1
-  if (tid == 0) kn_bits = 0;
-  if (tid < 64) live[tid] = (tid < bmax && klive[(int64_t)u * M + tid] > 0) ? 1 : 0;
-  __syncthreads();
-  // per block: valid, number of live candidates, how many to keep, whether that is a real choice
-  int want[NBLK];
-  bool valid[NBLK], choose[NBLK], any_choose = false;
-#pragma unroll
-  for (int i = 0; i < NBLK; ++i) {
-    const int b = b0 + i;
-    valid[i] = i < nbk && max(b * BK, pad0) < min((b + 1) * BK, s.L);
-    int nc = 0;
-    for (int j = 0; j < b && i < nbk; ++j) nc += live[j];
-    want[i] = min(s.topk - 1, nc);
-    choose[i] = valid[i] && nc > want[i] && want[i] > 0;
-    any_choose |= choose[i];
-  }
-
-  if (any_choose) {
-    for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {  // the 64 positions, fp32, invalid rows zero
-      const int lt = i / (D / 4), cc = (i % (D / 4)) * 4, t = b0 * BK + lt;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (t >= pad0 && t < s.L) v = ld4(q + row_offset(s, n, h, t) + cc);
-      *reinterpret_cast<float4 *>(qs + lt * P + cc) = v;
-    }
-    for (int i = tid; i < 64 * (D / 4); i += kFastThreads) {  // the candidate means
-      const int lj = i / (D / 4), cc = (i % (D / 4)) * 4;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (lj < bmax && live[lj])
-        v = *reinterpret_cast<const float4 *>(kmean32 + ((int64_t)u * M + lj) * D + cc);
-      *reinterpret_cast<float4 *>(ks + lj * P + cc) = v;
-    }
-    if (tid < bmax && live[tid]) {
-      const float km = knorm[(int64_t)u * M + tid];
-      if (km > 0.f) atomicMax(&kn_bits, __float_as_int(km));  // positive floats order like ints
-    }
-    __syncthreads();
-    if (tid < 64) {
-      float a = 0.f;
-      for (int cc = 0; cc < D; ++cc) a = fmaf(qs[tid * P + cc], qs[tid * P + cc], a);
-      rn[tid] = sqrtf(a) * 1.0001f;
-    }
-    const int ty = tid >> 4, tx = tid & 15;  // product: rows ty + 16 a, candidates tx + 16 e
-    const int ne = (bmax + 15) >> 4;         // groups of 16 candidates that hold any
-    float acc[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[a][e] = 0.f;
-#pragma unroll 4
-    for (int cc = 0; cc < D; cc += 4) {
-      float4 qa[4], kb[4];
-#pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + cc);
-        if (a < ne) kb[a] = *reinterpret_cast<const float4 *>(ks + (tx + 16 * a) * P + cc);
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-        if (e < ne) {
-#pragma unroll
-          for (int a = 0; a < 4; ++a) {
-            acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
-            acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
-            acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
-            acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
-          }
-        }
-    }
-    __syncthreads();  // everyone has read ks: it becomes zs
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) zs[(ty + 16 * a) * ZP + tx + 16 * e] = s.scale * acc[a][e];
-    __syncthreads();
-    {  // softmax of row rt over the live candidates before its own block, by 4 lanes, in registers
-      const int rt = tid >> 2, part = tid & 3, t = b0 * BK + rt, brow = b0 + rt / BK;
-      const bool row_valid = t >= pad0 && t < s.L;
-      float z[16], e[16];
-      unsigned lm = 0u;
-      float cm = -INFINITY;
-#pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int j = part + 4 * k;
-        const bool v = j < brow && live[j];
-        lm |= (v ? 1u : 0u) << k;
-        z[k] = v ? zs[rt * ZP + j] : -INFINITY;
-        cm = fmaxf(cm, z[k]);
-      }
-      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
-      cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
-      float sum = 0.f;
-#pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        e[k] = 0.f;
-        if (cm > -INFINITY && ((lm >> k) & 1u)) {
-          e[k] = __expf(z[k] - cm);
-          sum += e[k];
-        }
-      }
-      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-      const float inv = sum > 0.f ? 1.f / sum : 0.f;
-#pragma unroll
-      for (int k = 0; k < 16; ++k)
-        zs[rt * ZP + part + 4 * k] = (row_valid && ((lm >> k) & 1u)) ? e[k] * inv : 0.f;
-    }
-    __syncthreads();
-    {  // column sums of every 16-row quarter in a fixed order, then the blocks' sums of quarters
-      const int j = tid & 63, quarter = tid >> 6;
-      float a = 0.f;
-#pragma unroll
-      for (int t = 0; t < 16; ++t) a += zs[(quarter * 16 + t) * ZP + j];
-      csum[tid] = a;
-    }
-    __syncthreads();
-    for (int e = tid; e < NBLK * 64; e += kFastThreads) {
-      const int i = e >> 6, j = e & 63;
-      float a = csum[(i * QPB) * 64 + j];
-#pragma unroll
-      for (int qq = 1; qq < QPB; ++qq) a += csum[(i * QPB + qq) * 64 + j];
-      S[i][j] = a;
-    }
-    __syncthreads();
-  }
-
-  // Selection by rank within each block, 4 lanes per (block, candidate)
-  for (int e0 = 0; e0 < NBLK * 64; e0 += kFastThreads / 4) {
-    const int e = e0 + (tid >> 2), part = tid & 3, i = e >> 6, j = e & 63, b = b0 + i;
-    int rank = 0;
-    const bool cand = i < nbk && j < b && live[j];
-    bool ch = false;
-    int wt = 0;
-#pragma unroll
-    for (int ii = 0; ii < NBLK; ++ii)
-      if (ii == i) { ch = choose[ii]; wt = want[ii]; }
-    if (cand && ch) {
-      const float sj = S[i][j];
-      for (int x = part; x < b; x += 4)
-        if (live[x]) {
-          const float sx = S[i][x];
-          rank += (sx > sj || (sx == sj && x < j)) ? 1 : 0;
-        }
-    }
-    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
-    rank += __shfl_xor_sync(0xffffffffu, rank, 2);
-    if (part == 0 && i < nbk) {
-      if (ch) {
-        if (cand) {
-          taken[i][j] = rank < wt;
-          if (rank == wt - 1) bound_s[i][0] = S[i][j];  // the smallest kept score
-          if (rank == wt) bound_s[i][1] = S[i][j];      // the largest dropped score
-        } else {
-          taken[i][j] = 0;
-        }
-      } else {
-        taken[i][j] = (wt > 0 && cand) ? 1 : 0;
-      }
-    }
-  }
-  __syncthreads();
-
-  if (warp < nbk) {  // warp i finishes block b0 + i
-    const int i = warp, b = b0 + i;
-    bool ch = false, vd = false;
-#pragma unroll
-    for (int ii = 0; ii < NBLK; ++ii)
-      if (ii == i) { ch = choose[ii]; vd = valid[ii]; }
-    int32_t *row = idx + ((int64_t)u * M + b) * s.topk;
-    if (!vd) {  // the query block holds only padding
-      for (int x = lane; x < s.topk; x += 32) row[x] = -1;
-      return;
-    }
-    bool certain = true;
-    if (ch) {
       float qn = 0.f;
-      for (int x = lane; x < BK; x += 32) qn = fmaxf(qn, rn[i * BK + x]);
+      for (int x = lane; x < Bk; x += 32) qn = fmaxf(qn, rn[i * Bk + x]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, o));
       const float kn = __int_as_float(kn_bits);
-      const float uu = 5.9604645e-8f;  // 2^-24
-      const float bound = s.scale * qn * kn;  // >= every |logit|
+      const float uu = 5.9604645e-8f;          // 2^-24
+      const float bound = sh.scale * qn * kn;  // >= every |logit|
       const float E = (float)(D + 4) * uu * bound * 1.01f;
-      const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f + ((float)b * 0.25f + 80.f + 8.f + 1.f) * uu;
+      const float nchunks = (float)((nc + kChunk - 1) / kChunk);
+      const float R = 2.f * E + 4.77e-7f + 2.f * bound * 2.39e-7f +
+                      (16.f * nchunks + (float)(Bk / 4) + 2.f + (float)sh.G + (float)(g.rs * g.rl) + 40.f) * uu;
       const float smin = bound_s[i][0], umax = bound_s[i][1];
       certain = (smin - umax) > R * (smin + umax) * 1.001f;
     }
-    if (certain) {
-      int pos = 0;
-      for (int base = 0; base < b; base += 32) {
-        const int j = base + lane;
-        const bool f = j < b && taken[i][j];
-        const unsigned mm = __ballot_sync(0xffffffffu, f);
-        if (f) row[pos + __popc(mm & ((1u << lane) - 1u))] = j;
-        pos += __popc(mm);
+    __syncwarp();
+    if (certain) emit_row(row, tk, jmin, b, sh.topk, lane);
+    else if (lane == 0) worklist[atomicAdd(work_count, 1)] = u * M + b;  // re-scored in double precision
+  }
+}
+
+// ---- stage 2: the same scores in double precision ------------------------------------------
+// One CTA of 256 threads per query block of the work list (every query block when worklist ==
+// nullptr).  64 query rows at a time (the block's queries of the group's heads, head-major)
+// against 64 candidate means at a time: thread (row tid / 4, part tid % 4) forms the 16 logits of
+// candidates part + 4 k, so sixteen independent accumulation chains are in flight; softmax per row
+// by 4 lanes; the probabilities go through a shared tile for the column sums (fixed order).
+template <typename T, int D>
+__global__ void __launch_bounds__(256) score_exact_kernel(
+    Shape sh, SelGeom g, const T *__restrict__ q, const double *__restrict__ mean,
+    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, const int32_t *__restrict__ worklist,
+    const int32_t *__restrict__ work_count, int sc_len) {
+  constexpr int PD = D + 1;
+  extern __shared__ double dsm[];
+  __shared__ double bound_d[2];
+  double *qd = dsm;             // [64][PD] query rows
+  double *kd = qd + 64 * PD;    // [64] candidate means (pitch PD), then the probability tile (pitch 65)
+  double *csum = kd + 64 * 65;  // [256]
+  double *Sc = csum + 256;      // [sc_len] summed probabilities per candidate
+  double *S = Sc + sc_len;      // [M] scores of the selection blocks
+  uint8_t *taken = reinterpret_cast<uint8_t *>(S + sh.M);  // [M]
+
+  const int M = sh.M, Bk = sh.Bk;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rt = tid >> 2, part = tid & 3;
+  const int total = worklist ? *work_count : M * sh.B * sh.Hkv;
+  for (int wi = blockIdx.x; wi < total; wi += gridDim.x) {
+    const int row_id = worklist ? worklist[wi] : wi;
+    const int b = row_id % M, u = row_id / M, n = u / sh.Hkv, hk = u % sh.Hkv;
+    int len = seq_lens ? seq_lens[n] : sh.L;
+    len = min(max(len, 0), sh.L);
+    const int pad0 = sh.L - len;
+    const int qlo = max(b * Bk, pad0), qhi = min((b + 1) * Bk, sh.L);
+    int32_t *row = idx + ((int64_t)u * M + b) * sh.topk;
+    __syncthreads();  // shared memory is reused from the previous query block
+    if (qlo >= qhi) {  // the query block holds only padding
+      for (int i = tid; i < sh.topk; i += 256) row[i] = -1;
+      continue;
+    }
+    const int cmin = first_live_scored(g, pad0), jmin = pad0 / Bk;
+    const int nc = n_candidates(sh, g, b), ncand = max(0, nc - cmin);
+    const int nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
+    const bool choose = nsel > want && want > 0;
+
+    if (choose && ncand > 0) {
+      for (int c = cmin + tid; c < nc; c += 256) Sc[c] = 0.0;
+      const int nq = qhi - qlo, nrows = nq * sh.G;  // rows: head r / nq of the group, query qlo + r % nq
+      const int ch_lo = cmin / 64, ch_hi = (nc + 63) / 64;
+      const int npass = ch_hi - ch_lo > 1 ? 2 : 1;
+      const double *kbase = mean + (int64_t)u * g.n * D;
+      for (int r0 = 0; r0 < nrows; r0 += 64) {
+        const int nr = min(64, nrows - r0);
+        __syncthreads();
+        for (int i = tid; i < 64 * (D / 4); i += 256) {  // 64 query rows as doubles, missing rows zero
+          const int lr = i / (D / 4), c = (i % (D / 4)) * 4;
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (lr < nr) {
+            const int r = r0 + lr;
+            v = ld4(q + row_offset(sh, n, hk * sh.G + r / nq, qlo + r % nq) + c);
+          }
+          double *d = qd + lr * PD + c;
+          d[0] = (double)v.x; d[1] = (double)v.y; d[2] = (double)v.z; d[3] = (double)v.w;
+        }
+        const bool row_on = rt < nr;
+        double mx = -INFINITY, den = 0.0;
+        for (int pass = 0; pass < npass; ++pass) {
+          for (int ch = ch_lo; ch < ch_hi; ++ch) {
+            const int c0 = ch * 64, nb = min(64, nc - c0);
+            __syncthreads();  // previous users of kd are done
+            for (int i = tid; i < 64 * (D / 2); i += 256) {
+              const int lj = i / (D / 2), c = (i % (D / 2)) * 2;
+              double2 v = make_double2(0.0, 0.0);
+              if (lj < nb && c0 + lj >= cmin) v = *reinterpret_cast<const double2 *>(kbase + (int64_t)(c0 + lj) * D + c);
+              kd[lj * PD + c] = v.x;
+              kd[lj * PD + c + 1] = v.y;
+            }
+            __syncthreads();
+            double z[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) z[k] = 0.0;
+            const double *qr = qd + rt * PD;
+#pragma unroll 2
+            for (int c = 0; c < D; ++c) {
+              const double qv = qr[c];
+#pragma unroll
+              for (int k = 0; k < 16; ++k) z[k] = fma(qv, kd[(part + 4 * k) * PD + c], z[k]);
+            }
+            uint32_t on = 0u;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+              z[k] *= sh.scale_d;
+              if (row_on && part + 4 * k < nb && c0 + part + 4 * k >= cmin) on |= 1u << k;
+            }
+            if (pass == 0) {
+              double cm = -INFINITY;
+#pragma unroll
+              for (int k = 0; k < 16; ++k)
+                if ((on >> k) & 1u) cm = fmax(cm, z[k]);
+              cm = fmax(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+              cm = fmax(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+              const double nm = fmax(mx, cm);
+              double es = 0.0;
+              if (nm > -INFINITY) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k)
+                  if ((on >> k) & 1u) es += exp(z[k] - nm);
+              }
+              es += __shfl_xor_sync(0xffffffffu, es, 1);
+              es += __shfl_xor_sync(0xffffffffu, es, 2);
+              den = (mx > -INFINITY ? den * exp(mx - nm) : 0.0) + es;
+              mx = nm;
+            }
+            if (pass == npass - 1) {
+              __syncthreads();  // everyone has read kd: it becomes the probability tile
+#pragma unroll
+              for (int k = 0; k < 16; ++k)
+                kd[rt * 65 + part + 4 * k] = ((on >> k) & 1u) ? exp(z[k] - mx) / den : 0.0;
+              __syncthreads();
+              {  // column sums in a fixed order: four partial sums of 16 rows, then their tree
+                const int j = tid & 63, quarter = tid >> 6;
+                double a = 0.0;
+#pragma unroll
+                for (int t = 0; t < 16; ++t) a += kd[(quarter * 16 + t) * 65 + j];
+                csum[tid] = a;
+              }
+              __syncthreads();
+              if (tid < nb) Sc[c0 + tid] += (csum[tid] + csum[64 + tid]) + (csum[128 + tid] + csum[192 + tid]);
+            }
+          }
+        }
       }
-      if (lane == 0) row[pos] = b;
-      for (int x = pos + 1 + lane; x < s.topk; x += 32) row[x] = -1;
-    } else if (lane == 0) {
-      worklist[atomicAdd(work_count, 1)] = u * M + b;  // re-scored in double precision
+    }
+    __syncthreads();
+    if (warp == 0) {
+      if (!choose) {
+        for (int j = jmin + lane; j < b; j += 32) taken[j] = want > 0 ? 1 : 0;
+      } else if (ncand == 0) {
+        for (int j = jmin + lane; j < b; j += 32) taken[j] = j - jmin < want ? 1 : 0;
+      } else {
+        map_scores<double>(g, Sc, cmin, nc, jmin, b, S, lane);
+        __syncwarp();
+        rank_select<double>(S, jmin, b, want, taken, bound_d, lane);
+      }
+      __syncwarp();
+      emit_row(row, taken, jmin, b, sh.topk, lane);
     }
   }
 }
 
-size_t select_fast_smem_bytes(int M, int D) {
-  const int P = D + 4, ZP = 68;
-  return (size_t)(64 * P + 64 * (P > ZP ? P : ZP)) * sizeof(float) + (size_t)M * (sizeof(float) + 2 * sizeof(int));
-}
+// The arrays the selection kernels work in (the caller's workspace or the built-in scratch).
+struct SelBuffers {
+  double *mean;
+  int32_t *live;
+  float *mean32, *norm;
+  int32_t *list, *count;
+};
 
-size_t select_smem_bytes(int M, int D, bool kt_in_smem) {
-  size_t dbl = (size_t)kSelWarps * M * 2 + (size_t)kSelWarps * D + M;
-  size_t ints = 2 * (size_t)M;
-  size_t kt = kt_in_smem ? (size_t)M * (D + 1) : 0;
-  return (dbl + kt) * sizeof(double) + ints * sizeof(int);
+// Dynamic shared memory of the two scoring kernels; 0 = the single-precision stage does not take
+// this shape (more score slots per CTA than it keeps) and every query block goes to stage 2.
+size_t fast_smem_bytes(const Shape &sh, const SelGeom &g, int D, int *sc_pitch) {
+  const int nqb = kRowTile / sh.Bk;
+  *sc_pitch = ((g.n + kChunk - 1) / kChunk) * kChunk;
+  const size_t slots = (size_t)nqb * *sc_pitch + (g.plain ? 0 : (size_t)nqb * sh.M);
+  if (slots > 20480) return 0;
+  return ((size_t)(kRowTile + kChunk) * (D + 4) + 4 * 8 * 64 + slots) * sizeof(float) + (size_t)nqb * sh.M + 16;
+}
+size_t exact_smem_bytes(const Shape &sh, const SelGeom &g, int D, int *sc_len) {
+  *sc_len = ((g.n + 63) / 64) * 64;
+  return ((size_t)64 * (D + 1) + 64 * 65 + 256 + *sc_len + sh.M) * sizeof(double) + (size_t)sh.M + 16;
 }
 
 template <typename T, int D>
-int launch_select_t(const Shape &s, const T *q, const T *k, const int32_t *seq_lens, int32_t *idx,
-                    const Workspace &ws, cudaStream_t st) {
-  // block = (unit, query block), unit-major; a unit is a (batch, key/value head) pair
-  const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.Hkv);
-  {
+int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_lens, int32_t *idx,
+                    const SelBuffers &w, cudaStream_t st) {
+  const SelGeom g = sel_geom(sh);
+  const int64_t units = (int64_t)sh.B * sh.Hkv;
+  if (g.n > 0) {
     LaunchScope ls(K_SUMMARY, st);
-    summary_kernel<T, D><<<grid, 256, 0, st>>>(s, k, seq_lens, ws.kmean, ws.klive, ws.kmean32, ws.knorm,
-                                               ws.sel_count);
+    summary_kernel<T, D><<<(unsigned)((units * g.n + 7) / 8), 256, 0, st>>>(sh, g, k, seq_lens, w.mean, w.live,
+                                                                            w.mean32, w.norm, w.count);
+  } else if (cudaMemsetAsync(w.count, 0, sizeof(int32_t), st) != cudaSuccess) {
+    return BLOSSOM_ERR_CUDA;
   }
-  const bool exact_only = exact_select_only();
+  int sc_pitch = 0, sc_len = 0;
+  const size_t fsm = fast_smem_bytes(sh, g, D, &sc_pitch);
+  const bool exact_only = exact_select_only() || fsm == 0;
   if (!exact_only) {
-    if (s.G == 1 && s.M <= 64 && (s.Bk == 16 || s.Bk == 32)) {
-      // short sequences of small blocks: 64 / Bk query blocks per CTA
-      const int nblk = 64 / s.Bk;
-      const size_t psm = (size_t)(64 * (D + 4) + 64 * 68) * sizeof(float);
-      auto packed = nblk == 2 ? score_select_fast_packed_kernel<T, D, 2> : score_select_fast_packed_kernel<T, D, 4>;
-      const unsigned gpk = (unsigned)((s.M + nblk - 1) / nblk) * (unsigned)(s.B * s.Hkv);
-      LaunchScope ls(K_SCORE_FAST, st);
-      packed<<<gpk, kFastThreads, psm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive, seq_lens, idx, ws.sel_list,
-                                             ws.sel_count);
-    } else {
-    const size_t fsm = select_fast_smem_bytes(s.M, D);
-    auto fast = s.G > 1 ? score_select_fast_kernel<T, D, true> : score_select_fast_kernel<T, D, false>;
-    if (fsm > 48 * 1024 &&
-        cudaFuncSetAttribute(fast, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm) != cudaSuccess)
+    if (fsm > 48 * 1024 && cudaFuncSetAttribute(score_fast_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)fsm) != cudaSuccess)
       return BLOSSOM_ERR_CUDA;
+    const unsigned ntiles = (unsigned)((sh.L + kRowTile - 1) / kRowTile);
     LaunchScope ls(K_SCORE_FAST, st);
-    fast<<<grid, kFastThreads, fsm, st>>>(s, q, ws.kmean32, ws.knorm, ws.klive, seq_lens, idx, ws.sel_list,
-                                          ws.sel_count);
-    }
+    score_fast_kernel<T, D><<<ntiles * (unsigned)units, kFastThreads, fsm, st>>>(
+        sh, g, q, w.mean32, w.norm, seq_lens, idx, w.list, w.count, sc_pitch);
   }
-  bool in_smem = select_smem_bytes(s.M, D, true) <= 160 * 1024;
-  size_t smem = select_smem_bytes(s.M, D, in_smem);
-  if (smem > 48 * 1024) {
-    if (cudaFuncSetAttribute(score_select_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess)
-      return BLOSSOM_ERR_CUDA;
-  }
+  const size_t esm = exact_smem_bytes(sh, g, D, &sc_len);
+  if (esm > 48 * 1024 && cudaFuncSetAttribute(score_exact_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)esm) != cudaSuccess)
+    return BLOSSOM_ERR_CUDA;
   {
     // double precision: every query block (exact_only) or the work list of the kernel above
     LaunchScope ls(K_SCORE_SELECT, st);
-    const unsigned g2 = exact_only ? grid : (grid < 592u ? grid : 592u);
-    score_select_kernel<T, D><<<g2, kSelThreads, smem, st>>>(s, q, ws.kmean, ws.klive, seq_lens, idx,
-                                                            in_smem ? 1 : 0, exact_only ? nullptr : ws.sel_list,
-                                                            ws.sel_count);
+    const int64_t rows = units * sh.M;
+    const unsigned g2 = (unsigned)(rows < 592 ? rows : 592);
+    score_exact_kernel<T, D><<<g2, 256, esm, st>>>(sh, g, q, w.mean, seq_lens, idx, exact_only ? nullptr : w.list,
+                                                   w.count, sc_len);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
+int launch_select_buffers(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
+                          int32_t *idx, const SelBuffers &w, cudaStream_t st) {
+  typedef __nv_bfloat16 bf;
+  if (dtype == BLOSSOM_DTYPE_FP32) {
+    if (s.D == 32) return launch_select_t<float, 32>(s, (const float *)q, (const float *)k, seq_lens, idx, w, st);
+    return launch_select_t<float, 64>(s, (const float *)q, (const float *)k, seq_lens, idx, w, st);
+  }
+  if (s.D == 32) return launch_select_t<bf, 32>(s, (const bf *)q, (const bf *)k, seq_lens, idx, w, st);
+  return launch_select_t<bf, 64>(s, (const bf *)q, (const bf *)k, seq_lens, idx, w, st);
 }
 
 }  // namespace
 
 int launch_select(const Shape &s, int dtype, const void *q, const void *k, const int32_t *seq_lens,
                   int32_t *idx, const Workspace &ws, cudaStream_t st) {
-  if (s.cmp_l > 0) return launch_select_cmp(s, dtype, q, k, seq_lens, idx, ws, st);  // Eq. 8-11
-  if (dtype == BLOSSOM_DTYPE_FP32) {
-    if (s.D == 32) return launch_select_t<float, 32>(s, (const float *)q, (const float *)k, seq_lens, idx, ws, st);
-    return launch_select_t<float, 64>(s, (const float *)q, (const float *)k, seq_lens, idx, ws, st);
+  SelBuffers w;
+  if (s.cmp_l > 0) {  // the means of the overlapping compression blocks have arrays of their own
+    w.mean = ws.cmean; w.live = ws.clive; w.mean32 = ws.cmean32; w.norm = ws.cnorm;
+  } else {
+    w.mean = ws.kmean; w.live = ws.klive; w.mean32 = ws.kmean32; w.norm = ws.knorm;
   }
-  if (s.D == 32)
-    return launch_select_t<__nv_bfloat16, 32>(s, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, seq_lens, idx, ws, st);
-  return launch_select_t<__nv_bfloat16, 64>(s, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, seq_lens, idx, ws, st);
+  w.list = ws.sel_list;
+  w.count = ws.sel_count;
+  return launch_select_buffers(s, dtype, q, k, seq_lens, idx, w, st);
 }
 
 // ---- selection with built-in scratch (no allocation anywhere on the call path) -------------
@@ -815,8 +769,8 @@ int launch_select(const Shape &s, int dtype, const void *q, const void *k, const
 // live here in one array that is part of the loaded module.  Every launch overwrites each entry
 // it later reads, so nothing has to start at zero and stale contents of earlier calls are
 // harmless; two calls in flight at once on one device would overwrite each other's means.
-constexpr size_t kStaticMeanElems = 524288;  // doubles: batch * heads * M * head_dim may not exceed this
-constexpr size_t kStaticBlocks = 8192;       // int32:   batch * heads * M may not exceed this
+constexpr size_t kStaticMeanElems = 524288;  // doubles: batch * kv_heads * M * head_dim may not exceed this
+constexpr size_t kStaticBlocks = 8192;       // int32:   batch * kv_heads * M may not exceed this
 // doubles (means) | floats (fp32 means) | int32 live counts | float norms | int32 work list | counter
 constexpr size_t kStaticOffMean32 = kStaticMeanElems * sizeof(double);
 constexpr size_t kStaticOffLive = kStaticOffMean32 + kStaticMeanElems * sizeof(float);
@@ -846,14 +800,14 @@ int launch_select_static(const Shape &s, int dtype, const void *q, const void *k
     g_scratch_addr[dev] = p;
   }
   unsigned char *base = static_cast<unsigned char *>(g_scratch_addr[dev]);
-  Workspace ws = {};
-  ws.kmean = reinterpret_cast<double *>(base);
-  ws.kmean32 = reinterpret_cast<float *>(base + kStaticOffMean32);
-  ws.klive = reinterpret_cast<int32_t *>(base + kStaticOffLive);
-  ws.knorm = reinterpret_cast<float *>(base + kStaticOffNorm);
-  ws.sel_list = reinterpret_cast<int32_t *>(base + kStaticOffList);
-  ws.sel_count = reinterpret_cast<int32_t *>(base + kStaticOffCount);
-  return launch_select(s, dtype, q, k, seq_lens, idx, ws, st);
+  SelBuffers w;
+  w.mean = reinterpret_cast<double *>(base);
+  w.mean32 = reinterpret_cast<float *>(base + kStaticOffMean32);
+  w.live = reinterpret_cast<int32_t *>(base + kStaticOffLive);
+  w.norm = reinterpret_cast<float *>(base + kStaticOffNorm);
+  w.list = reinterpret_cast<int32_t *>(base + kStaticOffList);
+  w.count = reinterpret_cast<int32_t *>(base + kStaticOffCount);
+  return launch_select_buffers(s, dtype, q, k, seq_lens, idx, w, st);
 }
 
 }  // namespace blossom
