@@ -207,11 +207,13 @@ def time_oracle(ws):
     import oracle
     t0 = time.perf_counter()
     idx = None
-    if ws.cmp_block or ws.cmp_stride:   # selection through overlapping compression blocks (Eq. 8-11)
+    grouped = bool(ws.kv_heads) and ws.kv_heads != ws.H
+    if (ws.cmp_block or ws.cmp_stride) and not grouped:   # selection through overlapping compression blocks (Eq. 8-11)
         idx = oracle.select_blocks_cmp(ws.q, ws.k, ws.block, ws.topk, ws.cmp_block or ws.block,
                                        ws.cmp_stride or ws.block, ws.seq_lens)
-    if ws.kv_heads and ws.kv_heads != ws.H:   # grouped key/value heads: one selection per group (Eq. 12)
+    if grouped:   # grouped key/value heads: one selection per group (Eq. 12)
         f = oracle.forward_gqa(ws.q, ws.k, ws.v, ws.gate, ws.block, ws.topk, ws.window, ws.seq_lens,
+                               cmp_block=ws.cmp_block, cmp_stride=ws.cmp_stride,
                                stis_mode=ws.stis_mode, stis_block=ws.stis_block)
         oracle.backward_gqa(ws.q, ws.k, ws.v, ws.gate, ws.block, ws.topk, ws.window, f, ws.dout,
                             ws.seq_lens, stis_mode=ws.stis_mode, stis_block=ws.stis_block)
@@ -281,6 +283,9 @@ def main():
     ap.add_argument("--cmp-stride", type=int, default=0, help="their stride s")
     ap.add_argument("--kv-heads", type=int, default=0,
                     help="key/value heads shared by groups of query heads (0: one per query head)")
+    ap.add_argument("--paper-options", action="store_true",
+                    help="the paper's options together on the chosen shape: heads on 2 key/value heads, "
+                         "compression blocks of 2 x block at stride block / 2, power-law mask (window 8, block 1)")
     ap.add_argument("--no-secondary", action="store_true",
                     help="skip the L = 1024 case that the default run times beside the headline")
     ap.add_argument("--batch", type=int, default=0,
@@ -299,7 +304,12 @@ def main():
         kw["B"] = args.batch
     if args.kv_heads and args.config != 1:
         kw["kv_heads"] = args.kv_heads
+    if args.paper_options and args.config != 1:
+        kw["kv_heads"] = args.kv_heads or 2
+        args.short_term = "power-law"
     w = workloads.CONFIGS[args.config](**kw)
+    if args.paper_options and args.config != 1:
+        args.cmp_block, args.cmp_stride = args.cmp_block or 2 * w.block, args.cmp_stride or w.block // 2
     if w.kv_heads:
         w.name += f"+kv_heads{w.kv_heads}"
     if args.short_term == "power-law":

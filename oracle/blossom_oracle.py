@@ -214,15 +214,24 @@ def _group(H, Hkv):
     return H // Hkv
 
 
-def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False):
-    """q ``[B,H,L,D]``, k ``[B,Hkv,L,D]`` -> idx ``[B,Hkv,M,topk]`` from group-summed scores."""
+def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False,
+                      cmp_block=0, cmp_stride=0):
+    """q ``[B,H,L,D]``, k ``[B,Hkv,L,D]`` -> idx ``[B,Hkv,M,topk]`` from group-summed scores.
+
+    With ``cmp_block`` / ``cmp_stride`` the per-head scores are those of the overlapping
+    compression blocks mapped onto the selection blocks (Eq. 8-11); they are then summed over the
+    heads of the group (Eq. 12) and the top-k is taken (Eq. 13): the paper's full selection."""
     q, k = _f64(q), _f64(k)
     B, H, L, D = q.shape
     Hkv = k.shape[1]
     G = _group(H, Hkv)
     M = -(-L // block)
-    _, per_head = select_blocks(q, np.repeat(k, G, axis=1), block, topk, seq_lens, sm_scale,
-                                return_scores=True)
+    if cmp_block or cmp_stride:
+        _, per_head, _ = select_blocks_cmp(q, np.repeat(k, G, axis=1), block, topk, cmp_block or block,
+                                           cmp_stride or block, seq_lens, sm_scale, return_scores=True)
+    else:
+        _, per_head = select_blocks(q, np.repeat(k, G, axis=1), block, topk, seq_lens, sm_scale,
+                                    return_scores=True)
     scores = per_head.reshape(B, Hkv, G, M, M).sum(axis=2)            # Eq. 12
     idx = np.full((B, Hkv, M, topk), -1, dtype=np.int32)
     for n in range(B):
@@ -240,12 +249,14 @@ def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_sc
     return (idx, scores) if return_scores else idx
 
 
-def forward_gqa(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None, **kw):
+def forward_gqa(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None,
+                cmp_block=0, cmp_stride=0, **kw):
     """``forward`` for q ``[B,H,L,D]`` and k, v ``[B,Hkv,L,D]``; idx is ``[B,Hkv,M,topk]``."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     G = _group(q.shape[1], k.shape[1])
     if idx is None:
-        idx = select_blocks_gqa(q, k, block, topk, seq_lens, sm_scale)
+        idx = select_blocks_gqa(q, k, block, topk, seq_lens, sm_scale, cmp_block=cmp_block,
+                                cmp_stride=cmp_stride)
     idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
     f = forward(q, np.repeat(k, G, axis=1), np.repeat(v, G, axis=1), gate, block, topk, window,
                 seq_lens, sm_scale, idx=np.repeat(idx, G, axis=1), **kw)

@@ -31,7 +31,8 @@ def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
     if _grouped(w):
         ref_idx, scores = oracle.select_blocks_gqa(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
-                                                   return_scores=True)
+                                                   return_scores=True, cmp_block=w.cmp_block,
+                                                   cmp_stride=w.cmp_stride)
     elif w.cmp_block or w.cmp_stride:
         ref_idx, scores, _ = oracle.select_blocks_cmp(w.q, w.k, w.block, w.topk, w.cmp_block or w.block,
                                                       w.cmp_stride or w.block, w.seq_lens, sm_scale,

@@ -169,6 +169,21 @@ def test_grouped_query_heads(runner, dtype, L, D, H, Hkv, block, topk, window, l
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.parametrize("dtype,D", [("fp32", 32), ("bf16", 32), ("bf16", 64)])
+def test_paper_default_configuration_in_one_call(runner, dtype, D):
+    """The configuration the paper evaluates, all in one call: 8 query heads on 2 key/value heads
+    with one selection per group (Eq. 12), compression blocks of 32 at stride 16 scored and mapped
+    onto selection blocks of 16 (Eq. 8-11), top-4, and the power-law short-term mask with window 8
+    and mask block 1 (Eq. 15), at the paper's sequence length 200 with left padding."""
+    w = workloads.make("paper-default", dtype, 5, 8, 200, D, 16, 4, 8, seed=29, std=0.7, kv_heads=2,
+                       stis_mode=1, stis_block=1)
+    w.cmp_block, w.cmp_stride = 32, 16
+    w.seq_lens = np.asarray([200, 131, 33, 16, 0], dtype=np.int32)
+    _, res = run(runner, w)
+    assert res["idx"].shape == (5, 2, 13, 4) and res["dk"].shape == (5, 2, 200, D)
+    print(check_forward_backward(w, res))
+
+
 def test_explicit_scale_and_given_indices(runner):
     w = workloads.make("scale", "fp32", 2, 2, 96, 32, 16, 3, 20, seed=5)
     p, res = run(runner, w, sm_scale=0.37)
@@ -342,6 +357,17 @@ def test_config4_full_size_power_law(runner):
     print(errs)
 
 
+def test_config4_full_size_paper_options_together(runner):
+    """The headline shape with the paper's three options at once (8 heads on 2 key/value heads,
+    overlapping compression blocks 128 / 32 behind the 64-position selection blocks, power-law
+    mask with window 8 and mask block 1), as the benchmark's --paper-options times it."""
+    w = workloads.config4(kv_heads=2)
+    w.cmp_block, w.cmp_stride = 128, 32
+    w.stis_mode, w.stis_block, w.window = 1, 1, 8
+    errs, _ = _whole_batch(runner, w)
+    print(errs)
+
+
 def test_config2_full_size(runner):
     w = workloads.config2()
     errs, res = _whole_batch(runner, w)
@@ -388,7 +414,11 @@ def test_certified_selection_equals_double_precision_selection(runner):
     overlap2.cmp_block, overlap2.cmp_stride = 32, 16           # the paper's default sizes, padded rows
     small_stride = workloads.make("small-stride", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9)
     small_stride.cmp_block, small_stride.cmp_stride = 32, 8    # 253 compression blocks: four chunks
-    for w in (workloads.config4(B=1), workloads.config2(B=16), workloads.config3(B=1),
+    gqa_overlap = workloads.config2(B=16, kv_heads=1)
+    gqa_overlap.cmp_block, gqa_overlap.cmp_stride = 32, 16     # grouped heads through overlapping blocks
+    gqa_overlap4 = workloads.config4(B=1, kv_heads=2)
+    gqa_overlap4.cmp_block, gqa_overlap4.cmp_stride = 128, 32
+    for w in (workloads.config4(B=1), workloads.config2(B=16), workloads.config3(B=1), gqa_overlap, gqa_overlap4,
               workloads.config4(B=1, kv_heads=2), workloads.config2(B=16, kv_heads=1),
               workloads.config3(B=1, kv_heads=1),
               workloads.make("many-blocks", "bf16", 1, 2, 2048, 32, 16, 6, 16, seed=9),

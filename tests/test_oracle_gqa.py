@@ -85,6 +85,39 @@ def test_key_and_value_gradients_by_central_differences(lens):
     assert b["dk"].shape == k.shape and b["dq"].shape == q.shape
 
 
+def test_grouped_selection_through_overlapping_blocks():
+    """The paper's full selection (Eq. 8-13: overlapping compression blocks, score remap, scores
+    summed over the group's heads): one head per group is the single-head function bit for bit;
+    the group scores are the sum of an independent numpy scorer's per-head scores (Eq. 11 as a
+    convolution); the chosen set is the stable arg-sort of those sums."""
+    from test_oracle_overlap import numpy_scores
+    q, k, v, gate, dout, sl = rand_case(6, B=2, H=3, Hkv=3, L=96, D=8, lens=[96, 41])
+    idx, sc = oracle.select_blocks_gqa(q, k, 16, 3, sl, return_scores=True, cmp_block=32, cmp_stride=16)
+    idx0, sc0, _ = oracle.select_blocks_cmp(q, k, 16, 3, 32, 16, sl, return_scores=True)
+    np.testing.assert_array_equal(idx, idx0)
+    np.testing.assert_array_equal(sc, sc0)
+
+    q, k, v, gate, dout, sl = rand_case(7, B=2, H=4, Hkv=2, L=96, D=8, lens=[96, 50])
+    lp, l, s, topk, scale = 16, 32, 16, 3, 1.0 / math.sqrt(8)
+    idx, sc = oracle.select_blocks_gqa(q, k, lp, topk, sl, return_scores=True, cmp_block=l, cmp_stride=s)
+    M = 6
+    for n in range(2):
+        pad0 = 96 - int(sl[n])
+        for g in range(2):
+            tot = np.zeros((M, M))
+            for h in (2 * g, 2 * g + 1):
+                tot += numpy_scores(q[n, h], k[n, g], lp, l, s, pad0, scale)[1]
+            np.testing.assert_allclose(sc[n, g], tot, atol=1e-12)
+            for b in range(M):
+                if min((b + 1) * lp, 96) <= max(b * lp, pad0):
+                    assert list(idx[n, g, b]) == [-1] * topk
+                    continue
+                cand = [j for j in range(b) if (j + 1) * lp > pad0]
+                order = sorted(cand, key=lambda j: (-tot[b, j], j))[:topk - 1]
+                row = sorted(order) + [b]
+                assert list(idx[n, g, b][:len(row)]) == row and all(x == -1 for x in idx[n, g, b][len(row):])
+
+
 def test_heads_must_divide():
     q, k, v, gate, dout, sl = rand_case(5, H=3, Hkv=2)
     with pytest.raises(ValueError):
