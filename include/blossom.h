@@ -193,6 +193,15 @@ int blossom_attn_bwd(const blossom_params *params /* host */, const void *q, con
  * Returns BLOSSOM_ERR_CUDA if the synchronise or the copy fails. */
 int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out);
 
+/* Diagnostic (no counterpart in the paper): shows that a device-side wait that cannot complete
+ * ends in a report, not in a hang.  Launches one tiny kernel on `stream` that sets up tensor
+ * memory and an mbarrier like the attention kernels and then waits for an arrival nobody makes:
+ * the wait gives up after the library's limit (about 0.2 s of GPU time), the kernel runs to its
+ * normal end, frees its tensor memory and records BLOSSOM_ERR_TIMEOUT in the status words at the
+ * start of `workspace` (>= 256 bytes, 256-byte aligned), where blossom_device_status finds it.
+ * The context stays usable.  Returns BLOSSOM_OK if the kernel was launched. */
+int blossom_selftest_wait_timeout(void *workspace, size_t workspace_bytes, blossom_stream_t stream);
+
 /* Debugging switches (no counterpart in the paper), process-wide, host only, not thread-safe.
  * which = 0: route every call to the fp32 CUDA-core kernels instead of the tensor-core ones;
  * which = 1: score every query block in double precision (skip the certified fp32 stage).

@@ -28,6 +28,7 @@ EXPORTS = (
     "blossom_attn_fwd", "blossom_attn_bwd",
     "blossom_device_status", "blossom_status_string", "blossom_version", "blossom_launch_count",
     "blossom_profile_start", "blossom_profile_stop", "blossom_kernel_name", "blossom_debug_switch",
+    "blossom_selftest_wait_timeout",
 )
 
 
@@ -87,6 +88,8 @@ def load():
     lib.blossom_profile_stop.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     lib.blossom_kernel_name.restype = ctypes.c_char_p
     lib.blossom_kernel_name.argtypes = [ctypes.c_int]
+    lib.blossom_selftest_wait_timeout.restype = ctypes.c_int
+    lib.blossom_selftest_wait_timeout.argtypes = [vp, sz, vp]
     lib.blossom_debug_switch.restype = ctypes.c_int
     lib.blossom_debug_switch.argtypes = [ctypes.c_int, ctypes.c_int]
     _lib = lib
@@ -233,3 +236,11 @@ def blossom_debug_switch(which: int, value: int) -> None:
     rc = load().blossom_debug_switch(int(which), int(value))
     if rc:
         raise BlossomError(rc, "blossom_debug_switch")
+
+
+def blossom_selftest_wait_timeout(workspace, stream=None) -> None:
+    """Launch the diagnostic kernel whose only wait cannot complete; read the outcome with
+    ``blossom_device_status(workspace)`` (it must be BLOSSOM_ERR_TIMEOUT)."""
+    rc = load().blossom_selftest_wait_timeout(_ptr(workspace), _nbytes(workspace), _stream(stream))
+    if rc:
+        raise BlossomError(rc, "blossom_selftest_wait_timeout")

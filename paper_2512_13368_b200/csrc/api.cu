@@ -273,6 +273,12 @@ int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_
   return BLOSSOM_OK;
 }
 
+int blossom_selftest_wait_timeout(void *workspace, size_t workspace_bytes, blossom_stream_t stream) {
+  if (!workspace || misaligned(workspace, 256) || workspace_bytes < 256) return BLOSSOM_ERR_WORKSPACE;
+  ++g_launches;
+  return tc::launch_wait_selftest(static_cast<int32_t *>(workspace), (cudaStream_t)stream);
+}
+
 int blossom_debug_switch(int which, int value) {
   if (value < -1 || value > 1) return BLOSSOM_ERR_INVALID_ARG;
   if (which == 0) g_force_simt_override = value;

@@ -135,6 +135,7 @@ int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, flo
                      cudaStream_t st);
 
 namespace tc {
+int launch_wait_selftest(int32_t *status, cudaStream_t st);
 bool fwd_tc_supported(const Shape &s, int dtype);
 size_t tc_meta_bytes(const Shape &s);  // bytes of one of the two tile-list areas of the workspace
 int launch_bwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,

@@ -39,6 +39,40 @@ int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_
   return rc == CUDA_SUCCESS ? 0 : 1;
 }
 
+// Diagnostic kernel: the bounded-wait machinery of the attention kernels on a wait that cannot
+// complete.  One CTA allocates tensor memory like the attention kernels, initialises an mbarrier
+// that expects an arrival nobody makes, and every warp waits on it: the waits run out after the
+// common limit, the first one records its site, later ones return at once, and the common kernel
+// end frees the tensor memory and reports BLOSSOM_ERR_TIMEOUT, the site and the CTA through the
+// status words.  Nothing faults and nothing spins without bound.
+__global__ void __launch_bounds__(128) wait_selftest_kernel(int32_t *status) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const int warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc(smem_u32(&tmem_slot), 32);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  mbar_wait(smem_u32(&bar), 0, &abort_flag, 900 + warp);  // phase 0 never completes
+  finish(warp, tmem_slot, 32, &abort_flag, status);
+}
+
+int launch_wait_selftest(int32_t *status, cudaStream_t st) {
+  if (cudaMemsetAsync(status, 0, 32, st) != cudaSuccess) return BLOSSOM_ERR_CUDA;
+  wait_selftest_kernel<<<1, 128, 0, st>>>(status);
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
 bool fwd_tc_supported(const Shape &s, int dtype) {
   return dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;

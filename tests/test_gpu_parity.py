@@ -450,3 +450,93 @@ def test_certified_selection_on_random_small_block_shapes(runner):
         p = runner.DeviceProblem(w)
         fast, exact = _fast_and_exact_selection(p)
         assert np.array_equal(fast, exact), (it, L, Bk, D, H, B, topk, dtype, std)
+
+
+# ------------------------------------------- what stands in for a memory checker on this path
+def _guarded(shape, dtype, fill, device, pad=4096):
+    """A tensor carved out of a larger allocation with `pad` guard elements before and after it."""
+    import torch
+    n = int(np.prod(shape))
+    raw = torch.full((n + 2 * pad,), fill, dtype=dtype, device=device)
+    return raw, raw[pad:pad + n].view(shape)
+
+
+@pytest.mark.parametrize("L,D,block,topk,window,lens,kv_heads", [
+    (200, 32, 16, 4, 32, [200, 77, 5], 0),      # ragged last block and last tile, padded batch entries
+    (330, 64, 32, 5, 70, [330, 129], 0),        # L not a multiple of 64: the bulk stores are clipped at L
+    (257, 64, 64, 3, 300, None, 2),             # one row past a tile border, grouped heads
+])
+def test_no_write_outside_any_output(runner, L, D, block, topk, window, lens, kv_heads):
+    """Every output (out, out_lt, out_st, lse, dq, dk, dv, dgate, block_idx) sits between guard
+    regions that must come back untouched: the tensor-core kernels write their results with bulk
+    tensor stores that rely on the hardware clipping rows past L, and nothing else would notice a
+    store that strays."""
+    import torch
+    from paper_2512_13368_b200 import binding
+    B = len(lens) if lens else 2
+    H = 4
+    w = workloads.make("guards", "bf16", B, H, L, D, block, topk, window, seed=43, kv_heads=kv_heads)
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    p = runner.DeviceProblem(w)
+    dev = p.q.device
+    hkv = kv_heads or H
+    bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+    specs = {"out": ((B, H, L, D), bf), "out_lt": ((B, H, L, D), bf), "out_st": ((B, H, L, D), bf),
+             "dq": ((B, H, L, D), bf), "dk": ((B, hkv, L, D), bf), "dv": ((B, hkv, L, D), bf),
+             "lse": ((2, B, H, L), f32), "dgate": ((H, 2), f32), "idx": ((B, hkv, w.n_blocks, topk), i32)}
+    raws = {}
+    for name, (shape, dt) in specs.items():
+        fill = -7 if dt == i32 else 123.0
+        raws[name], view = _guarded(shape, dt, fill, dev)
+        setattr(p, name, view)
+    p.step()
+    assert binding.blossom_device_status(p.workspace) == 0
+    res = p.results()
+    for name, (shape, dt) in specs.items():
+        raw, n, fill = raws[name], int(np.prod(shape)), (-7 if dt == i32 else 123.0)
+        assert bool((raw[:4096] == fill).all()) and bool((raw[4096 + n:] == fill).all()), name
+    print(check_forward_backward(w, res))
+
+
+@pytest.mark.parametrize("cfg", ["cfg2", "cfg3", "edge"])
+def test_tensor_core_path_against_the_cuda_core_path(runner, cfg):
+    """A second opinion on the tensor-core kernels: the same bf16 problem through the fp32
+    CUDA-core kernels (debugging switch), which share none of their code.  Both round their
+    outputs to bf16, so they agree to a few bf16 units in the last place of the largest value."""
+    from paper_2512_13368_b200 import binding
+    if cfg == "cfg2":
+        w = workloads.config2(B=16)
+    elif cfg == "cfg3":
+        w = workloads.config3(B=1)
+    else:
+        w = workloads.make("edge-simt", "bf16", 2, 3, 700, 32, 16, 9, 48, seed=47, lengths=(100, 700))
+    _, tc = run(runner, w)
+    binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, 1)
+    try:
+        _, simt = run(runner, w)
+    finally:
+        binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, -1)
+    assert np.array_equal(tc["idx"], simt["idx"])
+    for key in ("out", "out_lt", "out_st", "lse", "dq", "dk", "dv", "dgate"):
+        ref = np.abs(simt[key]).max()
+        err = np.abs(tc[key] - simt[key]).max()
+        assert err <= 2e-2 * max(ref, 1e-3), (key, err, ref)
+    check_forward_backward(w, simt)      # and the CUDA-core path against the oracle
+
+
+def test_a_wait_that_cannot_complete_is_reported_and_the_context_stays_usable(runner):
+    """The timeout branch of the bounded device-side waits, in the allowed form: a diagnostic
+    kernel waits on a barrier nobody arrives at; the wait gives up after its limit, the kernel ends
+    normally, frees its tensor memory and leaves BLOSSOM_ERR_TIMEOUT, the site of the wait and the
+    CTA in the status words.  A normal step afterwards must still be right."""
+    import torch
+    from paper_2512_13368_b200 import binding
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda:0")
+    binding.blossom_selftest_wait_timeout(ws)
+    assert binding.blossom_device_status(ws) == binding.BLOSSOM_ERR_TIMEOUT
+    words = ws[:16].cpu().numpy().view(np.int32)
+    assert words[0] == binding.BLOSSOM_ERR_TIMEOUT and 900 <= words[1] < 904 and words[2] == 0
+    w = workloads.make("after-timeout", "bf16", 2, 2, 300, 64, 32, 3, 50, seed=53)
+    _, res = run(runner, w)                    # tensor memory was freed, barriers work, results are right
+    print(check_forward_backward(w, res))
