@@ -17,9 +17,11 @@
 // memory and written with whole-line TMA stores.
 //
 //  dQ     resident Q, dO (128 queries); streams K, V 64-key tiles (same walk as the forward) and
-//         works through them in half tiles of 32 keys.  Tensor memory: three buffers of 64
-//         columns (half tile x uses buffer x % 3: S in its first 32 columns, dP in the other 32)
-//         and dQ [192,192+D).  S = Q K^T, dP = dO V^T; P'_x = weight_x exp(S - lse_x);
+//         works through them in half tiles of 32 keys.  Tensor memory: two buffers of 64
+//         columns (half tile x uses buffer x % 2: S in its first 32 columns, dP in the other 32),
+//         Q and dO as first operands of the first-stage products [128,128+D/2), [160,160+D/2)
+//         (read from shared memory they cost 4 KB per product, more than the data pipe delivers
+//         in the product's run time), and dQ [192,192+D).  S = Q K^T, dP = dO V^T; P'_x = weight_x exp(S - lse_x);
 //         dS = P'_lt (dP - Delta_lt) + P'_st (dP - Delta_st) (one tile for both branches, they share
 //         K).  A thread owns 16 of the 32 columns and writes its dS (bf16 pairs) over the first 8
 //         of its own S columns, from where dQ += dS K reads it: the compute warps wait for one
@@ -165,9 +167,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   constexpr int STAGES = kDqStages;
   constexpr int OC = D / 2;  // accumulator columns per thread
   extern __shared__ uint8_t smem_raw[];
-  // barriers: full[STAGES], empty[STAGES], res, meta, then one per buffer: s_full[3], t_full[3],
-  // mma_done[3]
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 11];
+  // barriers: full[STAGES], empty[STAGES], res, meta, a_ready, then one per buffer: s_full[2],
+  // t_full[2], mma_done[2]
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 9];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ double red[kComputeWarps];
@@ -199,8 +201,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
 
   const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[STAGES]);
   const uint32_t b_res = smem_u32(&bars[2 * STAGES]), b_meta = smem_u32(&bars[2 * STAGES + 1]);
-  const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 2]), b_tfull = smem_u32(&bars[2 * STAGES + 5]);
-  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 8]);
+  const uint32_t b_aready = smem_u32(&bars[2 * STAGES + 2]);
+  const uint32_t b_sfull = smem_u32(&bars[2 * STAGES + 3]), b_tfull = smem_u32(&bars[2 * STAGES + 5]);
+  const uint32_t b_done = smem_u32(&bars[2 * STAGES + 7]);
 
   if (tid == 0) {
     abort_flag = (*status != 0) ? 1 : 0;
@@ -213,7 +216,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
       mbar_init(b_empty + 8 * i, 1);
     }
     mbar_init(b_res, 1);
-    for (int i = 0; i < 3; ++i) {
+    mbar_init(b_aready, kComputeWarps);
+    for (int i = 0; i < 2; ++i) {
       mbar_init(b_sfull + 8 * i, 1);
       mbar_init(b_tfull + 8 * i, kComputeWarps);
       mbar_init(b_done + 8 * i, 1);
@@ -238,7 +242,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   mbar_wait(b_meta, 0, &abort_flag, 223);
   const int nvis = *reinterpret_cast<const int *>(meta + ml.counts);
   const uint32_t tmem_base = tmem_slot;
-  const uint32_t tmem_dq = tmem_base + 192;  // buffers at tmem_base + 64 * (half tile % 3)
+  // buffers at tmem_base + 64 * (half tile % 2); Q and dO as first operands (bf16 pairs, D / 2
+  // columns each) at 128 and 160; the dQ accumulator at 192
+  const uint32_t tmem_qa = tmem_base + 128, tmem_ga = tmem_base + 160, tmem_dq = tmem_base + 192;
 
   if (warp >= kComputeWarps) {
     // ============ three single-thread roles, one converged warp each ============
@@ -259,16 +265,17 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         __syncwarp();
       }
     } else if (warp == kComputeWarps + 1 && nvis > 0) {
-      // ---- S = Q K^T and dP = dO V^T of a half tile (32 keys) into buffer x % 3 once
-      // dQ += dS K of half tile x-3 has read that buffer ----
+      // ---- S = Q K^T and dP = dO V^T of a half tile (32 keys) into buffer x % 2 once
+      // dQ += dS K of half tile x-2 has read that buffer.  Q and dO are read from tensor memory
+      // (the compute warps copied the resident tiles there), so a product fetches only its 32
+      // keys from shared memory instead of 128 rows of Q or dO as well ----
       constexpr uint32_t idesc_s = instr_desc(128, 32, 0, 0);
-      const uint64_t dqd = smem_desc(smem_u32(q_tile), 16, C::kAtomBytes, C::kSwizzle);
-      const uint64_t dgd = smem_desc(smem_u32(g_tile), 16, C::kAtomBytes, C::kSwizzle);
-      mbar_wait(b_res, 0, &abort_flag, 201);
-      for (int i = 0, x = 0, b = 0, ph = 0; i < nvis; ++i) {  // x = 2 i + hh, b = x % 3, ph = (x / 3) & 1
+      mbar_wait(b_aready, 0, &abort_flag, 201);
+      tc_fence_after();
+      for (int i = 0, x = 0, b = 0, ph = 0; i < nvis; ++i) {  // x = 2 i + hh, b = x % 2, ph = (x / 2) & 1
         mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 202);
         for (int hh = 0; hh < 2; ++hh, ++x) {
-          if (x >= 3) mbar_wait(b_done + 8 * b, ph ^ 1, &abort_flag, 203);
+          if (x >= 2) mbar_wait(b_done + 8 * b, ph ^ 1, &abort_flag, 203);
           tc_fence_after();
           const uint32_t kt = smem_u32(kv_tiles + (i % STAGES) * 2 * C::kSmallBytes) + hh * 32 * C::kRowBytes;
           const uint64_t dkd = smem_desc(kt, 16, C::kAtomBytes, C::kSwizzle);
@@ -276,13 +283,13 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
           const uint32_t ts = tmem_base + 64 * b;
           if (elect_one()) {
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) umma_bf16(ts, dqd + 2 * k, dkd + 2 * k, idesc_s, k > 0);
+            for (int k = 0; k < D / 16; ++k) umma_bf16_ts(ts, tmem_qa + 8 * k, dkd + 2 * k, idesc_s, k > 0);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) umma_bf16(ts + 32, dgd + 2 * k, dvd + 2 * k, idesc_s, k > 0);
+            for (int k = 0; k < D / 16; ++k) umma_bf16_ts(ts + 32, tmem_ga + 8 * k, dvd + 2 * k, idesc_s, k > 0);
             umma_commit(b_sfull + 8 * b);
           }
           __syncwarp();
-          if (++b == 3) {
+          if (++b == 2) {
             b = 0;
             ph ^= 1;
           }
@@ -307,7 +314,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
             if (hh == 1) umma_commit(b_empty + 8 * (i % STAGES));  // every product on this stage has completed
           }
           __syncwarp();
-          if (++b == 3) {
+          if (++b == 2) {
             b = 0;
             ph ^= 1;
           }
@@ -332,7 +339,25 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     }
     float2 dalL = make_float2(0.f, 0.f), dalS = make_float2(0.f, 0.f);  // sums of P' dP per branch
     const float sc2 = s.scale * kLog2e;
-    int b = 0, ph = 0;  // buffer x % 3 of half tile x = 2 i + hh and the parity (x / 3) & 1
+    int b = 0, ph = 0;  // buffer x % 2 of half tile x = 2 i + hh and the parity (x / 2) & 1
+    if (nvis > 0) {
+      // The resident tiles become first operands in tensor memory: row r of Q (warps 0..3) or of dO
+      // (warps 4..7) goes to lane r as it is stored, two bf16 per 32-bit column.
+      mbar_wait(b_res, 0, &abort_flag, 208);
+      const uint8_t *src = (half ? g_tile : q_tile) + r * C::kRowBytes;
+      uint32_t wr[D / 2];
+#pragma unroll
+      for (int ch = 0; ch < D / 8; ++ch) {
+        const int pos = D == 64 ? (ch ^ (r & 7)) : (ch ^ ((r >> 1) & 3));  // the TMA swizzle of the tile
+        const uint4 v4 = *reinterpret_cast<const uint4 *>(src + (pos << 4));
+        wr[4 * ch] = v4.x; wr[4 * ch + 1] = v4.y; wr[4 * ch + 2] = v4.z; wr[4 * ch + 3] = v4.w;
+      }
+      const uint32_t ta = (half ? tmem_ga : tmem_qa) + lane_off;
+      if constexpr (D == 64) tmem_st32u(ta, wr); else tmem_st16u(ta, wr);
+      tmem_wait_st();
+      tc_fence_before();
+      warp_arrive(b_aready, lane);
+    }
 
     int cls_n = nvis > 0 ? jcls[warp] : 0;
     for (int x = 0; x < 2 * nvis; ++x) {  // half tile x: keys 32 (x % 2) ... of tile list[x / 2]
@@ -377,14 +402,14 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
       tmem_wait_st();
       tc_fence_before();
       warp_arrive(b_tfull + 8 * b, lane);
-      if (++b == 3) {
+      if (++b == 2) {
         b = 0;
         ph ^= 1;
       }
     }
 
     if (nvis > 0) {
-      mbar_wait(b_done + 8 * ((2 * nvis - 1) % 3), ((2 * nvis - 1) / 3) & 1, &abort_flag, 209);
+      mbar_wait(b_done + 8, (nvis - 1) & 1, &abort_flag, 209);  // the last half tile used buffer 1
       __syncwarp();
       tc_fence_after();
     }
