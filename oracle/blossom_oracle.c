@@ -18,7 +18,9 @@
  *   score sharing        Eq. 12 rule (sum of the probabilities of everyone who
  *                               shares one selection) applied to the queries
  *                               of a query block
- *   top-k selection      Eq. 13 own block always kept, ties -> lower index
+ *   top-k selection      Eq. 13 own block always kept, ties -> lower index; per query block
+ *                               (summed probabilities) or per query position (as printed:
+ *                               blossom_oracle_select_pq)
  *   overlapping blocks   Eq. 8 with l, s != Bk and the score remap of Eq. 11
  *                               (blossom_oracle_select_cmp)
  *   selected-KV attention Eq. 14 + Eq. 16 (via Eq. 1 with the causal mask)
@@ -158,6 +160,89 @@ int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double s
       if (len > L) len = L;
       select_unit(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D,
                   idx + u * M * topk, scores ? scores + u * M * M : NULL);
+    }
+  return 0;
+}
+
+/* ---- selection per query position for one (n,h) unit: Eq. 8-10, 13 as printed -----------
+ * The paper selects for each query position: query t (in query block b = t / Bk) takes the softmax
+ * of Eq. 10 over the live blocks j < b (strictly-past blocks, whose summaries hold no key after
+ * t) and keeps the top_k - 1 largest probabilities, ties to the lower index, plus its own block b.
+ * idx is [L][topk] (one row per position, -1 rows for padding), probs [L][M] optional. */
+static void select_unit_pq(int L, int D, int Bk, int topk, double scale, int pad0,
+                           const double *q, const double *k, int32_t *idx, double *probs) {
+  const int M = n_blocks(L, Bk);
+  double *ktil = (double *)calloc((size_t)M * D, sizeof(double));
+  int *live = (int *)calloc((size_t)M, sizeof(int));
+  double *P = (double *)malloc(sizeof(double) * (size_t)M);
+  char *taken = (char *)malloc((size_t)M);
+  for (int j = 0; j < M; ++j) { /* Eq. 8 + Eq. 9 */
+    int lo = imax(j * Bk, pad0), hi = imin((j + 1) * Bk, L), cnt = 0;
+    for (int p = lo; p < hi; ++p) {
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] += k[(size_t)p * D + c];
+      ++cnt;
+    }
+    live[j] = cnt > 0;
+    if (cnt > 0)
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] /= (double)cnt;
+  }
+  for (int t = 0; t < L; ++t) {
+    int32_t *row = idx + (size_t)t * topk;
+    for (int s = 0; s < topk; ++s) row[s] = -1;
+    if (probs)
+      for (int j = 0; j < M; ++j) probs[(size_t)t * M + j] = 0.0;
+    if (t < pad0) continue;
+    const int b = t / Bk;
+    int ncand = 0;
+    double mx = -INFINITY;
+    for (int j = 0; j < b; ++j) {
+      P[j] = 0.0;
+      if (!live[j]) continue;
+      ++ncand;
+      double acc = 0.0;
+      for (int c = 0; c < D; ++c) acc += q[(size_t)t * D + c] * ktil[(size_t)j * D + c];
+      P[j] = scale * acc;
+      if (P[j] > mx) mx = P[j];
+    }
+    double den = 0.0;
+    for (int j = 0; j < b; ++j)
+      if (live[j]) den += exp(P[j] - mx);
+    for (int j = 0; j < b; ++j) /* Eq. 10 */
+      P[j] = live[j] ? exp(P[j] - mx) / den : 0.0;
+    if (probs)
+      for (int j = 0; j < b; ++j) probs[(size_t)t * M + j] = P[j];
+    int want = imin(topk - 1, ncand); /* Eq. 13 */
+    memset(taken, 0, (size_t)M);
+    for (int s = 0; s < want; ++s) {
+      int best = -1;
+      for (int j = 0; j < b; ++j) {
+        if (!live[j] || taken[j]) continue;
+        if (best < 0 || P[j] > P[best]) best = j;
+      }
+      taken[best] = 1;
+    }
+    int s = 0;
+    for (int j = 0; j < b; ++j)
+      if (taken[j]) row[s++] = j;
+    row[s++] = b;
+  }
+  free(ktil); free(live); free(P); free(taken);
+}
+
+int blossom_oracle_select_pq(int B, int H, int L, int D, int Bk, int topk, double scale,
+                             const double *q, const double *k, const int32_t *seq_lens,
+                             int32_t *idx, double *probs) {
+  if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
+  const int M = n_blocks(L, Bk);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int n = 0; n < B; ++n)
+    for (int h = 0; h < H; ++h) {
+      size_t u = (size_t)n * H + h;
+      int len = seq_lens ? seq_lens[n] : L;
+      if (len < 0) len = 0;
+      if (len > L) len = L;
+      select_unit_pq(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D,
+                     idx + u * L * topk, probs ? probs + u * L * M : NULL);
     }
   return 0;
 }
@@ -358,8 +443,10 @@ static int stis_keys(int mode, int w, int blk, int L, int pad0, int t, int *keys
 
 static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 
+/* per_query = 0: idx is [B][H][M][topk], one row per query block; 1: [B][H][L][topk], one row per
+ * query position (Eq. 13 as printed) */
 int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
-                           int stis_blk, double scale,
+                           int stis_blk, int per_query, double scale,
                            const double *q, const double *k, const double *v, const double *gate,
                            const int32_t *seq_lens, const int32_t *idx, double *out,
                            double *out_lt, double *out_st, double *lse) {
@@ -387,7 +474,8 @@ int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int win
         if (t < pad0) {
           for (int c = 0; c < D; ++c) oL[c] = oS[c] = 0.0;
         } else {
-          const int32_t *row = idx + (u * M + (size_t)(t / Bk)) * topk;
+          const int32_t *row = per_query ? idx + (u * L + (size_t)t) * topk
+                                         : idx + (u * M + (size_t)(t / Bk)) * topk;
           int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
           lL = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oL); /* Eq. 16 */
           nk = stis_keys(stis_mode, window, stis_blk, L, pad0, t, keys);
@@ -436,7 +524,7 @@ static void attend_row_bwd(int D, double scale, const double *qt, const double *
 }
 
 int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
-                            int stis_blk, double scale,
+                            int stis_blk, int per_query, double scale,
                             const double *q, const double *k, const double *v, const double *gate,
                             const int32_t *seq_lens, const int32_t *idx, const double *out_lt,
                             const double *out_st, const double *lse, const double *dout,
@@ -471,7 +559,8 @@ int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int wi
           gL[c] = alpha * dout[ro + c];
           gS[c] = (1.0 - alpha) * dout[ro + c];
         }
-        const int32_t *row = idx + (u * M + (size_t)(t / Bk)) * topk;
+        const int32_t *row = per_query ? idx + (u * L + (size_t)t) * topk
+                                       : idx + (u * M + (size_t)(t / Bk)) * topk;
         int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
         attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[u * L + t],
                        out_lt + ro, gL, dqu + (size_t)t * D, dku, dvu);

@@ -52,10 +52,12 @@ def _load():
         lib.blossom_oracle_select_cmp.restype = i
         lib.blossom_oracle_select_cmp.argtypes = [i, i, i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp, _dp]
         lib.blossom_oracle_forward.restype = i
-        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_select_pq.restype = i
+        lib.blossom_oracle_select_pq.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp]
+        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
         lib.blossom_oracle_backward.restype = i
-        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                 _ip, _dp, _dp, _dp, _dp, _dp, _dp, _dp, _dp]
         _lib = lib
     return _lib
@@ -102,6 +104,41 @@ def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores
     return (idx, scores) if return_scores else idx
 
 
+def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False):
+    """Eq. 8-10, 13 as printed: one selection per query position.  k may have fewer heads than q
+    (grouped heads: the probabilities of a group's heads are summed, Eq. 12, and the group's
+    queries at one position share the selection).  Returns idx ``[B,Hkv,L,topk]`` (ascending, -1
+    padded, the position's own block included) and, if asked, the probabilities ``[B,Hkv,L,M]``."""
+    q, k = _f64(q), _f64(k)
+    B, H, L, D = q.shape
+    Hkv = k.shape[1]
+    G = _group(H, Hkv)
+    M = -(-L // block)
+    idx = np.empty((B, H, L, topk), dtype=np.int32)
+    probs = np.zeros((B, H, L, M), dtype=np.float64) if (return_scores or G > 1) else None
+    sl = _lens(seq_lens, B)
+    kk = np.ascontiguousarray(np.repeat(k, G, axis=1))
+    rc = _load().blossom_oracle_select_pq(B, H, L, D, block, topk, _scale(sm_scale, D), _ptr(q, _dp),
+                                          _ptr(kk, _dp), _ptr(sl, _ip), _ptr(idx, _ip), _ptr(probs, _dp))
+    if rc:
+        raise ValueError("blossom_oracle_select_pq: bad arguments")
+    if G == 1:
+        return (idx, probs) if return_scores else idx
+    probs = probs.reshape(B, Hkv, G, L, M).sum(axis=2)               # Eq. 12
+    gidx = np.full((B, Hkv, L, topk), -1, dtype=np.int32)
+    for n in range(B):
+        pad0 = 0 if seq_lens is None else L - int(seq_lens[n])
+        live = np.array([min((j + 1) * block, L) > max(j * block, pad0) for j in range(M)])
+        for g in range(Hkv):
+            for t in range(pad0, L):
+                b = t // block
+                cand = [j for j in range(b) if live[j]]
+                best = sorted(cand, key=lambda j: (-probs[n, g, t, j], j))[:topk - 1]
+                row = sorted(best) + [b]
+                gidx[n, g, t, :len(row)] = row
+    return (gidx, probs) if return_scores else gidx
+
+
 def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, sm_scale=None,
                       return_scores=False):
     """Eq. 8-11, 13 with overlapping compression blocks (length ``cmp_block``, stride
@@ -135,11 +172,13 @@ def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, s
 
 
 def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None,
-            stis_mode=0, stis_block=1):
+            stis_mode=0, stis_block=1, per_query=False):
     """Eq. 14, 16, 17, 19.  ``idx`` overrides the selection when given.
 
     ``stis_mode`` 0: the short-term branch is the causal window (Eq. 15, first case);
     1: the power-law mask (all of Eq. 15, causal side) with mask block ``stis_block``.
+
+    ``per_query``: the selection is per query position, idx ``[B,H,L,topk]``.
 
     Returns a dict: out, out_lt, out_st ``[B,H,L,D]``, lse ``[2,B,H,L]``, idx.
     """
@@ -148,16 +187,16 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     M = -(-L // block)
     assert gate.shape == (H, 2)
     if idx is None:
-        idx = select_blocks(q, k, block, topk, seq_lens, sm_scale)
+        idx = (select_blocks_per_query if per_query else select_blocks)(q, k, block, topk, seq_lens, sm_scale)
     idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
-    assert idx.shape == (B, H, M, topk)
+    assert idx.shape == (B, H, L if per_query else M, topk)
     sl = _lens(seq_lens, B)
     out = np.empty_like(q)
     out_lt = np.empty_like(q)
     out_st = np.empty_like(q)
     lse = np.empty((2, B, H, L), dtype=np.float64)
     rc = _load().blossom_oracle_forward(B, H, L, D, block, topk, window, int(stis_mode),
-                                        int(stis_block), _scale(sm_scale, D),
+                                        int(stis_block), int(bool(per_query)), _scale(sm_scale, D),
                                         _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp), _ptr(gate, _dp),
                                         _ptr(sl, _ip), _ptr(idx, _ip), _ptr(out, _dp),
                                         _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp))
@@ -167,7 +206,7 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
 
 
 def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None,
-             stis_mode=0, stis_block=1):
+             stis_mode=0, stis_block=1, per_query=False):
     """Gradients of sum(out * dout) with the selection frozen.
 
     ``fwd`` is the dict ``forward`` returned.  Returns dq, dk, dv, dgate ``[H,2]``.
@@ -180,7 +219,7 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
     dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
     dgate = np.empty((H, 2), dtype=np.float64)
     rc = _load().blossom_oracle_backward(B, H, L, D, block, topk, window, int(stis_mode),
-                                         int(stis_block), _scale(sm_scale, D),
+                                         int(stis_block), int(bool(per_query)), _scale(sm_scale, D),
                                          _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp),
                                          _ptr(gate, _dp), _ptr(sl, _ip), _ptr(idx, _ip),
                                          _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp),
@@ -192,11 +231,12 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
 
 
 def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm_scale=None,
-                     idx=None, stis_mode=0, stis_block=1):
+                     idx=None, stis_mode=0, stis_block=1, per_query=False):
     """Convenience: forward then backward; returns the two dicts merged."""
-    f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx, stis_mode, stis_block)
+    f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx, stis_mode, stis_block,
+                per_query)
     b = backward(q, k, v, gate, block, topk, window, f, dout, seq_lens, sm_scale, stis_mode,
-                 stis_block)
+                 stis_block, per_query)
     f.update(b)
     return f
 
@@ -254,7 +294,9 @@ def forward_gqa(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None
     """``forward`` for q ``[B,H,L,D]`` and k, v ``[B,Hkv,L,D]``; idx is ``[B,Hkv,M,topk]``."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     G = _group(q.shape[1], k.shape[1])
-    if idx is None:
+    if idx is None and kw.get("per_query"):
+        idx = select_blocks_per_query(q, k, block, topk, seq_lens, sm_scale)
+    elif idx is None:
         idx = select_blocks_gqa(q, k, block, topk, seq_lens, sm_scale, cmp_block=cmp_block,
                                 cmp_stride=cmp_stride)
     idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
