@@ -20,7 +20,7 @@
  *     query rows produce 0 in out / out_lt / out_st / lse and in every gradient.
  *   - block_idx is int32 [B][H][M][top_k], M = ceil(seq_len / block_size): for each query block
  *     the selected key blocks in ascending order, -1 padded.  The query block's own block is
- *     always one of them.
+ *     always one of them.  (select_mode 1: a row per query position, [B][H][L][top_k].)
  *   - lse is float [2][B][H][L]: plane 0 long-term branch, plane 1 short-term branch; natural log
  *     of the sum over the branch's visible keys of exp(sm_scale * <q, k>).
  *   - gate_logits is float [H][2]: column 0 long-term, column 1 short-term logit;
@@ -70,7 +70,11 @@ typedef struct {
   int32_t window;      /* w >= 1: query t sees keys t - w < p <= t in the short-term branch (and
                         * more with stis_mode 1)                                                 */
   int32_t causal;      /* must be 1                                                              */
-  int32_t select_mode; /* 0 = one selection per query block (the only mode implemented)          */
+  int32_t select_mode; /* 0 = one selection per query block, from the probabilities summed over the
+                        * block's queries (tensor-core kernels for bf16); 1 = one selection per
+                        * query position (Eq. 13 as printed): block_idx is then
+                        * [B][kv_heads][L][top_k], a row per position, and the attention runs on
+                        * the CUDA-core kernels; not combined with cmp_block / cmp_stride          */
   int32_t dtype;       /* BLOSSOM_DTYPE_FP32 or BLOSSOM_DTYPE_BF16                               */
   float sm_scale;      /* 0 -> 1/sqrt(head_dim); scales block scores and attention logits alike  */
   int64_t stride_b, stride_h, stride_l; /* element strides of every q-shaped tensor              */

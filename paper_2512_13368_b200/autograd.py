@@ -63,7 +63,7 @@ def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True):
 class _BlossomAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
-                stis_mode, stis_block, cmp_block, cmp_stride):
+                stis_mode, stis_block, cmp_block, cmp_stride, per_query=0):
         seq_lens = check_arguments(q, k, v, gate_logits, seq_lens)
         B, H, L, D = q.shape
         Hkv = k.shape[1]
@@ -78,7 +78,7 @@ class _BlossomAttention(torch.autograd.Function):
         params = binding.make_params(B, H, L, D, block_size, top_k, window, _DT[q.dtype],
                                      sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
                                      stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride,
-                                     kv_heads=Hkv, kv_strides=k.stride()[:3])
+                                     kv_heads=Hkv, kv_strides=k.stride()[:3], select_mode=int(per_query))
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -86,7 +86,7 @@ class _BlossomAttention(torch.autograd.Function):
         workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         gate = gate_logits.detach().to(torch.float32).contiguous()
         M = -(-L // block_size)
-        idx = torch.empty((B, Hkv, M, top_k), dtype=torch.int32, device=dev)
+        idx = torch.empty((B, Hkv, L if per_query else M, top_k), dtype=torch.int32, device=dev)
         out, out_lt, out_st = _like(q), _like(q), _like(q)
         lse = torch.empty((2, B, H, L), dtype=torch.float32, device=dev)
         binding.blossom_attn_fwd(params, q, k, v, gate, seq_lens, idx, 0, out, out_lt, out_st, lse,
@@ -106,12 +106,12 @@ class _BlossomAttention(torch.autograd.Function):
         dgate = torch.empty((q.shape[1], 2), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
-        return dq, dk, dv, dgate.to(ctx.gate_dtype), None, None, None, None, None, None, None, None, None
+        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 10
 
 
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
                       return_indices=False, short_term="window", mask_block=1, cmp_block=0,
-                      cmp_stride=0):
+                      cmp_stride=0, select_per_query=False):
     """Gated two-branch sparse attention of q [B, H, L, D] and k, v [B, Hkv, L, D] (float32 or
     bfloat16, CUDA; Hkv divides H: with Hkv < H the query heads of a group share key/value head
     and selection, and the returned indices are [B, Hkv, M, top_k]).
@@ -125,11 +125,13 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     mask_block positions at power-of-two block distances, and the last mask_block positions).
     cmp_block / cmp_stride: length and stride of overlapping compression blocks for the selection
     (Eq. 8, 11); 0 = the selection blocks themselves.
+    select_per_query: one selection per query position (Eq. 13 as printed; indices [B, Hkv, L,
+    top_k]) instead of one per query block; runs on the CUDA-core kernels.
     """
     if short_term not in ("window", "power-law"):
         raise ValueError("short_term must be 'window' or 'power-law'")
     out, idx = _BlossomAttention.apply(q, k, v, gate_logits, seq_lens, int(block_size), int(top_k),
                                        int(window), float(sm_scale),
                                        1 if short_term == "power-law" else 0, int(mask_block),
-                                       int(cmp_block), int(cmp_stride))
+                                       int(cmp_block), int(cmp_stride), int(bool(select_per_query)))
     return (out, idx) if return_indices else out

@@ -106,7 +106,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   if (kv_given && (p->kv_stride_l < p->head_dim || p->kv_stride_h < 1 || p->kv_stride_b < 1 ||
                    p->kv_stride_l % 8 || p->kv_stride_h % 8 || p->kv_stride_b % 8))
     return BLOSSOM_ERR_INVALID_ARG;
-  if (p->causal != 1 || p->select_mode != 0) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->select_mode < 0 || p->select_mode > 1) return BLOSSOM_ERR_INVALID_ARG;
+  if (p->causal != 1) return BLOSSOM_ERR_UNSUPPORTED;
   if (p->stis_mode < 0 || p->stis_mode > 1 || p->stis_block < 0) return BLOSSOM_ERR_INVALID_ARG;
   if (p->head_dim != 32 && p->head_dim != 64) return BLOSSOM_ERR_UNSUPPORTED;
   if (p->block_size != 8 && p->block_size != 16 && p->block_size != 32 && p->block_size != 64)
@@ -135,6 +136,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.scale = (float)s.scale_d;
   s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;
   s.Hkv = p->kv_heads; s.G = p->heads / p->kv_heads;
+  s.pq = p->select_mode;
+  if (s.pq && s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // per-position selection scores the selection blocks themselves
   if (kv_given) {
     s.ksb = p->kv_stride_b; s.ksh = p->kv_stride_h; s.ksl = p->kv_stride_l;
   } else if (s.G == 1) {

@@ -63,6 +63,27 @@ __device__ __forceinline__ void build_visit_flags(const Shape &s, const int32_t 
   }
 }
 
+// Selection per query position (block_idx [B][Hkv][L][top_k]): every row of the query block has a
+// list of its own.  rowsel[r][w] = bit set of the blocks row r selected; flags[blk] bit 0 = some
+// row selected blk, bit 1 as above.  `active` rows only (thread (r, sub) takes every fourth entry).
+__device__ __forceinline__ void build_row_selections(const Shape &s, const int32_t *idxrow, int qb, int r,
+                                                     int sub, bool active, int *flags, uint32_t *rowsel) {
+  const int MW = (s.M + 31) >> 5;
+  const int t0 = qb * s.Bk, t1 = min(s.L, t0 + s.Bk) - 1;
+  for (int blk = threadIdx.x; blk <= qb; blk += blockDim.x)
+    flags[blk] = st_ranges_touch(s, t0, t1, blk * s.Bk, min(s.L, blk * s.Bk + s.Bk) - 1) ? 2 : 0;
+  for (int i = threadIdx.x; i < s.Bk * MW; i += blockDim.x) rowsel[i] = 0u;
+  __syncthreads();
+  if (active)
+    for (int i = sub; i < s.topk; i += 4) {
+      const int j = idxrow[i];
+      if (j >= 0 && j <= qb) {
+        atomicOr(&rowsel[r * MW + (j >> 5)], 1u << (j & 31));
+        atomicOr(&flags[j], 1);
+      }
+    }
+}
+
 // ------------------------------------------------------------------------------- forward
 template <typename T, int D>
 __global__ void __launch_bounds__(256) fwd_simt_kernel(
@@ -84,7 +105,13 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
   const bool inrange = t < s.L, active = inrange && t >= pad0;
 
   const int hk = h / s.G;  // key/value head of this query head; its group shares one selection
-  build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
+  uint32_t *rowsel = reinterpret_cast<uint32_t *>(flags + s.M);  // [Bk][ceil(M / 32)], per-position selection only
+  const int MW = (s.M + 31) >> 5;
+  if (s.pq)
+    build_row_selections(s, idx + (((int64_t)n * s.Hkv + hk) * s.L + (inrange ? t : 0)) * s.topk, qb, r, sub, active,
+                         flags, rowsel);
+  else
+    build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
 
   float4 qv[NV], aL[NV], aS[NV];
 #pragma unroll
@@ -109,7 +136,7 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
       if (!active) continue;
       const int p0 = blk * s.Bk;
       const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
-      const bool selb = f & 1;
+      const bool selb = s.pq ? (rowsel[r * MW + (blk >> 5)] >> (blk & 31)) & 1u : f & 1;
       for (int pi = pbeg; pi < pend; ++pi) {
         const bool inS = st_visible(s, t, p0 + pi);
         if (!selb && !inS) continue;
@@ -174,6 +201,8 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
   float *Ks = smf, *Vs = Ks + s.Bk * D;
   int *flags = reinterpret_cast<int *>(Vs + s.Bk * D);
   double *red = reinterpret_cast<double *>(flags + s.M + (s.M & 1));  // [Bk]
+  uint32_t *rowsel = reinterpret_cast<uint32_t *>(red + s.Bk);  // [Bk][ceil(M / 32)], per-position selection only
+  const int MW = (s.M + 31) >> 5;
   const int qb = blockIdx.x % s.M, u = blockIdx.x / s.M, n = u / s.H, h = u % s.H;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
@@ -186,7 +215,11 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
   const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
 
   const int hk = h / s.G;  // key/value head of this query head; its group shares one selection
-  build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
+  if (s.pq)
+    build_row_selections(s, idx + (((int64_t)n * s.Hkv + hk) * s.L + (inrange ? t : 0)) * s.topk, qb, r, sub, active,
+                         flags, rowsel);
+  else
+    build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
 
   float4 qv[NV], gv[NV], acc[NV];
   float dL = 0.f, dS = 0.f;
@@ -232,7 +265,7 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
       if (!active) continue;
       const int p0 = blk * s.Bk;
       const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
-      const bool selb = f & 1;
+      const bool selb = s.pq ? (rowsel[r * MW + (blk >> 5)] >> (blk & 31)) & 1u : f & 1;
       for (int pi = pbeg; pi < pend; ++pi) {
         const bool inS = st_visible(s, t, p0 + pi);
         if (!selb && !inS) continue;
@@ -288,6 +321,7 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   float *Qs = smf, *Gs = Qs + s.Bk * D;
   float *lLs = Gs + s.Bk * D, *lSs = lLs + s.Bk, *dLs = lSs + s.Bk, *dSs = dLs + s.Bk;
   int *flags = reinterpret_cast<int *>(dSs + s.Bk);
+  int *rsel = flags + s.M;  // [Bk] per-position selection only: which queries of the staged block selected this key block
   // uk counts (batch, key/value head) pairs: the key block collects from every query head of its group
   const int j = blockIdx.x % s.M, uk = blockIdx.x / s.M, n = uk / s.Hkv, hk = uk % s.Hkv;
   int len = seq_lens ? seq_lens[n] : s.L;
@@ -302,10 +336,11 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   // which query blocks visit this key block: bit 0 = selected it, bit 1 = their short-term branch
   // may reach it
   for (int qb = j + tid; qb < s.M; qb += blockDim.x) {
-    const int32_t *row = idx + ((int64_t)uk * s.M + qb) * s.topk;
+    const int32_t *row = idx + ((int64_t)uk * s.M + qb) * s.topk;  // (read only when the selection is per block)
     int f = st_ranges_touch(s, qb * s.Bk, min(s.L, qb * s.Bk + s.Bk) - 1, j * s.Bk,
                             min(s.L, j * s.Bk + s.Bk) - 1) ? 2 : 0;
-    for (int i = 0; i < s.topk; ++i) f |= (row[i] == j) ? 1 : 0;
+    if (!s.pq)
+      for (int i = 0; i < s.topk; ++i) f |= (row[i] == j) ? 1 : 0;
     flags[qb] = f;
   }
 
@@ -328,7 +363,22 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
       const int h = hk * s.G + x / (s.M - j), qb = j + x % (s.M - j);
       const int64_t u = (int64_t)n * s.H + h;
       const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
-      const int f = flags[qb];
+      int f = flags[qb];
+      if (s.pq) {  // every query position has a list of its own
+        __syncthreads();
+        int any = 0;
+        for (int i = tid; i < s.Bk; i += blockDim.x) {
+          const int t = qb * s.Bk + i;
+          int sel = 0;
+          if (t < s.L && t >= pad0) {
+            const int32_t *row = idx + ((int64_t)uk * s.L + t) * s.topk;
+            for (int e = 0; e < s.topk; ++e) sel |= (row[e] == j) ? 1 : 0;
+          }
+          rsel[i] = sel;
+          any |= sel;
+        }
+        f |= __syncthreads_or(any) ? 1 : 0;
+      }
       if (!f) continue;
       __syncthreads();
       stage_tile<T, D>(s, q, row_offset(s, n, h, 0), s.sl, qb * s.Bk, Qs);
@@ -345,8 +395,9 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
       if (!active) continue;
       const int t0 = qb * s.Bk;
       const int tbeg = max(0, p - t0), tend = min(s.Bk, s.L - t0);  // t >= p >= pad0
-      const bool selb = f & 1;
+      const bool sel_all = f & 1;
       for (int ti = tbeg; ti < tend; ++ti) {
+        const bool selb = s.pq ? rsel[ti] != 0 : sel_all;
         const bool inS = st_visible(s, t0 + ti, p);
         if (!selb && !inS) continue;
         const float4 *qr = reinterpret_cast<const float4 *>(Qs) + ti * CH;
@@ -422,7 +473,8 @@ int launch_fwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
                  const int32_t *seq_lens, const int32_t *idx, T *out, T *out_lt, T *out_st,
                  float *lse, cudaStream_t st) {
   const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.H);
-  const size_t smem = (size_t)2 * s.Bk * D * sizeof(float) + (size_t)s.M * sizeof(int);
+  const size_t rowsel = s.pq ? (size_t)s.Bk * ((s.M + 31) / 32) * sizeof(uint32_t) : 0;
+  const size_t smem = (size_t)2 * s.Bk * D * sizeof(float) + (size_t)s.M * sizeof(int) + rowsel;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(fwd_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
@@ -441,8 +493,9 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
                  const float *lse, const T *dout, T *dq, T *dk, T *dv, float *dgate,
                  const Workspace &ws, cudaStream_t st) {
   const unsigned grid = (unsigned)s.M * (unsigned)(s.B * s.H);
+  const size_t rowsel = s.pq ? (size_t)s.Bk * ((s.M + 31) / 32) * sizeof(uint32_t) : 0;
   const size_t smem_q = (size_t)2 * s.Bk * D * sizeof(float) +
-                        (size_t)(s.M + (s.M & 1)) * sizeof(int) + (size_t)s.Bk * sizeof(double);
+                        (size_t)(s.M + (s.M & 1)) * sizeof(int) + (size_t)s.Bk * sizeof(double) + rowsel;
   if (smem_q > 48 * 1024 &&
       cudaFuncSetAttribute(bwd_dq_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem_q) != cudaSuccess)
@@ -453,7 +506,7 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
                                                              out_st, lse, dout, dq, ws.delta,
                                                              ws.dalpha);
   }
-  const size_t smem_k = (size_t)(2 * s.Bk * D + 4 * s.Bk) * sizeof(float) + (size_t)s.M * sizeof(int);
+  const size_t smem_k = (size_t)(2 * s.Bk * D + 4 * s.Bk) * sizeof(float) + (size_t)(s.M + s.Bk) * sizeof(int);
   if (smem_k > 48 * 1024 &&
       cudaFuncSetAttribute(bwd_dkdv_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem_k) != cudaSuccess)

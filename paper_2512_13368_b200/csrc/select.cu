@@ -677,6 +677,81 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
   }
 }
 
+// ---- selection per query position (Eq. 13 as printed), double precision -------------------
+// One warp per (batch, key/value head, position t): the softmax of Eq. 10 over the live blocks
+// before t's block for every head of the group, the probabilities summed over the heads (Eq. 12),
+// the top_k - 1 largest kept together with t's own block, ties to the lower index.  block_idx is
+// [B][Hkv][L][top_k].  Lanes stride over the candidate blocks; the means come from global memory
+// (they are shared by the neighbouring positions and stay in L2).
+template <typename T, int D>
+__global__ void __launch_bounds__(256) score_per_query_kernel(
+    Shape sh, const T *__restrict__ q, const double *__restrict__ mean,
+    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx) {
+  extern __shared__ double dsm[];
+  __shared__ double bound_d[8][2];
+  const int M = sh.M, Bk = sh.Bk;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  double *P = dsm + (size_t)warp * (2 * M + D);  // [M] summed probabilities of this warp's position
+  double *Z = P + M;                             // [M] logits of the current head
+  double *qrow = Z + M;                          // [D]
+  uint8_t *taken = reinterpret_cast<uint8_t *>(dsm + (size_t)8 * (2 * M + D)) + (size_t)warp * M;
+  const int64_t pos = (int64_t)blockIdx.x * 8 + warp;
+  if (pos >= (int64_t)sh.B * sh.Hkv * sh.L) return;
+  const int t = (int)(pos % sh.L), u = (int)(pos / sh.L), n = u / sh.Hkv, hk = u % sh.Hkv;
+  int len = seq_lens ? seq_lens[n] : sh.L;
+  len = min(max(len, 0), sh.L);
+  const int pad0 = sh.L - len;
+  int32_t *row = idx + pos * sh.topk;
+  if (t < pad0) {
+    for (int i = lane; i < sh.topk; i += 32) row[i] = -1;
+    return;
+  }
+  const int b = t / Bk, jmin = pad0 / Bk;  // live blocks before the own one: jmin .. b - 1
+  const int nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
+  if (nsel > want && want > 0) {
+    for (int j = jmin + lane; j < b; j += 32) P[j] = 0.0;
+    const double *kbase = mean + (int64_t)u * M * D;
+    for (int hg = 0; hg < sh.G; ++hg) {
+      __syncwarp();
+      const T *qp = q + row_offset(sh, n, hk * sh.G + hg, t);
+      for (int c = lane; c < D; c += 32) qrow[c] = (double)ld1(qp + c);
+      __syncwarp();
+      double mx = -INFINITY;
+      for (int j = jmin + lane; j < b; j += 32) {
+        const double *kj = kbase + (int64_t)j * D;
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll 4
+        for (int c = 0; c < D; c += 4) {
+          a0 = fma(qrow[c], kj[c], a0);
+          a1 = fma(qrow[c + 1], kj[c + 1], a1);
+          a2 = fma(qrow[c + 2], kj[c + 2], a2);
+          a3 = fma(qrow[c + 3], kj[c + 3], a3);
+        }
+        const double z = sh.scale_d * ((a0 + a1) + (a2 + a3));
+        Z[j] = z;
+        mx = fmax(mx, z);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      double den = 0.0;
+      for (int j = jmin + lane; j < b; j += 32) {
+        const double e = exp(Z[j] - mx);
+        Z[j] = e;
+        den += e;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+      for (int j = jmin + lane; j < b; j += 32) P[j] += Z[j] / den;  // heads in ascending order
+    }
+    __syncwarp();
+    rank_select<double>(P, jmin, b, want, taken, bound_d[warp], lane);
+  } else {
+    for (int j = jmin + lane; j < b; j += 32) taken[j] = want > 0 ? 1 : 0;
+  }
+  __syncwarp();
+  emit_row(row, taken, jmin, b, sh.topk, lane);
+}
+
 // The arrays the selection kernels work in (the caller's workspace or the built-in scratch).
 struct SelBuffers {
   double *mean;
@@ -710,6 +785,15 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
                                                                             w.mean32, w.norm, w.count);
   } else if (cudaMemsetAsync(w.count, 0, sizeof(int32_t), st) != cudaSuccess) {
     return BLOSSOM_ERR_CUDA;
+  }
+  if (sh.pq) {  // one selection per query position: block_idx is [B][Hkv][L][top_k]
+    const size_t psm = (size_t)8 * (2 * sh.M + D) * sizeof(double) + (size_t)8 * sh.M + 16;
+    if (psm > 48 * 1024 && cudaFuncSetAttribute(score_per_query_kernel<T, D>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm) != cudaSuccess)
+      return BLOSSOM_ERR_CUDA;
+    LaunchScope ls(K_SCORE_SELECT, st);
+    score_per_query_kernel<T, D><<<(unsigned)((units * sh.L + 7) / 8), 256, psm, st>>>(sh, q, w.mean, seq_lens, idx);
+    return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
   }
   int sc_pitch = 0, sc_len = 0;
   const size_t fsm = fast_smem_bytes(sh, g, D, &sc_pitch);
@@ -787,7 +871,7 @@ size_t select_static_capacity_bytes() { return kStaticBytes; }
 
 int launch_select_static(const Shape &s, int dtype, const void *q, const void *k,
                          const int32_t *seq_lens, int32_t *idx, cudaStream_t st) {
-  if (s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // the built-in scratch has no room for that mode
+  if (s.cmp_l > 0 || s.pq) return BLOSSOM_ERR_UNSUPPORTED;  // the built-in scratch serves the plain selection
   const size_t blocks = (size_t)s.B * s.Hkv * s.M;  // every scratch array is per key/value head
   if (blocks > kStaticBlocks || blocks * (size_t)s.D > kStaticMeanElems) return BLOSSOM_ERR_TOO_LARGE;
   int dev = -1;

@@ -29,7 +29,8 @@ class DeviceProblem:
         self.params = binding.make_params(w.B, w.H, w.L, w.D, w.block, w.topk, w.window, w.dtype,
                                           sm_scale=sm_scale, stis_mode=w.stis_mode,
                                           stis_block=w.stis_block, cmp_block=w.cmp_block,
-                                          cmp_stride=w.cmp_stride, kv_heads=w.kv_heads or w.H)
+                                          cmp_stride=w.cmp_stride, kv_heads=w.kv_heads or w.H,
+                                          select_mode=w.per_query)
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):
@@ -38,7 +39,8 @@ class DeviceProblem:
         e = lambda: torch.empty(shape, dtype=self.dt, device=dev)  # noqa: E731
         hkv = w.kv_heads or w.H   # k, v, dk, dv and the selection are per key/value head
         ekv = lambda: torch.empty((w.B, hkv, w.L, w.D), dtype=self.dt, device=dev)  # noqa: E731
-        self.idx = torch.empty((w.B, hkv, w.n_blocks, w.topk), dtype=torch.int32, device=dev)
+        rows = w.L if w.per_query else w.n_blocks   # one index row per position or per query block
+        self.idx = torch.empty((w.B, hkv, rows, w.topk), dtype=torch.int32, device=dev)
         self.out = e()
         self.out_lt = e() if training else None
         self.out_st = e() if training else None

@@ -29,7 +29,11 @@ def _grouped(w):
 
 def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
-    if _grouped(w):
+    pq = bool(getattr(w, "per_query", 0))
+    if pq:
+        ref_idx, scores = oracle.select_blocks_per_query(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
+                                                         return_scores=True)
+    elif _grouped(w):
         ref_idx, scores = oracle.select_blocks_gqa(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
                                                    return_scores=True, cmp_block=w.cmp_block,
                                                    cmp_stride=w.cmp_stride)
@@ -44,11 +48,17 @@ def check_indices(w, gpu_idx, sm_scale=None):
     bad = np.argwhere((gpu_idx != ref_idx).any(-1))
     forgiven = 0
     for n, h, b in bad:
-        S = scores[n, h, b, :b]
-        ref_sel = [j for j in ref_idx[n, h, b] if 0 <= j < b]
-        gpu_sel = [j for j in gpu_idx[n, h, b] if 0 <= j < b]
+        if pq:          # a row per position t (= b here): its candidates are the blocks before t's block
+            t, b = b, b // w.block
+            S = scores[n, h, t, :b]
+            ref_row, gpu_row = ref_idx[n, h, t], gpu_idx[n, h, t]
+        else:
+            S = scores[n, h, b, :b]
+            ref_row, gpu_row = ref_idx[n, h, b], gpu_idx[n, h, b]
+        ref_sel = [j for j in ref_row if 0 <= j < b]
+        gpu_sel = [j for j in gpu_row if 0 <= j < b]
         # structure must still be valid
-        g = [int(j) for j in gpu_idx[n, h, b] if j >= 0]
+        g = [int(j) for j in gpu_row if j >= 0]
         assert g == sorted(set(g)) and g[-1] == b and len(g) == len(ref_sel) + 1, (n, h, b, g)
         dropped = np.setdiff1d(np.arange(b), ref_sel)
         kept_min = S[ref_sel].min()
@@ -72,13 +82,14 @@ def check_forward_backward(w, res, sm_scale=None, backward=True):
     """res: dict of numpy arrays from the CUDA path.  Returns a dict of max-abs errors."""
     forgiven = check_indices(w, res["idx"], sm_scale)
     fwd_fn, bwd_fn = (oracle.forward_gqa, oracle.backward_gqa) if _grouped(w) else (oracle.forward, oracle.backward)
+    kw = {"per_query": True} if getattr(w, "per_query", 0) else {}
     ref = fwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
-                 idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block)
+                 idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block, **kw)
     errs = {"near_tie_rows": forgiven}
     keys = ["out", "out_lt", "out_st", "lse"]
     if backward:
         ref.update(bwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, ref, w.dout,
-                          w.seq_lens, sm_scale, stis_mode=w.stis_mode, stis_block=w.stis_block))
+                          w.seq_lens, sm_scale, stis_mode=w.stis_mode, stis_block=w.stis_block, **kw))
         keys += ["dq", "dk", "dv", "dgate"]
     for key in keys:
         if res.get(key) is None:

@@ -540,3 +540,25 @@ def test_a_wait_that_cannot_complete_is_reported_and_the_context_stays_usable(ru
     w = workloads.make("after-timeout", "bf16", 2, 2, 300, 64, 32, 3, 50, seed=53)
     _, res = run(runner, w)                    # tensor memory was freed, barriers work, results are right
     print(check_forward_backward(w, res))
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens,power_law", [
+    (64, 32, 2, 2, 8, 2, 16, None, False),
+    (200, 32, 2, 2, 16, 4, 32, [200, 5, 77, 0], False),      # padded, ragged last block
+    (300, 64, 4, 2, 32, 4, 40, [300, 131], False),           # grouped heads share a per-position selection
+    (257, 64, 2, 2, 64, 3, 8, None, True),                   # with the power-law short-term mask
+    (1024, 64, 2, 2, 64, 8, 64, [1024, 700], False),
+])
+def test_selection_per_query_position(runner, dtype, L, D, H, Hkv, block, topk, window, lens, power_law):
+    """select_mode 1 (Eq. 13 as the paper prints it: every query position keeps its own top-k
+    blocks): indices, forward and backward against the oracle."""
+    B = len(lens) if lens else 2
+    w = workloads.make("per-query", dtype, B, H, L, D, block, topk, window, seed=59, kv_heads=Hkv if Hkv != H else 0,
+                       stis_mode=1 if power_law else 0)
+    w.per_query = 1
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    assert res["idx"].shape == (B, Hkv, L, topk)
+    print(check_forward_backward(w, res))
