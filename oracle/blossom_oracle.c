@@ -12,7 +12,8 @@
  *
  *   block splitting      Eq. 8  with l = s = l' = Bk (non-overlapping blocks,
  *                               0-based half-open, ragged last block kept)
- *   block compression    Eq. 9  with phi := mean over the valid keys of a block
+ *   block compression    Eq. 9  with phi := mean over the valid keys of a block, or a learnable
+ *                               softmax pooling over the block's positions (phi_weight)
  *   importance scoring   Eq. 10 softmax over the strictly-past live blocks,
  *                               logits scaled by sm_scale
  *   score sharing        Eq. 12 rule (sum of the probabilities of everyone who
@@ -66,9 +67,14 @@ int blossom_oracle_threads(void) {
 #endif
 }
 
+/* Eq. 9's learnable summary, in the one-layer form this oracle takes: a softmax pooling over the
+ * positions of a block, k~ = sum_i w_i k_i / sum_i w_i over the block's valid keys with
+ * w_i = exp(phi[i]), i the position inside the block.  phi == NULL (or all zeros) is the mean. */
+static double phi_weight(const double *phi, int i) { return phi ? exp(phi[i]) : 1.0; }
+
 /* ---- selection for one (n,h) unit: Eq. 8-10, 12, 13 --------------------- */
 static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0,
-                        const double *q, const double *k, int32_t *idx,
+                        const double *q, const double *k, const double *phi, int32_t *idx,
                         double *scores /* [M][M] or NULL */) {
   const int M = n_blocks(L, Bk);
   double *ktil = (double *)calloc((size_t)M * D, sizeof(double));
@@ -81,13 +87,16 @@ static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0,
   /* Eq. 8 + Eq. 9: block j = [j*Bk, min((j+1)*Bk, L)), summary = mean of its valid keys */
   for (int j = 0; j < M; ++j) {
     int lo = imax(j * Bk, pad0), hi = imin((j + 1) * Bk, L), cnt = 0;
+    double wsum = 0.0;
     for (int p = lo; p < hi; ++p) {
-      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] += k[(size_t)p * D + c];
+      const double w = phi_weight(phi, p - j * Bk);
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] += w * k[(size_t)p * D + c];
+      wsum += w;
       ++cnt;
     }
     live[j] = cnt > 0;
     if (cnt > 0)
-      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] /= (double)cnt;
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] /= wsum;
   }
 
   for (int b = 0; b < M; ++b) {
@@ -148,7 +157,7 @@ static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0,
 
 int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double scale,
                           const double *q, const double *k, const int32_t *seq_lens,
-                          int32_t *idx, double *scores) {
+                          const double *phi /* [Bk] or NULL */, int32_t *idx, double *scores) {
   if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
   const int M = n_blocks(L, Bk);
 #pragma omp parallel for collapse(2) schedule(dynamic)
@@ -158,7 +167,7 @@ int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double s
       int len = seq_lens ? seq_lens[n] : L;
       if (len < 0) len = 0;
       if (len > L) len = L;
-      select_unit(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D,
+      select_unit(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D, phi,
                   idx + u * M * topk, scores ? scores + u * M * M : NULL);
     }
   return 0;
@@ -170,7 +179,7 @@ int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double s
  * t) and keeps the top_k - 1 largest probabilities, ties to the lower index, plus its own block b.
  * idx is [L][topk] (one row per position, -1 rows for padding), probs [L][M] optional. */
 static void select_unit_pq(int L, int D, int Bk, int topk, double scale, int pad0,
-                           const double *q, const double *k, int32_t *idx, double *probs) {
+                           const double *q, const double *k, const double *phi, int32_t *idx, double *probs) {
   const int M = n_blocks(L, Bk);
   double *ktil = (double *)calloc((size_t)M * D, sizeof(double));
   int *live = (int *)calloc((size_t)M, sizeof(int));
@@ -178,13 +187,16 @@ static void select_unit_pq(int L, int D, int Bk, int topk, double scale, int pad
   char *taken = (char *)malloc((size_t)M);
   for (int j = 0; j < M; ++j) { /* Eq. 8 + Eq. 9 */
     int lo = imax(j * Bk, pad0), hi = imin((j + 1) * Bk, L), cnt = 0;
+    double wsum = 0.0;
     for (int p = lo; p < hi; ++p) {
-      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] += k[(size_t)p * D + c];
+      const double w = phi_weight(phi, p - j * Bk);
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] += w * k[(size_t)p * D + c];
+      wsum += w;
       ++cnt;
     }
     live[j] = cnt > 0;
     if (cnt > 0)
-      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] /= (double)cnt;
+      for (int c = 0; c < D; ++c) ktil[(size_t)j * D + c] /= wsum;
   }
   for (int t = 0; t < L; ++t) {
     int32_t *row = idx + (size_t)t * topk;
@@ -231,7 +243,7 @@ static void select_unit_pq(int L, int D, int Bk, int topk, double scale, int pad
 
 int blossom_oracle_select_pq(int B, int H, int L, int D, int Bk, int topk, double scale,
                              const double *q, const double *k, const int32_t *seq_lens,
-                             int32_t *idx, double *probs) {
+                             const double *phi /* [Bk] or NULL */, int32_t *idx, double *probs) {
   if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
   const int M = n_blocks(L, Bk);
 #pragma omp parallel for collapse(2) schedule(dynamic)
@@ -241,7 +253,7 @@ int blossom_oracle_select_pq(int B, int H, int L, int D, int Bk, int topk, doubl
       int len = seq_lens ? seq_lens[n] : L;
       if (len < 0) len = 0;
       if (len > L) len = L;
-      select_unit_pq(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D,
+      select_unit_pq(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D, phi,
                      idx + u * L * topk, probs ? probs + u * L * M : NULL);
     }
   return 0;
@@ -258,8 +270,8 @@ int blossom_oracle_select_pq(int B, int H, int L, int D, int Bk, int topk, doubl
  * terms whose index is out of range or not a candidate being zero.  Eq. 13 as in select_unit.
  * scores_cmp [M][Mc] and scores [M][M] are optional outputs. */
 static void select_unit_cmp(int L, int D, int Bk, int topk, int l, int s, double scale, int pad0,
-                            const double *q, const double *k, int32_t *idx, double *scores,
-                            double *scores_cmp) {
+                            const double *q, const double *k, const double *phi, int32_t *idx,
+                            double *scores, double *scores_cmp) {
   const int M = n_blocks(L, Bk);
   const int Mc = L >= l ? (L - l) / s + 1 : 0;
   const int rs = Bk / s, rl = l / s;
@@ -272,13 +284,16 @@ static void select_unit_cmp(int L, int D, int Bk, int topk, int l, int s, double
 
   for (int i = 0; i < Mc; ++i) { /* Eq. 8 + Eq. 9 */
     int lo = imax(i * s, pad0), hi = i * s + l, cnt = 0;
+    double wsum = 0.0;
     for (int p = lo; p < hi; ++p) {
-      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] += k[(size_t)p * D + c];
+      const double w = phi_weight(phi, p - i * s);
+      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] += w * k[(size_t)p * D + c];
+      wsum += w;
       ++cnt;
     }
     livec[i] = cnt > 0;
     if (cnt > 0)
-      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] /= (double)cnt;
+      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] /= wsum;
   }
 
   for (int b = 0; b < M; ++b) {
@@ -358,8 +373,8 @@ static void select_unit_cmp(int L, int D, int Bk, int topk, int l, int s, double
 
 int blossom_oracle_select_cmp(int B, int H, int L, int D, int Bk, int topk, int l, int s,
                               double scale, const double *q, const double *k,
-                              const int32_t *seq_lens, int32_t *idx, double *scores,
-                              double *scores_cmp) {
+                              const int32_t *seq_lens, const double *phi /* [l] or NULL */,
+                              int32_t *idx, double *scores, double *scores_cmp) {
   if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
   if (l < 1 || s < 1 || l % s || Bk % s) return 1;
   const int M = n_blocks(L, Bk);
@@ -371,7 +386,7 @@ int blossom_oracle_select_cmp(int B, int H, int L, int D, int Bk, int topk, int 
       int len = seq_lens ? seq_lens[n] : L;
       if (len < 0) len = 0;
       if (len > L) len = L;
-      select_unit_cmp(L, D, Bk, topk, l, s, scale, L - len, q + u * L * D, k + u * L * D,
+      select_unit_cmp(L, D, Bk, topk, l, s, scale, L - len, q + u * L * D, k + u * L * D, phi,
                       idx + u * M * topk, scores ? scores + u * M * M : NULL,
                       scores_cmp ? scores_cmp + u * M * Mc : NULL);
     }

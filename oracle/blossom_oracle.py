@@ -48,12 +48,12 @@ def _load():
         d = ctypes.c_double
         lib.blossom_oracle_threads.restype = i
         lib.blossom_oracle_select.restype = i
-        lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp]
+        lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
         lib.blossom_oracle_select_cmp.restype = i
-        lib.blossom_oracle_select_cmp.argtypes = [i, i, i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp, _dp]
+        lib.blossom_oracle_select_cmp.argtypes = [i, i, i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp, _dp]
         lib.blossom_oracle_forward.restype = i
         lib.blossom_oracle_select_pq.restype = i
-        lib.blossom_oracle_select_pq.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _ip, _dp]
+        lib.blossom_oracle_select_pq.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
         lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
         lib.blossom_oracle_backward.restype = i
@@ -84,27 +84,42 @@ def _lens(seq_lens, B):
     return s
 
 
+def _phi(phi_logits, length):
+    """The logits of the learnable block summary (softmax pooling over a block's positions), or
+    None for the mean."""
+    if phi_logits is None:
+        return None
+    p = np.ascontiguousarray(np.asarray(phi_logits, dtype=np.float64))
+    assert p.shape == (length,)
+    return p
+
+
 def _scale(sm_scale, D):
     return float(sm_scale) if sm_scale else 1.0 / math.sqrt(D)
 
 
-def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False):
-    """Eq. 8-10, 12, 13: block summaries, block scores and the top-k block set."""
+def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False, phi_logits=None):
+    """Eq. 8-10, 12, 13: block summaries, block scores and the top-k block set.
+
+    ``phi_logits`` ``[block]``: Eq. 9's learnable summary as a softmax pooling over the positions of
+    a block (weights exp(phi_logits[i]) over the valid keys); None = the mean."""
     q, k = _f64(q), _f64(k)
     B, H, L, D = q.shape
     M = -(-L // block)
     idx = np.empty((B, H, M, topk), dtype=np.int32)
     scores = np.zeros((B, H, M, M), dtype=np.float64) if return_scores else None
     sl = _lens(seq_lens, B)
+    ph = _phi(phi_logits, block)
     rc = _load().blossom_oracle_select(B, H, L, D, block, topk, _scale(sm_scale, D),
-                                       _ptr(q, _dp), _ptr(k, _dp), _ptr(sl, _ip),
+                                       _ptr(q, _dp), _ptr(k, _dp), _ptr(sl, _ip), _ptr(ph, _dp),
                                        _ptr(idx, _ip), _ptr(scores, _dp))
     if rc:
         raise ValueError("blossom_oracle_select: bad arguments")
     return (idx, scores) if return_scores else idx
 
 
-def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False):
+def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False,
+                            phi_logits=None):
     """Eq. 8-10, 13 as printed: one selection per query position.  k may have fewer heads than q
     (grouped heads: the probabilities of a group's heads are summed, Eq. 12, and the group's
     queries at one position share the selection).  Returns idx ``[B,Hkv,L,topk]`` (ascending, -1
@@ -118,8 +133,10 @@ def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, ret
     probs = np.zeros((B, H, L, M), dtype=np.float64) if (return_scores or G > 1) else None
     sl = _lens(seq_lens, B)
     kk = np.ascontiguousarray(np.repeat(k, G, axis=1))
+    ph = _phi(phi_logits, block)
     rc = _load().blossom_oracle_select_pq(B, H, L, D, block, topk, _scale(sm_scale, D), _ptr(q, _dp),
-                                          _ptr(kk, _dp), _ptr(sl, _ip), _ptr(idx, _ip), _ptr(probs, _dp))
+                                          _ptr(kk, _dp), _ptr(sl, _ip), _ptr(ph, _dp), _ptr(idx, _ip),
+                                          _ptr(probs, _dp))
     if rc:
         raise ValueError("blossom_oracle_select_pq: bad arguments")
     if G == 1:
@@ -140,7 +157,7 @@ def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, ret
 
 
 def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, sm_scale=None,
-                      return_scores=False):
+                      return_scores=False, phi_logits=None):
     """Eq. 8-11, 13 with overlapping compression blocks (length ``cmp_block``, stride
     ``cmp_stride``) scored and mapped onto selection blocks of ``block`` positions.
 
@@ -160,9 +177,10 @@ def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, s
         sc_arg = None
     else:
         sc_arg = scores_cmp
+    ph = _phi(phi_logits, int(cmp_block))
     rc = _load().blossom_oracle_select_cmp(B, H, L, D, block, topk, int(cmp_block), int(cmp_stride),
                                            _scale(sm_scale, D), _ptr(q, _dp), _ptr(k, _dp),
-                                           _ptr(sl, _ip), _ptr(idx, _ip), _ptr(scores, _dp),
+                                           _ptr(sl, _ip), _ptr(ph, _dp), _ptr(idx, _ip), _ptr(scores, _dp),
                                            _ptr(sc_arg, _dp))
     if rc:
         raise ValueError("blossom_oracle_select_cmp: bad arguments")
@@ -255,7 +273,7 @@ def _group(H, Hkv):
 
 
 def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False,
-                      cmp_block=0, cmp_stride=0):
+                      cmp_block=0, cmp_stride=0, phi_logits=None):
     """q ``[B,H,L,D]``, k ``[B,Hkv,L,D]`` -> idx ``[B,Hkv,M,topk]`` from group-summed scores.
 
     With ``cmp_block`` / ``cmp_stride`` the per-head scores are those of the overlapping
@@ -268,10 +286,11 @@ def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_sc
     M = -(-L // block)
     if cmp_block or cmp_stride:
         _, per_head, _ = select_blocks_cmp(q, np.repeat(k, G, axis=1), block, topk, cmp_block or block,
-                                           cmp_stride or block, seq_lens, sm_scale, return_scores=True)
+                                           cmp_stride or block, seq_lens, sm_scale, return_scores=True,
+                                           phi_logits=phi_logits)
     else:
         _, per_head = select_blocks(q, np.repeat(k, G, axis=1), block, topk, seq_lens, sm_scale,
-                                    return_scores=True)
+                                    return_scores=True, phi_logits=phi_logits)
     scores = per_head.reshape(B, Hkv, G, M, M).sum(axis=2)            # Eq. 12
     idx = np.full((B, Hkv, M, topk), -1, dtype=np.int32)
     for n in range(B):
