@@ -88,6 +88,13 @@ typedef struct {
   int32_t cmp_stride;  /* s: their stride; 0 = block_size; must divide cmp_block and block_size  */
   int64_t kv_stride_b, kv_stride_h, kv_stride_l; /* element strides of k, v, dk, dv; all 0 = the
                         * strides above if kv_heads == heads, else contiguous [B][kv_heads][L][D] */
+  const float *phi_logits; /* DEVICE pointer or NULL.  Eq. 9's learnable block summary, in the
+                        * one-layer form this library takes: a softmax pooling over the positions
+                        * of a scored block, summary = sum_i w_i k_i / sum_i w_i over the block's
+                        * valid keys, w_i = exp(phi_logits[i]), i the position inside the block;
+                        * float [cmp_block] (or [block_size] without compression blocks).  NULL =
+                        * the mean.  Only the selection reads it, and no gradient reaches it (the
+                        * top-k is piecewise constant), so it has no entry in the backward.       */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

@@ -63,7 +63,7 @@ def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True):
 class _BlossomAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
-                stis_mode, stis_block, cmp_block, cmp_stride, per_query=0):
+                stis_mode, stis_block, cmp_block, cmp_stride, per_query=0, phi_logits=None):
         seq_lens = check_arguments(q, k, v, gate_logits, seq_lens)
         B, H, L, D = q.shape
         Hkv = k.shape[1]
@@ -78,7 +78,8 @@ class _BlossomAttention(torch.autograd.Function):
         params = binding.make_params(B, H, L, D, block_size, top_k, window, _DT[q.dtype],
                                      sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
                                      stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride,
-                                     kv_heads=Hkv, kv_strides=k.stride()[:3], select_mode=int(per_query))
+                                     kv_heads=Hkv, kv_strides=k.stride()[:3], select_mode=int(per_query),
+                                     phi_logits=phi_logits)
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -92,6 +93,7 @@ class _BlossomAttention(torch.autograd.Function):
         binding.blossom_attn_fwd(params, q, k, v, gate, seq_lens, idx, 0, out, out_lt, out_st, lse,
                                  workspace)
         ctx.params, ctx.workspace, ctx.seq_lens = params, workspace, seq_lens
+        ctx.phi_logits = phi_logits  # the params hold its address: keep it alive until the backward
         ctx.gate_dtype = gate_logits.dtype
         ctx.save_for_backward(q, k, v, gate, idx, out_lt, out_st, lse)
         ctx.mark_non_differentiable(idx)
@@ -106,12 +108,12 @@ class _BlossomAttention(torch.autograd.Function):
         dgate = torch.empty((q.shape[1], 2), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
-        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 10
+        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 11
 
 
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
                       return_indices=False, short_term="window", mask_block=1, cmp_block=0,
-                      cmp_stride=0, select_per_query=False):
+                      cmp_stride=0, select_per_query=False, phi_logits=None):
     """Gated two-branch sparse attention of q [B, H, L, D] and k, v [B, Hkv, L, D] (float32 or
     bfloat16, CUDA; Hkv divides H: with Hkv < H the query heads of a group share key/value head
     and selection, and the returned indices are [B, Hkv, M, top_k]).
@@ -127,11 +129,20 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     (Eq. 8, 11); 0 = the selection blocks themselves.
     select_per_query: one selection per query position (Eq. 13 as printed; indices [B, Hkv, L,
     top_k]) instead of one per query block; runs on the CUDA-core kernels.
+    phi_logits: optional float32 CUDA tensor [cmp_block or block_size]: Eq. 9's learnable block
+    summary as a softmax pooling over a block's positions (None = the mean).  It only steers the
+    selection, which is not differentiated, so it receives no gradient here.
     """
+    if phi_logits is not None:
+        n = int(cmp_block) or int(block_size)
+        if not (isinstance(phi_logits, torch.Tensor) and phi_logits.is_cuda and phi_logits.device == q.device
+                and phi_logits.dtype == torch.float32 and tuple(phi_logits.shape) == (n,)):
+            raise ValueError(f"phi_logits must be a float32 CUDA tensor of shape [{n}] on q's device")
+        phi_logits = phi_logits.detach().contiguous()
     if short_term not in ("window", "power-law"):
         raise ValueError("short_term must be 'window' or 'power-law'")
     out, idx = _BlossomAttention.apply(q, k, v, gate_logits, seq_lens, int(block_size), int(top_k),
                                        int(window), float(sm_scale),
                                        1 if short_term == "power-law" else 0, int(mask_block),
-                                       int(cmp_block), int(cmp_stride), int(bool(select_per_query)))
+                                       int(cmp_block), int(cmp_stride), int(bool(select_per_query)), phi_logits)
     return (out, idx) if return_indices else out

@@ -42,6 +42,7 @@ class blossom_params(ctypes.Structure):
         ("stis_mode", ctypes.c_int32), ("stis_block", ctypes.c_int32),
         ("cmp_block", ctypes.c_int32), ("cmp_stride", ctypes.c_int32),
         ("kv_stride_b", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64), ("kv_stride_l", ctypes.c_int64),
+        ("phi_logits", ctypes.c_void_p),
     ]
 
 
@@ -121,9 +122,10 @@ def _stream(stream):
 
 def make_params(batch, heads, seq_len, head_dim, block_size, top_k, window, dtype, sm_scale=0.0,
                 strides=None, kv_heads=None, causal=1, select_mode=0, stis_mode=0,
-                stis_block=1, cmp_block=0, cmp_stride=0, kv_strides=None) -> blossom_params:
+                stis_block=1, cmp_block=0, cmp_stride=0, kv_strides=None, phi_logits=None) -> blossom_params:
     """Fill a ``blossom_params``; ``strides`` = (stride_b, stride_h, stride_l) in elements,
-    default contiguous [B, H, L, D]."""
+    default contiguous [B, H, L, D].  ``phi_logits``: float32 device tensor (the caller keeps it
+    alive) or None."""
     if strides is None:
         strides = (heads * seq_len * head_dim, seq_len * head_dim, head_dim)
     d = {"fp32": DTYPE_FP32, "bf16": DTYPE_BF16}.get(dtype, dtype)
@@ -131,7 +133,8 @@ def make_params(batch, heads, seq_len, head_dim, block_size, top_k, window, dtyp
                           block_size, top_k, window, causal, select_mode, d, float(sm_scale),
                           int(strides[0]), int(strides[1]), int(strides[2]), int(stis_mode),
                           int(stis_block), int(cmp_block), int(cmp_stride),
-                          *((0, 0, 0) if kv_strides is None else [int(x) for x in kv_strides]))
+                          *((0, 0, 0) if kv_strides is None else [int(x) for x in kv_strides]),
+                          _ptr(phi_logits))
 
 
 def blossom_status_string(status) -> str:

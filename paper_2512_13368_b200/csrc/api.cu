@@ -137,6 +137,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;
   s.Hkv = p->kv_heads; s.G = p->heads / p->kv_heads;
   s.pq = p->select_mode;
+  s.phi = p->phi_logits;
+  if (reinterpret_cast<uintptr_t>(s.phi) % 4) return BLOSSOM_ERR_INVALID_ARG;
   if (s.pq && s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // per-position selection scores the selection blocks themselves
   if (kv_given) {
     s.ksb = p->kv_stride_b; s.ksh = p->kv_stride_h; s.ksl = p->kv_stride_l;

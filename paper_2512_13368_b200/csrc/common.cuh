@@ -19,6 +19,7 @@ struct Shape {
   int64_t sb, sh, sl;  // element strides of q-shaped tensors
   int Hkv, G;             // key/value heads and query heads per key/value head (H = Hkv * G)
   int pq;                 // 1: one selection per query position (block_idx is [B][Hkv][L][top_k])
+  const float *phi;       // logits of the learnable block summary (Eq. 9) or nullptr = the mean
   int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
 };
 

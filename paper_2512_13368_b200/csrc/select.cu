@@ -95,8 +95,8 @@ struct Raw8<float> {
 // bf16, two of fp32) of every (32 / (D / 8))-th row and sums them in a fixed order with eight rows
 // in flight (kept as loaded until they are added); the lanes that share columns are combined by
 // shuffles in a fixed tree.
-template <typename T, int D>
-__global__ void __launch_bounds__(256, 4) summary_kernel(Shape sh, SelGeom g, const T *__restrict__ k,
+template <typename T, int D, bool PHI>
+__global__ void __launch_bounds__(256, PHI ? 2 : 4) summary_kernel(Shape sh, SelGeom g, const T *__restrict__ k,
                                                          const int32_t *__restrict__ seq_lens,
                                                          double *__restrict__ mean,
                                                          int32_t *__restrict__ live,
@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(256, 4) summary_kernel(Shape sh, SelGeom g, co
   const int lo = max(c * g.s, pad0), hi = min(c * g.s + g.l, sh.L);
   const int sub = lane / LPR, col = (lane % LPR) * 8;
   const T *base = k + row_offset_kv(sh, n, hk, 0) + col;
-  double a[8];
+  double a[8], wsum = 0.0;  // weighted column sums and the sum of the weights (Eq. 9)
 #pragma unroll
   for (int e = 0; e < 8; ++e) a[e] = 0.0;
   for (int p = lo + sub; p < hi; p += NF * RPI) {
@@ -128,12 +128,25 @@ __global__ void __launch_bounds__(256, 4) summary_kernel(Shape sh, SelGeom g, co
       if (pp < hi) x[r].load(base + (int64_t)pp * sh.ksl);
       else x[r].zero();
     }
+    if (PHI) {  // learnable summary: weight exp(phi[i]) for position i of the block
 #pragma unroll
-    for (int r = 0; r < NF; ++r) {
-      float f[8];
-      x[r].unpack(f);
+      for (int r = 0; r < NF; ++r) {
+        const int pp = p + r * RPI;
+        const double w = pp < hi ? exp((double)sh.phi[pp - c * g.s]) : 0.0;
+        float f[8];
+        x[r].unpack(f);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) a[e] += (double)f[e];
+        for (int e = 0; e < 8; ++e) a[e] = fma(w, (double)f[e], a[e]);
+        wsum += w;
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < NF; ++r) {
+        float f[8];
+        x[r].unpack(f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[e] += (double)f[e];
+      }
     }
   }
 #pragma unroll
@@ -141,13 +154,19 @@ __global__ void __launch_bounds__(256, 4) summary_kernel(Shape sh, SelGeom g, co
 #pragma unroll
     for (int e = 0; e < 8; ++e) a[e] += __shfl_xor_sync(0xffffffffu, a[e], o);
   const int cnt = max(hi - lo, 0);
+  if (PHI) {
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+  } else {
+    wsum = (double)cnt;
+  }
   float sq = 0.f;
   if (sub == 0) {
     double m[8];
     float f[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      m[e] = cnt > 0 ? a[e] / (double)cnt : 0.0;
+      m[e] = cnt > 0 ? a[e] / wsum : 0.0;
       f[e] = (float)m[e];
       sq = fmaf(f[e], f[e], sq);
     }
@@ -781,8 +800,9 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
   const int64_t units = (int64_t)sh.B * sh.Hkv;
   if (g.n > 0) {
     LaunchScope ls(K_SUMMARY, st);
-    summary_kernel<T, D><<<(unsigned)((units * g.n + 7) / 8), 256, 0, st>>>(sh, g, k, seq_lens, w.mean, w.live,
-                                                                            w.mean32, w.norm, w.count);
+    auto summary = sh.phi ? summary_kernel<T, D, true> : summary_kernel<T, D, false>;
+    summary<<<(unsigned)((units * g.n + 7) / 8), 256, 0, st>>>(sh, g, k, seq_lens, w.mean, w.live, w.mean32, w.norm,
+                                                               w.count);
   } else if (cudaMemsetAsync(w.count, 0, sizeof(int32_t), st) != cudaSuccess) {
     return BLOSSOM_ERR_CUDA;
   }

@@ -26,11 +26,14 @@ class DeviceProblem:
         self.seq_lens = None
         if w.seq_lens is not None:
             self.seq_lens = torch.from_numpy(w.seq_lens.astype(np.int32)).to(self.device)
+        self.phi = None   # logits of the learnable block summary, kept alive here (the params hold its address)
+        if getattr(w, "phi_logits", None) is not None:
+            self.phi = torch.from_numpy(np.ascontiguousarray(w.phi_logits, dtype=np.float32)).to(self.device)
         self.params = binding.make_params(w.B, w.H, w.L, w.D, w.block, w.topk, w.window, w.dtype,
                                           sm_scale=sm_scale, stis_mode=w.stis_mode,
                                           stis_block=w.stis_block, cmp_block=w.cmp_block,
                                           cmp_stride=w.cmp_stride, kv_heads=w.kv_heads or w.H,
-                                          select_mode=w.per_query)
+                                          select_mode=w.per_query, phi_logits=self.phi)
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):

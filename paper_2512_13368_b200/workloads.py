@@ -65,6 +65,7 @@ class Workload:
     cmp_stride: int = 0   # and its stride s (0 = block)
     kv_heads: int = 0     # key/value heads (0 = H): k, v are [B, kv_heads, L, D]
     per_query: int = 0    # 1: one selection per query position (Eq. 13 as printed) instead of per query block
+    phi_logits: np.ndarray | None = field(default=None, repr=False)  # learnable block summary (Eq. 9) or None = mean
 
     @property
     def n_blocks(self) -> int:
@@ -85,7 +86,7 @@ class Workload:
                         self.q[n:n + 1, hq].copy(), self.k[n:n + 1, h:h + 1].copy(),
                         self.v[n:n + 1, h:h + 1].copy(), self.gate[hq].copy(),
                         self.dout[n:n + 1, hq].copy(), sl, self.stis_mode, self.stis_block,
-                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0, self.per_query)
+                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0, self.per_query, self.phi_logits)
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,

@@ -30,20 +30,21 @@ def _grouped(w):
 def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
     pq = bool(getattr(w, "per_query", 0))
+    phi = getattr(w, "phi_logits", None)
     if pq:
         ref_idx, scores = oracle.select_blocks_per_query(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
-                                                         return_scores=True)
+                                                         return_scores=True, phi_logits=phi)
     elif _grouped(w):
         ref_idx, scores = oracle.select_blocks_gqa(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
                                                    return_scores=True, cmp_block=w.cmp_block,
-                                                   cmp_stride=w.cmp_stride)
+                                                   cmp_stride=w.cmp_stride, phi_logits=phi)
     elif w.cmp_block or w.cmp_stride:
         ref_idx, scores, _ = oracle.select_blocks_cmp(w.q, w.k, w.block, w.topk, w.cmp_block or w.block,
                                                       w.cmp_stride or w.block, w.seq_lens, sm_scale,
-                                                      return_scores=True)
+                                                      return_scores=True, phi_logits=phi)
     else:
         ref_idx, scores = oracle.select_blocks(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
-                                                return_scores=True)
+                                                return_scores=True, phi_logits=phi)
     assert gpu_idx.shape == ref_idx.shape and gpu_idx.dtype == np.int32
     bad = np.argwhere((gpu_idx != ref_idx).any(-1))
     forgiven = 0

@@ -562,3 +562,32 @@ def test_selection_per_query_position(runner, dtype, L, D, H, Hkv, block, topk, 
     _, res = run(runner, w)
     assert res["idx"].shape == (B, Hkv, L, topk)
     print(check_forward_backward(w, res))
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,H,Hkv,block,topk,cmp,lens,per_query", [
+    (200, 32, 2, 2, 16, 4, None, [200, 5, 77], False),
+    (512, 64, 4, 2, 32, 4, (64, 16), [512, 200], False),     # overlapping blocks, grouped heads
+    (1024, 64, 2, 2, 64, 6, None, None, False),
+    (192, 32, 2, 2, 16, 3, None, [192, 40], True),           # with a selection per query position
+])
+def test_learnable_block_summary(runner, dtype, L, D, H, Hkv, block, topk, cmp, lens, per_query):
+    """Eq. 9's learnable summary (softmax pooling over a block's positions, logits given by the
+    caller) behind the selection: indices bit-checked against the oracle, attention on them."""
+    B = len(lens) if lens else 2
+    w = workloads.make("phi", dtype, B, H, L, D, block, topk, 24, seed=61, kv_heads=Hkv if Hkv != H else 0)
+    if cmp:
+        w.cmp_block, w.cmp_stride = cmp
+    w.per_query = int(per_query)
+    w.phi_logits = np.random.default_rng(3).standard_normal(cmp[0] if cmp else block).astype(np.float32)
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    print(check_forward_backward(w, res))
+    # the logits matter: the mean selects something else somewhere
+    w0 = workloads.make("phi", dtype, B, H, L, D, block, topk, 24, seed=61, kv_heads=Hkv if Hkv != H else 0)
+    if cmp:
+        w0.cmp_block, w0.cmp_stride = cmp
+    w0.per_query, w0.seq_lens = w.per_query, w.seq_lens
+    _, res0 = run(runner, w0, backward=False)
+    assert not np.array_equal(res0["idx"], res["idx"])
