@@ -29,7 +29,8 @@
  *   power-law mask       Eq. 15 all three cases (stis_mode 1), causal side:
  *                               window, block-index distance a power of two,
  *                               the last blk positions
- *   gate combine         Eq. 19 with alpha_h = sigmoid(a[h][0] - a[h][1])
+ *   gate combine         Eq. 19 with alpha_h = sigmoid(a[h][0] - a[h][1]), or Eq. 18's
+ *                               input-dependent gate with a one-layer F_o (gate_mode 1)
  *   backward             chain rule through Eq. 19, Eq. 16/17 and Eq. 1 with
  *                        the selection frozen (top-k is piecewise constant)
  *
@@ -460,8 +461,12 @@ static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 
 /* per_query = 0: idx is [B][H][M][topk], one row per query block; 1: [B][H][L][topk], one row per
  * query position (Eq. 13 as printed) */
+/* gate_mode = 0: gate is [H][2], alpha_h = sigmoid(a[h][0] - a[h][1]) for the whole head;
+ * 1: the input-dependent gate of Eq. 18 with a one-layer F_o: gate is [H][2 D + 1] = (w_lt[D],
+ * w_st[D], b) and alpha_t = sigmoid(<w_lt, O_lt,t> + <w_st, O_st,t> + b), one weight per token
+ * and head, broadcast over the head's channels in Eq. 19 */
 int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
-                           int stis_blk, int per_query, double scale,
+                           int stis_blk, int per_query, int gate_mode, double scale,
                            const double *q, const double *k, const double *v, const double *gate,
                            const int32_t *seq_lens, const int32_t *idx, double *out,
                            double *out_lt, double *out_st, double *lse) {
@@ -478,7 +483,8 @@ int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int win
       if (len > L) len = L;
       const int pad0 = L - len;
       const double *qu = q + u * L * D, *ku = k + u * L * D, *vu = v + u * L * D;
-      const double alpha = sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]); /* Eq. 18 reduced to a scalar */
+      const int GW = 2 * D + 1;
+      const double alpha_h = gate_mode ? 0.0 : sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]); /* Eq. 18 reduced to a scalar */
       int *keys = (int *)malloc(sizeof(int) * (size_t)(L + 1));
       double *sbuf = (double *)malloc(sizeof(double) * (size_t)(L + 1));
       double *oL = (double *)malloc(sizeof(double) * (size_t)D);
@@ -495,6 +501,12 @@ int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int win
           lL = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oL); /* Eq. 16 */
           nk = stis_keys(stis_mode, window, stis_blk, L, pad0, t, keys);
           lS = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oS); /* Eq. 17 */
+        }
+        double alpha = alpha_h;
+        if (gate_mode) { /* Eq. 18: F_o of the concatenated branch outputs, then the sigmoid */
+          double a = gate[h * GW + 2 * D];
+          for (int c = 0; c < D; ++c) a += gate[h * GW + c] * oL[c] + gate[h * GW + D + c] * oS[c];
+          alpha = sigmoid(a);
         }
         for (int c = 0; c < D; ++c) {
           if (out_lt) out_lt[ro + c] = oL[c];
@@ -539,7 +551,7 @@ static void attend_row_bwd(int D, double scale, const double *qt, const double *
 }
 
 int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
-                            int stis_blk, int per_query, double scale,
+                            int stis_blk, int per_query, int gate_mode, double scale,
                             const double *q, const double *k, const double *v, const double *gate,
                             const int32_t *seq_lens, const int32_t *idx, const double *out_lt,
                             const double *out_st, const double *lse, const double *dout,
@@ -548,7 +560,9 @@ int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int wi
   if (stis_mode < 0 || stis_mode > 1 || stis_blk < 1) return 1;
   const int M = n_blocks(L, Bk);
   const size_t BHL = (size_t)B * H * L;
-  double *dalpha_unit = (double *)calloc((size_t)B * H, sizeof(double));
+  const int GW = 2 * D + 1;
+  /* per (n, h): d alpha (scalar gate) or the gradient of (w_lt, w_st, b) (input-dependent gate) */
+  double *dalpha_unit = (double *)calloc((size_t)B * H * (gate_mode ? GW : 1), sizeof(double));
   memset(dq, 0, sizeof(double) * BHL * D);
   memset(dk, 0, sizeof(double) * BHL * D);
   memset(dv, 0, sizeof(double) * BHL * D);
@@ -562,17 +576,34 @@ int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int wi
       const int pad0 = L - len;
       const double *qu = q + u * L * D, *ku = k + u * L * D, *vu = v + u * L * D;
       double *dqu = dq + u * L * D, *dku = dk + u * L * D, *dvu = dv + u * L * D;
-      const double alpha = sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]);
+      const double alpha_h = gate_mode ? 0.0 : sigmoid(gate[h * 2 + 0] - gate[h * 2 + 1]);
       int *keys = (int *)malloc(sizeof(int) * (size_t)(L + 1));
       double *gL = (double *)malloc(sizeof(double) * (size_t)D);
       double *gS = (double *)malloc(sizeof(double) * (size_t)D);
       double dalpha = 0.0;
+      double *dw = gate_mode ? dalpha_unit + u * GW : NULL;
       for (int t = pad0; t < L; ++t) {
         size_t ro = (u * L + t) * (size_t)D;
+        double alpha = alpha_h, da_t = 0.0; /* d loss / d alpha of this row */
+        for (int c = 0; c < D; ++c) da_t += dout[ro + c] * (out_lt[ro + c] - out_st[ro + c]); /* Eq. 19 */
+        dalpha += da_t;
+        double cpre = 0.0; /* d loss / d (pre-activation of the gate) of this row */
+        if (gate_mode) {
+          double a = gate[h * GW + 2 * D];
+          for (int c = 0; c < D; ++c)
+            a += gate[h * GW + c] * out_lt[ro + c] + gate[h * GW + D + c] * out_st[ro + c];
+          alpha = sigmoid(a);
+          cpre = alpha * (1.0 - alpha) * da_t;
+          for (int c = 0; c < D; ++c) { /* F_o's parameters */
+            dw[c] += cpre * out_lt[ro + c];
+            dw[D + c] += cpre * out_st[ro + c];
+          }
+          dw[2 * D] += cpre;
+        }
         for (int c = 0; c < D; ++c) {
-          dalpha += dout[ro + c] * (out_lt[ro + c] - out_st[ro + c]); /* d/d alpha of Eq. 19 */
-          gL[c] = alpha * dout[ro + c];
-          gS[c] = (1.0 - alpha) * dout[ro + c];
+          /* through Eq. 19 directly and, with the input-dependent gate, through alpha as well */
+          gL[c] = alpha * dout[ro + c] + (gate_mode ? cpre * gate[h * GW + c] : 0.0);
+          gS[c] = (1.0 - alpha) * dout[ro + c] + (gate_mode ? cpre * gate[h * GW + D + c] : 0.0);
         }
         const int32_t *row = per_query ? idx + (u * L + (size_t)t) * topk
                                        : idx + (u * M + (size_t)(t / Bk)) * topk;
@@ -583,9 +614,19 @@ int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int wi
         attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[BHL + u * L + t],
                        out_st + ro, gS, dqu + (size_t)t * D, dku, dvu);
       }
-      dalpha_unit[u] = dalpha;
+      if (!gate_mode) dalpha_unit[u] = dalpha;
       free(keys); free(gL); free(gS);
     }
+  if (gate_mode) { /* sum the parameter gradients over the batch, in batch order */
+    for (int h = 0; h < H; ++h)
+      for (int c = 0; c < GW; ++c) {
+        double a = 0.0;
+        for (int n = 0; n < B; ++n) a += dalpha_unit[((size_t)n * H + h) * GW + c];
+        dgate[h * GW + c] = a;
+      }
+    free(dalpha_unit);
+    return 0;
+  }
   /* gate logits: alpha = sigmoid(a0 - a1)  =>  d a0 = alpha (1 - alpha) d alpha = - d a1 */
   for (int h = 0; h < H; ++h) {
     double da = 0.0;

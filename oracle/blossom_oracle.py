@@ -54,10 +54,10 @@ def _load():
         lib.blossom_oracle_forward.restype = i
         lib.blossom_oracle_select_pq.restype = i
         lib.blossom_oracle_select_pq.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
-        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
         lib.blossom_oracle_backward.restype = i
-        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                 _ip, _dp, _dp, _dp, _dp, _dp, _dp, _dp, _dp]
         _lib = lib
     return _lib
@@ -190,20 +190,22 @@ def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, s
 
 
 def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None,
-            stis_mode=0, stis_block=1, per_query=False):
+            stis_mode=0, stis_block=1, per_query=False, gate_mode=0):
     """Eq. 14, 16, 17, 19.  ``idx`` overrides the selection when given.
 
     ``stis_mode`` 0: the short-term branch is the causal window (Eq. 15, first case);
     1: the power-law mask (all of Eq. 15, causal side) with mask block ``stis_block``.
 
     ``per_query``: the selection is per query position, idx ``[B,H,L,topk]``.
+    ``gate_mode`` 1: Eq. 18's input-dependent gate with a one-layer F_o; gate is ``[H, 2 D + 1]`` =
+    (w_lt, w_st, b) per head and alpha_t = sigmoid(<w_lt, O_lt,t> + <w_st, O_st,t> + b).
 
     Returns a dict: out, out_lt, out_st ``[B,H,L,D]``, lse ``[2,B,H,L]``, idx.
     """
     q, k, v, gate = _f64(q), _f64(k), _f64(v), _f64(gate)
     B, H, L, D = q.shape
     M = -(-L // block)
-    assert gate.shape == (H, 2)
+    assert gate.shape == ((H, 2 * D + 1) if gate_mode else (H, 2))
     if idx is None:
         idx = (select_blocks_per_query if per_query else select_blocks)(q, k, block, topk, seq_lens, sm_scale)
     idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
@@ -214,7 +216,8 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     out_st = np.empty_like(q)
     lse = np.empty((2, B, H, L), dtype=np.float64)
     rc = _load().blossom_oracle_forward(B, H, L, D, block, topk, window, int(stis_mode),
-                                        int(stis_block), int(bool(per_query)), _scale(sm_scale, D),
+                                        int(stis_block), int(bool(per_query)), int(gate_mode),
+                                        _scale(sm_scale, D),
                                         _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp), _ptr(gate, _dp),
                                         _ptr(sl, _ip), _ptr(idx, _ip), _ptr(out, _dp),
                                         _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp))
@@ -224,10 +227,10 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
 
 
 def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None,
-             stis_mode=0, stis_block=1, per_query=False):
+             stis_mode=0, stis_block=1, per_query=False, gate_mode=0):
     """Gradients of sum(out * dout) with the selection frozen.
 
-    ``fwd`` is the dict ``forward`` returned.  Returns dq, dk, dv, dgate ``[H,2]``.
+    ``fwd`` is the dict ``forward`` returned.  Returns dq, dk, dv, dgate (the shape of gate).
     """
     q, k, v, gate, dout = _f64(q), _f64(k), _f64(v), _f64(gate), _f64(dout)
     B, H, L, D = q.shape
@@ -235,9 +238,10 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
     idx = np.ascontiguousarray(fwd["idx"], dtype=np.int32)
     out_lt, out_st, lse = _f64(fwd["out_lt"]), _f64(fwd["out_st"]), _f64(fwd["lse"])
     dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
-    dgate = np.empty((H, 2), dtype=np.float64)
+    dgate = np.empty(gate.shape, dtype=np.float64)
     rc = _load().blossom_oracle_backward(B, H, L, D, block, topk, window, int(stis_mode),
-                                         int(stis_block), int(bool(per_query)), _scale(sm_scale, D),
+                                         int(stis_block), int(bool(per_query)), int(gate_mode),
+                                         _scale(sm_scale, D),
                                          _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp),
                                          _ptr(gate, _dp), _ptr(sl, _ip), _ptr(idx, _ip),
                                          _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp),
@@ -249,12 +253,12 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
 
 
 def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm_scale=None,
-                     idx=None, stis_mode=0, stis_block=1, per_query=False):
+                     idx=None, stis_mode=0, stis_block=1, per_query=False, gate_mode=0):
     """Convenience: forward then backward; returns the two dicts merged."""
     f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx, stis_mode, stis_block,
-                per_query)
+                per_query, gate_mode)
     b = backward(q, k, v, gate, block, topk, window, f, dout, seq_lens, sm_scale, stis_mode,
-                 stis_block, per_query)
+                 stis_block, per_query, gate_mode)
     f.update(b)
     return f
 
