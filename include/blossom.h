@@ -95,6 +95,12 @@ typedef struct {
                         * float [cmp_block] (or [block_size] without compression blocks).  NULL =
                         * the mean.  Only the selection reads it, and no gradient reaches it (the
                         * top-k is piecewise constant), so it has no entry in the backward.       */
+  int32_t gate_mode;   /* 0: gate_logits is float [H][2] and alpha_h = sigmoid(g[h][0] - g[h][1]);
+                        * 1: the input-dependent gate of Eq. 18 with a one-layer F_o: gate_logits
+                        * (and dgate) are float [H][2 D + 1] = (w_lt[D], w_st[D], b) per head and
+                        * alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row,
+                        * broadcast over the head's channels in Eq. 19; runs on the CUDA-core
+                        * kernels                                                                 */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

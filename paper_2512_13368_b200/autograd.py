@@ -28,7 +28,7 @@ def _like(t):
     return torch.empty_strided(t.shape, t.stride(), dtype=t.dtype, device=t.device)
 
 
-def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True):
+def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True, gate_mode=0):
     """Host-side validation before anything is launched: the library receives raw addresses, so a
     host tensor, a tensor on another device, a wrong integer width or a wrong shape would become a
     device memory fault instead of a Python error.  Returns seq_lens as the int32 CUDA tensor the
@@ -43,8 +43,9 @@ def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True):
     B, H, L, D = q.shape
     if k.shape[0] != B or k.shape[2] != L or k.shape[3] != D or k.shape[1] < 1 or H % k.shape[1]:
         raise ValueError("k, v must be [B, Hkv, L, D] with Hkv dividing the number of query heads")
-    if not isinstance(gate_logits, torch.Tensor) or tuple(gate_logits.shape) != (H, 2):
-        raise ValueError("gate_logits must be a tensor of shape [H, 2]")
+    gshape = (H, 2 * D + 1) if gate_mode else (H, 2)
+    if not isinstance(gate_logits, torch.Tensor) or tuple(gate_logits.shape) != gshape:
+        raise ValueError(f"gate_logits must be a tensor of shape {list(gshape)}")
     if (require_cuda and not gate_logits.is_cuda) or gate_logits.device != q.device:
         raise ValueError("gate_logits must be a CUDA tensor on q's device")
     if not gate_logits.dtype.is_floating_point:
@@ -63,8 +64,9 @@ def check_arguments(q, k, v, gate_logits, seq_lens, require_cuda=True):
 class _BlossomAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
-                stis_mode, stis_block, cmp_block, cmp_stride, per_query=0, phi_logits=None):
-        seq_lens = check_arguments(q, k, v, gate_logits, seq_lens)
+                stis_mode, stis_block, cmp_block, cmp_stride, per_query=0, phi_logits=None,
+                gate_mode=0):
+        seq_lens = check_arguments(q, k, v, gate_logits, seq_lens, gate_mode=gate_mode)
         B, H, L, D = q.shape
         Hkv = k.shape[1]
         # The library addresses every q-shaped buffer with q's strides and every k-shaped one with
@@ -79,7 +81,7 @@ class _BlossomAttention(torch.autograd.Function):
                                      sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
                                      stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride,
                                      kv_heads=Hkv, kv_strides=k.stride()[:3], select_mode=int(per_query),
-                                     phi_logits=phi_logits)
+                                     phi_logits=phi_logits, gate_mode=int(gate_mode))
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -105,15 +107,15 @@ class _BlossomAttention(torch.autograd.Function):
         if dout.stride() != q.stride() or dout.dtype != q.dtype:  # the library wants q's layout
             dout = _like(q).copy_(dout)
         dq, dk, dv = _like(q), _like(k), _like(k)
-        dgate = torch.empty((q.shape[1], 2), dtype=torch.float32, device=q.device)
+        dgate = torch.empty(tuple(gate.shape), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
-        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 11
+        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 12
 
 
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
                       return_indices=False, short_term="window", mask_block=1, cmp_block=0,
-                      cmp_stride=0, select_per_query=False, phi_logits=None):
+                      cmp_stride=0, select_per_query=False, phi_logits=None, input_dependent_gate=False):
     """Gated two-branch sparse attention of q [B, H, L, D] and k, v [B, Hkv, L, D] (float32 or
     bfloat16, CUDA; Hkv divides H: with Hkv < H the query heads of a group share key/value head
     and selection, and the returned indices are [B, Hkv, M, top_k]).
@@ -129,6 +131,9 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     (Eq. 8, 11); 0 = the selection blocks themselves.
     select_per_query: one selection per query position (Eq. 13 as printed; indices [B, Hkv, L,
     top_k]) instead of one per query block; runs on the CUDA-core kernels.
+    input_dependent_gate: Eq. 18's gate with a one-layer F_o: gate_logits is [H, 2 D + 1] = (w_lt,
+    w_st, b) per head and alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row
+    (differentiable in those parameters); runs on the CUDA-core kernels.
     phi_logits: optional float32 CUDA tensor [cmp_block or block_size]: Eq. 9's learnable block
     summary as a softmax pooling over a block's positions (None = the mean).  It only steers the
     selection, which is not differentiated, so it receives no gradient here.
@@ -144,5 +149,6 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     out, idx = _BlossomAttention.apply(q, k, v, gate_logits, seq_lens, int(block_size), int(top_k),
                                        int(window), float(sm_scale),
                                        1 if short_term == "power-law" else 0, int(mask_block),
-                                       int(cmp_block), int(cmp_stride), int(bool(select_per_query)), phi_logits)
+                                       int(cmp_block), int(cmp_stride), int(bool(select_per_query)), phi_logits,
+                                       int(bool(input_dependent_gate)))
     return (out, idx) if return_indices else out

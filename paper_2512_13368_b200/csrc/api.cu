@@ -84,6 +84,8 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.clive = reinterpret_cast<int32_t *>(take(units * (size_t)s.Mc * sizeof(int32_t)));
   w.cmean32 = reinterpret_cast<float *>(take(units * (size_t)s.Mc * s.D * sizeof(float)));
   w.cnorm = reinterpret_cast<float *>(take(units * (size_t)s.Mc * sizeof(float)));
+  w.gate_ac = reinterpret_cast<float *>(take(s.gate_mode ? 2 * units * s.L * sizeof(float) : 0));
+  w.dgate_part = reinterpret_cast<double *>(take(s.gate_mode ? units * s.M * (2 * s.D + 1) * sizeof(double) : 0));
   w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.bytes = off;
@@ -136,6 +138,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.scale = (float)s.scale_d;
   s.sb = p->stride_b; s.sh = p->stride_h; s.sl = p->stride_l;
   s.Hkv = p->kv_heads; s.G = p->heads / p->kv_heads;
+  if (p->gate_mode < 0 || p->gate_mode > 1) return BLOSSOM_ERR_INVALID_ARG;
+  s.gate_mode = p->gate_mode;
   s.pq = p->select_mode;
   s.phi = p->phi_logits;
   if (reinterpret_cast<uintptr_t>(s.phi) % 4) return BLOSSOM_ERR_INVALID_ARG;

@@ -34,6 +34,9 @@ __device__ __forceinline__ void scale_axpy4(float4 &y, float c, float a, const f
   y.x = fmaf(a, x.x, y.x * c); y.y = fmaf(a, x.y, y.y * c);
   y.z = fmaf(a, x.z, y.z * c); y.w = fmaf(a, x.w, y.w * c);
 }
+// four consecutive floats from an address that is only 4-byte aligned (the rows of F_o's
+// parameters are 2 D + 1 floats long)
+__device__ __forceinline__ float4 ldw4(const float *p) { return make_float4(p[0], p[1], p[2], p[3]); }
 __device__ __forceinline__ float4 zero4() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
 
@@ -165,20 +168,36 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
   }
 
   if (!inrange) return;
-  const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]);
   const float iL = lL > 0.f ? 1.f / lL : 0.f, iS = lS > 0.f ? 1.f / lS : 0.f;
   const int64_t ro = row_offset(s, n, h, t);
+  float4 oL[NV], oS[NV];
 #pragma unroll
   for (int c = 0; c < NV; ++c) {
-    const float4 oL = make_float4(aL[c].x * iL, aL[c].y * iL, aL[c].z * iL, aL[c].w * iL);
-    const float4 oS = make_float4(aS[c].x * iS, aS[c].y * iS, aS[c].z * iS, aS[c].w * iS);
+    oL[c] = make_float4(aL[c].x * iL, aL[c].y * iL, aL[c].z * iL, aL[c].w * iL);
+    oS[c] = make_float4(aS[c].x * iS, aS[c].y * iS, aS[c].z * iS, aS[c].w * iS);
+  }
+  float alpha;
+  if (s.gate_mode) {  // Eq. 18: alpha_t = sigmoid(<w_lt, O_lt,t> + <w_st, O_st,t> + b)
+    const float *gw = gate + (int64_t)h * (2 * D + 1);
+    float a = 0.f;
+#pragma unroll
+    for (int c = 0; c < NV; ++c) {
+      a = dot4(ldw4(gw + (c * 4 + sub) * 4), oL[c], a);
+      a = dot4(ldw4(gw + D + (c * 4 + sub) * 4), oS[c], a);
+    }
+    alpha = sigmoidf_(group_sum(a, gmask) + gw[2 * D]);
+  } else {
+    alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]);
+  }
+#pragma unroll
+  for (int c = 0; c < NV; ++c) {
     const float be = 1.f - alpha;
-    const float4 o = make_float4(alpha * oL.x + be * oS.x, alpha * oL.y + be * oS.y,
-                                 alpha * oL.z + be * oS.z, alpha * oL.w + be * oS.w);
+    const float4 o = make_float4(alpha * oL[c].x + be * oS[c].x, alpha * oL[c].y + be * oS[c].y,
+                                 alpha * oL[c].z + be * oS[c].z, alpha * oL[c].w + be * oS[c].w);
     const int64_t off = ro + (c * 4 + sub) * 4;
     st4(out + off, o);
-    if (out_lt) st4(out_lt + off, oL);
-    if (out_st) st4(out_st + off, oS);
+    if (out_lt) st4(out_lt + off, oL[c]);
+    if (out_st) st4(out_st + off, oS[c]);
   }
   if (sub == 0 && lse) {
     const int64_t BHL = (int64_t)s.B * s.H * s.L;
@@ -195,7 +214,8 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
     const int32_t *__restrict__ idx, const T *__restrict__ out_lt, const T *__restrict__ out_st,
     const float *__restrict__ lse, const T *__restrict__ dout, T *__restrict__ dq,
-    float *__restrict__ delta, double *__restrict__ dalpha_part) {
+    float *__restrict__ delta, double *__restrict__ dalpha_part, float *__restrict__ gate_ac,
+    double *__restrict__ dgate_part) {
   constexpr int NV = D / 16, CH = D / 4;
   extern __shared__ float smf[];
   float *Ks = smf, *Vs = Ks + s.Bk * D;
@@ -212,7 +232,10 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
   const int t = qb * s.Bk + r;
   const bool inrange = t < s.L, active = inrange && t >= pad0;
   const int64_t BHL = (int64_t)s.B * s.H * s.L;
-  const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
+  // scalar gate: one alpha per head; input-dependent gate (Eq. 18): one per row, and the row's
+  // upstream gradients of the two branches gain c w_lt, c w_st with c = alpha (1 - alpha) <G, O_lt - O_st>
+  float alpha = s.gate_mode ? 0.f : sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
+  const float *gw = gate + (int64_t)h * (2 * D + 1);
 
   const int hk = h / s.G;  // key/value head of this query head; its group shares one selection
   if (s.pq)
@@ -221,8 +244,8 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
   else
     build_visit_flags(s, idx + (((int64_t)n * s.Hkv + hk) * s.M + qb) * s.topk, qb, flags);
 
-  float4 qv[NV], gv[NV], acc[NV];
-  float dL = 0.f, dS = 0.f;
+  float4 qv[NV], gv[NV], acc[NV], wL[NV], wS[NV];
+  float dL = 0.f, dS = 0.f, woL = 0.f, woS = 0.f;
   const int64_t ro = row_offset(s, n, h, inrange ? t : 0);
 #pragma unroll
   for (int c = 0; c < NV; ++c) {
@@ -230,14 +253,31 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
     qv[c] = active ? ld4(q + off) : zero4();
     gv[c] = active ? ld4(dout + off) : zero4();
     acc[c] = zero4();
+    wL[c] = s.gate_mode ? ldw4(gw + (c * 4 + sub) * 4) : zero4();
+    wS[c] = s.gate_mode ? ldw4(gw + D + (c * 4 + sub) * 4) : zero4();
     if (active) {
-      dL = dot4(gv[c], ld4(out_lt + off), dL);
-      dS = dot4(gv[c], ld4(out_st + off), dS);
+      const float4 ol = ld4(out_lt + off), os = ld4(out_st + off);
+      dL = dot4(gv[c], ol, dL);
+      dS = dot4(gv[c], os, dS);
+      woL = dot4(wL[c], ol, woL);
+      woS = dot4(wS[c], os, woS);
     }
   }
   dL = group_sum(dL, gmask);
   dS = group_sum(dS, gmask);
-  const float deltaL = alpha * dL, deltaS = beta * dS;
+  float cpre = 0.f;
+  if (s.gate_mode) {
+    woL = group_sum(woL, gmask);
+    woS = group_sum(woS, gmask);
+    alpha = sigmoidf_(woL + woS + gw[2 * D]);
+    beta = 1.f - alpha;
+    cpre = active ? alpha * beta * (dL - dS) : 0.f;
+    if (inrange && sub == 0) {
+      gate_ac[(int64_t)u * s.L + t] = alpha;
+      gate_ac[(int64_t)s.B * s.H * s.L + (int64_t)u * s.L + t] = cpre;
+    }
+  }
+  const float deltaL = alpha * dL + cpre * woL, deltaS = beta * dS + cpre * woS;
   float lseL2 = 0.f, lseS2 = 0.f;
   if (active) {
     lseL2 = lse[(int64_t)u * s.L + t] * kLog2e;
@@ -271,23 +311,32 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
         if (!selb && !inS) continue;
         const float4 *kr = reinterpret_cast<const float4 *>(Ks) + pi * CH;
         const float4 *vr = reinterpret_cast<const float4 *>(Vs) + pi * CH;
-        float part = 0.f, dpart = 0.f;
+        float part = 0.f, dpart = 0.f, uL = 0.f, uS = 0.f;
 #pragma unroll
         for (int c = 0; c < NV; ++c) {
           part = dot4(qv[c], kr[c * 4 + sub], part);
           dpart = dot4(gv[c], vr[c * 4 + sub], dpart);
+        }
+        if (s.gate_mode) {  // <w_lt, v_p>, <w_st, v_p>: the part of dP that comes through alpha
+#pragma unroll
+          for (int c = 0; c < NV; ++c) {
+            uL = dot4(wL[c], vr[c * 4 + sub], uL);
+            uS = dot4(wS[c], vr[c * 4 + sub], uS);
+          }
+          uL = cpre * group_sum(uL, gmask);
+          uS = cpre * group_sum(uS, gmask);
         }
         const float sv = group_sum(part, gmask) * sc2;
         const float dP = group_sum(dpart, gmask);
         float dSsum = 0.f;
         if (selb) {
           const float P = exp2f(sv - lseL2);
-          dSsum = P * (alpha * dP - deltaL);
+          dSsum = P * (alpha * dP + uL - deltaL);
           dal = fmaf(P, dP, dal);
         }
         if (inS) {
           const float P = exp2f(sv - lseS2);
-          dSsum = fmaf(P, beta * dP - deltaS, dSsum);
+          dSsum = fmaf(P, beta * dP + uS - deltaS, dSsum);
           dal = fmaf(-P, dP, dal);
         }
         const float w = s.scale * dSsum;
@@ -303,6 +352,26 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
     for (int i = 0; i < s.Bk; ++i) a += red[i];  // fixed order
     dalpha_part[(int64_t)u * s.M + qb] = a;
   }
+  if (s.gate_mode) {
+    // gradient of F_o's parameters from this query block: sum_t c_t O_lt,t, sum_t c_t O_st,t, sum_t c_t
+    // (rows staged in the K / V tiles, which nobody reads any more; fixed order over the rows)
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < NV; ++c) {
+      const int64_t off = ro + (c * 4 + sub) * 4;
+      const float4 ol = active ? ld4(out_lt + off) : zero4(), os = active ? ld4(out_st + off) : zero4();
+      reinterpret_cast<float4 *>(Ks)[r * CH + c * 4 + sub] = make_float4(cpre * ol.x, cpre * ol.y, cpre * ol.z, cpre * ol.w);
+      reinterpret_cast<float4 *>(Vs)[r * CH + c * 4 + sub] = make_float4(cpre * os.x, cpre * os.y, cpre * os.z, cpre * os.w);
+    }
+    if (sub == 0) red[r] = (double)cpre;
+    __syncthreads();
+    for (int d = tid; d < 2 * D + 1; d += blockDim.x) {
+      double a = 0.0;
+      for (int i = 0; i < s.Bk; ++i)
+        a += d < D ? (double)Ks[i * D + d] : (d < 2 * D ? (double)Vs[i * D + d - D] : red[i]);
+      dgate_part[((int64_t)u * s.M + qb) * (2 * D + 1) + d] = a;
+    }
+  }
   if (!inrange) return;
 #pragma unroll
   for (int c = 0; c < NV; ++c) st4(dq + ro + (c * 4 + sub) * 4, acc[c]);
@@ -315,13 +384,14 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
     const int32_t *__restrict__ idx, const float *__restrict__ lse,
     const float *__restrict__ delta, const T *__restrict__ dout, T *__restrict__ dk,
-    T *__restrict__ dv) {
+    T *__restrict__ dv, const float *__restrict__ gate_ac) {
   constexpr int NV = D / 16, CH = D / 4;
   extern __shared__ float smf[];
   float *Qs = smf, *Gs = Qs + s.Bk * D;
   float *lLs = Gs + s.Bk * D, *lSs = lLs + s.Bk, *dLs = lSs + s.Bk, *dSs = dLs + s.Bk;
   int *flags = reinterpret_cast<int *>(dSs + s.Bk);
   int *rsel = flags + s.M;  // [Bk] per-position selection only: which queries of the staged block selected this key block
+  float *als = reinterpret_cast<float *>(rsel + s.Bk), *cs = als + s.Bk;  // [Bk] each: alpha_t, c_t (input-dependent gate)
   // uk counts (batch, key/value head) pairs: the key block collects from every query head of its group
   const int j = blockIdx.x % s.M, uk = blockIdx.x / s.M, n = uk / s.Hkv, hk = uk % s.Hkv;
   int len = seq_lens ? seq_lens[n] : s.L;
@@ -362,7 +432,7 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
     for (int x = 0; x < s.G * (s.M - j); ++x) {  // every query head of the group, every later query block
       const int h = hk * s.G + x / (s.M - j), qb = j + x % (s.M - j);
       const int64_t u = (int64_t)n * s.H + h;
-      const float alpha = sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]), beta = 1.f - alpha;
+      const float alpha_h = s.gate_mode ? 0.f : sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]);
       int f = flags[qb];
       if (s.pq) {  // every query position has a list of its own
         __syncthreads();
@@ -390,9 +460,26 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
         lSs[i] = ok ? lse[BHL + u * s.L + t] * kLog2e : 0.f;
         dLs[i] = ok ? delta[u * s.L + t] : 0.f;
         dSs[i] = ok ? delta[BHL + u * s.L + t] : 0.f;
+        als[i] = s.gate_mode ? (ok ? gate_ac[u * s.L + t] : 0.f) : alpha_h;
+        cs[i] = (s.gate_mode && ok) ? gate_ac[BHL + u * s.L + t] : 0.f;
       }
       __syncthreads();
       if (!active) continue;
+      // input-dependent gate: <w_lt, v_p>, <w_st, v_p> of this thread's key row and the weights' chunks
+      float4 wL[NV], wS[NV];
+      float uL = 0.f, uS = 0.f;
+      if (s.gate_mode) {
+        const float *gw = gate + (int64_t)h * (2 * D + 1);
+#pragma unroll
+        for (int c = 0; c < NV; ++c) {
+          wL[c] = ldw4(gw + (c * 4 + sub) * 4);
+          wS[c] = ldw4(gw + D + (c * 4 + sub) * 4);
+          uL = dot4(wL[c], vv[c], uL);
+          uS = dot4(wS[c], vv[c], uS);
+        }
+        uL = group_sum(uL, gmask);
+        uS = group_sum(uS, gmask);
+      }
       const int t0 = qb * s.Bk;
       const int tbeg = max(0, p - t0), tend = min(s.Bk, s.L - t0);  // t >= p >= pad0
       const bool sel_all = f & 1;
@@ -410,22 +497,32 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
         }
         const float sv = group_sum(part, gmask) * sc2;
         const float dP = group_sum(dpart, gmask);
-        float wv = 0.f, dSsum = 0.f;
+        const float alpha = als[ti], beta = 1.f - alpha, ct = cs[ti];
+        float wv = 0.f, dSsum = 0.f, cwL = 0.f, cwS = 0.f;
         if (selb) {
           const float P = exp2f(sv - lLs[ti]);
           wv = alpha * P;
-          dSsum = P * (alpha * dP - dLs[ti]);
+          cwL = ct * P;
+          dSsum = P * (alpha * dP + ct * uL - dLs[ti]);
         }
         if (inS) {
           const float P = exp2f(sv - lSs[ti]);
           wv = fmaf(beta, P, wv);
-          dSsum = fmaf(P, beta * dP - dSs[ti], dSsum);
+          cwS = ct * P;
+          dSsum = fmaf(P, beta * dP + ct * uS - dSs[ti], dSsum);
         }
         const float wk = s.scale * dSsum;
 #pragma unroll
         for (int c = 0; c < NV; ++c) {
           axpy4(dva[c], wv, gr[c * 4 + sub]);
           axpy4(dka[c], wk, qr[c * 4 + sub]);
+        }
+        if (s.gate_mode) {  // dV_p += P_lt c_t w_lt + P_st c_t w_st
+#pragma unroll
+          for (int c = 0; c < NV; ++c) {
+            axpy4(dva[c], cwL, wL[c]);
+            axpy4(dva[c], cwS, wS[c]);
+          }
         }
       }
     }
@@ -463,6 +560,19 @@ __global__ void __launch_bounds__(256) gate_grad_kernel(Shape s, const float *__
     const double g0 = al * (1.0 - al) * red[0];
     dgate[h * 2 + 0] = (float)g0;
     dgate[h * 2 + 1] = (float)(-g0);
+  }
+}
+
+// Gradient of F_o's parameters (input-dependent gate): per head, the per-query-block partial sums
+// added over batch entries and query blocks in a fixed order.  One block per head.
+__global__ void __launch_bounds__(256) gate_param_grad_kernel(Shape s, const double *__restrict__ part,
+                                                              float *__restrict__ dgate) {
+  const int h = blockIdx.x, GW = 2 * s.D + 1;
+  for (int d = threadIdx.x; d < GW; d += 256) {
+    double a = 0.0;
+    for (int n = 0; n < s.B; ++n)
+      for (int qb = 0; qb < s.M; ++qb) a += part[(((int64_t)n * s.H + h) * s.M + qb) * GW + d];
+    dgate[(int64_t)h * GW + d] = (float)a;
   }
 }
 
@@ -504,9 +614,9 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
     LaunchScope ls(K_BWD_DQ_SIMT, st);
     bwd_dq_simt_kernel<T, D><<<grid, s.Bk * 4, smem_q, st>>>(s, q, k, v, gate, seq_lens, idx, out_lt,
                                                              out_st, lse, dout, dq, ws.delta,
-                                                             ws.dalpha);
+                                                             ws.dalpha, ws.gate_ac, ws.dgate_part);
   }
-  const size_t smem_k = (size_t)(2 * s.Bk * D + 4 * s.Bk) * sizeof(float) + (size_t)(s.M + s.Bk) * sizeof(int);
+  const size_t smem_k = (size_t)(2 * s.Bk * D + 6 * s.Bk) * sizeof(float) + (size_t)(s.M + s.Bk) * sizeof(int);
   if (smem_k > 48 * 1024 &&
       cudaFuncSetAttribute(bwd_dkdv_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem_k) != cudaSuccess)
@@ -515,7 +625,12 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
     LaunchScope ls(K_BWD_DKDV_SIMT, st);
     const unsigned grid_k = (unsigned)s.M * (unsigned)(s.B * s.Hkv);
     bwd_dkdv_simt_kernel<T, D><<<grid_k, s.Bk * 4, smem_k, st>>>(s, q, k, v, gate, seq_lens, idx, lse,
-                                                               ws.delta, dout, dk, dv);
+                                                               ws.delta, dout, dk, dv, ws.gate_ac);
+  }
+  if (s.gate_mode) {
+    LaunchScope ls(K_GATE_GRAD, st);
+    gate_param_grad_kernel<<<s.H, 256, 0, st>>>(s, ws.dgate_part, dgate);
+    return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
   }
   return launch_gate_grad(s, gate, ws, dgate, st);
 }

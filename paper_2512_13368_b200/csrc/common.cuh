@@ -19,6 +19,7 @@ struct Shape {
   int64_t sb, sh, sl;  // element strides of q-shaped tensors
   int Hkv, G;             // key/value heads and query heads per key/value head (H = Hkv * G)
   int pq;                 // 1: one selection per query position (block_idx is [B][Hkv][L][top_k])
+  int gate_mode;          // 0: one gate weight per head from two logits; 1: Eq. 18's input-dependent gate
   const float *phi;       // logits of the learnable block summary (Eq. 9) or nullptr = the mean
   int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
 };
@@ -41,6 +42,8 @@ struct Workspace {
   int32_t *clive;    // [B][H][Mc]     their numbers of valid keys
   float *cmean32;    // [B][H][Mc][D]  the means rounded to fp32
   float *cnorm;      // [B][H][Mc]     upper bounds of the norms of the fp32 means
+  float *gate_ac;    // [2][B][H][L]  input-dependent gate: alpha_t and c_t of every row (backward)
+  double *dgate_part;// [B][H][M][2 D + 1]  per query block partial of the gradient of F_o's parameters
   uint8_t *qmeta;    // per query-major CTA of the tensor-core kernels: tile lists (tc_meta_kernel)
   uint8_t *kmeta;    // per key-major CTA (dK/dV kernel): tile lists
   size_t bytes;

@@ -33,7 +33,8 @@ class DeviceProblem:
                                           sm_scale=sm_scale, stis_mode=w.stis_mode,
                                           stis_block=w.stis_block, cmp_block=w.cmp_block,
                                           cmp_stride=w.cmp_stride, kv_heads=w.kv_heads or w.H,
-                                          select_mode=w.per_query, phi_logits=self.phi)
+                                          select_mode=w.per_query, phi_logits=self.phi,
+                                          gate_mode=getattr(w, "gate_mode", 0))
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):
@@ -49,7 +50,7 @@ class DeviceProblem:
         self.out_st = e() if training else None
         self.lse = torch.empty((2, w.B, w.H, w.L), dtype=torch.float32, device=dev) if training else None
         self.dq, self.dk, self.dv = (e(), ekv(), ekv()) if training else (None, None, None)
-        self.dgate = torch.empty((w.H, 2), dtype=torch.float32, device=dev)
+        self.dgate = torch.empty(tuple(w.gate.shape), dtype=torch.float32, device=dev)
         nbytes = binding.blossom_workspace_bytes(self.params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")

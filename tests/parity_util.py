@@ -84,6 +84,8 @@ def check_forward_backward(w, res, sm_scale=None, backward=True):
     forgiven = check_indices(w, res["idx"], sm_scale)
     fwd_fn, bwd_fn = (oracle.forward_gqa, oracle.backward_gqa) if _grouped(w) else (oracle.forward, oracle.backward)
     kw = {"per_query": True} if getattr(w, "per_query", 0) else {}
+    if getattr(w, "gate_mode", 0):
+        kw["gate_mode"] = 1
     ref = fwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
                  idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block, **kw)
     errs = {"near_tie_rows": forgiven}

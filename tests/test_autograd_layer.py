@@ -72,6 +72,32 @@ def test_autograd_packed_projection_views_and_grouped_heads():
         assert err <= tolerance(w, ref[key]), (key, err)
 
 
+def test_autograd_options_input_dependent_gate_per_query_selection_learned_summary():
+    """The front end's newer options together: Eq. 18's gate (gradient of F_o's parameters), a
+    selection per query position, the learnable block summary."""
+    import torch
+    import oracle
+    from paper_2512_13368_b200.autograd import blossom_attention
+    dev = torch.device("cuda:0")
+    w = workloads.make("autograd-opts", "fp32", 2, 2, 96, 32, 16, 3, 20, seed=71)
+    gw = (0.3 * np.random.default_rng(1).standard_normal((2, 65))).astype(np.float32)
+    phi = np.random.default_rng(2).standard_normal(16).astype(np.float32)
+    t = lambda a: torch.from_numpy(a).to(dev).requires_grad_(True)  # noqa: E731
+    q, k, v, gate = t(w.q), t(w.k), t(w.v), t(gw)
+    out, idx = blossom_attention(q, k, v, gate, w.block, w.topk, w.window, return_indices=True,
+                                 select_per_query=True, phi_logits=torch.from_numpy(phi).to(dev),
+                                 input_dependent_gate=True)
+    out.backward(torch.from_numpy(w.dout).to(dev))
+    ref_idx = oracle.select_blocks_per_query(w.q, w.k, w.block, w.topk, phi_logits=phi)
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    ref = oracle.forward_backward(w.q, w.k, w.v, gw, w.dout, w.block, w.topk, w.window, idx=ref_idx,
+                                  per_query=True, gate_mode=1)
+    got = {"out": out, "dq": q.grad, "dk": k.grad, "dv": v.grad, "dgate": gate.grad}
+    for key, val in got.items():
+        err = float(np.abs(val.detach().float().cpu().numpy() - ref[key]).max())
+        assert err <= 1e-4, (key, err)
+
+
 def test_layer_step_runs_and_reports_attention_share():
     from paper_2512_13368_b200 import layer_step
     r = layer_step.attention_share(batch=8, seq_len=256, n_items=2000, negatives=15, steps=2, warmup=1)

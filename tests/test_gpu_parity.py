@@ -591,3 +591,24 @@ def test_learnable_block_summary(runner, dtype, L, D, H, Hkv, block, topk, cmp, 
     w0.per_query, w0.seq_lens = w.per_query, w.seq_lens
     _, res0 = run(runner, w0, backward=False)
     assert not np.array_equal(res0["idx"], res["idx"])
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens,per_query", [
+    (64, 32, 2, 2, 8, 2, 16, None, False),
+    (200, 32, 2, 2, 16, 4, 32, [200, 5, 77, 0], False),
+    (300, 64, 4, 2, 32, 4, 40, [300, 131], False),            # grouped heads
+    (257, 64, 2, 2, 64, 3, 8, None, True),                    # with a selection per query position
+])
+def test_input_dependent_gate(runner, dtype, L, D, H, Hkv, block, topk, window, lens, per_query):
+    """gate_mode 1 (Eq. 18: alpha = sigmoid(F_o([O_lt; O_st])) per query row with a one-layer F_o,
+    Eq. 19): forward, the gradients of q, k, v and of F_o's parameters against the oracle."""
+    B = len(lens) if lens else 2
+    w = workloads.make("gate-mlp", dtype, B, H, L, D, block, topk, window, seed=67, kv_heads=Hkv if Hkv != H else 0)
+    w.gate_mode, w.per_query = 1, int(per_query)
+    w.gate = (0.3 * np.random.default_rng(5).standard_normal((H, 2 * D + 1))).astype(np.float32)
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    assert res["dgate"].shape == (H, 2 * D + 1)
+    print(check_forward_backward(w, res))
