@@ -74,7 +74,9 @@ int blossom_oracle_threads(void) {
 static double phi_weight(const double *phi, int i) { return phi ? exp(phi[i]) : 1.0; }
 
 /* ---- selection for one (n,h) unit: Eq. 8-10, 12, 13 --------------------- */
-static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0,
+/* causal = 1: the candidates of query block b are the live blocks before it; causal = 0 (a
+ * bidirectional encoder): every live block but b itself.  The own block is always kept. */
+static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0, int causal,
                         const double *q, const double *k, const double *phi, int32_t *idx,
                         double *scores /* [M][M] or NULL */) {
   const int M = n_blocks(L, Bk);
@@ -108,55 +110,56 @@ static void select_unit(int L, int D, int Bk, int topk, double scale, int pad0,
     int qlo = imax(b * Bk, pad0), qhi = imin((b + 1) * Bk, L);
     if (qlo >= qhi) continue; /* query block holds only padding */
 
+    const int hi = causal ? b : M; /* candidates: j < hi, j != b */
     int ncand = 0;
-    for (int j = 0; j < b; ++j) {
+    for (int j = 0; j < hi; ++j) {
       S[j] = 0.0;
-      ncand += live[j];
+      if (j != b) ncand += live[j];
     }
     /* Eq. 10 per query, summed over the queries that share the selection (Eq. 12's rule) */
     if (ncand > 0) {
       for (int t = qlo; t < qhi; ++t) {
         double mx = -INFINITY;
-        for (int j = 0; j < b; ++j) {
-          if (!live[j]) continue;
+        for (int j = 0; j < hi; ++j) {
+          if (!live[j] || j == b) continue;
           double acc = 0.0;
           for (int c = 0; c < D; ++c) acc += q[(size_t)t * D + c] * ktil[(size_t)j * D + c];
           z[j] = scale * acc;
           if (z[j] > mx) mx = z[j];
         }
         double den = 0.0;
-        for (int j = 0; j < b; ++j)
-          if (live[j]) den += exp(z[j] - mx);
-        for (int j = 0; j < b; ++j)
-          if (live[j]) S[j] += exp(z[j] - mx) / den;
+        for (int j = 0; j < hi; ++j)
+          if (live[j] && j != b) den += exp(z[j] - mx);
+        for (int j = 0; j < hi; ++j)
+          if (live[j] && j != b) S[j] += exp(z[j] - mx) / den;
       }
     }
     if (scores)
-      for (int j = 0; j < b; ++j)
-        if (live[j]) scores[(size_t)b * M + j] = S[j];
+      for (int j = 0; j < hi; ++j)
+        if (live[j] && j != b) scores[(size_t)b * M + j] = S[j];
 
-    /* Eq. 13: the own block plus the (topk-1) best past blocks, ties to the lower index */
+    /* Eq. 13: the own block plus the (topk-1) best candidates, ties to the lower index */
     int want = imin(topk - 1, ncand), nch = 0;
     memset(taken, 0, (size_t)M);
     for (int s = 0; s < want; ++s) {
       int best = -1;
-      for (int j = 0; j < b; ++j) {
-        if (!live[j] || taken[j]) continue;
+      for (int j = 0; j < hi; ++j) {
+        if (!live[j] || j == b || taken[j]) continue;
         if (best < 0 || S[j] > S[best]) best = j; /* strict > keeps the lower index on ties */
       }
       taken[best] = 1;
       chosen[nch++] = best;
     }
-    /* ascending order: walk the flags, then the own block (largest index) */
+    /* ascending order: walk the flags, the own block in its place */
+    taken[b] = 1;
     int s = 0;
-    for (int j = 0; j < b; ++j)
+    for (int j = 0; j < M; ++j)
       if (taken[j]) row[s++] = j;
-    row[s++] = b;
   }
   free(ktil); free(live); free(S); free(z); free(taken); free(chosen);
 }
 
-int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double scale,
+int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, int causal, double scale,
                           const double *q, const double *k, const int32_t *seq_lens,
                           const double *phi /* [Bk] or NULL */, int32_t *idx, double *scores) {
   if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
@@ -168,7 +171,7 @@ int blossom_oracle_select(int B, int H, int L, int D, int Bk, int topk, double s
       int len = seq_lens ? seq_lens[n] : L;
       if (len < 0) len = 0;
       if (len > L) len = L;
-      select_unit(L, D, Bk, topk, scale, L - len, q + u * L * D, k + u * L * D, phi,
+      select_unit(L, D, Bk, topk, scale, L - len, causal, q + u * L * D, k + u * L * D, phi,
                   idx + u * M * topk, scores ? scores + u * M * M : NULL);
     }
   return 0;
@@ -420,13 +423,14 @@ static double attend_row(int D, double scale, const double *qt, const double *k,
 
 /* key list of the long-term branch for query t (Eq. 14 + causal mask): valid p <= t inside the
  * selected blocks of t's query block */
-static int ltis_keys(int L, int Bk, int topk, int pad0, const int32_t *row, int t, int *keys) {
+static int ltis_keys(int L, int Bk, int topk, int pad0, int causal, const int32_t *row, int t, int *keys) {
   int nk = 0;
   const int M = n_blocks(L, Bk);
   for (int s = 0; s < topk; ++s) {
     int j = row[s];
     if (j < 0 || j >= M) continue;
-    int lo = imax(j * Bk, pad0), hi = imin(imin((j + 1) * Bk, L), t + 1);
+    int lo = imax(j * Bk, pad0), hi = imin((j + 1) * Bk, L);
+    if (causal) hi = imin(hi, t + 1);
     for (int p = lo; p < hi; ++p) keys[nk++] = p;
   }
   return nk;
@@ -450,9 +454,9 @@ static int stis_mask(int mode, int w, int blk, int L, int i, int j) {
 
 /* key list of the short-term branch: Eq. 15 restricted to the causal side (p <= t) and to the
  * valid (non-padding) positions */
-static int stis_keys(int mode, int w, int blk, int L, int pad0, int t, int *keys) {
+static int stis_keys(int mode, int w, int blk, int L, int pad0, int causal, int t, int *keys) {
   int nk = 0;
-  for (int p = pad0; p <= t; ++p)
+  for (int p = pad0; p <= (causal ? t : L - 1); ++p)
     if (stis_mask(mode, w, blk, L, t, p)) keys[nk++] = p;
   return nk;
 }
@@ -466,7 +470,7 @@ static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
  * w_st[D], b) and alpha_t = sigmoid(<w_lt, O_lt,t> + <w_st, O_st,t> + b), one weight per token
  * and head, broadcast over the head's channels in Eq. 19 */
 int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
-                           int stis_blk, int per_query, int gate_mode, double scale,
+                           int stis_blk, int per_query, int gate_mode, int causal, double scale,
                            const double *q, const double *k, const double *v, const double *gate,
                            const int32_t *seq_lens, const int32_t *idx, double *out,
                            double *out_lt, double *out_st, double *lse) {
@@ -497,9 +501,9 @@ int blossom_oracle_forward(int B, int H, int L, int D, int Bk, int topk, int win
         } else {
           const int32_t *row = per_query ? idx + (u * L + (size_t)t) * topk
                                          : idx + (u * M + (size_t)(t / Bk)) * topk;
-          int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
+          int nk = ltis_keys(L, Bk, topk, pad0, causal, row, t, keys);
           lL = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oL); /* Eq. 16 */
-          nk = stis_keys(stis_mode, window, stis_blk, L, pad0, t, keys);
+          nk = stis_keys(stis_mode, window, stis_blk, L, pad0, causal, t, keys);
           lS = attend_row(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, sbuf, oS); /* Eq. 17 */
         }
         double alpha = alpha_h;
@@ -551,7 +555,7 @@ static void attend_row_bwd(int D, double scale, const double *qt, const double *
 }
 
 int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int window, int stis_mode,
-                            int stis_blk, int per_query, int gate_mode, double scale,
+                            int stis_blk, int per_query, int gate_mode, int causal, double scale,
                             const double *q, const double *k, const double *v, const double *gate,
                             const int32_t *seq_lens, const int32_t *idx, const double *out_lt,
                             const double *out_st, const double *lse, const double *dout,
@@ -607,10 +611,10 @@ int blossom_oracle_backward(int B, int H, int L, int D, int Bk, int topk, int wi
         }
         const int32_t *row = per_query ? idx + (u * L + (size_t)t) * topk
                                        : idx + (u * M + (size_t)(t / Bk)) * topk;
-        int nk = ltis_keys(L, Bk, topk, pad0, row, t, keys);
+        int nk = ltis_keys(L, Bk, topk, pad0, causal, row, t, keys);
         attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[u * L + t],
                        out_lt + ro, gL, dqu + (size_t)t * D, dku, dvu);
-        nk = stis_keys(stis_mode, window, stis_blk, L, pad0, t, keys);
+        nk = stis_keys(stis_mode, window, stis_blk, L, pad0, causal, t, keys);
         attend_row_bwd(D, scale, qu + (size_t)t * D, ku, vu, keys, nk, lse[BHL + u * L + t],
                        out_st + ro, gS, dqu + (size_t)t * D, dku, dvu);
       }

@@ -48,16 +48,16 @@ def _load():
         d = ctypes.c_double
         lib.blossom_oracle_threads.restype = i
         lib.blossom_oracle_select.restype = i
-        lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
+        lib.blossom_oracle_select.argtypes = [i, i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
         lib.blossom_oracle_select_cmp.restype = i
         lib.blossom_oracle_select_cmp.argtypes = [i, i, i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp, _dp]
         lib.blossom_oracle_forward.restype = i
         lib.blossom_oracle_select_pq.restype = i
         lib.blossom_oracle_select_pq.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
-        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
         lib.blossom_oracle_backward.restype = i
-        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
+        lib.blossom_oracle_backward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                 _ip, _dp, _dp, _dp, _dp, _dp, _dp, _dp, _dp]
         _lib = lib
     return _lib
@@ -98,11 +98,13 @@ def _scale(sm_scale, D):
     return float(sm_scale) if sm_scale else 1.0 / math.sqrt(D)
 
 
-def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False, phi_logits=None):
+def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False, phi_logits=None,
+                  causal=True):
     """Eq. 8-10, 12, 13: block summaries, block scores and the top-k block set.
 
     ``phi_logits`` ``[block]``: Eq. 9's learnable summary as a softmax pooling over the positions of
-    a block (weights exp(phi_logits[i]) over the valid keys); None = the mean."""
+    a block (weights exp(phi_logits[i]) over the valid keys); None = the mean.
+    ``causal=False`` (a bidirectional encoder): a query block scores every live block but itself."""
     q, k = _f64(q), _f64(k)
     B, H, L, D = q.shape
     M = -(-L // block)
@@ -110,7 +112,7 @@ def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores
     scores = np.zeros((B, H, M, M), dtype=np.float64) if return_scores else None
     sl = _lens(seq_lens, B)
     ph = _phi(phi_logits, block)
-    rc = _load().blossom_oracle_select(B, H, L, D, block, topk, _scale(sm_scale, D),
+    rc = _load().blossom_oracle_select(B, H, L, D, block, topk, int(bool(causal)), _scale(sm_scale, D),
                                        _ptr(q, _dp), _ptr(k, _dp), _ptr(sl, _ip), _ptr(ph, _dp),
                                        _ptr(idx, _ip), _ptr(scores, _dp))
     if rc:
@@ -190,7 +192,7 @@ def select_blocks_cmp(q, k, block, topk, cmp_block, cmp_stride, seq_lens=None, s
 
 
 def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, idx=None,
-            stis_mode=0, stis_block=1, per_query=False, gate_mode=0):
+            stis_mode=0, stis_block=1, per_query=False, gate_mode=0, causal=True):
     """Eq. 14, 16, 17, 19.  ``idx`` overrides the selection when given.
 
     ``stis_mode`` 0: the short-term branch is the causal window (Eq. 15, first case);
@@ -199,6 +201,8 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     ``per_query``: the selection is per query position, idx ``[B,H,L,topk]``.
     ``gate_mode`` 1: Eq. 18's input-dependent gate with a one-layer F_o; gate is ``[H, 2 D + 1]`` =
     (w_lt, w_st, b) per head and alpha_t = sigmoid(<w_lt, O_lt,t> + <w_st, O_st,t> + b).
+    ``causal=False``: no causal mask (the bidirectional encoders the paper also plugs the
+    mechanism into): a query sees every valid key of its selected blocks, and Eq. 15 is symmetric.
 
     Returns a dict: out, out_lt, out_st ``[B,H,L,D]``, lse ``[2,B,H,L]``, idx.
     """
@@ -207,7 +211,10 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     M = -(-L // block)
     assert gate.shape == ((H, 2 * D + 1) if gate_mode else (H, 2))
     if idx is None:
-        idx = (select_blocks_per_query if per_query else select_blocks)(q, k, block, topk, seq_lens, sm_scale)
+        if per_query:
+            idx = select_blocks_per_query(q, k, block, topk, seq_lens, sm_scale)
+        else:
+            idx = select_blocks(q, k, block, topk, seq_lens, sm_scale, causal=causal)
     idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int32))
     assert idx.shape == (B, H, L if per_query else M, topk)
     sl = _lens(seq_lens, B)
@@ -217,7 +224,7 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
     lse = np.empty((2, B, H, L), dtype=np.float64)
     rc = _load().blossom_oracle_forward(B, H, L, D, block, topk, window, int(stis_mode),
                                         int(stis_block), int(bool(per_query)), int(gate_mode),
-                                        _scale(sm_scale, D),
+                                        int(bool(causal)), _scale(sm_scale, D),
                                         _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp), _ptr(gate, _dp),
                                         _ptr(sl, _ip), _ptr(idx, _ip), _ptr(out, _dp),
                                         _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp))
@@ -227,7 +234,7 @@ def forward(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None, id
 
 
 def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_scale=None,
-             stis_mode=0, stis_block=1, per_query=False, gate_mode=0):
+             stis_mode=0, stis_block=1, per_query=False, gate_mode=0, causal=True):
     """Gradients of sum(out * dout) with the selection frozen.
 
     ``fwd`` is the dict ``forward`` returned.  Returns dq, dk, dv, dgate (the shape of gate).
@@ -241,7 +248,7 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
     dgate = np.empty(gate.shape, dtype=np.float64)
     rc = _load().blossom_oracle_backward(B, H, L, D, block, topk, window, int(stis_mode),
                                          int(stis_block), int(bool(per_query)), int(gate_mode),
-                                         _scale(sm_scale, D),
+                                         int(bool(causal)), _scale(sm_scale, D),
                                          _ptr(q, _dp), _ptr(k, _dp), _ptr(v, _dp),
                                          _ptr(gate, _dp), _ptr(sl, _ip), _ptr(idx, _ip),
                                          _ptr(out_lt, _dp), _ptr(out_st, _dp), _ptr(lse, _dp),
@@ -253,12 +260,12 @@ def backward(q, k, v, gate, block, topk, window, fwd, dout, seq_lens=None, sm_sc
 
 
 def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm_scale=None,
-                     idx=None, stis_mode=0, stis_block=1, per_query=False, gate_mode=0):
+                     idx=None, stis_mode=0, stis_block=1, per_query=False, gate_mode=0, causal=True):
     """Convenience: forward then backward; returns the two dicts merged."""
     f = forward(q, k, v, gate, block, topk, window, seq_lens, sm_scale, idx, stis_mode, stis_block,
-                per_query, gate_mode)
+                per_query, gate_mode, causal)
     b = backward(q, k, v, gate, block, topk, window, f, dout, seq_lens, sm_scale, stis_mode,
-                 stis_block, per_query, gate_mode)
+                 stis_block, per_query, gate_mode, causal)
     f.update(b)
     return f
 
