@@ -284,7 +284,7 @@ def _group(H, Hkv):
 
 
 def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False,
-                      cmp_block=0, cmp_stride=0, phi_logits=None):
+                      cmp_block=0, cmp_stride=0, phi_logits=None, causal=True):
     """q ``[B,H,L,D]``, k ``[B,Hkv,L,D]`` -> idx ``[B,Hkv,M,topk]`` from group-summed scores.
 
     With ``cmp_block`` / ``cmp_stride`` the per-head scores are those of the overlapping
@@ -301,7 +301,7 @@ def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_sc
                                            phi_logits=phi_logits)
     else:
         _, per_head = select_blocks(q, np.repeat(k, G, axis=1), block, topk, seq_lens, sm_scale,
-                                    return_scores=True, phi_logits=phi_logits)
+                                    return_scores=True, phi_logits=phi_logits, causal=causal)
     scores = per_head.reshape(B, Hkv, G, M, M).sum(axis=2)            # Eq. 12
     idx = np.full((B, Hkv, M, topk), -1, dtype=np.int32)
     for n in range(B):
@@ -311,10 +311,10 @@ def select_blocks_gqa(q, k, block, topk, seq_lens=None, sm_scale=None, return_sc
             for b in range(M):
                 if not live[b]:
                     continue
-                cand = [j for j in range(b) if live[j]]
+                cand = [j for j in (range(b) if causal else range(M)) if live[j] and j != b]
                 # Eq. 13: largest scores first, ties to the lower index; the own block always
                 best = sorted(cand, key=lambda j: (-scores[n, g, b, j], j))[:topk - 1]
-                row = sorted(best) + [b]
+                row = sorted(best + [b])
                 idx[n, g, b, :len(row)] = row
     return (idx, scores) if return_scores else idx
 

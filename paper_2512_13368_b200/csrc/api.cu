@@ -109,7 +109,7 @@ static int make_shape(const blossom_params *p, Shape *out) {
                    p->kv_stride_l % 8 || p->kv_stride_h % 8 || p->kv_stride_b % 8))
     return BLOSSOM_ERR_INVALID_ARG;
   if (p->select_mode < 0 || p->select_mode > 1) return BLOSSOM_ERR_INVALID_ARG;
-  if (p->causal != 1) return BLOSSOM_ERR_UNSUPPORTED;
+  if (p->causal != 0 && p->causal != 1) return BLOSSOM_ERR_INVALID_ARG;
   if (p->stis_mode < 0 || p->stis_mode > 1 || p->stis_block < 0) return BLOSSOM_ERR_INVALID_ARG;
   if (p->head_dim != 32 && p->head_dim != 64) return BLOSSOM_ERR_UNSUPPORTED;
   if (p->block_size != 8 && p->block_size != 16 && p->block_size != 32 && p->block_size != 64)
@@ -141,6 +141,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   if (p->gate_mode < 0 || p->gate_mode > 1) return BLOSSOM_ERR_INVALID_ARG;
   s.gate_mode = p->gate_mode;
   s.pq = p->select_mode;
+  s.causal = p->causal;
+  if (!s.causal && (s.pq || s.cmp_l > 0)) return BLOSSOM_ERR_UNSUPPORTED;  // bidirectional: plain per-block selection
   s.phi = p->phi_logits;
   if (reinterpret_cast<uintptr_t>(s.phi) % 4) return BLOSSOM_ERR_INVALID_ARG;
   if (s.pq && s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // per-position selection scores the selection blocks themselves

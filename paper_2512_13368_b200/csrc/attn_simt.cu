@@ -59,7 +59,8 @@ __device__ __forceinline__ void stage_tile(const Shape &s, const T *base, int64_
 __device__ __forceinline__ void build_visit_flags(const Shape &s, const int32_t *idxrow, int qb,
                                                   int *flags) {
   const int t0 = qb * s.Bk, t1 = min(s.L, t0 + s.Bk) - 1;
-  for (int blk = threadIdx.x; blk <= qb; blk += blockDim.x) {
+  const int last = s.causal ? qb : s.M - 1;  // without the causal mask later blocks are visited too
+  for (int blk = threadIdx.x; blk <= last; blk += blockDim.x) {
     int f = st_ranges_touch(s, t0, t1, blk * s.Bk, min(s.L, blk * s.Bk + s.Bk) - 1) ? 2 : 0;
     for (int i = 0; i < s.topk; ++i) f |= (idxrow[i] == blk) ? 1 : 0;
     flags[blk] = f;
@@ -129,7 +130,7 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
   __syncthreads();
 
   if (block_live) {
-    for (int blk = 0; blk <= qb; ++blk) {
+    for (int blk = 0; blk <= (s.causal ? qb : s.M - 1); ++blk) {
       const int f = flags[blk];
       if (!f) continue;
       __syncthreads();
@@ -138,7 +139,7 @@ __global__ void __launch_bounds__(256) fwd_simt_kernel(
       __syncthreads();
       if (!active) continue;
       const int p0 = blk * s.Bk;
-      const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
+      const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), s.causal ? t - p0 + 1 : s.Bk);
       const bool selb = s.pq ? (rowsel[r * MW + (blk >> 5)] >> (blk & 31)) & 1u : f & 1;
       for (int pi = pbeg; pi < pend; ++pi) {
         const bool inS = st_visible(s, t, p0 + pi);
@@ -295,7 +296,7 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
   __syncthreads();
 
   if (block_live) {
-    for (int blk = 0; blk <= qb; ++blk) {
+    for (int blk = 0; blk <= (s.causal ? qb : s.M - 1); ++blk) {
       const int f = flags[blk];
       if (!f) continue;
       __syncthreads();
@@ -304,7 +305,7 @@ __global__ void __launch_bounds__(256) bwd_dq_simt_kernel(
       __syncthreads();
       if (!active) continue;
       const int p0 = blk * s.Bk;
-      const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), t - p0 + 1);
+      const int pbeg = max(0, pad0 - p0), pend = min(min(s.Bk, s.L - p0), s.causal ? t - p0 + 1 : s.Bk);
       const bool selb = s.pq ? (rowsel[r * MW + (blk >> 5)] >> (blk & 31)) & 1u : f & 1;
       for (int pi = pbeg; pi < pend; ++pi) {
         const bool inS = st_visible(s, t, p0 + pi);
@@ -405,7 +406,8 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
 
   // which query blocks visit this key block: bit 0 = selected it, bit 1 = their short-term branch
   // may reach it
-  for (int qb = j + tid; qb < s.M; qb += blockDim.x) {
+  const int q0 = s.causal ? j : 0, nqv = s.M - q0;  // the query blocks that may visit this key block
+  for (int qb = q0 + tid; qb < s.M; qb += blockDim.x) {
     const int32_t *row = idx + ((int64_t)uk * s.M + qb) * s.topk;  // (read only when the selection is per block)
     int f = st_ranges_touch(s, qb * s.Bk, min(s.L, qb * s.Bk + s.Bk) - 1, j * s.Bk,
                             min(s.L, j * s.Bk + s.Bk) - 1) ? 2 : 0;
@@ -429,8 +431,8 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
   __syncthreads();
 
   if (block_live) {
-    for (int x = 0; x < s.G * (s.M - j); ++x) {  // every query head of the group, every later query block
-      const int h = hk * s.G + x / (s.M - j), qb = j + x % (s.M - j);
+    for (int x = 0; x < s.G * nqv; ++x) {  // every query head of the group, every query block that may visit
+      const int h = hk * s.G + x / nqv, qb = q0 + x % nqv;
       const int64_t u = (int64_t)n * s.H + h;
       const float alpha_h = s.gate_mode ? 0.f : sigmoidf_(gate[h * 2 + 0] - gate[h * 2 + 1]);
       int f = flags[qb];
@@ -481,7 +483,7 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
         uS = group_sum(uS, gmask);
       }
       const int t0 = qb * s.Bk;
-      const int tbeg = max(0, p - t0), tend = min(s.Bk, s.L - t0);  // t >= p >= pad0
+      const int tbeg = s.causal ? max(0, p - t0) : max(0, pad0 - t0), tend = min(s.Bk, s.L - t0);  // valid t (>= p if causal)
       const bool sel_all = f & 1;
       for (int ti = tbeg; ti < tend; ++ti) {
         const bool selb = s.pq ? rsel[ti] != 0 : sel_all;

@@ -19,6 +19,7 @@ struct Shape {
   int64_t sb, sh, sl;  // element strides of q-shaped tensors
   int Hkv, G;             // key/value heads and query heads per key/value head (H = Hkv * G)
   int pq;                 // 1: one selection per query position (block_idx is [B][Hkv][L][top_k])
+  int causal;             // 1: causal mask (default); 0: bidirectional (CUDA-core kernels)
   int gate_mode;          // 0: one gate weight per head from two logits; 1: Eq. 18's input-dependent gate
   const float *phi;       // logits of the learnable block summary (Eq. 9) or nullptr = the mean
   int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
@@ -100,19 +101,22 @@ __device__ __forceinline__ int64_t row_offset_kv(const Shape &s, int n, int hk, 
 }
 
 // ---- the short-term mask (Eq. 15), shared by the CUDA-core and the tensor-core kernels ----
-// Eq. 15 on the causal side: may query t attend to key p <= t in the short-term branch?
-// Mode 0: the window alone.  Mode 1 (power-law mask): the window, or the block-index distance
-// floor(t / blk) - floor(p / blk) is a power of two, or p is one of the last blk positions.
+// Eq. 15: may query t attend to key p in the short-term branch?  (Under the causal mask callers
+// only ask for p <= t.)  Mode 0: the window alone, |t - p| < w.  Mode 1 (power-law mask): the
+// window, or the block-index distance |floor(t / blk) - floor(p / blk)| is a power of two, or p is
+// one of the last blk positions.
 __device__ __forceinline__ bool st_visible(const Shape &s, int t, int p) {
-  if (t - p < s.window) return true;
+  if (abs(t - p) < s.window) return true;
   if (s.stis_mode == 0) return false;
-  const int bd = t / s.stis_blk - p / s.stis_blk;
+  const int bd = abs(t / s.stis_blk - p / s.stis_blk);
   return (bd >= 1 && (bd & (bd - 1)) == 0) || p >= s.L - s.stis_blk;
 }
 // May some query in [t0, t1] see some key in [p0, p1] (p0 <= t1) through the short-term branch?
 // Exact for the window; for the power-law mask a superset (any power of two inside the range of
 // block distances counts), which only costs a visit: st_visible decides every pair.
 __device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, int p0, int p1) {
+  if (!s.causal)  // keys on both sides: exact for the window, every range for the power-law mask
+    return s.stis_mode != 0 || (t0 - p1 < s.window && p0 - t1 < s.window);
   if (t0 - p1 < s.window) return true;
   if (s.stis_mode == 0) return false;
   if (p1 >= s.L - s.stis_blk) return true;

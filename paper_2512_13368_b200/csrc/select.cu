@@ -253,6 +253,19 @@ __device__ __forceinline__ void row_group_sums(const float (&p)[8][8], float *pa
     }
 }
 
+// ascending: the flagged blocks of [lo, hi), then -1
+__device__ __forceinline__ void emit_flags(int32_t *row, const uint8_t *taken, int lo, int hi, int topk, int lane) {
+  int pos = 0;
+  for (int base = lo; base < hi; base += 32) {
+    const int j = base + lane;
+    const bool f = j < hi && taken[j];
+    const unsigned m = __ballot_sync(0xffffffffu, f);
+    if (f) row[pos + __popc(m & ((1u << lane) - 1u))] = j;
+    pos += __popc(m);
+  }
+  for (int i = pos + lane; i < topk; i += 32) row[i] = -1;
+}
+
 // ---- stage 1: single-precision scoring with an error bound ----------------------------------
 // A CTA of 128 threads takes 128 consecutive positions of one (batch, key/value head): 128 / Bk
 // query blocks.  Logits against 64 candidate means at a time come from a register-blocked fp32
@@ -587,8 +600,11 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
       continue;
     }
     const int cmin = first_live_scored(g, pad0), jmin = pad0 / Bk;
-    const int nc = n_candidates(sh, g, b), ncand = max(0, nc - cmin);
-    const int nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
+    // without the causal mask (plain selection only) every other live block is a candidate
+    const int hi = sh.causal ? b : M;
+    const int nc = sh.causal ? n_candidates(sh, g, b) : g.n;
+    const int ncand = max(0, nc - cmin - (sh.causal ? 0 : 1));
+    const int nsel = max(0, hi - jmin - (sh.causal ? 0 : 1)), want = min(sh.topk - 1, nsel);
     const bool choose = nsel > want && want > 0;
 
     if (choose && ncand > 0) {
@@ -638,7 +654,8 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
               z[k] *= sh.scale_d;
-              if (row_on && part + 4 * k < nb && c0 + part + 4 * k >= cmin) on |= 1u << k;
+              const int c = c0 + part + 4 * k;
+              if (row_on && part + 4 * k < nb && c >= cmin && (sh.causal || c != b)) on |= 1u << k;
             }
             if (pass == 0) {
               double cm = -INFINITY;
@@ -682,16 +699,24 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
     __syncthreads();
     if (warp == 0) {
       if (!choose) {
-        for (int j = jmin + lane; j < b; j += 32) taken[j] = want > 0 ? 1 : 0;
+        for (int j = jmin + lane; j < hi; j += 32) taken[j] = want > 0 ? 1 : 0;
       } else if (ncand == 0) {
-        for (int j = jmin + lane; j < b; j += 32) taken[j] = j - jmin < want ? 1 : 0;
+        for (int j = jmin + lane; j < hi; j += 32) taken[j] = j - jmin < want ? 1 : 0;
       } else {
-        map_scores<double>(g, Sc, cmin, nc, jmin, b, S, lane);
+        map_scores<double>(g, Sc, cmin, nc, jmin, hi, S, lane);
         __syncwarp();
-        rank_select<double>(S, jmin, b, want, taken, bound_d, lane);
+        if (!sh.causal && lane == 0) S[b] = -INFINITY;  // the own block is not ranked: it is kept anyway
+        __syncwarp();
+        rank_select<double>(S, jmin, hi, want, taken, bound_d, lane);
       }
       __syncwarp();
-      emit_row(row, taken, jmin, b, sh.topk, lane);
+      if (sh.causal) {
+        emit_row(row, taken, jmin, b, sh.topk, lane);
+      } else {  // the own block takes its place in the ascending row
+        if (lane == 0) taken[b] = 1;
+        __syncwarp();
+        emit_flags(row, taken, jmin, hi, sh.topk, lane);
+      }
     }
   }
 }
@@ -817,7 +842,8 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
   }
   int sc_pitch = 0, sc_len = 0;
   const size_t fsm = fast_smem_bytes(sh, g, D, &sc_pitch);
-  const bool exact_only = exact_select_only() || fsm == 0;
+  // (without the causal mask the candidates are not a prefix of the blocks: double precision only)
+  const bool exact_only = exact_select_only() || fsm == 0 || !sh.causal;
   if (!exact_only) {
     if (fsm > 48 * 1024 && cudaFuncSetAttribute(score_fast_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)fsm) != cudaSuccess)

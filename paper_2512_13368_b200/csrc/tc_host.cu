@@ -76,7 +76,7 @@ int launch_wait_selftest(int32_t *status, cudaStream_t st) {
 bool fwd_tc_supported(const Shape &s, int dtype) {
   // (a selection per query position gives every row its own key blocks: CUDA-core kernels)
   // (and so does the input-dependent gate, whose backward adds rank-one terms to both branches)
-  return !s.pq && !s.gate_mode && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  return s.causal && !s.pq && !s.gate_mode && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 

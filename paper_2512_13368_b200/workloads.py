@@ -67,6 +67,7 @@ class Workload:
     per_query: int = 0    # 1: one selection per query position (Eq. 13 as printed) instead of per query block
     phi_logits: np.ndarray | None = field(default=None, repr=False)  # learnable block summary (Eq. 9) or None = mean
     gate_mode: int = 0    # 1: Eq. 18's input-dependent gate, gate is [H, 2 D + 1] = (w_lt, w_st, b)
+    causal: int = 1       # 0: no causal mask (bidirectional encoder)
 
     @property
     def n_blocks(self) -> int:
@@ -87,7 +88,7 @@ class Workload:
                         self.q[n:n + 1, hq].copy(), self.k[n:n + 1, h:h + 1].copy(),
                         self.v[n:n + 1, h:h + 1].copy(), self.gate[hq].copy(),
                         self.dout[n:n + 1, hq].copy(), sl, self.stis_mode, self.stis_block,
-                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0, self.per_query, self.phi_logits, self.gate_mode)
+                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0, self.per_query, self.phi_logits, self.gate_mode, self.causal)
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,

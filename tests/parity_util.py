@@ -37,14 +37,16 @@ def check_indices(w, gpu_idx, sm_scale=None):
     elif _grouped(w):
         ref_idx, scores = oracle.select_blocks_gqa(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
                                                    return_scores=True, cmp_block=w.cmp_block,
-                                                   cmp_stride=w.cmp_stride, phi_logits=phi)
+                                                   cmp_stride=w.cmp_stride, phi_logits=phi,
+                                                   causal=bool(getattr(w, "causal", 1)))
     elif w.cmp_block or w.cmp_stride:
         ref_idx, scores, _ = oracle.select_blocks_cmp(w.q, w.k, w.block, w.topk, w.cmp_block or w.block,
                                                       w.cmp_stride or w.block, w.seq_lens, sm_scale,
                                                       return_scores=True, phi_logits=phi)
     else:
         ref_idx, scores = oracle.select_blocks(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
-                                                return_scores=True, phi_logits=phi)
+                                                return_scores=True, phi_logits=phi,
+                                                causal=bool(getattr(w, "causal", 1)))
     assert gpu_idx.shape == ref_idx.shape and gpu_idx.dtype == np.int32
     bad = np.argwhere((gpu_idx != ref_idx).any(-1))
     forgiven = 0
@@ -56,12 +58,19 @@ def check_indices(w, gpu_idx, sm_scale=None):
         else:
             S = scores[n, h, b, :b]
             ref_row, gpu_row = ref_idx[n, h, b], gpu_idx[n, h, b]
-        ref_sel = [j for j in ref_row if 0 <= j < b]
-        gpu_sel = [j for j in gpu_row if 0 <= j < b]
+        causal = bool(getattr(w, "causal", 1))
+        own = b
+        cand = np.arange(b) if causal else np.array([j for j in range(scores.shape[-1]) if j != b])
+        if not causal:
+            S = scores[n, h, b]
+        ref_sel = [j for j in ref_row if j >= 0 and j != own]
+        gpu_sel = [j for j in gpu_row if j >= 0 and j != own]
         # structure must still be valid
         g = [int(j) for j in gpu_row if j >= 0]
-        assert g == sorted(set(g)) and g[-1] == b and len(g) == len(ref_sel) + 1, (n, h, b, g)
-        dropped = np.setdiff1d(np.arange(b), ref_sel)
+        assert g == sorted(set(g)) and own in g and len(g) == len(ref_sel) + 1, (n, h, b, g)
+        if causal:
+            assert g[-1] == own
+        dropped = np.setdiff1d(cand, ref_sel)
         kept_min = S[ref_sel].min()
         drop_max = S[dropped].max()
         gap = abs(kept_min - drop_max) / max(abs(kept_min), abs(drop_max))
@@ -86,6 +95,8 @@ def check_forward_backward(w, res, sm_scale=None, backward=True):
     kw = {"per_query": True} if getattr(w, "per_query", 0) else {}
     if getattr(w, "gate_mode", 0):
         kw["gate_mode"] = 1
+    if not getattr(w, "causal", 1):
+        kw["causal"] = False
     ref = fwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, w.seq_lens, sm_scale,
                  idx=res["idx"], stis_mode=w.stis_mode, stis_block=w.stis_block, **kw)
     errs = {"near_tie_rows": forgiven}

@@ -48,7 +48,7 @@ def test_workspace_bytes(lib):
     assert n > 0 and n % 256 == 0
     assert binding.blossom_workspace_bytes(good(batch=8)) > n
     for bad in (dict(batch=0), dict(head_dim=48), dict(block_size=12), dict(top_k=0), dict(window=0),
-                dict(kv_heads=3), dict(kv_heads=0), dict(kv_strides=(4096, 2048, 31)), dict(causal=0), dict(select_mode=2), dict(select_mode=1, cmp_block=16, cmp_stride=4), dict(dtype=7),
+                dict(kv_heads=3), dict(kv_heads=0), dict(kv_strides=(4096, 2048, 31)), dict(causal=2), dict(causal=0, select_mode=1), dict(select_mode=2), dict(select_mode=1, cmp_block=16, cmp_stride=4), dict(dtype=7),
                 dict(seq_len=8 * 1025), dict(strides=(4096, 2048, 33)), dict(sm_scale=-1.0),
                 dict(stis_mode=2), dict(stis_mode=-1), dict(stis_mode=1, stis_block=-3),
                 dict(cmp_block=12, cmp_stride=8), dict(cmp_block=16, cmp_stride=3), dict(cmp_block=-8)):

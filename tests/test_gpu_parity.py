@@ -612,3 +612,23 @@ def test_input_dependent_gate(runner, dtype, L, D, H, Hkv, block, topk, window, 
     _, res = run(runner, w)
     assert res["dgate"].shape == (H, 2 * D + 1)
     print(check_forward_backward(w, res))
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens,power_law", [
+    (64, 32, 2, 2, 8, 3, 5, None, False),
+    (200, 32, 2, 2, 16, 4, 9, [200, 5, 77, 0], False),       # padded, ragged last block
+    (300, 64, 4, 2, 32, 4, 17, [300, 131], True),            # grouped heads, symmetric power-law mask
+    (512, 64, 2, 2, 64, 8, 600, None, False),                # everything visible: dense bidirectional attention
+])
+def test_without_the_causal_mask(runner, dtype, L, D, H, Hkv, block, topk, window, lens, power_law):
+    """causal = 0 (the bidirectional encoders of the paper's transfer experiment): selection among
+    all other live blocks, attention over whole selected blocks, symmetric Eq. 15."""
+    B = len(lens) if lens else 2
+    w = workloads.make("non-causal", dtype, B, H, L, D, block, topk, window, seed=73, kv_heads=Hkv if Hkv != H else 0,
+                       stis_mode=1 if power_law else 0, stis_block=2 if power_law else 1)
+    w.causal = 0
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    _, res = run(runner, w)
+    print(check_forward_backward(w, res))
