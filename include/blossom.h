@@ -105,6 +105,12 @@ typedef struct {
                         * alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row,
                         * broadcast over the head's channels in Eq. 19; runs on the CUDA-core
                         * kernels                                                                 */
+  float rope_theta;    /* 0 = q and k are used as given.  > 0 (>= 1, e.g. 10000): rotary position
+                        * embedding inside the library: q and k are rotated by position before the
+                        * selection and both branches (pairs (x[2i], x[2i+1]), angle
+                        * t * rope_theta^(-2i / D) at array position t, evaluated in double precision
+                        * and rounded once to the storage type; the copies live in the workspace),
+                        * and blossom_attn_bwd returns dq, dk with respect to the unrotated inputs  */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

@@ -9,6 +9,6 @@ from .blossom_oracle import (  # noqa: F401
     forward,
     backward,
     forward_backward,
-    select_blocks, select_blocks_cmp, select_blocks_gqa, select_blocks_per_query, forward_gqa, backward_gqa,
+    select_blocks, select_blocks_cmp, select_blocks_gqa, select_blocks_per_query, rope, forward_gqa, backward_gqa,
     threads,
 )

@@ -270,6 +270,42 @@ def forward_backward(q, k, v, gate, dout, block, topk, window, seq_lens=None, sm
     return f
 
 
+# ---------------------------------------------------------------------------- rotary positions
+# The paper applies RoPE to Q and K before both branches.  Original formulation: the pairs
+# (x[2i], x[2i+1]) of a row at position t are rotated by the angle t * theta^(-2i / D).
+def _round_to_bf16(x):
+    """float64 -> the nearest bfloat16 value (ties to even), returned as float64."""
+    x = np.asarray(x, dtype=np.float64)
+    f = x.astype(np.float32)
+    u = f.view(np.uint32)
+    lo = (u & np.uint32(0xFFFF0000)).view(np.float32).astype(np.float64)       # toward zero
+    hi = ((u & np.uint32(0xFFFF0000)) + np.uint32(0x10000)).view(np.float32).astype(np.float64)
+    dl, dh = np.abs(x - lo), np.abs(hi - x)
+    lo_even = ((u >> np.uint32(16)) & np.uint32(1)) == 0
+    return np.where((dl < dh) | ((dl == dh) & lo_even), lo, hi)
+
+
+def rope(x, theta, dtype=None, transpose=False):
+    """Rotate ``x [..., L, D]`` by position; ``transpose`` applies the inverse rotation (what the
+    chain rule needs for the gradient with respect to the unrotated tensor).  ``dtype`` 'bf16' /
+    'fp32' rounds the result once to that storage type; None keeps float64."""
+    x = _f64(x)
+    L, D = x.shape[-2], x.shape[-1]
+    i = np.arange(D // 2, dtype=np.float64)
+    ang = np.arange(L, dtype=np.float64)[:, None] * np.power(float(theta), -2.0 * i / D)[None, :]
+    if transpose:
+        ang = -ang
+    cs, sn = np.cos(ang), np.sin(ang)
+    out = np.empty_like(x)
+    out[..., 0::2] = x[..., 0::2] * cs - x[..., 1::2] * sn
+    out[..., 1::2] = x[..., 0::2] * sn + x[..., 1::2] * cs
+    if dtype == "bf16":
+        return _round_to_bf16(out)
+    if dtype == "fp32":
+        return out.astype(np.float32).astype(np.float64)
+    return out
+
+
 # ---------------------------------------------------------------------------- grouped-query
 # Grouped-query attention: H query heads share Hkv key/value heads, G = H / Hkv query heads per
 # group, query head h using key/value head h // G.  The importance scores of the heads of a group

@@ -65,7 +65,7 @@ class _BlossomAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, gate_logits, seq_lens, block_size, top_k, window, sm_scale,
                 stis_mode, stis_block, cmp_block, cmp_stride, per_query=0, phi_logits=None,
-                gate_mode=0, causal=1):
+                gate_mode=0, causal=1, rope_theta=0.0):
         seq_lens = check_arguments(q, k, v, gate_logits, seq_lens, gate_mode=gate_mode)
         B, H, L, D = q.shape
         Hkv = k.shape[1]
@@ -81,7 +81,8 @@ class _BlossomAttention(torch.autograd.Function):
                                      sm_scale=sm_scale, strides=q.stride()[:3], stis_mode=stis_mode,
                                      stis_block=stis_block, cmp_block=cmp_block, cmp_stride=cmp_stride,
                                      kv_heads=Hkv, kv_strides=k.stride()[:3], select_mode=int(per_query),
-                                     phi_logits=phi_logits, gate_mode=int(gate_mode), causal=int(causal))
+                                     phi_logits=phi_logits, gate_mode=int(gate_mode), causal=int(causal),
+                                     rope_theta=float(rope_theta))
         nbytes = binding.blossom_workspace_bytes(params)
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
@@ -110,12 +111,12 @@ class _BlossomAttention(torch.autograd.Function):
         dgate = torch.empty(tuple(gate.shape), dtype=torch.float32, device=q.device)
         binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
-        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 13
+        return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 14
 
 
 def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=None, sm_scale=0.0,
                       return_indices=False, short_term="window", mask_block=1, cmp_block=0,
-                      cmp_stride=0, select_per_query=False, phi_logits=None, input_dependent_gate=False, causal=True):
+                      cmp_stride=0, select_per_query=False, phi_logits=None, input_dependent_gate=False, causal=True, rope_theta=0.0):
     """Gated two-branch sparse attention of q [B, H, L, D] and k, v [B, Hkv, L, D] (float32 or
     bfloat16, CUDA; Hkv divides H: with Hkv < H the query heads of a group share key/value head
     and selection, and the returned indices are [B, Hkv, M, top_k]).
@@ -137,6 +138,8 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     causal: False drops the causal mask (bidirectional encoders): a query block scores every other
     live block, a query sees all valid keys of its selected blocks, Eq. 15 is symmetric; runs on the
     CUDA-core kernels.
+    rope_theta: > 0 applies rotary position embedding to q and k inside the library (interleaved
+    pairs, angle t * rope_theta^(-2i / D)); the gradients returned are those of the unrotated q, k.
     phi_logits: optional float32 CUDA tensor [cmp_block or block_size]: Eq. 9's learnable block
     summary as a softmax pooling over a block's positions (None = the mean).  It only steers the
     selection, which is not differentiated, so it receives no gradient here.
@@ -153,5 +156,5 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
                                        int(window), float(sm_scale),
                                        1 if short_term == "power-law" else 0, int(mask_block),
                                        int(cmp_block), int(cmp_stride), int(bool(select_per_query)), phi_logits,
-                                       int(bool(input_dependent_gate)), int(bool(causal)))
+                                       int(bool(input_dependent_gate)), int(bool(causal)), float(rope_theta))
     return (out, idx) if return_indices else out

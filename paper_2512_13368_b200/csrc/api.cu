@@ -84,6 +84,13 @@ Workspace carve_workspace(const Shape &s, void *base) {
   w.clive = reinterpret_cast<int32_t *>(take(units * (size_t)s.Mc * sizeof(int32_t)));
   w.cmean32 = reinterpret_cast<float *>(take(units * (size_t)s.Mc * s.D * sizeof(float)));
   w.cnorm = reinterpret_cast<float *>(take(units * (size_t)s.Mc * sizeof(float)));
+  {
+    // rotated copies of q and k span what the originals span (same strides)
+    const size_t qspan = (size_t)((s.B - 1) * s.sb + (s.H - 1) * s.sh + (int64_t)(s.L - 1) * s.sl + s.D);
+    const size_t kspan = (size_t)((s.B - 1) * s.ksb + (s.Hkv - 1) * s.ksh + (int64_t)(s.L - 1) * s.ksl + s.D);
+    w.q_rot = take(s.rope_theta > 0 ? qspan * s.esz : 0);
+    w.k_rot = take(s.rope_theta > 0 ? kspan * s.esz : 0);
+  }
   w.gate_ac = reinterpret_cast<float *>(take(s.gate_mode ? 2 * units * s.L * sizeof(float) : 0));
   w.dgate_part = reinterpret_cast<double *>(take(s.gate_mode ? units * s.M * (2 * s.D + 1) * sizeof(double) : 0));
   w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
@@ -140,6 +147,10 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.Hkv = p->kv_heads; s.G = p->heads / p->kv_heads;
   if (p->gate_mode < 0 || p->gate_mode > 1) return BLOSSOM_ERR_INVALID_ARG;
   s.gate_mode = p->gate_mode;
+  if (!(p->rope_theta >= 0.f) || isinf(p->rope_theta) || (p->rope_theta > 0.f && p->rope_theta < 1.f))
+    return BLOSSOM_ERR_INVALID_ARG;
+  s.rope_theta = (double)p->rope_theta;
+  s.esz = p->dtype == BLOSSOM_DTYPE_BF16 ? 2 : 4;
   s.pq = p->select_mode;
   s.causal = p->causal;
   if (!s.causal && (s.pq || s.cmp_l > 0)) return BLOSSOM_ERR_UNSUPPORTED;  // bidirectional: plain per-block selection
@@ -154,6 +165,19 @@ static int make_shape(const blossom_params *p, Shape *out) {
     s.ksl = s.D; s.ksh = (int64_t)s.L * s.D; s.ksb = (int64_t)s.Hkv * s.L * s.D;
   }
   *out = s;
+  return BLOSSOM_OK;
+}
+
+// With rope_theta > 0: rotated copies of q and k go to the workspace and *q, *k point at them.
+static int rotate_inputs(const Shape &s, int dtype, const Workspace &ws, const void **q, const void **k,
+                         cudaStream_t st) {
+  if (s.rope_theta <= 0) return BLOSSOM_OK;
+  int rc = launch_rope(s, dtype, false, +1, *q, ws.q_rot, st);
+  if (rc) return rc;
+  rc = launch_rope(s, dtype, true, +1, *k, ws.k_rot, st);
+  if (rc) return rc;
+  *q = ws.q_rot;
+  *k = ws.k_rot;
   return BLOSSOM_OK;
 }
 
@@ -198,6 +222,8 @@ int blossom_select_blocks(const blossom_params *params, const void *q, const voi
   Workspace ws;
   rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
   if (rc) return rc;
+  rc = rotate_inputs(s, params->dtype, ws, &q, &k, (cudaStream_t)stream);
+  if (rc) return rc;
   return launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, (cudaStream_t)stream);
 }
 
@@ -233,6 +259,8 @@ int blossom_attn_fwd(const blossom_params *params, const void *q, const void *k,
   rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
+  rc = rotate_inputs(s, params->dtype, ws, &q, &k, st);
+  if (rc) return rc;
   if (!idx_is_input) {
     rc = launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, st);
     if (rc) return rc;
@@ -264,14 +292,22 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
   Workspace ws;
   rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws, true);
   if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  rc = rotate_inputs(s, params->dtype, ws, &q, &k, st);
+  if (rc) return rc;
   if (!force_simt() && tc::fwd_tc_supported(s, params->dtype)) {
     rc = tc::launch_bwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out_lt, out_st, lse, dout, dq,
-                           dk, dv, ws, (cudaStream_t)stream);
-    if (rc) return rc;
-    return launch_gate_grad(s, gate_logits, ws, dgate, (cudaStream_t)stream);
+                           dk, dv, ws, st);
+    if (!rc) rc = launch_gate_grad(s, gate_logits, ws, dgate, st);
+  } else {
+    rc = launch_bwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out_lt,
+                         out_st, lse, dout, dq, dk, dv, dgate, ws, st);
   }
-  return launch_bwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out_lt,
-                         out_st, lse, dout, dq, dk, dv, dgate, ws, (cudaStream_t)stream);
+  if (rc || s.rope_theta <= 0) return rc;
+  // dq, dk hold the gradients of the rotated tensors: turn them back (the transpose), in place
+  rc = launch_rope(s, params->dtype, false, -1, dq, dq, st);
+  if (rc) return rc;
+  return launch_rope(s, params->dtype, true, -1, dk, dk, st);
 }
 
 int blossom_device_status(const void *workspace, blossom_stream_t stream, int32_t *host_out) {
@@ -355,7 +391,7 @@ int blossom_profile_stop(int32_t *kernel_ids, float *ms, int capacity) {
 const char *blossom_kernel_name(int id) {
   static const char *names[K_COUNT] = {
       "summary", "score_select", "fwd_simt", "bwd_dq_simt", "bwd_dkdv_simt", "gate_grad",
-      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast", "bwd_prep", "tc_meta"};
+      "fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc", "score_fast", "bwd_prep", "tc_meta", "rope"};
   return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

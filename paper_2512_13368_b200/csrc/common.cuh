@@ -19,6 +19,8 @@ struct Shape {
   int64_t sb, sh, sl;  // element strides of q-shaped tensors
   int Hkv, G;             // key/value heads and query heads per key/value head (H = Hkv * G)
   int pq;                 // 1: one selection per query position (block_idx is [B][Hkv][L][top_k])
+  double rope_theta;      // > 0: q and k are rotated by position inside the library (base of the angles)
+  int esz;                // bytes per element of the q-shaped tensors (2 or 4)
   int causal;             // 1: causal mask (default); 0: bidirectional (CUDA-core kernels)
   int gate_mode;          // 0: one gate weight per head from two logits; 1: Eq. 18's input-dependent gate
   const float *phi;       // logits of the learnable block summary (Eq. 9) or nullptr = the mean
@@ -43,6 +45,7 @@ struct Workspace {
   int32_t *clive;    // [B][H][Mc]     their numbers of valid keys
   float *cmean32;    // [B][H][Mc][D]  the means rounded to fp32
   float *cnorm;      // [B][H][Mc]     upper bounds of the norms of the fp32 means
+  void *q_rot, *k_rot;  // rotated copies of q and k (rope_theta > 0), laid out with the originals' strides
   float *gate_ac;    // [2][B][H][L]  input-dependent gate: alpha_t and c_t of every row (backward)
   double *dgate_part;// [B][H][M][2 D + 1]  per query block partial of the gradient of F_o's parameters
   uint8_t *qmeta;    // per query-major CTA of the tensor-core kernels: tile lists (tc_meta_kernel)
@@ -57,7 +60,7 @@ extern unsigned long long g_launches;  // host-side launch counter
 // Kernel identifiers reported by the optional per-launch event profile.
 enum KernelId {
   K_SUMMARY = 0, K_SCORE_SELECT, K_FWD_SIMT, K_BWD_DQ_SIMT, K_BWD_DKDV_SIMT, K_GATE_GRAD,
-  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_BWD_PREP, K_TC_META, K_COUNT
+  K_FWD_TC, K_BWD_DQ_TC, K_BWD_DKDV_TC, K_SCORE_FAST, K_BWD_PREP, K_TC_META, K_ROPE, K_COUNT
 };
 void prof_mark(int id, int phase, cudaStream_t st);  // no-op unless a profile is running
 
@@ -142,6 +145,7 @@ int launch_select_static(const Shape &s, int dtype, const void *q, const void *k
 size_t select_static_capacity_bytes();
 int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, float *dgate,
                      cudaStream_t st);
+int launch_rope(const Shape &s, int dtype, bool kv, int dir, const void *src, void *dst, cudaStream_t st);
 
 namespace tc {
 int launch_wait_selftest(int32_t *status, cudaStream_t st);

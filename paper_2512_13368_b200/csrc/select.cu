@@ -917,7 +917,8 @@ size_t select_static_capacity_bytes() { return kStaticBytes; }
 
 int launch_select_static(const Shape &s, int dtype, const void *q, const void *k,
                          const int32_t *seq_lens, int32_t *idx, cudaStream_t st) {
-  if (s.cmp_l > 0 || s.pq) return BLOSSOM_ERR_UNSUPPORTED;  // the built-in scratch serves the plain selection
+  // the built-in scratch serves the plain selection (and has no room for rotated copies of q and k)
+  if (s.cmp_l > 0 || s.pq || s.rope_theta > 0) return BLOSSOM_ERR_UNSUPPORTED;
   const size_t blocks = (size_t)s.B * s.Hkv * s.M;  // every scratch array is per key/value head
   if (blocks > kStaticBlocks || blocks * (size_t)s.D > kStaticMeanElems) return BLOSSOM_ERR_TOO_LARGE;
   int dev = -1;

@@ -34,7 +34,8 @@ class DeviceProblem:
                                           stis_block=w.stis_block, cmp_block=w.cmp_block,
                                           cmp_stride=w.cmp_stride, kv_heads=w.kv_heads or w.H,
                                           select_mode=w.per_query, phi_logits=self.phi,
-                                          gate_mode=getattr(w, "gate_mode", 0), causal=getattr(w, "causal", 1))
+                                          gate_mode=getattr(w, "gate_mode", 0), causal=getattr(w, "causal", 1),
+                                          rope_theta=getattr(w, "rope_theta", 0.0))
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):

@@ -68,6 +68,7 @@ class Workload:
     phi_logits: np.ndarray | None = field(default=None, repr=False)  # learnable block summary (Eq. 9) or None = mean
     gate_mode: int = 0    # 1: Eq. 18's input-dependent gate, gate is [H, 2 D + 1] = (w_lt, w_st, b)
     causal: int = 1       # 0: no causal mask (bidirectional encoder)
+    rope_theta: float = 0.0  # > 0: q and k are rotated by position inside the library
 
     @property
     def n_blocks(self) -> int:
@@ -88,7 +89,7 @@ class Workload:
                         self.q[n:n + 1, hq].copy(), self.k[n:n + 1, h:h + 1].copy(),
                         self.v[n:n + 1, h:h + 1].copy(), self.gate[hq].copy(),
                         self.dout[n:n + 1, hq].copy(), sl, self.stis_mode, self.stis_block,
-                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0, self.per_query, self.phi_logits, self.gate_mode, self.causal)
+                        self.cmp_block, self.cmp_stride, 1 if G > 1 else 0, self.per_query, self.phi_logits, self.gate_mode, self.causal, self.rope_theta)
 
 
 def make(name, dtype, B, H, L, D, block, topk, window, seed, std=1.0, lengths=None,

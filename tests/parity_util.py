@@ -27,8 +27,22 @@ def _grouped(w):
     return bool(w.kv_heads) and w.kv_heads != w.H
 
 
+def _rotated(w):
+    """With rotary positions the library works on q, k rotated and rounded to the storage type."""
+    theta = getattr(w, "rope_theta", 0.0)
+    if not theta:
+        return w
+    import copy
+    w2 = copy.copy(w)
+    w2.q = oracle.rope(w.q, theta, w.dtype)
+    w2.k = oracle.rope(w.k, theta, w.dtype)
+    w2.rope_theta = 0.0
+    return w2
+
+
 def check_indices(w, gpu_idx, sm_scale=None):
     """Returns the number of forgiven near-tie rows; asserts on any real mismatch."""
+    w = _rotated(w)
     pq = bool(getattr(w, "per_query", 0))
     phi = getattr(w, "phi_logits", None)
     if pq:
@@ -90,6 +104,8 @@ def tolerance(w, ref):
 
 def check_forward_backward(w, res, sm_scale=None, backward=True):
     """res: dict of numpy arrays from the CUDA path.  Returns a dict of max-abs errors."""
+    theta = getattr(w, "rope_theta", 0.0)
+    w = _rotated(w)
     forgiven = check_indices(w, res["idx"], sm_scale)
     fwd_fn, bwd_fn = (oracle.forward_gqa, oracle.backward_gqa) if _grouped(w) else (oracle.forward, oracle.backward)
     kw = {"per_query": True} if getattr(w, "per_query", 0) else {}
@@ -104,6 +120,9 @@ def check_forward_backward(w, res, sm_scale=None, backward=True):
     if backward:
         ref.update(bwd_fn(w.q, w.k, w.v, w.gate, w.block, w.topk, w.window, ref, w.dout,
                           w.seq_lens, sm_scale, stis_mode=w.stis_mode, stis_block=w.stis_block, **kw))
+        if theta:   # gradients with respect to the unrotated q, k: the transpose of the rotation
+            ref["dq"] = oracle.rope(ref["dq"], theta, transpose=True)
+            ref["dk"] = oracle.rope(ref["dk"], theta, transpose=True)
         keys += ["dq", "dk", "dv", "dgate"]
     for key in keys:
         if res.get(key) is None:

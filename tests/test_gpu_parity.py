@@ -632,3 +632,24 @@ def test_without_the_causal_mask(runner, dtype, L, D, H, Hkv, block, topk, windo
         w.seq_lens = np.asarray(lens, dtype=np.int32)
     _, res = run(runner, w)
     print(check_forward_backward(w, res))
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens", [
+    (64, 32, 2, 2, 8, 2, 16, None),
+    (200, 32, 2, 2, 16, 4, 32, [200, 5, 77, 0]),
+    (700, 64, 4, 2, 32, 5, 70, [700, 129]),              # tensor-core kernels (bf16) on the rotated copies
+    (1024, 64, 2, 2, 64, 8, 256, None),
+])
+def test_rotary_positions_inside_the_library(runner, dtype, L, D, H, Hkv, block, topk, window, lens):
+    """rope_theta > 0: q and k are rotated by position inside the library before the selection and
+    both branches, and the backward returns gradients with respect to the unrotated q and k."""
+    B = len(lens) if lens else 2
+    w = workloads.make("rope", dtype, B, H, L, D, block, topk, window, seed=79, kv_heads=Hkv if Hkv != H else 0)
+    w.rope_theta = 10000.0
+    if lens is not None:
+        w.seq_lens = np.asarray(lens, dtype=np.int32)
+    p, res = run(runner, w)
+    print(check_forward_backward(w, res))
+    # the inputs are left as they were (the rotated copies live in the workspace)
+    assert np.array_equal(p.q.float().cpu().numpy(), w.q) and np.array_equal(p.k.float().cpu().numpy(), w.k)
