@@ -26,7 +26,11 @@
 // want them.
 #include "common.cuh"
 
+#include <cooperative_groups.h>
+
 namespace blossom {
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -567,6 +571,12 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
 // against 64 candidate means at a time: thread (row tid / 4, part tid % 4) forms the 16 logits of
 // candidates part + 4 k, so sixteen independent accumulation chains are in flight; softmax per row
 // by 4 lanes; the probabilities go through a shared tile for the column sums (fixed order).
+// Launched in thread-block clusters when a query block has more than 64 rows (grouped heads): CTA
+// r of a cluster takes the row chunks r, r + cluster size, ..., and CTA 0 adds the other CTAs'
+// column sums to its own in rank order out of their shared memory, which with one chunk per CTA
+// is the order a single CTA adds them in.  The work of a query block is otherwise serial, and the
+// work list is short (a few per cent of the query blocks), so without the split the kernel's time
+// is that of one CTA walking G * Bk rows.
 template <typename T, int D>
 __global__ void __launch_bounds__(256) score_exact_kernel(
     Shape sh, SelGeom g, const T *__restrict__ q, const double *__restrict__ mean,
@@ -586,7 +596,10 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rt = tid >> 2, part = tid & 3;
   const int total = worklist ? *work_count : M * sh.B * sh.Hkv;
-  for (int wi = blockIdx.x; wi < total; wi += gridDim.x) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int nrank = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  // (every CTA of a cluster walks the same query blocks, so the cluster barriers below match up)
+  for (int wi = blockIdx.x / nrank; wi < total; wi += gridDim.x / nrank) {
     const int row_id = worklist ? worklist[wi] : wi;
     const int b = row_id % M, u = row_id / M, n = u / sh.Hkv, hk = u % sh.Hkv;
     int len = seq_lens ? seq_lens[n] : sh.L;
@@ -596,7 +609,8 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
     int32_t *row = idx + ((int64_t)u * M + b) * sh.topk;
     __syncthreads();  // shared memory is reused from the previous query block
     if (qlo >= qhi) {  // the query block holds only padding
-      for (int i = tid; i < sh.topk; i += 256) row[i] = -1;
+      if (rank == 0)
+        for (int i = tid; i < sh.topk; i += 256) row[i] = -1;
       continue;
     }
     const int cmin = first_live_scored(g, pad0), jmin = pad0 / Bk;
@@ -613,7 +627,7 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
       const int ch_lo = cmin / 64, ch_hi = (nc + 63) / 64;
       const int npass = ch_hi - ch_lo > 1 ? 2 : 1;
       const double *kbase = mean + (int64_t)u * g.n * D;
-      for (int r0 = 0; r0 < nrows; r0 += 64) {
+      for (int r0 = 64 * rank; r0 < nrows; r0 += 64 * nrank) {
         const int nr = min(64, nrows - r0);
         __syncthreads();
         for (int i = tid; i < 64 * (D / 4); i += 256) {  // 64 query rows as doubles, missing rows zero
@@ -695,6 +709,18 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
           }
         }
       }
+    }
+    if (nrank > 1) {
+      cluster.sync();  // every CTA's column sums are complete
+      if (rank == 0 && choose && ncand > 0) {
+        for (int c = cmin + tid; c < nc; c += 256) {
+          double a = Sc[c];
+          for (int r = 1; r < nrank; ++r) a += cluster.map_shared_rank(Sc, r)[c];
+          Sc[c] = a;
+        }
+      }
+      cluster.sync();  // the other CTAs' sums have been read: they may go on (or exit)
+      if (rank != 0) continue;
     }
     __syncthreads();
     if (warp == 0) {
@@ -861,9 +887,25 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
     // double precision: every query block (exact_only) or the work list of the kernel above
     LaunchScope ls(K_SCORE_SELECT, st);
     const int64_t rows = units * sh.M;
-    const unsigned g2 = (unsigned)(rows < 592 ? rows : 592);
-    score_exact_kernel<T, D><<<g2, 256, esm, st>>>(sh, g, q, w.mean, seq_lens, idx, exact_only ? nullptr : w.list,
-                                                   w.count, sc_len);
+    const int chunks = (sh.G * sh.Bk + 63) / 64;  // 64-row chunks of a query block
+    const unsigned cl = chunks >= 8 ? 8u : chunks >= 4 ? 4u : chunks >= 2 ? 2u : 1u;
+    const int64_t max_clusters = 592 / cl;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(rows < max_clusters ? rows : max_clusters) * cl);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = esm;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cl;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, score_exact_kernel<T, D>, sh, g, q, (const double *)w.mean, seq_lens, idx,
+                           (const int32_t *)(exact_only ? nullptr : w.list), (const int32_t *)w.count,
+                           sc_len) != cudaSuccess)
+      return BLOSSOM_ERR_CUDA;
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
