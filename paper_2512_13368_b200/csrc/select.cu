@@ -577,8 +577,8 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
 // is the order a single CTA adds them in.  The work of a query block is otherwise serial, and the
 // work list is short (a few per cent of the query blocks), so without the split the kernel's time
 // is that of one CTA walking G * Bk rows.
-template <typename T, int D>
-__global__ void __launch_bounds__(256) score_exact_kernel(
+template <typename T, int D, int NZ>  // NZ: chunks of 64 candidates whose logits a thread may keep in registers
+__global__ void __launch_bounds__(256, 2) score_exact_kernel(
     Shape sh, SelGeom g, const T *__restrict__ q, const double *__restrict__ mean,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, const int32_t *__restrict__ worklist,
     const int32_t *__restrict__ work_count, int sc_len) {
@@ -625,7 +625,6 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
       for (int c = cmin + tid; c < nc; c += 256) Sc[c] = 0.0;
       const int nq = qhi - qlo, nrows = nq * sh.G;  // rows: head r / nq of the group, query qlo + r % nq
       const int ch_lo = cmin / 64, ch_hi = (nc + 63) / 64;
-      const int npass = ch_hi - ch_lo > 1 ? 2 : 1;
       const double *kbase = mean + (int64_t)u * g.n * D;
       for (int r0 = 64 * rank; r0 < nrows; r0 += 64 * nrank) {
         const int nr = min(64, nrows - r0);
@@ -641,71 +640,103 @@ __global__ void __launch_bounds__(256) score_exact_kernel(
           d[0] = (double)v.x; d[1] = (double)v.y; d[2] = (double)v.z; d[3] = (double)v.w;
         }
         const bool row_on = rt < nr;
-        double mx = -INFINITY, den = 0.0;
-        for (int pass = 0; pass < npass; ++pass) {
-          for (int ch = ch_lo; ch < ch_hi; ++ch) {
-            const int c0 = ch * 64, nb = min(64, nc - c0);
-            __syncthreads();  // previous users of kd are done
-            for (int i = tid; i < 64 * (D / 2); i += 256) {
-              const int lj = i / (D / 2), c = (i % (D / 2)) * 2;
-              double2 v = make_double2(0.0, 0.0);
-              if (lj < nb && c0 + lj >= cmin) v = *reinterpret_cast<const double2 *>(kbase + (int64_t)(c0 + lj) * D + c);
-              kd[lj * PD + c] = v.x;
-              kd[lj * PD + c + 1] = v.y;
-            }
-            __syncthreads();
-            double z[16];
+        const double *qr = qd + rt * PD;
+        // logits of this thread's row against the 16 candidates part + 4 k of chunk ch, and which
+        // of them count
+        auto logits = [&](int ch, double (&z)[16], uint32_t &on) {
+          const int c0 = ch * 64, nb = min(64, nc - c0);
+          __syncthreads();  // previous users of kd are done
+          for (int i = tid; i < 64 * (D / 2); i += 256) {
+            const int lj = i / (D / 2), c = (i % (D / 2)) * 2;
+            double2 v = make_double2(0.0, 0.0);
+            if (lj < nb && c0 + lj >= cmin) v = *reinterpret_cast<const double2 *>(kbase + (int64_t)(c0 + lj) * D + c);
+            kd[lj * PD + c] = v.x;
+            kd[lj * PD + c + 1] = v.y;
+          }
+          __syncthreads();
 #pragma unroll
-            for (int k = 0; k < 16; ++k) z[k] = 0.0;
-            const double *qr = qd + rt * PD;
+          for (int k = 0; k < 16; ++k) z[k] = 0.0;
 #pragma unroll 2
-            for (int c = 0; c < D; ++c) {
-              const double qv = qr[c];
+          for (int c = 0; c < D; ++c) {
+            const double qv = qr[c];
 #pragma unroll
-              for (int k = 0; k < 16; ++k) z[k] = fma(qv, kd[(part + 4 * k) * PD + c], z[k]);
+            for (int k = 0; k < 16; ++k) z[k] = fma(qv, kd[(part + 4 * k) * PD + c], z[k]);
+          }
+          on = 0u;
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            z[k] *= sh.scale_d;
+            const int c = c0 + part + 4 * k;
+            if (row_on && part + 4 * k < nb && c >= cmin && (sh.causal || c != b)) on |= 1u << k;
+          }
+        };
+        // running maximum and normaliser of the row over the chunks seen so far
+        auto fold = [&](const double (&z)[16], uint32_t on, double &mx, double &den) {
+          double cm = -INFINITY;
+#pragma unroll
+          for (int k = 0; k < 16; ++k)
+            if ((on >> k) & 1u) cm = fmax(cm, z[k]);
+          cm = fmax(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+          cm = fmax(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+          const double nm = fmax(mx, cm);
+          double es = 0.0;
+          if (nm > -INFINITY) {
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+              if ((on >> k) & 1u) es += exp(z[k] - nm);
+          }
+          es += __shfl_xor_sync(0xffffffffu, es, 1);
+          es += __shfl_xor_sync(0xffffffffu, es, 2);
+          den = (mx > -INFINITY ? den * exp(mx - nm) : 0.0) + es;
+          mx = nm;
+        };
+        // probabilities of chunk ch and their column sums, added to Sc
+        auto columns = [&](int ch, const double (&z)[16], uint32_t on, double mx, double den) {
+          const int c0 = ch * 64, nb = min(64, nc - c0);
+          __syncthreads();  // everyone has read kd: it becomes the probability tile
+#pragma unroll
+          for (int k = 0; k < 16; ++k)
+            kd[rt * 65 + part + 4 * k] = ((on >> k) & 1u) ? exp(z[k] - mx) / den : 0.0;
+          __syncthreads();
+          {  // column sums in a fixed order: four partial sums of 16 rows, then their tree
+            const int j = tid & 63, quarter = tid >> 6;
+            double a = 0.0;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) a += kd[(quarter * 16 + t) * 65 + j];
+            csum[tid] = a;
+          }
+          __syncthreads();
+          if (tid < nb) Sc[c0 + tid] += (csum[tid] + csum[64 + tid]) + (csum[128 + tid] + csum[192 + tid]);
+        };
+        double mx = -INFINITY, den = 0.0;
+        if (ch_hi - ch_lo <= NZ) {
+          // the logits of all (one or two) chunks stay in registers
+          double za[16], zb[NZ > 1 ? 16 : 1];
+          uint32_t ona = 0u, onb = 0u;
+          const bool two = NZ > 1 && ch_hi - ch_lo == 2;
+          logits(ch_lo, za, ona);
+          fold(za, ona, mx, den);
+          if constexpr (NZ > 1) {
+            if (two) {
+              logits(ch_lo + 1, zb, onb);
+              fold(zb, onb, mx, den);
             }
-            uint32_t on = 0u;
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-              z[k] *= sh.scale_d;
-              const int c = c0 + part + 4 * k;
-              if (row_on && part + 4 * k < nb && c >= cmin && (sh.causal || c != b)) on |= 1u << k;
-            }
-            if (pass == 0) {
-              double cm = -INFINITY;
-#pragma unroll
-              for (int k = 0; k < 16; ++k)
-                if ((on >> k) & 1u) cm = fmax(cm, z[k]);
-              cm = fmax(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
-              cm = fmax(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
-              const double nm = fmax(mx, cm);
-              double es = 0.0;
-              if (nm > -INFINITY) {
-#pragma unroll
-                for (int k = 0; k < 16; ++k)
-                  if ((on >> k) & 1u) es += exp(z[k] - nm);
-              }
-              es += __shfl_xor_sync(0xffffffffu, es, 1);
-              es += __shfl_xor_sync(0xffffffffu, es, 2);
-              den = (mx > -INFINITY ? den * exp(mx - nm) : 0.0) + es;
-              mx = nm;
-            }
-            if (pass == npass - 1) {
-              __syncthreads();  // everyone has read kd: it becomes the probability tile
-#pragma unroll
-              for (int k = 0; k < 16; ++k)
-                kd[rt * 65 + part + 4 * k] = ((on >> k) & 1u) ? exp(z[k] - mx) / den : 0.0;
-              __syncthreads();
-              {  // column sums in a fixed order: four partial sums of 16 rows, then their tree
-                const int j = tid & 63, quarter = tid >> 6;
-                double a = 0.0;
-#pragma unroll
-                for (int t = 0; t < 16; ++t) a += kd[(quarter * 16 + t) * 65 + j];
-                csum[tid] = a;
-              }
-              __syncthreads();
-              if (tid < nb) Sc[c0 + tid] += (csum[tid] + csum[64 + tid]) + (csum[128 + tid] + csum[192 + tid]);
-            }
+          }
+          columns(ch_lo, za, ona, mx, den);
+          if constexpr (NZ > 1) {
+            if (two) columns(ch_lo + 1, zb, onb, mx, den);
+          }
+        } else {
+          // more: one pass for the maxima and normalisers, a second one for the probabilities
+          double z[16];
+          uint32_t on;
+          for (int ch = ch_lo; ch < ch_hi; ++ch) {
+            logits(ch, z, on);
+            fold(z, on, mx, den);
+          }
+          for (int ch = ch_lo; ch < ch_hi; ++ch) {
+            logits(ch, z, on);
+            columns(ch, z, on, mx, den);
           }
         }
       }
@@ -880,8 +911,9 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
         sh, g, q, w.mean32, w.norm, seq_lens, idx, w.list, w.count, sc_pitch);
   }
   const size_t esm = exact_smem_bytes(sh, g, D, &sc_len);
-  if (esm > 48 * 1024 && cudaFuncSetAttribute(score_exact_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)esm) != cudaSuccess)
+  auto exact = g.n > 64 ? score_exact_kernel<T, D, 2> : score_exact_kernel<T, D, 1>;
+  if (esm > 48 * 1024 &&
+      cudaFuncSetAttribute(exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)esm) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   {
     // double precision: every query block (exact_only) or the work list of the kernel above
@@ -902,7 +934,7 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, score_exact_kernel<T, D>, sh, g, q, (const double *)w.mean, seq_lens, idx,
+    if (cudaLaunchKernelEx(&cfg, exact, sh, g, q, (const double *)w.mean, seq_lens, idx,
                            (const int32_t *)(exact_only ? nullptr : w.list), (const int32_t *)w.count,
                            sc_len) != cudaSuccess)
       return BLOSSOM_ERR_CUDA;
