@@ -286,6 +286,16 @@ def main():
     ap.add_argument("--paper-options", action="store_true",
                     help="the paper's options together on the chosen shape: heads on 2 key/value heads, "
                          "compression blocks of 2 x block at stride block / 2, power-law mask (window 8, block 1)")
+    ap.add_argument("--per-query", action="store_true",
+                    help="one selection per query position (Eq. 13 as printed); CUDA-core attention kernels")
+    ap.add_argument("--learned-summary", action="store_true",
+                    help="softmax-pooled block summaries (Eq. 9) with seeded pooling logits")
+    ap.add_argument("--input-gate", action="store_true",
+                    help="input-dependent gate (Eq. 18, one linear layer); CUDA-core attention kernels")
+    ap.add_argument("--non-causal", action="store_true",
+                    help="no causal mask (bidirectional encoder); CUDA-core attention kernels")
+    ap.add_argument("--rope-theta", type=float, default=0.0,
+                    help="rotate q and k by position inside the library (0 = off)")
     ap.add_argument("--no-secondary", action="store_true",
                     help="skip the L = 1024 case that the default run times beside the headline")
     ap.add_argument("--batch", type=int, default=0,
@@ -318,6 +328,24 @@ def main():
     if args.cmp_block or args.cmp_stride:
         w.cmp_block, w.cmp_stride = args.cmp_block or w.block, args.cmp_stride or w.block
         w.name += f"+cmp(l{w.cmp_block},s{w.cmp_stride})"
+    import numpy as np
+    opt_rng = np.random.default_rng(1000 + w.seed)   # inputs of the options below, seeded like the rest
+    if args.per_query:
+        w.per_query = 1
+        w.name += "+per-query-selection"
+    if args.learned_summary:
+        w.phi_logits = opt_rng.standard_normal(w.cmp_block or w.block).astype(np.float32)
+        w.name += "+softmax-pooled-summary"
+    if args.input_gate:
+        w.gate_mode = 1
+        w.gate = (opt_rng.standard_normal((w.H, 2 * w.D + 1)) / np.sqrt(w.D)).astype(np.float32)
+        w.name += "+input-gate"
+    if args.non_causal:
+        w.causal = 0
+        w.name += "+non-causal"
+    if args.rope_theta > 0:
+        w.rope_theta = float(args.rope_theta)
+        w.name += f"+rope({args.rope_theta:g})"
     cfg_desc = {"workload": w.name, "batch": w.B, "heads": w.H, "kv_heads": w.kv_heads or w.H, "seq_len": w.L, "head_dim": w.D,
                 "block_size": w.block, "top_k": w.topk, "window": w.window, "short_term": args.short_term,
                 "mask_block": w.stis_block if w.stis_mode else None,

@@ -30,36 +30,52 @@ __device__ __forceinline__ double2 load_pair(const __nv_bfloat16 *p) {
   return make_double2((double)__bfloat162float(v.x), (double)__bfloat162float(v.y));
 }
 
-// One thread per (row, pair).  heads / strides describe the tensor ([B][heads][L][D]); dir = +1
-// rotates by the position's angle, -1 by its negative (the transpose).  src may equal dst.
+// One thread per (position t, pair i) and slice of the (batch, head) rows: the angle, its sine and
+// cosine are evaluated once and applied to that pair of every row of the slice, so the
+// double-precision transcendental work is shared by all rows that sit at the same position.  A
+// warp's 32 pairs are 32 consecutive pairs of one row: whole 128-byte (bf16) lines.  heads /
+// strides describe the tensor ([B][heads][L][D]); dir = +1 rotates by the position's angle, -1 by
+// its negative (the transpose).  src may equal dst.
 template <typename T>
 __global__ void __launch_bounds__(256) rope_kernel(int B, int heads, int L, int D, int64_t sb, int64_t sh,
                                                    int64_t sl, double theta, int dir, const T *__restrict__ src,
                                                    T *__restrict__ dst) {
   const int half = D / 2;
-  const int64_t total = (int64_t)B * heads * L * half;
-  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-    const int i = (int)(e % half);
-    const int64_t row = e / half;
-    const int t = (int)(row % L);
-    const int h = (int)((row / L) % heads), n = (int)(row / ((int64_t)L * heads));
-    const int64_t off = (int64_t)n * sb + (int64_t)h * sh + (int64_t)t * sl + 2 * i;
-    const double ang = (double)t * pow(theta, -2.0 * (double)i / (double)D) * (double)dir;
-    double sn, cs;
-    sincos(ang, &sn, &cs);
-    const double2 x = load_pair(src + off);
-    store_pair(dst + off, x.x * cs - x.y * sn, x.x * sn + x.y * cs);
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (int64_t)L * half) return;
+  const int i = (int)(e % half), t = (int)(e / half);
+  const double ang = (double)t * pow(theta, -2.0 * (double)i / (double)D) * (double)dir;
+  double sn, cs;
+  sincos(ang, &sn, &cs);
+  const int rows = B * heads;
+  const int64_t base = (int64_t)t * sl + 2 * i;
+  for (int r0 = (int)blockIdx.y * 4; r0 < rows; r0 += (int)gridDim.y * 4) {
+    double2 x[4];
+    int64_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {  // four rows in flight
+      const int r = r0 + j;
+      off[j] = base + (int64_t)(r / heads) * sb + (int64_t)(r % heads) * sh;
+      if (r < rows) x[j] = load_pair(src + off[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (r0 + j < rows) store_pair(dst + off[j], x[j].x * cs - x[j].y * sn, x[j].x * sn + x[j].y * cs);
   }
 }
 
 template <typename T>
 int launch_rope_t(int B, int heads, int L, int D, int64_t sb, int64_t sh, int64_t sl, double theta, int dir,
                   const T *src, T *dst, cudaStream_t st) {
-  const int64_t total = (int64_t)B * heads * L * (D / 2);
-  const unsigned grid = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+  const int64_t per_row = (int64_t)L * (D / 2);
+  const unsigned gx = (unsigned)((per_row + 255) / 256);
+  // enough slices of the rows to fill the GPU about eight CTAs deep, each of at least four rows
+  const int64_t want = (148 * 8 + gx - 1) / gx, most = ((int64_t)B * heads + 3) / 4;
+  int64_t gy = want < 1 ? 1 : (want > most ? most : want);
+  if (gy > 65535) gy = 65535;
   {
     LaunchScope ls(K_ROPE, st);
-    rope_kernel<T><<<grid, 256, 0, st>>>(B, heads, L, D, sb, sh, sl, theta, dir, src, dst);
+    rope_kernel<T><<<dim3(gx, (unsigned)gy), 256, 0, st>>>(B, heads, L, D, sb, sh, sl, theta, dir, src, dst);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
