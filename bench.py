@@ -291,7 +291,7 @@ def main():
     ap.add_argument("--learned-summary", action="store_true",
                     help="softmax-pooled block summaries (Eq. 9) with seeded pooling logits")
     ap.add_argument("--input-gate", action="store_true",
-                    help="input-dependent gate (Eq. 18, one linear layer); CUDA-core attention kernels")
+                    help="input-dependent gate (Eq. 18, one linear layer)")
     ap.add_argument("--non-causal", action="store_true",
                     help="no causal mask (bidirectional encoder); CUDA-core attention kernels")
     ap.add_argument("--rope-theta", type=float, default=0.0,
@@ -403,7 +403,7 @@ def main():
         sampler.start()
         time.sleep(0.3)
         launches0 = binding.blossom_launch_count()
-        cap = 16 * steps
+        cap = 32 * steps
         binding.blossom_profile_start(cap)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         step_events = []

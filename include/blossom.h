@@ -103,8 +103,10 @@ typedef struct {
                         * 1: the input-dependent gate of Eq. 18 with a one-layer F_o: gate_logits
                         * (and dgate) are float [H][2 D + 1] = (w_lt[D], w_st[D], b) per head and
                         * alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row,
-                        * broadcast over the head's channels in Eq. 19; runs on the CUDA-core
-                        * kernels                                                                 */
+                        * broadcast over the head's channels in Eq. 19.  The out_lt, out_st that
+                        * enter F_o are the rows as stored (bf16 roundings for bf16 tensors on
+                        * the tensor-core kernels, which then run the backward once per branch
+                        * and need about seven q-sized scratch tensors in the workspace)          */
   float rope_theta;    /* 0 = q and k are used as given.  > 0 (>= 1, e.g. 10000): rotary position
                         * embedding inside the library: q and k are rotated by position before the
                         * selection and both branches (pairs (x[2i], x[2i+1]), angle

@@ -134,7 +134,7 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     top_k]) instead of one per query block; runs on the CUDA-core kernels.
     input_dependent_gate: Eq. 18's gate with a one-layer F_o: gate_logits is [H, 2 D + 1] = (w_lt,
     w_st, b) per head and alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row
-    (differentiable in those parameters); runs on the CUDA-core kernels.
+    (differentiable in those parameters).
     causal: False drops the causal mask (bidirectional encoders): a query block scores every other
     live block, a query sees all valid keys of its selected blocks, Eq. 15 is symmetric; runs on the
     CUDA-core kernels.

@@ -93,6 +93,20 @@ Workspace carve_workspace(const Shape &s, void *base) {
   }
   w.gate_ac = reinterpret_cast<float *>(take(s.gate_mode ? 2 * units * s.L * sizeof(float) : 0));
   w.dgate_part = reinterpret_cast<double *>(take(s.gate_mode ? units * s.M * (2 * s.D + 1) * sizeof(double) : 0));
+  {
+    // input-dependent gate on the tensor-core kernels (bf16): scratch tensors of the two passes
+    const bool on = s.gate_mode && s.esz == 2;
+    const size_t qspan = (size_t)((s.B - 1) * s.sb + (s.H - 1) * s.sh + (int64_t)(s.L - 1) * s.sl + s.D);
+    const size_t kspan = (size_t)((s.B - 1) * s.ksb + (s.Hkv - 1) * s.ksh + (int64_t)(s.L - 1) * s.ksl + s.D);
+    w.gate_glt = take(on ? qspan * 2 : 0);
+    w.gate_gst = take(on ? qspan * 2 : 0);
+    w.gate_dq = take(on ? qspan * 2 : 0);
+    w.gate_olt = take(on ? qspan * 2 : 0);
+    w.gate_ost = take(on ? qspan * 2 : 0);
+    w.gate_dk = take(on ? kspan * 2 : 0);
+    w.gate_dv = take(on ? kspan * 2 : 0);
+    w.qstats2 = reinterpret_cast<float4 *>(take(on ? units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4) : 0));
+  }
   w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
   w.bytes = off;
@@ -265,9 +279,13 @@ int blossom_attn_fwd(const blossom_params *params, const void *q, const void *k,
     rc = launch_select(s, params->dtype, q, k, seq_lens, block_idx, ws, st);
     if (rc) return rc;
   }
-  if (!force_simt() && tc::fwd_tc_supported(s, params->dtype))
+  if (!force_simt() && tc::fwd_tc_supported(s, params->dtype)) {
+    if (s.gate_mode)
+      return tc::launch_fwd_tc_gate(s, q, k, v, gate_logits, seq_lens, block_idx, out, out_lt, out_st, lse,
+                                    ws, st);
     return tc::launch_fwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out, out_lt, out_st, lse, ws,
                              st);
+  }
   return launch_fwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out, out_lt,
                          out_st, lse, ws, st);
 }
@@ -296,9 +314,14 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
   rc = rotate_inputs(s, params->dtype, ws, &q, &k, st);
   if (rc) return rc;
   if (!force_simt() && tc::fwd_tc_supported(s, params->dtype)) {
-    rc = tc::launch_bwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out_lt, out_st, lse, dout, dq,
-                           dk, dv, ws, st);
-    if (!rc) rc = launch_gate_grad(s, gate_logits, ws, dgate, st);
+    if (s.gate_mode) {
+      rc = tc::launch_bwd_tc_gate(s, q, k, v, gate_logits, seq_lens, block_idx, out_lt, out_st, lse, dout,
+                                  dq, dk, dv, dgate, ws, st);
+    } else {
+      rc = tc::launch_bwd_tc(s, q, k, v, gate_logits, seq_lens, block_idx, out_lt, out_st, lse, dout, dq,
+                             dk, dv, ws, st);
+      if (!rc) rc = launch_gate_grad(s, gate_logits, ws, dgate, st);
+    }
   } else {
     rc = launch_bwd_simt(s, params->dtype, q, k, v, gate_logits, seq_lens, block_idx, out_lt,
                          out_st, lse, dout, dq, dk, dv, dgate, ws, st);

@@ -639,6 +639,14 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
 
 }  // namespace
 
+int launch_gate_param_grad(const Shape &s, const Workspace &ws, float *dgate, cudaStream_t st) {
+  {
+    LaunchScope ls(K_GATE_GRAD, st);
+    gate_param_grad_kernel<<<s.H, 256, 0, st>>>(s, ws.dgate_part, dgate);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+}
+
 int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, float *dgate,
                      cudaStream_t st) {
   {

@@ -780,7 +780,7 @@ template <int D>
 int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                     const int32_t *seq_lens, const int32_t *idx, const void *out_lt,
                     const void *out_st, const float *lse, const void *dout, void *dq, void *dk,
-                    void *dv, const Workspace &ws, cudaStream_t st) {
+                    void *dv, const Workspace &ws, cudaStream_t st, int branches, const float4 *records) {
   typedef __nv_bfloat16 bf;
   using C = Cfg<D>;
   CUtensorMap q128, k64, v64, g128, q64, k128, v128, g64, tdq, tdk, tdv;
@@ -799,8 +799,9 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
-  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, ws.kmeta, st)) return rc;
-  {
+  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, ws.kmeta, st, branches)) return rc;
+  const float4 *rec = records ? records : ws.qstats;
+  if (!records) {
     LaunchScope ls(K_BWD_PREP, st);
     const int Lpad = nT * 64, rpb = 256 / (D / 8);
     const unsigned gp = (unsigned)(s.B * s.H) * (unsigned)((Lpad + rpb - 1) / rpb);
@@ -810,14 +811,14 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   {
     LaunchScope ls(K_BWD_DQ_TC, st);
     bwd_dq_tc_kernel<D><<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
-                                                           tdq, ws.qstats, ws.dalpha,
+                                                           tdq, rec, ws.dalpha,
                                                            ws.status_bwd, nT);
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
     const unsigned grid_k = (unsigned)nST * (unsigned)(s.B * s.Hkv);
     bwd_dkdv_tc_kernel<D><<<grid_k, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
-                                                             ws.qstats, tdk, tdv, ws.status_bwd, nT);
+                                                             rec, tdk, tdv, ws.status_bwd, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
@@ -825,11 +826,11 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
 template int launch_bwd_tc_t<32>(const Shape &, const void *, const void *, const void *, const float *,
                                  const int32_t *, const int32_t *, const void *, const void *,
                                  const float *, const void *, void *, void *, void *, const Workspace &,
-                                 cudaStream_t);
+                                 cudaStream_t, int, const float4 *);
 template int launch_bwd_tc_t<64>(const Shape &, const void *, const void *, const void *, const float *,
                                  const int32_t *, const int32_t *, const void *, const void *,
                                  const float *, const void *, void *, void *, void *, const Workspace &,
-                                 cudaStream_t);
+                                 cudaStream_t, int, const float4 *);
 
 }  // namespace tc
 }  // namespace blossom

@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                                                                   const int32_t *__restrict__ idx,
                                                                   uint8_t *__restrict__ qmeta,
                                                                   uint8_t *__restrict__ kmeta, int nT,
-                                                                  int n_query_ctas, int n_images) {
+                                                                  int n_query_ctas, int n_images, int branches) {
   extern __shared__ __align__(16) uint8_t meta_all[];
   const MetaLayout ml = meta_layout(nT);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         if (jt <= jt_max && row_last >= pad0 && jt * 64 + 63 >= pad0) {
           for (int g = 0; g < G; ++g) f |= selb[g * nT + jt] ? 1 : 0;
           if (st_ranges_touch(s, row0, row_last, jt * 64, jt * 64 + 63)) f |= 2;
+          f &= branches;
         }
         const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
         if (f) {
@@ -295,6 +296,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       if (qt <= qt_max && key_last >= pad0) {
         for (int g = 0; g < G; ++g) f |= selb[g * nT + qt] ? 1 : 0;
         if (st_ranges_touch(s, qt * 64, min(qt * 64 + 63, s.L - 1), key0, key_last)) f |= 2;
+        f &= branches;
       }
       const unsigned bal = __ballot_sync(0xffffffffu, f != 0);
       if (f) {
@@ -344,7 +346,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
 }  // namespace
 
 int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
-                   uint8_t *kmeta, cudaStream_t st) {
+                   uint8_t *kmeta, cudaStream_t st, int branches) {
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const int nq = nST * s.B * s.H, n_images = kmeta ? nq + nST * s.B * s.Hkv : nq;
   const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT) + ((3 * nT + 15) / 16) * 16);
@@ -354,7 +356,7 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
   {
     LaunchScope ls(K_TC_META, st);
     tc_meta_kernel<<<(unsigned)((n_images + kMetaWarps - 1) / kMetaWarps), kMetaWarps * 32, smem, st>>>(
-        s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images);
+        s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images, branches);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

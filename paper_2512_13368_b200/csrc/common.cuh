@@ -48,6 +48,12 @@ struct Workspace {
   void *q_rot, *k_rot;  // rotated copies of q and k (rope_theta > 0), laid out with the originals' strides
   float *gate_ac;    // [2][B][H][L]  input-dependent gate: alpha_t and c_t of every row (backward)
   double *dgate_part;// [B][H][M][2 D + 1]  per query block partial of the gradient of F_o's parameters
+  // input-dependent gate on the tensor-core kernels (bf16 only): the two branches' upstream
+  // tensors, the second pass's gradients (added to the first pass's afterwards), its records, and
+  // the branch outputs of a forward call that does not return them; q-shaped ones laid out with
+  // q's strides, k-shaped ones with k's
+  void *gate_glt, *gate_gst, *gate_dq, *gate_dk, *gate_dv, *gate_olt, *gate_ost;
+  float4 *qstats2;
   uint8_t *qmeta;    // per query-major CTA of the tensor-core kernels: tile lists (tc_meta_kernel)
   uint8_t *kmeta;    // per key-major CTA (dK/dV kernel): tile lists
   size_t bytes;
@@ -145,16 +151,30 @@ int launch_select_static(const Shape &s, int dtype, const void *q, const void *k
 size_t select_static_capacity_bytes();
 int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, float *dgate,
                      cudaStream_t st);
+// input-dependent gate: fixed-order reduction of ws.dgate_part into dgate [H][2 D + 1]
+int launch_gate_param_grad(const Shape &s, const Workspace &ws, float *dgate, cudaStream_t st);
 int launch_rope(const Shape &s, int dtype, bool kv, int dir, const void *src, void *dst, cudaStream_t st);
 
 namespace tc {
 int launch_wait_selftest(int32_t *status, cudaStream_t st);
 bool fwd_tc_supported(const Shape &s, int dtype);
 size_t tc_meta_bytes(const Shape &s);  // bytes of one of the two tile-list areas of the workspace
+// branches: bit 0 long-term, bit 1 short-term branch: the tile lists hold only the tiles those
+// branches need.  records: null = computed from out_lt, out_st, lse, dout and the per-head gate by
+// the pre-pass; otherwise the caller's per-row records (layout of Workspace::qstats) are used as
+// they are.
 int launch_bwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                   const int32_t *seq_lens, const int32_t *idx, const void *out_lt, const void *out_st,
                   const float *lse, const void *dout, void *dq, void *dk, void *dv,
-                  const Workspace &ws, cudaStream_t st);
+                  const Workspace &ws, cudaStream_t st, int branches = 3, const float4 *records = nullptr);
+// the same two calls with the input-dependent gate (gate = F_o's parameters [H][2 D + 1])
+int launch_fwd_tc_gate(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                       const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt, void *out_st,
+                       float *lse, const Workspace &ws, cudaStream_t st);
+int launch_bwd_tc_gate(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
+                       const int32_t *seq_lens, const int32_t *idx, const void *out_lt, const void *out_st,
+                       const float *lse, const void *dout, void *dq, void *dk, void *dv, float *dgate,
+                       const Workspace &ws, cudaStream_t st);
 int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                   const int32_t *seq_lens, const int32_t *idx, void *out, void *out_lt, void *out_st,
                   float *lse, const Workspace &ws, cudaStream_t st);

@@ -467,8 +467,9 @@ int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_
 
 // Builds the bookkeeping of every query-major CTA (forward, dQ) into qmeta and, if kmeta is not
 // null, of every key-major CTA (dK/dV) into kmeta: meta_bytes(nT) bytes per CTA, CTA-major.
+// branches: bit 0 long-term, bit 1 short-term: tiles that only the other branch needs are left out.
 int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
-                   uint8_t *kmeta, cudaStream_t st);
+                   uint8_t *kmeta, cudaStream_t st, int branches = 3);
 
 // per-file launchers behind launch_fwd_tc / launch_bwd_tc
 template <int D>
@@ -479,7 +480,7 @@ template <int D>
 int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                     const int32_t *seq_lens, const int32_t *idx, const void *out_lt,
                     const void *out_st, const float *lse, const void *dout, void *dq, void *dk,
-                    void *dv, const Workspace &ws, cudaStream_t st);
+                    void *dv, const Workspace &ws, cudaStream_t st, int branches, const float4 *records);
 
 }  // namespace tc
 }  // namespace blossom

@@ -75,8 +75,8 @@ int launch_wait_selftest(int32_t *status, cudaStream_t st) {
 
 bool fwd_tc_supported(const Shape &s, int dtype) {
   // (a selection per query position gives every row its own key blocks: CUDA-core kernels)
-  // (and so does the input-dependent gate, whose backward adds rank-one terms to both branches)
-  return s.causal && !s.pq && !s.gate_mode && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  // (the input-dependent gate goes through launch_fwd_tc_gate / launch_bwd_tc_gate)
+  return s.causal && !s.pq && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 
@@ -95,10 +95,12 @@ int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, c
 int launch_bwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
                   const int32_t *seq_lens, const int32_t *idx, const void *out_lt, const void *out_st,
                   const float *lse, const void *dout, void *dq, void *dk, void *dv,
-                  const Workspace &ws, cudaStream_t st) {
+                  const Workspace &ws, cudaStream_t st, int branches, const float4 *records) {
   if (s.D == 32)
-    return launch_bwd_tc_t<32>(s, q, k, v, gate, seq_lens, idx, out_lt, out_st, lse, dout, dq, dk, dv, ws, st);
-  return launch_bwd_tc_t<64>(s, q, k, v, gate, seq_lens, idx, out_lt, out_st, lse, dout, dq, dk, dv, ws, st);
+    return launch_bwd_tc_t<32>(s, q, k, v, gate, seq_lens, idx, out_lt, out_st, lse, dout, dq, dk, dv, ws, st,
+                               branches, records);
+  return launch_bwd_tc_t<64>(s, q, k, v, gate, seq_lens, idx, out_lt, out_st, lse, dout, dq, dk, dv, ws, st,
+                             branches, records);
 }
 
 }  // namespace tc

@@ -149,6 +149,43 @@ def test_overlapping_compression_blocks(runner, dtype, L, D, block, topk, l, s, 
 
 
 @pytest.mark.gpu
+def test_input_dependent_gate_runs_on_the_tensor_core_kernels(runner):
+    """bf16 shapes the tensor-core kernels take keep them with gate_mode 1 (one forward kernel plus
+    a row-wise mix; one backward pass per branch plus an addition): the launch record shows those
+    kernels, the results agree with the oracle and with the CUDA-core path, and a forward call
+    that returns no branch outputs gives the same output bits."""
+    from paper_2512_13368_b200 import binding
+    w = workloads.make("gate-tc", "bf16", 3, 4, 1000, 64, 32, 6, 70, seed=71, kv_heads=2, lengths=(300, 1000))
+    w.gate_mode = 1
+    w.gate = (0.3 * np.random.default_rng(6).standard_normal((w.H, 2 * w.D + 1))).astype(np.float32)
+    binding.blossom_profile_start(64)
+    _, tc = run(runner, w)
+    names = {name for name, _ in binding.blossom_profile_stop(64)}
+    assert {"fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc"} <= names and not any("simt" in x for x in names), names
+    print(check_forward_backward(w, tc))
+    q, _ = run(runner, w, training=False, backward=False)
+    assert np.array_equal(q.results()["out"], tc["out"])
+    binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, 1)
+    try:
+        _, simt = run(runner, w)
+    finally:
+        binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, -1)
+    for key in ("out", "out_lt", "out_st", "lse", "dq", "dk", "dv", "dgate"):
+        ref = np.abs(simt[key]).max()
+        err = np.abs(tc[key] - simt[key]).max()
+        assert err <= 2e-2 * max(ref, 1e-3), (key, err, ref)
+
+
+def test_config4_full_size_input_dependent_gate(runner):
+    """The headline shape with Eq. 18's gate, as the benchmark's --input-gate option times it."""
+    w = workloads.config4()
+    w.gate_mode = 1
+    w.gate = (np.random.default_rng(1004).standard_normal((w.H, 2 * w.D + 1)) / np.sqrt(w.D)).astype(np.float32)
+    errs, res = _whole_batch(runner, w)
+    print(errs)
+    assert res["dgate"].shape == (w.H, 2 * w.D + 1)
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens,power_law", [
     (64, 32, 4, 2, 8, 2, 16, None, False),
