@@ -287,7 +287,7 @@ def main():
                     help="the paper's options together on the chosen shape: heads on 2 key/value heads, "
                          "compression blocks of 2 x block at stride block / 2, power-law mask (window 8, block 1)")
     ap.add_argument("--per-query", action="store_true",
-                    help="one selection per query position (Eq. 13 as printed); CUDA-core attention kernels")
+                    help="one selection per query position (Eq. 13 as printed)")
     ap.add_argument("--learned-summary", action="store_true",
                     help="softmax-pooled block summaries (Eq. 9) with seeded pooling logits")
     ap.add_argument("--input-gate", action="store_true",

@@ -131,7 +131,7 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     cmp_block / cmp_stride: length and stride of overlapping compression blocks for the selection
     (Eq. 8, 11); 0 = the selection blocks themselves.
     select_per_query: one selection per query position (Eq. 13 as printed; indices [B, Hkv, L,
-    top_k]) instead of one per query block; runs on the CUDA-core kernels.
+    top_k]) instead of one per query block.
     input_dependent_gate: Eq. 18's gate with a one-layer F_o: gate_logits is [H, 2 D + 1] = (w_lt,
     w_st, b) per head and alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row
     (differentiable in those parameters).

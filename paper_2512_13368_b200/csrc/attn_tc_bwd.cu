@@ -193,8 +193,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   uint8_t *g_tile = q_tile + C::kBigBytes;
   uint8_t *kv_tiles = g_tile + C::kBigBytes;
   uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;  // image built by tc_meta_kernel
-  const MetaLayout ml = meta_layout(nT);
+  const MetaLayout ml = meta_layout(nT, s.pq);
   const uint8_t *selb = meta;
+  const uint8_t *rowb = meta + ml.rows;  // (selection per query position) [128 rows][nT]
   const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
   const uint8_t *lflags = meta + ml.flags;
   const uint8_t *jcls = meta + ml.jcls;  // [tile][half tile][compute warp]
@@ -370,7 +371,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         uint64_t maskL = 0ull, maskS = 0ull;
         if (row_valid) {
           const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
-          if (f & 1) maskL = mc & expand_block_bits(selb[g * nT + jt], s.Bk);
+          if (f & 1) maskL = mc & expand_block_bits(s.pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk);
           if (f & 2) maskS = mc & st_key_cols(s, t, p0);
         }
         hL = (uint32_t)(maskL >> (32 * (x & 1) + 16 * half)) & 0xffffu;
@@ -538,7 +539,8 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   uint8_t *v_tile = k_tile + C::kBigBytes;
   uint8_t *qg_tiles = v_tile + C::kBigBytes;  // [stage][Q, dO, row records]
   uint8_t *meta = qg_tiles + STAGES * kStageBytes;  // image built by tc_meta_kernel
-  const MetaLayout ml = meta_layout(nT);
+  const MetaLayout ml = meta_layout(nT, s.pq);
+  const uint64_t *inv64 = reinterpret_cast<const uint64_t *>(meta + ml.rows);  // (selection per query position) [8][nT]
   const uint8_t *invb = meta;                           // [8][nT] bytes: per key block, per query tile
   const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
   const uint8_t *lflags = meta + ml.flags;
@@ -686,7 +688,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       if (cls2[0] == 8 || cls2[8] == 8) {  // a mixed half tile: per-lane column masks
         if (row_valid) {
           const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
-          if (f & 1) maskL = mc & expand_block_bits(invb[g * nT + qt], s.Bk);
+          if (f & 1) maskL = mc & (s.pq ? inv64[g * nT + qt] : expand_block_bits(invb[g * nT + qt], s.Bk));
           if (f & 2) maskS = mc & st_query_cols(s, p, t0);
         }
       }
@@ -793,9 +795,9 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
-  const size_t smem_dq = 1024 + 2 * C::kBigBytes + kDqStages * 2 * C::kSmallBytes + meta_bytes(nT);
+  const size_t smem_dq = 1024 + 2 * C::kBigBytes + kDqStages * 2 * C::kSmallBytes + meta_bytes(nT, s.pq);
   const size_t smem_kv =
-      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT);
+      1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT, s.pq);
   if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;

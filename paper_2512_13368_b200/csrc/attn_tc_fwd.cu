@@ -151,8 +151,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   uint8_t *kv_tiles = q_tile + C::kBigBytes;                  // [stage][K, V]
   uint8_t *sl = kv_tiles + STAGES * 2 * C::kSmallBytes;       // the long-term rows, staged when their phase ends
   uint8_t *meta = sl + C::kBigBytes;                          // image built by tc_meta_kernel
-  const MetaLayout ml = meta_layout(nT);
+  const MetaLayout ml = meta_layout(nT, s.pq);
   const uint8_t *selb = meta;
+  const uint8_t *rowb = meta + ml.rows;  // (selection per query position) [128 rows][nT]
   const uint16_t *items = reinterpret_cast<const uint16_t *>(meta + ml.items);  // [2 nT]
   const uint8_t *icls = meta + ml.icls;                                         // [2 nT][4]
   const int *counts = reinterpret_cast<const int *>(meta + ml.counts);
@@ -371,7 +372,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       if (cls == 2) {
         if (row_ok) {
           uint64_t mask = cols_le(t - p0) & cols_ge(pad0 - p0);
-          mask &= isL ? expand_block_bits(selb[g * nT + jt], s.Bk) : st_key_cols(s, t, p0);
+          mask &= isL ? expand_block_bits(s.pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk) : st_key_cols(s, t, p0);
           hm = (uint32_t)(mask >> (32 * grp));
         }
         doB = __any_sync(0xffffffffu, hm != 0u);
@@ -466,7 +467,7 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
       make_tensor_map(&tos, training ? out_st : out, s, 128))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
-  const size_t smem = 1024 + 2 * C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT);
+  const size_t smem = 1024 + 2 * C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT, s.pq);
   if (cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return BLOSSOM_ERR_CUDA;

@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                                                                   uint8_t *__restrict__ kmeta, int nT,
                                                                   int n_query_ctas, int n_images, int branches) {
   extern __shared__ __align__(16) uint8_t meta_all[];
-  const MetaLayout ml = meta_layout(nT);
+  const MetaLayout ml = meta_layout(nT, s.pq);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int image = (int)blockIdx.x * kMetaWarps + warp;
   if (image >= n_images) return;
@@ -70,6 +70,22 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   if (!key_major) {
     const int st = nST - 1 - cta % nST;  // the attention kernels take long rows first
     const int row0 = st * 128, row_last = min(s.L - 1, row0 + 127);
+    if (s.pq) {
+      // a selection per query position: every row's own bytes, and their union per query block
+      // (which is what the tile list and the item order below are built from)
+      uint32_t *roww = reinterpret_cast<uint32_t *>(meta + ml.rows);
+      for (int i = lane; i < 128 * s.topk; i += 32) {
+        const int r = i / s.topk, slot = i % s.topk, t = row0 + r;
+        if (t < s.L) {
+          const int blk = idx[((int64_t)uk * s.L + t) * s.topk + slot];
+          if (blk >= 0 && blk <= (t >> bk_shift)) {
+            const int a = (r >> bk_shift) * nT + blk / nb, b2 = r * nT + blk / nb;
+            atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
+            atomicOr(&roww[b2 >> 2], (1u << (blk % nb)) << ((b2 & 3) * 8));
+          }
+        }
+      }
+    } else {
     for (int i = lane; i < G * s.topk; i += 32) {  // the selections of the CTA's query blocks
       const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
       if (qb < s.M) {
@@ -79,6 +95,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
           atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
         }
       }
+    }
     }
     __syncwarp();
     int nv = 0;
@@ -171,7 +188,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
           if (!uni) cls = 2;
           else {
             const uint32_t bits = selb[((w * 32) / s.Bk) * nT + jt];
-            cls = bits == 0u ? 0 : ((inner && bits == allbits) ? 1 : 2);
+            cls = bits == 0u ? 0 : ((!s.pq && inner && bits == allbits) ? 1 : 2);  // (per position: the rows differ)
           }
         } else if (st_ranges_touch(s, t_lo, t_lo + 31, p0, p0 + 63)) {
           cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;  // 1: inside every row's window
@@ -257,7 +274,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
           any_sel |= sel;
           all_sel &= sel;
         }
-        if (any_sel) cL = (all_sel && past) ? 1 : 2;
+        if (any_sel) cL = (all_sel && past && !s.pq) ? 1 : 2;
       }
       if ((f & 2) && reach && st_ranges_touch(s, t_lo, t_hi, k_lo, k_hi))
         cS = (past && k_lo >= t_hi - s.window + 1) ? 1 : 2;  // 1: inside every row's window
@@ -266,7 +283,30 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   } else {
     const int kt = cta % nST;  // the dK/dV kernel takes early keys first
     const int key0 = kt * 128, key_last = min(s.L - 1, key0 + 127);
-    {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
+    if (s.pq) {
+      // a selection per query position: which positions selected each of this CTA's key blocks
+      // (one bit per position), and per 64-query tile which query blocks hold such a position
+      uint32_t *invw = reinterpret_cast<uint32_t *>(meta + ml.rows);
+      const int qb0 = kt * G, total = (s.L - key0) * s.topk;
+      const int32_t *rows = idx + ((int64_t)uk * s.L + key0) * s.topk;
+      for (int base = 0; base < total; base += 256) {
+        int blk[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = base + e * 32 + lane;
+          blk[e] = i < total ? rows[i] : -1;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = base + e * 32 + lane, t = key0 + i / s.topk;
+          if (blk[e] >= qb0 && blk[e] < qb0 + G && blk[e] <= (t >> bk_shift)) {
+            const int a = (blk[e] - qb0) * nT + (t >> 6);
+            atomicOr(&selw[a >> 2], (1u << ((t >> bk_shift) % nb)) << ((a & 3) * 8));
+            atomicOr(&invw[2 * a + ((t & 63) >> 5)], 1u << (t & 31));
+          }
+        }
+      }
+    } else {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
       // (the index rows of query blocks qb0 .. M-1 are contiguous; eight loads in flight per lane)
       const int qb0 = kt * G, total = (s.M - qb0) * s.topk;
       const int32_t *rows = idx + ((int64_t)uk * s.M + qb0) * s.topk;
@@ -330,7 +370,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
             all_sel &= sel;
           }
         }
-        if (any_sel) cL = (all_sel && past) ? 1 : 2;
+        if (any_sel) cL = (all_sel && past && !s.pq) ? 1 : 2;
       }
       if ((f & 2) && reach && st_ranges_touch(s, t_lo, min(t_hi, s.L - 1), p_lo, min(p_hi, s.L - 1)))
         cS = (past && p_lo >= t_hi - s.window + 1) ? 1 : 2;  // 1: inside every query's window
@@ -349,7 +389,7 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
                    uint8_t *kmeta, cudaStream_t st, int branches) {
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const int nq = nST * s.B * s.H, n_images = kmeta ? nq + nST * s.B * s.Hkv : nq;
-  const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT) + ((3 * nT + 15) / 16) * 16);
+  const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT, s.pq) + ((3 * nT + 15) / 16) * 16);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(tc_meta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;

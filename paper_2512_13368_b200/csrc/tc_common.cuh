@@ -412,10 +412,15 @@ struct Cfg {
 // items with 4 class bytes each, (dQ kernel) 16 class bytes per listed tile, and the counts {tiles
 // on the list, long-term items, short-term items}.  Offsets in bytes; every part starts on a
 // 16-byte boundary where a copy needs it.
+// With a selection per query position (pq) an area of 128 nT bytes follows: in a query-major
+// image [128 rows][nT] bytes, bit c of byte (r, jt): row r of the CTA selected key block
+// jt * (64 / Bk) + c (the [8][nT] bytes at the start are then the union over a query block's
+// rows); in a key-major image [8][nT] 64-bit words, bit i of word (g, qt): query position
+// 64 qt + i selected key block g of the CTA.
 struct MetaLayout {
-  int list, flags, items, icls, jcls, counts, bytes;
+  int list, flags, items, icls, jcls, counts, rows, bytes;
 };
-__host__ __device__ inline MetaLayout meta_layout(int nT) {
+__host__ __device__ inline MetaLayout meta_layout(int nT, int pq = 0) {
   MetaLayout m;
   m.list = ((8 * nT + 15) / 16) * 16;
   m.flags = m.list + 2 * nT;
@@ -423,10 +428,11 @@ __host__ __device__ inline MetaLayout meta_layout(int nT) {
   m.icls = m.items + 4 * nT;
   m.jcls = ((m.icls + 8 * nT + 15) / 16) * 16;
   m.counts = m.jcls + 16 * nT;
-  m.bytes = m.counts + 16;
+  m.rows = m.counts + 16;
+  m.bytes = m.rows + (pq ? 128 * nT : 0);
   return m;
 }
-__host__ __device__ inline int meta_bytes(int nT) { return meta_layout(nT).bytes; }
+__host__ __device__ inline int meta_bytes(int nT, int pq = 0) { return meta_layout(nT, pq).bytes; }
 
 // one arrival per warp, after all its lanes are done
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {

@@ -74,15 +74,16 @@ int launch_wait_selftest(int32_t *status, cudaStream_t st) {
 }
 
 bool fwd_tc_supported(const Shape &s, int dtype) {
-  // (a selection per query position gives every row its own key blocks: CUDA-core kernels)
+  // (a selection per query position adds 128 bytes per tile to a CTA's bookkeeping in shared
+  // memory: up to 64 tiles, i.e. L <= 4096; longer sequences take the CUDA-core kernels)
   // (the input-dependent gate goes through launch_fwd_tc_gate / launch_bwd_tc_gate)
-  return s.causal && !s.pq && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  return s.causal && (!s.pq || (s.L + 63) / 64 <= 64) && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 
 size_t tc_meta_bytes(const Shape &s) {
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
-  return (size_t)s.B * s.H * nST * (size_t)meta_bytes(nT);
+  return (size_t)s.B * s.H * nST * (size_t)meta_bytes(nT, s.pq);
 }
 
 int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,

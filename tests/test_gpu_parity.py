@@ -601,6 +601,44 @@ def test_selection_per_query_position(runner, dtype, L, D, H, Hkv, block, topk, 
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.parametrize("block,power_law", [(16, False), (32, True), (64, False)])
+def test_selection_per_query_position_runs_on_the_tensor_core_kernels(runner, block, power_law):
+    """bf16 shapes of up to 4096 positions keep the tensor-core kernels with select_mode 1 (their
+    tile lists are the union of a query block's rows, every row masks with its own selection):
+    the launch record shows those kernels, and the results agree with the oracle and with the
+    CUDA-core path."""
+    from paper_2512_13368_b200 import binding
+    w = workloads.make("per-query-tc", "bf16", 3, 4, 1000, 64, block, 5, 70, seed=79, kv_heads=2, lengths=(300, 1000),
+                       stis_mode=1 if power_law else 0, stis_block=2 if power_law else 1)
+    w.per_query = 1
+    binding.blossom_profile_start(64)
+    _, tc = run(runner, w)
+    names = {name for name, _ in binding.blossom_profile_stop(64)}
+    assert {"fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc"} <= names and not any("simt" in x for x in names), names
+    assert tc["idx"].shape == (w.B, 2, w.L, w.topk)
+    print(check_forward_backward(w, tc))
+    binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, 1)
+    try:
+        _, simt = run(runner, w)
+    finally:
+        binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, -1)
+    assert np.array_equal(tc["idx"], simt["idx"])
+    for key in ("out", "out_lt", "out_st", "lse", "dq", "dk", "dv", "dgate"):
+        ref = np.abs(simt[key]).max()
+        err = np.abs(tc[key] - simt[key]).max()
+        assert err <= 2e-2 * max(ref, 1e-3), (key, err, ref)
+
+
+def test_config4_full_size_selection_per_query_position(runner):
+    """The headline shape with a selection per query position, as the benchmark's --per-query
+    option times it."""
+    w = workloads.config4()
+    w.per_query = 1
+    errs, res = _whole_batch(runner, w)
+    print(errs)
+    assert res["idx"].shape == (w.B, w.H, w.L, w.topk)
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("L,D,H,Hkv,block,topk,cmp,lens,per_query", [
     (200, 32, 2, 2, 16, 4, None, [200, 5, 77], False),
