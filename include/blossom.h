@@ -77,8 +77,9 @@ typedef struct {
   int32_t select_mode; /* 0 = one selection per query block, from the probabilities summed over the
                         * block's queries (tensor-core kernels for bf16); 1 = one selection per
                         * query position (Eq. 13 as printed): block_idx is then
-                        * [B][kv_heads][L][top_k], a row per position, and the attention runs on
-                        * the CUDA-core kernels; not combined with cmp_block / cmp_stride          */
+                        * [B][kv_heads][L][top_k], a row per position (tensor-core kernels for
+                        * bf16 up to 4096 positions, CUDA-core kernels beyond); not combined with
+                        * cmp_block / cmp_stride                                                   */
   int32_t dtype;       /* BLOSSOM_DTYPE_FP32 or BLOSSOM_DTYPE_BF16                               */
   float sm_scale;      /* 0 -> 1/sqrt(head_dim); scales block scores and attention logits alike  */
   int64_t stride_b, stride_h, stride_l; /* element strides of every q-shaped tensor              */
