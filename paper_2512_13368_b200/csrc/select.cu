@@ -853,6 +853,135 @@ __global__ void __launch_bounds__(256) score_per_query_kernel(
   emit_row(row, taken, jmin, b, sh.topk, lane);
 }
 
+// The same selection, tiled: one CTA of 256 threads per 64 consecutive positions of a (batch,
+// key/value head), for up to 64 NZ candidate blocks.  The 64 query rows of one head at a time and
+// 64 candidate means at a time sit in shared memory as doubles; thread (row tid / 4, part tid % 4)
+// forms the 16 logits of candidates part + 4 k per chunk (sixteen independent accumulation
+// chains) and keeps the logits of all chunks in registers; the row's softmax takes 4 lanes; the
+// probabilities are added, head after head, into a [64 rows][64 NZ] table in shared memory, from
+// which one warp per row ranks and emits.  The means are read once per tile and head instead of
+// once per position and head.
+template <typename T, int D, int NZ>
+__global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_kernel(
+    Shape sh, const T *__restrict__ q, const double *__restrict__ mean,
+    const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx) {
+  constexpr int PD = D + 1, MP = 64 * NZ;
+  extern __shared__ double dsm[];
+  __shared__ double bound_d[8][2];
+  double *qd = dsm;                // [64][PD] query rows of the current head
+  double *kd = qd + 64 * PD;       // [64][PD] a chunk of candidate means
+  double *P = kd + 64 * PD;        // [64][MP] probabilities summed over the group's heads
+  uint8_t *taken_all = reinterpret_cast<uint8_t *>(P + 64 * MP);  // [8 warps][MP]
+  const int M = sh.M, Bk = sh.Bk;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rt = tid >> 2, part = tid & 3;
+  const int ntile = (sh.L + 63) / 64;
+  const int u = (int)(blockIdx.x / ntile), tile = (int)(blockIdx.x % ntile), n = u / sh.Hkv, hk = u % sh.Hkv;
+  int len = seq_lens ? seq_lens[n] : sh.L;
+  len = min(max(len, 0), sh.L);
+  const int pad0 = sh.L - len;
+  const int t0 = tile * 64, t_last = min(t0 + 63, sh.L - 1);
+  const int jmin = pad0 / Bk;
+  const int nc = t_last / Bk;  // candidates of the tile's rows: blocks jmin .. nc - 1 (row t: those before t / Bk)
+  const int t = t0 + rt;
+  const bool row_on = t >= pad0 && t < sh.L;
+  const int b_row = row_on ? t / Bk : 0;
+
+  if (t_last >= pad0 && nc > jmin) {
+    for (int i = tid; i < 64 * MP; i += 256) P[i] = 0.0;
+    const int ch_lo = jmin / 64, ch_hi = (nc + 63) / 64;  // at most NZ chunks apart (host-checked: M <= 64 NZ)
+    const double *kbase = mean + (int64_t)u * M * D;
+    for (int hg = 0; hg < sh.G; ++hg) {
+      __syncthreads();  // the previous head's rows are no longer read
+      for (int i = tid; i < 64 * (D / 4); i += 256) {
+        const int lr = i / (D / 4), c = (i % (D / 4)) * 4, tt = t0 + lr;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (tt >= pad0 && tt < sh.L) v = ld4(q + row_offset(sh, n, hk * sh.G + hg, tt) + c);
+        double *d = qd + lr * PD + c;
+        d[0] = (double)v.x; d[1] = (double)v.y; d[2] = (double)v.z; d[3] = (double)v.w;
+      }
+      const double *qr = qd + rt * PD;
+      double z[NZ][16];
+      uint32_t on[NZ];
+      double mx = -INFINITY;
+#pragma unroll
+      for (int ci = 0; ci < NZ; ++ci) {
+        on[ci] = 0u;
+        const int ch = ch_lo + ci;
+        if (ch < ch_hi) {  // (block-uniform)
+          const int c0 = ch * 64, nb = min(64, nc - c0);
+          __syncthreads();  // previous users of kd are done (and qd is complete)
+          for (int i = tid; i < 64 * (D / 2); i += 256) {
+            const int lj = i / (D / 2), c = (i % (D / 2)) * 2;
+            double2 v = make_double2(0.0, 0.0);
+            if (lj < nb && c0 + lj >= jmin) v = *reinterpret_cast<const double2 *>(kbase + (int64_t)(c0 + lj) * D + c);
+            kd[lj * PD + c] = v.x;
+            kd[lj * PD + c + 1] = v.y;
+          }
+          __syncthreads();
+#pragma unroll
+          for (int k = 0; k < 16; ++k) z[ci][k] = 0.0;
+#pragma unroll 2
+          for (int c = 0; c < D; ++c) {
+            const double qv = qr[c];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) z[ci][k] = fma(qv, kd[(part + 4 * k) * PD + c], z[ci][k]);
+          }
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            z[ci][k] *= sh.scale_d;
+            const int c = c0 + part + 4 * k;
+            if (row_on && c >= jmin && c < b_row) {
+              on[ci] |= 1u << k;
+              mx = fmax(mx, z[ci][k]);
+            }
+          }
+        }
+      }
+      mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      double den = 0.0;
+#pragma unroll
+      for (int ci = 0; ci < NZ; ++ci)
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+          if ((on[ci] >> k) & 1u) {
+            z[ci][k] = exp(z[ci][k] - mx);
+            den += z[ci][k];
+          }
+      den += __shfl_xor_sync(0xffffffffu, den, 1);
+      den += __shfl_xor_sync(0xffffffffu, den, 2);
+#pragma unroll
+      for (int ci = 0; ci < NZ; ++ci)
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+          if ((on[ci] >> k) & 1u) P[rt * MP + (ch_lo + ci) * 64 - ch_lo * 64 + part + 4 * k] += z[ci][k] / den;  // heads in ascending order
+    }
+  }
+  __syncthreads();
+  // one warp per row: Eq. 13 from the row's summed probabilities (table column = block - 64 ch_lo)
+  const int col0 = (jmin / 64) * 64;
+  uint8_t *taken = taken_all + warp * MP;
+  for (int lr = warp; lr < 64; lr += 8) {
+    const int tt = t0 + lr;
+    if (tt >= sh.L) break;
+    int32_t *row = idx + ((int64_t)u * sh.L + tt) * sh.topk;
+    if (tt < pad0) {
+      for (int i = lane; i < sh.topk; i += 32) row[i] = -1;
+      continue;
+    }
+    const int b = tt / Bk, nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
+    __syncwarp();
+    if (nsel > want && want > 0) {
+      rank_select<double>(P + lr * MP - col0, jmin, b, want, taken - col0, bound_d[warp], lane);
+    } else {
+      for (int j = jmin + lane; j < b; j += 32) taken[j - col0] = want > 0 ? 1 : 0;
+    }
+    __syncwarp();
+    emit_row(row, taken - col0, jmin, b, sh.topk, lane);
+  }
+}
+
 // The arrays the selection kernels work in (the caller's workspace or the built-in scratch).
 struct SelBuffers {
   double *mean;
@@ -889,6 +1018,16 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
     return BLOSSOM_ERR_CUDA;
   }
   if (sh.pq) {  // one selection per query position: block_idx is [B][Hkv][L][top_k]
+    if (sh.M <= 128) {  // the tiled kernel keeps the logits of up to two chunks of 64 blocks in registers
+      const int nz = sh.M <= 64 ? 1 : 2;
+      const size_t tsm = ((size_t)2 * 64 * (D + 1) + (size_t)64 * 64 * nz) * sizeof(double) + (size_t)8 * 64 * nz + 16;
+      auto kern = nz == 1 ? score_per_query_tile_kernel<T, D, 1> : score_per_query_tile_kernel<T, D, 2>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tsm) != cudaSuccess)
+        return BLOSSOM_ERR_CUDA;
+      LaunchScope ls(K_SCORE_SELECT, st);
+      kern<<<(unsigned)(units * ((sh.L + 63) / 64)), 256, tsm, st>>>(sh, q, w.mean, seq_lens, idx);
+      return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
+    }
     const size_t psm = (size_t)8 * (2 * sh.M + D) * sizeof(double) + (size_t)8 * sh.M + 16;
     if (psm > 48 * 1024 && cudaFuncSetAttribute(score_per_query_kernel<T, D>,
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm) != cudaSuccess)
