@@ -293,7 +293,7 @@ def main():
     ap.add_argument("--input-gate", action="store_true",
                     help="input-dependent gate (Eq. 18, one linear layer)")
     ap.add_argument("--non-causal", action="store_true",
-                    help="no causal mask (bidirectional encoder); CUDA-core attention kernels")
+                    help="no causal mask (bidirectional encoder)")
     ap.add_argument("--rope-theta", type=float, default=0.0,
                     help="rotate q and k by position inside the library (0 = off)")
     ap.add_argument("--no-secondary", action="store_true",

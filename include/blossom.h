@@ -72,8 +72,8 @@ typedef struct {
   int32_t causal;      /* 1 = causal mask: key p <= query t everywhere, the selection scores the
                         * blocks before the query block.  0 = none (bidirectional encoders): a
                         * query block scores every other live block, a query sees every valid key of
-                        * its selected blocks, and Eq. 15 is taken as printed (symmetric); CUDA-core
-                        * kernels; not combined with select_mode 1 or cmp_block / cmp_stride       */
+                        * its selected blocks, and Eq. 15 is taken as printed (symmetric); not
+                        * combined with select_mode 1 or cmp_block / cmp_stride                    */
   int32_t select_mode; /* 0 = one selection per query block, from the probabilities summed over the
                         * block's queries (tensor-core kernels for bf16); 1 = one selection per
                         * query position (Eq. 13 as printed): block_idx is then

@@ -136,8 +136,7 @@ def blossom_attention(q, k, v, gate_logits, block_size, top_k, window, seq_lens=
     w_st, b) per head and alpha = sigmoid(<w_lt, out_lt> + <w_st, out_st> + b) per query row
     (differentiable in those parameters).
     causal: False drops the causal mask (bidirectional encoders): a query block scores every other
-    live block, a query sees all valid keys of its selected blocks, Eq. 15 is symmetric; runs on the
-    CUDA-core kernels.
+    live block, a query sees all valid keys of its selected blocks, Eq. 15 is symmetric.
     rope_theta: > 0 applies rotary position embedding to q and k inside the library (interleaved
     pairs, angle t * rope_theta^(-2i / D)); the gradients returned are those of the unrotated q, k.
     phi_logits: optional float32 CUDA tensor [cmp_block or block_size]: Eq. 9's learnable block

@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         const int i = x >> 1, jt = list[i], f = lflags[i], p0 = jt * 64;
         uint64_t maskL = 0ull, maskS = 0ull;
         if (row_valid) {
-          const uint64_t mc = cols_le(t - p0) & cols_ge(pad0 - p0);
+          const uint64_t mc = cols_le((s.causal ? t : s.L - 1) - p0) & cols_ge(pad0 - p0);
           if (f & 1) maskL = mc & expand_block_bits(s.pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk);
           if (f & 2) maskS = mc & st_key_cols(s, t, p0);
         }
@@ -687,7 +687,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       uint64_t maskL = 0ull, maskS = 0ull;
       if (cls2[0] == 8 || cls2[8] == 8) {  // a mixed half tile: per-lane column masks
         if (row_valid) {
-          const uint64_t mc = cols_ge(p - t0) & cols_le(s.L - 1 - t0);
+          const uint64_t mc = cols_ge((s.causal ? p : pad0) - t0) & cols_le(s.L - 1 - t0);
           if (f & 1) maskL = mc & (s.pq ? inv64[g * nT + qt] : expand_block_bits(invb[g * nT + qt], s.Bk));
           if (f & 2) maskS = mc & st_query_cols(s, p, t0);
         }

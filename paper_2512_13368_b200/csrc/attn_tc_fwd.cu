@@ -370,8 +370,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       uint32_t hm = 0u;  // this thread's 32 keys of the tile that the row sees
       bool doB = cls == 1, fullB = cls == 1;
       if (cls == 2) {
-        if (row_ok) {
-          uint64_t mask = cols_le(t - p0) & cols_ge(pad0 - p0);
+        if (row_ok && t >= pad0) {  // (a padded row sees nothing; under the causal mask the bounds below say so by themselves)
+          uint64_t mask = cols_le((s.causal ? t : s.L - 1) - p0) & cols_ge(pad0 - p0);
           mask &= isL ? expand_block_bits(s.pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk) : st_key_cols(s, t, p0);
           hm = (uint32_t)(mask >> (32 * grp));
         }

@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
       if (qb < s.M) {
         const int blk = idx[((int64_t)uk * s.M + qb) * s.topk + slot];
-        if (blk >= 0 && blk <= qb) {
+        if (blk >= 0 && blk < s.M && (blk <= qb || !s.causal)) {
           const int a = g * nT + blk / nb;
           atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
         }
@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     __syncwarp();
     int nv = 0;
     {  // the tiles any row of the CTA needs, ascending
-      const int jt_max = row_last >> 6;
+      const int jt_max = (s.causal ? row_last : s.L - 1) >> 6;
       for (int base = 0; base <= jt_max; base += 32) {
         const int jt = base + lane;
         int f = 0;
@@ -180,8 +180,9 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     for (int e = lane; e < count * 4; e += 32) {
       const int it = e >> 2, w = e & 3;
       const int jt = items[it], p0 = jt * 64, t_lo = row0 + w * 32;
-      const bool some = p0 <= t_lo + 31 && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
-      const bool inner = t_lo >= pad0 && t_lo + 31 < s.L && p0 >= pad0 && p0 + 63 <= t_lo;
+      const bool some = (p0 <= t_lo + 31 || !s.causal) && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
+      // every row of the warp may see every key of the tile as far as validity and causality go
+      const bool inner = t_lo >= pad0 && t_lo + 31 < s.L && p0 >= pad0 && (s.causal ? p0 + 63 <= t_lo : p0 + 63 < s.L);
       int cls = 0;
       if (some) {
         if (it < nl) {
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
             cls = bits == 0u ? 0 : ((!s.pq && inner && bits == allbits) ? 1 : 2);  // (per position: the rows differ)
           }
         } else if (st_ranges_touch(s, t_lo, t_lo + 31, p0, p0 + 63)) {
-          cls = (inner && p0 >= t_lo + 31 - s.window + 1) ? 1 : 2;  // 1: inside every row's window
+          cls = (inner && p0 >= t_lo + 31 - s.window + 1 && (s.causal || p0 + 63 <= t_lo + s.window - 1)) ? 1 : 2;  // 1: inside every row's window
         }
       }
       icls[e] = (uint8_t)cls;
@@ -218,7 +219,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                 if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
             if (lflags[j] & 2)
               for (int hf = 0; hf < 2; ++hf)
-                if (p0 <= row0 + 64 * hf + 63 &&
+                if ((p0 <= row0 + 64 * hf + 63 || !s.causal) &&
                     st_ranges_touch(s, row0 + 64 * hf, row0 + 64 * hf + 63, p0, p0 + 63))
                   c |= 1 << hf;
             if (c == 0) c = 3;
@@ -263,8 +264,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       const int jt = list[it], f = lflags[it];
       const int k_lo = jt * 64 + 32 * hh + 16 * c, k_hi = k_lo + 15, t_lo = row0 + qtr * 32, t_hi = t_lo + 31;
       const bool rows_in = t_lo >= pad0 && t_hi < s.L, rows_none = t_hi < pad0 || t_lo >= s.L;
-      const bool past = rows_in && k_lo >= pad0 && k_hi <= t_lo;  // every key causally visible to every row
-      const bool reach = !rows_none && k_lo <= t_hi && k_hi >= pad0;  // some key may be visible to some row
+      const bool past = rows_in && k_lo >= pad0 && (s.causal ? k_hi <= t_lo : k_hi < s.L);  // every key visible to every row (validity, causality)
+      const bool reach = !rows_none && (k_lo <= t_hi || !s.causal) && k_hi >= pad0 && k_lo < s.L;  // some key may be visible to some row
       int cL = 0, cS = 0;  // 0 none, 1 all, 2 mixed
       if ((f & 1) && reach) {
         const int kb = (32 * hh + 16 * c) >> bk_shift;  // key block within the tile
@@ -277,7 +278,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         if (any_sel) cL = (all_sel && past && !s.pq) ? 1 : 2;
       }
       if ((f & 2) && reach && st_ranges_touch(s, t_lo, t_hi, k_lo, k_hi))
-        cS = (past && k_lo >= t_hi - s.window + 1) ? 1 : 2;  // 1: inside every row's window
+        cS = (past && k_lo >= t_hi - s.window + 1 && (s.causal || k_hi <= t_lo + s.window - 1)) ? 1 : 2;  // 1: inside every row's window
       jcls[e] = (uint8_t)((cL == 2 || cS == 2) ? 8 : (cL | (cS << 1)));
     }
   } else {
@@ -308,8 +309,9 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
     } else {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
       // (the index rows of query blocks qb0 .. M-1 are contiguous; eight loads in flight per lane)
-      const int qb0 = kt * G, total = (s.M - qb0) * s.topk;
-      const int32_t *rows = idx + ((int64_t)uk * s.M + qb0) * s.topk;
+      // (without the causal mask every query block may have selected them: the rows start at block 0)
+      const int qb0 = kt * G, qb_first = s.causal ? qb0 : 0, total = (s.M - qb_first) * s.topk;
+      const int32_t *rows = idx + ((int64_t)uk * s.M + qb_first) * s.topk;
       for (int base = 0; base < total; base += 256) {
         int blk[8];
 #pragma unroll
@@ -319,8 +321,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         }
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const int i = base + e * 32 + lane, qb = qb0 + i / s.topk;
-          if (blk[e] >= qb0 && blk[e] < qb0 + G && blk[e] <= qb) {
+          const int i = base + e * 32 + lane, qb = qb_first + i / s.topk;
+          if (blk[e] >= qb0 && blk[e] < qb0 + G && (blk[e] <= qb || !s.causal)) {
             const int a = (blk[e] - qb0) * nT + qb / nb;
             atomicOr(&selw[a >> 2], (1u << (qb % nb)) << ((a & 3) * 8));
           }
@@ -328,7 +330,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
     }
     __syncwarp();
-    const int qt_min = key0 >> 6, qt_max = (s.L - 1) >> 6;
+    const int qt_min = s.causal ? key0 >> 6 : 0, qt_max = (s.L - 1) >> 6;
     int count = 0;
     for (int base = qt_min; base <= qt_max; base += 32) {
       const int qt = base + lane;
@@ -357,8 +359,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       const int qt = list[it], f = lflags[it], c_lo = 32 * hh + 16 * hf;
       const int p_lo = key0 + 32 * qtr, p_hi = p_lo + 31, t_lo = qt * 64 + c_lo, t_hi = t_lo + 15;
       const bool rows_in = p_lo >= pad0 && p_hi < s.L, rows_none = p_hi < pad0 || p_lo >= s.L;
-      const bool past = rows_in && t_hi < s.L && t_lo >= p_hi;  // every query causally sees every key
-      const bool reach = !rows_none && t_hi >= p_lo && t_lo < s.L;  // some query may see some key
+      const bool past = rows_in && t_hi < s.L && (s.causal ? t_lo >= p_hi : t_lo >= pad0);  // every query sees every key (validity, causality)
+      const bool reach = !rows_none && (t_hi >= p_lo || !s.causal) && t_hi >= pad0 && t_lo < s.L;  // some query may see some key
       int cL = 0, cS = 0;  // 0 none, 1 all, 2 mixed
       if ((f & 1) && reach) {
         bool any_sel = false, all_sel = true;
@@ -373,7 +375,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
         if (any_sel) cL = (all_sel && past && !s.pq) ? 1 : 2;
       }
       if ((f & 2) && reach && st_ranges_touch(s, t_lo, min(t_hi, s.L - 1), p_lo, min(p_hi, s.L - 1)))
-        cS = (past && p_lo >= t_hi - s.window + 1) ? 1 : 2;  // 1: inside every query's window
+        cS = (past && p_lo >= t_hi - s.window + 1 && (s.causal || p_hi <= t_lo + s.window - 1)) ? 1 : 2;  // 1: inside every query's window
       jcls[e] = (uint8_t)((cL == 2 || cS == 2) ? 8 : (cL | (cS << 1)));
     }
   }

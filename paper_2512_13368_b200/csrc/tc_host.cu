@@ -77,7 +77,7 @@ bool fwd_tc_supported(const Shape &s, int dtype) {
   // (a selection per query position adds 128 bytes per tile to a CTA's bookkeeping in shared
   // memory: up to 64 tiles, i.e. L <= 4096; longer sequences take the CUDA-core kernels)
   // (the input-dependent gate goes through launch_fwd_tc_gate / launch_bwd_tc_gate)
-  return s.causal && (!s.pq || (s.L + 63) / 64 <= 64) && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
+  return (!s.pq || (s.L + 63) / 64 <= 64) && dtype == BLOSSOM_DTYPE_BF16 && (s.D == 32 || s.D == 64) &&
          (s.Bk == 16 || s.Bk == 32 || s.Bk == 64) && (s.L + 63) / 64 <= 1024;
 }
 

@@ -709,6 +709,40 @@ def test_without_the_causal_mask(runner, dtype, L, D, H, Hkv, block, topk, windo
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.parametrize("block,power_law", [(16, False), (32, True), (64, False)])
+def test_without_the_causal_mask_runs_on_the_tensor_core_kernels(runner, block, power_law):
+    """bf16 shapes keep the tensor-core kernels with causal = 0 (tile lists over both sides of the
+    diagonal, whole selected blocks, the symmetric short-term mask): the launch record shows those
+    kernels, and the results agree with the oracle and with the CUDA-core path."""
+    from paper_2512_13368_b200 import binding
+    w = workloads.make("non-causal-tc", "bf16", 3, 4, 1000, 64, block, 5, 70, seed=83, kv_heads=2, lengths=(300, 1000),
+                       stis_mode=1 if power_law else 0, stis_block=2 if power_law else 1)
+    w.causal = 0
+    binding.blossom_profile_start(64)
+    _, tc = run(runner, w)
+    names = {name for name, _ in binding.blossom_profile_stop(64)}
+    assert {"fwd_tc", "bwd_dq_tc", "bwd_dkdv_tc"} <= names and not any("simt" in x for x in names), names
+    print(check_forward_backward(w, tc))
+    binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, 1)
+    try:
+        _, simt = run(runner, w)
+    finally:
+        binding.blossom_debug_switch(binding.SWITCH_FORCE_SIMT, -1)
+    assert np.array_equal(tc["idx"], simt["idx"])
+    for key in ("out", "out_lt", "out_st", "lse", "dq", "dk", "dv", "dgate"):
+        ref = np.abs(simt[key]).max()
+        err = np.abs(tc[key] - simt[key]).max()
+        assert err <= 2e-2 * max(ref, 1e-3), (key, err, ref)
+
+
+def test_config4_full_size_without_the_causal_mask(runner):
+    """The headline shape without the causal mask, as the benchmark's --non-causal option times it."""
+    w = workloads.config4()
+    w.causal = 0
+    errs, _ = _whole_batch(runner, w)
+    print(errs)
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("L,D,H,Hkv,block,topk,window,lens", [
     (64, 32, 2, 2, 8, 2, 16, None),
