@@ -397,6 +397,117 @@ int blossom_oracle_select_cmp(int B, int H, int L, int D, int Bk, int topk, int 
   return 0;
 }
 
+/* ---- selection per query position through overlapping compression blocks ---- */
+/* Eq. 8-11 and Eq. 13 as printed (one selection per position): position t, in selection block
+ * b = t / Bk, scores the live compression blocks that end before its block starts (the rule of
+ * the per-block selection above, so no summary holds a key the position must not see), takes its
+ * own softmax over them (Eq. 10), maps the probabilities onto the selection blocks j < b with
+ * Eq. 11, and keeps its own block plus the top-(k-1) selectable past blocks, ties to the lower
+ * index.  scores, if given, receives the mapped scores [L][M] (zero where not selectable). */
+static void select_unit_pq_cmp(int L, int D, int Bk, int topk, int l, int s, double scale, int pad0,
+                               const double *q, const double *k, const double *phi, int32_t *idx,
+                               double *scores) {
+  const int M = n_blocks(L, Bk);
+  const int Mc = L >= l ? (L - l) / s + 1 : 0;
+  const int rs = Bk / s, rl = l / s;
+  double *ktil = (double *)calloc((size_t)(Mc > 0 ? Mc : 1) * D, sizeof(double));
+  int *livec = (int *)calloc((size_t)(Mc > 0 ? Mc : 1), sizeof(int));
+  double *P = (double *)malloc(sizeof(double) * (size_t)(Mc > 0 ? Mc : 1));
+  double *S = (double *)malloc(sizeof(double) * (size_t)M);
+  char *taken = (char *)malloc((size_t)M);
+  for (int i = 0; i < Mc; ++i) { /* Eq. 8 + Eq. 9 */
+    int lo = imax(i * s, pad0), hi = i * s + l, cnt = 0;
+    double wsum = 0.0;
+    for (int p = lo; p < hi; ++p) {
+      const double w = phi_weight(phi, p - i * s);
+      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] += w * k[(size_t)p * D + c];
+      wsum += w;
+      ++cnt;
+    }
+    livec[i] = cnt > 0;
+    if (cnt > 0)
+      for (int c = 0; c < D; ++c) ktil[(size_t)i * D + c] /= wsum;
+  }
+  for (int t = 0; t < L; ++t) {
+    int32_t *row = idx + (size_t)t * topk;
+    for (int e = 0; e < topk; ++e) row[e] = -1;
+    if (scores)
+      for (int j = 0; j < M; ++j) scores[(size_t)t * M + j] = 0.0;
+    if (t < pad0) continue;
+    const int b = t / Bk;
+    int nc = 0; /* compression blocks 0 .. nc-1 end before block b starts */
+    while (nc < Mc && nc * s + l <= b * Bk) ++nc;
+    double mx = -INFINITY;
+    int ncand = 0;
+    for (int i = 0; i < nc; ++i) {
+      P[i] = 0.0;
+      if (!livec[i]) continue;
+      ++ncand;
+      double acc = 0.0;
+      for (int c = 0; c < D; ++c) acc += q[(size_t)t * D + c] * ktil[(size_t)i * D + c];
+      P[i] = scale * acc;
+      if (P[i] > mx) mx = P[i];
+    }
+    if (ncand > 0) { /* Eq. 10 */
+      double den = 0.0;
+      for (int i = 0; i < nc; ++i)
+        if (livec[i]) den += exp(P[i] - mx);
+      for (int i = 0; i < nc; ++i) P[i] = livec[i] ? exp(P[i] - mx) / den : 0.0;
+    }
+    int nlive = 0;
+    for (int j = 0; j < b; ++j) { /* Eq. 11 */
+      double acc = 0.0;
+      for (int m = 0; m < rs; ++m)
+        for (int n = 0; n < rl; ++n) {
+          int i = rs * j - m - n;
+          if (i >= 0 && i < nc && livec[i]) acc += P[i];
+        }
+      S[j] = acc;
+      taken[j] = 0;
+      if (imin((j + 1) * Bk, L) > imax(j * Bk, pad0)) {
+        ++nlive;
+        if (scores) scores[(size_t)t * M + j] = acc;
+      } else {
+        taken[j] = 2; /* not selectable */
+      }
+    }
+    int want = imin(topk - 1, nlive); /* Eq. 13 */
+    for (int e = 0; e < want; ++e) {
+      int best = -1;
+      for (int j = 0; j < b; ++j) {
+        if (taken[j]) continue;
+        if (best < 0 || S[j] > S[best]) best = j;
+      }
+      taken[best] = 1;
+    }
+    int e = 0;
+    for (int j = 0; j < b; ++j)
+      if (taken[j] == 1) row[e++] = j;
+    row[e++] = b;
+  }
+  free(ktil); free(livec); free(P); free(S); free(taken);
+}
+
+int blossom_oracle_select_pq_cmp(int B, int H, int L, int D, int Bk, int topk, int l, int s,
+                                 double scale, const double *q, const double *k,
+                                 const int32_t *seq_lens, const double *phi /* [l] or NULL */,
+                                 int32_t *idx /* [B][H][L][topk] */, double *scores /* [B][H][L][M] or NULL */) {
+  if (B < 1 || H < 1 || L < 1 || D < 1 || Bk < 1 || topk < 1) return 1;
+  if (l < 1 || s < 1 || l % s || Bk % s) return 1;
+  const int M = n_blocks(L, Bk);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+  for (int n = 0; n < B; ++n)
+    for (int h = 0; h < H; ++h) {
+      size_t u = (size_t)n * H + h;
+      int len = seq_lens ? seq_lens[n] : L;
+      if (len < 0) len = 0;
+      if (len > L) len = L;
+      select_unit_pq_cmp(L, D, Bk, topk, l, s, scale, L - len, q + u * L * D, k + u * L * D, phi,
+                         idx + u * (size_t)L * topk, scores ? scores + u * (size_t)L * M : NULL);
+    }
+  return 0;
+}
+
 /* ---- one softmax-attention row over an explicit key list: Eq. 1 ---------- */
 /* keys[0..nk) are key positions; writes out[D], returns lse (0 and zeros if nk == 0) */
 static double attend_row(int D, double scale, const double *qt, const double *k, const double *v,

@@ -54,6 +54,8 @@ def _load():
         lib.blossom_oracle_forward.restype = i
         lib.blossom_oracle_select_pq.restype = i
         lib.blossom_oracle_select_pq.argtypes = [i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
+        lib.blossom_oracle_select_pq_cmp.restype = i
+        lib.blossom_oracle_select_pq_cmp.argtypes = [i, i, i, i, i, i, i, i, d, _dp, _dp, _ip, _dp, _ip, _dp]
         lib.blossom_oracle_forward.argtypes = [i, i, i, i, i, i, i, i, i, i, i, i, d, _dp, _dp, _dp, _dp, _ip,
                                                _ip, _dp, _dp, _dp, _dp]
         lib.blossom_oracle_backward.restype = i
@@ -121,11 +123,14 @@ def select_blocks(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores
 
 
 def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, return_scores=False,
-                            phi_logits=None):
+                            phi_logits=None, cmp_block=0, cmp_stride=0):
     """Eq. 8-10, 13 as printed: one selection per query position.  k may have fewer heads than q
     (grouped heads: the probabilities of a group's heads are summed, Eq. 12, and the group's
-    queries at one position share the selection).  Returns idx ``[B,Hkv,L,topk]`` (ascending, -1
-    padded, the position's own block included) and, if asked, the probabilities ``[B,Hkv,L,M]``."""
+    queries at one position share the selection).  With ``cmp_block`` / ``cmp_stride`` the position
+    scores overlapping compression blocks and Eq. 11 maps its probabilities onto the selection
+    blocks (the paper's selection in full).  Returns idx ``[B,Hkv,L,topk]`` (ascending, -1
+    padded, the position's own block included) and, if asked, the (mapped) probabilities
+    ``[B,Hkv,L,M]``."""
     q, k = _f64(q), _f64(k)
     B, H, L, D = q.shape
     Hkv = k.shape[1]
@@ -135,10 +140,17 @@ def select_blocks_per_query(q, k, block, topk, seq_lens=None, sm_scale=None, ret
     probs = np.zeros((B, H, L, M), dtype=np.float64) if (return_scores or G > 1) else None
     sl = _lens(seq_lens, B)
     kk = np.ascontiguousarray(np.repeat(k, G, axis=1))
-    ph = _phi(phi_logits, block)
-    rc = _load().blossom_oracle_select_pq(B, H, L, D, block, topk, _scale(sm_scale, D), _ptr(q, _dp),
-                                          _ptr(kk, _dp), _ptr(sl, _ip), _ptr(ph, _dp), _ptr(idx, _ip),
-                                          _ptr(probs, _dp))
+    if cmp_block or cmp_stride:
+        l, s = int(cmp_block or block), int(cmp_stride or block)
+        ph = _phi(phi_logits, l)
+        rc = _load().blossom_oracle_select_pq_cmp(B, H, L, D, block, topk, l, s, _scale(sm_scale, D),
+                                                  _ptr(q, _dp), _ptr(kk, _dp), _ptr(sl, _ip), _ptr(ph, _dp),
+                                                  _ptr(idx, _ip), _ptr(probs, _dp))
+    else:
+        ph = _phi(phi_logits, block)
+        rc = _load().blossom_oracle_select_pq(B, H, L, D, block, topk, _scale(sm_scale, D), _ptr(q, _dp),
+                                              _ptr(kk, _dp), _ptr(sl, _ip), _ptr(ph, _dp), _ptr(idx, _ip),
+                                              _ptr(probs, _dp))
     if rc:
         raise ValueError("blossom_oracle_select_pq: bad arguments")
     if G == 1:
@@ -361,7 +373,8 @@ def forward_gqa(q, k, v, gate, block, topk, window, seq_lens=None, sm_scale=None
     q, k, v = _f64(q), _f64(k), _f64(v)
     G = _group(q.shape[1], k.shape[1])
     if idx is None and kw.get("per_query"):
-        idx = select_blocks_per_query(q, k, block, topk, seq_lens, sm_scale)
+        idx = select_blocks_per_query(q, k, block, topk, seq_lens, sm_scale, cmp_block=cmp_block,
+                                      cmp_stride=cmp_stride)
     elif idx is None:
         idx = select_blocks_gqa(q, k, block, topk, seq_lens, sm_scale, cmp_block=cmp_block,
                                 cmp_stride=cmp_stride)

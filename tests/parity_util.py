@@ -47,7 +47,8 @@ def check_indices(w, gpu_idx, sm_scale=None):
     phi = getattr(w, "phi_logits", None)
     if pq:
         ref_idx, scores = oracle.select_blocks_per_query(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
-                                                         return_scores=True, phi_logits=phi)
+                                                         return_scores=True, phi_logits=phi,
+                                                         cmp_block=w.cmp_block, cmp_stride=w.cmp_stride)
     elif _grouped(w):
         ref_idx, scores = oracle.select_blocks_gqa(w.q, w.k, w.block, w.topk, w.seq_lens, sm_scale,
                                                    return_scores=True, cmp_block=w.cmp_block,

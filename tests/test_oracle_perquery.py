@@ -157,3 +157,79 @@ def test_grouped_heads_share_one_per_position_selection():
     np.testing.assert_array_equal(f["idx"], idx)
     g = oracle.backward_gqa(q, k, v, gate, 8, 3, 5, f, dout, per_query=True)
     assert g["dk"].shape == k.shape
+
+
+# ---- per position through overlapping compression blocks (Eq. 8-11, 13 as printed) ------------
+def test_compression_blocks_equal_to_the_selection_blocks_change_nothing():
+    q, k, *_ = rand_case(11, L=72)
+    sl = np.asarray([72, 31], dtype=np.int32)
+    a, pa = oracle.select_blocks_per_query(q, k, 8, 3, sl, return_scores=True)
+    b, pb = oracle.select_blocks_per_query(q, k, 8, 3, sl, return_scores=True, cmp_block=8, cmp_stride=8)
+    np.testing.assert_array_equal(a, b)
+    np.testing.assert_allclose(pa, pb, rtol=0, atol=1e-15)
+
+
+def test_equal_queries_in_a_block_select_what_the_block_selects_through_compression_blocks():
+    q, k, *_ = rand_case(12, L=96)
+    q = np.repeat(q[:, :, ::8], 8, axis=2)           # every query of a block of 8 is the same vector
+    per_block, sb, _ = oracle.select_blocks_cmp(q, k, 8, 3, 16, 4, return_scores=True)
+    per_query, sq = oracle.select_blocks_per_query(q, k, 8, 3, return_scores=True, cmp_block=16, cmp_stride=4)
+    np.testing.assert_array_equal(per_query, np.repeat(per_block, 8, axis=2))
+    # a block's score is the sum over its 8 equal queries of the position's score
+    np.testing.assert_allclose(np.repeat(sb, 8, axis=2), 8.0 * sq, rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("lens", [None, [70, 27]])
+@pytest.mark.parametrize("Bk,l,s", [(8, 16, 4), (16, 32, 16), (8, 8, 4)])
+def test_compression_blocks_against_a_numpy_scorer(lens, Bk, l, s):
+    """Means by slicing, one softmax per position over the compression blocks that end before the
+    position's block, Eq. 11 as a double sum, stable arg-sort: written without the oracle's code."""
+    L, topk, D = 70, 3, 8
+    q, k, *_ = rand_case(13, L=L, D=D)
+    sl = None if lens is None else np.asarray(lens, dtype=np.int32)
+    idx, sc = oracle.select_blocks_per_query(q, k, Bk, topk, sl, return_scores=True, cmp_block=l, cmp_stride=s)
+    M, Mc = -(-L // Bk), (L - l) // s + 1
+    for n in range(2):
+        pad0 = 0 if sl is None else L - int(sl[n])
+        for h in range(2):
+            means, live = np.zeros((Mc, D)), np.zeros(Mc, dtype=bool)
+            for i in range(Mc):
+                lo = max(i * s, pad0)
+                if lo < i * s + l:
+                    means[i], live[i] = k[n, h, lo:i * s + l].mean(axis=0), True
+            for t in range(L):
+                if t < pad0:
+                    assert list(idx[n, h, t]) == [-1] * topk
+                    continue
+                b = t // Bk
+                cands = [i for i in range(Mc) if i * s + l <= b * Bk and live[i]]
+                p = np.zeros(Mc)
+                if cands:
+                    z = (means[cands] @ q[n, h, t]) / math.sqrt(D)
+                    e = np.exp(z - z.max())
+                    p[cands] = e / e.sum()
+                S = np.zeros(M)
+                for j in range(b):
+                    for m in range(Bk // s):
+                        for r in range(l // s):
+                            i = (Bk // s) * j - m - r
+                            if 0 <= i < Mc and i * s + l <= b * Bk:
+                                S[j] += p[i]
+                sel = [j for j in range(b) if min((j + 1) * Bk, L) > max(j * Bk, pad0)]
+                order = sorted(sel, key=lambda j: (-S[j], j))[:topk - 1]
+                want = sorted(order) + [b]
+                assert [int(x) for x in idx[n, h, t] if x >= 0] == want, (n, h, t)
+                np.testing.assert_allclose(sc[n, h, t, sel], S[sel], rtol=1e-12, atol=1e-14)
+
+
+def test_grouped_heads_sum_the_mapped_probabilities_of_a_position():
+    q, k, *_ = rand_case(14, H=4, Hkv=2, L=64)
+    idx, sc = oracle.select_blocks_per_query(q, k, 8, 3, return_scores=True, cmp_block=16, cmp_stride=8)
+    assert idx.shape == (2, 2, 64, 3)
+    _, per_head = oracle.select_blocks_per_query(q, np.repeat(k, 2, axis=1), 8, 3, return_scores=True,
+                                                 cmp_block=16, cmp_stride=8)
+    np.testing.assert_allclose(sc, per_head.reshape(2, 2, 2, 64, 8).sum(axis=2), rtol=1e-13, atol=1e-15)
+    t = 63
+    row = [int(x) for x in idx[0, 1, t] if x >= 0]
+    best = sorted(range(7), key=lambda j: (-sc[0, 1, t, j], j))[:2]
+    assert row == sorted(best) + [7]
