@@ -78,8 +78,10 @@ typedef struct {
                         * block's queries (tensor-core kernels for bf16); 1 = one selection per
                         * query position (Eq. 13 as printed): block_idx is then
                         * [B][kv_heads][L][top_k], a row per position (tensor-core kernels for
-                        * bf16 up to 4096 positions, CUDA-core kernels beyond); not combined with
-                        * cmp_block / cmp_stride                                                   */
+                        * bf16 up to 4096 positions, CUDA-core kernels beyond).  With cmp_block /
+                        * cmp_stride a position scores the compression blocks that end before its
+                        * selection block starts (up to 128 selection and 128 compression blocks,
+                        * else BLOSSOM_ERR_UNSUPPORTED)                                            */
   int32_t dtype;       /* BLOSSOM_DTYPE_FP32 or BLOSSOM_DTYPE_BF16                               */
   float sm_scale;      /* 0 -> 1/sqrt(head_dim); scales block scores and attention logits alike  */
   int64_t stride_b, stride_h, stride_l; /* element strides of every q-shaped tensor              */

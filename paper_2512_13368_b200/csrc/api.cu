@@ -170,7 +170,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   if (!s.causal && (s.pq || s.cmp_l > 0)) return BLOSSOM_ERR_UNSUPPORTED;  // bidirectional: plain per-block selection
   s.phi = p->phi_logits;
   if (reinterpret_cast<uintptr_t>(s.phi) % 4) return BLOSSOM_ERR_INVALID_ARG;
-  if (s.pq && s.cmp_l > 0) return BLOSSOM_ERR_UNSUPPORTED;  // per-position selection scores the selection blocks themselves
+  // per-position selection through compression blocks: the tiled kernel only (up to 128 blocks of either kind)
+  if (s.pq && s.cmp_l > 0 && (s.Mc > 128 || s.M > 128)) return BLOSSOM_ERR_UNSUPPORTED;
   if (kv_given) {
     s.ksb = p->kv_stride_b; s.ksh = p->kv_stride_h; s.ksl = p->kv_stride_l;
   } else if (s.G == 1) {

@@ -854,7 +854,8 @@ __global__ void __launch_bounds__(256) score_per_query_kernel(
 }
 
 // The same selection, tiled: one CTA of 256 threads per 64 consecutive positions of a (batch,
-// key/value head), for up to 64 NZ candidate blocks.  The 64 query rows of one head at a time and
+// key/value head), for up to 64 NZ scored blocks (the selection blocks themselves, or overlapping
+// compression blocks whose probabilities Eq. 11 maps onto the selection blocks, row by row).  The 64 query rows of one head at a time and
 // 64 candidate means at a time sit in shared memory as doubles; thread (row tid / 4, part tid % 4)
 // forms the 16 logits of candidates part + 4 k per chunk (sixteen independent accumulation
 // chains) and keeps the logits of all chunks in registers; the row's softmax takes 4 lanes; the
@@ -863,7 +864,7 @@ __global__ void __launch_bounds__(256) score_per_query_kernel(
 // once per position and head.
 template <typename T, int D, int NZ>
 __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_kernel(
-    Shape sh, const T *__restrict__ q, const double *__restrict__ mean,
+    Shape sh, SelGeom g, const T *__restrict__ q, const double *__restrict__ mean,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx) {
   constexpr int PD = D + 1, MP = 64 * NZ;
   extern __shared__ double dsm[];
@@ -871,7 +872,8 @@ __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_ker
   double *qd = dsm;                // [64][PD] query rows of the current head
   double *kd = qd + 64 * PD;       // [64][PD] a chunk of candidate means
   double *P = kd + 64 * PD;        // [64][MP] probabilities summed over the group's heads
-  uint8_t *taken_all = reinterpret_cast<uint8_t *>(P + 64 * MP);  // [8 warps][MP]
+  double *Smap = P + 64 * MP;      // [8 warps][MP] a row's scores of the selection blocks (Eq. 11; overlapping mode)
+  uint8_t *taken_all = reinterpret_cast<uint8_t *>(Smap + (g.plain ? 0 : 8 * MP));  // [8 warps][MP]
   const int M = sh.M, Bk = sh.Bk;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rt = tid >> 2, part = tid & 3;
@@ -881,16 +883,18 @@ __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_ker
   len = min(max(len, 0), sh.L);
   const int pad0 = sh.L - len;
   const int t0 = tile * 64, t_last = min(t0 + 63, sh.L - 1);
-  const int jmin = pad0 / Bk;
-  const int nc = t_last / Bk;  // candidates of the tile's rows: blocks jmin .. nc - 1 (row t: those before t / Bk)
+  const int jmin = pad0 / Bk;                    // selectable selection blocks: j >= jmin
+  const int cmin = first_live_scored(g, pad0);   // live scored blocks: c >= cmin
+  // candidates of the tile's rows: scored blocks cmin .. nc - 1 (row t: those that end before block t / Bk)
+  const int nc = n_candidates(sh, g, t_last / Bk);
   const int t = t0 + rt;
   const bool row_on = t >= pad0 && t < sh.L;
-  const int b_row = row_on ? t / Bk : 0;
+  const int nc_row = row_on ? n_candidates(sh, g, t / Bk) : 0;
 
-  if (t_last >= pad0 && nc > jmin) {
+  if (t_last >= pad0 && nc > cmin) {
     for (int i = tid; i < 64 * MP; i += 256) P[i] = 0.0;
-    const int ch_lo = jmin / 64, ch_hi = (nc + 63) / 64;  // at most NZ chunks apart (host-checked: M <= 64 NZ)
-    const double *kbase = mean + (int64_t)u * M * D;
+    const int ch_lo = cmin / 64, ch_hi = (nc + 63) / 64;  // at most NZ chunks apart (host-checked: blocks <= 64 NZ)
+    const double *kbase = mean + (int64_t)u * g.n * D;
     for (int hg = 0; hg < sh.G; ++hg) {
       __syncthreads();  // the previous head's rows are no longer read
       for (int i = tid; i < 64 * (D / 4); i += 256) {
@@ -914,7 +918,7 @@ __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_ker
           for (int i = tid; i < 64 * (D / 2); i += 256) {
             const int lj = i / (D / 2), c = (i % (D / 2)) * 2;
             double2 v = make_double2(0.0, 0.0);
-            if (lj < nb && c0 + lj >= jmin) v = *reinterpret_cast<const double2 *>(kbase + (int64_t)(c0 + lj) * D + c);
+            if (lj < nb && c0 + lj >= cmin) v = *reinterpret_cast<const double2 *>(kbase + (int64_t)(c0 + lj) * D + c);
             kd[lj * PD + c] = v.x;
             kd[lj * PD + c + 1] = v.y;
           }
@@ -931,7 +935,7 @@ __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_ker
           for (int k = 0; k < 16; ++k) {
             z[ci][k] *= sh.scale_d;
             const int c = c0 + part + 4 * k;
-            if (row_on && c >= jmin && c < b_row) {
+            if (row_on && c >= cmin && c < nc_row) {
               on[ci] |= 1u << k;
               mx = fmax(mx, z[ci][k]);
             }
@@ -959,9 +963,11 @@ __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_ker
     }
   }
   __syncthreads();
-  // one warp per row: Eq. 13 from the row's summed probabilities (table column = block - 64 ch_lo)
-  const int col0 = (jmin / 64) * 64;
+  // one warp per row: Eq. 11 and Eq. 13 from the row's summed probabilities (table column =
+  // scored block - 64 ch_lo)
+  const int col0 = (cmin / 64) * 64;
   uint8_t *taken = taken_all + warp * MP;
+  double *Srow = Smap + warp * MP;
   for (int lr = warp; lr < 64; lr += 8) {
     const int tt = t0 + lr;
     if (tt >= sh.L) break;
@@ -973,12 +979,20 @@ __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_ker
     const int b = tt / Bk, nsel = max(0, b - jmin), want = min(sh.topk - 1, nsel);
     __syncwarp();
     if (nsel > want && want > 0) {
-      rank_select<double>(P + lr * MP - col0, jmin, b, want, taken - col0, bound_d[warp], lane);
+      if (g.plain) {
+        rank_select<double>(P + lr * MP - col0, jmin, b, want, taken, bound_d[warp], lane);
+      } else if (n_candidates(sh, g, b) > cmin) {
+        map_scores<double>(g, P + lr * MP - col0, cmin, n_candidates(sh, g, b), jmin, b, Srow, lane);
+        __syncwarp();
+        rank_select<double>(Srow, jmin, b, want, taken, bound_d[warp], lane);
+      } else {  // no compression block lies in the past yet: all scores are zero, the lowest blocks win the ties
+        for (int j = jmin + lane; j < b; j += 32) taken[j] = j - jmin < want ? 1 : 0;
+      }
     } else {
-      for (int j = jmin + lane; j < b; j += 32) taken[j - col0] = want > 0 ? 1 : 0;
+      for (int j = jmin + lane; j < b; j += 32) taken[j] = want > 0 ? 1 : 0;
     }
     __syncwarp();
-    emit_row(row, taken - col0, jmin, b, sh.topk, lane);
+    emit_row(row, taken, jmin, b, sh.topk, lane);
   }
 }
 
@@ -1018,16 +1032,18 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
     return BLOSSOM_ERR_CUDA;
   }
   if (sh.pq) {  // one selection per query position: block_idx is [B][Hkv][L][top_k]
-    if (sh.M <= 128) {  // the tiled kernel keeps the logits of up to two chunks of 64 blocks in registers
-      const int nz = sh.M <= 64 ? 1 : 2;
-      const size_t tsm = ((size_t)2 * 64 * (D + 1) + (size_t)64 * 64 * nz) * sizeof(double) + (size_t)8 * 64 * nz + 16;
+    if (g.n <= 128 && sh.M <= 128) {  // the tiled kernel keeps the logits of up to two chunks of 64 blocks in registers
+      const int nz = (g.n <= 64 && sh.M <= 64) ? 1 : 2;
+      const size_t tsm = ((size_t)2 * 64 * (D + 1) + (size_t)64 * 64 * nz + (g.plain ? 0 : (size_t)8 * 64 * nz)) * sizeof(double) +
+                         (size_t)8 * 64 * nz + 16;
       auto kern = nz == 1 ? score_per_query_tile_kernel<T, D, 1> : score_per_query_tile_kernel<T, D, 2>;
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tsm) != cudaSuccess)
         return BLOSSOM_ERR_CUDA;
       LaunchScope ls(K_SCORE_SELECT, st);
-      kern<<<(unsigned)(units * ((sh.L + 63) / 64)), 256, tsm, st>>>(sh, q, w.mean, seq_lens, idx);
+      kern<<<(unsigned)(units * ((sh.L + 63) / 64)), 256, tsm, st>>>(sh, g, q, w.mean, seq_lens, idx);
       return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
     }
+    if (!g.plain) return BLOSSOM_ERR_UNSUPPORTED;  // (more than 128 blocks: the per-warp kernel scores selection blocks only)
     const size_t psm = (size_t)8 * (2 * sh.M + D) * sizeof(double) + (size_t)8 * sh.M + 16;
     if (psm > 48 * 1024 && cudaFuncSetAttribute(score_per_query_kernel<T, D>,
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm) != cudaSuccess)

@@ -48,7 +48,7 @@ def test_workspace_bytes(lib):
     assert n > 0 and n % 256 == 0
     assert binding.blossom_workspace_bytes(good(batch=8)) > n
     for bad in (dict(batch=0), dict(head_dim=48), dict(block_size=12), dict(top_k=0), dict(window=0),
-                dict(kv_heads=3), dict(kv_heads=0), dict(kv_strides=(4096, 2048, 31)), dict(causal=2), dict(causal=0, select_mode=1), dict(select_mode=2), dict(select_mode=1, cmp_block=16, cmp_stride=4), dict(dtype=7),
+                dict(kv_heads=3), dict(kv_heads=0), dict(kv_strides=(4096, 2048, 31)), dict(causal=2), dict(causal=0, select_mode=1), dict(select_mode=2), dict(select_mode=1, cmp_block=16, cmp_stride=4, seq_len=2048), dict(dtype=7),
                 dict(seq_len=8 * 1025), dict(strides=(4096, 2048, 33)), dict(sm_scale=-1.0),
                 dict(stis_mode=2), dict(stis_mode=-1), dict(stis_mode=1, stis_block=-3),
                 dict(cmp_block=12, cmp_stride=8), dict(cmp_block=16, cmp_stride=3), dict(cmp_block=-8)):
@@ -77,7 +77,7 @@ def test_argument_validation_precedes_any_launch(lib):
     assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, A + 64, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
     assert E.blossom_attn_fwd(p, A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes - 1, stream=0, check=False) == E.BLOSSOM_ERR_WORKSPACE
     # unsupported but legal requests
-    assert E.blossom_attn_fwd(good(select_mode=1, cmp_block=16, cmp_stride=4), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
+    assert E.blossom_attn_fwd(good(select_mode=1, cmp_block=16, cmp_stride=4, seq_len=2048), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
     assert E.blossom_attn_fwd(good(kv_heads=3), A, A, A, A, None, A, 0, A, A, A, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_INVALID_ARG
     assert E.blossom_select_blocks(good(head_dim=128), A, A, None, A, A, ws_bytes, stream=0, check=False) == E.BLOSSOM_ERR_UNSUPPORTED
     # one block more than the 1024 the lists are laid out for

@@ -221,6 +221,19 @@ def test_paper_default_configuration_in_one_call(runner, dtype, D):
     print(check_forward_backward(w, res))
 
 
+@pytest.mark.parametrize("dtype,D", [("fp32", 32), ("bf16", 32), ("bf16", 64)])
+def test_paper_default_configuration_with_its_selection_per_query_position(runner, dtype, D):
+    """The same configuration with the selection as the paper prints it (Eq. 13 per query
+    position, through the compression blocks and Eq. 11, shared by the heads of a group)."""
+    w = workloads.make("paper-exact", dtype, 5, 8, 200, D, 16, 4, 8, seed=37, std=0.7, kv_heads=2,
+                       stis_mode=1, stis_block=1)
+    w.cmp_block, w.cmp_stride, w.per_query = 32, 16, 1
+    w.seq_lens = np.asarray([200, 131, 33, 16, 0], dtype=np.int32)
+    _, res = run(runner, w)
+    assert res["idx"].shape == (5, 2, 200, 4) and res["dk"].shape == (5, 2, 200, D)
+    print(check_forward_backward(w, res))
+
+
 def test_explicit_scale_and_given_indices(runner):
     w = workloads.make("scale", "fp32", 2, 2, 96, 32, 16, 3, 20, seed=5)
     p, res = run(runner, w, sm_scale=0.37)
@@ -405,6 +418,17 @@ def test_config4_full_size_paper_options_together(runner):
     print(errs)
 
 
+def test_config4_full_size_paper_options_with_the_selection_per_query_position(runner):
+    """The headline shape with all of the paper's options and its per-position selection, as the
+    benchmark's --paper-options --per-query times it."""
+    w = workloads.config4(kv_heads=2)
+    w.cmp_block, w.cmp_stride, w.per_query = 128, 32, 1
+    w.stis_mode, w.stis_block, w.window = 1, 1, 8
+    errs, res = _whole_batch(runner, w)
+    print(errs)
+    assert res["idx"].shape == (w.B, 2, w.L, w.topk)
+
+
 def test_config2_full_size(runner):
     w = workloads.config2()
     errs, res = _whole_batch(runner, w)
@@ -586,14 +610,18 @@ def test_a_wait_that_cannot_complete_is_reported_and_the_context_stays_usable(ru
     (300, 64, 4, 2, 32, 4, 40, [300, 131], False),           # grouped heads share a per-position selection
     (257, 64, 2, 2, 64, 3, 8, None, True),                   # with the power-law short-term mask
     (1024, 64, 2, 2, 64, 8, 64, [1024, 700], False),
+    (300, 64, 4, 2, 32, 4, 40, [300, 131], "cmp64/16"),      # through overlapping compression blocks
+    (1000, 32, 2, 2, 16, 5, 30, [1000, 404], "cmp32/8"),     # 122 compression blocks: two chunks
 ])
 def test_selection_per_query_position(runner, dtype, L, D, H, Hkv, block, topk, window, lens, power_law):
     """select_mode 1 (Eq. 13 as the paper prints it: every query position keeps its own top-k
     blocks): indices, forward and backward against the oracle."""
     B = len(lens) if lens else 2
     w = workloads.make("per-query", dtype, B, H, L, D, block, topk, window, seed=59, kv_heads=Hkv if Hkv != H else 0,
-                       stis_mode=1 if power_law else 0)
+                       stis_mode=1 if power_law is True else 0)
     w.per_query = 1
+    if isinstance(power_law, str):
+        w.cmp_block, w.cmp_stride = (int(x) for x in power_law[3:].split("/"))
     if lens is not None:
         w.seq_lens = np.asarray(lens, dtype=np.int32)
     _, res = run(runner, w)
