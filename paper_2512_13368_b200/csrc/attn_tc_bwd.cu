@@ -155,7 +155,9 @@ __device__ __forceinline__ void dq_tile(const float (&sv)[16], const float (&dp)
   }
 }
 
-template <int D>
+// PLAIN (both kernels below): the causal mask and one selection per query block (the measured
+// path): the other modes' tests fold away at compile time.
+template <int D, bool PLAIN>
 __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
@@ -193,7 +195,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   uint8_t *g_tile = q_tile + C::kBigBytes;
   uint8_t *kv_tiles = g_tile + C::kBigBytes;
   uint8_t *meta = kv_tiles + STAGES * 2 * C::kSmallBytes;  // image built by tc_meta_kernel
-  const MetaLayout ml = meta_layout(nT, s.pq);
+  const bool causal = PLAIN || s.causal;
+  const int pq = PLAIN ? 0 : s.pq;
+  const MetaLayout ml = meta_layout(nT, pq);
   const uint8_t *selb = meta;
   const uint8_t *rowb = meta + ml.rows;  // (selection per query position) [128 rows][nT]
   const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
@@ -370,9 +374,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
         const int i = x >> 1, jt = list[i], f = lflags[i], p0 = jt * 64;
         uint64_t maskL = 0ull, maskS = 0ull;
         if (row_valid) {
-          const uint64_t mc = cols_le((s.causal ? t : s.L - 1) - p0) & cols_ge(pad0 - p0);
-          if (f & 1) maskL = mc & expand_block_bits(s.pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk);
-          if (f & 2) maskS = mc & st_key_cols(s, t, p0);
+          const uint64_t mc = cols_le((causal ? t : s.L - 1) - p0) & cols_ge(pad0 - p0);
+          if (f & 1) maskL = mc & expand_block_bits(pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk);
+          if (f & 2) maskS = mc & st_key_cols(s, t, p0, causal);
         }
         hL = (uint32_t)(maskL >> (32 * (x & 1) + 16 * half)) & 0xffffu;
         hS = (uint32_t)(maskS >> (32 * (x & 1) + 16 * half)) & 0xffffu;
@@ -503,7 +507,7 @@ __device__ __forceinline__ void dkdv_tile(const float (&sv)[16], const float (&d
   }
 }
 
-template <int D>
+template <int D, bool PLAIN>
 __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
@@ -539,7 +543,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
   uint8_t *v_tile = k_tile + C::kBigBytes;
   uint8_t *qg_tiles = v_tile + C::kBigBytes;  // [stage][Q, dO, row records]
   uint8_t *meta = qg_tiles + STAGES * kStageBytes;  // image built by tc_meta_kernel
-  const MetaLayout ml = meta_layout(nT, s.pq);
+  const bool causal = PLAIN || s.causal;
+  const int pq = PLAIN ? 0 : s.pq;
+  const MetaLayout ml = meta_layout(nT, pq);
   const uint64_t *inv64 = reinterpret_cast<const uint64_t *>(meta + ml.rows);  // (selection per query position) [8][nT]
   const uint8_t *invb = meta;                           // [8][nT] bytes: per key block, per query tile
   const uint16_t *list = reinterpret_cast<const uint16_t *>(meta + ml.list);
@@ -687,9 +693,9 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
       uint64_t maskL = 0ull, maskS = 0ull;
       if (cls2[0] == 8 || cls2[8] == 8) {  // a mixed half tile: per-lane column masks
         if (row_valid) {
-          const uint64_t mc = cols_ge((s.causal ? p : pad0) - t0) & cols_le(s.L - 1 - t0);
-          if (f & 1) maskL = mc & (s.pq ? inv64[g * nT + qt] : expand_block_bits(invb[g * nT + qt], s.Bk));
-          if (f & 2) maskS = mc & st_query_cols(s, p, t0);
+          const uint64_t mc = cols_ge((causal ? p : pad0) - t0) & cols_le(s.L - 1 - t0);
+          if (f & 1) maskL = mc & (pq ? inv64[g * nT + qt] : expand_block_bits(invb[g * nT + qt], s.Bk));
+          if (f & 2) maskS = mc & st_query_cols(s, p, t0, causal);
         }
       }
       mbar_wait(b_full + 8 * (i % STAGES), (i / STAGES) & 1, &abort_flag, 216);  // the row records have landed
@@ -798,8 +804,11 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   const size_t smem_dq = 1024 + 2 * C::kBigBytes + kDqStages * 2 * C::kSmallBytes + meta_bytes(nT, s.pq);
   const size_t smem_kv =
       1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT, s.pq);
-  if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
-      cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
+  const bool plain = s.causal && !s.pq;
+  auto kern_dq = plain ? bwd_dq_tc_kernel<D, true> : bwd_dq_tc_kernel<D, false>;
+  auto kern_kv = plain ? bwd_dkdv_tc_kernel<D, true> : bwd_dkdv_tc_kernel<D, false>;
+  if (cudaFuncSetAttribute(kern_dq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
+      cudaFuncSetAttribute(kern_kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, ws.kmeta, st, branches)) return rc;
   const float4 *rec = records ? records : ws.qstats;
@@ -812,14 +821,14 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   }
   {
     LaunchScope ls(K_BWD_DQ_TC, st);
-    bwd_dq_tc_kernel<D><<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
+    kern_dq<<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
                                                            tdq, rec, ws.dalpha,
                                                            ws.status_bwd, nT);
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
     const unsigned grid_k = (unsigned)nST * (unsigned)(s.B * s.Hkv);
-    bwd_dkdv_tc_kernel<D><<<grid_k, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
+    kern_kv<<<grid_k, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
                                                              rec, tdk, tdv, ws.status_bwd, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;

@@ -116,7 +116,9 @@ __device__ __forceinline__ uint4 load_row_chunk(const uint8_t *tile, int r, int 
   else return *reinterpret_cast<const uint4 *>(tile + r * 64 + ((ch ^ ((r >> 1) & 3)) << 4));
 }
 
-template <int D>
+// PLAIN: the causal mask and one selection per query block (the measured path): the other modes'
+// tests fold away at compile time.
+template <int D, bool PLAIN>
 __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
@@ -151,7 +153,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   uint8_t *kv_tiles = q_tile + C::kBigBytes;                  // [stage][K, V]
   uint8_t *sl = kv_tiles + STAGES * 2 * C::kSmallBytes;       // the long-term rows, staged when their phase ends
   uint8_t *meta = sl + C::kBigBytes;                          // image built by tc_meta_kernel
-  const MetaLayout ml = meta_layout(nT, s.pq);
+  const bool causal = PLAIN || s.causal;
+  const int pq = PLAIN ? 0 : s.pq;
+  const MetaLayout ml = meta_layout(nT, pq);
   const uint8_t *selb = meta;
   const uint8_t *rowb = meta + ml.rows;  // (selection per query position) [128 rows][nT]
   const uint16_t *items = reinterpret_cast<const uint16_t *>(meta + ml.items);  // [2 nT]
@@ -370,9 +374,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
       uint32_t hm = 0u;  // this thread's 32 keys of the tile that the row sees
       bool doB = cls == 1, fullB = cls == 1;
       if (cls == 2) {
-        if (row_ok && t >= pad0) {  // (a padded row sees nothing; under the causal mask the bounds below say so by themselves)
-          uint64_t mask = cols_le((s.causal ? t : s.L - 1) - p0) & cols_ge(pad0 - p0);
-          mask &= isL ? expand_block_bits(s.pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk) : st_key_cols(s, t, p0);
+        if (row_ok && (causal || t >= pad0)) {  // (a padded row sees nothing; under the causal mask the bounds below say so)
+          uint64_t mask = cols_le((causal ? t : s.L - 1) - p0) & cols_ge(pad0 - p0);
+          mask &= isL ? expand_block_bits(pq ? rowb[r * nT + jt] : selb[g * nT + jt], s.Bk) : st_key_cols(s, t, p0, causal);
           hm = (uint32_t)(mask >> (32 * grp));
         }
         doB = __any_sync(0xffffffffu, hm != 0u);
@@ -468,14 +472,14 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const size_t smem = 1024 + 2 * C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT, s.pq);
-  if (cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-      cudaSuccess)
+  auto kern = (s.causal && !s.pq) ? fwd_tc_kernel<D, true> : fwd_tc_kernel<D, false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
   if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, nullptr, st)) return rc;
   {
     LaunchScope ls(K_FWD_TC, st);
-    fwd_tc_kernel<D><<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, ws.qmeta,
+    kern<<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, ws.qmeta,
                                                      training, lse, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;

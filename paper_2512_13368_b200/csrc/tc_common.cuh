@@ -352,10 +352,11 @@ __device__ __forceinline__ uint64_t expand_block_bits(uint32_t bits, int bk) {
 
 // Short-term mask of Eq. 15 over the 64 keys p0 ... p0 + 63 for query t, without the causal and
 // the padding condition (the caller ANDs those): the window, and with the power-law mask the key
-// blocks at power-of-two block distances and the last block.
-__device__ __forceinline__ uint64_t st_key_cols(const Shape &s, int t, int p0) {
+// blocks at power-of-two block distances and the last block.  `causal` is the caller's (often
+// compile-time) copy of s.causal.
+__device__ __forceinline__ uint64_t st_key_cols(const Shape &s, int t, int p0, bool causal) {
   uint64_t m = cols_ge(t - s.window + 1 - p0);
-  if (!s.causal) m &= cols_le(t + s.window - 1 - p0);  // (without the causal mask the window has two sides)
+  if (!causal) m &= cols_le(t + s.window - 1 - p0);  // (without the causal mask the window has two sides)
   if (s.stis_mode) {
     m |= cols_ge(s.L - s.stis_blk - p0);
     const int bq = t / s.stis_blk;
@@ -364,7 +365,7 @@ __device__ __forceinline__ uint64_t st_key_cols(const Shape &s, int t, int p0) {
       if (a + s.stis_blk - 1 < p0) break;
       if (a <= p0 + 63) m |= cols_ge(a - p0) & cols_le(a + s.stis_blk - 1 - p0);
     }
-    if (!s.causal) {
+    if (!causal) {
       for (int d = 1;; d <<= 1) {  // and key block bq + d: later d lie further right
         const int a = (bq + d) * s.stis_blk;
         if (a > p0 + 63 || a >= s.L) break;
@@ -376,9 +377,9 @@ __device__ __forceinline__ uint64_t st_key_cols(const Shape &s, int t, int p0) {
 }
 // The same mask seen from key p over the 64 queries t0 ... t0 + 63 (again without causality and
 // padding).
-__device__ __forceinline__ uint64_t st_query_cols(const Shape &s, int p, int t0) {
+__device__ __forceinline__ uint64_t st_query_cols(const Shape &s, int p, int t0, bool causal) {
   uint64_t m = cols_le(p + s.window - 1 - t0);
-  if (!s.causal) m &= cols_ge(p - s.window + 1 - t0);
+  if (!causal) m &= cols_ge(p - s.window + 1 - t0);
   if (s.stis_mode) {
     if (p >= s.L - s.stis_blk) return ~0ull;
     const int bk = p / s.stis_blk;
@@ -387,7 +388,7 @@ __device__ __forceinline__ uint64_t st_query_cols(const Shape &s, int p, int t0)
       if (a > t0 + 63 || a >= s.L) break;
       if (a + s.stis_blk - 1 >= t0) m |= cols_ge(a - t0) & cols_le(a + s.stis_blk - 1 - t0);
     }
-    if (!s.causal) {
+    if (!causal) {
       for (int d = 1; d <= bk; d <<= 1) {  // and query block bk - d
         const int a = (bk - d) * s.stis_blk;
         if (a + s.stis_blk - 1 < t0) break;

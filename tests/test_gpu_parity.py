@@ -513,6 +513,53 @@ def test_certified_selection_on_random_small_block_shapes(runner):
         assert np.array_equal(fast, exact), (it, L, Bk, D, H, B, topk, dtype, std)
 
 
+def _random_option_workload(rng, it):
+    """A small bf16 / fp32 problem with a random legal combination of the options."""
+    Bk = int(rng.choice([16, 32, 64]))
+    D = int(rng.choice([32, 64]))
+    Hkv = int(rng.choice([1, 2]))
+    H = Hkv * int(rng.choice([1, 2]))
+    L = int(rng.integers(Bk + 1, 700))
+    topk, window = int(rng.integers(1, 7)), int(rng.integers(1, 90))
+    dtype = "bf16" if rng.random() < 0.8 else "fp32"
+    lens = None if rng.random() < 0.4 else (0, L)
+    power_law = rng.random() < 0.4
+    w = workloads.make(f"rand-options-{it}", dtype, 3, H, L, D, Bk, topk, window, seed=2000 + it, lengths=lens,
+                       kv_heads=Hkv if Hkv != H else 0, stis_mode=1 if power_law else 0,
+                       stis_block=int(rng.choice([1, 2, 4])) if power_law else 1)
+    w.causal = 0 if rng.random() < 0.3 else 1
+    if w.causal:
+        if rng.random() < 0.4:
+            w.per_query = 1
+        if rng.random() < 0.4:
+            s = int(rng.choice([x for x in (4, 8, 16, 32, 64) if Bk % x == 0]))
+            w.cmp_block, w.cmp_stride = s * int(rng.choice([1, 2, 4])), s
+            if w.per_query and ((L - w.cmp_block) // s + 1 > 128 or -(-L // Bk) > 128):
+                w.cmp_block = w.cmp_stride = 0
+    if rng.random() < 0.3:
+        w.gate_mode = 1
+        w.gate = (0.3 * rng.standard_normal((H, 2 * D + 1))).astype(np.float32)
+    if rng.random() < 0.3:
+        w.rope_theta = 10000.0
+    if rng.random() < 0.3:
+        w.phi_logits = rng.standard_normal(w.cmp_block or Bk).astype(np.float32)
+    return w
+
+
+def test_random_combinations_of_the_options(runner):
+    """Forty seeded problems with random shapes, lengths and legal combinations of the options
+    (power-law mask, compression blocks, grouped heads, per-position selection, pooled summaries,
+    input-dependent gate, no causal mask, rotary positions), each against the oracle."""
+    rng = np.random.default_rng(2024)
+    for it in range(40):
+        w = _random_option_workload(rng, it)
+        _, res = run(runner, w)
+        try:
+            check_forward_backward(w, res)
+        except AssertionError as e:
+            raise AssertionError(f"case {it}: {w}: {e}") from e
+
+
 # ------------------------------------------- what stands in for a memory checker on this path
 def _guarded(shape, dtype, fill, device, pad=4096):
     """A tensor carved out of a larger allocation with `pad` guard elements before and after it."""
