@@ -565,17 +565,23 @@ __global__ void __launch_bounds__(256) gate_grad_kernel(Shape s, const float *__
   }
 }
 
-// Gradient of F_o's parameters (input-dependent gate): per head, the per-query-block partial sums
-// added over batch entries and query blocks in a fixed order.  One block per head.
+// Gradient of F_o's parameters (input-dependent gate): the per-query-block partial sums added
+// over batch entries and query blocks in a fixed order.  One warp per (head, parameter): lane i
+// adds the entries i, i + 32, ... in ascending order, then a fixed shuffle tree joins the lanes.
 __global__ void __launch_bounds__(256) gate_param_grad_kernel(Shape s, const double *__restrict__ part,
                                                               float *__restrict__ dgate) {
-  const int h = blockIdx.x, GW = 2 * s.D + 1;
-  for (int d = threadIdx.x; d < GW; d += 256) {
-    double a = 0.0;
-    for (int n = 0; n < s.B; ++n)
-      for (int qb = 0; qb < s.M; ++qb) a += part[(((int64_t)n * s.H + h) * s.M + qb) * GW + d];
-    dgate[(int64_t)h * GW + d] = (float)a;
+  const int GW = 2 * s.D + 1;
+  const int w = (int)blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (w >= s.H * GW) return;
+  const int h = w / GW, d = w % GW, n_entries = s.B * s.M;
+  double a = 0.0;
+  for (int e = lane; e < n_entries; e += 32) {
+    const int n = e / s.M, qb = e % s.M;
+    a += part[(((int64_t)n * s.H + h) * s.M + qb) * GW + d];
   }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+  if (lane == 0) dgate[(int64_t)h * GW + d] = (float)a;
 }
 
 namespace {
@@ -631,7 +637,7 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
   }
   if (s.gate_mode) {
     LaunchScope ls(K_GATE_GRAD, st);
-    gate_param_grad_kernel<<<s.H, 256, 0, st>>>(s, ws.dgate_part, dgate);
+    gate_param_grad_kernel<<<(unsigned)((s.H * (2 * s.D + 1) + 7) / 8), 256, 0, st>>>(s, ws.dgate_part, dgate);
     return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
   }
   return launch_gate_grad(s, gate, ws, dgate, st);
@@ -642,7 +648,7 @@ int launch_bwd_t(const Shape &s, const T *q, const T *k, const T *v, const float
 int launch_gate_param_grad(const Shape &s, const Workspace &ws, float *dgate, cudaStream_t st) {
   {
     LaunchScope ls(K_GATE_GRAD, st);
-    gate_param_grad_kernel<<<s.H, 256, 0, st>>>(s, ws.dgate_part, dgate);
+    gate_param_grad_kernel<<<(unsigned)((s.H * (2 * s.D + 1) + 7) / 8), 256, 0, st>>>(s, ws.dgate_part, dgate);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }
