@@ -116,6 +116,14 @@ typedef struct {
                         * t * rope_theta^(-2i / D) at array position t, evaluated in double precision
                         * and rounded once to the storage type; the copies live in the workspace),
                         * and blossom_attn_bwd returns dq, dk with respect to the unrotated inputs  */
+  int32_t reuse_tile_lists; /* read by blossom_attn_bwd only.  0: the call builds the tile lists its
+                        * kernels walk from block_idx (one more launch).  1: the caller promises that
+                        * the last call on this workspace was a blossom_attn_fwd in training mode
+                        * (out_lt, out_st given) with the same params, seq_lens and block_idx contents:
+                        * that call has left the backward's lists in the workspace and they are used
+                        * as they are.  A broken promise gives wrong gradients, not a fault (lists of
+                        * another shape are never read: the shape is part of the promise).  Ignored
+                        * on the CUDA-core path and with gate_mode 1                               */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

@@ -109,7 +109,11 @@ class _BlossomAttention(torch.autograd.Function):
             dout = _like(q).copy_(dout)
         dq, dk, dv = _like(q), _like(k), _like(k)
         dgate = torch.empty(tuple(gate.shape), dtype=torch.float32, device=q.device)
-        binding.blossom_attn_bwd(ctx.params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
+        # the workspace is this call's own and its last user was the training forward above (or an
+        # earlier backward, which leaves the lists alone): the backward may reuse that call's tile lists
+        params = binding.blossom_params.from_buffer_copy(ctx.params)
+        params.reuse_tile_lists = 1
+        binding.blossom_attn_bwd(params, q, k, v, gate, ctx.seq_lens, idx, out_lt, out_st, lse,
                                  dout, dq, dk, dv, dgate, ctx.workspace)
         return (dq, dk, dv, dgate.to(ctx.gate_dtype)) + (None,) * 14
 

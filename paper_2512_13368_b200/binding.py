@@ -44,6 +44,7 @@ class blossom_params(ctypes.Structure):
         ("kv_stride_b", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64), ("kv_stride_l", ctypes.c_int64),
         ("phi_logits", ctypes.c_void_p), ("gate_mode", ctypes.c_int32),
         ("rope_theta", ctypes.c_float),
+        ("reuse_tile_lists", ctypes.c_int32),
     ]
 
 
@@ -124,7 +125,7 @@ def _stream(stream):
 def make_params(batch, heads, seq_len, head_dim, block_size, top_k, window, dtype, sm_scale=0.0,
                 strides=None, kv_heads=None, causal=1, select_mode=0, stis_mode=0,
                 stis_block=1, cmp_block=0, cmp_stride=0, kv_strides=None, phi_logits=None,
-                gate_mode=0, rope_theta=0.0) -> blossom_params:
+                gate_mode=0, rope_theta=0.0, reuse_tile_lists=0) -> blossom_params:
     """Fill a ``blossom_params``; ``strides`` = (stride_b, stride_h, stride_l) in elements,
     default contiguous [B, H, L, D].  ``phi_logits``: float32 device tensor (the caller keeps it
     alive) or None."""
@@ -136,7 +137,7 @@ def make_params(batch, heads, seq_len, head_dim, block_size, top_k, window, dtyp
                           int(strides[0]), int(strides[1]), int(strides[2]), int(stis_mode),
                           int(stis_block), int(cmp_block), int(cmp_stride),
                           *((0, 0, 0) if kv_strides is None else [int(x) for x in kv_strides]),
-                          _ptr(phi_logits), int(gate_mode), float(rope_theta))
+                          _ptr(phi_logits), int(gate_mode), float(rope_theta), int(reuse_tile_lists))
 
 
 def blossom_status_string(status) -> str:

@@ -164,6 +164,8 @@ static int make_shape(const blossom_params *p, Shape *out) {
   if (!(p->rope_theta >= 0.f) || isinf(p->rope_theta) || (p->rope_theta > 0.f && p->rope_theta < 1.f))
     return BLOSSOM_ERR_INVALID_ARG;
   s.rope_theta = (double)p->rope_theta;
+  if (p->reuse_tile_lists < 0 || p->reuse_tile_lists > 1) return BLOSSOM_ERR_INVALID_ARG;
+  s.reuse_lists = p->reuse_tile_lists;
   s.esz = p->dtype == BLOSSOM_DTYPE_BF16 ? 2 : 4;
   s.pq = p->select_mode;
   s.causal = p->causal;

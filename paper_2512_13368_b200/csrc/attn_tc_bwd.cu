@@ -810,7 +810,8 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   if (cudaFuncSetAttribute(kern_dq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(kern_kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
-  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, ws.kmeta, st, branches)) return rc;
+  if (!(s.reuse_lists && branches == 3 && !records))  // (the passes of the input-dependent gate build their own)
+    if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, ws.kmeta, st, branches)) return rc;
   const float4 *rec = records ? records : ws.qstats;
   if (!records) {
     LaunchScope ls(K_BWD_PREP, st);

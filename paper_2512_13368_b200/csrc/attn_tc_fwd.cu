@@ -476,7 +476,9 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
-  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, nullptr, st)) return rc;
+  // A training call also builds the backward's tile lists (the same launch: one warp per image):
+  // a backward call told to reuse them (blossom_params::reuse_tile_lists) then builds none.
+  if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, training ? ws.kmeta : nullptr, st, 3, 1)) return rc;
   {
     LaunchScope ls(K_FWD_TC, st);
     kern<<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, ws.qmeta,

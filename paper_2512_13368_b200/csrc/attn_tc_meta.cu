@@ -34,7 +34,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                                                                   const int32_t *__restrict__ idx,
                                                                   uint8_t *__restrict__ qmeta,
                                                                   uint8_t *__restrict__ kmeta, int nT,
-                                                                  int n_query_ctas, int n_images, int branches) {
+                                                                  int n_query_ctas, int n_images, int branches,
+                                                                  int with_fwd) {
   extern __shared__ __align__(16) uint8_t meta_all[];
   const MetaLayout ml = meta_layout(nT, s.pq);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     __syncwarp();
     const int gh = G / 2;
     if (lane == 0) counts[0] = nv;
-    if (!kmeta) {  // ---- forward-only call: the forward's items and their classes ----
+    if (with_fwd) {  // ---- the forward's items and their classes ----
     // Long-term items: the tiles both 64-row halves of the CTA need, then alternately a tile only
     // rows 0..63 need and a tile only rows 64..127 need.  A softmax warp may run ahead of the
     // slowest one, so with alternating items both pairs of warps have work at once.
@@ -197,7 +198,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
       icls[e] = (uint8_t)cls;
     }
-    }  // forward-only
+    }  // the forward's part
     __syncwarp();
     // The dQ kernel walks `list` itself (a tile serves both branches there).  Same idea as above:
     // tiles both 64-row halves need first, then alternately a tile only rows 0..63 need and one
@@ -388,7 +389,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
 }  // namespace
 
 int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
-                   uint8_t *kmeta, cudaStream_t st, int branches) {
+                   uint8_t *kmeta, cudaStream_t st, int branches, int with_fwd) {
+  if (with_fwd < 0) with_fwd = kmeta == nullptr;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const int nq = nST * s.B * s.H, n_images = kmeta ? nq + nST * s.B * s.Hkv : nq;
   const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT, s.pq) + ((3 * nT + 15) / 16) * 16);
@@ -398,7 +400,7 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
   {
     LaunchScope ls(K_TC_META, st);
     tc_meta_kernel<<<(unsigned)((n_images + kMetaWarps - 1) / kMetaWarps), kMetaWarps * 32, smem, st>>>(
-        s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images, branches);
+        s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images, branches, with_fwd);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -24,6 +24,7 @@ struct Shape {
   int causal;             // 1: causal mask (default); 0: bidirectional (CUDA-core kernels)
   int gate_mode;          // 0: one gate weight per head from two logits; 1: Eq. 18's input-dependent gate
   const float *phi;       // logits of the learnable block summary (Eq. 9) or nullptr = the mean
+  int reuse_lists;        // backward: the tile lists of the preceding training forward are in the workspace
   int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
 };
 

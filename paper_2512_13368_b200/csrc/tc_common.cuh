@@ -491,8 +491,11 @@ int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_
 // Builds the bookkeeping of every query-major CTA (forward, dQ) into qmeta and, if kmeta is not
 // null, of every key-major CTA (dK/dV) into kmeta: meta_bytes(nT) bytes per CTA, CTA-major.
 // branches: bit 0 long-term, bit 1 short-term: tiles that only the other branch needs are left out.
+// with_fwd: 1 = the query-major images carry the forward's items, 0 = not, -1 = only when no
+// key-major images are asked for (a forward call builds the forward's part, a backward call the
+// rest; a training forward may build everything at once for a backward that reuses it).
 int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, uint8_t *qmeta,
-                   uint8_t *kmeta, cudaStream_t st, int branches = 3);
+                   uint8_t *kmeta, cudaStream_t st, int branches = 3, int with_fwd = -1);
 
 // per-file launchers behind launch_fwd_tc / launch_bwd_tc
 template <int D>

@@ -36,6 +36,10 @@ class DeviceProblem:
                                           select_mode=w.per_query, phi_logits=self.phi,
                                           gate_mode=getattr(w, "gate_mode", 0), causal=getattr(w, "causal", 1),
                                           rope_theta=getattr(w, "rope_theta", 0.0))
+        # the backward of a step follows its training forward on the same workspace: it reuses the
+        # tile lists that forward left there
+        self.params_bwd = binding.blossom_params.from_buffer_copy(self.params)
+        self.params_bwd.reuse_tile_lists = 1
         self.alloc_outputs(training)
 
     def alloc_outputs(self, training=True):
@@ -67,8 +71,8 @@ class DeviceProblem:
                                  self.idx, int(idx_is_input), self.out, self.out_lt, self.out_st,
                                  self.lse, self.workspace, stream=stream)
 
-    def backward(self, stream=None):
-        binding.blossom_attn_bwd(self.params, self.q, self.k, self.v, self.gate, self.seq_lens,
+    def backward(self, stream=None, reuse_tile_lists=True):
+        binding.blossom_attn_bwd(self.params_bwd if reuse_tile_lists else self.params, self.q, self.k, self.v, self.gate, self.seq_lens,
                                  self.idx, self.out_lt, self.out_st, self.lse, self.dout, self.dq,
                                  self.dk, self.dv, self.dgate, self.workspace, stream=stream)
 

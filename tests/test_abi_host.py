@@ -98,8 +98,8 @@ def test_argument_validation_precedes_any_launch(lib):
 def test_params_struct_layout_matches_header():
     # 12 x 4-byte fields, three int64 strides, the two short-term mask fields, the two
     # compression-block fields, three int64 key/value strides and the pointer to the summary
-    # logits, the gate mode: 128 bytes with natural alignment
-    assert ctypes.sizeof(binding.blossom_params) == 128
+    # logits, the gate mode, the rotary base, the tile-list promise: 136 bytes with natural alignment
+    assert ctypes.sizeof(binding.blossom_params) == 136
     assert binding.blossom_params.phi_logits.offset == 112 and binding.blossom_params.gate_mode.offset == 120
     assert binding.blossom_params.kv_stride_b.offset == 88
     assert binding.blossom_params.cmp_block.offset == 80 and binding.blossom_params.cmp_stride.offset == 84

@@ -268,6 +268,28 @@ def test_inference_mode_and_select_only(runner):
     assert np.array_equal(q.results()["idx"], res["idx"])
 
 
+@pytest.mark.parametrize("opts", [{}, {"kv_heads": 2}, {"per_query": 1}, {"causal": 0}])
+def test_backward_on_the_forward_s_tile_lists_gives_the_same_bits(runner, opts):
+    """reuse_tile_lists = 1: a backward call that follows a training forward on the same workspace
+    walks the lists that forward built; the gradients are those of a backward that builds its own,
+    bit for bit."""
+    w = workloads.make("reuse-lists", "bf16", 3, 4, 900, 64, 32, 5, 70, seed=89, lengths=(200, 900),
+                       kv_heads=opts.get("kv_heads", 0))
+    w.per_query, w.causal = opts.get("per_query", 0), opts.get("causal", 1)
+    p = runner.DeviceProblem(w)
+    p.forward()
+    p.backward(reuse_tile_lists=False)
+    own = p.results()
+    for t in (p.dq, p.dk, p.dv, p.dgate):
+        t.fill_(7.0)
+    p.forward()
+    p.backward(reuse_tile_lists=True)
+    reused = p.results()
+    for key in ("dq", "dk", "dv", "dgate"):
+        assert np.array_equal(own[key], reused[key]), key
+    print(check_forward_backward(w, reused))
+
+
 def test_host_pipeline_returns_the_device_resident_results(runner):
     """Steps streamed from and to pinned host memory over alternating device slots give, step
     after step, the bits of a device-resident step."""
