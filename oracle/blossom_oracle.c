@@ -23,7 +23,8 @@
  *                               (summed probabilities) or per query position (as printed:
  *                               blossom_oracle_select_pq)
  *   overlapping blocks   Eq. 8 with l, s != Bk and the score remap of Eq. 11
- *                               (blossom_oracle_select_cmp)
+ *                               (blossom_oracle_select_cmp; per query position:
+ *                               blossom_oracle_select_pq_cmp)
  *   selected-KV attention Eq. 14 + Eq. 16 (via Eq. 1 with the causal mask)
  *   window attention     Eq. 15 first case (|i-j| < w), causal side, Eq. 17
  *   power-law mask       Eq. 15 all three cases (stis_mode 1), causal side:
@@ -38,8 +39,11 @@
  * Eq. 1, softmax/causality invariants, reductions to dense causal attention,
  * constructed selections with known answers, an independent numpy scorer,
  * finite differences, and Table 5's key-budget closed form.  The readings of
- * the paper that no printed value pins (selection per query block, phi = mean,
- * scalar gate, own block always selected) are "parity unpinned by the paper".
+ * the paper that no printed value pins (selection per query block, phi = mean
+ * or a softmax pooling, scalar gate or one-layer F_o, own block always
+ * selected, which compression blocks a position may score) are "parity
+ * unpinned by the paper": the pins above fix the arithmetic of each reading,
+ * not the choice of the reading.
  *
  * Layout: q, k, v, out*, dout, dq, dk, dv are contiguous [B][H][L][D] doubles;
  * lse is [2][B][H][L] (0 = long-term branch, 1 = short-term branch), natural
