@@ -367,6 +367,10 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
         tc_fence_after();
         merge(true, false);
         tc_fence_before();
+        // Both groups read both accumulators in the merge, and the first product of the next phase
+        // overwrites an accumulator as soon as ITS group has stored the next probabilities: no
+        // warp may go on before every warp has read.
+        named_bar_sync(3, kSoftmaxWarps * 32);
         m = -INFINITY;
         l = 0.f;
         acc = 0;

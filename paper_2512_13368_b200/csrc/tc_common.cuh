@@ -350,6 +350,9 @@ __device__ __forceinline__ uint64_t expand_block_bits(uint32_t bits, int bk) {
   return m;
 }
 
+// the smallest power of two >= x (1 for x <= 1)
+__device__ __forceinline__ int pow2_at_least(int x) { return x <= 1 ? 1 : 1 << (32 - __clz(x - 1)); }
+
 // Short-term mask of Eq. 15 over the 64 keys p0 ... p0 + 63 for query t, without the causal and
 // the padding condition (the caller ANDs those): the window, and with the power-law mask the key
 // blocks at power-of-two block distances and the last block.  `causal` is the caller's (often
@@ -360,13 +363,17 @@ __device__ __forceinline__ uint64_t st_key_cols(const Shape &s, int t, int p0, b
   if (s.stis_mode) {
     m |= cols_ge(s.L - s.stis_blk - p0);
     const int bq = t / s.stis_blk;
-    for (int d = 1; d <= bq; d <<= 1) {  // key block bq - d: later d lie further left
+    // key block bq - d, d a power of two: later d lie further left.  The walk starts at the first d
+    // that can reach the tile from the right, the smallest power of two >= bq - (last block of the
+    // tile), instead of at 1: a far tile then costs one or two steps, not log2 of its distance.
+    const int dmin = bq - (p0 + 63) / s.stis_blk;
+    for (int d = pow2_at_least(dmin); d <= bq; d <<= 1) {
       const int a = (bq - d) * s.stis_blk;
       if (a + s.stis_blk - 1 < p0) break;
       if (a <= p0 + 63) m |= cols_ge(a - p0) & cols_le(a + s.stis_blk - 1 - p0);
     }
     if (!causal) {
-      for (int d = 1;; d <<= 1) {  // and key block bq + d: later d lie further right
+      for (int d = pow2_at_least(p0 / s.stis_blk - bq);; d <<= 1) {  // and key block bq + d: later d lie further right
         const int a = (bq + d) * s.stis_blk;
         if (a > p0 + 63 || a >= s.L) break;
         if (a + s.stis_blk - 1 >= p0) m |= cols_ge(a - p0) & cols_le(a + s.stis_blk - 1 - p0);
@@ -383,13 +390,13 @@ __device__ __forceinline__ uint64_t st_query_cols(const Shape &s, int p, int t0,
   if (s.stis_mode) {
     if (p >= s.L - s.stis_blk) return ~0ull;
     const int bk = p / s.stis_blk;
-    for (int d = 1;; d <<= 1) {  // query block bk + d: later d lie further right
+    for (int d = pow2_at_least(t0 / s.stis_blk - bk);; d <<= 1) {  // query block bk + d: later d lie further right
       const int a = (bk + d) * s.stis_blk;
       if (a > t0 + 63 || a >= s.L) break;
       if (a + s.stis_blk - 1 >= t0) m |= cols_ge(a - t0) & cols_le(a + s.stis_blk - 1 - t0);
     }
     if (!causal) {
-      for (int d = 1; d <= bk; d <<= 1) {  // and query block bk - d
+      for (int d = pow2_at_least(bk - (t0 + 63) / s.stis_blk); d <= bk; d <<= 1) {  // and query block bk - d
         const int a = (bk - d) * s.stis_blk;
         if (a + s.stis_blk - 1 < t0) break;
         if (a <= t0 + 63) m |= cols_ge(a - t0) & cols_le(a + s.stis_blk - 1 - t0);

@@ -3,6 +3,8 @@ workspace with PyTorch, call the library, hand results back.  No arithmetic of t
 happens here."""
 from __future__ import annotations
 
+import os
+
 import numpy as np
 import torch
 
@@ -60,6 +62,14 @@ class DeviceProblem:
         if nbytes == 0:
             raise binding.BlossomError(binding.BLOSSOM_ERR_UNSUPPORTED, "blossom_workspace_bytes")
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        if os.environ.get("BLOSSOM_POISON_BUFFERS", "0") not in ("", "0"):
+            # debugging aid: every output and the workspace start as 0xFF bytes (NaN in bf16 and
+            # fp32, -1 as int32), so that a read of memory nobody has written shows in the results
+            # instead of finding the still-correct leftovers of an earlier, identical run
+            for t in (self.idx, self.out, self.out_lt, self.out_st, self.lse, self.dq, self.dk, self.dv,
+                      self.dgate, self.workspace):
+                if t is not None:
+                    t.view(torch.uint8).fill_(0xFF)
 
     # -- calls ---------------------------------------------------------------------------
     def select(self, stream=None):
