@@ -121,12 +121,19 @@ __device__ __forceinline__ bool st_visible(const Shape &s, int t, int p) {
   const int bd = abs(t / s.stis_blk - p / s.stis_blk);
   return (bd >= 1 && (bd & (bd - 1)) == 0) || p >= s.L - s.stis_blk;
 }
-// May some query in [t0, t1] see some key in [p0, p1] (p0 <= t1) through the short-term branch?
+// May some query in [t0, t1] see some key in [p0, p1] (p0 <= t1 under the causal mask) through the short-term branch?
 // Exact for the window; for the power-law mask a superset (any power of two inside the range of
 // block distances counts), which only costs a visit: st_visible decides every pair.
 __device__ __forceinline__ bool st_ranges_touch(const Shape &s, int t0, int t1, int p0, int p1) {
-  if (!s.causal)  // keys on both sides: exact for the window, every range for the power-law mask
-    return s.stis_mode != 0 || (t0 - p1 < s.window && p0 - t1 < s.window);
+  if (!s.causal) {  // keys on both sides of the queries
+    if (t0 - p1 < s.window && p0 - t1 < s.window) return true;
+    if (s.stis_mode == 0) return false;
+    if (p1 >= s.L - s.stis_blk) return true;
+    // is a power of two among the block distances of keys before the queries, or of keys after?
+    const int bq0 = t0 / s.stis_blk, bq1 = t1 / s.stis_blk, bk0 = p0 / s.stis_blk, bk1 = p1 / s.stis_blk;
+    const int lmax = bq1 - bk0, lmin = max(1, bq0 - bk1), rmax = bk1 - bq0, rmin = max(1, bk0 - bq1);
+    return (lmax >= lmin && (1 << (31 - __clz(lmax))) >= lmin) || (rmax >= rmin && (1 << (31 - __clz(rmax))) >= rmin);
+  }
   if (t0 - p1 < s.window) return true;
   if (s.stis_mode == 0) return false;
   if (p1 >= s.L - s.stis_blk) return true;
