@@ -157,7 +157,9 @@ __device__ __forceinline__ void dq_tile(const float (&sv)[16], const float (&dp)
 
 // PLAIN (both kernels below): the causal mask and one selection per query block (the measured
 // path): the other modes' tests fold away at compile time.
-template <int D, bool PLAIN>
+// PACK (dQ kernel): rows 0..63 and 64..127 of the CTA are the same 64 positions of two query heads
+// with a common key/value head, as in the forward kernel.
+template <int D, bool PLAIN, bool PACK>
 __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmg, Shape s,
@@ -179,14 +181,15 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
   // long rows first, tile-major: every unit's last tile, then every unit's last but one, ...
-  const int nU = s.B * s.H;
-  const int st = nST - 1 - (int)(blockIdx.x / nU);
-  const int u = (int)(blockIdx.x % nU), n = u / s.H, h = u % s.H;
+  // (PACK: a unit is a pair of heads, a tile 64 positions; h = the pair's first head)
+  const int nU = PACK ? s.B * (s.H / 2) : s.B * s.H, nQT = PACK ? nT : nST;
+  const int st = nQT - 1 - (int)(blockIdx.x / nU);
+  const int u = (int)(blockIdx.x % nU);
+  const int n = PACK ? u / (s.H / 2) : u / s.H, h = PACK ? 2 * (u % (s.H / 2)) : u % s.H;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
-  const int row0 = st * 128;
-  const int G = 128 / s.Bk;
+  const int row0 = PACK ? st * 64 : st * 128;
   const int Lpad = nT * 64;
 
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -231,7 +234,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     mbar_fence_init();
     // the CTA's tile lists and its resident tiles
     mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
-    bulk_load(smem_u32(meta), qmeta + ((size_t)u * nST + (nST - 1 - st)) * ml.bytes, (uint32_t)ml.bytes, b_meta);
+    bulk_load(smem_u32(meta), qmeta + ((size_t)u * nQT + (nQT - 1 - st)) * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, 2 * C::kBigBytes);
     tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
     tma_load_4d(smem_u32(g_tile), &tmg, b_res, 0, row0, h, n);
@@ -329,14 +332,16 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   } else {
     setmaxnreg_inc<kKvComputeRegs>();
     const int quarter = warp & 3, half = warp >> 2;
-    const int r = quarter * 32 + lane, t = row0 + r, g = r / s.Bk;
+    const int r = quarter * 32 + lane, t = PACK ? row0 + (r & 63) : row0 + r, g = r / s.Bk;
+    const int hr = PACK ? h + (r >> 6) : h;  // this row's head
     const bool row_ok = t < s.L, row_valid = row_ok && t >= pad0;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
+    const float alpha = gate_alpha(gate, hr), beta = 1.f - alpha;
     // this row's record from the pre-pass: nl = -(lse * log2e - log2 weight), nD = -Delta
     float nlL = 0.f, nlS = 0.f, nDL = 0.f, nDS = 0.f;
     if (row_valid) {
-      const float *rec = reinterpret_cast<const float *>(qstats) + ((int64_t)u * Lpad + (t & ~1)) * 4 + (t & 1);
+      const float *rec =
+          reinterpret_cast<const float *>(qstats) + (((int64_t)n * s.H + hr) * Lpad + (t & ~1)) * 4 + (t & 1);
       nlL = rec[0];
       nDL = rec[2];
       nlS = rec[4];
@@ -455,12 +460,25 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
   }
   tc_fence_before();
   __syncthreads();
-  // d alpha partial of this CTA -> first query-block slot of the super-tile, zeros in the rest
+  // d alpha partial of this CTA -> first query-block slot of its rows, zeros in the rest
+  // (PACK: one partial per head, from the warps of that head's 64 rows)
   if (tid == 0) {
-    double a = 0.0;
-    for (int i = 0; i < kComputeWarps; ++i) a += red[i];  // fixed order
-    for (int gq = 0; gq < G; ++gq)
-      if (st * G + gq < s.M) dalpha_part[(int64_t)u * s.M + st * G + gq] = gq == 0 ? a : 0.0;
+    if (PACK) {
+      const int nb = 64 / s.Bk;
+      for (int hh = 0; hh < 2; ++hh) {
+        double a = 0.0;
+        for (int i = 0; i < kComputeWarps; ++i)
+          if (((i & 3) >> 1) == hh) a += red[i];  // fixed order
+        for (int gq = 0; gq < nb; ++gq)
+          if (st * nb + gq < s.M) dalpha_part[((int64_t)n * s.H + h + hh) * s.M + st * nb + gq] = gq == 0 ? a : 0.0;
+      }
+    } else {
+      const int G = 128 / s.Bk;
+      double a = 0.0;
+      for (int i = 0; i < kComputeWarps; ++i) a += red[i];  // fixed order
+      for (int gq = 0; gq < G; ++gq)
+        if (st * G + gq < s.M) dalpha_part[(int64_t)u * s.M + st * G + gq] = gq == 0 ? a : 0.0;
+    }
   }
   if (nvis == 0 && tid == 0) mbar_wait(b_res, 0, &abort_flag, 221);  // no load may outlive the CTA
   finish(warp, tmem_base, kBwdTmemCols, &abort_flag, status);
@@ -792,11 +810,13 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   typedef __nv_bfloat16 bf;
   using C = Cfg<D>;
   CUtensorMap q128, k64, v64, g128, q64, k128, v128, g64, tdq, tdk, tdv;
-  if (make_tensor_map(&q128, q, s, 128) || make_tensor_map(&k64, k, s, 64, true) ||
-      make_tensor_map(&v64, v, s, 64, true) || make_tensor_map(&g128, dout, s, 128) ||
+  // (head-packed dQ kernel: a query-side box is 64 positions of two heads)
+  const int qrows = s.pack ? 64 : 128, qheads = s.pack ? 2 : 1;
+  if (make_tensor_map(&q128, q, s, qrows, false, qheads) || make_tensor_map(&k64, k, s, 64, true) ||
+      make_tensor_map(&v64, v, s, 64, true) || make_tensor_map(&g128, dout, s, qrows, false, qheads) ||
       make_tensor_map(&q64, q, s, 64) || make_tensor_map(&k128, k, s, 128, true) ||
       make_tensor_map(&v128, v, s, 128, true) || make_tensor_map(&g64, dout, s, 64) ||
-      make_tensor_map(&tdq, dq, s, 128) || make_tensor_map(&tdk, dk, s, 128, true) ||
+      make_tensor_map(&tdq, dq, s, qrows, false, qheads) || make_tensor_map(&tdk, dk, s, 128, true) ||
       make_tensor_map(&tdv, dv, s, 128, true))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
@@ -805,7 +825,8 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   const size_t smem_kv =
       1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT, s.pq);
   const bool plain = s.causal && !s.pq;
-  auto kern_dq = plain ? bwd_dq_tc_kernel<D, true> : bwd_dq_tc_kernel<D, false>;
+  auto kern_dq = s.pack ? (s.causal ? bwd_dq_tc_kernel<D, true, true> : bwd_dq_tc_kernel<D, false, true>)
+                        : (plain ? bwd_dq_tc_kernel<D, true, false> : bwd_dq_tc_kernel<D, false, false>);
   auto kern_kv = plain ? bwd_dkdv_tc_kernel<D, true> : bwd_dkdv_tc_kernel<D, false>;
   if (cudaFuncSetAttribute(kern_dq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||
       cudaFuncSetAttribute(kern_kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv) != cudaSuccess)
@@ -822,7 +843,8 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   }
   {
     LaunchScope ls(K_BWD_DQ_TC, st);
-    kern_dq<<<grid, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
+    const unsigned grid_q = s.pack ? (unsigned)nT * (unsigned)(s.B * (s.H / 2)) : grid;
+    kern_dq<<<grid_q, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
                                                            tdq, rec, ws.dalpha,
                                                            ws.status_bwd, nT);
   }

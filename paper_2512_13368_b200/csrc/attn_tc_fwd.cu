@@ -118,7 +118,10 @@ __device__ __forceinline__ uint4 load_row_chunk(const uint8_t *tile, int r, int 
 
 // PLAIN: the causal mask and one selection per query block (the measured path): the other modes'
 // tests fold away at compile time.
-template <int D, bool PLAIN>
+// PACK: rows 0..63 and 64..127 of the CTA are the same 64 positions of two query heads with a common
+// key/value head: by Eq. 12 they selected the same blocks and their windows reach the same tiles,
+// so every tile the CTA loads has work for all its rows.
+template <int D, bool PLAIN, bool PACK>
 __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
     const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
@@ -139,13 +142,15 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nST = (s.L + 127) >> 7;
   // long rows first, tile-major: every unit's last tile, then every unit's last but one, ...
-  const int nU = s.B * s.H;
-  const int st = nST - 1 - (int)(blockIdx.x / nU);
-  const int u = (int)(blockIdx.x % nU), n = u / s.H, h = u % s.H;
+  // (PACK: a unit is a pair of heads, a tile 64 positions; h = the pair's first head)
+  const int nU = PACK ? s.B * (s.H / 2) : s.B * s.H, nQT = PACK ? nT : nST;
+  const int st = nQT - 1 - (int)(blockIdx.x / nU);
+  const int u = (int)(blockIdx.x % nU);
+  const int n = PACK ? u / (s.H / 2) : u / s.H, h = PACK ? 2 * (u % (s.H / 2)) : u % s.H;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
-  const int row0 = st * 128;
+  const int row0 = PACK ? st * 64 : st * 128;
 
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t *tiles = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
@@ -187,7 +192,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     mbar_fence_init();
     // the CTA's tile lists and its query tile
     mbar_expect_tx(b_meta, (uint32_t)ml.bytes);
-    bulk_load(smem_u32(meta), qmeta + ((size_t)u * nST + (nST - 1 - st)) * ml.bytes, (uint32_t)ml.bytes, b_meta);
+    bulk_load(smem_u32(meta), qmeta + ((size_t)u * nQT + (nQT - 1 - st)) * ml.bytes, (uint32_t)ml.bytes, b_meta);
     mbar_expect_tx(b_res, C::kBigBytes);
     tma_load_4d(smem_u32(q_tile), &tmq, b_res, 0, row0, h, n);
   }
@@ -277,7 +282,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     // ================================ softmax =================================
     setmaxnreg_inc<kSoftmaxRegs>();
     const int quarter = warp & 3, grp = warp >> 2;  // TMEM lane quarter; key half of every tile
-    const int r = quarter * 32 + lane, t = row0 + r, g = r / s.Bk;
+    const int r = quarter * 32 + lane, t = PACK ? row0 + (r & 63) : row0 + r, g = r / s.Bk;
+    const int hr = PACK ? h + (r >> 6) : h;  // this row's head
     const bool row_ok = t < s.L;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const uint32_t acc_own = (grp ? tmem_ob : tmem_oa) + lane_off;
@@ -286,7 +292,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     bool haveL = false, haveS = false;
     int acc = 0;  // the current phase has written the accumulators
     const float sc2 = s.scale * kLog2e;
-    const float alpha = gate_alpha(gate, h), beta = 1.f - alpha;
+    const float alpha = gate_alpha(gate, hr), beta = 1.f - alpha;
     int jt_n = nI > 0 ? items[0] : 0, cls_n = nI > 0 ? icls[quarter] : 0;
     uint8_t *so = kv_tiles, *ss = so + C::kBigBytes;  // staging of out / out_st (the K/V stages, free by then)
 
@@ -452,8 +458,9 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     }
     if (grp == 0 && row_ok && lse) {
       const int64_t BHL = (int64_t)s.B * s.H * s.L;
-      lse[(int64_t)u * s.L + t] = haveL ? lseL : 0.f;
-      lse[BHL + (int64_t)u * s.L + t] = haveS ? lseS : 0.f;
+      const int64_t row = ((int64_t)n * s.H + hr) * s.L + t;
+      lse[row] = haveL ? lseL : 0.f;
+      lse[BHL + row] = haveS ? lseS : 0.f;
     }
   }
   if (nI == 0 && tid == 0) mbar_wait(b_res, 0, &abort_flag, 112);  // no load may outlive the CTA
@@ -469,17 +476,20 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   using C = Cfg<D>;
   CUtensorMap tq, tk, tv, to, tol, tos;
   const int training = out_lt != nullptr;
-  if (make_tensor_map(&tq, q, s, 128) || make_tensor_map(&tk, k, s, 64, true) ||
-      make_tensor_map(&tv, v, s, 64, true) ||
-      make_tensor_map(&to, out, s, 128) || make_tensor_map(&tol, training ? out_lt : out, s, 128) ||
-      make_tensor_map(&tos, training ? out_st : out, s, 128))
+  // (head-packed: a query-side box is 64 positions of two heads)
+  const int qrows = s.pack ? 64 : 128, qheads = s.pack ? 2 : 1;
+  if (make_tensor_map(&tq, q, s, qrows, false, qheads) || make_tensor_map(&tk, k, s, 64, true) ||
+      make_tensor_map(&tv, v, s, 64, true) || make_tensor_map(&to, out, s, qrows, false, qheads) ||
+      make_tensor_map(&tol, training ? out_lt : out, s, qrows, false, qheads) ||
+      make_tensor_map(&tos, training ? out_st : out, s, qrows, false, qheads))
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const size_t smem = 1024 + 2 * C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT, s.pq);
-  auto kern = (s.causal && !s.pq) ? fwd_tc_kernel<D, true> : fwd_tc_kernel<D, false>;
+  auto kern = s.pack ? (s.causal ? fwd_tc_kernel<D, true, true> : fwd_tc_kernel<D, false, true>)
+                     : ((s.causal && !s.pq) ? fwd_tc_kernel<D, true, false> : fwd_tc_kernel<D, false, false>);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
-  const unsigned grid = (unsigned)nST * (unsigned)(s.B * s.H);
+  const unsigned grid = s.pack ? (unsigned)nT * (unsigned)(s.B * (s.H / 2)) : (unsigned)nST * (unsigned)(s.B * s.H);
   // A training call also builds the backward's tile lists (the same launch: one warp per image):
   // a backward call told to reuse them (blossom_params::reuse_tile_lists) then builds none.
   if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, training ? ws.kmeta : nullptr, st, 3, 1)) return rc;

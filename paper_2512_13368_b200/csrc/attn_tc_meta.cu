@@ -16,6 +16,9 @@
 //                             class of every (item, softmax warp)
 //   jcls[nT][2][8]            (dQ) class of every (listed tile, half tile, compute warp)
 //   counts                    {tiles on the list, long-term items, short-term items}
+// Head-packed variant (Shape::pack): the CTA's rows 0..63 and 64..127 are the same 64 positions of
+// two query heads with a common key/value head, so both halves have the same selection bytes and
+// every listed tile concerns both.
 // Key-major image (dK/dV kernel): [8][nT] bytes: bit c of byte (g, qt): query block
 // qt * (64 / Bk) + c selected key block g of the CTA; list / flags of the 64-query tiles that
 // visit the CTA's keys; jcls[nT][2][8] class of every (listed tile, half tile, compute warp);
@@ -48,8 +51,11 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   const int cta = key_major ? image - n_query_ctas : image;
   // query-major CTAs count (batch, query head) pairs, key-major CTAs (batch, key/value head) pairs;
   // uk = the (batch, key/value head) pair whose selection the image is built from
-  const int u = cta / nST, n = key_major ? u / s.Hkv : u / s.H;
-  const int uk = key_major ? u : n * s.Hkv + (u % s.H) / s.G;
+  // (head-packed query-major CTAs count (batch, pair of query heads) pairs, one CTA per 64 positions)
+  const bool pack = !key_major && s.pack;
+  const int u = pack ? cta / nT : cta / nST;
+  const int n = key_major ? u / s.Hkv : (pack ? u / (s.H / 2) : u / s.H);
+  const int uk = key_major ? u : n * s.Hkv + (pack ? 2 * (u % (s.H / 2)) : u % s.H) / s.G;
   int len = seq_lens ? seq_lens[n] : s.L;
   len = min(max(len, 0), s.L);
   const int pad0 = s.L - len;
@@ -69,8 +75,11 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
   __syncwarp();
 
   if (!key_major) {
-    const int st = nST - 1 - cta % nST;  // the attention kernels take long rows first
-    const int row0 = st * 128, row_last = min(s.L - 1, row0 + 127);
+    const int st = pack ? nT - 1 - cta % nT : nST - 1 - cta % nST;  // the attention kernels take long rows first
+    const int row0 = pack ? st * 64 : st * 128, row_last = min(s.L - 1, row0 + (pack ? 63 : 127));
+    // first position of the 32 rows of TMEM lane quarter w, and of the 64-row half hf
+    auto quarter_row0 = [&](int w) { return row0 + 32 * (pack ? (w & 1) : w); };
+    auto half_row0 = [&](int hf) { return pack ? row0 : row0 + 64 * hf; };
     if (s.pq) {
       // a selection per query position: every row's own bytes, and their union per query block
       // (which is what the tile list and the item order below are built from)
@@ -88,7 +97,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       }
     } else {
     for (int i = lane; i < G * s.topk; i += 32) {  // the selections of the CTA's query blocks
-      const int g = i / s.topk, slot = i % s.topk, qb = st * G + g;
+      const int g = i / s.topk, slot = i % s.topk, qb = pack ? st * nb + g % nb : st * G + g;
       if (qb < s.M) {
         const int blk = idx[((int64_t)uk * s.M + qb) * s.topk + slot];
         if (blk >= 0 && blk < s.M && (blk <= qb || !s.causal)) {
@@ -180,7 +189,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     const uint32_t allbits = (1u << (64 / s.Bk)) - 1u;
     for (int e = lane; e < count * 4; e += 32) {
       const int it = e >> 2, w = e & 3;
-      const int jt = items[it], p0 = jt * 64, t_lo = row0 + w * 32;
+      const int jt = items[it], p0 = jt * 64, t_lo = quarter_row0(w);
       const bool some = (p0 <= t_lo + 31 || !s.causal) && p0 + 63 >= pad0 && t_lo + 31 >= pad0 && t_lo < s.L;
       // every row of the warp may see every key of the tile as far as validity and causality go
       const bool inner = t_lo >= pad0 && t_lo + 31 < s.L && p0 >= pad0 && (s.causal ? p0 + 63 <= t_lo : p0 + 63 < s.L);
@@ -220,8 +229,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                 if (selb[g * nT + jt]) c |= g < gh ? 1 : 2;
             if (lflags[j] & 2)
               for (int hf = 0; hf < 2; ++hf)
-                if ((p0 <= row0 + 64 * hf + 63 || !s.causal) &&
-                    st_ranges_touch(s, row0 + 64 * hf, row0 + 64 * hf + 63, p0, p0 + 63))
+                if ((p0 <= half_row0(hf) + 63 || !s.causal) &&
+                    st_ranges_touch(s, half_row0(hf), half_row0(hf) + 63, p0, p0 + 63))
                   c |= 1 << hf;
             if (c == 0) c = 3;
           }
@@ -263,7 +272,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     for (int e = lane; e < (kmeta ? nv * 16 : 0); e += 32) {
       const int it = e >> 4, hh = (e >> 3) & 1, w = e & 7, qtr = w & 3, c = w >> 2;
       const int jt = list[it], f = lflags[it];
-      const int k_lo = jt * 64 + 32 * hh + 16 * c, k_hi = k_lo + 15, t_lo = row0 + qtr * 32, t_hi = t_lo + 31;
+      const int k_lo = jt * 64 + 32 * hh + 16 * c, k_hi = k_lo + 15, t_lo = quarter_row0(qtr), t_hi = t_lo + 31;
       const bool rows_in = t_lo >= pad0 && t_hi < s.L, rows_none = t_hi < pad0 || t_lo >= s.L;
       const bool past = rows_in && k_lo >= pad0 && (s.causal ? k_hi <= t_lo : k_hi < s.L);  // every key visible to every row (validity, causality)
       const bool reach = !rows_none && (k_lo <= t_hi || !s.causal) && k_hi >= pad0 && k_lo < s.L;  // some key may be visible to some row
@@ -392,7 +401,7 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
                    uint8_t *kmeta, cudaStream_t st, int branches, int with_fwd) {
   if (with_fwd < 0) with_fwd = kmeta == nullptr;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
-  const int nq = nST * s.B * s.H, n_images = kmeta ? nq + nST * s.B * s.Hkv : nq;
+  const int nq = s.pack ? nT * s.B * (s.H / 2) : nST * s.B * s.H, n_images = kmeta ? nq + nST * s.B * s.Hkv : nq;
   const size_t smem = (size_t)kMetaWarps * (meta_bytes(nT, s.pq) + ((3 * nT + 15) / 16) * 16);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(tc_meta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

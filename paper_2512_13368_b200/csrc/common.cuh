@@ -25,6 +25,9 @@ struct Shape {
   int gate_mode;          // 0: one gate weight per head from two logits; 1: Eq. 18's input-dependent gate
   const float *phi;       // logits of the learnable block summary (Eq. 9) or nullptr = the mean
   int reuse_lists;        // backward: the tile lists of the preceding training forward are in the workspace
+  int pack;               // tensor-core forward and dQ kernel: a CTA's 128 rows are the same 64 positions of
+                          // two query heads that share a key/value head (they select the same blocks,
+                          // Eq. 12, and their windows reach the same tiles), not 128 positions of one head
   int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
 };
 

@@ -493,7 +493,8 @@ __device__ __forceinline__ void store_row_chunk(uint8_t *tile, int r, int ch, ui
 }
 
 // ---- host: TMA descriptor of a q-shaped bf16 tensor, box = (D, rows, 1, 1) -----------------
-int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows, bool kv = false);
+int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows, bool kv = false,
+                    int box_heads = 1);
 
 // Builds the bookkeeping of every query-major CTA (forward, dQ) into qmeta and, if kmeta is not
 // null, of every key-major CTA (dK/dV) into kmeta: meta_bytes(nT) bytes per CTA, CTA-major.

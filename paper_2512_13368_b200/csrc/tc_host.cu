@@ -21,16 +21,16 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// q-shaped bf16 tensor [B][H][L][D] with the caller's strides, box = (D, box_rows, 1, 1); rows
-// past L read as zeros.  The swizzle matches the shared-memory descriptors of the kernels.
-int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows, bool kv) {
+// q-shaped bf16 tensor [B][H][L][D] with the caller's strides, box = (D, box_rows, box_heads, 1)
+// (the box's heads follow one another in shared memory, box_rows rows each); rows past L read as zeros.  The swizzle matches the shared-memory descriptors of the kernels.
+int make_tensor_map(CUtensorMap *map, const void *base, const Shape &s, int box_rows, bool kv, int box_heads) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return 1;
   // kv: a key/value-shaped tensor [B][Hkv][L][D] with its own strides
   const cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.L, (cuuint64_t)(kv ? s.Hkv : s.H), (cuuint64_t)s.B};
   const cuuint64_t strides[3] = {(cuuint64_t)(kv ? s.ksl : s.sl) * 2, (cuuint64_t)(kv ? s.ksh : s.sh) * 2,
                                  (cuuint64_t)(kv ? s.ksb : s.sb) * 2};
-  const cuuint32_t box[4] = {(cuuint32_t)s.D, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t box[4] = {(cuuint32_t)s.D, (cuuint32_t)box_rows, (cuuint32_t)box_heads, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   const CUtensorMapSwizzle sw = s.D == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
   CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,

@@ -193,6 +193,9 @@ def test_config4_full_size_input_dependent_gate(runner):
     (300, 64, 6, 3, 32, 4, 40, [300, 131], False),
     (256, 64, 4, 1, 64, 3, 8, None, True),               # one key/value head, power-law short-term mask
     (1024, 64, 8, 2, 64, 8, 256, [1024, 640], False),
+    (448, 64, 6, 2, 32, 4, 40, [448, 131], False),       # an odd number of heads per key/value head
+    (330, 32, 4, 2, 16, 3, 24, [330, 9, 200], True),     # pairs of heads, six 64-position tiles, the last ragged
+    (577, 64, 4, 2, 64, 5, 100, [577, 64, 65], False),   # pairs of heads, an odd number of tiles
 ])
 def test_grouped_query_heads(runner, dtype, L, D, H, Hkv, block, topk, window, lens, power_law):
     """Query heads share key/value heads and one selection per group (summed scores, Eq. 12)."""
