@@ -169,7 +169,7 @@ static int make_shape(const blossom_params *p, Shape *out) {
   s.esz = p->dtype == BLOSSOM_DTYPE_BF16 ? 2 : 4;
   s.pq = p->select_mode;
   s.causal = p->causal;
-  s.pack = (s.G % 2 == 0 && !s.pq) ? 1 : 0;
+  s.pack = s.G % 2 == 0 ? 1 : 0;
   if (!s.causal && (s.pq || s.cmp_l > 0)) return BLOSSOM_ERR_UNSUPPORTED;  // bidirectional: plain per-block selection
   s.phi = p->phi_logits;
   if (reinterpret_cast<uintptr_t>(s.phi) % 4) return BLOSSOM_ERR_INVALID_ARG;

@@ -825,7 +825,7 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   const size_t smem_kv =
       1024 + 2 * C::kBigBytes + kKvStages * (2 * C::kSmallBytes + kStatBytes) + meta_bytes(nT, s.pq);
   const bool plain = s.causal && !s.pq;
-  auto kern_dq = s.pack ? (s.causal ? bwd_dq_tc_kernel<D, true, true> : bwd_dq_tc_kernel<D, false, true>)
+  auto kern_dq = s.pack ? (plain ? bwd_dq_tc_kernel<D, true, true> : bwd_dq_tc_kernel<D, false, true>)
                         : (plain ? bwd_dq_tc_kernel<D, true, false> : bwd_dq_tc_kernel<D, false, false>);
   auto kern_kv = plain ? bwd_dkdv_tc_kernel<D, true> : bwd_dkdv_tc_kernel<D, false>;
   if (cudaFuncSetAttribute(kern_dq, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq) != cudaSuccess ||

@@ -485,8 +485,9 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
     return BLOSSOM_ERR_CUDA;
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
   const size_t smem = 1024 + 2 * C::kBigBytes + kFwdStages * 2 * C::kSmallBytes + meta_bytes(nT, s.pq);
-  auto kern = s.pack ? (s.causal ? fwd_tc_kernel<D, true, true> : fwd_tc_kernel<D, false, true>)
-                     : ((s.causal && !s.pq) ? fwd_tc_kernel<D, true, false> : fwd_tc_kernel<D, false, false>);
+  const bool plain = s.causal && !s.pq;
+  auto kern = s.pack ? (plain ? fwd_tc_kernel<D, true, true> : fwd_tc_kernel<D, false, true>)
+                     : (plain ? fwd_tc_kernel<D, true, false> : fwd_tc_kernel<D, false, false>);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
   const unsigned grid = s.pack ? (unsigned)nT * (unsigned)(s.B * (s.H / 2)) : (unsigned)nST * (unsigned)(s.B * s.H);

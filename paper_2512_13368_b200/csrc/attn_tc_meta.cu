@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       // (which is what the tile list and the item order below are built from)
       uint32_t *roww = reinterpret_cast<uint32_t *>(meta + ml.rows);
       for (int i = lane; i < 128 * s.topk; i += 32) {
-        const int r = i / s.topk, slot = i % s.topk, t = row0 + r;
+        const int r = i / s.topk, slot = i % s.topk, t = pack ? row0 + (r & 63) : row0 + r;
         if (t < s.L) {
           const int blk = idx[((int64_t)uk * s.L + t) * s.topk + slot];
           if (blk >= 0 && blk <= (t >> bk_shift)) {

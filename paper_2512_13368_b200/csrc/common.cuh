@@ -27,7 +27,8 @@ struct Shape {
   int reuse_lists;        // backward: the tile lists of the preceding training forward are in the workspace
   int pack;               // tensor-core forward and dQ kernel: a CTA's 128 rows are the same 64 positions of
                           // two query heads that share a key/value head (they select the same blocks,
-                          // Eq. 12, and their windows reach the same tiles), not 128 positions of one head
+                          // Eq. 12, and their windows reach the same tiles), not 128 positions of one head;
+                          // set whenever the heads per key/value head are even
   int64_t ksb, ksh, ksl;  // element strides of k, v, dk, dv ([B][Hkv][L][D])
 };
 

@@ -586,7 +586,7 @@ def test_random_combinations_of_the_options(runner):
 
 
 @pytest.mark.parametrize("opts", [{}, {"causal": 0}, {"per_query": 1}, {"gate_mode": 1}, {"power_law": True, "kv_heads": 2},
-                                  {"full": True}, {"full": True, "causal": 0}])
+                                  {"full": True}, {"full": True, "causal": 0}, {"full": True, "kv_heads": 2}])
 def test_repeated_steps_give_the_same_bits(runner, opts):
     """Nothing in the path is allowed to depend on the order in which warps or CTAs happen to run
     (no atomics on results, fixed reduction orders, every hand-off behind a barrier): repeated
@@ -594,7 +594,7 @@ def test_repeated_steps_give_the_same_bits(runner, opts):
     (thirty steps of a mid-size problem, twelve of the headline shape)."""
     import torch
     if opts.get("full"):
-        w, reps = workloads.config4(), 12
+        w, reps = workloads.config4(kv_heads=opts.get("kv_heads", 0)), 12
     else:
         w, reps = workloads.make("repeat", "bf16", 4, 4, 2048, 64, 64, 8, 200, seed=97, lengths=(700, 2048),
                                  kv_heads=opts.get("kv_heads", 0), stis_mode=1 if opts.get("power_law") else 0), 30
