@@ -10,7 +10,7 @@
  *     buffer; except where an entry point says otherwise the library allocates nothing,
  *     launches only on the given stream and never synchronises.  State kept between calls: none
  *     that a result depends on; process-wide there are a launch counter, the optional event
- *     profile below, and the two debugging switches (blossom_debug_switch).
+ *     profile below, and the debugging switches (blossom_debug_switch).
  *   - q-shaped tensors (q, k, v, out, out_lt, out_st, dout, dq, dk, dv) are [B][H][L][D] with
  *     element strides (stride_b, stride_h, stride_l, 1) shared by all of them; the element type
  *     is params.dtype.  Base pointers must be 16-byte aligned and the three strides multiples
@@ -244,10 +244,14 @@ int blossom_selftest_wait_timeout(void *workspace, size_t workspace_bytes, bloss
 
 /* Debugging switches (no counterpart in the paper), process-wide, host only, not thread-safe.
  * which = 0: route every call to the fp32 CUDA-core kernels instead of the tensor-core ones;
- * which = 1: score every query block in double precision (skip the certified fp32 stage).
+ * which = 1: score every query block in double precision (skip the certified fp32 stage);
+ * which = 2: launch every kernel fully serialised behind its predecessor (by default the kernels
+ * of a call are chained by programmatic dependent launches: a kernel may become resident while
+ * the last CTAs of the one before it still run, and waits for that kernel's completion before it
+ * touches global memory; results do not depend on the switch).
  * value 1 = on, 0 = off, -1 = back to the default, which is the environment variable
- * BLOSSOM_FORCE_SIMT resp. BLOSSOM_EXACT_SELECT as it stood when the library was loaded
- * (unset or "0" = off).  Returns BLOSSOM_ERR_INVALID_ARG for other arguments. */
+ * BLOSSOM_FORCE_SIMT, BLOSSOM_EXACT_SELECT resp. BLOSSOM_SERIAL_LAUNCH as it stood when the
+ * library was loaded (unset or "0" = off).  Returns BLOSSOM_ERR_INVALID_ARG for other arguments. */
 int blossom_debug_switch(int which, int value);
 
 /* Human-readable name of a blossom_status (host string, static storage). */
@@ -269,8 +273,14 @@ uint64_t blossom_launch_count(void);
  * entries), destroys the events and returns the number of launches written (-1 on error or if
  * no profile is running).  Process-wide and not thread-safe; off by default; launches beyond
  * max_launches are not recorded.  blossom_kernel_name maps an id to a static host string.
+ * An event record between two kernels keeps the second from becoming resident before the first
+ * has completed (see blossom_debug_switch, which = 2) and costs a few microseconds itself;
+ * blossom_profile_every(n), called while no profile is running, makes the following profiles
+ * bracket only every n-th launch of each kernel (n >= 1, default 1; BLOSSOM_ERR_INVALID_ARG
+ * otherwise), so that a timed loop of several steps is disturbed in one step out of n.
  */
 int blossom_profile_start(int max_launches);
+int blossom_profile_every(int n);
 int blossom_profile_stop(int32_t *kernel_ids /* host */, float *ms /* host */, int capacity);
 const char *blossom_kernel_name(int kernel_id);
 

@@ -27,7 +27,8 @@ EXPORTS = (
     "blossom_workspace_bytes", "blossom_select_blocks", "blossom_select_blocks_static",
     "blossom_attn_fwd", "blossom_attn_bwd",
     "blossom_device_status", "blossom_status_string", "blossom_version", "blossom_launch_count",
-    "blossom_profile_start", "blossom_profile_stop", "blossom_kernel_name", "blossom_debug_switch",
+    "blossom_profile_start", "blossom_profile_every", "blossom_profile_stop", "blossom_kernel_name",
+    "blossom_debug_switch",
     "blossom_selftest_wait_timeout",
 )
 
@@ -87,6 +88,8 @@ def load():
     lib.blossom_launch_count.restype = ctypes.c_uint64
     lib.blossom_profile_start.restype = ctypes.c_int
     lib.blossom_profile_start.argtypes = [ctypes.c_int]
+    lib.blossom_profile_every.restype = ctypes.c_int
+    lib.blossom_profile_every.argtypes = [ctypes.c_int]
     lib.blossom_profile_stop.restype = ctypes.c_int
     lib.blossom_profile_stop.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     lib.blossom_kernel_name.restype = ctypes.c_char_p
@@ -219,6 +222,12 @@ def blossom_profile_start(max_launches: int) -> None:
         raise BlossomError(rc, "blossom_profile_start")
 
 
+def blossom_profile_every(n: int) -> None:
+    rc = load().blossom_profile_every(int(n))
+    if rc:
+        raise BlossomError(rc, "blossom_profile_every")
+
+
 def blossom_profile_stop(capacity: int):
     """Returns a list of (kernel name, milliseconds), one entry per recorded launch."""
     ids = (ctypes.c_int32 * capacity)()
@@ -235,6 +244,7 @@ def blossom_kernel_name(kernel_id: int) -> str:
 
 SWITCH_FORCE_SIMT = 0
 SWITCH_EXACT_SELECT = 1
+SWITCH_SERIAL_LAUNCH = 2
 
 
 def blossom_debug_switch(which: int, value: int) -> None:

@@ -16,10 +16,18 @@ static int *g_prof_start = nullptr;           // index of the event a record's t
 static int g_prof_cap = 0, g_prof_n = 0;
 static cudaStream_t g_prof_chain_stream = nullptr;
 static bool g_prof_chain = false;  // the last thing put on g_prof_chain_stream was a record's end event
+static int g_prof_every = 1;       // blossom_profile_every: every n-th launch of each kernel is bracketed
+static unsigned g_prof_seen[K_COUNT];
+static bool g_prof_skip = false;   // the launch in progress is not bracketed
 
 void prof_mark(int id, int phase, cudaStream_t st) {
   if (!g_prof_events) return;
   if (phase == 0) {
+    g_prof_skip = (g_prof_seen[id]++ % (unsigned)g_prof_every) != 0;
+    if (g_prof_skip) {
+      g_prof_chain = false;  // the next bracketed launch records its own start
+      return;
+    }
     if (g_prof_n >= g_prof_cap) return;
     g_prof_ids[g_prof_n] = id;
     // back-to-back launches of one call share an event: the end of one is the start of the next
@@ -30,7 +38,7 @@ void prof_mark(int id, int phase, cudaStream_t st) {
       cudaEventRecord(g_prof_events[2 * g_prof_n], st);
     }
   } else {
-    if (g_prof_n >= g_prof_cap) return;
+    if (g_prof_skip || g_prof_n >= g_prof_cap) return;
     cudaEventRecord(g_prof_events[2 * g_prof_n + 1], st);
     g_prof_chain = true;
     g_prof_chain_stream = st;
@@ -42,16 +50,21 @@ void prof_mark(int id, int phase, cudaStream_t st) {
 // last call must not be charged to this call's first kernel.
 void prof_break() { g_prof_chain = false; }
 
-// The two environment switches are read once, when the library is loaded.
+// The environment switches are read once, when the library is loaded.
 static bool env_flag(const char *name) {
   const char *e = getenv(name);
   return e && e[0] && e[0] != '0';
 }
 static const bool g_force_simt = env_flag("BLOSSOM_FORCE_SIMT");
 static const bool g_exact_select = env_flag("BLOSSOM_EXACT_SELECT");
-static int g_force_simt_override = -1, g_exact_select_override = -1;  // blossom_debug_switch
+static const bool g_serial_launch = env_flag("BLOSSOM_SERIAL_LAUNCH");
+static int g_force_simt_override = -1, g_exact_select_override = -1, g_serial_launch_override = -1;  // blossom_debug_switch
 
 bool force_simt() { return g_force_simt_override >= 0 ? g_force_simt_override != 0 : g_force_simt; }
+
+bool chained_launches() {
+  return !(g_serial_launch_override >= 0 ? g_serial_launch_override != 0 : g_serial_launch);
+}
 
 bool exact_select_only() {
   return g_exact_select_override >= 0 ? g_exact_select_override != 0 : g_exact_select;
@@ -357,6 +370,7 @@ int blossom_debug_switch(int which, int value) {
   if (value < -1 || value > 1) return BLOSSOM_ERR_INVALID_ARG;
   if (which == 0) g_force_simt_override = value;
   else if (which == 1) g_exact_select_override = value;
+  else if (which == 2) g_serial_launch_override = value;
   else return BLOSSOM_ERR_INVALID_ARG;
   return BLOSSOM_OK;
 }
@@ -387,10 +401,18 @@ int blossom_profile_start(int max_launches) {
     }
   g_prof_ids = new int[max_launches];
   g_prof_start = new int[max_launches];
+  for (int i = 0; i < K_COUNT; ++i) g_prof_seen[i] = 0;
+  g_prof_skip = false;
   g_prof_chain = false;
   g_prof_cap = max_launches;
   g_prof_n = 0;
   g_prof_events = ev;
+  return BLOSSOM_OK;
+}
+
+int blossom_profile_every(int n) {
+  if (n < 1 || g_prof_events) return BLOSSOM_ERR_INVALID_ARG;
+  g_prof_every = n;
   return BLOSSOM_OK;
 }
 

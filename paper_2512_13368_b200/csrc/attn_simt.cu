@@ -543,6 +543,7 @@ __global__ void __launch_bounds__(256) bwd_dkdv_simt_kernel(
 __global__ void __launch_bounds__(256) gate_grad_kernel(Shape s, const float *__restrict__ gate,
                                                         const double *__restrict__ dalpha_part,
                                                         float *__restrict__ dgate) {
+  grid_chain_enter();
   __shared__ double red[256];
   const int h = blockIdx.x;
   double a = 0.0;
@@ -657,7 +658,7 @@ int launch_gate_grad(const Shape &s, const float *gate, const Workspace &ws, flo
                      cudaStream_t st) {
   {
     LaunchScope ls(K_GATE_GRAD, st);
-    gate_grad_kernel<<<s.H, 256, 0, st>>>(s, gate, ws.dalpha, dgate);
+    launch_chained(gate_grad_kernel, dim3(s.H), dim3(256), 0, st, s, gate, (const double *)ws.dalpha, dgate);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -69,6 +69,7 @@ __global__ void __launch_bounds__(256) bwd_prep_kernel(Shape s, const float *__r
                                                        const float *__restrict__ lse,
                                                        const __nv_bfloat16 *__restrict__ dout,
                                                        float4 *__restrict__ qstats, int Lpad) {
+  grid_chain_enter();
   constexpr int LPR = D / 8;         // lanes per row
   constexpr int RPB = 256 / LPR;     // rows per block
   const int blocks_per_unit = (Lpad + RPB - 1) / RPB;
@@ -167,6 +168,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dq_tc_kernel(
     const uint8_t *__restrict__ qmeta, const __grid_constant__ CUtensorMap tmdq,
     const float4 *__restrict__ qstats, double *__restrict__ dalpha_part, int32_t *__restrict__ status,
     int nT) {
+  grid_chain_enter();
   using C = Cfg<D>;
   constexpr int STAGES = kDqStages;
   constexpr int OC = D / 2;  // accumulator columns per thread
@@ -532,6 +534,7 @@ __global__ void __launch_bounds__(kKvThreads, 2) bwd_dkdv_tc_kernel(
     const int32_t *__restrict__ seq_lens, const uint8_t *__restrict__ kmeta,
     const float4 *__restrict__ qstats, const __grid_constant__ CUtensorMap tmdk,
     const __grid_constant__ CUtensorMap tmdv, int32_t *__restrict__ status, int nT) {
+  grid_chain_enter();
   using C = Cfg<D>;
   constexpr int STAGES = kKvStages;
   constexpr int OC = D / 2;
@@ -838,21 +841,20 @@ int launch_bwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
     LaunchScope ls(K_BWD_PREP, st);
     const int Lpad = nT * 64, rpb = 256 / (D / 8);
     const unsigned gp = (unsigned)(s.B * s.H) * (unsigned)((Lpad + rpb - 1) / rpb);
-    bwd_prep_kernel<D><<<gp, 256, 0, st>>>(s, gate, seq_lens, (const bf *)out_lt, (const bf *)out_st, lse,
-                                          (const bf *)dout, ws.qstats, Lpad);
+    launch_chained(bwd_prep_kernel<D>, dim3(gp), dim3(256), 0, st, s, gate, seq_lens, (const bf *)out_lt,
+                   (const bf *)out_st, lse, (const bf *)dout, ws.qstats, Lpad);
   }
   {
     LaunchScope ls(K_BWD_DQ_TC, st);
     const unsigned grid_q = s.pack ? (unsigned)nT * (unsigned)(s.B * (s.H / 2)) : grid;
-    kern_dq<<<grid_q, kKvThreads, smem_dq, st>>>(q128, k64, v64, g128, s, gate, seq_lens, ws.qmeta,
-                                                           tdq, rec, ws.dalpha,
-                                                           ws.status_bwd, nT);
+    launch_chained(kern_dq, dim3(grid_q), dim3(kKvThreads), smem_dq, st, q128, k64, v64, g128, s, gate, seq_lens,
+                   (const uint8_t *)ws.qmeta, tdq, rec, ws.dalpha, ws.status_bwd, nT);
   }
   {
     LaunchScope ls(K_BWD_DKDV_TC, st);
     const unsigned grid_k = (unsigned)nST * (unsigned)(s.B * s.Hkv);
-    kern_kv<<<grid_k, kKvThreads, smem_kv, st>>>(q64, k128, v128, g64, s, seq_lens, ws.kmeta,
-                                                             rec, tdk, tdv, ws.status_bwd, nT);
+    launch_chained(kern_kv, dim3(grid_k), dim3(kKvThreads), smem_kv, st, q64, k128, v128, g64, s, seq_lens,
+                   (const uint8_t *)ws.kmeta, rec, tdk, tdv, ws.status_bwd, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -129,6 +129,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) fwd_tc_kernel(
     const float *__restrict__ gate, const int32_t *__restrict__ seq_lens,
     const uint8_t *__restrict__ qmeta, int training, float *__restrict__ lse,
     int32_t *__restrict__ status, int nT) {
+  grid_chain_enter();
   using C = Cfg<D>;
   constexpr int STAGES = kFwdStages;
   constexpr int DC = D / 2;  // output columns a softmax thread merges and stages
@@ -496,8 +497,8 @@ int launch_fwd_tc_t(const Shape &s, const void *q, const void *k, const void *v,
   if (int rc = launch_tc_meta(s, seq_lens, idx, ws.qmeta, training ? ws.kmeta : nullptr, st, 3, 1)) return rc;
   {
     LaunchScope ls(K_FWD_TC, st);
-    kern<<<grid, kFwdThreads, smem, st>>>(tq, tk, tv, to, tol, tos, s, gate, seq_lens, ws.qmeta,
-                                                     training, lse, ws.status, nT);
+    launch_chained(kern, dim3(grid), dim3(kFwdThreads), smem, st, tq, tk, tv, to, tol, tos, s, gate, seq_lens,
+                   (const uint8_t *)ws.qmeta, training, lse, ws.status, nT);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                                                                   uint8_t *__restrict__ kmeta, int nT,
                                                                   int n_query_ctas, int n_images, int branches,
                                                                   int with_fwd) {
+  grid_chain_enter();
   extern __shared__ __align__(16) uint8_t meta_all[];
   const MetaLayout ml = meta_layout(nT, s.pq);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -408,8 +409,8 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
     return BLOSSOM_ERR_CUDA;
   {
     LaunchScope ls(K_TC_META, st);
-    tc_meta_kernel<<<(unsigned)((n_images + kMetaWarps - 1) / kMetaWarps), kMetaWarps * 32, smem, st>>>(
-        s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images, branches, with_fwd);
+    launch_chained(tc_meta_kernel, dim3((unsigned)((n_images + kMetaWarps - 1) / kMetaWarps)), dim3(kMetaWarps * 32),
+                   smem, st, s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images, branches, with_fwd);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/blossom.h"
 
 namespace blossom {
@@ -82,6 +84,37 @@ struct LaunchScope {
   LaunchScope(int id_, cudaStream_t st_) : id(id_), st(st_) { ++g_launches; prof_mark(id, 0, st); }
   ~LaunchScope() { prof_mark(id, 1, st); }
 };
+
+// ---- chained launches ---------------------------------------------------------------------
+// The kernels of a call follow one another on the caller's stream, each reading what the one before
+// wrote.  A kernel launched with launch_chained() may become resident while its predecessor's last
+// CTAs still run (programmatic dependent launch), which hides the launch latency and part of the
+// predecessor's tail; such a kernel calls grid_chain_enter() as its first statement, in every
+// thread: it lets the kernel behind it do the same and then waits until the kernel before it has
+// completed and its writes are visible.  Nothing before that call may touch global memory.  Behind
+// anything but a kernel (a memset, an event) and with the switch off (chained_launches()) the
+// launch is an ordinary one and the call returns at once.
+__device__ __forceinline__ void grid_chain_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+bool chained_launches();  // blossom_debug_switch(2, ...) / BLOSSOM_SERIAL_LAUNCH
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = chained_launches() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 // ---- element access: 4 consecutive elements as float4 ------------------------------------
 __device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }

@@ -107,6 +107,7 @@ __global__ void __launch_bounds__(256, PHI ? 2 : 4) summary_kernel(Shape sh, Sel
                                                          float *__restrict__ mean32,
                                                          float *__restrict__ norm,
                                                          int32_t *__restrict__ sel_count) {
+  grid_chain_enter();
   constexpr int LPR = D / 8;     // lanes per row
   constexpr int RPI = 32 / LPR;  // rows per warp iteration
   constexpr int NF = sizeof(T) == 2 ? 8 : 2;  // rows in flight per lane
@@ -295,6 +296,7 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
     Shape sh, SelGeom g, const T *__restrict__ q, const float *__restrict__ mean32,
     const float *__restrict__ norm, const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx,
     int32_t *__restrict__ worklist, int32_t *__restrict__ work_count, int sc_pitch) {
+  grid_chain_enter();
   constexpr int P = D + 4;  // row pitch of the operand tiles (floats): conflict-free 128-bit reads
   extern __shared__ float fsm[];
   __shared__ float rn[kRowTile];  // norm bound of every query row (largest over the group's heads)
@@ -582,6 +584,7 @@ __global__ void __launch_bounds__(256, 2) score_exact_kernel(
     Shape sh, SelGeom g, const T *__restrict__ q, const double *__restrict__ mean,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx, const int32_t *__restrict__ worklist,
     const int32_t *__restrict__ work_count, int sc_len) {
+  grid_chain_enter();
   constexpr int PD = D + 1;
   extern __shared__ double dsm[];
   __shared__ double bound_d[2];
@@ -788,6 +791,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256) score_per_query_kernel(
     Shape sh, const T *__restrict__ q, const double *__restrict__ mean,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx) {
+  grid_chain_enter();
   extern __shared__ double dsm[];
   __shared__ double bound_d[8][2];
   const int M = sh.M, Bk = sh.Bk;
@@ -866,6 +870,7 @@ template <typename T, int D, int NZ>
 __global__ void __launch_bounds__(256, NZ == 1 ? 2 : 1) score_per_query_tile_kernel(
     Shape sh, SelGeom g, const T *__restrict__ q, const double *__restrict__ mean,
     const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx) {
+  grid_chain_enter();
   constexpr int PD = D + 1, MP = 64 * NZ;
   extern __shared__ double dsm[];
   __shared__ double bound_d[8][2];
@@ -1040,7 +1045,8 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tsm) != cudaSuccess)
         return BLOSSOM_ERR_CUDA;
       LaunchScope ls(K_SCORE_SELECT, st);
-      kern<<<(unsigned)(units * ((sh.L + 63) / 64)), 256, tsm, st>>>(sh, g, q, w.mean, seq_lens, idx);
+      launch_chained(kern, dim3((unsigned)(units * ((sh.L + 63) / 64))), dim3(256), tsm, st, sh, g, q,
+                     (const double *)w.mean, seq_lens, idx);
       return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
     }
     if (!g.plain) return BLOSSOM_ERR_UNSUPPORTED;  // (more than 128 blocks: the per-warp kernel scores selection blocks only)
@@ -1049,7 +1055,8 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm) != cudaSuccess)
       return BLOSSOM_ERR_CUDA;
     LaunchScope ls(K_SCORE_SELECT, st);
-    score_per_query_kernel<T, D><<<(unsigned)((units * sh.L + 7) / 8), 256, psm, st>>>(sh, q, w.mean, seq_lens, idx);
+    launch_chained(score_per_query_kernel<T, D>, dim3((unsigned)((units * sh.L + 7) / 8)), dim3(256), psm, st, sh, q,
+                   (const double *)w.mean, seq_lens, idx);
     return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
   }
   int sc_pitch = 0, sc_len = 0;
@@ -1062,8 +1069,8 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
       return BLOSSOM_ERR_CUDA;
     const unsigned ntiles = (unsigned)((sh.L + kRowTile - 1) / kRowTile);
     LaunchScope ls(K_SCORE_FAST, st);
-    score_fast_kernel<T, D><<<ntiles * (unsigned)units, kFastThreads, fsm, st>>>(
-        sh, g, q, w.mean32, w.norm, seq_lens, idx, w.list, w.count, sc_pitch);
+    launch_chained(score_fast_kernel<T, D>, dim3(ntiles * (unsigned)units), dim3(kFastThreads), fsm, st, sh, g, q,
+                   (const float *)w.mean32, (const float *)w.norm, seq_lens, idx, w.list, w.count, sc_pitch);
   }
   const size_t esm = exact_smem_bytes(sh, g, D, &sc_len);
   auto exact = g.n > 64 ? score_exact_kernel<T, D, 2> : score_exact_kernel<T, D, 1>;
@@ -1082,13 +1089,15 @@ int launch_select_t(const Shape &sh, const T *q, const T *k, const int32_t *seq_
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = esm;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = cl;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // chained behind the kernel before it
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = chained_launches() ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, exact, sh, g, q, (const double *)w.mean, seq_lens, idx,
                            (const int32_t *)(exact_only ? nullptr : w.list), (const int32_t *)w.count,
                            sc_len) != cudaSuccess)

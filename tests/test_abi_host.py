@@ -165,7 +165,8 @@ def test_every_q_shaped_buffer_gets_q_strides():
 
 def test_debug_switch_arguments(lib):
     assert lib.blossom_debug_switch(0, -1) == 0 and lib.blossom_debug_switch(1, -1) == 0
-    assert lib.blossom_debug_switch(2, 0) == binding.BLOSSOM_ERR_INVALID_ARG
+    assert lib.blossom_debug_switch(2, -1) == 0
+    assert lib.blossom_debug_switch(3, 0) == binding.BLOSSOM_ERR_INVALID_ARG
     assert lib.blossom_debug_switch(0, 2) == binding.BLOSSOM_ERR_INVALID_ARG
 
 

@@ -625,6 +625,63 @@ def test_repeated_steps_give_the_same_bits(runner, opts):
         print(check_forward_backward(w, p.results()))
 
 
+@pytest.mark.parametrize("opts", [{}, {"kv_heads": 2, "power_law": True}, {"per_query": 1}, {"gate_mode": 1}])
+def test_chained_and_serial_launches_give_the_same_bits(runner, opts):
+    """By default a kernel of a call may become resident while the last CTAs of the kernel before it
+    still run, and waits for that kernel's completion before it touches global memory; with the
+    debugging switch every launch is fully serialised.  Same bits either way, steps alternating."""
+    import torch
+    from paper_2512_13368_b200 import binding
+    w = workloads.make("chained", "bf16", 4, 4, 1500, 64, 32, 6, 100, seed=53, lengths=(300, 1500),
+                       kv_heads=opts.get("kv_heads", 0), stis_mode=1 if opts.get("power_law") else 0)
+    w.per_query, w.gate_mode = opts.get("per_query", 0), opts.get("gate_mode", 0)
+    if w.gate_mode:
+        w.gate = (0.3 * np.random.default_rng(9).standard_normal((w.H, 2 * w.D + 1))).astype(np.float32)
+    p = runner.DeviceProblem(w)
+    keys = ("idx", "out", "out_lt", "out_st", "lse", "dq", "dk", "dv", "dgate")
+    try:
+        binding.blossom_debug_switch(binding.SWITCH_SERIAL_LAUNCH, 1)
+        p.step()
+        first = {k: getattr(p, k).clone() for k in keys}
+        for it in range(12):
+            binding.blossom_debug_switch(binding.SWITCH_SERIAL_LAUNCH, it % 2)
+            for k in keys:
+                getattr(p, k).view(torch.uint8).fill_(0xFF)
+            for _ in range(3):
+                p.step()
+            for k in keys:
+                assert torch.equal(first[k].view(torch.uint8), getattr(p, k).view(torch.uint8)), (it, k)
+    finally:
+        binding.blossom_debug_switch(binding.SWITCH_SERIAL_LAUNCH, -1)
+    assert binding.blossom_device_status(p.workspace) == 0
+    print(check_forward_backward(w, p.results()))
+
+
+def test_profile_of_every_nth_launch(runner):
+    """blossom_profile_every(n): only every n-th launch of each kernel is bracketed by events."""
+    from paper_2512_13368_b200 import binding
+    w = workloads.make("sampled", "bf16", 2, 2, 512, 64, 64, 4, 100, seed=5)
+    p = runner.DeviceProblem(w)
+    p.step()
+    counts = {}
+    for every in (1, 3):
+        binding.blossom_profile_every(every)
+        binding.blossom_profile_start(256)
+        for _ in range(6):
+            p.step()
+        rec = binding.blossom_profile_stop(256)
+        counts[every] = {}
+        for name, ms in rec:
+            assert ms > 0.0
+            counts[every][name] = counts[every].get(name, 0) + 1
+    binding.blossom_profile_every(1)
+    assert counts[1]["fwd_tc"] == 6 and counts[3]["fwd_tc"] == 2
+    assert set(counts[1]) == set(counts[3])
+    assert all(counts[3][k] * 3 == counts[1][k] for k in counts[1])
+    with pytest.raises(binding.BlossomError):
+        binding.blossom_profile_every(0)
+
+
 # ------------------------------------------- what stands in for a memory checker on this path
 def _guarded(shape, dtype, fill, device, pad=4096):
     """A tensor carved out of a larger allocation with `pad` guard elements before and after it."""
