@@ -16,7 +16,8 @@
 // 16-column passes, two columns per FMA / ADD / MUL (packed f32x2); outputs are staged in shared
 // memory and written with whole-line TMA stores.
 //
-//  dQ     resident Q, dO (128 queries); streams K, V 64-key tiles (same walk as the forward) and
+//  dQ     resident Q, dO (128 queries: 128 positions of a head, or with grouped heads 64 positions
+//         of two heads of a group, as in the forward); streams K, V 64-key tiles (same walk as the forward) and
 //         works through them in half tiles of 32 keys.  Tensor memory: two buffers of 64
 //         columns (half tile x uses buffer x % 2: S in its first 32 columns, dP in the other 32),
 //         Q and dO as first operands of the first-stage products [128,128+D/2), [160,160+D/2)

@@ -3,7 +3,9 @@
 // A CTA owns 128 query rows (128 / Bk query blocks) and walks a list of items, one 64-key tile of
 // one branch each: first the tiles any of its query blocks selected (Eq. 14, 16), then the tiles
 // its rows reach through the window (Eq. 15, 17).  A tile that belongs to both branches is visited
-// once per phase.
+// once per phase.  With grouped heads (an even number per key/value head) the 128 rows are instead
+// the same 64 positions of two heads of a group, which share their selection (Eq. 12), their window
+// tiles and their K/V: every tile on the list then has work for every row (template flag PACK).
 //
 // CTA = 384 threads.  Warps 0..7 are softmax warps: a query row (= TMEM lane) is shared by two
 // threads, warp w and warp w + 4, which split the KEYS of every tile: group 0 (warps 0..3) takes
