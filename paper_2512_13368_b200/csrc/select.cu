@@ -276,7 +276,9 @@ __device__ __forceinline__ void emit_flags(int32_t *row, const uint8_t *taken, i
 // query blocks.  Logits against 64 candidate means at a time come from a register-blocked fp32
 // product out of shared memory: thread (ty, tx) owns rows ty + 16 a and candidates tx + 8 e
 // (a, e < 8), so a row's 64 logits sit in the eight lanes tx = 0..7 and the softmax of a row needs
-// three shuffles.  Probabilities are summed over groups of four rows by shuffles and over a query
+// three shuffles.  The candidates e = 2 e2 and 2 e2 + 1 of a thread sit interleaved in shared
+// memory, so one 16-byte load brings two dimensions of both and one packed instruction does two of
+// the thread's multiply-adds (each accumulator still adds its D products one after the other).  Probabilities are summed over groups of four rows by shuffles and over a query
 // block's groups in a fixed order through shared memory.
 //
 // Error bound.  With u = 2^-24: every logit is within E = (D + 4) u scale max|q_t| max|mean_c| of
@@ -288,6 +290,17 @@ __device__ __forceinline__ void emit_flags(int32_t *row, const uint8_t *taken, i
 // Eq. 11, and a margin of 40.  R is the total, relative; two scores a > b are in certain order
 // when a - b > R (a + b).
 constexpr int kFastThreads = 128;
+
+// d = a * b + c on two packed fp32 values: two IEEE fused multiply-adds in one instruction (the
+// same rounding, and the same flush of denormals, as the scalar fmaf of this build)
+__device__ __forceinline__ float2 fma_pair(float2 a, float2 b, float2 c) {
+  uint64_t d;
+  asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<uint64_t *>(&a)), "l"(*reinterpret_cast<uint64_t *>(&b)),
+        "l"(*reinterpret_cast<uint64_t *>(&c)));
+  return *reinterpret_cast<float2 *>(&d);
+}
 constexpr int kRowTile = 128;  // positions per CTA
 constexpr int kChunk = 64;     // candidates per product
 
@@ -297,7 +310,8 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
     const float *__restrict__ norm, const int32_t *__restrict__ seq_lens, int32_t *__restrict__ idx,
     int32_t *__restrict__ worklist, int32_t *__restrict__ work_count, int sc_pitch) {
   grid_chain_enter();
-  constexpr int P = D + 4;  // row pitch of the operand tiles (floats): conflict-free 128-bit reads
+  constexpr int P = D + 4;  // row pitch of the query tile (floats): conflict-free 128-bit reads
+  constexpr int PK = D + 2;  // row pitch of the interleaved means (pairs of floats): the same
   extern __shared__ float fsm[];
   __shared__ float rn[kRowTile];  // norm bound of every query row (largest over the group's heads)
   __shared__ float bound_s[16][2];
@@ -305,7 +319,8 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
   const int M = sh.M, Bk = sh.Bk;
   const int nqb_full = kRowTile / Bk;
   float *qs = fsm;                                      // [128][P]  the tile's queries of one head
-  float *ks = qs + kRowTile * P;                        // [64][P]   a chunk of candidate means
+  float *ks = qs + kRowTile * P;                        // [4 e2][8 tx][PK][2] a chunk of candidate means: candidates
+                                                        // tx + 16 e2 and tx + 16 e2 + 8 interleaved per dimension
   float *part = ks + kChunk * P;                        // [4 warps][8][64] sums over groups of four rows
   float *Sc = part + 4 * 8 * 64;                        // [nqb][sc_pitch] summed probabilities per candidate
   float *Ssel = Sc + nqb_full * sc_pitch;               // [nqb][M] selection-block scores (overlapping mode)
@@ -390,7 +405,8 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
 #pragma unroll
         for (int it = 0; it < NK; ++it) {
           const int i = tid + it * kFastThreads, lj = i / (D / 4), c = (i % (D / 4)) * 4;
-          *reinterpret_cast<float4 *>(ks + lj * P + c) = v[it];
+          float *dst = ks + ((((lj >> 4) * 8 + (lj & 7)) * PK + c) << 1) + ((lj >> 3) & 1);
+          dst[0] = v[it].x; dst[2] = v[it].y; dst[4] = v[it].z; dst[6] = v[it].w;
         }
       }
       __syncthreads();
@@ -424,36 +440,52 @@ __global__ void __launch_bounds__(kFastThreads, 3) score_fast_kernel(
 #pragma unroll
             for (int it = 0; it < NK; ++it) {
               const int i = tid + it * kFastThreads, lj = i / (D / 4), c = (i % (D / 4)) * 4;
-              *reinterpret_cast<float4 *>(ks + lj * P + c) = v[it];
+              float *dst = ks + ((((lj >> 4) * 8 + (lj & 7)) * PK + c) << 1) + ((lj >> 3) & 1);
+              dst[0] = v[it].x; dst[2] = v[it].y; dst[4] = v[it].z; dst[6] = v[it].w;
             }
             __syncthreads();
+          }
+          float2 acc2[8][4];  // (row a; candidates e = 2 e2, 2 e2 + 1)
+#pragma unroll
+          for (int a = 0; a < 8; ++a)
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2) acc2[a][e2] = make_float2(0.f, 0.f);
+          const int ne = (nb + 7) >> 3;  // groups of 8 candidates that hold any (block-uniform)
+          const int ne2 = (ne + 1) >> 1;  // (the odd group's partner holds zeros)
+#pragma unroll 2
+          for (int c = 0; c < D; c += 4) {
+            float4 qa[8], kb[4][2];  // kb[e2][h]: dimensions c + 2 h, c + 2 h + 1 of the two candidates
+#pragma unroll
+            for (int a = 0; a < 8; ++a) qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + c);
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2)
+              if (e2 < ne2) {
+                const float *src = ks + (((e2 * 8 + tx) * PK + c) << 1);
+                kb[e2][0] = *reinterpret_cast<const float4 *>(src);
+                kb[e2][1] = *reinterpret_cast<const float4 *>(src + 4);
+              }
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2)
+              if (e2 < ne2) {
+#pragma unroll
+                for (int a = 0; a < 8; ++a) {
+                  float2 r = acc2[a][e2];
+                  r = fma_pair(make_float2(qa[a].x, qa[a].x), make_float2(kb[e2][0].x, kb[e2][0].y), r);
+                  r = fma_pair(make_float2(qa[a].y, qa[a].y), make_float2(kb[e2][0].z, kb[e2][0].w), r);
+                  r = fma_pair(make_float2(qa[a].z, qa[a].z), make_float2(kb[e2][1].x, kb[e2][1].y), r);
+                  r = fma_pair(make_float2(qa[a].w, qa[a].w), make_float2(kb[e2][1].z, kb[e2][1].w), r);
+                  acc2[a][e2] = r;
+                }
+              }
           }
           float acc[8][8];
 #pragma unroll
           for (int a = 0; a < 8; ++a)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[a][e] = 0.f;
-          const int ne = (nb + 7) >> 3;  // groups of 8 candidates that hold any (block-uniform)
-#pragma unroll 2
-          for (int c = 0; c < D; c += 4) {
-            float4 qa[8], kb[8];
-#pragma unroll
-            for (int a = 0; a < 8; ++a) qa[a] = *reinterpret_cast<const float4 *>(qs + (ty + 16 * a) * P + c);
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-              if (e < ne) kb[e] = *reinterpret_cast<const float4 *>(ks + (tx + 8 * e) * P + c);
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-              if (e < ne) {
-#pragma unroll
-                for (int a = 0; a < 8; ++a) {
-                  acc[a][e] = fmaf(qa[a].x, kb[e].x, acc[a][e]);
-                  acc[a][e] = fmaf(qa[a].y, kb[e].y, acc[a][e]);
-                  acc[a][e] = fmaf(qa[a].z, kb[e].z, acc[a][e]);
-                  acc[a][e] = fmaf(qa[a].w, kb[e].w, acc[a][e]);
-                }
-              }
-          }
+            for (int e2 = 0; e2 < 4; ++e2) {
+              acc[a][2 * e2] = acc2[a][e2].x;
+              acc[a][2 * e2 + 1] = acc2[a][e2].y;
+            }
           // logits; pairs that do not take part (dead candidates, candidates not before the row's
           // block, invalid rows) become -inf and drop out of every sum below
 #pragma unroll
