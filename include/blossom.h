@@ -122,8 +122,10 @@ typedef struct {
                         * (out_lt, out_st given) with the same params, seq_lens and block_idx contents:
                         * that call has left the backward's lists in the workspace and they are used
                         * as they are.  A broken promise gives wrong gradients, not a fault (lists of
-                        * another shape are never read: the shape is part of the promise).  Ignored
-                        * on the CUDA-core path and with gate_mode 1                               */
+                        * another shape are never read: the shape is part of the promise).  The lists
+                        * are ignored on the CUDA-core path and with gate_mode 1.  With rope_theta > 0
+                        * the promise extends to q and k: the rotated copies that forward left in the
+                        * workspace are used instead of being formed again (every path)             */
 } blossom_params;
 
 /* Bytes of device scratch the calls below need for these params (one size serves all three);

@@ -200,13 +200,17 @@ static int make_shape(const blossom_params *p, Shape *out) {
 }
 
 // With rope_theta > 0: rotated copies of q and k go to the workspace and *q, *k point at them.
+// reuse: the copies of the preceding forward on this workspace are still there (the backward's
+// reuse_tile_lists promise).
 static int rotate_inputs(const Shape &s, int dtype, const Workspace &ws, const void **q, const void **k,
-                         cudaStream_t st) {
+                         cudaStream_t st, bool reuse = false) {
   if (s.rope_theta <= 0) return BLOSSOM_OK;
-  int rc = launch_rope(s, dtype, false, +1, *q, ws.q_rot, st);
-  if (rc) return rc;
-  rc = launch_rope(s, dtype, true, +1, *k, ws.k_rot, st);
-  if (rc) return rc;
+  if (!reuse) {
+    int rc = launch_rope(s, dtype, false, +1, *q, ws.q_rot, st);
+    if (rc) return rc;
+    rc = launch_rope(s, dtype, true, +1, *k, ws.k_rot, st);
+    if (rc) return rc;
+  }
   *q = ws.q_rot;
   *k = ws.k_rot;
   return BLOSSOM_OK;
@@ -328,7 +332,7 @@ int blossom_attn_bwd(const blossom_params *params, const void *q, const void *k,
   rc = check_workspace(s, workspace, workspace_bytes, (cudaStream_t)stream, &ws, true);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  rc = rotate_inputs(s, params->dtype, ws, &q, &k, st);
+  rc = rotate_inputs(s, params->dtype, ws, &q, &k, st, s.reuse_lists != 0);
   if (rc) return rc;
   if (!force_simt() && tc::fwd_tc_supported(s, params->dtype)) {
     if (s.gate_mode) {

@@ -271,14 +271,16 @@ def test_inference_mode_and_select_only(runner):
     assert np.array_equal(q.results()["idx"], res["idx"])
 
 
-@pytest.mark.parametrize("opts", [{}, {"kv_heads": 2}, {"per_query": 1}, {"causal": 0}])
+@pytest.mark.parametrize("opts", [{}, {"kv_heads": 2}, {"per_query": 1}, {"causal": 0}, {"rope_theta": 10000.0},
+                                  {"rope_theta": 500.0, "dtype": "fp32"}])
 def test_backward_on_the_forward_s_tile_lists_gives_the_same_bits(runner, opts):
     """reuse_tile_lists = 1: a backward call that follows a training forward on the same workspace
-    walks the lists that forward built; the gradients are those of a backward that builds its own,
-    bit for bit."""
-    w = workloads.make("reuse-lists", "bf16", 3, 4, 900, 64, 32, 5, 70, seed=89, lengths=(200, 900),
+    walks the lists that forward built and, with rotary positions, reads the rotated q and k that
+    forward left there; the gradients are those of a backward that builds its own, bit for bit."""
+    w = workloads.make("reuse-lists", opts.get("dtype", "bf16"), 3, 4, 900, 64, 32, 5, 70, seed=89, lengths=(200, 900),
                        kv_heads=opts.get("kv_heads", 0))
     w.per_query, w.causal = opts.get("per_query", 0), opts.get("causal", 1)
+    w.rope_theta = opts.get("rope_theta", 0.0)
     p = runner.DeviceProblem(w)
     p.forward()
     p.backward(reuse_tile_lists=False)
