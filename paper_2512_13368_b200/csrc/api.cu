@@ -121,7 +121,7 @@ Workspace carve_workspace(const Shape &s, void *base) {
     w.qstats2 = reinterpret_cast<float4 *>(take(on ? units * (size_t)((s.L + 63) / 64 * 64) * sizeof(float4) : 0));
   }
   w.qmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
-  w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s)));
+  w.kmeta = reinterpret_cast<uint8_t *>(take(tc::tc_meta_bytes(s) + tc::tc_inv_bits_bytes(s)));
   w.bytes = off;
   return w;
 }

@@ -19,6 +19,10 @@
 // Head-packed variant (Shape::pack): the CTA's rows 0..63 and 64..127 are the same 64 positions of
 // two query heads with a common key/value head, so both halves have the same selection bytes and
 // every listed tile concerns both.
+// With a selection per query position the key-major images would each have to scan the index rows
+// of every later position; instead the query-major images, which read every index row once, set
+// one bit per (key block, position) in a table in global memory (launch 1), and the key-major
+// images copy the words of their key blocks from it (launch 2).
 // Key-major image (dK/dV kernel): [8][nT] bytes: bit c of byte (g, qt): query block
 // qt * (64 / Bk) + c selected key block g of the CTA; list / flags of the 64-query tiles that
 // visit the CTA's keys; jcls[nT][2][8] class of every (listed tile, half tile, compute warp);
@@ -37,14 +41,16 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
                                                                   const int32_t *__restrict__ idx,
                                                                   uint8_t *__restrict__ qmeta,
                                                                   uint8_t *__restrict__ kmeta, int nT,
-                                                                  int n_query_ctas, int n_images, int branches,
-                                                                  int with_fwd) {
+                                                                  int n_query_ctas, int image0, int image_end,
+                                                                  int branches, int with_fwd,
+                                                                  uint32_t *__restrict__ inv_bits) {
   grid_chain_enter();
   extern __shared__ __align__(16) uint8_t meta_all[];
   const MetaLayout ml = meta_layout(nT, s.pq);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int image = (int)blockIdx.x * kMetaWarps + warp;
-  if (image >= n_images) return;
+  const int image = image0 + (int)blockIdx.x * kMetaWarps + warp;  // this launch builds [image0, image_end)
+  if (image >= image_end) return;
+  const int Lw = (s.L + 31) >> 5;  // words per key block of the bit table
   const int slice = ml.bytes + ((3 * nT + 15) / 16) * 16;  // the image and a scratch list behind it
   uint8_t *meta = meta_all + (size_t)warp * slice;
   const int nST = (s.L + 127) >> 7;
@@ -85,6 +91,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
       // a selection per query position: every row's own bytes, and their union per query block
       // (which is what the tile list and the item order below are built from)
       uint32_t *roww = reinterpret_cast<uint32_t *>(meta + ml.rows);
+      // the bit table is per key/value head: the group's first query head (or pair of heads) fills it
+      const bool fills = inv_bits && (pack ? (2 * (u % (s.H / 2))) % s.G == 0 : (u % s.H) % s.G == 0);
       for (int i = lane; i < 128 * s.topk; i += 32) {
         const int r = i / s.topk, slot = i % s.topk, t = pack ? row0 + (r & 63) : row0 + r;
         if (t < s.L) {
@@ -93,6 +101,8 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
             const int a = (r >> bk_shift) * nT + blk / nb, b2 = r * nT + blk / nb;
             atomicOr(&selw[a >> 2], (1u << (blk % nb)) << ((a & 3) * 8));
             atomicOr(&roww[b2 >> 2], (1u << (blk % nb)) << ((b2 & 3) * 8));
+            if (fills && (!pack || r < 64))
+              atomicOr(&inv_bits[((int64_t)uk * s.M + blk) * Lw + (t >> 5)], 1u << (t & 31));
           }
         }
       }
@@ -298,25 +308,22 @@ __global__ void __launch_bounds__(kMetaWarps * 32) tc_meta_kernel(Shape s, const
     if (s.pq) {
       // a selection per query position: which positions selected each of this CTA's key blocks
       // (one bit per position), and per 64-query tile which query blocks hold such a position
+      // (the words of this CTA's key blocks from the bit table the query-major images filled: word w
+      // of a block holds positions 32 w ...; a position before the block never selected it)
       uint32_t *invw = reinterpret_cast<uint32_t *>(meta + ml.rows);
-      const int qb0 = kt * G, total = (s.L - key0) * s.topk;
-      const int32_t *rows = idx + ((int64_t)uk * s.L + key0) * s.topk;
-      for (int base = 0; base < total; base += 256) {
-        int blk[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int i = base + e * 32 + lane;
-          blk[e] = i < total ? rows[i] : -1;
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int i = base + e * 32 + lane, t = key0 + i / s.topk;
-          if (blk[e] >= qb0 && blk[e] < qb0 + G && blk[e] <= (t >> bk_shift)) {
-            const int a = (blk[e] - qb0) * nT + (t >> 6);
-            atomicOr(&selw[a >> 2], (1u << ((t >> bk_shift) % nb)) << ((a & 3) * 8));
-            atomicOr(&invw[2 * a + ((t & 63) >> 5)], 1u << (t & 31));
-          }
-        }
+      const int qb0 = kt * G, w_lo = key0 >> 5;
+      for (int i = lane; i < G * (Lw - w_lo); i += 32) {
+        const int g = i / (Lw - w_lo), w = w_lo + i % (Lw - w_lo);
+        if (qb0 + g >= s.M) continue;
+        const uint32_t bits = inv_bits[((int64_t)uk * s.M + qb0 + g) * Lw + w];
+        if (!bits) continue;
+        const int a = g * nT + (w >> 1);
+        invw[2 * a + (w & 1)] = bits;
+        // the 32 positions lie in one query block (Bk >= 32) or in two (Bk = 16)
+        uint32_t qbits;
+        if (s.Bk >= 32) qbits = 1u << (((w & 1) * 32) >> bk_shift);
+        else qbits = (((bits & 0xffffu) ? 1u : 0u) | ((bits >> 16) ? 2u : 0u)) << ((w & 1) * 2);
+        atomicOr(&selw[a >> 2], qbits << ((a & 3) * 8));
       }
     } else {  // which query blocks selected each of this CTA's key blocks, per 64-query tile
       // (the index rows of query blocks qb0 .. M-1 are contiguous; eight loads in flight per lane)
@@ -407,10 +414,20 @@ int launch_tc_meta(const Shape &s, const int32_t *seq_lens, const int32_t *idx, 
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(tc_meta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return BLOSSOM_ERR_CUDA;
-  {
+  auto launch = [&](int image0, int image_end, uint32_t *inv_bits) {
     LaunchScope ls(K_TC_META, st);
-    launch_chained(tc_meta_kernel, dim3((unsigned)((n_images + kMetaWarps - 1) / kMetaWarps)), dim3(kMetaWarps * 32),
-                   smem, st, s, seq_lens, idx, qmeta, kmeta, nT, nq, n_images, branches, with_fwd);
+    launch_chained(tc_meta_kernel, dim3((unsigned)((image_end - image0 + kMetaWarps - 1) / kMetaWarps)),
+                   dim3(kMetaWarps * 32), smem, st, s, seq_lens, idx, qmeta, kmeta, nT, nq, image0, image_end, branches,
+                   with_fwd, inv_bits);
+  };
+  if (s.pq && kmeta) {
+    // selection per position: the query-major images fill the bit table, then the key-major ones read it
+    uint32_t *inv_bits = reinterpret_cast<uint32_t *>(kmeta + tc_meta_bytes(s));
+    if (cudaMemsetAsync(inv_bits, 0, tc_inv_bits_bytes(s), st) != cudaSuccess) return BLOSSOM_ERR_CUDA;
+    launch(0, nq, inv_bits);
+    launch(nq, n_images, inv_bits);
+  } else {
+    launch(0, n_images, nullptr);
   }
   return cudaGetLastError() == cudaSuccess ? BLOSSOM_OK : BLOSSOM_ERR_CUDA;
 }

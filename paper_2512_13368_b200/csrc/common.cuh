@@ -204,6 +204,7 @@ namespace tc {
 int launch_wait_selftest(int32_t *status, cudaStream_t st);
 bool fwd_tc_supported(const Shape &s, int dtype);
 size_t tc_meta_bytes(const Shape &s);  // bytes of one of the two tile-list areas of the workspace
+size_t tc_inv_bits_bytes(const Shape &s);  // (selection per position) bytes of the bit table behind the second
 // branches: bit 0 long-term, bit 1 short-term branch: the tile lists hold only the tiles those
 // branches need.  records: null = computed from out_lt, out_st, lse, dout and the per-head gate by
 // the pre-pass; otherwise the caller's per-row records (layout of Workspace::qstats) are used as

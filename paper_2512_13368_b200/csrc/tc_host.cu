@@ -83,7 +83,14 @@ bool fwd_tc_supported(const Shape &s, int dtype) {
 
 size_t tc_meta_bytes(const Shape &s) {
   const int nT = (s.L + 63) / 64, nST = (s.L + 127) / 128;
-  return (size_t)s.B * s.H * nST * (size_t)meta_bytes(nT, s.pq);
+  return ((size_t)s.B * s.H * nST * (size_t)meta_bytes(nT, s.pq) + 255) / 256 * 256;
+}
+
+// Selection per query position: one bit per (batch, key/value head, key block, position) = that
+// position selected that block; written while the query-major images are built, read by the
+// key-major ones.  It lies behind the key-major images in the workspace.
+size_t tc_inv_bits_bytes(const Shape &s) {
+  return s.pq ? (size_t)s.B * s.Hkv * s.M * (size_t)((s.L + 31) / 32) * sizeof(uint32_t) : 0;
 }
 
 int launch_fwd_tc(const Shape &s, const void *q, const void *k, const void *v, const float *gate,
